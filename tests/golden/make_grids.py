@@ -1,0 +1,42 @@
+"""Writes the stored grids tests use: Lloyd fits (Algorithm 2) computed by the fp64 oracle ONLY.
+
+Run from the repository root:  python -m tests.golden.make_grids
+Each grid is fitted on 2^18 seeded N(0, I_p) samples (seed = synth.inputs.grid_sample_seed(p, n)),
+started from the first n samples, run until no assignment changes, and stored as fp32-exact
+decimal text (the values are rounded to fp32 first, because the library's grid table is fp32 and
+both sides of a parity test must see the same table).
+"""
+import os
+
+import numpy as np
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+GRIDS = [(2, 256), (2, 64), (1, 16), (2, 16)]
+
+
+def path(p, n):
+    return os.path.join(HERE, f"grid_p{p}_n{n}.txt")
+
+
+def load(p, n):
+    g = np.loadtxt(path(p, n), dtype=np.float64, comments="#", ndmin=2)
+    return g.reshape(n, p)
+
+
+def main():
+    import oracle
+    from synth import inputs
+
+    for p, n in GRIDS:
+        s = inputs.gaussian_samples(p, inputs.grid_sample_seed(p, n))
+        res = oracle.make_grid_lloyd(p, n, s, max_iters=6000)
+        g32 = res.grid.astype(np.float32)
+        hdr = (f"Lloyd fit of the Gaussian-MSE-optimal grid (Algorithm 2), p={p} n={n}, 2^18 samples, seed "
+               f"{inputs.grid_sample_seed(p, n)}, iterations {res.iters}, converged {res.converged}; "
+               f"written by tests/golden/make_grids.py from the fp64 oracle; values are fp32-exact")
+        np.savetxt(path(p, n), g32.astype(np.float64), fmt="%.9g", header=hdr)
+        print(p, n, res.iters, res.converged, res.mse_hist[-1])
+
+
+if __name__ == "__main__":
+    main()
