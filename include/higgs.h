@@ -1,0 +1,176 @@
+/*
+ * higgs.h - C ABI of the B200 (sm_100a) HIGGS quantized linear layer.
+ *
+ * The library implements the data-parallel hot path of HIGGS ("Hadamard
+ * Incoherence and Gaussian MSE-optimal GridS"): the encoder of Algorithm 1
+ * (RHT-VQ) with the grid of Algorithm 2, and the rotated-space product of
+ * Appendix F ("Rotating Activations") with the lookup-table dequantisation
+ * discussed in Section 4.3.
+ *
+ * Symbols: N = output features (rows of W), K = input features, B = tokens,
+ * g = scale / rotation group size along K, p = grid dimension, n = grid size,
+ * xi = RHT seed.  W is [N][K] row-major; groups are W[r, i*g:(i+1)*g]
+ * (Appendix F).  Codes are 0-based (Algorithm 1 prints them 1-based).
+ *
+ * Conventions for every entry point
+ *   - Pointers marked "device" are caller-allocated device memory; the library
+ *     never allocates, frees, retains or reallocates them.  Pointers marked
+ *     "host" are ordinary host memory.
+ *   - All device work is enqueued on the caller's stream (a cudaStream_t passed
+ *     as void*; NULL = the legacy default stream).  No call synchronises.
+ *   - The return value is a higgs_status; HIGGS_OK means the work was enqueued.
+ *     Nothing is enqueued when another value is returned.
+ *   - Inputs must be finite; this is a precondition, not checked on the device.
+ *   - There is no CPU fallback: without a CUDA device every compute call
+ *     returns HIGGS_ERR_CUDA.
+ *
+ * The sign function of the randomised Hadamard transform (part of the ABI):
+ *   z = xi + (j+1) * 0x9E3779B97F4A7C15            (mod 2^64)
+ *   z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9
+ *   z = (z ^ (z >> 27)) * 0x94D049BB133111EB
+ *   z =  z ^ (z >> 31)
+ *   sign(xi, j) = -1 if the top bit of z is set, else +1
+ * i.e. output j of the splitmix64 stream seeded with xi.  One sign per input
+ * index j in [0, K), shared by every row of W and every token, so that the
+ * activations are rotated once (Appendix F: "same xi ... same groups").
+ *
+ * The transform itself: RHT(v) = H * diag(sign) * v on each group of g values,
+ * H the Sylvester-ordered Hadamard matrix H[i][j] = (-1)^popcount(i & j).
+ * The encoder uses H unnormalised (Algorithm 1: entries of the rotated unit
+ * vector are approximately N(0,1)); the activations use H / sqrt(g) (Appendix
+ * F: "additional scale 1/sqrt(g) ... making it a random rotation").
+ */
+#ifndef HIGGS_H_
+#define HIGGS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum higgs_status {
+    HIGGS_OK = 0,
+    HIGGS_ERR_INVALID_ARG = 1,   /* null pointer, negative size, misaligned pointer            */
+    HIGGS_ERR_UNSUPPORTED = 2,   /* (p, n, g, dtype, shape) combination has no kernel          */
+    HIGGS_ERR_WORKSPACE = 3,     /* workspace smaller than higgs_workspace_bytes() asks        */
+    HIGGS_ERR_CUDA = 4,          /* a CUDA runtime call failed (no device, launch error)        */
+    HIGGS_ERR_TIMEOUT = 5        /* a bounded device-side wait ran out (read from a status word) */
+} higgs_status;
+
+typedef enum higgs_dtype { HIGGS_F32 = 0, HIGGS_F16 = 1, HIGGS_BF16 = 2 } higgs_dtype;
+
+typedef enum higgs_op { HIGGS_OP_QUANTIZE = 0, HIGGS_OP_LINEAR = 1, HIGGS_OP_MAKE_GRID = 2 } higgs_op;
+
+/*
+ * Description of one quantized matrix.  Supported: g = 1024; (p, n) in
+ * {(2,256), (2,64), (1,16)}; N a multiple of 16, K a multiple of g.
+ * Anything else returns HIGGS_ERR_UNSUPPORTED (never padded silently).
+ * scale_dtype must be HIGGS_F16: one 16-bit scale per (row, group), which is
+ * what the paper's bit counts imply (4.02 = 4 + 16/1024, Appendix G).
+ */
+typedef struct higgs_desc {
+    int32_t p;
+    int32_t n;
+    int32_t g;
+    int32_t scale_dtype;
+    uint64_t rht_seed; /* xi */
+    int64_t N;
+    int64_t K;
+} higgs_desc;
+
+/* Text for a status code (static storage, never NULL). */
+const char* higgs_status_string(int status);
+
+/* Host evaluation of the ABI's sign function: returns +1 or -1. */
+int higgs_sign(uint64_t rht_seed, int64_t j);
+
+/* Bytes of the packed code stream (kernel-native, opaque layout; log2(n)/p
+ * bits per weight), of the scale array ([N][K/g] of scale_dtype), and of the
+ * canonical code array ([N][K/p], one byte per code).  0 if unsupported.   */
+size_t higgs_packed_bytes(const higgs_desc* desc);
+size_t higgs_scales_bytes(const higgs_desc* desc);
+size_t higgs_canonical_bytes(const higgs_desc* desc);
+
+/* Scratch bytes the given operation needs for batch B (B ignored unless
+ * op == HIGGS_OP_LINEAR; for HIGGS_OP_MAKE_GRID desc->K holds the number of
+ * samples and desc->p, desc->n the grid).  Workspaces must be 256-byte
+ * aligned.  Contents need not be initialised and are undefined afterwards.  */
+size_t higgs_workspace_bytes(const higgs_desc* desc, int op, int64_t B);
+
+/*
+ * Algorithm 2, first line: the Gaussian-MSE-optimal grid.  The paper names the
+ * procedure (CLVQ) without its parameters; this library runs the batch (Lloyd)
+ * fixed-point iteration on the caller's samples of N(0, I_p): centres start at
+ * the first n samples; every iteration assigns each sample to its nearest
+ * centre (ties to the lowest index) and moves each centre to the mean of its
+ * samples (an empty cell keeps its centre); it stops when no assignment
+ * changes or after max_iters iterations; centres are then sorted
+ * lexicographically.
+ *   samples      device, [num_samples][p] fp32, num_samples >= n
+ *   grid_out     device, [n][p] fp32
+ *   mse_out      device, optional: per-dimension MSE of the final assignment on
+ *                the samples
+ *   iters_out    device, optional: iterations run (int32), negative if
+ *                max_iters was reached without convergence
+ * Distances are fp32, sums fp64; the result is a fixed point of the same
+ * iteration the fp64 definition runs but need not be bit-identical to it.
+ */
+int higgs_make_grid(int p, int n, const float* samples, int64_t num_samples, int max_iters,
+                    float* grid_out, float* mse_out, int32_t* iters_out,
+                    void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Algorithm 1 (RHT-VQ) on every row of W.  Per (row r, group i):
+ *   s = ||w||_2;  w+ = H diag(sign) (w / s);  code_t = nearest grid point of
+ *   the t-th consecutive p-tuple of w+ (exhaustive search, fp32 squared
+ *   distances, lowest index on exact ties);  stored scale = s / sqrt(g).
+ * A group of zeros gets scale 0 and the code of the point nearest the origin.
+ *   W              device, [N][K] row-major, w_dtype in {HIGGS_F32, HIGGS_BF16}
+ *   grid           device, [n][p] fp32
+ *   packed_out     device, higgs_packed_bytes() bytes, 16-byte aligned
+ *   scales_out     device, [N][K/g] of desc->scale_dtype
+ *   canonical_out  device, optional, [N][K/p] one byte per code (for checking)
+ */
+int higgs_quantize(const higgs_desc* desc, const void* W, int w_dtype, const float* grid,
+                   void* packed_out, void* scales_out, uint8_t* canonical_out,
+                   void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Appendix F, "Rotating Activations": y = x W^T computed in the rotated space.
+ *   x+ = (H / sqrt(g)) diag(sign) x per token and K-group (same xi as the
+ *   encoder);  y[b][r] = sum_i scale[r][i] * sum_t < G[code[r][i][t]], x+[b][i][tp:(t+1)p] >.
+ * Grid entries and x+ are rounded to fp16 for the tensor-core operands;
+ * products are exact and accumulation is fp32; scales are applied in fp32.
+ *   x        device, [B][K] row-major bf16, B >= 1
+ *   packed   device, from higgs_quantize / higgs_pack_codes
+ *   scales   device, [N][K/g]
+ *   grid     device, [n][p] fp32
+ *   y        device, [B][N] row-major, y_dtype in {HIGGS_F32, HIGGS_BF16}
+ * When K is split over several thread blocks the partial sums meet in fp32
+ * atomics, so the last bits of y may differ from run to run.
+ */
+int higgs_linear(const higgs_desc* desc, const void* x, int64_t B,
+                 const void* packed, const void* scales, const float* grid,
+                 void* y, int y_dtype,
+                 void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---- validation helpers (not on the hot path) --------------------------- */
+
+/* The transform alone on `rows` rows of length K: out[r] = RHT of x[r] per
+ * group (Algorithm 1 / Appendix F).  x_dtype in {HIGGS_F32, HIGGS_BF16};
+ * out is device [rows][K] fp32; normalised != 0 divides by sqrt(g).        */
+int higgs_rht(const higgs_desc* desc, const void* x, int x_dtype, int64_t rows,
+              float* out, int normalised, void* stream);
+
+/* Canonical codes ([N][K/p] bytes, device) -> packed stream, and back.  They
+ * let codes produced elsewhere (e.g. by a reference encoder) be fed to
+ * higgs_linear, and the packed output of higgs_quantize be inspected.       */
+int higgs_pack_codes(const higgs_desc* desc, const uint8_t* canonical, void* packed_out, void* stream);
+int higgs_unpack_codes(const higgs_desc* desc, const void* packed, uint8_t* canonical_out, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HIGGS_H_ */

@@ -1,0 +1,190 @@
+"""Thin ctypes binding of the C ABI declared in include/higgs.h.
+
+Argument marshalling only: every step of the path runs in the CUDA library.
+torch is used for device memory and streams.  There is no CPU fallback: if the
+shared library is missing, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libhiggs_b200.so")
+
+HIGGS_OK, HIGGS_ERR_INVALID_ARG, HIGGS_ERR_UNSUPPORTED, HIGGS_ERR_WORKSPACE, HIGGS_ERR_CUDA, HIGGS_ERR_TIMEOUT = range(6)
+HIGGS_F32, HIGGS_F16, HIGGS_BF16 = 0, 1, 2
+HIGGS_OP_QUANTIZE, HIGGS_OP_LINEAR, HIGGS_OP_MAKE_GRID = 0, 1, 2
+
+EXPORTS = [
+    "higgs_status_string", "higgs_sign", "higgs_packed_bytes", "higgs_scales_bytes", "higgs_canonical_bytes",
+    "higgs_workspace_bytes", "higgs_make_grid", "higgs_quantize", "higgs_linear", "higgs_rht",
+    "higgs_pack_codes", "higgs_unpack_codes",
+]
+
+
+class higgs_desc(ctypes.Structure):
+    _fields_ = [
+        ("p", ctypes.c_int32), ("n", ctypes.c_int32), ("g", ctypes.c_int32), ("scale_dtype", ctypes.c_int32),
+        ("rht_seed", ctypes.c_uint64), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+    ]
+
+
+class HiggsError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2411_17525_b200.build` "
+            "(there is no CPU or PyTorch fallback for the HIGGS kernels)")
+    lib = ctypes.CDLL(LIB_PATH)
+    P, vp, sz, i64, i32, u64 = ctypes.POINTER(higgs_desc), ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int64, ctypes.c_int, ctypes.c_uint64
+    lib.higgs_status_string.restype = ctypes.c_char_p
+    lib.higgs_status_string.argtypes = [i32]
+    lib.higgs_sign.restype = i32
+    lib.higgs_sign.argtypes = [u64, i64]
+    for f in ("higgs_packed_bytes", "higgs_scales_bytes", "higgs_canonical_bytes"):
+        getattr(lib, f).restype = sz
+        getattr(lib, f).argtypes = [P]
+    lib.higgs_workspace_bytes.restype = sz
+    lib.higgs_workspace_bytes.argtypes = [P, i32, i64]
+    lib.higgs_make_grid.restype = i32
+    lib.higgs_make_grid.argtypes = [i32, i32, vp, i64, i32, vp, vp, vp, vp, sz, vp]
+    lib.higgs_quantize.restype = i32
+    lib.higgs_quantize.argtypes = [P, vp, i32, vp, vp, vp, vp, vp, sz, vp]
+    lib.higgs_linear.restype = i32
+    lib.higgs_linear.argtypes = [P, vp, i64, vp, vp, vp, vp, i32, vp, sz, vp]
+    lib.higgs_rht.restype = i32
+    lib.higgs_rht.argtypes = [P, vp, i32, i64, vp, i32, vp]
+    lib.higgs_pack_codes.restype = i32
+    lib.higgs_pack_codes.argtypes = [P, vp, vp, vp]
+    lib.higgs_unpack_codes.restype = i32
+    lib.higgs_unpack_codes.argtypes = [P, vp, vp, vp]
+    return lib
+
+
+lib = _load()
+
+
+def make_desc(p: int, n: int, N: int, K: int, rht_seed: int, g: int = 1024) -> higgs_desc:
+    return higgs_desc(p, n, g, HIGGS_F16, rht_seed & (2**64 - 1), N, K)
+
+
+def status_string(status: int) -> str:
+    return lib.higgs_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != HIGGS_OK:
+        raise HiggsError(status, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    return {torch.float32: HIGGS_F32, torch.float16: HIGGS_F16, torch.bfloat16: HIGGS_BF16}[t.dtype]
+
+
+def higgs_sign(rht_seed: int, j: int) -> int:
+    return int(lib.higgs_sign(ctypes.c_uint64(rht_seed & (2**64 - 1)), int(j)))
+
+
+def higgs_packed_bytes(desc: higgs_desc) -> int:
+    return int(lib.higgs_packed_bytes(ctypes.byref(desc)))
+
+
+def higgs_scales_bytes(desc: higgs_desc) -> int:
+    return int(lib.higgs_scales_bytes(ctypes.byref(desc)))
+
+
+def higgs_canonical_bytes(desc: higgs_desc) -> int:
+    return int(lib.higgs_canonical_bytes(ctypes.byref(desc)))
+
+
+def higgs_workspace_bytes(desc: higgs_desc, op: int, B: int = 0) -> int:
+    return int(lib.higgs_workspace_bytes(ctypes.byref(desc), int(op), int(B)))
+
+
+def _workspace(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
+
+
+def higgs_make_grid(p: int, n: int, samples: torch.Tensor, max_iters: int = 4000, workspace: Optional[torch.Tensor] = None):
+    """samples: cuda fp32 [m][p].  Returns (grid [n][p] fp32, mse fp32 scalar tensor, iters int32 scalar tensor)."""
+    assert samples.is_cuda and samples.dtype == torch.float32 and samples.is_contiguous()
+    m = samples.numel() // p
+    d = higgs_desc(p, n, 0, HIGGS_F16, 0, 0, m)
+    if workspace is None:
+        workspace = _workspace(higgs_workspace_bytes(d, HIGGS_OP_MAKE_GRID), samples.device)
+    grid = torch.empty((n, p), dtype=torch.float32, device=samples.device)
+    mse = torch.empty((), dtype=torch.float32, device=samples.device)
+    iters = torch.empty((), dtype=torch.int32, device=samples.device)
+    _check(lib.higgs_make_grid(p, n, _ptr(samples), m, int(max_iters), _ptr(grid), _ptr(mse), _ptr(iters),
+                               _ptr(workspace), workspace.numel(), _stream()), "higgs_make_grid")
+    return grid, mse, iters
+
+
+def higgs_quantize(desc: higgs_desc, W: torch.Tensor, grid: torch.Tensor, want_canonical: bool = False,
+                   workspace: Optional[torch.Tensor] = None):
+    """W: cuda [N][K] fp32 or bf16; grid: cuda [n][p] fp32.  Returns (packed u8, scales fp16 [N][K/g], canonical u8 or None)."""
+    assert W.is_cuda and W.is_contiguous() and grid.is_cuda and grid.dtype == torch.float32 and grid.is_contiguous()
+    dev = W.device
+    packed = torch.empty(max(higgs_packed_bytes(desc), 16), dtype=torch.uint8, device=dev)
+    scales = torch.empty((desc.N, max(desc.K // desc.g, 0)), dtype=torch.float16, device=dev)
+    canonical = torch.empty((desc.N, desc.K // desc.p), dtype=torch.uint8, device=dev) if want_canonical else None
+    if workspace is None:
+        workspace = _workspace(higgs_workspace_bytes(desc, HIGGS_OP_QUANTIZE), dev)
+    _check(lib.higgs_quantize(ctypes.byref(desc), _ptr(W), _dtype_code(W), _ptr(grid), _ptr(packed), _ptr(scales),
+                              _ptr(canonical), _ptr(workspace), workspace.numel(), _stream()), "higgs_quantize")
+    return packed, scales, canonical
+
+
+def higgs_linear(desc: higgs_desc, x: torch.Tensor, packed: torch.Tensor, scales: torch.Tensor, grid: torch.Tensor,
+                 out_dtype: torch.dtype = torch.float32, workspace: Optional[torch.Tensor] = None,
+                 y: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """x: cuda [B][K] bf16.  Returns y [B][N] of out_dtype (fp32 or bf16)."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous()
+    B = x.shape[0]
+    if y is None:
+        y = torch.empty((B, desc.N), dtype=out_dtype, device=x.device)
+    if workspace is None:
+        workspace = _workspace(higgs_workspace_bytes(desc, HIGGS_OP_LINEAR, B), x.device)
+    _check(lib.higgs_linear(ctypes.byref(desc), _ptr(x), B, _ptr(packed), _ptr(scales), _ptr(grid), _ptr(y),
+                            _dtype_code(y), _ptr(workspace), workspace.numel(), _stream()), "higgs_linear")
+    return y
+
+
+def higgs_rht(desc: higgs_desc, x: torch.Tensor, normalised: bool) -> torch.Tensor:
+    """x: cuda [rows][K] fp32 or bf16 -> fp32 [rows][K], the transform of Algorithm 1 / Appendix F per group."""
+    assert x.is_cuda and x.is_contiguous()
+    out = torch.empty(x.shape, dtype=torch.float32, device=x.device)
+    _check(lib.higgs_rht(ctypes.byref(desc), _ptr(x), _dtype_code(x), x.shape[0], _ptr(out), int(bool(normalised)),
+                         _stream()), "higgs_rht")
+    return out
+
+
+def higgs_pack_codes(desc: higgs_desc, canonical: torch.Tensor) -> torch.Tensor:
+    assert canonical.is_cuda and canonical.dtype == torch.uint8 and canonical.is_contiguous()
+    packed = torch.empty(max(higgs_packed_bytes(desc), 16), dtype=torch.uint8, device=canonical.device)
+    _check(lib.higgs_pack_codes(ctypes.byref(desc), _ptr(canonical), _ptr(packed), _stream()), "higgs_pack_codes")
+    return packed
+
+
+def higgs_unpack_codes(desc: higgs_desc, packed: torch.Tensor) -> torch.Tensor:
+    assert packed.is_cuda and packed.dtype == torch.uint8
+    canonical = torch.empty((desc.N, desc.K // desc.p), dtype=torch.uint8, device=packed.device)
+    _check(lib.higgs_unpack_codes(ctypes.byref(desc), _ptr(packed), _ptr(canonical), _stream()), "higgs_unpack_codes")
+    return canonical

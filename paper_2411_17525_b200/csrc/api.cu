@@ -1,0 +1,168 @@
+// C-ABI entry points: argument checking, workspace carving, kernel sequencing.
+#include "common.cuh"
+
+namespace higgs {
+
+int check_desc(const higgs_desc* d) {
+    if (!d) return HIGGS_ERR_INVALID_ARG;
+    if (d->N < 0 || d->K < 0) return HIGGS_ERR_INVALID_ARG;
+    if (d->g != kGroup) return HIGGS_ERR_UNSUPPORTED;
+    if (format_of(d->p, d->n) == Format::kNone) return HIGGS_ERR_UNSUPPORTED;
+    if (d->scale_dtype != HIGGS_F16) return HIGGS_ERR_UNSUPPORTED;
+    if (d->N % kRowTile || d->K % kGroup) return HIGGS_ERR_UNSUPPORTED;
+    if (d->N > (int64_t)1 << 30 || d->K > (int64_t)1 << 30) return HIGGS_ERR_UNSUPPORTED;
+    return HIGGS_OK;
+}
+
+static bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+}  // namespace higgs
+
+using namespace higgs;
+
+extern "C" {
+
+const char* higgs_status_string(int status) {
+    switch (status) {
+        case HIGGS_OK: return "ok";
+        case HIGGS_ERR_INVALID_ARG: return "invalid argument";
+        case HIGGS_ERR_UNSUPPORTED: return "unsupported (p, n, g, dtype, shape) combination";
+        case HIGGS_ERR_WORKSPACE: return "workspace too small";
+        case HIGGS_ERR_CUDA: return "CUDA runtime error";
+        case HIGGS_ERR_TIMEOUT: return "bounded device-side wait ran out";
+        default: return "unknown status";
+    }
+}
+
+int higgs_sign(uint64_t rht_seed, int64_t j) { return sign_bit(rht_seed, j) ? -1 : 1; }
+
+size_t higgs_packed_bytes(const higgs_desc* d) {
+    if (check_desc(d) != HIGGS_OK) return 0;
+    const size_t pairs = (size_t)d->N * (size_t)d->K / 2;
+    return format_of(d->p, d->n) == Format::kSixBit ? pairs / 4 * 3 : pairs;
+}
+
+size_t higgs_scales_bytes(const higgs_desc* d) {
+    if (check_desc(d) != HIGGS_OK) return 0;
+    return (size_t)d->N * (size_t)(d->K / d->g) * 2;
+}
+
+size_t higgs_canonical_bytes(const higgs_desc* d) {
+    if (check_desc(d) != HIGGS_OK) return 0;
+    return (size_t)d->N * (size_t)d->K / (size_t)d->p;
+}
+
+size_t higgs_workspace_bytes(const higgs_desc* d, int op, int64_t B) {
+    if (!d) return 0;
+    if (op == HIGGS_OP_MAKE_GRID) {
+        if (!((d->p == 1 || d->p == 2) && d->n >= 1 && d->n <= 256 && d->K >= d->n)) return 0;
+        return make_grid_workspace(d->p, d->n, d->K);
+    }
+    if (check_desc(d) != HIGGS_OK) return 0;
+    if (op == HIGGS_OP_QUANTIZE) return align_up(higgs_canonical_bytes(d), 256) + 256;
+    if (op == HIGGS_OP_LINEAR) {
+        if (B < 1) return 0;
+        return align_up((size_t)B * d->K * 2, 256) + align_up((size_t)B * d->N * 4, 256) + 256;
+    }
+    return 0;
+}
+
+int higgs_make_grid(int p, int n, const float* samples, int64_t num_samples, int max_iters, float* grid_out,
+                    float* mse_out, int32_t* iters_out, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!samples || !grid_out || !workspace || max_iters < 1) return HIGGS_ERR_INVALID_ARG;
+    if (!(p == 1 || p == 2) || n < 1 || n > 256) return HIGGS_ERR_UNSUPPORTED;
+    if (num_samples < n || num_samples > ((int64_t)1 << 31) - 1) return HIGGS_ERR_INVALID_ARG;
+    if (!aligned(workspace, 256)) return HIGGS_ERR_INVALID_ARG;
+    if (workspace_bytes < make_grid_workspace(p, n, num_samples)) return HIGGS_ERR_WORKSPACE;
+    return launch_make_grid(p, n, samples, num_samples, max_iters, grid_out, mse_out, iters_out, workspace,
+                            as_stream(stream));
+}
+
+int higgs_quantize(const higgs_desc* d, const void* W, int w_dtype, const float* grid, void* packed_out,
+                   void* scales_out, uint8_t* canonical_out, void* workspace, size_t workspace_bytes, void* stream) {
+    int rc = check_desc(d);
+    if (rc != HIGGS_OK) return rc;
+    if (w_dtype != HIGGS_F32 && w_dtype != HIGGS_BF16) return HIGGS_ERR_UNSUPPORTED;
+    if (d->N == 0 || d->K == 0) return HIGGS_OK;
+    if (!W || !grid || !packed_out || !scales_out) return HIGGS_ERR_INVALID_ARG;
+    if (!aligned(W, 16) || !aligned(packed_out, 16) || !aligned(scales_out, 2)) return HIGGS_ERR_INVALID_ARG;
+    uint8_t* canonical = canonical_out;
+    if (!canonical) {
+        if (!workspace || !aligned(workspace, 256)) return HIGGS_ERR_INVALID_ARG;
+        if (workspace_bytes < higgs_workspace_bytes(d, HIGGS_OP_QUANTIZE, 0)) return HIGGS_ERR_WORKSPACE;
+        canonical = static_cast<uint8_t*>(workspace);
+    } else if (!aligned(canonical, 8)) {
+        return HIGGS_ERR_INVALID_ARG;
+    }
+    cudaStream_t st = as_stream(stream);
+    rc = launch_encode(*d, W, w_dtype, grid, canonical, scales_out, st);
+    if (rc != HIGGS_OK) return rc;
+    return launch_pack(*d, canonical, packed_out, st);
+}
+
+int higgs_linear(const higgs_desc* d, const void* x, int64_t B, const void* packed, const void* scales,
+                 const float* grid, void* y, int y_dtype, void* workspace, size_t workspace_bytes, void* stream) {
+    int rc = check_desc(d);
+    if (rc != HIGGS_OK) return rc;
+    if (y_dtype != HIGGS_F32 && y_dtype != HIGGS_BF16) return HIGGS_ERR_UNSUPPORTED;
+    if (B < 0) return HIGGS_ERR_INVALID_ARG;
+    if (B == 0 || d->N == 0) return HIGGS_OK;
+    if (d->K == 0) return HIGGS_ERR_UNSUPPORTED;
+    if (!x || !packed || !scales || !grid || !y || !workspace) return HIGGS_ERR_INVALID_ARG;
+    if (!aligned(x, 16) || !aligned(packed, 16) || !aligned(scales, 2) || !aligned(workspace, 256) ||
+        !aligned(y, y_dtype == HIGGS_F32 ? 4 : 2))
+        return HIGGS_ERR_INVALID_ARG;
+    if (workspace_bytes < higgs_workspace_bytes(d, HIGGS_OP_LINEAR, B)) return HIGGS_ERR_WORKSPACE;
+    cudaStream_t st = as_stream(stream);
+
+    __half* xdag = static_cast<__half*>(workspace);
+    float* y32 = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up((size_t)B * d->K * 2, 256));
+    const int chunks = linear_k_chunks(*d, B);
+    const bool split = chunks > 1;
+    float* acc_target = split ? (y_dtype == HIGGS_F32 ? static_cast<float*>(y) : y32) : nullptr;
+
+    // D1: rotate the activations once (and clear the accumulation target of a K-split product)
+    rc = launch_rht_activations(*d, x, B, xdag, acc_target, split ? (size_t)B * d->N : 0, st);
+    if (rc != HIGGS_OK) return rc;
+
+    // D2-D5: stream codes, look up, contract, reduce
+    for (int64_t b0 = 0; b0 < B; b0 += 16) {
+        const int64_t bn = B - b0 < 16 ? B - b0 : 16;
+        void* yo;
+        int mode;
+        if (split) { yo = acc_target + b0 * d->N; mode = 2; }
+        else if (y_dtype == HIGGS_F32) { yo = static_cast<float*>(y) + b0 * d->N; mode = 0; }
+        else { yo = static_cast<__nv_bfloat16*>(y) + b0 * d->N; mode = 1; }
+        rc = launch_linear_mma(*d, xdag + b0 * d->K, bn, packed, scales, grid, yo, d->N, mode, st);
+        if (rc != HIGGS_OK) return rc;
+    }
+    if (split && y_dtype == HIGGS_BF16) return launch_convert_out(y32, y, y_dtype, (size_t)B * d->N, st);
+    return HIGGS_OK;
+}
+
+int higgs_rht(const higgs_desc* d, const void* x, int x_dtype, int64_t rows, float* out, int normalised, void* stream) {
+    int rc = check_desc(d);
+    if (rc != HIGGS_OK) return rc;
+    if (rows < 0) return HIGGS_ERR_INVALID_ARG;
+    if (rows == 0 || d->K == 0) return HIGGS_OK;
+    if (!x || !out || !aligned(x, 16) || !aligned(out, 16)) return HIGGS_ERR_INVALID_ARG;
+    return launch_rht_debug(*d, x, x_dtype, rows, out, normalised, as_stream(stream));
+}
+
+int higgs_pack_codes(const higgs_desc* d, const uint8_t* canonical, void* packed_out, void* stream) {
+    int rc = check_desc(d);
+    if (rc != HIGGS_OK) return rc;
+    if (d->N == 0 || d->K == 0) return HIGGS_OK;
+    if (!canonical || !packed_out || !aligned(packed_out, 16)) return HIGGS_ERR_INVALID_ARG;
+    return launch_pack(*d, canonical, packed_out, as_stream(stream));
+}
+
+int higgs_unpack_codes(const higgs_desc* d, const void* packed, uint8_t* canonical_out, void* stream) {
+    int rc = check_desc(d);
+    if (rc != HIGGS_OK) return rc;
+    if (d->N == 0 || d->K == 0) return HIGGS_OK;
+    if (!packed || !canonical_out || !aligned(packed, 16)) return HIGGS_ERR_INVALID_ARG;
+    return launch_unpack(*d, packed, canonical_out, as_stream(stream));
+}
+
+}  // extern "C"

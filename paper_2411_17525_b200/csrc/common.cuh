@@ -1,0 +1,100 @@
+// Shared declarations of the HIGGS CUDA library (sm_100a only).
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "higgs.h"
+
+namespace higgs {
+
+constexpr int kGroup = 1024;     // the only supported group size g
+constexpr int kRowTile = 16;     // rows of W per mma tile (m16n8k16)
+constexpr int kBlockK = 64;      // k-extent of one 512-byte packed block
+
+// Top bit of output j of the splitmix64 stream seeded with xi: 1 -> sign -1.
+__host__ __device__ __forceinline__ uint32_t sign_bit(uint64_t xi, int64_t j) {
+    uint64_t z = xi + ((uint64_t)j + 1ull) * 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    z = z ^ (z >> 31);
+    return (uint32_t)(z >> 63);
+}
+
+// How codes are stored in the packed stream.
+//   kByteLut : one byte looks up one fp16x2 table entry (two consecutive k).
+//              p=2,n=256: the byte is the code.  p=1,n=16: the byte holds the
+//              codes of k (low nibble) and k+1 (high nibble).
+//   kSixBit  : p=2,n=64: 6-bit codes, low nibbles and high bit-pairs in
+//              separate planes (bit slices), see pack.cu.
+enum class Format : int { kNone = 0, kByteLut = 1, kSixBit = 2 };
+
+__host__ __device__ inline Format format_of(int p, int n) {
+    if (p == 2 && n == 256) return Format::kByteLut;
+    if (p == 1 && n == 16) return Format::kByteLut;
+    if (p == 2 && n == 64) return Format::kSixBit;
+    return Format::kNone;
+}
+
+// Validates the descriptor; returns HIGGS_OK or the error to hand back.
+int check_desc(const higgs_desc* d);
+
+inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
+
+inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? HIGGS_OK : HIGGS_ERR_CUDA; }
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// ---- in-register / warp-shuffle fast Walsh-Hadamard transform over 1024 ----
+// A warp owns one group.  Lane l holds 32 values v[r], r = c*8 + e, standing
+// for element index  idx = c*256 + l*8 + e  (c in 0..3, e in 0..7), so that a
+// lane's four chunks are 8 consecutive elements each and a warp-wide chunk load
+// is one contiguous 256-element run.  Butterflies over the e and c bits run in
+// registers, the five lane bits through shfl.bfly.  The transform is the
+// unnormalised Sylvester one (stages commute, so any bit order gives H v).
+__device__ __forceinline__ void fwht1024_warp(float (&v)[32], int lane) {
+#pragma unroll
+    for (int h = 1; h < 32; h <<= 1) {
+#pragma unroll
+        for (int r = 0; r < 32; ++r) {
+            if ((r & h) == 0) {
+                float a = v[r], b = v[r | h];
+                v[r] = a + b;
+                v[r | h] = a - b;
+            }
+        }
+    }
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+        const bool upper = (lane & m) != 0;
+#pragma unroll
+        for (int r = 0; r < 32; ++r) {
+            float o = __shfl_xor_sync(0xffffffffu, v[r], m);
+            v[r] = upper ? (o - v[r]) : (v[r] + o);
+        }
+    }
+}
+
+// element index inside the group of register r of lane l (see above)
+__device__ __forceinline__ int fwht_index(int lane, int r) { return (r >> 3) * 256 + lane * 8 + (r & 7); }
+
+// ---- kernels' host-side launchers (defined in the .cu files) ---------------
+int launch_rht_activations(const higgs_desc& d, const void* x, int64_t B, __half* xdag, float* zero_ptr,
+                           size_t zero_floats, cudaStream_t st);
+int launch_rht_debug(const higgs_desc& d, const void* x, int x_dtype, int64_t rows, float* out, int normalised,
+                     cudaStream_t st);
+int launch_encode(const higgs_desc& d, const void* W, int w_dtype, const float* grid, uint8_t* canonical,
+                  void* scales, cudaStream_t st);
+int launch_pack(const higgs_desc& d, const uint8_t* canonical, void* packed, cudaStream_t st);
+int launch_unpack(const higgs_desc& d, const void* packed, uint8_t* canonical, cudaStream_t st);
+int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const void* packed, const void* scales,
+                      const float* grid, void* y, int64_t ldy, int y_mode, cudaStream_t st);
+int launch_convert_out(const float* y32, void* y, int y_dtype, size_t count, cudaStream_t st);
+size_t make_grid_workspace(int p, int n, int64_t m);
+int launch_make_grid(int p, int n, const float* samples, int64_t m, int max_iters, float* grid_out, float* mse_out,
+                     int32_t* iters_out, void* ws, cudaStream_t st);
+int linear_k_chunks(const higgs_desc& d, int64_t B);
+
+}  // namespace higgs

@@ -1,0 +1,153 @@
+// Grid fit of Algorithm 2 ("CLVQ(n, p), computed once"), run as Lloyd's batch
+// iteration on caller-provided samples of N(0, I_p): the assignment step is the
+// encoder's exhaustive nearest-point search, the update a segmented mean.
+#include "common.cuh"
+
+namespace higgs {
+
+namespace {
+
+struct GridWs {
+    float* centres;               // [n][p]
+    double* sums;                 // [n][p]
+    unsigned long long* counts;   // [n]
+    int32_t* assign;              // [m]
+    double* err;                  // [2]: running, last completed
+    int32_t* flags;               // [0] changed, [1] done, [2] iterations
+};
+
+__host__ __device__ inline size_t up256(size_t v) { return (v + 255) / 256 * 256; }
+
+GridWs carve(void* ws, int p, int n, int64_t m) {
+    uint8_t* b = static_cast<uint8_t*>(ws);
+    GridWs w;
+    w.centres = reinterpret_cast<float*>(b); b += up256(sizeof(float) * n * p);
+    w.sums = reinterpret_cast<double*>(b); b += up256(sizeof(double) * n * p);
+    w.counts = reinterpret_cast<unsigned long long*>(b); b += up256(sizeof(unsigned long long) * n);
+    w.err = reinterpret_cast<double*>(b); b += 256;
+    w.flags = reinterpret_cast<int32_t*>(b); b += 256;
+    w.assign = reinterpret_cast<int32_t*>(b);
+    (void)m;
+    return w;
+}
+
+__global__ void grid_init_kernel(GridWs w, const float* __restrict__ samples, int p, int n, int64_t m) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < m) w.assign[i] = -1;
+    if (i < (int64_t)n * p) { w.centres[i] = samples[i]; w.sums[i] = 0.0; }
+    if (i < n) w.counts[i] = 0ull;
+    if (i < 2) w.err[i] = 0.0;
+    if (i < 3) w.flags[i] = 0;
+}
+
+template <int P>
+__global__ void __launch_bounds__(256) grid_assign_kernel(GridWs w, const float* __restrict__ samples, int n, int64_t m) {
+    __shared__ float sc[256 * 2];
+    __shared__ double ssum[256 * 2];
+    __shared__ unsigned int scnt[256];
+    __shared__ double serr;
+    __shared__ int schanged;
+    if (w.flags[1]) return;
+    for (int i = threadIdx.x; i < n * P; i += blockDim.x) { sc[i] = w.centres[i]; ssum[i] = 0.0; }
+    for (int i = threadIdx.x; i < n; i += blockDim.x) scnt[i] = 0u;
+    if (threadIdx.x == 0) { serr = 0.0; schanged = 0; }
+    __syncthreads();
+    double err = 0.0;
+    int changed = 0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < m; i += (int64_t)gridDim.x * blockDim.x) {
+        float x0 = samples[i * P], x1 = P == 2 ? samples[i * P + 1] : 0.f;
+        float best = INFINITY;
+        int bi = 0;
+        for (int c = 0; c < n; ++c) {
+            float d;
+            if (P == 2) {
+                const float dx = x0 - sc[2 * c], dy = x1 - sc[2 * c + 1];
+                d = fmaf(dy, dy, dx * dx);
+            } else {
+                const float dx = x0 - sc[c];
+                d = dx * dx;
+            }
+            if (d < best) { best = d; bi = c; }
+        }
+        if (w.assign[i] != bi) { w.assign[i] = bi; ++changed; }
+        err += (double)best;
+        atomicAdd(&ssum[bi * P], (double)x0);
+        if (P == 2) atomicAdd(&ssum[bi * P + 1], (double)x1);
+        atomicAdd(&scnt[bi], 1u);
+    }
+    atomicAdd(&serr, err);
+    if (changed) atomicAdd(&schanged, changed);
+    __syncthreads();
+    for (int i = threadIdx.x; i < n * P; i += blockDim.x)
+        if (ssum[i] != 0.0) atomicAdd(&w.sums[i], ssum[i]);
+    for (int i = threadIdx.x; i < n; i += blockDim.x)
+        if (scnt[i]) atomicAdd(&w.counts[i], (unsigned long long)scnt[i]);
+    if (threadIdx.x == 0) {
+        atomicAdd(&w.err[0], serr);
+        if (schanged) atomicAdd(&w.flags[0], schanged);
+    }
+}
+
+__global__ void grid_update_kernel(GridWs w, int p, int n) {
+    if (w.flags[1]) return;
+    const int changed = w.flags[0];
+    __syncthreads();
+    for (int i = threadIdx.x; i < n * p; i += blockDim.x) {
+        const unsigned long long cnt = w.counts[i / p];
+        if (changed && cnt) w.centres[i] = (float)(w.sums[i] / (double)cnt);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < n * p; i += blockDim.x) w.sums[i] = 0.0;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) w.counts[i] = 0ull;
+    if (threadIdx.x == 0) {
+        w.err[1] = w.err[0];
+        w.err[0] = 0.0;
+        w.flags[2] += 1;
+        w.flags[0] = 0;
+        if (!changed) w.flags[1] = 1;
+    }
+}
+
+__global__ void grid_finalize_kernel(GridWs w, int p, int n, int64_t m, float* __restrict__ grid_out,
+                                     float* __restrict__ mse_out, int32_t* __restrict__ iters_out) {
+    for (int c = threadIdx.x; c < n; c += blockDim.x) {
+        const float a0 = w.centres[c * p], a1 = p == 2 ? w.centres[c * p + 1] : 0.f;
+        int rank = 0;
+        for (int o = 0; o < n; ++o) {
+            const float b0 = w.centres[o * p], b1 = p == 2 ? w.centres[o * p + 1] : 0.f;
+            const bool less = (b0 < a0) || (b0 == a0 && (b1 < a1 || (b1 == a1 && o < c)));
+            rank += less ? 1 : 0;
+        }
+        grid_out[rank * p] = a0;
+        if (p == 2) grid_out[rank * p + 1] = a1;
+    }
+    if (threadIdx.x == 0) {
+        if (mse_out) *mse_out = (float)(w.err[1] / ((double)m * p));
+        if (iters_out) *iters_out = w.flags[1] ? w.flags[2] : -w.flags[2];
+    }
+}
+
+}  // namespace
+
+size_t make_grid_workspace(int p, int n, int64_t m) {
+    return up256(sizeof(float) * n * p) + up256(sizeof(double) * n * p) + up256(sizeof(unsigned long long) * n) + 512 +
+           up256(sizeof(int32_t) * (size_t)m);
+}
+
+int launch_make_grid(int p, int n, const float* samples, int64_t m, int max_iters, float* grid_out, float* mse_out,
+                     int32_t* iters_out, void* ws, cudaStream_t st) {
+    GridWs w = carve(ws, p, n, m);
+    const int64_t init_threads = m > (int64_t)n * p ? m : (int64_t)n * p;
+    grid_init_kernel<<<(unsigned)((init_threads + 255) / 256), 256, 0, st>>>(w, samples, p, n, m);
+    int64_t blocks = (m + 255) / 256;
+    if (blocks > 592) blocks = 592;
+    for (int it = 0; it < max_iters; ++it) {
+        if (p == 2) grid_assign_kernel<2><<<(unsigned)blocks, 256, 0, st>>>(w, samples, n, m);
+        else grid_assign_kernel<1><<<(unsigned)blocks, 256, 0, st>>>(w, samples, n, m);
+        grid_update_kernel<<<1, 256, 0, st>>>(w, p, n);
+    }
+    grid_finalize_kernel<<<1, 256, 0, st>>>(w, p, n, m, grid_out, mse_out, iters_out);
+    return cuda_status(cudaGetLastError());
+}
+
+}  // namespace higgs

@@ -1,0 +1,280 @@
+// Encoder of Algorithm 1 (RHT-VQ): group norm, randomised Hadamard transform,
+// exhaustive nearest-grid-point search, canonical codes and fp16 scales; plus the
+// conversion between canonical codes and the packed, kernel-native code stream.
+#include "common.cuh"
+
+namespace higgs {
+
+namespace {
+
+template <typename T>
+__device__ __forceinline__ void load32(const T* __restrict__ src, int lane, float (&v)[32]);
+
+template <>
+__device__ __forceinline__ void load32<__nv_bfloat16>(const __nv_bfloat16* __restrict__ src, int lane, float (&v)[32]) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        uint4 q = __ldg(reinterpret_cast<const uint4*>(src + c * 256 + lane * 8));
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            v[c * 8 + 2 * e] = __uint_as_float(w[e] << 16);
+            v[c * 8 + 2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+        }
+    }
+}
+
+template <>
+__device__ __forceinline__ void load32<float>(const float* __restrict__ src, int lane, float (&v)[32]) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        float4 a = __ldg(reinterpret_cast<const float4*>(src + c * 256 + lane * 8));
+        float4 b = __ldg(reinterpret_cast<const float4*>(src + c * 256 + lane * 8 + 4));
+        v[c * 8 + 0] = a.x; v[c * 8 + 1] = a.y; v[c * 8 + 2] = a.z; v[c * 8 + 3] = a.w;
+        v[c * 8 + 4] = b.x; v[c * 8 + 5] = b.y; v[c * 8 + 6] = b.z; v[c * 8 + 7] = b.w;
+    }
+}
+
+// One warp per (row, group).  Steps in the order of Algorithm 1:
+//   s = ||w||_2 ; w+ = H diag(sign) (w/s) ; code = argmin_c ||w+_t - G[c]||^2 ; scale = s/sqrt(g).
+// Distances are fp32 in the plain (x-g)^2 form; '<' keeps the lowest index on ties.
+template <typename T, int P>
+__global__ void __launch_bounds__(128) encode_kernel(const T* __restrict__ W, const float* __restrict__ grid, int n,
+                                                     uint8_t* __restrict__ canonical, __half* __restrict__ scales,
+                                                     int64_t N, int64_t K, uint64_t xi) {
+    __shared__ float sgrid[256 * 2];
+    for (int i = threadIdx.x; i < n * P; i += blockDim.x) sgrid[i] = grid[i];
+    __syncthreads();
+
+    const int lane = threadIdx.x & 31;
+    const int64_t groups = K / kGroup;
+    const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (warp >= N * groups) return;
+    const int64_t row = warp / groups, gi = warp % groups;
+
+    float v[32];
+    load32<T>(W + row * K + gi * kGroup, lane, v);
+
+    float ss = 0.0f;
+#pragma unroll
+    for (int r = 0; r < 32; ++r) ss = fmaf(v[r], v[r], ss);
+#pragma unroll
+    for (int m = 16; m >= 1; m >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, m);
+    const float s = sqrtf(ss);
+    const float inv = s > 0.0f ? 1.0f / s : 0.0f;
+
+#pragma unroll
+    for (int r = 0; r < 32; ++r) {
+        uint32_t sb = sign_bit(xi, gi * kGroup + fwht_index(lane, r));
+        v[r] = __uint_as_float(__float_as_uint(v[r] * inv) ^ (sb << 31));
+    }
+    fwht1024_warp(v, lane);
+
+    if (lane == 0) scales[row * groups + gi] = __float2half_rn(s * 0.03125f);
+
+    if (P == 2) {
+        float best[16];
+        int bi[16];
+#pragma unroll
+        for (int t = 0; t < 16; ++t) { best[t] = INFINITY; bi[t] = 0; }
+#pragma unroll 2
+        for (int c = 0; c < n; ++c) {
+            const float2 gp = *reinterpret_cast<const float2*>(&sgrid[2 * c]);
+#pragma unroll
+            for (int t = 0; t < 16; ++t) {
+                const float dx = v[2 * t] - gp.x, dy = v[2 * t + 1] - gp.y;
+                const float d = fmaf(dy, dy, dx * dx);
+                if (d < best[t]) { best[t] = d; bi[t] = c; }
+            }
+        }
+        // pair t of chunk c sits at tuple index c*128 + lane*4 + (t&3): 4 consecutive bytes per chunk
+        uint8_t* dst = canonical + row * (K / 2) + gi * (kGroup / 2);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            uint32_t w = (uint32_t)bi[c * 4] | ((uint32_t)bi[c * 4 + 1] << 8) | ((uint32_t)bi[c * 4 + 2] << 16) |
+                         ((uint32_t)bi[c * 4 + 3] << 24);
+            *reinterpret_cast<uint32_t*>(dst + c * 128 + lane * 4) = w;
+        }
+    } else {
+        float best[32];
+        int bi[32];
+#pragma unroll
+        for (int t = 0; t < 32; ++t) { best[t] = INFINITY; bi[t] = 0; }
+#pragma unroll 2
+        for (int c = 0; c < n; ++c) {
+            const float gp = sgrid[c];
+#pragma unroll
+            for (int t = 0; t < 32; ++t) {
+                const float dx = v[t] - gp;
+                const float d = dx * dx;
+                if (d < best[t]) { best[t] = d; bi[t] = c; }
+            }
+        }
+        uint8_t* dst = canonical + row * K + gi * kGroup;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            uint32_t w0 = (uint32_t)bi[c * 8] | ((uint32_t)bi[c * 8 + 1] << 8) | ((uint32_t)bi[c * 8 + 2] << 16) |
+                          ((uint32_t)bi[c * 8 + 3] << 24);
+            uint32_t w1 = (uint32_t)bi[c * 8 + 4] | ((uint32_t)bi[c * 8 + 5] << 8) | ((uint32_t)bi[c * 8 + 6] << 16) |
+                          ((uint32_t)bi[c * 8 + 7] << 24);
+            *reinterpret_cast<uint2*>(dst + c * 256 + lane * 8) = make_uint2(w0, w1);
+        }
+    }
+}
+
+// ---- packed layout -----------------------------------------------------------
+// The packed stream is a sequence of blocks, block (rt, kb) covering rows
+// [16 rt, 16 rt + 16) and inputs [64 kb, 64 kb + 64), stored at block index
+// rt * (K/64) + kb.  Inside a block, lane L of the consuming warp owns a
+// contiguous run of bytes holding exactly the table indices of the A-fragment
+// registers it feeds to four m16n8k16 tensor-core steps: step m (inputs
+// 16m..16m+15 of the block), register a in 0..3 is the fp16 pair
+//   row   = 16 rt + (L>>2) + 8 (a&1)
+//   pairs = inputs 64 kb + 16 m + 2 (L&3) + 8 (a>>1) + {0, 1}.
+// "Slot" s = 4m + a, 16 slots per lane.
+//   byte-LUT format: 16 bytes per lane, byte s = table index of slot s; a block is
+//                    512 contiguous bytes, lane L at byte offset 16 L.
+//   six-bit format : three 32-bit words per lane and block.  Words 0 and 1 hold the
+//                    low nibbles: slot 4m+a sits in word m>>1 at bit 8a + 4(m&1).
+//                    Word 2 holds the high bit-pairs: slot 4m+a at bit 8a + 2m.
+//                    (The consumer rebuilds four byte-aligned indices with one shift
+//                    and one three-input logic operation each, see linear_mma.cu.)
+//                    Two neighbouring blocks (2j, 2j+1 along K) form a 768-byte
+//                    super-block of three 256-byte planes; plane w stores word w of
+//                    lane L, block half h at 32-bit index 2L + h, so a warp reads
+//                    each plane with one coalesced 64-bit load per lane.
+__device__ __forceinline__ void slot_coords(int64_t rt, int64_t kb, int L, int s, int64_t& row, int64_t& pair) {
+    const int m = s >> 2, a = s & 3;
+    row = rt * 16 + (L >> 2) + 8 * (a & 1);
+    pair = kb * 32 + m * 8 + (L & 3) + 4 * (a >> 1);   // index of the 2-input pair along K
+}
+
+// table index of a pair of inputs (2 consecutive k) from the canonical codes
+template <int P>
+__device__ __forceinline__ uint32_t pair_index(const uint8_t* __restrict__ canonical, int64_t K, int64_t row,
+                                               int64_t pair) {
+    if (P == 2) return canonical[row * (K / 2) + pair];
+    const uint8_t* q = canonical + row * K + 2 * pair;
+    return (uint32_t)(q[0] & 15) | ((uint32_t)(q[1] & 15) << 4);
+}
+
+__device__ __forceinline__ void six_bit_store(uint32_t (&w)[3], int s, uint32_t code) {
+    const int m = s >> 2, a = s & 3;
+    w[m >> 1] |= (code & 15u) << (8 * a + 4 * (m & 1));
+    w[2] |= ((code >> 4) & 3u) << (8 * a + 2 * m);
+}
+__device__ __forceinline__ uint32_t six_bit_load(const uint32_t (&w)[3], int s) {
+    const int m = s >> 2, a = s & 3;
+    const uint32_t lo = (w[m >> 1] >> (8 * a + 4 * (m & 1))) & 15u;
+    const uint32_t hi = (w[2] >> (8 * a + 2 * m)) & 3u;
+    return lo | (hi << 4);
+}
+// 32-bit index of word w of (block kb, lane L) in the six-bit stream
+__device__ __forceinline__ int64_t six_bit_word(int64_t rt, int64_t kb, int64_t kblocks, int L, int w) {
+    return ((rt * (kblocks >> 1) + (kb >> 1)) * 3 + w) * 64 + 2 * L + (kb & 1);
+}
+
+template <int P, bool SIX>
+__global__ void __launch_bounds__(256) pack_kernel(const uint8_t* __restrict__ canonical, uint32_t* __restrict__ packed,
+                                                   int64_t N, int64_t K) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t kblocks = K / kBlockK;
+    const int64_t total = (N / 16) * kblocks * 32;
+    if (t >= total) return;
+    const int L = (int)(t & 31);
+    const int64_t blk = t >> 5, rt = blk / kblocks, kb = blk % kblocks;
+    if (SIX) {
+        uint32_t w[3] = {0u, 0u, 0u};
+        for (int s = 0; s < 16; ++s) {
+            int64_t row, pair;
+            slot_coords(rt, kb, L, s, row, pair);
+            six_bit_store(w, s, pair_index<P>(canonical, K, row, pair) & 63u);
+        }
+        for (int i = 0; i < 3; ++i) packed[six_bit_word(rt, kb, kblocks, L, i)] = w[i];
+    } else {
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
+        for (int s = 0; s < 16; ++s) {
+            int64_t row, pair;
+            slot_coords(rt, kb, L, s, row, pair);
+            w[s >> 2] |= pair_index<P>(canonical, K, row, pair) << (8 * (s & 3));
+        }
+        reinterpret_cast<uint4*>(packed)[t] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
+template <int P, bool SIX>
+__global__ void __launch_bounds__(256) unpack_kernel(const uint32_t* __restrict__ packed, uint8_t* __restrict__ canonical,
+                                                     int64_t N, int64_t K) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t kblocks = K / kBlockK;
+    const int64_t total = (N / 16) * kblocks * 32;
+    if (t >= total) return;
+    const int L = (int)(t & 31);
+    const int64_t blk = t >> 5, rt = blk / kblocks, kb = blk % kblocks;
+    uint32_t w6[3] = {0u, 0u, 0u};
+    uint32_t w8[4] = {0u, 0u, 0u, 0u};
+    if (SIX) {
+        for (int i = 0; i < 3; ++i) w6[i] = packed[six_bit_word(rt, kb, kblocks, L, i)];
+    } else {
+        uint4 q = reinterpret_cast<const uint4*>(packed)[t];
+        w8[0] = q.x; w8[1] = q.y; w8[2] = q.z; w8[3] = q.w;
+    }
+    for (int s = 0; s < 16; ++s) {
+        int64_t row, pair;
+        slot_coords(rt, kb, L, s, row, pair);
+        const uint32_t idx = SIX ? six_bit_load(w6, s) : ((w8[s >> 2] >> (8 * (s & 3))) & 255u);
+        if (P == 2) {
+            canonical[row * (K / 2) + pair] = (uint8_t)idx;
+        } else {
+            canonical[row * K + 2 * pair] = (uint8_t)(idx & 15u);
+            canonical[row * K + 2 * pair + 1] = (uint8_t)(idx >> 4);
+        }
+    }
+}
+
+}  // namespace
+
+int launch_encode(const higgs_desc& d, const void* W, int w_dtype, const float* grid, uint8_t* canonical, void* scales,
+                  cudaStream_t st) {
+    const int64_t warps = d.N * (d.K / kGroup);
+    if (warps == 0) return HIGGS_OK;
+    const unsigned blocks = (unsigned)((warps + 3) / 4);
+    __half* sc = static_cast<__half*>(scales);
+#define HIGGS_ENC(T, P) \
+    encode_kernel<T, P><<<blocks, 128, 0, st>>>(static_cast<const T*>(W), grid, d.n, canonical, sc, d.N, d.K, d.rht_seed)
+    if (w_dtype == HIGGS_F32 && d.p == 2) HIGGS_ENC(float, 2);
+    else if (w_dtype == HIGGS_F32 && d.p == 1) HIGGS_ENC(float, 1);
+    else if (w_dtype == HIGGS_BF16 && d.p == 2) HIGGS_ENC(__nv_bfloat16, 2);
+    else if (w_dtype == HIGGS_BF16 && d.p == 1) HIGGS_ENC(__nv_bfloat16, 1);
+    else return HIGGS_ERR_UNSUPPORTED;
+#undef HIGGS_ENC
+    return cuda_status(cudaGetLastError());
+}
+
+int launch_pack(const higgs_desc& d, const uint8_t* canonical, void* packed, cudaStream_t st) {
+    const int64_t total = (d.N / 16) * (d.K / kBlockK) * 32;
+    if (total == 0) return HIGGS_OK;
+    const unsigned blocks = (unsigned)((total + 255) / 256);
+    uint32_t* out = static_cast<uint32_t*>(packed);
+    const Format f = format_of(d.p, d.n);
+    if (f == Format::kByteLut && d.p == 2) pack_kernel<2, false><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K);
+    else if (f == Format::kByteLut && d.p == 1) pack_kernel<1, false><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K);
+    else if (f == Format::kSixBit) pack_kernel<2, true><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K);
+    else return HIGGS_ERR_UNSUPPORTED;
+    return cuda_status(cudaGetLastError());
+}
+
+int launch_unpack(const higgs_desc& d, const void* packed, uint8_t* canonical, cudaStream_t st) {
+    const int64_t total = (d.N / 16) * (d.K / kBlockK) * 32;
+    if (total == 0) return HIGGS_OK;
+    const unsigned blocks = (unsigned)((total + 255) / 256);
+    const uint32_t* in = static_cast<const uint32_t*>(packed);
+    const Format f = format_of(d.p, d.n);
+    if (f == Format::kByteLut && d.p == 2) unpack_kernel<2, false><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K);
+    else if (f == Format::kByteLut && d.p == 1) unpack_kernel<1, false><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K);
+    else if (f == Format::kSixBit) unpack_kernel<2, true><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K);
+    else return HIGGS_ERR_UNSUPPORTED;
+    return cuda_status(cudaGetLastError());
+}
+
+}  // namespace higgs

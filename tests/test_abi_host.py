@@ -1,0 +1,94 @@
+"""CPU-only checks of the C-ABI library: it loads, exports every declared symbol, and its host logic
+(size queries, argument validation, the sign function) behaves as include/higgs.h documents."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2411_17525_b200 as hb
+from paper_2411_17525_b200 import binding
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if fn.endswith(".h"):
+            src = open(os.path.join(ROOT, "include", fn)).read()
+            src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+            names |= set(re.findall(r"\b(higgs_[a-z0-9_]+)\s*\(", src))
+    return sorted(names)
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_symbols()
+    assert len(names) >= 12 and "higgs_linear" in names and "higgs_quantize" in names and "higgs_make_grid" in names
+    lib = ctypes.CDLL(hb.LIB_PATH)
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(binding.EXPORTS) <= set(names)
+
+
+def test_sign_function_matches_oracle_statement():
+    for seed in (0, 1, 0x48494747, 2**64 - 1, 0x123456789ABCDEF0):
+        got = [hb.higgs_sign(seed, j) for j in range(512)]
+        want = [int(oracle.sign(seed, j)) for j in range(512)]
+        assert got == want
+    assert hb.higgs_sign(7, 10**12) == int(oracle.sign(7, 10**12))
+
+
+def test_size_queries():
+    d = hb.make_desc(2, 256, 4096, 14336, 1)
+    assert hb.higgs_packed_bytes(d) == 4096 * 14336 // 2          # 4 bits per weight
+    assert hb.higgs_scales_bytes(d) == 4096 * 14 * 2              # one fp16 per (row, group)
+    assert hb.higgs_canonical_bytes(d) == 4096 * 14336 // 2
+    d = hb.make_desc(2, 64, 4096, 4096, 1)
+    assert hb.higgs_packed_bytes(d) == 4096 * 4096 * 3 // 8       # 3 bits per weight
+    d = hb.make_desc(1, 16, 1024, 4096, 1)
+    assert hb.higgs_packed_bytes(d) == 1024 * 4096 // 2
+    assert hb.higgs_canonical_bytes(d) == 1024 * 4096
+    assert hb.higgs_workspace_bytes(d, hb.HIGGS_OP_LINEAR, 16) >= 16 * 4096 * 2
+    assert hb.higgs_workspace_bytes(d, hb.HIGGS_OP_LINEAR, 0) == 0
+    # effective bits per weight incl. scales, as the paper counts them: 4 + 16/1024
+    d = hb.make_desc(2, 256, 4096, 4096, 1)
+    bpw = 8.0 * (hb.higgs_packed_bytes(d) + hb.higgs_scales_bytes(d)) / (4096 * 4096)
+    assert round(bpw, 2) == 4.02
+
+
+@pytest.mark.parametrize("p,n,g,N,K", [(2, 100, 1024, 16, 1024), (3, 256, 1024, 16, 1024), (2, 256, 512, 16, 1024),
+                                       (2, 256, 1024, 15, 1024), (2, 256, 1024, 16, 1000), (1, 256, 1024, 16, 1024)])
+def test_unsupported_descriptors_are_refused(p, n, g, N, K):
+    d = hb.make_desc(p, n, N, K, 1, g=g)
+    assert hb.higgs_packed_bytes(d) == 0
+    rc = binding.lib.higgs_linear(ctypes.byref(d), None, 1, None, None, None, None, 0, None, 0, None)
+    assert rc == hb.HIGGS_ERR_UNSUPPORTED
+    rc = binding.lib.higgs_quantize(ctypes.byref(d), None, 0, None, None, None, None, None, 0, None)
+    assert rc == hb.HIGGS_ERR_UNSUPPORTED
+
+
+def test_invalid_arguments_are_refused_before_any_cuda_call():
+    d = hb.make_desc(2, 256, 16, 1024, 1)
+    L = binding.lib
+    assert L.higgs_linear(None, None, 1, None, None, None, None, 0, None, 0, None) == hb.HIGGS_ERR_INVALID_ARG
+    assert L.higgs_linear(ctypes.byref(d), None, 1, None, None, None, None, 0, None, 0, None) == hb.HIGGS_ERR_INVALID_ARG
+    assert L.higgs_linear(ctypes.byref(d), None, -1, None, None, None, None, 0, None, 0, None) == hb.HIGGS_ERR_INVALID_ARG
+    assert L.higgs_linear(ctypes.byref(d), None, 0, None, None, None, None, 0, None, 0, None) == hb.HIGGS_OK  # empty batch
+    assert L.higgs_linear(ctypes.byref(d), None, 1, None, None, None, None, 7, None, 0, None) == hb.HIGGS_ERR_UNSUPPORTED
+    assert L.higgs_quantize(ctypes.byref(d), None, 0, None, None, None, None, None, 0, None) == hb.HIGGS_ERR_INVALID_ARG
+    assert L.higgs_quantize(ctypes.byref(d), None, 1, None, None, None, None, None, 0, None) == hb.HIGGS_ERR_UNSUPPORTED
+    # misaligned and undersized workspace (fake non-null addresses are never dereferenced on these paths)
+    a = ctypes.c_void_p(0x1000)
+    assert L.higgs_linear(ctypes.byref(d), a, 1, a, a, a, a, 0, ctypes.c_void_p(0x1010), 1 << 20, None) == hb.HIGGS_ERR_INVALID_ARG
+    assert L.higgs_linear(ctypes.byref(d), a, 1, a, a, a, a, 0, a, 16, None) == hb.HIGGS_ERR_WORKSPACE
+    assert L.higgs_quantize(ctypes.byref(d), a, 0, a, a, a, None, a, 16, None) == hb.HIGGS_ERR_WORKSPACE
+    assert L.higgs_make_grid(2, 256, a, 100, 10, a, None, None, a, 1 << 30, None) == hb.HIGGS_ERR_INVALID_ARG  # fewer samples than points
+    assert L.higgs_make_grid(3, 256, a, 1000, 10, a, None, None, a, 1 << 30, None) == hb.HIGGS_ERR_UNSUPPORTED
+    assert L.higgs_make_grid(2, 256, a, 1000, 10, a, None, None, a, 16, None) == hb.HIGGS_ERR_WORKSPACE
+    empty = hb.make_desc(2, 256, 0, 1024, 1)
+    assert L.higgs_quantize(ctypes.byref(empty), None, 0, None, None, None, None, None, 0, None) == hb.HIGGS_OK
+    for s in range(7):
+        assert isinstance(hb.status_string(s), str) and hb.status_string(s)

@@ -1,0 +1,208 @@
+"""GPU parity tests: the CUDA path (through the C ABI) against the fp64 oracle on the same seeded inputs.
+
+Bars: codes bit-exact except near-ties (oracle margin < 1e-5, GPU code = oracle runner-up, fewer than 1e-4 of
+all codes); layer outputs, given identical codes, within max|dy|/max|y| <= 2e-3.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2411_17525_b200 as hb
+from synth import inputs
+from tests import gpu_util as U
+
+pytestmark = pytest.mark.gpu
+
+G = 1024
+Y_TOL = 2e-3
+
+
+# ----------------------------------------------------------------------------- RHT
+@pytest.mark.parametrize("rows,K,dtype", [(1, 1024, "f32"), (3, 2048, "f32"), (5, 4096, "bf16"), (17, 1024, "bf16")])
+def test_rht_matches_oracle(rows, K, dtype):
+    rng = np.random.default_rng(rows * K)
+    x = rng.standard_normal((rows, K)).astype(np.float32)
+    xi = inputs.rht_seed(0)
+    d = hb.make_desc(2, 256, 16, K, xi)
+    if dtype == "bf16":
+        x = inputs.bf16_round(x)
+        xt = U.bf16_tensor(x)
+    else:
+        xt = U.f32_tensor(x)
+    sg = oracle.signs(xi, K)
+    for normalised in (False, True):
+        got = hb.higgs_rht(d, xt, normalised).cpu().numpy().astype(np.float64)
+        want = np.stack([np.concatenate([oracle.rht(x[r, i * G:(i + 1) * G].astype(np.float64), sg[i * G:(i + 1) * G], normalised)
+                                         for i in range(K // G)]) for r in range(rows)])
+        scale = np.abs(want).max()
+        assert np.max(np.abs(got - want)) <= 2e-6 * scale
+
+
+# ----------------------------------------------------------------------------- encoder
+def run_quantize(W32, p, n, xi, bf16):
+    N, K = W32.shape
+    d = hb.make_desc(p, n, N, K, xi)
+    g64, gt = U.grid32(p, n)
+    Wt = U.bf16_tensor(W32) if bf16 else U.f32_tensor(W32)
+    packed, scales, canon = hb.higgs_quantize(d, Wt, gt, want_canonical=True)
+    torch.cuda.synchronize()
+    return d, g64, gt, packed, scales, canon
+
+
+@pytest.mark.parametrize("p,n,N,K,bf16", [
+    (2, 256, 512, 1024, False),     # the single-layer reference configuration (fp32 weights, one group per row)
+    (2, 256, 48, 3072, True),       # several groups per row, ragged against any block size
+    (2, 64, 80, 2048, True),
+    (1, 16, 64, 2048, True),
+    (2, 256, 16, 1024, False),      # smallest supported matrix
+])
+def test_quantize_codes_and_scales(p, n, N, K, bf16):
+    W = inputs.make_weights(N, K, seed=inputs.weight_seed(0, n + N), bf16=bf16)
+    xi = inputs.rht_seed(0)
+    d, g64, gt, packed, scales, canon = run_quantize(W, p, n, xi, bf16)
+    q, sc16 = U.oracle_encode(W, G, g64, xi)
+    gpu_codes = canon.cpu().numpy()
+    assert gpu_codes.shape == q.codes.shape and gpu_codes.max() < n
+    U.compare_codes(gpu_codes, q)
+    # scales: fp32 norm then fp16 rounding; at most one fp16 ulp from the oracle's, almost all identical
+    s_gpu = scales.cpu().numpy()
+    ulp = np.abs(s_gpu.view(np.int16).astype(np.int64) - sc16.view(np.int16).astype(np.int64))
+    assert ulp.max() <= 1 and (ulp == 0).mean() > 0.98
+    # the packed stream holds exactly the canonical codes
+    back = hb.higgs_unpack_codes(d, packed).cpu().numpy()
+    assert np.array_equal(back, gpu_codes)
+    repacked = hb.higgs_pack_codes(d, canon)
+    assert torch.equal(repacked[: hb.higgs_packed_bytes(d)], packed[: hb.higgs_packed_bytes(d)])
+    # without the optional canonical output (codes staged in the workspace) the stream is the same
+    Wt = U.bf16_tensor(W) if bf16 else U.f32_tensor(W)
+    packed2, scales2, none = hb.higgs_quantize(d, Wt, gt, want_canonical=False)
+    assert none is None and torch.equal(packed2, packed) and torch.equal(scales2, scales)
+
+
+def test_quantize_invariants_on_gpu():
+    """Power-of-two scaling leaves codes unchanged and scales exact; zero groups stay finite."""
+    p, n, N, K = 2, 256, 32, 2048
+    xi = 99
+    W = inputs.make_weights(N, K, seed=5, bf16=False)
+    d, g64, gt, packed, scales, canon = run_quantize(W, p, n, xi, False)
+    d2, _, _, packed2, scales2, canon2 = run_quantize(W * 4.0, p, n, xi, False)
+    assert torch.equal(canon, canon2) and torch.equal(scales * 4.0, scales2)
+    Wz = W.copy()
+    Wz[3, :1024] = 0.0
+    dz, _, _, _, scz, cz = run_quantize(Wz, p, n, xi, False)
+    origin = int(np.argmin((g64 ** 2).sum(1)))
+    assert float(scz[3, 0]) == 0.0 and bool((cz[3, :512] == origin).all())
+    assert torch.equal(cz[4:], canon[4:]) and bool(torch.isfinite(scz.float()).all())
+
+
+# ----------------------------------------------------------------------------- decode
+def run_linear_case(p, n, N, K, B, xi, wseed, xseed, out_dtype=torch.float32, lognormal=False):
+    W = inputs.make_weights(N, K, seed=wseed, bf16=True)
+    x = inputs.make_activations(B, K, seed=xseed, lognormal_channels=lognormal)
+    g64, gt = U.grid32(p, n)
+    q, sc16 = U.oracle_encode(W, G, g64, xi)
+    d = hb.make_desc(p, n, N, K, xi)
+    canon = torch.from_numpy(q.codes.astype(np.uint8)).to(U.dev())
+    packed = hb.higgs_pack_codes(d, canon)                       # identical codes on both sides
+    scales = torch.from_numpy(sc16).to(U.dev())
+    y = hb.higgs_linear(d, U.bf16_tensor(x), packed, scales, gt, out_dtype=out_dtype)
+    torch.cuda.synchronize()
+    y_ref = oracle.linear_dense(x.astype(np.float64), q.codes, sc16.astype(np.float64), G, g64, xi)
+    return y, y_ref
+
+
+@pytest.mark.parametrize("p,n,N,K,B", [
+    (2, 256, 512, 1024, 1),      # reference configuration
+    (2, 256, 48, 2048, 1),
+    (2, 256, 48, 2048, 3),
+    (2, 256, 272, 4096, 8),
+    (2, 256, 272, 4096, 9),
+    (2, 256, 64, 8192, 16),      # K split over several blocks (atomic accumulation)
+    (2, 256, 32, 14336, 1),
+    (2, 256, 32, 14336, 16),
+    (2, 64, 48, 2048, 1),
+    (2, 64, 272, 4096, 4),
+    (2, 64, 64, 8192, 16),
+    (2, 64, 32, 1024, 12),
+    (1, 16, 48, 2048, 1),
+    (1, 16, 64, 4096, 16),
+    (2, 256, 16, 1024, 17),      # more tokens than one launch takes
+    (2, 256, 32, 2048, 40),
+])
+def test_linear_matches_oracle_given_identical_codes(p, n, N, K, B):
+    y, y_ref = run_linear_case(p, n, N, K, B, xi=inputs.rht_seed(2), wseed=100 + N, xseed=200 + B)
+    assert y.shape == (B, N) and y.dtype == torch.float32
+    err = U.linear_error(y.cpu().numpy(), y_ref)
+    assert err <= Y_TOL, err
+    assert err <= 6e-4, err   # expected level for fp16 operands with fp32 accumulation
+
+
+def test_linear_bf16_output_and_outlier_channels():
+    y, y_ref = run_linear_case(2, 256, 64, 8192, 8, xi=3, wseed=7, xseed=8, out_dtype=torch.bfloat16, lognormal=True)
+    assert y.dtype == torch.bfloat16
+    # bf16 output rounding (2^-9 relative per element) sits on top of the fp32 result
+    err = U.linear_error(y.float().cpu().numpy(), y_ref)
+    assert err <= Y_TOL + 2.0 ** -9
+    y32, _ = run_linear_case(2, 256, 64, 8192, 8, xi=3, wseed=7, xseed=8, lognormal=True)
+    assert U.linear_error(y32.cpu().numpy(), y_ref) <= Y_TOL
+    y1, y1_ref = run_linear_case(2, 256, 64, 2048, 2, xi=3, wseed=7, xseed=8, out_dtype=torch.bfloat16)
+    assert U.linear_error(y1.float().cpu().numpy(), y1_ref) <= Y_TOL + 2.0 ** -9
+
+
+def test_end_to_end_quantize_then_linear():
+    """GPU encoder feeding GPU decode approximates the unquantised layer at the level the grid's MSE predicts
+    (Appendix E: relative error^2 ~= t^2(grid)), and equals the oracle's layer on the oracle's own codes except
+    for the few near-tie codes."""
+    p, n, N, K, B = 2, 256, 256, 4096, 4
+    xi = inputs.rht_seed(2)
+    W = inputs.make_weights(N, K, seed=31, bf16=True)
+    x = inputs.make_activations(B, K, seed=32)
+    d, g64, gt, packed, scales, canon = run_quantize(W, p, n, xi, True)
+    y = hb.higgs_linear(d, U.bf16_tensor(x), packed, scales, gt).cpu().numpy().astype(np.float64)
+    y0 = x.astype(np.float64) @ W.astype(np.float64).T
+    rel = np.linalg.norm(y - y0) / np.linalg.norm(y0)
+    assert 0.06 < rel < 0.12          # sqrt(0.0078) = 0.088
+    q, sc16 = U.oracle_encode(W, G, g64, xi)
+    y_ref = oracle.linear_dense(x.astype(np.float64), q.codes, sc16.astype(np.float64), G, g64, xi)
+    assert U.linear_error(y, y_ref) <= Y_TOL
+
+
+def test_empty_inputs():
+    d = hb.make_desc(2, 256, 0, 1024, 1)
+    _, gt = U.grid32(2, 256)
+    W = torch.empty((0, 1024), dtype=torch.float32, device=U.dev())
+    packed, scales, canon = hb.higgs_quantize(d, W, gt, want_canonical=True)
+    assert scales.shape == (0, 1) and canon.shape == (0, 512)
+    d = hb.make_desc(2, 256, 16, 1024, 1)
+    x = torch.empty((0, 1024), dtype=torch.bfloat16, device=U.dev())
+    y = hb.higgs_linear(d, x, torch.zeros(16 * 512, dtype=torch.uint8, device=U.dev()),
+                        torch.zeros((16, 1), dtype=torch.float16, device=U.dev()), gt)
+    assert y.shape == (0, 16)
+
+
+# ----------------------------------------------------------------------------- grid fit
+@pytest.mark.parametrize("p,n", [(2, 64), (1, 16)])
+def test_make_grid_is_a_lloyd_fixed_point_at_the_oracle_mse(p, n):
+    s = inputs.gaussian_samples(p, inputs.grid_sample_seed(p, n), log2_count=16)
+    st = U.f32_tensor(s)
+    grid, mse, iters = hb.higgs_make_grid(p, n, st, max_iters=3000)
+    torch.cuda.synchronize()
+    g = grid.cpu().numpy().astype(np.float64)
+    assert int(iters) > 5, int(iters)                 # converged (negative = ran out of iterations)
+    # sorted lexicographically
+    keys = [tuple(r) for r in g]
+    assert keys == sorted(keys)
+    s32 = s.astype(np.float32).astype(np.float64)
+    # reported MSE equals the oracle's evaluation of the device grid on the same samples
+    assert abs(float(mse) - oracle.grid_mse(g, s32)) <= 1e-5 * float(mse)
+    # fixed point: one more oracle Lloyd step from the device grid leaves it in place
+    d2 = ((s32[:, None, :] - g[None, :, :]) ** 2).sum(-1)
+    a = d2.argmin(1)
+    means = np.stack([s32[a == c].mean(0) for c in range(n)])
+    assert np.max(np.abs(means - g)) < 5e-6
+    # quality: held-out MSE within 1% of the oracle's own fit on the same samples
+    ref = oracle.make_grid_lloyd(p, n, s32, max_iters=4000)
+    fresh = inputs.gaussian_samples(p, 777, log2_count=20)
+    m_dev, m_ref = oracle.grid_mse(g, fresh), oracle.grid_mse(ref.grid, fresh)
+    assert abs(m_dev - m_ref) <= 0.01 * m_ref
