@@ -19,8 +19,9 @@ def path(p, n):
 
 
 def load(p, n):
+    """The stored table as float64 holding exactly the fp32 values (9 printed digits identify an fp32)."""
     g = np.loadtxt(path(p, n), dtype=np.float64, comments="#", ndmin=2)
-    return g.reshape(n, p)
+    return g.astype(np.float32).astype(np.float64).reshape(n, p)
 
 
 def main():
