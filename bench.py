@@ -1,0 +1,432 @@
+#!/usr/bin/env python
+"""Benchmark of the HIGGS quantized linear layer on B200.
+
+One "step" = one decode pass (Appendix F: rotate activations, stream codes, table lookup, contraction, reduce)
+over every layer of a Llama-shaped layer set for one batch of synthetic activations.  The headline value is the
+effective weight bandwidth (packed codes + scales bytes of the layer set / time per step).  The encoder
+(Algorithm 1) and the grid fit (Algorithm 2) run once during set-up, on the GPU, and are reported separately.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama-3.2-1b] [--batch 1] [--grid 2,256]
+    python bench.py --impl reference ...      # the fp64 CPU oracle timed on the host cores (reported baseline)
+
+Under torchrun (N > 1) every rank runs an independent replica of the same layer set on its own GPU (the layer
+needs no collective); the reported value is the sum over ranks divided by the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from synth import inputs  # noqa: E402
+
+G = 1024
+L2_BYTES = 126 * 1024 * 1024
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", default="llama-3.2-1b", choices=list(inputs.LAYER_SETS))
+    ap.add_argument("--batch", type=int, default=1)
+    ap.add_argument("--grid", default="2,256", help="p,n")
+    ap.add_argument("--no-graph", action="store_true", help="launch kernels directly instead of replaying CUDA graphs")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-detail", action="store_true", help="skip the per-layer / other-batch detail measurements")
+    return ap.parse_args()
+
+
+def layer_bytes(N, K, p, n):
+    bits = {(2, 256): 4, (1, 16): 4, (2, 64): 3}[(p, n)]
+    return N * K * bits // 8 + N * (K // G) * 2
+
+
+def algorithmic_bytes(N, K, p, n, B):
+    """codes + scales + activations in + outputs out + grid table (per launch of the product kernel)."""
+    return layer_bytes(N, K, p, n) + B * K * 2 + B * N * 4 + n * p * 4
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [c.strip() for c in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------- reference arm
+def run_reference(args):
+    """The fp64 oracle (as it stands) on the host cores: the same metric on a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from tests.golden import make_grids
+
+    p, n = (int(v) for v in args.grid.split(","))
+    layers = inputs.LAYER_SETS[args.workload]
+    cfg = inputs.CONFIG_OF_SET[args.workload]
+    xi = inputs.rht_seed(cfg)
+    grid = make_grids.load(p, n)
+    B = args.batch
+    rows = 64  # rows of every layer per step: rows are independent, so this is a plain sample of the layer set
+    sample = []
+    for li, (name, N, K) in enumerate(layers):
+        r = min(rows, N)
+        W = inputs.make_weights(r, K, inputs.weight_seed(cfg, li), bf16=True).astype(np.float64)
+        q = oracle.quantize(W, G, grid, xi)
+        sc = oracle.round_scales_fp16(q.scales).astype(np.float64)
+        x = inputs.make_activations(B, K, inputs.activation_seed(cfg, B) + li).astype(np.float64)
+        sample.append((q.codes, sc, x, r, K))
+    nbytes = sum(layer_bytes(r, K, p, n) for _, _, _, r, K in sample)
+
+    def step():
+        for codes, sc, x, r, K in sample:
+            oracle.linear_dense(x, codes, sc, G, grid, xi)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / max(args.steps, 1)
+    value = nbytes / dt / 1e9
+    desc = f"{rows} rows of each of the {len(layers)} layers per step (rows are independent), dequantise + fp64 matmul"
+    line = {
+        "impl": "reference", "metric": "higgs_linear_effective_weight_bandwidth", "value": value, "unit": "GB/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{args.workload} layer set, grid p={p} n={n}, g=1024, batch {B}", "sample": desc},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": oracle.threads(), "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------------------------- our arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2411_17525_b200 as hb
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the HIGGS kernels have no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    p, n = (int(v) for v in args.grid.split(","))
+    layers = inputs.LAYER_SETS[args.workload]
+    cfg = inputs.CONFIG_OF_SET[args.workload]
+    xi = inputs.rht_seed(cfg)
+    B = args.batch
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    # ---- E0: grid fit on the device (Algorithm 2), 2^18 seeded Gaussian samples
+    samples = torch.from_numpy(inputs.gaussian_samples(p, inputs.grid_sample_seed(p, n)).astype(np.float32)).to(dev)
+    e0, e1 = ev(), ev()
+    e0.record()
+    grid, grid_mse, grid_iters = hb.higgs_make_grid(p, n, samples, max_iters=3000)
+    e1.record()
+    torch.cuda.synchronize()
+    grid_ms = e0.elapsed_time(e1)
+    del samples
+
+    # ---- E1-E4: encode every layer once on the device (Algorithm 1)
+    set_bytes = sum(layer_bytes(N, K, p, n) for _, N, K in layers)
+    copies = max(2, -(-2 * L2_BYTES // set_bytes))          # rotating copies so that no step finds its codes in L2
+    copies = min(copies, 64)
+    descs, packed, scales, xs, xs_host, ws, ys = [], [], [], [], [], [], []
+    enc_ms, enc_weights = 0.0, 0
+    for li, (name, N, K) in enumerate(layers):
+        d = hb.make_desc(p, n, N, K, xi)
+        W = torch.from_numpy(inputs.make_weights(N, K, inputs.weight_seed(cfg, li), bf16=True)).to(dev).to(torch.bfloat16)
+        e0, e1 = ev(), ev()
+        e0.record()
+        pk, sc, _ = hb.higgs_quantize(d, W, grid)
+        e1.record()
+        torch.cuda.synchronize()
+        enc_ms += e0.elapsed_time(e1)
+        enc_weights += N * K
+        del W
+        descs.append(d)
+        packed.append([pk] + [pk.clone() for _ in range(copies - 1)])
+        scales.append([sc] + [sc.clone() for _ in range(copies - 1)])
+        xh = torch.from_numpy(inputs.make_activations(B, K, inputs.activation_seed(cfg, B) + li)).to(torch.bfloat16)
+        xs_host.append(xh.pin_memory())
+        xs.append(xh.to(dev))
+        ws.append(torch.empty(hb.higgs_linear_host_workspace_bytes(d, B), dtype=torch.uint8, device=dev))
+        ys.append(torch.empty((B, N), dtype=torch.float32, device=dev))
+    ys_host = [torch.empty((B, N), dtype=torch.float32).pin_memory() for _, N, _ in layers]
+    launches_per_step = sum(hb.higgs_linear_launch_count(d, B) for d in descs)
+
+    def step(i):
+        c = i % copies
+        for li, d in enumerate(descs):
+            hb.higgs_linear(d, xs[li], packed[li][c], scales[li][c], grid, workspace=ws[li], y=ys[li])
+
+    def step_host(i):
+        c = i % copies
+        for li, d in enumerate(descs):
+            hb.higgs_linear_host(d, xs_host[li], packed[li][c], scales[li][c], grid, ys_host[li], ws[li])
+        torch.cuda.current_stream().synchronize()   # the step's results are read on the host
+
+    # ---- graphs: one per weight copy, replayed in rotation
+    stream = torch.cuda.Stream()
+    graphs = None
+    with torch.cuda.stream(stream):
+        step(0)
+        stream.synchronize()
+        if not args.no_graph:
+            graphs = []
+            for c in range(copies):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    step(c)
+                graphs.append(g)
+
+    def run_step(i):
+        if graphs is not None:
+            graphs[i % copies].replay()
+        else:
+            step(i)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    def timed(fn, steps, warmup):
+        with torch.cuda.stream(stream):
+            for i in range(warmup):
+                fn(i)
+            stream.synchronize()
+            barrier()
+            torch.cuda.synchronize()
+            a, b = ev(), ev()
+            a.record(stream)
+            for i in range(steps):
+                fn(warmup + i)
+            b.record(stream)
+            torch.cuda.synchronize()
+            barrier()
+            ms = a.elapsed_time(b)
+        if world > 1:
+            t = torch.tensor([ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ms = timed(run_step, args.steps, max(args.warmup, 3))
+    ms_e2e = timed(step_host, args.steps, max(args.warmup, 3))
+    clocks = sampler.stop() if rank == 0 else None
+
+    ms_per_step = ms / args.steps
+    value = world * set_bytes / (ms_per_step * 1e-3) / 1e9
+    e2e_value = world * set_bytes / (ms_e2e / args.steps * 1e-3) / 1e9
+    h2d = sum(B * K * 2 for _, _, K in layers)
+    d2h = sum(B * N * 4 for _, N, _ in layers)
+
+    # ---- dominant kernel: the product kernel on the largest layer, timed alone with CUDA events
+    peak, peak_src = measured_peaks()
+    big = max(range(len(layers)), key=lambda i: layers[i][1] * layers[i][2])
+    _, Nb, Kb = layers[big]
+    db = descs[big]
+
+    def kernel_time(li, d, Bk, reps=200):
+        """Average duration of one launch of the product kernel (pre-rotated activations), rotating weight copies."""
+        xdag = hb.higgs_rotate_activations(d, xs[li] if Bk == B else
+                                           torch.from_numpy(inputs.make_activations(Bk, d.K, 1)).to(torch.bfloat16).to(dev))
+        yk = torch.empty((Bk, d.N), dtype=torch.float32, device=dev)
+        wk = torch.empty(hb.higgs_workspace_bytes(d, hb.HIGGS_OP_LINEAR, Bk), dtype=torch.uint8, device=dev)
+        per_launch_bytes = layer_bytes(d.N, d.K, p, n)
+        need = max(2, -(-2 * L2_BYTES // per_launch_bytes))
+        pks = list(packed[li])
+        scs = list(scales[li])
+        while len(pks) < min(need, 64):
+            pks.append(pks[0].clone())
+            scs.append(scs[0].clone())
+        with torch.cuda.stream(stream):
+            g = torch.cuda.CUDAGraph()
+            hb.higgs_linear_prerotated(d, xdag, pks[0], scs[0], grid, workspace=wk, y=yk)
+            stream.synchronize()
+            with torch.cuda.graph(g, stream=stream):
+                for c in range(len(pks)):
+                    hb.higgs_linear_prerotated(d, xdag, pks[c], scs[c], grid, workspace=wk, y=yk)
+            rounds = max(1, reps // len(pks))
+            for _ in range(2):
+                g.replay()
+            stream.synchronize()
+            a, b = ev(), ev()
+            a.record(stream)
+            for _ in range(rounds):
+                g.replay()
+            b.record(stream)
+            stream.synchronize()
+        nodes = hb.higgs_linear_launch_count(d, Bk) - 1
+        return a.elapsed_time(b) * 1e3 / (rounds * len(pks)), nodes   # microseconds per call
+
+    us_big, nodes_big = kernel_time(big, db, B)
+    alg = algorithmic_bytes(Nb, Kb, p, n, B)
+    achieved = alg / (us_big * 1e-6) / 1e9
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tpath):
+        try:
+            with open(tpath) as f:
+                traffic = json.load(f).get(f"{args.workload}:{layers[big][0]}:p{p}n{n}:B{B}")
+        except Exception:
+            traffic = None
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": traffic, "peak_source": f"of {peak_src}", "kernel": "linear_mma_kernel",
+                "layer": f"{layers[big][0]} {Nb}x{Kb}", "us_per_launch": us_big, "algorithmic_bytes": alg,
+                "frac_of_8TBps": achieved / 8000.0}
+
+    detail = None
+    if not args.no_detail and rank == 0:
+        detail = {"layers": []}
+        for li, (name, N, K) in enumerate(layers):
+            if any(l["shape"] == f"{N}x{K}" for l in detail["layers"]):
+                continue
+            us, _ = kernel_time(li, descs[li], B)
+            wb = layer_bytes(N, K, p, n)
+            detail["layers"].append({"name": name, "shape": f"{N}x{K}", "B": B, "us": round(us, 3),
+                                     "weight_GBps": round(wb / us / 1e3, 1), "frac_of_measured": round(wb / us / 1e3 / peak, 4)})
+        if B != 16:
+            us16, _ = kernel_time(big, db, 16)
+            wb = layer_bytes(Nb, Kb, p, n)
+            detail["batch16_largest_layer"] = {"us": round(us16, 3), "weight_GBps": round(wb / us16 / 1e3, 1),
+                                               "frac_of_measured": round(wb / us16 / 1e3 / peak, 4)}
+
+    # ---- CPU baseline: the oracle as it stands on this machine's cores (rank 0, single-GPU runs only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        rows = 256
+        smp = []
+        for li, (name, N, K) in enumerate(layers):
+            r = min(rows, N)
+            W = inputs.make_weights(r, K, inputs.weight_seed(cfg, li), bf16=True).astype(np.float64)
+            g64 = grid.cpu().numpy().astype(np.float64)
+            q = oracle.quantize(W, G, g64, xi)
+            smp.append((q.codes, oracle.round_scales_fp16(q.scales).astype(np.float64), xs_host[li].float().numpy().astype(np.float64), r, K))
+        nb = sum(layer_bytes(r, K, p, n) for *_, r, K in smp)
+        reps, t0 = 0, time.perf_counter()
+        while reps < 3 or time.perf_counter() - t0 < 10.0:
+            for codes, sc, x, r, K in smp:
+                oracle.linear_dense(x, codes, sc, G, g64, xi)
+            reps += 1
+            if time.perf_counter() - t0 > 30.0:
+                break
+        dt = (time.perf_counter() - t0) / reps
+        cpu = {"value": nb / dt / 1e9, "unit": "GB/s", "cores": oracle.threads(), "kind": "oracle",
+               "sample": f"{rows} rows of each of the {len(layers)} layers (rows are independent), dequantise + fp64 matmul, {reps} passes"}
+
+    if rank == 0:
+        line = {
+            "metric": "higgs_linear_effective_weight_bandwidth", "value": value, "unit": "GB/s", "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f16xf16->f32", "data": "synthetic",
+            "config": {"workload": f"{args.workload} layer set ({len(layers)} matrices), grid p={p} n={n}, g=1024, batch {B}",
+                       "global_batch": B * world, "parallelism": f"replicas x{world}",
+                       "l2": f"rotating {copies} weight copies ({copies * set_bytes / 1e6:.0f} MB > 126 MB L2)",
+                       "launch": "direct" if graphs is None else "one CUDA graph per weight copy"},
+            "us_per_layer": ms_per_step * 1e3 / len(layers),
+            "weight_bytes_per_step": set_bytes,
+            "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "ms_per_step": ms_e2e / args.steps},
+            "gpu_launches": launches_per_step * args.steps,
+            "clocks": clocks,
+            "roofline": roofline,
+            "cpu_baseline": cpu,
+            "quantize": {"weights_per_s": enc_weights / (enc_ms * 1e-3), "ms": enc_ms, "weights": enc_weights,
+                         "grid_fit_ms": grid_ms, "grid_fit_iters": int(grid_iters), "grid_mse": float(grid_mse)},
+            "detail": detail,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

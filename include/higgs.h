@@ -68,7 +68,8 @@ typedef enum higgs_op { HIGGS_OP_QUANTIZE = 0, HIGGS_OP_LINEAR = 1, HIGGS_OP_MAK
  * {(2,256), (2,64), (1,16)}; N a multiple of 16, K a multiple of g.
  * Anything else returns HIGGS_ERR_UNSUPPORTED (never padded silently).
  * scale_dtype must be HIGGS_F16: one 16-bit scale per (row, group), which is
- * what the paper's bit counts imply (4.02 = 4 + 16/1024, Appendix G).
+ * what the paper's bit counts imply (4.02 = 4 + 16/1024 in the appendix on
+ * experiment configurations).
  */
 typedef struct higgs_desc {
     int32_t p;
@@ -155,6 +156,38 @@ int higgs_linear(const higgs_desc* desc, const void* x, int64_t B,
                  const void* packed, const void* scales, const float* grid,
                  void* y, int y_dtype,
                  void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The two halves of higgs_linear as separate calls (Section 4.3: the Hadamard
+ * transform "can be fully isolated from the matrix multiplication itself").
+ *   higgs_rotate_activations: x (device [B][K] bf16) -> xdag_out (device [B][K]
+ *     fp16) = (H / sqrt(g)) diag(sign) x per K-group.
+ *   higgs_linear_prerotated: the product of Appendix F on already rotated
+ *     activations xdag (device [B][K] fp16); other arguments as higgs_linear.
+ * higgs_linear(x) == higgs_linear_prerotated(higgs_rotate_activations(x)).
+ */
+int higgs_rotate_activations(const higgs_desc* desc, const void* x, int64_t B, void* xdag_out, void* stream);
+int higgs_linear_prerotated(const higgs_desc* desc, const void* xdag, int64_t B,
+                            const void* packed, const void* scales, const float* grid,
+                            void* y, int y_dtype,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * higgs_linear with HOST activations and HOST output (Appendix F product; the
+ * weights stay resident on the device): copies x_host ([B][K] bf16, ideally
+ * pinned) to the device, runs higgs_linear, copies y ([B][N] of y_dtype) back to
+ * y_host, all enqueued on `stream`; the caller synchronises the stream before
+ * reading y_host.  workspace is DEVICE memory of at least
+ * higgs_linear_host_workspace_bytes() bytes (it also stages x and y).
+ */
+int higgs_linear_host(const higgs_desc* desc, const void* x_host, int64_t B,
+                      const void* packed, const void* scales, const float* grid,
+                      void* y_host, int y_dtype,
+                      void* workspace, size_t workspace_bytes, void* stream);
+size_t higgs_linear_host_workspace_bytes(const higgs_desc* desc, int64_t B, int y_dtype);
+
+/* Number of kernels one higgs_linear call enqueues for this shape and batch. */
+int higgs_linear_launch_count(const higgs_desc* desc, int64_t B, int y_dtype);
 
 /* ---- validation helpers (not on the hot path) --------------------------- */
 

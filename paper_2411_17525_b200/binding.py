@@ -22,7 +22,8 @@ HIGGS_OP_QUANTIZE, HIGGS_OP_LINEAR, HIGGS_OP_MAKE_GRID = 0, 1, 2
 EXPORTS = [
     "higgs_status_string", "higgs_sign", "higgs_packed_bytes", "higgs_scales_bytes", "higgs_canonical_bytes",
     "higgs_workspace_bytes", "higgs_make_grid", "higgs_quantize", "higgs_linear", "higgs_rht",
-    "higgs_pack_codes", "higgs_unpack_codes",
+    "higgs_pack_codes", "higgs_unpack_codes", "higgs_rotate_activations", "higgs_linear_prerotated",
+    "higgs_linear_host", "higgs_linear_host_workspace_bytes", "higgs_linear_launch_count",
 ]
 
 
@@ -61,6 +62,16 @@ def _load() -> ctypes.CDLL:
     lib.higgs_quantize.argtypes = [P, vp, i32, vp, vp, vp, vp, vp, sz, vp]
     lib.higgs_linear.restype = i32
     lib.higgs_linear.argtypes = [P, vp, i64, vp, vp, vp, vp, i32, vp, sz, vp]
+    lib.higgs_rotate_activations.restype = i32
+    lib.higgs_rotate_activations.argtypes = [P, vp, i64, vp, vp]
+    lib.higgs_linear_prerotated.restype = i32
+    lib.higgs_linear_prerotated.argtypes = [P, vp, i64, vp, vp, vp, vp, i32, vp, sz, vp]
+    lib.higgs_linear_host.restype = i32
+    lib.higgs_linear_host.argtypes = [P, vp, i64, vp, vp, vp, vp, i32, vp, sz, vp]
+    lib.higgs_linear_host_workspace_bytes.restype = sz
+    lib.higgs_linear_host_workspace_bytes.argtypes = [P, i64, i32]
+    lib.higgs_linear_launch_count.restype = i32
+    lib.higgs_linear_launch_count.argtypes = [P, i64, i32]
     lib.higgs_rht.restype = i32
     lib.higgs_rht.argtypes = [P, vp, i32, i64, vp, i32, vp]
     lib.higgs_pack_codes.restype = i32
@@ -165,6 +176,53 @@ def higgs_linear(desc: higgs_desc, x: torch.Tensor, packed: torch.Tensor, scales
     _check(lib.higgs_linear(ctypes.byref(desc), _ptr(x), B, _ptr(packed), _ptr(scales), _ptr(grid), _ptr(y),
                             _dtype_code(y), _ptr(workspace), workspace.numel(), _stream()), "higgs_linear")
     return y
+
+
+def higgs_rotate_activations(desc: higgs_desc, x: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """x: cuda [B][K] bf16 -> rotated activations, cuda [B][K] fp16."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous()
+    if out is None:
+        out = torch.empty(x.shape, dtype=torch.float16, device=x.device)
+    _check(lib.higgs_rotate_activations(ctypes.byref(desc), _ptr(x), x.shape[0], _ptr(out), _stream()),
+           "higgs_rotate_activations")
+    return out
+
+
+def higgs_linear_prerotated(desc: higgs_desc, xdag: torch.Tensor, packed: torch.Tensor, scales: torch.Tensor,
+                            grid: torch.Tensor, out_dtype: torch.dtype = torch.float32,
+                            workspace: Optional[torch.Tensor] = None, y: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """xdag: cuda [B][K] fp16 from higgs_rotate_activations.  Returns y [B][N]."""
+    assert xdag.is_cuda and xdag.dtype == torch.float16 and xdag.is_contiguous()
+    B = xdag.shape[0]
+    if y is None:
+        y = torch.empty((B, desc.N), dtype=out_dtype, device=xdag.device)
+    if workspace is None:
+        workspace = _workspace(higgs_workspace_bytes(desc, HIGGS_OP_LINEAR, B), xdag.device)
+    _check(lib.higgs_linear_prerotated(ctypes.byref(desc), _ptr(xdag), B, _ptr(packed), _ptr(scales), _ptr(grid),
+                                       _ptr(y), _dtype_code(y), _ptr(workspace), workspace.numel(), _stream()),
+           "higgs_linear_prerotated")
+    return y
+
+
+def higgs_linear_host_workspace_bytes(desc: higgs_desc, B: int, y_dtype: int = HIGGS_F32) -> int:
+    return int(lib.higgs_linear_host_workspace_bytes(ctypes.byref(desc), int(B), int(y_dtype)))
+
+
+def higgs_linear_host(desc: higgs_desc, x_host: torch.Tensor, packed: torch.Tensor, scales: torch.Tensor,
+                      grid: torch.Tensor, y_host: torch.Tensor, workspace: torch.Tensor) -> torch.Tensor:
+    """x_host: CPU (pinned) [B][K] bf16; y_host: CPU (pinned) [B][N] fp32/bf16; workspace: cuda uint8.
+    Enqueues copy-in, the layer and copy-out on the current stream; synchronise before reading y_host."""
+    assert (not x_host.is_cuda) and x_host.dtype == torch.bfloat16 and x_host.is_contiguous()
+    assert (not y_host.is_cuda) and y_host.is_contiguous() and workspace.is_cuda
+    B = x_host.shape[0]
+    _check(lib.higgs_linear_host(ctypes.byref(desc), _ptr(x_host), B, _ptr(packed), _ptr(scales), _ptr(grid),
+                                 _ptr(y_host), _dtype_code(y_host), _ptr(workspace), workspace.numel(), _stream()),
+           "higgs_linear_host")
+    return y_host
+
+
+def higgs_linear_launch_count(desc: higgs_desc, B: int, y_dtype: int = HIGGS_F32) -> int:
+    return int(lib.higgs_linear_launch_count(ctypes.byref(desc), int(B), int(y_dtype)))
 
 
 def higgs_rht(desc: higgs_desc, x: torch.Tensor, normalised: bool) -> torch.Tensor:

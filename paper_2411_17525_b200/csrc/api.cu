@@ -100,32 +100,24 @@ int higgs_quantize(const higgs_desc* d, const void* W, int w_dtype, const float*
     return launch_pack(*d, canonical, packed_out, st);
 }
 
-int higgs_linear(const higgs_desc* d, const void* x, int64_t B, const void* packed, const void* scales,
-                 const float* grid, void* y, int y_dtype, void* workspace, size_t workspace_bytes, void* stream) {
+int higgs_rotate_activations(const higgs_desc* d, const void* x, int64_t B, void* xdag_out, void* stream) {
     int rc = check_desc(d);
     if (rc != HIGGS_OK) return rc;
-    if (y_dtype != HIGGS_F32 && y_dtype != HIGGS_BF16) return HIGGS_ERR_UNSUPPORTED;
     if (B < 0) return HIGGS_ERR_INVALID_ARG;
-    if (B == 0 || d->N == 0) return HIGGS_OK;
-    if (d->K == 0) return HIGGS_ERR_UNSUPPORTED;
-    if (!x || !packed || !scales || !grid || !y || !workspace) return HIGGS_ERR_INVALID_ARG;
-    if (!aligned(x, 16) || !aligned(packed, 16) || !aligned(scales, 2) || !aligned(workspace, 256) ||
-        !aligned(y, y_dtype == HIGGS_F32 ? 4 : 2))
-        return HIGGS_ERR_INVALID_ARG;
-    if (workspace_bytes < higgs_workspace_bytes(d, HIGGS_OP_LINEAR, B)) return HIGGS_ERR_WORKSPACE;
-    cudaStream_t st = as_stream(stream);
+    if (B == 0 || d->K == 0) return HIGGS_OK;
+    if (!x || !xdag_out || !aligned(x, 16) || !aligned(xdag_out, 16)) return HIGGS_ERR_INVALID_ARG;
+    return launch_rht_activations(*d, x, B, static_cast<__half*>(xdag_out), nullptr, 0, as_stream(stream));
+}
 
-    __half* xdag = static_cast<__half*>(workspace);
-    float* y32 = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up((size_t)B * d->K * 2, 256));
+// Shared tail of higgs_linear / higgs_linear_prerotated: D2-D5 on rotated activations.
+static int linear_tail(const higgs_desc* d, const __half* xdag, int64_t B, const void* packed, const void* scales,
+                       const float* grid, void* y, int y_dtype, float* y32, bool target_is_clear, cudaStream_t st) {
     const int chunks = linear_k_chunks(*d, B);
     const bool split = chunks > 1;
     float* acc_target = split ? (y_dtype == HIGGS_F32 ? static_cast<float*>(y) : y32) : nullptr;
-
-    // D1: rotate the activations once (and clear the accumulation target of a K-split product)
-    rc = launch_rht_activations(*d, x, B, xdag, acc_target, split ? (size_t)B * d->N : 0, st);
-    if (rc != HIGGS_OK) return rc;
-
-    // D2-D5: stream codes, look up, contract, reduce
+    if (split && !target_is_clear) {
+        if (cudaMemsetAsync(acc_target, 0, (size_t)B * d->N * sizeof(float), st) != cudaSuccess) return HIGGS_ERR_CUDA;
+    }
     for (int64_t b0 = 0; b0 < B; b0 += 16) {
         const int64_t bn = B - b0 < 16 ? B - b0 : 16;
         void* yo;
@@ -133,11 +125,92 @@ int higgs_linear(const higgs_desc* d, const void* x, int64_t B, const void* pack
         if (split) { yo = acc_target + b0 * d->N; mode = 2; }
         else if (y_dtype == HIGGS_F32) { yo = static_cast<float*>(y) + b0 * d->N; mode = 0; }
         else { yo = static_cast<__nv_bfloat16*>(y) + b0 * d->N; mode = 1; }
-        rc = launch_linear_mma(*d, xdag + b0 * d->K, bn, packed, scales, grid, yo, d->N, mode, st);
+        int rc = launch_linear_mma(*d, xdag + b0 * d->K, bn, packed, scales, grid, yo, d->N, mode, st);
         if (rc != HIGGS_OK) return rc;
     }
     if (split && y_dtype == HIGGS_BF16) return launch_convert_out(y32, y, y_dtype, (size_t)B * d->N, st);
     return HIGGS_OK;
+}
+
+static int linear_args(const higgs_desc* d, int64_t B, const void* x, const void* packed, const void* scales,
+                       const float* grid, void* y, int y_dtype, void* workspace, size_t workspace_bytes) {
+    int rc = check_desc(d);
+    if (rc != HIGGS_OK) return rc;
+    if (y_dtype != HIGGS_F32 && y_dtype != HIGGS_BF16) return HIGGS_ERR_UNSUPPORTED;
+    if (B < 0) return HIGGS_ERR_INVALID_ARG;
+    if (B == 0 || d->N == 0) return -1;   // nothing to do
+    if (d->K == 0) return HIGGS_ERR_UNSUPPORTED;
+    if (!x || !packed || !scales || !grid || !y || !workspace) return HIGGS_ERR_INVALID_ARG;
+    if (!aligned(x, 16) || !aligned(packed, 16) || !aligned(scales, 2) || !aligned(workspace, 256) ||
+        !aligned(y, y_dtype == HIGGS_F32 ? 4 : 2))
+        return HIGGS_ERR_INVALID_ARG;
+    if (workspace_bytes < higgs_workspace_bytes(d, HIGGS_OP_LINEAR, B)) return HIGGS_ERR_WORKSPACE;
+    return HIGGS_OK;
+}
+
+int higgs_linear(const higgs_desc* d, const void* x, int64_t B, const void* packed, const void* scales,
+                 const float* grid, void* y, int y_dtype, void* workspace, size_t workspace_bytes, void* stream) {
+    int rc = linear_args(d, B, x, packed, scales, grid, y, y_dtype, workspace, workspace_bytes);
+    if (rc != HIGGS_OK) return rc < 0 ? HIGGS_OK : rc;
+    cudaStream_t st = as_stream(stream);
+    __half* xdag = static_cast<__half*>(workspace);
+    float* y32 = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up((size_t)B * d->K * 2, 256));
+    const bool split = linear_k_chunks(*d, B) > 1;
+    float* acc_target = split ? (y_dtype == HIGGS_F32 ? static_cast<float*>(y) : y32) : nullptr;
+    // D1: rotate the activations once (and clear the accumulation target of a K-split product)
+    rc = launch_rht_activations(*d, x, B, xdag, acc_target, split ? (size_t)B * d->N : 0, st);
+    if (rc != HIGGS_OK) return rc;
+    // D2-D5: stream codes, look up, contract, reduce
+    return linear_tail(d, xdag, B, packed, scales, grid, y, y_dtype, y32, true, st);
+}
+
+int higgs_linear_prerotated(const higgs_desc* d, const void* xdag, int64_t B, const void* packed, const void* scales,
+                            const float* grid, void* y, int y_dtype, void* workspace, size_t workspace_bytes,
+                            void* stream) {
+    int rc = linear_args(d, B, xdag, packed, scales, grid, y, y_dtype, workspace, workspace_bytes);
+    if (rc != HIGGS_OK) return rc < 0 ? HIGGS_OK : rc;
+    float* y32 = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up((size_t)B * d->K * 2, 256));
+    return linear_tail(d, static_cast<const __half*>(xdag), B, packed, scales, grid, y, y_dtype, y32, false,
+                       as_stream(stream));
+}
+
+int higgs_linear_host(const higgs_desc* d, const void* x_host, int64_t B, const void* packed, const void* scales,
+                      const float* grid, void* y_host, int y_dtype, void* workspace, size_t workspace_bytes,
+                      void* stream) {
+    int rc = check_desc(d);
+    if (rc != HIGGS_OK) return rc;
+    if (y_dtype != HIGGS_F32 && y_dtype != HIGGS_BF16) return HIGGS_ERR_UNSUPPORTED;
+    if (B < 0) return HIGGS_ERR_INVALID_ARG;
+    if (B == 0 || d->N == 0) return HIGGS_OK;
+    if (!x_host || !y_host || !workspace || !aligned(workspace, 256)) return HIGGS_ERR_INVALID_ARG;
+    const size_t inner = higgs_workspace_bytes(d, HIGGS_OP_LINEAR, B);
+    const size_t xb = align_up((size_t)B * d->K * 2, 256);
+    const size_t yb = align_up((size_t)B * d->N * (y_dtype == HIGGS_F32 ? 4 : 2), 256);
+    if (workspace_bytes < inner + xb + yb) return HIGGS_ERR_WORKSPACE;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    void* x_dev = ws + inner;
+    void* y_dev = ws + inner + xb;
+    cudaStream_t st = as_stream(stream);
+    if (cudaMemcpyAsync(x_dev, x_host, (size_t)B * d->K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return HIGGS_ERR_CUDA;
+    rc = higgs_linear(d, x_dev, B, packed, scales, grid, y_dev, y_dtype, workspace, inner, stream);
+    if (rc != HIGGS_OK) return rc;
+    if (cudaMemcpyAsync(y_host, y_dev, (size_t)B * d->N * (y_dtype == HIGGS_F32 ? 4 : 2), cudaMemcpyDeviceToHost, st) !=
+        cudaSuccess)
+        return HIGGS_ERR_CUDA;
+    return HIGGS_OK;
+}
+
+size_t higgs_linear_host_workspace_bytes(const higgs_desc* d, int64_t B, int y_dtype) {
+    const size_t inner = higgs_workspace_bytes(d, HIGGS_OP_LINEAR, B);
+    if (inner == 0) return 0;
+    return inner + align_up((size_t)B * d->K * 2, 256) + align_up((size_t)B * d->N * (y_dtype == HIGGS_F32 ? 4 : 2), 256);
+}
+
+int higgs_linear_launch_count(const higgs_desc* d, int64_t B, int y_dtype) {
+    if (check_desc(d) != HIGGS_OK || B < 1 || d->N == 0) return 0;
+    const bool split = linear_k_chunks(*d, B) > 1;
+    return 1 + (int)((B + 15) / 16) + ((split && y_dtype == HIGGS_BF16) ? 1 : 0);
 }
 
 int higgs_rht(const higgs_desc* d, const void* x, int x_dtype, int64_t rows, float* out, int normalised, void* stream) {
