@@ -88,7 +88,7 @@ const char* higgs_status_string(int status);
 int higgs_sign(uint64_t rht_seed, int64_t j);
 
 /* Bytes of the packed code stream (kernel-native, opaque layout; log2(n)/p
- * bits per weight), of the scale array ([N][K/g] of scale_dtype), and of the
+ * bits per weight), of the scale array (N * K/g values of scale_dtype), and of the
  * canonical code array ([N][K/p], one byte per code).  0 if unsupported.   */
 size_t higgs_packed_bytes(const higgs_desc* desc);
 size_t higgs_scales_bytes(const higgs_desc* desc);
@@ -131,7 +131,8 @@ int higgs_make_grid(int p, int n, const float* samples, int64_t num_samples, int
  *   W              device, [N][K] row-major, w_dtype in {HIGGS_F32, HIGGS_BF16}
  *   grid           device, [n][p] fp32
  *   packed_out     device, higgs_packed_bytes() bytes, 16-byte aligned
- *   scales_out     device, [N][K/g] of desc->scale_dtype
+ *   scales_out     device, higgs_scales_bytes() bytes, 16-byte aligned: fp16 scales stored
+ *                  tile-major, element (r, i) at index ((r / 16) * (K/g) + i) * 16 + r % 16
  *   canonical_out  device, optional, [N][K/p] one byte per code (for checking)
  */
 int higgs_quantize(const higgs_desc* desc, const void* W, int w_dtype, const float* grid,
@@ -146,7 +147,7 @@ int higgs_quantize(const higgs_desc* desc, const void* W, int w_dtype, const flo
  * products are exact and accumulation is fp32; scales are applied in fp32.
  *   x        device, [B][K] row-major bf16, B >= 1
  *   packed   device, from higgs_quantize / higgs_pack_codes
- *   scales   device, [N][K/g]
+ *   scales   device, tile-major fp16 scales as written by higgs_quantize
  *   grid     device, [n][p] fp32
  *   y        device, [B][N] row-major, y_dtype in {HIGGS_F32, HIGGS_BF16}
  * When K is split over several thread blocks the partial sums meet in fp32
@@ -185,6 +186,15 @@ int higgs_linear_host(const higgs_desc* desc, const void* x_host, int64_t B,
                       void* y_host, int y_dtype,
                       void* workspace, size_t workspace_bytes, void* stream);
 size_t higgs_linear_host_workspace_bytes(const higgs_desc* desc, int64_t B, int y_dtype);
+
+/*
+ * Every device-side wait in this library is bounded.  If one runs out, the kernel
+ * gives up, and the library's device status word becomes HIGGS_ERR_TIMEOUT.
+ * This call synchronises `stream`, returns the word (HIGGS_OK if no wait ever
+ * ran out) and, if clear != 0, resets it.  Results computed by a launch that
+ * timed out are undefined.
+ */
+int higgs_device_status(void* stream, int clear);
 
 /* Number of kernels one higgs_linear call enqueues for this shape and batch. */
 int higgs_linear_launch_count(const higgs_desc* desc, int64_t B, int y_dtype);

@@ -23,7 +23,7 @@ EXPORTS = [
     "higgs_status_string", "higgs_sign", "higgs_packed_bytes", "higgs_scales_bytes", "higgs_canonical_bytes",
     "higgs_workspace_bytes", "higgs_make_grid", "higgs_quantize", "higgs_linear", "higgs_rht",
     "higgs_pack_codes", "higgs_unpack_codes", "higgs_rotate_activations", "higgs_linear_prerotated",
-    "higgs_linear_host", "higgs_linear_host_workspace_bytes", "higgs_linear_launch_count",
+    "higgs_linear_host", "higgs_linear_host_workspace_bytes", "higgs_linear_launch_count", "higgs_device_status",
 ]
 
 
@@ -72,6 +72,8 @@ def _load() -> ctypes.CDLL:
     lib.higgs_linear_host_workspace_bytes.argtypes = [P, i64, i32]
     lib.higgs_linear_launch_count.restype = i32
     lib.higgs_linear_launch_count.argtypes = [P, i64, i32]
+    lib.higgs_device_status.restype = i32
+    lib.higgs_device_status.argtypes = [vp, i32]
     lib.higgs_rht.restype = i32
     lib.higgs_rht.argtypes = [P, vp, i32, i64, vp, i32, vp]
     lib.higgs_pack_codes.restype = i32
@@ -150,11 +152,11 @@ def higgs_make_grid(p: int, n: int, samples: torch.Tensor, max_iters: int = 4000
 
 def higgs_quantize(desc: higgs_desc, W: torch.Tensor, grid: torch.Tensor, want_canonical: bool = False,
                    workspace: Optional[torch.Tensor] = None):
-    """W: cuda [N][K] fp32 or bf16; grid: cuda [n][p] fp32.  Returns (packed u8, scales fp16 [N][K/g], canonical u8 or None)."""
+    """W: cuda [N][K] fp32 or bf16; grid: cuda [n][p] fp32.  Returns (packed u8, scales fp16 tile-major [N/16][K/g][16], canonical u8 or None)."""
     assert W.is_cuda and W.is_contiguous() and grid.is_cuda and grid.dtype == torch.float32 and grid.is_contiguous()
     dev = W.device
     packed = torch.empty(max(higgs_packed_bytes(desc), 16), dtype=torch.uint8, device=dev)
-    scales = torch.empty((desc.N, max(desc.K // desc.g, 0)), dtype=torch.float16, device=dev)
+    scales = torch.empty((desc.N // 16, max(desc.K // desc.g, 0), 16), dtype=torch.float16, device=dev)
     canonical = torch.empty((desc.N, desc.K // desc.p), dtype=torch.uint8, device=dev) if want_canonical else None
     if workspace is None:
         workspace = _workspace(higgs_workspace_bytes(desc, HIGGS_OP_QUANTIZE), dev)
@@ -219,6 +221,24 @@ def higgs_linear_host(desc: higgs_desc, x_host: torch.Tensor, packed: torch.Tens
                                  _ptr(y_host), _dtype_code(y_host), _ptr(workspace), workspace.numel(), _stream()),
            "higgs_linear_host")
     return y_host
+
+
+def higgs_device_status(clear: bool = True) -> int:
+    """Synchronises the current stream and returns the library's device status word (HIGGS_OK unless a bounded
+    device-side wait ran out)."""
+    return int(lib.higgs_device_status(_stream(), int(bool(clear))))
+
+
+def scales_to_tile_major(scales: torch.Tensor) -> torch.Tensor:
+    """[N][K/g] fp16 -> the tile-major storage order higgs_linear reads (pure data movement)."""
+    N, Gn = scales.shape
+    return scales.reshape(N // 16, 16, Gn).permute(0, 2, 1).contiguous()
+
+
+def scales_from_tile_major(scales: torch.Tensor, N: int) -> torch.Tensor:
+    """Inverse of scales_to_tile_major: returns [N][K/g]."""
+    Gn = scales.numel() // N
+    return scales.reshape(N // 16, Gn, 16).permute(0, 2, 1).reshape(N, Gn).contiguous()
 
 
 def higgs_linear_launch_count(desc: higgs_desc, B: int, y_dtype: int = HIGGS_F32) -> int:

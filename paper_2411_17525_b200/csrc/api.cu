@@ -85,7 +85,7 @@ int higgs_quantize(const higgs_desc* d, const void* W, int w_dtype, const float*
     if (w_dtype != HIGGS_F32 && w_dtype != HIGGS_BF16) return HIGGS_ERR_UNSUPPORTED;
     if (d->N == 0 || d->K == 0) return HIGGS_OK;
     if (!W || !grid || !packed_out || !scales_out) return HIGGS_ERR_INVALID_ARG;
-    if (!aligned(W, 16) || !aligned(packed_out, 16) || !aligned(scales_out, 2)) return HIGGS_ERR_INVALID_ARG;
+    if (!aligned(W, 16) || !aligned(packed_out, 16) || !aligned(scales_out, 16)) return HIGGS_ERR_INVALID_ARG;
     uint8_t* canonical = canonical_out;
     if (!canonical) {
         if (!workspace || !aligned(workspace, 256)) return HIGGS_ERR_INVALID_ARG;
@@ -141,8 +141,7 @@ static int linear_args(const higgs_desc* d, int64_t B, const void* x, const void
     if (B == 0 || d->N == 0) return -1;   // nothing to do
     if (d->K == 0) return HIGGS_ERR_UNSUPPORTED;
     if (!x || !packed || !scales || !grid || !y || !workspace) return HIGGS_ERR_INVALID_ARG;
-    if (!aligned(x, 16) || !aligned(packed, 16) || !aligned(scales, 2) || !aligned(workspace, 256) ||
-        !aligned(y, y_dtype == HIGGS_F32 ? 4 : 2))
+    if (!aligned(x, 16) || !aligned(packed, 16) || !aligned(scales, 16) || !aligned(workspace, 256) || !aligned(y, 16))
         return HIGGS_ERR_INVALID_ARG;
     if (workspace_bytes < higgs_workspace_bytes(d, HIGGS_OP_LINEAR, B)) return HIGGS_ERR_WORKSPACE;
     return HIGGS_OK;
@@ -212,6 +211,8 @@ int higgs_linear_launch_count(const higgs_desc* d, int64_t B, int y_dtype) {
     const bool split = linear_k_chunks(*d, B) > 1;
     return 1 + (int)((B + 15) / 16) + ((split && y_dtype == HIGGS_BF16) ? 1 : 0);
 }
+
+int higgs_device_status(void* stream, int clear) { return read_device_status(as_stream(stream), clear); }
 
 int higgs_rht(const higgs_desc* d, const void* x, int x_dtype, int64_t rows, float* out, int normalised, void* stream) {
     int rc = check_desc(d);

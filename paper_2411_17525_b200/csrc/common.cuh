@@ -11,7 +11,7 @@
 namespace higgs {
 
 constexpr int kGroup = 1024;     // the only supported group size g
-constexpr int kRowTile = 16;     // rows of W per mma tile (m16n8k16)
+constexpr int kRowTile = 16;     // rows of W per mma tile (m16n8k16) and per scale tile
 constexpr int kBlockK = 64;      // k-extent of one 512-byte packed block
 
 // Top bit of output j of the splitmix64 stream seeded with xi: 1 -> sign -1.
@@ -96,5 +96,6 @@ size_t make_grid_workspace(int p, int n, int64_t m);
 int launch_make_grid(int p, int n, const float* samples, int64_t m, int max_iters, float* grid_out, float* mse_out,
                      int32_t* iters_out, void* ws, cudaStream_t st);
 int linear_k_chunks(const higgs_desc& d, int64_t B);
+int read_device_status(cudaStream_t st, int clear);
 
 }  // namespace higgs

@@ -70,7 +70,8 @@ __global__ void __launch_bounds__(128) encode_kernel(const T* __restrict__ W, co
     }
     fwht1024_warp(v, lane);
 
-    if (lane == 0) scales[row * groups + gi] = __float2half_rn(s * 0.03125f);
+    // scales are stored tile-major: [row / 16][group][row % 16]
+    if (lane == 0) scales[((row >> 4) * groups + gi) * 16 + (row & 15)] = __float2half_rn(s * 0.03125f);
 
     if (P == 2) {
         float best[16];

@@ -66,7 +66,8 @@ def test_quantize_codes_and_scales(p, n, N, K, bf16):
     assert gpu_codes.shape == q.codes.shape and gpu_codes.max() < n
     U.compare_codes(gpu_codes, q)
     # scales: fp32 norm then fp16 rounding; at most one fp16 ulp from the oracle's, almost all identical
-    s_gpu = scales.cpu().numpy()
+    s_gpu = hb.scales_from_tile_major(scales, N).cpu().numpy()
+    assert s_gpu.shape == sc16.shape
     ulp = np.abs(s_gpu.view(np.int16).astype(np.int64) - sc16.view(np.int16).astype(np.int64))
     assert ulp.max() <= 1 and (ulp == 0).mean() > 0.98
     # the packed stream holds exactly the canonical codes
@@ -92,6 +93,7 @@ def test_quantize_invariants_on_gpu():
     Wz[3, :1024] = 0.0
     dz, _, _, _, scz, cz = run_quantize(Wz, p, n, xi, False)
     origin = int(np.argmin((g64 ** 2).sum(1)))
+    scz = hb.scales_from_tile_major(scz, N)
     assert float(scz[3, 0]) == 0.0 and bool((cz[3, :512] == origin).all())
     assert torch.equal(cz[4:], canon[4:]) and bool(torch.isfinite(scz.float()).all())
 
@@ -105,9 +107,9 @@ def run_linear_case(p, n, N, K, B, xi, wseed, xseed, out_dtype=torch.float32, lo
     d = hb.make_desc(p, n, N, K, xi)
     canon = torch.from_numpy(q.codes.astype(np.uint8)).to(U.dev())
     packed = hb.higgs_pack_codes(d, canon)                       # identical codes on both sides
-    scales = torch.from_numpy(sc16).to(U.dev())
+    scales = hb.scales_to_tile_major(torch.from_numpy(sc16).to(U.dev()))   # storage order only
     y = hb.higgs_linear(d, U.bf16_tensor(x), packed, scales, gt, out_dtype=out_dtype)
-    torch.cuda.synchronize()
+    assert hb.higgs_device_status() == hb.HIGGS_OK
     y_ref = oracle.linear_dense(x.astype(np.float64), q.codes, sc16.astype(np.float64), G, g64, xi)
     return y, y_ref
 
@@ -173,11 +175,11 @@ def test_empty_inputs():
     _, gt = U.grid32(2, 256)
     W = torch.empty((0, 1024), dtype=torch.float32, device=U.dev())
     packed, scales, canon = hb.higgs_quantize(d, W, gt, want_canonical=True)
-    assert scales.shape == (0, 1) and canon.shape == (0, 512)
+    assert scales.numel() == 0 and canon.shape == (0, 512)
     d = hb.make_desc(2, 256, 16, 1024, 1)
     x = torch.empty((0, 1024), dtype=torch.bfloat16, device=U.dev())
     y = hb.higgs_linear(d, x, torch.zeros(16 * 512, dtype=torch.uint8, device=U.dev()),
-                        torch.zeros((16, 1), dtype=torch.float16, device=U.dev()), gt)
+                        torch.zeros((1, 1, 16), dtype=torch.float16, device=U.dev()), gt)
     assert y.shape == (0, 16)
 
 
