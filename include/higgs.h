@@ -56,7 +56,8 @@ typedef enum higgs_status {
     HIGGS_ERR_UNSUPPORTED = 2,   /* (p, n, g, dtype, shape) combination has no kernel          */
     HIGGS_ERR_WORKSPACE = 3,     /* workspace smaller than higgs_workspace_bytes() asks        */
     HIGGS_ERR_CUDA = 4,          /* a CUDA runtime call failed (no device, launch error)        */
-    HIGGS_ERR_TIMEOUT = 5        /* a bounded device-side wait ran out (read from a status word) */
+    HIGGS_ERR_TIMEOUT = 5,       /* a bounded device-side wait ran out (read from a status word) */
+    HIGGS_ERR_STATIC_SCRATCH = 6 /* request does not fit the library's built-in scratch array       */
 } higgs_status;
 
 typedef enum higgs_dtype { HIGGS_F32 = 0, HIGGS_F16 = 1, HIGGS_BF16 = 2 } higgs_dtype;
@@ -186,6 +187,34 @@ int higgs_linear_host(const higgs_desc* desc, const void* x_host, int64_t B,
                       void* y_host, int y_dtype,
                       void* workspace, size_t workspace_bytes, void* stream);
 size_t higgs_linear_host_workspace_bytes(const higgs_desc* desc, int64_t B, int y_dtype);
+
+/*
+ * higgs_linear without a workspace argument, for callers that cannot allocate
+ * device memory (code running where cudaMalloc is off limits, plugins that are
+ * only handed their input and output buffers, processes whose memory pool
+ * belongs to another component).  The paper has no counterpart: this is purely
+ * an interface convenience.  The result is the same as higgs_linear's.
+ *
+ * The scratch lives in one fixed array of higgs_linear_static_capacity() bytes
+ * (4 MiB) inside the library image; every GPU that loads the library holds it
+ * until the process exits.  A call whose higgs_workspace_bytes(desc,
+ * HIGGS_OP_LINEAR, B) exceeds that capacity returns HIGGS_ERR_STATIC_SCRATCH and
+ * enqueues nothing; 4 MiB covers every Llama-shaped layer up to 28672 x 8192
+ * at B <= 16.
+ *
+ * The call allocates nothing and calls no allocating routine.  Its first call on
+ * a device looks the array's address up (once per device, with that device
+ * current); make that first call before starting any stream capture.  All calls
+ * on a device share the one array: it keeps whatever the previous call left, the
+ * kernels overwrite or clear everything they read, and two calls that overlap on
+ * the GPU (different streams, or the same shape replayed concurrently) race on
+ * it - serialise them.  x, packed, scales, grid and y are caller-owned device
+ * buffers exactly as for higgs_linear.
+ */
+int higgs_linear_static(const higgs_desc* desc, const void* x, int64_t B,
+                        const void* packed, const void* scales, const float* grid,
+                        void* y, int y_dtype, void* stream);
+size_t higgs_linear_static_capacity(void);
 
 /*
  * Every device-side wait in this library is bounded.  If one runs out, the kernel

@@ -15,7 +15,7 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libhiggs_b200.so")
 
-HIGGS_OK, HIGGS_ERR_INVALID_ARG, HIGGS_ERR_UNSUPPORTED, HIGGS_ERR_WORKSPACE, HIGGS_ERR_CUDA, HIGGS_ERR_TIMEOUT = range(6)
+HIGGS_OK, HIGGS_ERR_INVALID_ARG, HIGGS_ERR_UNSUPPORTED, HIGGS_ERR_WORKSPACE, HIGGS_ERR_CUDA, HIGGS_ERR_TIMEOUT, HIGGS_ERR_STATIC_SCRATCH = range(7)
 HIGGS_F32, HIGGS_F16, HIGGS_BF16 = 0, 1, 2
 HIGGS_OP_QUANTIZE, HIGGS_OP_LINEAR, HIGGS_OP_MAKE_GRID = 0, 1, 2
 
@@ -24,6 +24,7 @@ EXPORTS = [
     "higgs_workspace_bytes", "higgs_make_grid", "higgs_quantize", "higgs_linear", "higgs_rht",
     "higgs_pack_codes", "higgs_unpack_codes", "higgs_rotate_activations", "higgs_linear_prerotated",
     "higgs_linear_host", "higgs_linear_host_workspace_bytes", "higgs_linear_launch_count", "higgs_device_status",
+    "higgs_linear_static", "higgs_linear_static_capacity",
 ]
 
 
@@ -72,6 +73,10 @@ def _load() -> ctypes.CDLL:
     lib.higgs_linear_host_workspace_bytes.argtypes = [P, i64, i32]
     lib.higgs_linear_launch_count.restype = i32
     lib.higgs_linear_launch_count.argtypes = [P, i64, i32]
+    lib.higgs_linear_static.restype = i32
+    lib.higgs_linear_static.argtypes = [P, vp, i64, vp, vp, vp, vp, i32, vp]
+    lib.higgs_linear_static_capacity.restype = sz
+    lib.higgs_linear_static_capacity.argtypes = []
     lib.higgs_device_status.restype = i32
     lib.higgs_device_status.argtypes = [vp, i32]
     lib.higgs_rht.restype = i32
@@ -221,6 +226,21 @@ def higgs_linear_host(desc: higgs_desc, x_host: torch.Tensor, packed: torch.Tens
                                  _ptr(y_host), _dtype_code(y_host), _ptr(workspace), workspace.numel(), _stream()),
            "higgs_linear_host")
     return y_host
+
+
+def higgs_linear_static_capacity() -> int:
+    return int(lib.higgs_linear_static_capacity())
+
+
+def higgs_linear_static(desc: higgs_desc, x: torch.Tensor, packed: torch.Tensor, scales: torch.Tensor,
+                        grid: torch.Tensor, y: torch.Tensor) -> torch.Tensor:
+    """higgs_linear for callers that cannot allocate: no workspace argument, the scratch is the library's own
+    fixed array.  x: cuda [B][K] bf16; y: caller-owned cuda [B][N] fp32 or bf16, written in place.  Raises
+    HiggsError(HIGGS_ERR_STATIC_SCRATCH) when the shape does not fit the array."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and y.is_cuda and y.is_contiguous()
+    _check(lib.higgs_linear_static(ctypes.byref(desc), _ptr(x), x.shape[0], _ptr(packed), _ptr(scales), _ptr(grid),
+                                   _ptr(y), _dtype_code(y), _stream()), "higgs_linear_static")
+    return y
 
 
 def higgs_device_status(clear: bool = True) -> int:

@@ -30,6 +30,7 @@ const char* higgs_status_string(int status) {
         case HIGGS_ERR_WORKSPACE: return "workspace too small";
         case HIGGS_ERR_CUDA: return "CUDA runtime error";
         case HIGGS_ERR_TIMEOUT: return "bounded device-side wait ran out";
+        case HIGGS_ERR_STATIC_SCRATCH: return "request exceeds the library's built-in scratch array";
         default: return "unknown status";
     }
 }
