@@ -47,6 +47,30 @@ inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? HIGGS_OK : HIG
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// ---- programmatic dependent launch -----------------------------------------------------------
+// Every kernel of the decode path is launched with the programmatic-stream-serialization
+// attribute: it may start while the previous kernel of the stream is still running, does the work
+// that depends on nothing (table build, weight prefetch) and then calls pdl_wait() before it
+// touches anything the previous kernel may read or write.  pdl_trigger() lets the next kernel
+// start as early as possible.
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---- in-register / warp-shuffle fast Walsh-Hadamard transform over 1024 ----
 // A warp owns one group.  Lane l holds 32 values v[r], r = c*8 + e, standing
 // for element index  idx = c*256 + l*8 + e  (c in 0..3, e in 0..7), so that a

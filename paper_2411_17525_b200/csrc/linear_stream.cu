@@ -29,6 +29,15 @@ namespace higgs {
 
 __device__ int g_device_status = 0;
 
+// Optional timeline tracing of one block (build with -DHIGGS_TRACE): SM cycle stamps per warp and event.
+#ifdef HIGGS_TRACE
+__device__ long long g_trace[17][64];
+__device__ __forceinline__ long long trace_now() { return clock64(); }   // SM cycles (cheap); one block only, so one clock domain
+#define TRACE(warp_, slot_) do { if (blockIdx.x == 7 && (threadIdx.x & 31) == 0 && (slot_) < 64) g_trace[warp_][slot_] = trace_now(); } while (0)
+#else
+#define TRACE(warp_, slot_) do { } while (0)
+#endif
+
 namespace {
 
 struct StreamParams {
@@ -38,7 +47,7 @@ struct StreamParams {
     const float* grid;     // [n][p]
     void* y;               // [B][ldy]
     int64_t N, K, ldy;
-    int64_t items;         // chunks * (N/16), numbered chunk-major
+    int chunks;            // K / ck; the grid is chunks x parts blocks
     int B, n, p;
     int ck;                // inputs per item
     int y_mode;            // 0: store fp32, 1: store bf16, 2: atomicAdd fp32
@@ -67,12 +76,6 @@ __device__ __forceinline__ uint2 lds64(uint32_t addr) {
     uint2 v;
     asm volatile("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
     return v;
-}
-__device__ __forceinline__ void sts128(uint32_t addr, float a, float b, float c, float d) {
-    asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
-__device__ __forceinline__ void red_shared_add(uint32_t addr, float v) {
-    asm volatile("red.shared.add.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
 }
 __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                          uint32_t b1) {
@@ -188,7 +191,7 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     using Codes = TaskCodes<KS, SIX>;
 
     // ---- shared memory map (all offsets derived from the runtime base address) ----
-    //   [base, base+4 KB)    ring mbarriers (0..1023), table seed (1024..2047), item mbarriers and
+    //   [base, base+4 KB)    ring mbarriers (0..1023), item mbarriers and
     //                        recycle counters of the partial-tile slots (2048..2559), abort flag (2560)
     //   [base+4 KB, lut)     ring slots, region A
     //   [lut, lut+64 KB)     table rows of 256 B: bytes 0..127 = the entry replicated per lane,
@@ -198,7 +201,6 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     const uint32_t dyn_end = base + kMaxDynSmem;
     const uint32_t lut = (base + kSmallBytes + 0xffffu) & ~0xffffu;   // 64 KB aligned: byte 1 of an address is free for the code
     const uint32_t bars = base;
-    const uint32_t seed = base + 1024u;
     const uint32_t item_bars = base + 2048u;                                        // [kMaxAccSlots] mbarriers, NS arrivals each
     volatile int* recycled = reinterpret_cast<volatile int*>(smem_raw + 2048 + 8 * kMaxAccSlots);   // [kMaxAccSlots] generations
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + 2560);
@@ -221,11 +223,11 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     // ---- this block's items and this warp's share of them ----
     // (all per-task bookkeeping below is incremental 32-bit arithmetic)
     const int tiles = (int)(prm.N / kRowTile);
-    const int64_t it_begin = prm.items * blockIdx.x / gridDim.x;
-    const int64_t it_end = prm.items * (blockIdx.x + 1) / gridDim.x;
-    const int n_items = (int)(it_end - it_begin);
+    const int parts = (int)gridDim.x / prm.chunks;
+    const int chunk_begin = (int)blockIdx.x / parts, part = (int)blockIdx.x % parts;   // this block's K-chunk
+    const int rt_begin = (int)((int64_t)tiles * part / parts);
+    const int n_items = (int)((int64_t)tiles * (part + 1) / parts) - rt_begin;          // its row tiles
     const int groups = (int)(prm.K / kGroup);
-    const int chunk_begin = (int)(it_begin / tiles), rt_begin = (int)(it_begin - (int64_t)chunk_begin * tiles);
     const int NS = prm.ck / KS;                // slices per item = warps per item
     const int PG = kWarps / NS;                // warps sharing a slice take every PG-th item
     const bool flusher = warp == kWarps;
@@ -271,6 +273,41 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
         for (; issued < n_tasks && issued < D; ++issued) issue(issued);
     }
 
+    TRACE(warp, 0);
+    pdl_trigger();
+    // Table: entry(idx) replicated once per lane (bank = lane): conflict-free gathers.  Warp w fills rows
+    // w, w+17, ...; all lanes of a warp read the same grid entry (one broadcast transaction), and the 16 loads of
+    // a warp are independent, so the whole build costs one global round trip.  (The grid is a constant of the layer.)
+    {
+        constexpr int kRowsPerWarp = (256 + kWarps) / (kWarps + 1);     // 16 rows for 17 warps (last one partly idle)
+        uint32_t ent[kRowsPerWarp];
+#pragma unroll
+        for (int r = 0; r < kRowsPerWarp; ++r) {
+            const int idx = warp + r * (kWarps + 1);
+            float lo = 0.f, hi = 0.f;
+            if (idx < 256) {
+                if (prm.p == 2) {
+                    const float2 gp = __ldg(reinterpret_cast<const float2*>(prm.grid) + (idx & (prm.n - 1)));
+                    lo = gp.x; hi = gp.y;
+                } else {
+                    lo = __ldg(prm.grid + (idx & 15));
+                    hi = __ldg(prm.grid + (idx >> 4));
+                }
+            }
+            __half2 h = __floats2half2_rn(lo, hi);
+            ent[r] = *reinterpret_cast<uint32_t*>(&h);
+        }
+#pragma unroll
+        for (int r = 0; r < kRowsPerWarp; ++r) {
+            const int idx = warp + r * (kWarps + 1);
+            if (idx < 256) *reinterpret_cast<uint32_t*>(smem_raw + (lut - base) + idx * 256 + lane * 4) = ent[r];
+        }
+    }
+    // Everything above depends only on the weights.  The activations (and y, which the previous kernel in the
+    // stream may still be reading or clearing) are touched only after the previous kernel has completed.
+    pdl_wait();
+    TRACE(warp, 1);
+
     // B fragments of this warp's K-slice for the first chunk (global loads, overlapped with the table build)
     uint32_t bfrag[KS / 16][NB][2];
     int cur_chunk = -1;
@@ -299,29 +336,8 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
         load_bfrag(cur_chunk);
     }
 
-    // table seed: one fp16 pair per index, loaded coalesced
-    if (tid < 256) {
-        float lo, hi;
-        if (prm.p == 2) {
-            const int c = tid & (prm.n - 1);
-            const float2 gp = __ldg(reinterpret_cast<const float2*>(prm.grid) + c);
-            lo = gp.x; hi = gp.y;
-        } else {
-            lo = __ldg(prm.grid + (tid & 15));
-            hi = __ldg(prm.grid + (tid >> 4));
-        }
-        __half2 h = __floats2half2_rn(lo, hi);
-        *reinterpret_cast<uint32_t*>(smem_raw + (seed - base) + tid * 4) = *reinterpret_cast<uint32_t*>(&h);
-    }
-    __syncthreads();
-    // table: entry(idx) replicated once per lane (bank = lane): conflict-free gathers
-    for (int i = tid; i < 256 * 32; i += blockDim.x) {
-        const int idx = i >> 5, l = i & 31;
-        const uint32_t e = *reinterpret_cast<const uint32_t*>(smem_raw + (seed - base) + idx * 4);
-        *reinterpret_cast<uint32_t*>(smem_raw + (lut - base) + idx * 256 + l * 4) = e;
-    }
-    __syncthreads();
-
+    __syncthreads();     // table and barriers visible to every warp
+    TRACE(warp, 2);
     // ---- flusher warp: one item after the other, in item order ----
     if (flusher) {
         int f_chunk = chunk_begin, f_rt = rt_begin;
@@ -329,25 +345,42 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
         for (int j = 0; j < n_items; ++j) {
             const int q = j & (acc_slots - 1), gen = j >> acc_shift;
             if (!mbar_wait_relaxed(item_bars + 8u * q, (uint32_t)(gen & 1), abort_flag)) return;
+            TRACE(16, 4 + 2 * j);
+            float4 sums[NB];
 #pragma unroll
             for (int qq = 0; qq < NB; ++qq) {
                 const int e = (qq * 32 + lane) * 4;      // 4 consecutive rows of one column
-                const int col = e >> 4, row = e & 15;
-                if (col < prm.B) {
-                    float4 v[16];
+                sums[qq] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if ((e >> 4) < prm.B) {
+                    // unconditional loads (clamped slice index), issued back to back; unused ones are dropped below
+                    uint4 raw[16];
+#pragma unroll
+                    for (int ns = 0; ns < 16; ++ns)
+                        raw[ns] = lds128(part_addr((q * NS + (ns < NS ? ns : 0)) * prm.B * 16 + e));
+                    float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                     for (int ns = 0; ns < 16; ++ns) {
-                        if (ns < NS) {
-                            const uint4 raw = lds128(part_addr((q * NS + ns) * prm.B * 16 + e));
-                            v[ns] = make_float4(__uint_as_float(raw.x), __uint_as_float(raw.y), __uint_as_float(raw.z),
-                                                __uint_as_float(raw.w));
-                        } else {
-                            v[ns] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        }
+                        const float m = ns < NS ? 1.f : 0.f;
+                        sum.x = fmaf(m, __uint_as_float(raw[ns].x), sum.x);
+                        sum.y = fmaf(m, __uint_as_float(raw[ns].y), sum.y);
+                        sum.z = fmaf(m, __uint_as_float(raw[ns].z), sum.z);
+                        sum.w = fmaf(m, __uint_as_float(raw[ns].w), sum.w);
                     }
-                    float4 sum = v[0];
+                    sums[qq] = sum;
+                }
+            }
+            // The partial tiles are in registers (the sums above consumed every load): hand the slot back first,
+            // then write y.  No fence follows the global write, so the warp never waits for its round trip.
+            if (sums[0].x != 1.2345e-30f) TRACE(16, 30 + 3 * j);
+            __syncwarp();
+            if (lane == 0) recycled[q] = gen + 1;
+            TRACE(16, 31 + 3 * j);
 #pragma unroll
-                    for (int ns = 1; ns < 16; ++ns) { sum.x += v[ns].x; sum.y += v[ns].y; sum.z += v[ns].z; sum.w += v[ns].w; }
+            for (int qq = 0; qq < NB; ++qq) {
+                const int e = (qq * 32 + lane) * 4;
+                const int col = e >> 4, row = e & 15;
+                if (col < prm.B) {
+                    const float4 sum = sums[qq];
                     const int64_t o = (int64_t)col * prm.ldy + (int64_t)f_rt * 16 + row;
                     if (prm.y_mode == 0) {
                         *reinterpret_cast<float4*>(static_cast<float*>(prm.y) + o) = sum;
@@ -362,11 +395,7 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
                     }
                 }
             }
-            __syncwarp();
-            if (lane == 0) {
-                __threadfence_block();
-                recycled[q] = gen + 1;               // the slot's partial tiles have been read: next generation may park
-            }
+            TRACE(16, 5 + 2 * j);
             if (++f_rt == tiles) { f_rt = 0; ++f_chunk; }
         }
         return;
@@ -379,11 +408,9 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     bool ok = true;
     int done = 0;                                // tasks whose slot has been consumed
     for (int i = 0; i < n_tasks; ++i) {
-        if (c_chunk != cur_chunk) {              // this block's range crossed into the next K-chunk
-            cur_chunk = c_chunk;
-            load_bfrag(c_chunk);
-        }
+        TRACE(warp, 4 + 3 * i);
         if (!mbar_wait(full_bar(d), ph, abort_flag)) { ok = false; break; }
+        TRACE(warp, 5 + 3 * i);
         const uint32_t slot = slot_addr(d);
         Codes codes;
         codes.load(slot, lane);
@@ -449,6 +476,7 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
             }
         }
         __syncwarp();
+        TRACE(warp, 6 + 3 * i);
         if (lane == 0) {                         // release: the partial tile is visible before the arrival counts
             asm volatile("{ .reg .b64 st; mbarrier.arrive.shared::cta.b64 st, [%0]; }" ::"r"(item_bars + 8u * q) : "memory");
         }
@@ -467,6 +495,8 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
 
 __global__ void convert_out_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, size_t count) {
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_trigger();
+    pdl_wait();
     if (i < count) dst[i] = __float2bfloat16_rn(src[i]);
 }
 
@@ -483,11 +513,14 @@ int sm_count() {
 }
 
 struct Plan {
-    int nb, ks, ck, chunks, blocks;
+    int nb, ks, ck, chunks, parts, blocks;
     int64_t items;
 };
 
-// Picks the item width CK (inputs per item) so that the items divide evenly over the SMs.
+// Picks the item width CK (inputs per item).  A block never leaves its K-chunk (its B fragments are loaded
+// once), so the grid is chunks x parts with parts = floor(SMs / chunks).  The score is the fraction of the
+// busiest block's time that is useful; splitting K is penalised because the partial results then meet in global
+// atomics and the output must be cleared first.
 Plan make_plan(const higgs_desc& d, int64_t B) {
     Plan best{};
     const int nb = B <= 8 ? 1 : 2;
@@ -500,17 +533,17 @@ Plan make_plan(const higgs_desc& d, int64_t B) {
         if (d.K % ck) continue;
         if (ck / ks > kWarps) continue;
         if (force && atoi(force) != ck) continue;
-        const int64_t items = tiles * (d.K / ck);
-        const int64_t blocks = items < sms ? items : sms;
-        const int64_t per = (items + blocks - 1) / blocks;
-        // fraction of the busiest block's time that is useful, with a mild preference for wide items
-        // (fewer K-splits to merge through global atomics)
-        const double eff = (double)items / (double)(per * blocks);
-        const double score = eff * (ck == 4096 ? 1.0 : ck == 2048 ? 0.97 : 0.94);
+        const int chunks = (int)(d.K / ck);
+        int64_t parts = sms / chunks;
+        if (parts < 1) parts = 1;
+        if (parts > tiles) parts = tiles;
+        const int64_t per = (tiles + parts - 1) / parts;          // row tiles of the busiest block
+        const double eff = (double)tiles * chunks / (double)(per * sms);
+        const double score = eff * (chunks == 1 ? 1.0 : 0.45);
         if (score > best_score) {
             best_score = score;
-            best.nb = nb; best.ks = ks; best.ck = ck; best.chunks = (int)(d.K / ck);
-            best.blocks = (int)blocks; best.items = items;
+            best.nb = nb; best.ks = ks; best.ck = ck; best.chunks = chunks;
+            best.parts = (int)parts; best.blocks = (int)(parts * chunks); best.items = tiles * chunks;
         }
     }
     return best;
@@ -527,8 +560,8 @@ int launch_one(const StreamParams& prm, int blocks, cudaStream_t st) {
         if (e != cudaSuccess) return HIGGS_ERR_CUDA;
         configured[dev] = true;
     }
-    linear_stream_kernel<NB, KS, SIX><<<(unsigned)blocks, (kWarps + 1) * 32, kMaxDynSmem, st>>>(prm);
-    return cuda_status(cudaGetLastError());
+    return cuda_status(launch_pdl(linear_stream_kernel<NB, KS, SIX>, dim3((unsigned)blocks), dim3((kWarps + 1) * 32),
+                                  kMaxDynSmem, st, prm));
 }
 
 }  // namespace
@@ -548,7 +581,7 @@ int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const 
     prm.grid = grid;
     prm.y = y;
     prm.N = d.N; prm.K = d.K; prm.ldy = ldy;
-    prm.items = pl.items;
+    prm.chunks = pl.chunks;
     prm.B = (int)B;
     prm.n = d.n; prm.p = d.p;
     prm.ck = pl.ck;
@@ -563,9 +596,13 @@ int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const 
 int launch_convert_out(const float* y32, void* y, int y_dtype, size_t count, cudaStream_t st) {
     if (y_dtype != HIGGS_BF16) return HIGGS_ERR_UNSUPPORTED;
     if (count == 0) return HIGGS_OK;
-    convert_out_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(y32, static_cast<__nv_bfloat16*>(y), count);
-    return cuda_status(cudaGetLastError());
+    return cuda_status(launch_pdl(convert_out_kernel, dim3((unsigned)((count + 255) / 256)), dim3(256), 0, st, y32,
+                                  static_cast<__nv_bfloat16*>(y), count));
 }
+
+#ifdef HIGGS_TRACE
+extern "C" int higgs_trace_read(long long* out) { return (int)cudaMemcpyFromSymbol(out, g_trace, sizeof(long long) * 17 * 64); }
+#endif
 
 int read_device_status(cudaStream_t st, int clear) {
     int v = 0;

@@ -57,6 +57,8 @@ __global__ void __launch_bounds__(256) rht_activations_kernel(const T* __restric
     const int64_t groups = K / kGroup;
     const size_t gtid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     const size_t gthreads = (size_t)gridDim.x * blockDim.x;
+    pdl_trigger();     // the product kernel may start its table build and weight prefetch now
+    pdl_wait();        // x may be the previous kernel's output; the buffers written below may still be read by it
     for (size_t i = gtid; i < zero_floats; i += gthreads) zero_ptr[i] = 0.0f;
     if (warp >= B * groups) return;
     const int64_t b = warp / groups, gi = warp % groups;
@@ -110,9 +112,8 @@ int launch_rht_activations(const higgs_desc& d, const void* x, int64_t B, __half
         if (zb > 1184) zb = 1184;
         if (zb > blocks) blocks = zb;
     }
-    rht_activations_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, st>>>(
-        static_cast<const __nv_bfloat16*>(x), xdag, B, d.K, d.rht_seed, zero_ptr, zero_floats);
-    return cuda_status(cudaGetLastError());
+    return cuda_status(launch_pdl(rht_activations_kernel<__nv_bfloat16>, dim3((unsigned)blocks), dim3(256), 0, st,
+                                  static_cast<const __nv_bfloat16*>(x), xdag, B, d.K, d.rht_seed, zero_ptr, zero_floats));
 }
 
 int launch_rht_debug(const higgs_desc& d, const void* x, int x_dtype, int64_t rows, float* out, int normalised,
