@@ -2,7 +2,8 @@
 """Benchmark of the HIGGS quantized linear layer on B200.
 
 One "step" = one decode pass (Appendix F: rotate activations, stream codes, table lookup, contraction, reduce)
-over every layer of a Llama-shaped layer set for one batch of synthetic activations.  The headline value is the
+over the seven linear layers of one Llama-shaped transformer block for one batch of synthetic activations, wired as
+in the block: q, k, v read one input (rotated once), o its own, gate and up one (rotated once), down its own.  The headline value is the
 effective weight bandwidth (packed codes + scales bytes of the layer set / time per step).  The encoder
 (Algorithm 1) and the grid fit (Algorithm 2) run once during set-up, on the GPU, and are reported separately.
 
@@ -228,12 +229,31 @@ def run_ours(args):
         ws.append(torch.empty(hb.higgs_linear_host_workspace_bytes(d, B), dtype=torch.uint8, device=dev))
         ys.append(torch.empty((B, N), dtype=torch.float32, device=dev))
     ys_host = [torch.empty((B, N), dtype=torch.float32).pin_memory() for _, N, _ in layers]
-    launches_per_step = sum(hb.higgs_linear_launch_count(d, B) for d in descs)
+
+    # layers that read the same block input share one rotation (the transform is isolated from the product, Sec. 4.3);
+    # a layer whose K is split across thread blocks goes through higgs_linear, whose rotation kernel also clears y
+    names = [nm for nm, _, _ in layers]
+    share = {"q": "attn", "k": "attn", "v": "attn", "gate": "mlp", "up": "mlp"}
+    groups_of = {}
+    for li, nm in enumerate(names):
+        split = hb.higgs_linear_k_splits(descs[li], B) > 1
+        key = share.get(nm) if not split else None
+        groups_of.setdefault(key if key else f"own{li}", []).append(li)
+    xdags = {k: torch.empty((B, descs[v[0]].K), dtype=torch.float16, device=dev) for k, v in groups_of.items() if len(v) > 1}
+    launches_per_step = 0
+    for k, v in groups_of.items():
+        launches_per_step += (1 + len(v) * ((B + 15) // 16)) if len(v) > 1 else hb.higgs_linear_launch_count(descs[v[0]], B)
 
     def step(i):
         c = i % copies
-        for li, d in enumerate(descs):
-            hb.higgs_linear(d, xs[li], packed[li][c], scales[li][c], grid, workspace=ws[li], y=ys[li])
+        for key, lis in groups_of.items():
+            if len(lis) > 1:
+                hb.higgs_rotate_activations(descs[lis[0]], xs[lis[0]], out=xdags[key])
+                for li in lis:
+                    hb.higgs_linear_prerotated(descs[li], xdags[key], packed[li][c], scales[li][c], grid, workspace=ws[li], y=ys[li])
+            else:
+                li = lis[0]
+                hb.higgs_linear(descs[li], xs[li], packed[li][c], scales[li][c], grid, workspace=ws[li], y=ys[li])
 
     def step_host(i):
         c = i % copies
@@ -402,7 +422,8 @@ def run_ours(args):
             "config": {"workload": f"{args.workload} layer set ({len(layers)} matrices), grid p={p} n={n}, g=1024, batch {B}",
                        "global_batch": B * world, "parallelism": f"replicas x{world}",
                        "l2": f"rotating {copies} weight copies ({copies * set_bytes / 1e6:.0f} MB > 126 MB L2)",
-                       "launch": "direct" if graphs is None else "one CUDA graph per weight copy"},
+                       "launch": "direct" if graphs is None else "one CUDA graph per weight copy",
+                       "step": "one transformer block: 4 activation rotations (q/k/v and gate/up share theirs) + 7 products"},
             "us_per_layer": ms_per_step * 1e3 / len(layers),
             "weight_bytes_per_step": set_bytes,
             "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

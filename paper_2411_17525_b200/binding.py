@@ -24,7 +24,7 @@ EXPORTS = [
     "higgs_workspace_bytes", "higgs_make_grid", "higgs_quantize", "higgs_linear", "higgs_rht",
     "higgs_pack_codes", "higgs_unpack_codes", "higgs_rotate_activations", "higgs_linear_prerotated",
     "higgs_linear_host", "higgs_linear_host_workspace_bytes", "higgs_linear_launch_count", "higgs_device_status",
-    "higgs_linear_static", "higgs_linear_static_capacity",
+    "higgs_linear_static", "higgs_linear_static_capacity", "higgs_linear_k_splits",
 ]
 
 
@@ -71,6 +71,8 @@ def _load() -> ctypes.CDLL:
     lib.higgs_linear_host.argtypes = [P, vp, i64, vp, vp, vp, vp, i32, vp, sz, vp]
     lib.higgs_linear_host_workspace_bytes.restype = sz
     lib.higgs_linear_host_workspace_bytes.argtypes = [P, i64, i32]
+    lib.higgs_linear_k_splits.restype = i32
+    lib.higgs_linear_k_splits.argtypes = [P, i64]
     lib.higgs_linear_launch_count.restype = i32
     lib.higgs_linear_launch_count.argtypes = [P, i64, i32]
     lib.higgs_linear_static.restype = i32
@@ -259,6 +261,10 @@ def scales_from_tile_major(scales: torch.Tensor, N: int) -> torch.Tensor:
     """Inverse of scales_to_tile_major: returns [N][K/g]."""
     Gn = scales.numel() // N
     return scales.reshape(N // 16, Gn, 16).permute(0, 2, 1).reshape(N, Gn).contiguous()
+
+
+def higgs_linear_k_splits(desc: higgs_desc, B: int) -> int:
+    return int(lib.higgs_linear_k_splits(ctypes.byref(desc), int(B)))
 
 
 def higgs_linear_launch_count(desc: higgs_desc, B: int, y_dtype: int = HIGGS_F32) -> int:

@@ -207,6 +207,11 @@ size_t higgs_linear_host_workspace_bytes(const higgs_desc* d, int64_t B, int y_d
     return inner + align_up((size_t)B * d->K * 2, 256) + align_up((size_t)B * d->N * (y_dtype == HIGGS_F32 ? 4 : 2), 256);
 }
 
+int higgs_linear_k_splits(const higgs_desc* d, int64_t B) {
+    if (check_desc(d) != HIGGS_OK || B < 1 || d->N == 0 || d->K == 0) return 0;
+    return linear_k_chunks(*d, B);
+}
+
 int higgs_linear_launch_count(const higgs_desc* d, int64_t B, int y_dtype) {
     if (check_desc(d) != HIGGS_OK || B < 1 || d->N == 0) return 0;
     const bool split = linear_k_chunks(*d, B) > 1;
