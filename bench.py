@@ -70,6 +70,22 @@ def measured_peaks():
         return 6650.0, "fallback"
 
 
+def max_over_ranks(ms: float, device, world: int) -> float:
+    """Duration of the timed region as the slowest rank saw it (replicas run independently; no data-path collective)."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(bytes_per_step: int, steps: int, ms: float, world: int) -> float:
+    """Whole-job effective weight bandwidth in GB/s: every rank processed bytes_per_step per step."""
+    return world * bytes_per_step / (ms / steps * 1e-3) / 1e9
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
 
@@ -300,11 +316,7 @@ def run_ours(args):
             torch.cuda.synchronize()
             barrier()
             ms = a.elapsed_time(b)
-        if world > 1:
-            t = torch.tensor([ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(ms, dev, world)
 
     sampler = ClockSampler(local)
     if rank == 0:
@@ -314,8 +326,8 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else None
 
     ms_per_step = ms / args.steps
-    value = world * set_bytes / (ms_per_step * 1e-3) / 1e9
-    e2e_value = world * set_bytes / (ms_e2e / args.steps * 1e-3) / 1e9
+    value = aggregate_value(set_bytes, args.steps, ms, world)
+    e2e_value = aggregate_value(set_bytes, args.steps, ms_e2e, world)
     h2d = sum(B * K * 2 for _, _, K in layers)
     d2h = sum(B * N * 4 for _, N, _ in layers)
 

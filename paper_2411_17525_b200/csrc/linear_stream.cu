@@ -207,18 +207,17 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
 
     constexpr uint32_t kSlotBytes = Codes::kBytes + 64u;       // codes + 16 fp16 scales (padded)
     const uint32_t ringA = base + kSmallBytes, ringB = lut + kLutBytes;
+    // Every warp's D slots are contiguous and lie entirely in one region, so slot d is one multiply-add away.
     const int nA = (int)((lut - ringA) / kSlotBytes);
     const int nB = (int)((dyn_end - ringB) / kSlotBytes);
-    int D = (nA + nB) / kWarps;
-    if (D > kMaxDepth) D = kMaxDepth;
-    auto slot_addr = [&](int d) {
-        const int idx = warp * D + d;
-        return idx < nA ? ringA + (uint32_t)idx * kSlotBytes : ringB + (uint32_t)(idx - nA) * kSlotBytes;
-    };
-    auto full_bar = [&](int d) { return bars + 8u * (uint32_t)(warp * kMaxDepth + d); };
-    // Partial tiles live in the upper halves of the table rows (8192 floats in 256 pieces of 32).  The tile of
-    // (item slot q, slice ns) holds B columns of 16 rows: float index ((q * NS + ns) * B + col) * 16 + row.
-    auto part_addr = [&](int fidx) { return lut + 128u + (uint32_t)((fidx >> 5) * 256 + (fidx & 31) * 4); };
+    int D = kMaxDepth;
+    while (D > 1 && nA / D + nB / D < kWarps) --D;
+    const int warps_in_A = nA / D;
+    const uint32_t slot0 = warp < warps_in_A ? ringA + (uint32_t)(warp * D) * kSlotBytes
+                                             : ringB + (uint32_t)((warp - warps_in_A) * D) * kSlotBytes;
+    const uint32_t bar0 = bars + 8u * (uint32_t)(warp * kMaxDepth);
+    auto slot_addr = [&](int d) { return slot0 + (uint32_t)d * kSlotBytes; };
+    auto full_bar = [&](int d) { return bar0 + 8u * (uint32_t)d; };
 
     // ---- this block's items and this warp's share of them ----
     // (all per-task bookkeeping below is incremental 32-bit arithmetic)
@@ -235,9 +234,16 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     const int n_tasks = (!flusher && n_items > phase) ? (n_items - phase + PG - 1) / PG : 0;
     const int gl = (slice * KS) >> 10;         // group of this slice inside the item
     const int ng = prm.ck >> 10;               // groups per item
-    int acc_slots = 512 / (NS * prm.B);        // power of two because NS and the slot count are; B rounds it down
+    // Partial tiles live in the upper halves of the table rows: 256 pieces of 32 floats (128 B), piece i at
+    // lut + 128 + 256 i.  A tile holds B columns of 16 rows ([col][row]) in tile_pieces whole pieces; the tile of
+    // (item slot q, slice ns) is tile q * NS + ns.  Element (col, row) of a tile sits in piece (col*16+row) >> 5.
+    const int tile_pieces = (16 * prm.B + 31) >> 5;
+    int acc_slots = 256 / (NS * tile_pieces);
     { int p2 = 1; while (p2 * 2 <= acc_slots && p2 < kMaxAccSlots) p2 *= 2; acc_slots = p2; }
     const int acc_shift = 31 - __clz(acc_slots);
+    const uint32_t part0 = lut + 128u;
+    const uint32_t tile_stride = (uint32_t)tile_pieces * 256u;         // bytes between consecutive tiles
+    const uint32_t q_stride = (uint32_t)NS * tile_stride;              // bytes between consecutive item slots
 
     // ---- prologue ----
     if (lane == 0 && !flusher) {
@@ -252,20 +258,22 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncwarp();
 
-    // task cursor used for issuing copies (runs D tasks ahead of the compute cursor)
-    int i_chunk = chunk_begin, i_rt = rt_begin + phase;
-    while (i_rt >= tiles) { i_rt -= tiles; ++i_chunk; }
-    auto issue = [&](int d) {   // lane 0: start the copies of the task at the issue cursor into slot d, advance the cursor
-        const uint32_t dst = slot_addr(d);
-        const int64_t kslice = (int64_t)i_chunk * prm.ck + (int64_t)slice * KS;
-        const uint8_t* src = prm.packed + (SIX ? (((int64_t)i_rt * (prm.K / 128) + kslice / 128) * 768)
-                                               : (((int64_t)i_rt * (prm.K / 64) + kslice / 64) * 512));
-        const __half* ssrc = prm.scales + ((int64_t)i_rt * groups + i_chunk * ng + gl) * 16;
-        mbar_expect_tx(full_bar(d), Codes::kBytes + 32u);
-        bulk_load(dst, src, Codes::kBytes, full_bar(d));
-        bulk_load(dst + Codes::kBytes, ssrc, 32u, full_bar(d));
-        i_rt += PG;
-        while (i_rt >= tiles) { i_rt -= tiles; ++i_chunk; }
+    // Copy cursor (runs D tasks ahead of the compute cursor): this warp's tasks are rt_begin + phase, + PG, ... of
+    // one K-chunk, so source addresses advance by constant strides.
+    const int64_t kslice = (int64_t)chunk_begin * prm.ck + (int64_t)slice * KS;
+    const int64_t rt_first = rt_begin + phase;
+    const uint8_t* src_next = prm.packed + (SIX ? ((rt_first * (prm.K / 128) + kslice / 128) * 768)
+                                                : ((rt_first * (prm.K / 64) + kslice / 64) * 512));
+    const __half* ssrc_next = prm.scales + (rt_first * groups + chunk_begin * ng + gl) * 16;
+    const int64_t src_stride = (int64_t)PG * (SIX ? prm.K * 6 : prm.K * 8);
+    const int64_t ssrc_stride = (int64_t)PG * groups * 16;
+    auto issue = [&](int d) {   // lane 0: start the copies of the next task into slot d
+        const uint32_t dst = slot_addr(d), bar = full_bar(d);
+        mbar_expect_tx(bar, Codes::kBytes + 32u);
+        bulk_load(dst, src_next, Codes::kBytes, bar);
+        bulk_load(dst + Codes::kBytes, ssrc_next, 32u, bar);
+        src_next += src_stride;
+        ssrc_next += ssrc_stride;
     };
     // the weight stream depends on nothing this kernel computes: start it before anything else
     int issued = 0;
@@ -356,7 +364,8 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
                     uint4 raw[16];
 #pragma unroll
                     for (int ns = 0; ns < 16; ++ns)
-                        raw[ns] = lds128(part_addr((q * NS + (ns < NS ? ns : 0)) * prm.B * 16 + e));
+                        raw[ns] = lds128(part0 + (uint32_t)q * q_stride + (uint32_t)(ns < NS ? ns : 0) * tile_stride +
+                                         (uint32_t)((e >> 5) * 256 + (e & 31) * 4));
                     float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                     for (int ns = 0; ns < 16; ++ns) {
@@ -403,6 +412,7 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
 
     // ---- main loop: this warp's tasks ----
     const uint32_t lut_lane = lut + lane * 4;
+    const uint32_t part_lane = part0 + (uint32_t)slice * tile_stride + (uint32_t)(t * 256 + g * 4);
     int d = 0;
     uint32_t ph = 0;
     bool ok = true;
@@ -458,7 +468,8 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
             }
         }
         if (!ok) break;
-        const int tile0 = (q * NS + slice) * prm.B * 16;       // first float of this warp's partial tile
+        // this lane's elements of the tile: (col 2t, row g) at piece t, float g; the others at fixed offsets
+        const uint32_t pa = part_lane + (uint32_t)q * q_stride;
 #pragma unroll
         for (int nb = 0; nb < NB; ++nb) {
             const int c0 = nb * 8 + 2 * t;           // this lane holds columns c0, c0+1 of rows g and g+8
@@ -467,12 +478,12 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
             const float v2 = (acc4[0][nb][2] + acc4[1][nb][2]) + (acc4[2][nb][2] + acc4[3][nb][2]);
             const float v3 = (acc4[0][nb][3] + acc4[1][nb][3]) + (acc4[2][nb][3] + acc4[3][nb][3]);
             if (c0 < prm.B) {                        // only the B valid columns exist
-                asm volatile("st.shared.f32 [%0], %1;" ::"r"(part_addr(tile0 + c0 * 16 + g)), "f"(v0 * s_lo) : "memory");
-                asm volatile("st.shared.f32 [%0], %1;" ::"r"(part_addr(tile0 + c0 * 16 + g + 8)), "f"(v2 * s_hi) : "memory");
+                asm volatile("st.shared.f32 [%0], %1;" ::"r"(pa + (uint32_t)(nb * 1024)), "f"(v0 * s_lo) : "memory");
+                asm volatile("st.shared.f32 [%0], %1;" ::"r"(pa + (uint32_t)(nb * 1024 + 32)), "f"(v2 * s_hi) : "memory");
             }
             if (c0 + 1 < prm.B) {
-                asm volatile("st.shared.f32 [%0], %1;" ::"r"(part_addr(tile0 + (c0 + 1) * 16 + g)), "f"(v1 * s_lo) : "memory");
-                asm volatile("st.shared.f32 [%0], %1;" ::"r"(part_addr(tile0 + (c0 + 1) * 16 + g + 8)), "f"(v3 * s_hi) : "memory");
+                asm volatile("st.shared.f32 [%0], %1;" ::"r"(pa + (uint32_t)(nb * 1024 + 64)), "f"(v1 * s_lo) : "memory");
+                asm volatile("st.shared.f32 [%0], %1;" ::"r"(pa + (uint32_t)(nb * 1024 + 96)), "f"(v3 * s_hi) : "memory");
             }
         }
         __syncwarp();
