@@ -25,14 +25,15 @@
  *     returns HIGGS_ERR_CUDA.
  *
  * The sign function of the randomised Hadamard transform (part of the ABI):
- *   z = xi + (j+1) * 0x9E3779B97F4A7C15            (mod 2^64)
- *   z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9
- *   z = (z ^ (z >> 27)) * 0x94D049BB133111EB
- *   z =  z ^ (z >> 31)
- *   sign(xi, j) = -1 if the top bit of z is set, else +1
- * i.e. output j of the splitmix64 stream seeded with xi.  One sign per input
- * index j in [0, K), shared by every row of W and every token, so that the
- * activations are rotated once (Appendix F: "same xi ... same groups").
+ *   out(xi, m):  z = xi + (m+1) * 0x9E3779B97F4A7C15            (mod 2^64)
+ *                z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9
+ *                z = (z ^ (z >> 27)) * 0x94D049BB133111EB
+ *                z =  z ^ (z >> 31)
+ *   i.e. output number m of the splitmix64 stream seeded with xi, and
+ *   sign(xi, j) = -1 if bit (j mod 64) of out(xi, floor(j / 64)) is set, else +1.
+ * One sign per input index j in [0, K), shared by every row of W and every
+ * token, so that the activations are rotated once (Appendix F: "same xi ...
+ * same groups").
  *
  * The transform itself: RHT(v) = H * diag(sign) * v on each group of g values,
  * H the Sylvester-ordered Hadamard matrix H[i][j] = (-1)^popcount(i & j).

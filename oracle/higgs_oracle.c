@@ -53,16 +53,20 @@ void higgs_oracle_set_threads(int t) {
 /* ------------------------------------------------------------------------- */
 /* Sign of the RHT for input index j (Algorithm 1, "RHT seed xi").            */
 /* The paper fixes no generator.  Reading used here: one independent          */
-/* Rademacher sign per input index j, the same for every row and token,       */
-/* obtained from a counter-based 64-bit mixer (the splitmix64 finaliser) of   */
-/* z = xi + (j+1)*0x9E3779B97F4A7C15; the top bit of the mixed word is the    */
-/* sign bit (set -> -1).                                                      */
-double higgs_oracle_sign(uint64_t xi, int64_t j) {
-    uint64_t z = xi + ((uint64_t)j + 1u) * 0x9E3779B97F4A7C15ull;
+/* Rademacher sign per input index j, the same for every row and token, taken */
+/* from the splitmix64 stream seeded with xi: output number m of that stream  */
+/* is mix(xi + (m+1)*0x9E3779B97F4A7C15) with the splitmix64 finaliser, and    */
+/* sign j is bit (j mod 64) of output number floor(j/64) (bit set -> -1).      */
+static uint64_t splitmix64_output(uint64_t xi, uint64_t m) {
+    uint64_t z = xi + (m + 1u) * 0x9E3779B97F4A7C15ull;
     z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
     z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
-    z = z ^ (z >> 31);
-    return (z >> 63) ? -1.0 : 1.0;
+    return z ^ (z >> 31);
+}
+
+double higgs_oracle_sign(uint64_t xi, int64_t j) {
+    uint64_t z = splitmix64_output(xi, (uint64_t)j >> 6);
+    return ((z >> ((uint64_t)j & 63u)) & 1u) ? -1.0 : 1.0;
 }
 
 /* ------------------------------------------------------------------------- */

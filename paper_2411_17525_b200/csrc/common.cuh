@@ -14,13 +14,16 @@ constexpr int kGroup = 1024;     // the only supported group size g
 constexpr int kRowTile = 16;     // rows of W per mma tile (m16n8k16) and per scale tile
 constexpr int kBlockK = 64;      // k-extent of one 512-byte packed block
 
-// Top bit of output j of the splitmix64 stream seeded with xi: 1 -> sign -1.
-__host__ __device__ __forceinline__ uint32_t sign_bit(uint64_t xi, int64_t j) {
-    uint64_t z = xi + ((uint64_t)j + 1ull) * 0x9E3779B97F4A7C15ull;
+// Output number m of the splitmix64 stream seeded with xi: 64 sign bits, for inputs 64 m .. 64 m + 63.
+__host__ __device__ __forceinline__ uint64_t sign_word(uint64_t xi, uint64_t m) {
+    uint64_t z = xi + (m + 1ull) * 0x9E3779B97F4A7C15ull;
     z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
     z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
-    z = z ^ (z >> 31);
-    return (uint32_t)(z >> 63);
+    return z ^ (z >> 31);
+}
+// sign of input j: bit (j mod 64) of output floor(j / 64); 1 -> sign -1.
+__host__ __device__ __forceinline__ uint32_t sign_bit(uint64_t xi, int64_t j) {
+    return (uint32_t)((sign_word(xi, (uint64_t)j >> 6) >> ((uint64_t)j & 63ull)) & 1ull);
 }
 
 // How codes are stored in the packed stream.
@@ -98,6 +101,19 @@ __device__ __forceinline__ void fwht1024_warp(float (&v)[32], int lane) {
             float o = __shfl_xor_sync(0xffffffffu, v[r], m);
             v[r] = upper ? (o - v[r]) : (v[r] + o);
         }
+    }
+}
+
+// Flips the signs of the 32 values of this lane (mapping above) for the group starting at input k0 (a multiple
+// of 1024): chunk c covers inputs k0 + c*256 + lane*8 .. +7, eight consecutive bits of one 64-bit sign word.
+__device__ __forceinline__ void apply_signs1024(float (&v)[32], uint64_t xi, int64_t k0, int lane) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const uint64_t j0 = (uint64_t)k0 + (uint64_t)(c * 256 + lane * 8);
+        const uint32_t bits = (uint32_t)(sign_word(xi, j0 >> 6) >> (j0 & 63ull)) & 0xffu;
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+            v[c * 8 + e] = __uint_as_float(__float_as_uint(v[c * 8 + e]) ^ (((bits >> e) & 1u) << 31));
     }
 }
 

@@ -64,10 +64,8 @@ __global__ void __launch_bounds__(128) encode_kernel(const T* __restrict__ W, co
     const float inv = s > 0.0f ? 1.0f / s : 0.0f;
 
 #pragma unroll
-    for (int r = 0; r < 32; ++r) {
-        uint32_t sb = sign_bit(xi, gi * kGroup + fwht_index(lane, r));
-        v[r] = __uint_as_float(__float_as_uint(v[r] * inv) ^ (sb << 31));
-    }
+    for (int r = 0; r < 32; ++r) v[r] *= inv;
+    apply_signs1024(v, xi, gi * kGroup, lane);
     fwht1024_warp(v, lane);
 
     // scales are stored tile-major: [row / 16][group][row % 16]

@@ -37,14 +37,6 @@ __device__ __forceinline__ void load_group<float>(const float* __restrict__ src,
     }
 }
 
-__device__ __forceinline__ void apply_signs(float (&v)[32], uint64_t xi, int64_t k0, int lane) {
-#pragma unroll
-    for (int r = 0; r < 32; ++r) {
-        uint32_t sb = sign_bit(xi, k0 + fwht_index(lane, r));
-        v[r] = __uint_as_float(__float_as_uint(v[r]) ^ (sb << 31));
-    }
-}
-
 // One warp per (token, group): x+ = (H/32) diag(sign) x, written as fp16 in natural
 // order.  Extra threads beyond the transform work clear `zero_ptr` (the fp32
 // accumulation target of a K-split product) so no separate memset launch is needed.
@@ -64,7 +56,7 @@ __global__ void __launch_bounds__(256) rht_activations_kernel(const T* __restric
     const int64_t b = warp / groups, gi = warp % groups;
     float v[32];
     load_group<T>(x + b * K + gi * kGroup, lane, v);
-    apply_signs(v, xi, gi * kGroup, lane);
+    apply_signs1024(v, xi, gi * kGroup, lane);
     fwht1024_warp(v, lane);
     __half* dst = xdag + b * K + gi * kGroup;
 #pragma unroll
@@ -89,7 +81,7 @@ __global__ void __launch_bounds__(256) rht_debug_kernel(const T* __restrict__ x,
     const int64_t b = warp / groups, gi = warp % groups;
     float v[32];
     load_group<T>(x + b * K + gi * kGroup, lane, v);
-    apply_signs(v, xi, gi * kGroup, lane);
+    apply_signs1024(v, xi, gi * kGroup, lane);
     fwht1024_warp(v, lane);
     float* dst = out + b * K + gi * kGroup;
 #pragma unroll

@@ -62,9 +62,13 @@ def test_orthogonality_norm_involution(g):
 
 
 def test_sign_stream_matches_published_splitmix64_vectors(golden):
-    want = golden("splitmix64.txt")["topbits_seed0"]
-    got = [oracle.sign(0, j) for j in range(len(want))]
-    assert got == [(-1.0 if b else 1.0) for b in want]
+    g = golden("splitmix64.txt")
+    words = [(int(h) << 32) | int(l) for h, l in zip(g["hi32"], g["lo32"])]
+    assert words[0] == 0xE220A8397B1DCDAF and words[4] == 0x1B39896A51A8749B
+    for m, w in enumerate(words):
+        for b in range(64):
+            want = -1.0 if (w >> b) & 1 else 1.0
+            assert oracle.sign(0, 64 * m + b) == want, (m, b)
 
 
 def test_sign_properties():
