@@ -63,7 +63,9 @@ size_t higgs_workspace_bytes(const higgs_desc* d, int op, int64_t B) {
     if (op == HIGGS_OP_QUANTIZE) return align_up(higgs_canonical_bytes(d), 256) + 256;
     if (op == HIGGS_OP_LINEAR) {
         if (B < 1) return 0;
-        return align_up((size_t)B * d->K * 2, 256) + align_up((size_t)B * d->N * 4, 256) + 256;
+        const size_t stream_path = align_up((size_t)B * d->K * 2, 256) + align_up((size_t)B * d->N * 4, 256) + 256;
+        const size_t tc_path = tc_eligible(*d, B) ? align_up(tc_workspace_bytes(*d, B), 256) + 256 : 0;
+        return stream_path > tc_path ? stream_path : tc_path;
     }
     return 0;
 }
@@ -153,6 +155,11 @@ int higgs_linear(const higgs_desc* d, const void* x, int64_t B, const void* pack
     int rc = linear_args(d, B, x, packed, scales, grid, y, y_dtype, workspace, workspace_bytes);
     if (rc != HIGGS_OK) return rc < 0 ? HIGGS_OK : rc;
     cudaStream_t st = as_stream(stream);
+    if (tc_eligible(*d, B)) {
+        // dense-contraction regime: rotate into the blocked operand layout, then one tcgen05 pass over the codes
+        return launch_linear_tc(*d, x, B, packed, scales, grid, y, y_dtype == HIGGS_F32 ? 0 : 1,
+                                static_cast<__half*>(workspace), st);
+    }
     __half* xdag = static_cast<__half*>(workspace);
     float* y32 = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up((size_t)B * d->K * 2, 256));
     const bool split = linear_k_chunks(*d, B) > 1;
@@ -214,6 +221,7 @@ int higgs_linear_k_splits(const higgs_desc* d, int64_t B) {
 
 int higgs_linear_launch_count(const higgs_desc* d, int64_t B, int y_dtype) {
     if (check_desc(d) != HIGGS_OK || B < 1 || d->N == 0) return 0;
+    if (tc_eligible(*d, B)) return 2;
     const bool split = linear_k_chunks(*d, B) > 1;
     return 1 + (int)((B + 15) / 16) + ((split && y_dtype == HIGGS_BF16) ? 1 : 0);
 }

@@ -136,6 +136,12 @@ size_t make_grid_workspace(int p, int n, int64_t m);
 int launch_make_grid(int p, int n, const float* samples, int64_t m, int max_iters, float* grid_out, float* mse_out,
                      int32_t* iters_out, void* ws, cudaStream_t st);
 int linear_k_chunks(const higgs_desc& d, int64_t B);
+// tensor-core path (B > 16)
+bool tc_eligible(const higgs_desc& d, int64_t B);
+size_t tc_workspace_bytes(const higgs_desc& d, int64_t B);
+int launch_linear_tc(const higgs_desc& d, const void* x, int64_t B, const void* packed, const void* scales,
+                     const float* grid, void* y, int y_mode, __half* xdag_tc, cudaStream_t st);
+int read_tc_status(int clear);
 int read_device_status(cudaStream_t st, int clear);
 
 }  // namespace higgs

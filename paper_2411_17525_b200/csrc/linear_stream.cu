@@ -623,7 +623,8 @@ int read_device_status(cudaStream_t st, int clear) {
         const int zero = 0;
         if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return HIGGS_ERR_CUDA;
     }
-    return v;
+    const int tc = read_tc_status(clear);
+    return v != 0 ? v : tc;
 }
 
 }  // namespace higgs

@@ -1,0 +1,425 @@
+// Large-batch product in the rotated space (Appendix F, "Rotating Activations") on the 5th-generation tensor
+// cores:  y[b][r] = sum_i scale[r][i] * sum_t < G[code[r][i][t]], x+[b][i][2t:2t+2] >  for 17 <= B tokens.
+// Here the path is a dense contraction, so it runs as tcgen05.mma with the accumulator in tensor memory (TMEM).
+//
+// One block computes a 128-row x BN-token tile of y over all of K ("swap-AB": the weights are the M = 128 side).
+//   producer lane    streams, per 64-input stage, the codes of the 128 rows (8 bulk copies of 512 B) and the BN x 64
+//                    tile of rotated activations (one bulk copy) into shared memory (TMA, cp.async.bulk + mbarrier);
+//   16 dequant warps each thread owns one row of the tile: it turns the row's 32 code bytes of the stage into table
+//                    lookups (fp16 pairs), multiplies by the row's group scale and writes them with tcgen05.st
+//                    straight into the TMEM columns the MMA reads as its A operand - dequantisation is fused into
+//                    the operand load and the dequantised weights never touch shared or global memory;
+//   MMA lane         issues four tcgen05.mma (M=128, N=BN, K=16, A from TMEM, B through a shared-memory
+//                    descriptor) per stage and commits them to an mbarrier that frees the stage;
+//   epilogue         the first four dequant warps read the fp32 accumulator with tcgen05.ld and store y.
+// The group scale is folded into the fp16 A operand (relative rounding 2^-11, the same size as the rounding of the
+// table entry itself), so one accumulation runs over all of K.  Every wait is bounded; TMEM is always released.
+#include "common.cuh"
+
+namespace higgs {
+
+__device__ int g_tc_status = 0;
+
+namespace {
+
+struct TcParams {
+    const uint8_t* packed;   // packed code stream (byte format)
+    const __half* scales;    // tile-major scales [N/16][K/g][16]
+    const float* grid;       // [n][p]
+    const __half* xdag;      // rotated activations, blocked: [batch tile][K/64][BN/8][8 k-cores][8 tokens][8 inputs]
+    void* y;                 // [B][N]
+    int64_t N, K;
+    int B, BN, n, p, y_mode; // y_mode 0: fp32, 1: bf16
+};
+
+constexpr uint32_t kTcSmem = 232448;
+constexpr int kTcStages = 4;
+constexpr int kTcDequantWarps = 16;
+constexpr int kTcThreads = (2 + kTcDequantWarps) * 32;
+constexpr uint32_t kTcCodeStage = 4096;      // 128 rows x 64 inputs, one byte per input pair
+constexpr uint32_t kTcWait = 1u << 22;
+constexpr uint32_t kTcACol = 256;            // TMEM columns [0, BN) accumulator, [256, 256 + 32*stages) A operand
+
+__device__ __forceinline__ uint32_t t_lds32(uint32_t a) { uint32_t v; asm("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(a)); return v; }
+__device__ __forceinline__ uint4 t_lds128(uint32_t a) {
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ void t_mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void t_mbar_arrive(uint32_t bar) {
+    asm volatile("{ .reg .b64 st; mbarrier.arrive.shared::cta.b64 st, [%0]; }" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void t_mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("{ .reg .b64 st; mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1; }" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t t_mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok;
+}
+// Bounded wait: false when the block is aborting or this wait ran out (then it raises the abort flag and the status).
+__device__ __forceinline__ bool t_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t it = 0;; ++it) {
+        if (t_mbar_try(bar, parity)) return true;
+        if ((it & 63u) == 63u) {
+            if (*abort_flag) return false;
+            if (it > kTcWait) {
+                *abort_flag = 1;
+                atomicExch(&g_tc_status, (int)HIGGS_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ void t_bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major operand without swizzle: 8-row x 16-byte core matrices, the two
+// K-adjacent cores of an MMA step `lbo` bytes apart, cores adjacent along N `sbo` bytes apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+    const uint64_t lo = (uint64_t)((addr & 0x3ffffu) >> 4) | ((uint64_t)(lbo >> 4) << 16);
+    const uint64_t hi = (uint64_t)(sbo >> 4) | (1ull << 14);     // bits 46-47: descriptor version 1; layout type 0
+    return lo | (hi << 32);
+}
+// D[tmem] (+)= A[tmem] * B[smem descriptor], one thread issues
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}\n"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+          "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+          "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,"
+        "%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams prm) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    // ---- shared memory map ----
+    //   [base, base+2 KB)    mbarriers, TMEM base address, abort flag
+    //   [base+2 KB, lut)     code stages (4 x 4 KB) and activation stage 3
+    //   [lut, lut+64 KB)     lookup table, 256-byte rows (bytes 0..127 = the entry replicated per lane)
+    //   [lut+64 KB, end)     activation stages 0..2 (BN x 128 B each, at most 32 KB)
+    const uint32_t base = (uint32_t)__cvta_generic_to_shared(smem_raw);
+    const uint32_t lut = (base + 2048u + 0xffffu) & ~0xffffu;
+    const uint32_t bars = base;
+    auto load_full = [&](int s) { return bars + 8u * (uint32_t)s; };
+    auto a_full = [&](int s) { return bars + 8u * (uint32_t)(kTcStages + s); };
+    auto mma_done = [&](int s) { return bars + 8u * (uint32_t)(2 * kTcStages + s); };
+    const uint32_t d_full = bars + 8u * (uint32_t)(3 * kTcStages);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_raw + 256);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + 264);
+    const uint32_t code0 = base + 2048u;                                   // 16 KB of code stages
+    const uint32_t bstage3 = (code0 + kTcStages * kTcCodeStage + 1023u) & ~1023u;
+    auto code_stage = [&](int s) { return code0 + (uint32_t)s * kTcCodeStage; };
+    auto b_stage = [&](int s) { return s < 3 ? lut + 65536u + (uint32_t)s * 32768u : bstage3; };
+
+    const int BN = prm.BN;
+    const int ksteps = (int)(prm.K / 64);
+    const int64_t row0 = (int64_t)blockIdx.x * 128;
+    const int bt = blockIdx.y;
+    const uint32_t b_bytes = (uint32_t)BN * 128u;
+
+    // ---- prologue ----
+    if (tid == 0) {
+        for (int s = 0; s < kTcStages; ++s) { t_mbar_init(load_full(s), 1); t_mbar_init(a_full(s), 4); t_mbar_init(mma_done(s), 1); }
+        t_mbar_init(d_full, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {   // one warp allocates all 512 TMEM columns (one block per SM, so nobody else wants them)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + 256u), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    pdl_trigger();
+    {   // lookup table: warp w fills rows w, w+18, ...; the grid is a constant of the layer
+        constexpr int kW = kTcThreads / 32;
+        constexpr int kRows = (256 + kW - 1) / kW;
+        uint32_t ent[kRows];
+#pragma unroll
+        for (int r = 0; r < kRows; ++r) {
+            const int idx = warp + r * kW;
+            float lo = 0.f, hi = 0.f;
+            if (idx < 256) {
+                if (prm.p == 2) {
+                    const float2 gp = __ldg(reinterpret_cast<const float2*>(prm.grid) + (idx & (prm.n - 1)));
+                    lo = gp.x; hi = gp.y;
+                } else {
+                    lo = __ldg(prm.grid + (idx & 15));
+                    hi = __ldg(prm.grid + (idx >> 4));
+                }
+            }
+            __half2 h = __floats2half2_rn(lo, hi);
+            ent[r] = *reinterpret_cast<uint32_t*>(&h);
+        }
+#pragma unroll
+        for (int r = 0; r < kRows; ++r) {
+            const int idx = warp + r * kW;
+            if (idx < 256) *reinterpret_cast<uint32_t*>(smem_raw + (lut - base) + idx * 256 + lane * 4) = ent[r];
+        }
+    }
+    pdl_wait();            // the rotated activations are the previous kernel's output
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        // =============================== producer ===============================
+        if (lane == 0) {
+            int issued = 0;
+            for (int j = 0; j < ksteps; ++j) {
+                const int s = j & (kTcStages - 1), it = j / kTcStages;
+                if (it >= 1 && !t_wait(mma_done(s), (uint32_t)((it - 1) & 1), abort_flag)) break;
+                t_mbar_expect_tx(load_full(s), kTcCodeStage + b_bytes);
+#pragma unroll
+                for (int rtl = 0; rtl < 8; ++rtl)
+                    t_bulk_load(code_stage(s) + rtl * 512, prm.packed + ((row0 / 16 + rtl) * (prm.K / 64) + j) * 512, 512u,
+                                load_full(s));
+                t_bulk_load(b_stage(s), prm.xdag + ((int64_t)bt * ksteps + j) * BN * 64, b_bytes, load_full(s));
+                ++issued;
+            }
+            // never leave with copies in flight: wait (bounded) for the last stages issued
+            const int first = issued > kTcStages ? issued - kTcStages : 0;
+            for (int j = first; j < issued; ++j) {
+                const int s = j & (kTcStages - 1);
+                for (uint32_t it = 0; it < kTcWait && !t_mbar_try(load_full(s), (uint32_t)((j / kTcStages) & 1)); ++it) {}
+            }
+        }
+    } else if (warp == 1) {
+        // =============================== MMA issuer ===============================
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | (8u << 24);   // f32 accumulate, f16 x f16, K-major, M=128
+            bool ok = true;
+            for (int j = 0; j < ksteps && ok; ++j) {
+                const int s = j & (kTcStages - 1), it = j / kTcStages;
+                ok = t_wait(load_full(s), (uint32_t)(it & 1), abort_flag) && t_wait(a_full(s), (uint32_t)(it & 1), abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    tc_mma(tmem, tmem + kTcACol + 32u * s + 8u * c, smem_desc(b_stage(s) + 256u * c, 128u, 1024u), idesc,
+                           (uint32_t)((j | c) != 0));
+                tc_commit(mma_done(s));       // frees the stage (shared memory and the A columns) when these MMAs are done
+            }
+            tc_commit(d_full);                // all MMAs issued so far are done -> the accumulator is final
+        }
+    } else {
+        // =============================== dequant warps (then epilogue) ===============================
+        // A warp may touch only the TMEM lanes 32 (warp % 4) .. +31; the four warps sharing a quadrant take the
+        // stages s = 0..3 in turn (warp group sg works on ring slot sg).
+        const int q = warp & 3, sg = (warp - 2) >> 2;
+        const int i = 32 * q + lane;               // row of the tile = TMEM lane
+        const int rtl = i >> 4, g = i & 7, h = (i >> 3) & 1;
+        const uint32_t lut_lane = lut + lane * 4;
+        const uint32_t sel0 = 0x7604u + ((uint32_t)h << 4), sel1 = 0x7624u + ((uint32_t)h << 4);   // bytes h and h+2 of a word
+        const int rot = g >> 1;                    // chunk rotation that makes the 16-byte code loads conflict-free
+        const int groups = (int)(prm.K / kGroup);
+        const __half* sc_row = prm.scales + ((row0 / 16 + rtl) * groups) * 16 + (i & 15);
+        const uint32_t t_lane = tmem + ((uint32_t)(32 * q) << 16);
+        int cur_group = -1;
+        uint32_t sc2 = 0;
+        bool ok = true;
+        for (int j = sg; j < ksteps; j += kTcStages) {
+            const int s = sg, it = j / kTcStages;
+            if (it >= 1 && !t_wait(mma_done(s), (uint32_t)((it - 1) & 1), abort_flag)) { ok = false; break; }
+            if (!t_wait(load_full(s), (uint32_t)(it & 1), abort_flag)) { ok = false; break; }
+            if ((j >> 4) != cur_group) {           // new group of 1024 inputs: this row's scale
+                cur_group = j >> 4;
+                const __half sc = sc_row[cur_group * 16];
+                const __half2 s2 = __half2half2(sc);
+                sc2 = *reinterpret_cast<const uint32_t*>(&s2);
+            }
+            // the row's codes of this stage: the 16-byte chunks of lanes (g, t = 0..3) of row tile rtl; instruction jj
+            // reads chunk (jj + rot) & 3 so that the eight g of a warp hit eight different bank groups
+            uint4 c4[4];
+#pragma unroll
+            for (int jj = 0; jj < 4; ++jj)
+                c4[jj] = t_lds128(code_stage(s) + (uint32_t)(rtl * 512 + (g * 4 + ((jj + rot) & 3)) * 16));
+            // undo the rotation: chunk t was loaded by instruction (t - rot) & 3
+            if (rot & 1) { const uint4 t0 = c4[0]; c4[0] = c4[3]; c4[3] = c4[2]; c4[2] = c4[1]; c4[1] = t0; }
+            if (rot & 2) { uint4 t0 = c4[0]; c4[0] = c4[2]; c4[2] = t0; t0 = c4[1]; c4[1] = c4[3]; c4[3] = t0; }
+            uint32_t a[32];
+#pragma unroll
+            for (int m = 0; m < 4; ++m) {
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const uint32_t w = m == 0 ? c4[t].x : m == 1 ? c4[t].y : m == 2 ? c4[t].z : c4[t].w;
+                    // input pairs 8m + t (byte h) and 8m + 4 + t (byte h + 2) of the 64-input block
+                    const uint32_t e0 = t_lds32(__byte_perm(w, lut_lane, sel0));
+                    const uint32_t e1 = t_lds32(__byte_perm(w, lut_lane, sel1));
+                    const __half2 p0 = __hmul2(*reinterpret_cast<const __half2*>(&e0), *reinterpret_cast<const __half2*>(&sc2));
+                    const __half2 p1 = __hmul2(*reinterpret_cast<const __half2*>(&e1), *reinterpret_cast<const __half2*>(&sc2));
+                    a[m * 8 + t] = *reinterpret_cast<const uint32_t*>(&p0);
+                    a[m * 8 + 4 + t] = *reinterpret_cast<const uint32_t*>(&p1);
+                }
+            }
+            tc_st32(t_lane + kTcACol + 32u * s, a);          // columns 8m + jj of the stage = input pair 8m + jj
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) t_mbar_arrive(a_full(s));
+        }
+        if (sg == 0 && ok) {
+            // epilogue: accumulator row i, 32 token columns at a time
+            if (t_wait(d_full, 0u, abort_flag)) {
+                tc_fence_after();
+                const int64_t row = row0 + i;
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    uint32_t d[32];
+                    tc_ld32(t_lane + (uint32_t)c0, d);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int r = 0; r < 32; ++r) {
+                        const int b = bt * BN + c0 + r;
+                        if (c0 + r < BN && b < prm.B) {
+                            const float v = __uint_as_float(d[r]);
+                            if (prm.y_mode == 0) static_cast<float*>(prm.y)[(int64_t)b * prm.N + row] = v;
+                            else static_cast<__nv_bfloat16*>(prm.y)[(int64_t)b * prm.N + row] = __float2bfloat16_rn(v);
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- every role ends here, aborted or not: TMEM must be handed back ----
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+    }
+}
+
+}  // namespace
+
+namespace {
+
+// Rotation of the activations (Appendix F) for the tensor-core path: one warp per (token, group), output written in
+// the blocked order the MMA's shared-memory descriptor expects, so that one stage (BN tokens x 64 inputs) is one
+// contiguous run:  [batch tile][K/64][BN/8 token blocks][8 input cores][8 tokens][8 inputs] fp16.
+__global__ void __launch_bounds__(256) rht_activations_tc_kernel(const __nv_bfloat16* __restrict__ x, __half* __restrict__ xdag,
+                                                                 int64_t B, int64_t K, uint64_t xi, int BN) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int64_t groups = K / kGroup;
+    pdl_trigger();
+    pdl_wait();
+    if (warp >= B * groups) return;
+    const int64_t b = warp / groups, gi = warp % groups;
+    const __nv_bfloat16* src = x + b * K + gi * kGroup;
+    float v[32];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(src + c * 256 + lane * 8));
+        const uint32_t w4[4] = {q4.x, q4.y, q4.z, q4.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            v[c * 8 + 2 * e] = __uint_as_float(w4[e] << 16);
+            v[c * 8 + 2 * e + 1] = __uint_as_float(w4[e] & 0xffff0000u);
+        }
+    }
+    apply_signs1024(v, xi, gi * kGroup, lane);
+    fwht1024_warp(v, lane);
+    const int64_t bt = b / BN, nloc = b % BN;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        uint32_t w4[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            __half2 h = __floats2half2_rn(v[c * 8 + 2 * e] * 0.03125f, v[c * 8 + 2 * e + 1] * 0.03125f);
+            w4[e] = *reinterpret_cast<uint32_t*>(&h);
+        }
+        const int64_t k = gi * kGroup + c * 256 + lane * 8;        // 8 consecutive inputs = one core-matrix row
+        const int64_t off = ((bt * (K / 64) + k / 64) * BN * 64) + (nloc / 8) * 512 + ((k % 64) / 8) * 64 + (nloc % 8) * 8;
+        *reinterpret_cast<uint4*>(xdag + off) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+    }
+}
+
+}  // namespace
+
+// Token-tile width of the tensor-core path for batch B: a multiple of 16, at most 256, balanced over the tiles.
+int tc_batch_tile(int64_t B) {
+    const int64_t tiles = (B + 255) / 256;
+    const int64_t per = (B + tiles - 1) / tiles;
+    return (int)((per + 15) / 16 * 16);
+}
+
+// The tensor-core path takes batches above 16 of byte-coded layers whose row count is a multiple of 128.
+bool tc_eligible(const higgs_desc& d, int64_t B) {
+    return B > 16 && d.N % 128 == 0 && d.N > 0 && format_of(d.p, d.n) == Format::kByteLut;
+}
+
+size_t tc_workspace_bytes(const higgs_desc& d, int64_t B) {
+    const int BN = tc_batch_tile(B);
+    const int64_t tiles = (B + BN - 1) / BN;
+    return (size_t)tiles * BN * d.K * 2;
+}
+
+int launch_linear_tc(const higgs_desc& d, const void* x, int64_t B, const void* packed, const void* scales,
+                     const float* grid, void* y, int y_mode, __half* xdag_tc, cudaStream_t st) {
+    const int BN = tc_batch_tile(B);
+    const int64_t tiles = (B + BN - 1) / BN;
+    const int64_t warps = B * (d.K / kGroup);
+    cudaError_t e = launch_pdl(rht_activations_tc_kernel, dim3((unsigned)((warps + 7) / 8)), dim3(256), 0, st,
+                               static_cast<const __nv_bfloat16*>(x), xdag_tc, B, d.K, d.rht_seed, BN);
+    if (e != cudaSuccess) return HIGGS_ERR_CUDA;
+    static bool configured[64] = {false};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        if (cudaFuncSetAttribute(linear_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem) != cudaSuccess)
+            return HIGGS_ERR_CUDA;
+        configured[dev] = true;
+    }
+    TcParams prm;
+    prm.packed = static_cast<const uint8_t*>(packed);
+    prm.scales = static_cast<const __half*>(scales);
+    prm.grid = grid;
+    prm.xdag = xdag_tc;
+    prm.y = y;
+    prm.N = d.N; prm.K = d.K;
+    prm.B = (int)B; prm.BN = BN; prm.n = d.n; prm.p = d.p; prm.y_mode = y_mode;
+    return cuda_status(launch_pdl(linear_tc_kernel, dim3((unsigned)(d.N / 128), (unsigned)tiles), dim3(kTcThreads), kTcSmem, st, prm));
+}
+
+int read_tc_status(int clear) {
+    int v = 0;
+    if (cudaMemcpyFromSymbol(&v, g_tc_status, sizeof(int)) != cudaSuccess) return HIGGS_ERR_CUDA;
+    if (clear && v != 0) {
+        const int zero = 0;
+        if (cudaMemcpyToSymbol(g_tc_status, &zero, sizeof(int)) != cudaSuccess) return HIGGS_ERR_CUDA;
+    }
+    return v;
+}
+
+}  // namespace higgs

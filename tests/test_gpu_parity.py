@@ -208,3 +208,25 @@ def test_make_grid_is_a_lloyd_fixed_point_at_the_oracle_mse(p, n):
     fresh = inputs.gaussian_samples(p, 777, log2_count=20)
     m_dev, m_ref = oracle.grid_mse(g, fresh), oracle.grid_mse(ref.grid, fresh)
     assert abs(m_dev - m_ref) <= 0.01 * m_ref
+
+
+# ----------------------------------------------------------------------------- tensor-core path (B > 16, N % 128 == 0)
+@pytest.mark.parametrize("p,n,N,K,B", [
+    (2, 256, 128, 1024, 17),     # smallest tile: one block, 16 stages, token tile of 32
+    (2, 256, 256, 2048, 64),
+    (2, 256, 384, 4096, 100),    # ragged batch (token tile 112)
+    (1, 16, 128, 2048, 48),
+    (2, 256, 128, 8192, 256),    # full 256-token tile, long K
+    (2, 256, 256, 1024, 300),    # two token tiles
+])
+def test_linear_tensor_core_path_matches_oracle(p, n, N, K, B):
+    y, y_ref = run_linear_case(p, n, N, K, B, xi=inputs.rht_seed(3), wseed=300 + N, xseed=400 + B, lognormal=(B == 64))
+    assert y.shape == (B, N)
+    err = U.linear_error(y.cpu().numpy(), y_ref)
+    assert err <= Y_TOL, err
+
+
+def test_linear_tensor_core_path_bf16_output():
+    y, y_ref = run_linear_case(2, 256, 128, 2048, 32, xi=5, wseed=9, xseed=10, out_dtype=torch.bfloat16)
+    assert y.dtype == torch.bfloat16
+    assert U.linear_error(y.float().cpu().numpy(), y_ref) <= Y_TOL + 2.0 ** -8
