@@ -249,6 +249,7 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     if (lane == 0 && !flusher) {
         for (int d = 0; d < kMaxDepth; ++d) mbar_init(full_bar(d), 1);
     }
+    __syncwarp();
     if (flusher) {
         mbar_init(item_bars + 8u * lane, (uint32_t)NS);
         recycled[lane] = 0;
@@ -267,17 +268,23 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     const __half* ssrc_next = prm.scales + (rt_first * groups + chunk_begin * ng + gl) * 16;
     const int64_t src_stride = (int64_t)PG * (SIX ? prm.K * 6 : prm.K * 8);
     const int64_t ssrc_stride = (int64_t)PG * groups * 16;
-    auto issue = [&](int d) {   // lane 0: start the copies of the next task into slot d
+    uint32_t elected;
+    asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(elected));
+    auto issue = [&](int d) {   // whole warp: start the copies of the next task into slot d (elected lane issues)
         const uint32_t dst = slot_addr(d), bar = full_bar(d);
-        mbar_expect_tx(bar, Codes::kBytes + 32u);
-        bulk_load(dst, src_next, Codes::kBytes, bar);
-        bulk_load(dst + Codes::kBytes, ssrc_next, 32u, bar);
+        if (elected) {
+            mbar_expect_tx(bar, Codes::kBytes + 32u);
+            bulk_load(dst, src_next, Codes::kBytes, bar);
+            bulk_load(dst + Codes::kBytes, ssrc_next, 32u, bar);
+        }
         src_next += src_stride;
         ssrc_next += ssrc_stride;
     };
     // the weight stream depends on nothing this kernel computes: start it before anything else
+    // (every lane runs the loop so that addresses stay warp-uniform - bulk copies take uniform operands - and one
+    // elected lane issues)
     int issued = 0;
-    if (lane == 0 && !flusher) {
+    if (!flusher) {
         for (; issued < n_tasks && issued < D; ++issued) issue(issued);
     }
 
@@ -429,7 +436,7 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
         asm volatile("ld.shared.u16 %0, [%1];" : "=h"(shi16) : "r"(slot + Codes::kBytes + (uint32_t)g * 2u + 16u));
         __syncwarp();
         ++done;
-        if (lane == 0 && issued < n_tasks) {     // the slot's words are in registers: re-arm it for task i + D
+        if (issued < n_tasks) {                  // the slot's words are in registers: re-arm it for task i + D
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             issue(d);
             ++issued;

@@ -3,8 +3,9 @@
 // Here the path is a dense contraction, so it runs as tcgen05.mma with the accumulator in tensor memory (TMEM).
 //
 // One block computes a 128-row x BN-token tile of y over all of K ("swap-AB": the weights are the M = 128 side).
-//   producer lane    streams, per 64-input stage, the codes of the 128 rows (8 bulk copies of 512 B) and the BN x 64
-//                    tile of rotated activations (one bulk copy) into shared memory (TMA, cp.async.bulk + mbarrier);
+//   producer lanes   stream, per 64-input stage, the codes of the 128 rows (8 bulk copies of 512 B, a deep ring: they
+//                    are the HBM stream) and the BN x 64 tile of rotated activations (one bulk copy, from L2) into
+//                    shared memory (TMA, cp.async.bulk + mbarrier);
 //   16 dequant warps each thread owns one row of the tile: it turns the row's 32 code bytes of the stage into table
 //                    lookups (fp16 pairs), multiplies by the row's group scale and writes them with tcgen05.st
 //                    straight into the TMEM columns the MMA reads as its A operand - dequantisation is fused into
@@ -20,6 +21,13 @@ namespace higgs {
 
 __device__ int g_tc_status = 0;
 
+#ifdef HIGGS_TRACE
+__device__ long long g_tc_trace[4][256];
+#define TTRACE(row_, slot_) do { if (blockIdx.x == 3 && blockIdx.y == 0 && (threadIdx.x & 31) == 0 && (slot_) < 256) g_tc_trace[row_][slot_] = clock64(); } while (0)
+#else
+#define TTRACE(row_, slot_) do { } while (0)
+#endif
+
 namespace {
 
 struct TcParams {
@@ -33,9 +41,12 @@ struct TcParams {
 };
 
 constexpr uint32_t kTcSmem = 232448;
-constexpr int kTcStages = 4;
-constexpr int kTcDequantWarps = 16;
-constexpr int kTcThreads = (2 + kTcDequantWarps) * 32;
+constexpr int kTcGroups = 4;                 // dequant warp groups (4 warps each, one per TMEM lane quadrant)
+constexpr int kTcAStages = 8;                // A-operand stages in TMEM (32 columns each)
+constexpr int kTcBStages = 3;                // activation-tile stages in shared memory (at most 32 KB each)
+constexpr int kTcMaxCodeStages = 14;         // code stages in shared memory (4 KB each)
+constexpr int kTcDequantWarps = 4 * kTcGroups;
+constexpr int kTcThreads = (3 + kTcDequantWarps) * 32;
 constexpr uint32_t kTcCodeStage = 4096;      // 128 rows x 64 inputs, one byte per input pair
 constexpr uint32_t kTcWait = 1u << 22;
 constexpr uint32_t kTcACol = 256;            // TMEM columns [0, BN) accumulator, [256, 256 + 32*stages) A operand
@@ -125,22 +136,28 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
 
     // ---- shared memory map ----
     //   [base, base+2 KB)    mbarriers, TMEM base address, abort flag
-    //   [base+2 KB, lut)     code stages (4 x 4 KB) and activation stage 3
+    //   [base+2 KB, lut)     code stages (CS x 4 KB): deep, because the codes are the HBM stream
     //   [lut, lut+64 KB)     lookup table, 256-byte rows (bytes 0..127 = the entry replicated per lane)
-    //   [lut+64 KB, end)     activation stages 0..2 (BN x 128 B each, at most 32 KB)
+    //   [lut+64 KB, end)     activation-tile stages (3 x at most 32 KB; they come from L2)
+    // Three rings: codes (freed when the four dequant warps of a stage have read them), activation tiles and the
+    // A operand in TMEM (both freed by tcgen05.commit when the stage's MMAs are done).
     const uint32_t base = (uint32_t)__cvta_generic_to_shared(smem_raw);
     const uint32_t lut = (base + 2048u + 0xffffu) & ~0xffffu;
     const uint32_t bars = base;
-    auto load_full = [&](int s) { return bars + 8u * (uint32_t)s; };
-    auto a_full = [&](int s) { return bars + 8u * (uint32_t)(kTcStages + s); };
-    auto mma_done = [&](int s) { return bars + 8u * (uint32_t)(2 * kTcStages + s); };
-    const uint32_t d_full = bars + 8u * (uint32_t)(3 * kTcStages);
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_raw + 256);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + 264);
-    const uint32_t code0 = base + 2048u;                                   // 16 KB of code stages
-    const uint32_t bstage3 = (code0 + kTcStages * kTcCodeStage + 1023u) & ~1023u;
+    auto code_full = [&](int s) { return bars + 8u * (uint32_t)s; };
+    auto code_empty = [&](int s) { return bars + 8u * (uint32_t)(16 + s); };
+    auto b_full = [&](int s) { return bars + 8u * (uint32_t)(32 + s); };
+    auto b_free = [&](int s) { return bars + 8u * (uint32_t)(36 + s); };
+    auto a_full = [&](int s) { return bars + 8u * (uint32_t)(40 + s); };
+    auto a_free = [&](int s) { return bars + 8u * (uint32_t)(48 + s); };
+    const uint32_t d_full = bars + 8u * 56u;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_raw + 1024);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + 1032);
+    const uint32_t code0 = base + 2048u;
+    int CS = (int)((lut - code0) / kTcCodeStage);
+    if (CS > kTcMaxCodeStages) CS = kTcMaxCodeStages;
     auto code_stage = [&](int s) { return code0 + (uint32_t)s * kTcCodeStage; };
-    auto b_stage = [&](int s) { return s < 3 ? lut + 65536u + (uint32_t)s * 32768u : bstage3; };
+    auto b_stage = [&](int s) { return lut + 65536u + (uint32_t)s * 32768u; };
 
     const int BN = prm.BN;
     const int ksteps = (int)(prm.K / 64);
@@ -150,18 +167,20 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
 
     // ---- prologue ----
     if (tid == 0) {
-        for (int s = 0; s < kTcStages; ++s) { t_mbar_init(load_full(s), 1); t_mbar_init(a_full(s), 4); t_mbar_init(mma_done(s), 1); }
+        for (int s = 0; s < 16; ++s) { t_mbar_init(code_full(s), 1); t_mbar_init(code_empty(s), 4); }
+        for (int s = 0; s < 4; ++s) { t_mbar_init(b_full(s), 1); t_mbar_init(b_free(s), 1); }
+        for (int s = 0; s < kTcAStages; ++s) { t_mbar_init(a_full(s), 4); t_mbar_init(a_free(s), 1); }
         t_mbar_init(d_full, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) {   // one warp allocates all 512 TMEM columns (one block per SM, so nobody else wants them)
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + 256u), "r"(512u) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + 1024u), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     pdl_trigger();
-    {   // lookup table: warp w fills rows w, w+18, ...; the grid is a constant of the layer
+    {   // lookup table: warp w fills rows w, w+19, ...; the grid is a constant of the layer
         constexpr int kW = kTcThreads / 32;
         constexpr int kRows = (256 + kW - 1) / kW;
         uint32_t ent[kRows];
@@ -187,57 +206,86 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
             if (idx < 256) *reinterpret_cast<uint32_t*>(smem_raw + (lut - base) + idx * 256 + lane * 4) = ent[r];
         }
     }
-    pdl_wait();            // the rotated activations are the previous kernel's output
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
     if (warp == 0) {
-        // =============================== producer ===============================
-        if (lane == 0) {
-            int issued = 0;
-            for (int j = 0; j < ksteps; ++j) {
-                const int s = j & (kTcStages - 1), it = j / kTcStages;
-                if (it >= 1 && !t_wait(mma_done(s), (uint32_t)((it - 1) & 1), abort_flag)) break;
-                t_mbar_expect_tx(load_full(s), kTcCodeStage + b_bytes);
+        // =============================== code producer (weights: no dependency on earlier kernels) ===============
+        // (whole warp in the loop, one elected lane issues: bulk copies take warp-uniform operands)
+        uint32_t elected;
+        asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(elected));
+        int issued = 0;
+        const uint8_t* src0 = prm.packed + (row0 / 16) * (prm.K / 64) * 512;
+        const int64_t tile_stride = (prm.K / 64) * 512;            // bytes between consecutive 16-row tiles
+        for (int j = 0; j < ksteps; ++j) {
+            const int s = j % CS, it = j / CS;
+            if (it >= 1 && !t_wait(code_empty(s), (uint32_t)((it - 1) & 1), abort_flag)) break;
+            if (elected) {
+                t_mbar_expect_tx(code_full(s), kTcCodeStage);
 #pragma unroll
                 for (int rtl = 0; rtl < 8; ++rtl)
-                    t_bulk_load(code_stage(s) + rtl * 512, prm.packed + ((row0 / 16 + rtl) * (prm.K / 64) + j) * 512, 512u,
-                                load_full(s));
-                t_bulk_load(b_stage(s), prm.xdag + ((int64_t)bt * ksteps + j) * BN * 64, b_bytes, load_full(s));
-                ++issued;
+                    t_bulk_load(code_stage(s) + rtl * 512, src0 + rtl * tile_stride + (int64_t)j * 512, 512u, code_full(s));
             }
-            // never leave with copies in flight: wait (bounded) for the last stages issued
-            const int first = issued > kTcStages ? issued - kTcStages : 0;
-            for (int j = first; j < issued; ++j) {
-                const int s = j & (kTcStages - 1);
-                for (uint32_t it = 0; it < kTcWait && !t_mbar_try(load_full(s), (uint32_t)((j / kTcStages) & 1)); ++it) {}
-            }
+            ++issued;
+            __syncwarp();
         }
+        // never leave with copies in flight: wait (bounded) for the last stages issued
+        for (int j = issued > CS ? issued - CS : 0; j < issued; ++j)
+            for (uint32_t it = 0; it < kTcWait && !t_mbar_try(code_full(j % CS), (uint32_t)((j / CS) & 1)); ++it) {}
+    } else if (warp == 2) {
+        // =============================== activation-tile producer ===============================
+        uint32_t elected;
+        asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(elected));
+        pdl_wait();            // the rotated activations are the previous kernel's output
+        int issued = 0;
+        const __half* xsrc = prm.xdag + (int64_t)bt * ksteps * BN * 64;
+        for (int j = 0; j < ksteps; ++j) {
+            const int s = j % kTcBStages, it = j / kTcBStages;
+            if (it >= 1 && !t_wait(b_free(s), (uint32_t)((it - 1) & 1), abort_flag)) break;
+            if (elected) {
+                t_mbar_expect_tx(b_full(s), b_bytes);
+                t_bulk_load(b_stage(s), xsrc + (int64_t)j * BN * 64, b_bytes, b_full(s));
+            }
+            ++issued;
+            __syncwarp();
+        }
+        for (int j = issued > kTcBStages ? issued - kTcBStages : 0; j < issued; ++j)
+            for (uint32_t it = 0; it < kTcWait && !t_mbar_try(b_full(j % kTcBStages), (uint32_t)((j / kTcBStages) & 1)); ++it) {}
     } else if (warp == 1) {
         // =============================== MMA issuer ===============================
-        if (lane == 0) {
-            const uint32_t idesc = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | (8u << 24);   // f32 accumulate, f16 x f16, K-major, M=128
-            bool ok = true;
-            for (int j = 0; j < ksteps && ok; ++j) {
-                const int s = j & (kTcStages - 1), it = j / kTcStages;
-                ok = t_wait(load_full(s), (uint32_t)(it & 1), abort_flag) && t_wait(a_full(s), (uint32_t)(it & 1), abort_flag);
-                if (!ok) break;
-                tc_fence_after();
+        // The whole warp runs the loop so that addresses and descriptors stay warp-uniform (tcgen05.mma takes its
+        // operands from uniform registers); one elected lane issues.
+        const uint32_t idesc = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | (8u << 24);   // f32 accumulate, f16 x f16, K-major, M=128
+        uint32_t elected;
+        asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(elected));
+        for (int j = 0; j < ksteps; ++j) {
+            const int sb = j % kTcBStages, sa = j % kTcAStages;
+            TTRACE(1, 3 * j);
+            if (!t_wait(b_full(sb), (uint32_t)((j / kTcBStages) & 1), abort_flag)) break;
+            TTRACE(1, 3 * j + 1);
+            if (!t_wait(a_full(sa), (uint32_t)((j / kTcAStages) & 1), abort_flag)) break;
+            TTRACE(1, 3 * j + 2);
+            tc_fence_after();
+            if (elected) {
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
-                    tc_mma(tmem, tmem + kTcACol + 32u * s + 8u * c, smem_desc(b_stage(s) + 256u * c, 128u, 1024u), idesc,
+                    tc_mma(tmem, tmem + kTcACol + 32u * sa + 8u * c, smem_desc(b_stage(sb) + 256u * c, 128u, 1024u), idesc,
                            (uint32_t)((j | c) != 0));
-                tc_commit(mma_done(s));       // frees the stage (shared memory and the A columns) when these MMAs are done
+                TTRACE(2, 2 * j);
+                tc_commit(a_free(sa));        // both arrive when the MMAs issued so far are done
+                tc_commit(b_free(sb));
+                TTRACE(2, 2 * j + 1);
             }
-            tc_commit(d_full);                // all MMAs issued so far are done -> the accumulator is final
+            __syncwarp();
         }
+        if (elected) tc_commit(d_full);       // -> the accumulator is final
     } else {
         // =============================== dequant warps (then epilogue) ===============================
         // A warp may touch only the TMEM lanes 32 (warp % 4) .. +31; the four warps sharing a quadrant take the
         // stages s = 0..3 in turn (warp group sg works on ring slot sg).
-        const int q = warp & 3, sg = (warp - 2) >> 2;
+        const int q = warp & 3, sg = (warp - 3) >> 2;
         const int i = 32 * q + lane;               // row of the tile = TMEM lane
         const int rtl = i >> 4, g = i & 7, h = (i >> 3) & 1;
         const uint32_t lut_lane = lut + lane * 4;
@@ -249,10 +297,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
         int cur_group = -1;
         uint32_t sc2 = 0;
         bool ok = true;
-        for (int j = sg; j < ksteps; j += kTcStages) {
-            const int s = sg, it = j / kTcStages;
-            if (it >= 1 && !t_wait(mma_done(s), (uint32_t)((it - 1) & 1), abort_flag)) { ok = false; break; }
-            if (!t_wait(load_full(s), (uint32_t)(it & 1), abort_flag)) { ok = false; break; }
+        for (int j = sg; j < ksteps; j += kTcGroups) {
+            const int sa = j % kTcAStages, ua = j / kTcAStages, cs = j % CS;
+            if (warp == 3) TTRACE(0, 4 * (j / kTcGroups));
+            if (!t_wait(code_full(cs), (uint32_t)((j / CS) & 1), abort_flag)) { ok = false; break; }
+            if (warp == 3) TTRACE(0, 4 * (j / kTcGroups) + 1);
             if ((j >> 4) != cur_group) {           // new group of 1024 inputs: this row's scale
                 cur_group = j >> 4;
                 const __half sc = sc_row[cur_group * 16];
@@ -264,7 +313,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
             uint4 c4[4];
 #pragma unroll
             for (int jj = 0; jj < 4; ++jj)
-                c4[jj] = t_lds128(code_stage(s) + (uint32_t)(rtl * 512 + (g * 4 + ((jj + rot) & 3)) * 16));
+                c4[jj] = t_lds128(code_stage(cs) + (uint32_t)(rtl * 512 + (g * 4 + ((jj + rot) & 3)) * 16));
+            __syncwarp();
+            if (lane == 0) t_mbar_arrive(code_empty(cs));     // the code words are in registers: hand the stage back
             // undo the rotation: chunk t was loaded by instruction (t - rot) & 3
             if (rot & 1) { const uint4 t0 = c4[0]; c4[0] = c4[3]; c4[3] = c4[2]; c4[2] = c4[1]; c4[1] = t0; }
             if (rot & 2) { uint4 t0 = c4[0]; c4[0] = c4[2]; c4[2] = t0; t0 = c4[1]; c4[1] = c4[3]; c4[3] = t0; }
@@ -283,11 +334,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
                     a[m * 8 + 4 + t] = *reinterpret_cast<const uint32_t*>(&p1);
                 }
             }
-            tc_st32(t_lane + kTcACol + 32u * s, a);          // columns 8m + jj of the stage = input pair 8m + jj
+            // the A stage must have been consumed by the MMAs that used it last
+            if (warp == 3 && a[31] != 0x12345u) TTRACE(0, 4 * (j / kTcGroups) + 2);
+            if (ua >= 1 && !t_wait(a_free(sa), (uint32_t)((ua - 1) & 1), abort_flag)) { ok = false; break; }
+            if (warp == 3) TTRACE(0, 4 * (j / kTcGroups) + 3);
+            tc_fence_after();
+            tc_st32(t_lane + kTcACol + 32u * sa, a);         // columns 8m + jj of the stage = input pair 8m + jj
             asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) t_mbar_arrive(a_full(s));
+            if (lane == 0) t_mbar_arrive(a_full(sa));
         }
         if (sg == 0 && ok) {
             // epilogue: accumulator row i, 32 token columns at a time
@@ -411,6 +467,10 @@ int launch_linear_tc(const higgs_desc& d, const void* x, int64_t B, const void* 
     prm.B = (int)B; prm.BN = BN; prm.n = d.n; prm.p = d.p; prm.y_mode = y_mode;
     return cuda_status(launch_pdl(linear_tc_kernel, dim3((unsigned)(d.N / 128), (unsigned)tiles), dim3(kTcThreads), kTcSmem, st, prm));
 }
+
+#ifdef HIGGS_TRACE
+extern "C" int higgs_tc_trace_read(long long* out) { return (int)cudaMemcpyFromSymbol(out, g_tc_trace, sizeof(long long) * 4 * 256); }
+#endif
 
 int read_tc_status(int clear) {
     int v = 0;
