@@ -61,13 +61,14 @@ def algorithmic_bytes(N, K, p, n, B):
 
 
 def measured_peaks():
+    """(HBM GB/s, dense 16-bit tensor TFLOP/s burst, source) from the generated file, else the stated fallback."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
         with open(path) as f:
             d = json.load(f)
-        return float(d["hbm_gbs"]), "measured"
+        return float(d["hbm_gbs"]), float(d["bf16_tflops"]), "measured"
     except Exception:
-        return 6650.0, "fallback"
+        return 6650.0, 1590.0, "fallback"
 
 
 def max_over_ranks(ms: float, device, world: int) -> float:
@@ -252,13 +253,16 @@ def run_ours(args):
     share = {"q": "attn", "k": "attn", "v": "attn", "gate": "mlp", "up": "mlp"}
     groups_of = {}
     for li, nm in enumerate(names):
-        split = hb.higgs_linear_k_splits(descs[li], B) > 1
-        key = share.get(nm) if not split else None
+        tiled = hb.higgs_rotated_layout(descs[li], B) > 0          # tensor-core path: never split
+        split = (not tiled) and hb.higgs_linear_k_splits(descs[li], B) > 1
+        key = (share.get(nm) + f":{hb.higgs_rotated_layout(descs[li], B)}") if (share.get(nm) and not split) else None
         groups_of.setdefault(key if key else f"own{li}", []).append(li)
-    xdags = {k: torch.empty((B, descs[v[0]].K), dtype=torch.float16, device=dev) for k, v in groups_of.items() if len(v) > 1}
+    xdags = {k: torch.empty(hb.higgs_rotated_bytes(descs[v[0]], B) // 2, dtype=torch.float16, device=dev)
+             for k, v in groups_of.items() if len(v) > 1}
     launches_per_step = 0
     for k, v in groups_of.items():
-        launches_per_step += (1 + len(v) * ((B + 15) // 16)) if len(v) > 1 else hb.higgs_linear_launch_count(descs[v[0]], B)
+        launches_per_step += (1 + sum(hb.higgs_linear_launch_count(descs[li], B) - 1 for li in v)) if len(v) > 1 \
+            else hb.higgs_linear_launch_count(descs[v[0]], B)
 
     def step(i):
         c = i % copies
@@ -266,7 +270,8 @@ def run_ours(args):
             if len(lis) > 1:
                 hb.higgs_rotate_activations(descs[lis[0]], xs[lis[0]], out=xdags[key])
                 for li in lis:
-                    hb.higgs_linear_prerotated(descs[li], xdags[key], packed[li][c], scales[li][c], grid, workspace=ws[li], y=ys[li])
+                    hb.higgs_linear_prerotated(descs[li], xdags[key], packed[li][c], scales[li][c], grid, workspace=ws[li],
+                                               y=ys[li], B=B)
             else:
                 li = lis[0]
                 hb.higgs_linear(descs[li], xs[li], packed[li][c], scales[li][c], grid, workspace=ws[li], y=ys[li])
@@ -332,7 +337,7 @@ def run_ours(args):
     d2h = sum(B * N * 4 for _, N, _ in layers)
 
     # ---- dominant kernel: the product kernel on the largest layer, timed alone with CUDA events
-    peak, peak_src = measured_peaks()
+    peak, peak_tf, peak_src = measured_peaks()
     big = max(range(len(layers)), key=lambda i: layers[i][1] * layers[i][2])
     _, Nb, Kb = layers[big]
     db = descs[big]
@@ -352,11 +357,11 @@ def run_ours(args):
             scs.append(scs[0].clone())
         with torch.cuda.stream(stream):
             g = torch.cuda.CUDAGraph()
-            hb.higgs_linear_prerotated(d, xdag, pks[0], scs[0], grid, workspace=wk, y=yk)
+            hb.higgs_linear_prerotated(d, xdag, pks[0], scs[0], grid, workspace=wk, y=yk, B=Bk)
             stream.synchronize()
             with torch.cuda.graph(g, stream=stream):
                 for c in range(len(pks)):
-                    hb.higgs_linear_prerotated(d, xdag, pks[c], scs[c], grid, workspace=wk, y=yk)
+                    hb.higgs_linear_prerotated(d, xdag, pks[c], scs[c], grid, workspace=wk, y=yk, B=Bk)
             rounds = max(1, reps // len(pks))
             for _ in range(2):
                 g.replay()
@@ -381,10 +386,20 @@ def run_ours(args):
                 traffic = json.load(f).get(f"{args.workload}:{layers[big][0]}:p{p}n{n}:B{B}")
         except Exception:
             traffic = None
-    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": traffic, "peak_source": f"of {peak_src}", "kernel": "linear_mma_kernel",
-                "layer": f"{layers[big][0]} {Nb}x{Kb}", "us_per_launch": us_big, "algorithmic_bytes": alg,
-                "frac_of_8TBps": achieved / 8000.0}
+    tiled_big = hb.higgs_rotated_layout(db, B) > 0
+    kname = "linear_tc_kernel" if tiled_big else "linear_stream_kernel"
+    if B >= 64 and tiled_big:
+        # dense-contraction regime: tensor roofline (fp16 operands; nominal fp16 peak = bf16 peak)
+        tf = 2.0 * B * Nb * Kb / (us_big * 1e-6) / 1e12
+        roofline = {"bound": "tensor", "achieved": tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": tf / peak_tf,
+                    "traffic": traffic, "peak_source": f"of {peak_src} (cuBLAS bf16 burst)", "kernel": kname,
+                    "layer": f"{layers[big][0]} {Nb}x{Kb}", "us_per_launch": us_big, "flops": 2.0 * B * Nb * Kb,
+                    "weight_GBps": layer_bytes(Nb, Kb, p, n) / us_big / 1e3}
+    else:
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                    "traffic": traffic, "peak_source": f"of {peak_src}", "kernel": kname,
+                    "layer": f"{layers[big][0]} {Nb}x{Kb}", "us_per_launch": us_big, "algorithmic_bytes": alg,
+                    "frac_of_8TBps": achieved / 8000.0}
 
     detail = None
     if not args.no_detail and rank == 0:
@@ -435,7 +450,7 @@ def run_ours(args):
                        "global_batch": B * world, "parallelism": f"replicas x{world}",
                        "l2": f"rotating {copies} weight copies ({copies * set_bytes / 1e6:.0f} MB > 126 MB L2)",
                        "launch": "direct" if graphs is None else "one CUDA graph per weight copy",
-                       "step": "one transformer block: 4 activation rotations (q/k/v and gate/up share theirs) + 7 products"},
+                       "step": "one transformer block: activation rotations (q/k/v and gate/up share theirs where the layout allows) + 7 products"},
             "us_per_layer": ms_per_step * 1e3 / len(layers),
             "weight_bytes_per_step": set_bytes,
             "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

@@ -163,13 +163,19 @@ int higgs_linear(const higgs_desc* desc, const void* x, int64_t B,
 /*
  * The two halves of higgs_linear as separate calls (Section 4.3: the Hadamard
  * transform "can be fully isolated from the matrix multiplication itself").
- *   higgs_rotate_activations: x (device [B][K] bf16) -> xdag_out (device [B][K]
- *     fp16) = (H / sqrt(g)) diag(sign) x per K-group.
+ *   higgs_rotate_activations: x (device [B][K] bf16) -> xdag_out (device,
+ *     higgs_rotated_bytes(desc, B) bytes of fp16) = (H / sqrt(g)) diag(sign) x
+ *     per K-group.  The storage order is higgs_rotated_layout(desc, B): 0 = row
+ *     major [B][K] (B <= 16, or layers the tensor-core path does not take),
+ *     t > 0 = blocked operand tiles of t tokens for the tensor-core path.
  *   higgs_linear_prerotated: the product of Appendix F on already rotated
- *     activations xdag (device [B][K] fp16); other arguments as higgs_linear.
+ *     activations; other arguments as higgs_linear.  xdag may be shared by
+ *     layers with the same K, seed and higgs_rotated_layout (e.g. q, k, v).
  * higgs_linear(x) == higgs_linear_prerotated(higgs_rotate_activations(x)).
  */
 int higgs_rotate_activations(const higgs_desc* desc, const void* x, int64_t B, void* xdag_out, void* stream);
+size_t higgs_rotated_bytes(const higgs_desc* desc, int64_t B);
+int higgs_rotated_layout(const higgs_desc* desc, int64_t B);
 int higgs_linear_prerotated(const higgs_desc* desc, const void* xdag, int64_t B,
                             const void* packed, const void* scales, const float* grid,
                             void* y, int y_dtype,

@@ -24,7 +24,8 @@ EXPORTS = [
     "higgs_workspace_bytes", "higgs_make_grid", "higgs_quantize", "higgs_linear", "higgs_rht",
     "higgs_pack_codes", "higgs_unpack_codes", "higgs_rotate_activations", "higgs_linear_prerotated",
     "higgs_linear_host", "higgs_linear_host_workspace_bytes", "higgs_linear_launch_count", "higgs_device_status",
-    "higgs_linear_static", "higgs_linear_static_capacity", "higgs_linear_k_splits",
+    "higgs_linear_static", "higgs_linear_static_capacity", "higgs_linear_k_splits", "higgs_rotated_bytes",
+    "higgs_rotated_layout",
 ]
 
 
@@ -71,6 +72,10 @@ def _load() -> ctypes.CDLL:
     lib.higgs_linear_host.argtypes = [P, vp, i64, vp, vp, vp, vp, i32, vp, sz, vp]
     lib.higgs_linear_host_workspace_bytes.restype = sz
     lib.higgs_linear_host_workspace_bytes.argtypes = [P, i64, i32]
+    lib.higgs_rotated_bytes.restype = sz
+    lib.higgs_rotated_bytes.argtypes = [P, i64]
+    lib.higgs_rotated_layout.restype = i32
+    lib.higgs_rotated_layout.argtypes = [P, i64]
     lib.higgs_linear_k_splits.restype = i32
     lib.higgs_linear_k_splits.argtypes = [P, i64]
     lib.higgs_linear_launch_count.restype = i32
@@ -188,10 +193,12 @@ def higgs_linear(desc: higgs_desc, x: torch.Tensor, packed: torch.Tensor, scales
 
 
 def higgs_rotate_activations(desc: higgs_desc, x: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """x: cuda [B][K] bf16 -> rotated activations, cuda [B][K] fp16."""
+    """x: cuda [B][K] bf16 -> rotated activations, cuda fp16 (higgs_rotated_bytes(desc, B) bytes; row-major [B][K]
+    when higgs_rotated_layout(desc, B) == 0)."""
     assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous()
     if out is None:
-        out = torch.empty(x.shape, dtype=torch.float16, device=x.device)
+        nb = higgs_rotated_bytes(desc, x.shape[0])
+        out = torch.empty(x.shape if nb == x.numel() * 2 else (nb // 2,), dtype=torch.float16, device=x.device)
     _check(lib.higgs_rotate_activations(ctypes.byref(desc), _ptr(x), x.shape[0], _ptr(out), _stream()),
            "higgs_rotate_activations")
     return out
@@ -199,10 +206,12 @@ def higgs_rotate_activations(desc: higgs_desc, x: torch.Tensor, out: Optional[to
 
 def higgs_linear_prerotated(desc: higgs_desc, xdag: torch.Tensor, packed: torch.Tensor, scales: torch.Tensor,
                             grid: torch.Tensor, out_dtype: torch.dtype = torch.float32,
-                            workspace: Optional[torch.Tensor] = None, y: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """xdag: cuda [B][K] fp16 from higgs_rotate_activations.  Returns y [B][N]."""
+                            workspace: Optional[torch.Tensor] = None, y: Optional[torch.Tensor] = None,
+                            B: Optional[int] = None) -> torch.Tensor:
+    """xdag: cuda fp16 from higgs_rotate_activations for the same batch B (pass B when xdag is not [B][K]).
+    Returns y [B][N]."""
     assert xdag.is_cuda and xdag.dtype == torch.float16 and xdag.is_contiguous()
-    B = xdag.shape[0]
+    B = xdag.shape[0] if B is None else B
     if y is None:
         y = torch.empty((B, desc.N), dtype=out_dtype, device=xdag.device)
     if workspace is None:
@@ -261,6 +270,14 @@ def scales_from_tile_major(scales: torch.Tensor, N: int) -> torch.Tensor:
     """Inverse of scales_to_tile_major: returns [N][K/g]."""
     Gn = scales.numel() // N
     return scales.reshape(N // 16, Gn, 16).permute(0, 2, 1).reshape(N, Gn).contiguous()
+
+
+def higgs_rotated_bytes(desc: higgs_desc, B: int) -> int:
+    return int(lib.higgs_rotated_bytes(ctypes.byref(desc), int(B)))
+
+
+def higgs_rotated_layout(desc: higgs_desc, B: int) -> int:
+    return int(lib.higgs_rotated_layout(ctypes.byref(desc), int(B)))
 
 
 def higgs_linear_k_splits(desc: higgs_desc, B: int) -> int:

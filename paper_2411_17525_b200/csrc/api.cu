@@ -109,6 +109,7 @@ int higgs_rotate_activations(const higgs_desc* d, const void* x, int64_t B, void
     if (B < 0) return HIGGS_ERR_INVALID_ARG;
     if (B == 0 || d->K == 0) return HIGGS_OK;
     if (!x || !xdag_out || !aligned(x, 16) || !aligned(xdag_out, 16)) return HIGGS_ERR_INVALID_ARG;
+    if (tc_eligible(*d, B)) return launch_rht_tc(*d, x, B, static_cast<__half*>(xdag_out), as_stream(stream));
     return launch_rht_activations(*d, x, B, static_cast<__half*>(xdag_out), nullptr, 0, as_stream(stream));
 }
 
@@ -157,8 +158,10 @@ int higgs_linear(const higgs_desc* d, const void* x, int64_t B, const void* pack
     cudaStream_t st = as_stream(stream);
     if (tc_eligible(*d, B)) {
         // dense-contraction regime: rotate into the blocked operand layout, then one tcgen05 pass over the codes
-        return launch_linear_tc(*d, x, B, packed, scales, grid, y, y_dtype == HIGGS_F32 ? 0 : 1,
-                                static_cast<__half*>(workspace), st);
+        rc = launch_rht_tc(*d, x, B, static_cast<__half*>(workspace), st);
+        if (rc != HIGGS_OK) return rc;
+        return launch_linear_tc(*d, static_cast<const __half*>(workspace), B, packed, scales, grid, y,
+                                y_dtype == HIGGS_F32 ? 0 : 1, st);
     }
     __half* xdag = static_cast<__half*>(workspace);
     float* y32 = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up((size_t)B * d->K * 2, 256));
@@ -176,6 +179,9 @@ int higgs_linear_prerotated(const higgs_desc* d, const void* xdag, int64_t B, co
                             void* stream) {
     int rc = linear_args(d, B, xdag, packed, scales, grid, y, y_dtype, workspace, workspace_bytes);
     if (rc != HIGGS_OK) return rc < 0 ? HIGGS_OK : rc;
+    if (tc_eligible(*d, B))
+        return launch_linear_tc(*d, static_cast<const __half*>(xdag), B, packed, scales, grid, y,
+                                y_dtype == HIGGS_F32 ? 0 : 1, as_stream(stream));
     float* y32 = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up((size_t)B * d->K * 2, 256));
     return linear_tail(d, static_cast<const __half*>(xdag), B, packed, scales, grid, y, y_dtype, y32, false,
                        as_stream(stream));
@@ -212,6 +218,16 @@ size_t higgs_linear_host_workspace_bytes(const higgs_desc* d, int64_t B, int y_d
     const size_t inner = higgs_workspace_bytes(d, HIGGS_OP_LINEAR, B);
     if (inner == 0) return 0;
     return inner + align_up((size_t)B * d->K * 2, 256) + align_up((size_t)B * d->N * (y_dtype == HIGGS_F32 ? 4 : 2), 256);
+}
+
+size_t higgs_rotated_bytes(const higgs_desc* d, int64_t B) {
+    if (check_desc(d) != HIGGS_OK || B < 1) return 0;
+    return tc_eligible(*d, B) ? tc_workspace_bytes(*d, B) : (size_t)B * d->K * 2;
+}
+
+int higgs_rotated_layout(const higgs_desc* d, int64_t B) {
+    if (check_desc(d) != HIGGS_OK || B < 1) return -1;
+    return tc_eligible(*d, B) ? tc_batch_tile(B) : 0;
 }
 
 int higgs_linear_k_splits(const higgs_desc* d, int64_t B) {

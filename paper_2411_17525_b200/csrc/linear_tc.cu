@@ -441,14 +441,19 @@ size_t tc_workspace_bytes(const higgs_desc& d, int64_t B) {
     return (size_t)tiles * BN * d.K * 2;
 }
 
-int launch_linear_tc(const higgs_desc& d, const void* x, int64_t B, const void* packed, const void* scales,
-                     const float* grid, void* y, int y_mode, __half* xdag_tc, cudaStream_t st) {
+// D1 for the tensor-core path: rotated activations in the blocked operand layout (tc_workspace_bytes() bytes).
+int launch_rht_tc(const higgs_desc& d, const void* x, int64_t B, __half* xdag_tc, cudaStream_t st) {
+    const int BN = tc_batch_tile(B);
+    const int64_t warps = B * (d.K / kGroup);
+    return cuda_status(launch_pdl(rht_activations_tc_kernel, dim3((unsigned)((warps + 7) / 8)), dim3(256), 0, st,
+                                  static_cast<const __nv_bfloat16*>(x), xdag_tc, B, d.K, d.rht_seed, BN));
+}
+
+// D2-D5 on the tensor cores, from activations rotated by launch_rht_tc for the same B.
+int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, const void* packed, const void* scales,
+                     const float* grid, void* y, int y_mode, cudaStream_t st) {
     const int BN = tc_batch_tile(B);
     const int64_t tiles = (B + BN - 1) / BN;
-    const int64_t warps = B * (d.K / kGroup);
-    cudaError_t e = launch_pdl(rht_activations_tc_kernel, dim3((unsigned)((warps + 7) / 8)), dim3(256), 0, st,
-                               static_cast<const __nv_bfloat16*>(x), xdag_tc, B, d.K, d.rht_seed, BN);
-    if (e != cudaSuccess) return HIGGS_ERR_CUDA;
     static bool configured[64] = {false};
     int dev = 0;
     cudaGetDevice(&dev);

@@ -226,6 +226,22 @@ def test_linear_tensor_core_path_matches_oracle(p, n, N, K, B):
     assert err <= Y_TOL, err
 
 
+def test_tensor_core_rotate_then_product_equals_one_call():
+    p, n, N, K, B = 2, 256, 256, 2048, 80
+    W = inputs.make_weights(N, K, seed=77, bf16=True)
+    d = hb.make_desc(p, n, N, K, 11)
+    _, gt = U.grid32(p, n)
+    packed, scales, _ = hb.higgs_quantize(d, U.bf16_tensor(W), gt)
+    x = U.bf16_tensor(inputs.make_activations(B, K, seed=78))
+    assert hb.higgs_rotated_layout(d, B) == 80 and hb.higgs_rotated_layout(d, 16) == 0
+    y1 = hb.higgs_linear(d, x, packed, scales, gt)
+    xd = hb.higgs_rotate_activations(d, x)
+    assert xd.numel() * 2 == hb.higgs_rotated_bytes(d, B)
+    y2 = hb.higgs_linear_prerotated(d, xd, packed, scales, gt, B=B)
+    assert hb.higgs_device_status() == hb.HIGGS_OK
+    assert torch.equal(y1, y2)
+
+
 def test_linear_tensor_core_path_bf16_output():
     y, y_ref = run_linear_case(2, 256, 128, 2048, 32, xi=5, wseed=9, xseed=10, out_dtype=torch.bfloat16)
     assert y.dtype == torch.bfloat16
