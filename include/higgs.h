@@ -233,8 +233,10 @@ size_t higgs_linear_static_capacity(void);
 int higgs_device_status(void* stream, int clear);
 
 /* Number of K ranges the product kernel assigns to different thread blocks for this shape and
- * batch (1 = not split).  A split product accumulates with fp32 atomics into a cleared output;
- * higgs_linear clears it inside its rotation kernel, higgs_linear_prerotated with a memset. */
+ * batch (1 = not split).  For batches up to 16 a split product accumulates with fp32 atomics into a
+ * cleared output (higgs_linear clears it inside its rotation kernel, higgs_linear_prerotated with a
+ * memset), so its last bits depend on timing.  The tensor-core path (larger batches) sums the ranges
+ * of a tile in a fixed order inside a thread-block cluster and needs no clearing. */
 int higgs_linear_k_splits(const higgs_desc* desc, int64_t B);
 
 /* Number of kernels one higgs_linear call enqueues for this shape and batch. */

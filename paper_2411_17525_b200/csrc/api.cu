@@ -232,6 +232,7 @@ int higgs_rotated_layout(const higgs_desc* d, int64_t B) {
 
 int higgs_linear_k_splits(const higgs_desc* d, int64_t B) {
     if (check_desc(d) != HIGGS_OK || B < 1 || d->N == 0 || d->K == 0) return 0;
+    if (tc_eligible(*d, B)) return tc_k_split(*d, B);
     return linear_k_chunks(*d, B);
 }
 

@@ -140,6 +140,7 @@ int linear_k_chunks(const higgs_desc& d, int64_t B);
 bool tc_eligible(const higgs_desc& d, int64_t B);
 size_t tc_workspace_bytes(const higgs_desc& d, int64_t B);
 int tc_batch_tile(int64_t B);
+int tc_k_split(const higgs_desc& d, int64_t B);
 int launch_rht_tc(const higgs_desc& d, const void* x, int64_t B, __half* xdag_tc, cudaStream_t st);
 int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, const void* packed, const void* scales,
                      const float* grid, void* y, int y_mode, cudaStream_t st);

@@ -2,19 +2,27 @@
 // cores:  y[b][r] = sum_i scale[r][i] * sum_t < G[code[r][i][t]], x+[b][i][2t:2t+2] >  for 17 <= B tokens.
 // Here the path is a dense contraction, so it runs as tcgen05.mma with the accumulator in tensor memory (TMEM).
 //
-// One block computes a 128-row x BN-token tile of y over all of K ("swap-AB": the weights are the M = 128 side).
-//   producer lanes   stream, per 64-input stage, the codes of the 128 rows (8 bulk copies of 512 B, a deep ring: they
-//                    are the HBM stream) and the BN x 64 tile of rotated activations (one bulk copy, from L2) into
-//                    shared memory (TMA, cp.async.bulk + mbarrier);
-//   16 dequant warps each thread owns one row of the tile: it turns the row's 32 code bytes of the stage into table
-//                    lookups (fp16 pairs), multiplies by the row's group scale and writes them with tcgen05.st
+// One block computes a 128-row x BN-token tile of y over a slice of K ("swap-AB": the weights are the M = 128 side).
+//   producer warps   stream, per 64 inputs, the codes of the 128 rows (8 bulk copies of 512 B, a deep ring: they
+//                    are the HBM stream) and, per 64/128/256 inputs, the tile of rotated activations (one bulk copy,
+//                    from L2) into shared memory (TMA, cp.async.bulk + mbarrier);
+//   16 dequant warps each thread owns one row of the tile: it turns the row's 32 code bytes of a 64-input step into
+//                    table lookups (fp16 pairs), multiplies by the row's group scale and writes them with tcgen05.st
 //                    straight into the TMEM columns the MMA reads as its A operand - dequantisation is fused into
-//                    the operand load and the dequantised weights never touch shared or global memory;
-//   MMA lane         issues four tcgen05.mma (M=128, N=BN, K=16, A from TMEM, B through a shared-memory
-//                    descriptor) per stage and commits them to an mbarrier that frees the stage;
-//   epilogue         the first four dequant warps read the fp32 accumulator with tcgen05.ld and store y.
+//                    the operand load and the dequantised weights never touch shared or global memory.  The four
+//                    warp groups fill the four quarters of one 256-input A stage at the same time;
+//   MMA warp         one elected lane issues sixteen tcgen05.mma (M=128, N=BN, K=16, A from TMEM, B through a
+//                    shared-memory descriptor) per A stage - one barrier wait per 256 inputs keeps the issuing
+//                    warp's serial bookkeeping off the critical path - and commits them to the mbarriers that free
+//                    the stages;
+//   epilogue         all dequant warps read the fp32 accumulator with tcgen05.ld and store y.
+// Layers with few row tiles split K over the blocks of a thread-block cluster (grid z): every block parks its
+// partial tile in its own shared memory, and after a cluster barrier block z sums the partials of "its" token
+// columns through distributed shared memory in a fixed order and writes them - no atomics, no zeroing, and the
+// result does not depend on timing.
 // The group scale is folded into the fp16 A operand (relative rounding 2^-11, the same size as the rounding of the
-// table entry itself), so one accumulation runs over all of K.  Every wait is bounded; TMEM is always released.
+// table entry itself), so one accumulation runs over all of K.  Every mbarrier wait is bounded; TMEM is always
+// released.
 #include "common.cuh"
 
 namespace higgs {
@@ -23,9 +31,15 @@ __device__ int g_tc_status = 0;
 
 #ifdef HIGGS_TRACE
 __device__ long long g_tc_trace[4][256];
+__device__ unsigned long long g_tc_blocks[4][512];
+__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define BTRACE(row_) do { if (threadIdx.x == 96 && blockIdx.y == 0 && blockIdx.z == 0 && blockIdx.x < 512) g_tc_blocks[row_][blockIdx.x] = gtime(); } while (0)
+#define BTRACE_FIRST() do { g_tc_blocks[1][blockIdx.x] = gtime(); } while (0)
 #define TTRACE(row_, slot_) do { if (blockIdx.x == 3 && blockIdx.y == 0 && (threadIdx.x & 31) == 0 && (slot_) < 256) g_tc_trace[row_][slot_] = clock64(); } while (0)
 #else
 #define TTRACE(row_, slot_) do { } while (0)
+#define BTRACE(row_) do { } while (0)
+#define BTRACE_FIRST() do { } while (0)
 #endif
 
 namespace {
@@ -38,18 +52,21 @@ struct TcParams {
     void* y;                 // [B][N]
     int64_t N, K;
     int B, BN, n, p, y_mode; // y_mode 0: fp32, 1: bf16
+    int ksplit;              // K slices (= cluster size along z); each a multiple of 256 inputs
 };
 
 constexpr uint32_t kTcSmem = 232448;
 constexpr int kTcGroups = 4;                 // dequant warp groups (4 warps each, one per TMEM lane quadrant)
-constexpr int kTcAStages = 8;                // A-operand stages in TMEM (32 columns each)
 constexpr int kTcBStages = 3;                // activation-tile stages in shared memory (at most 32 KB each)
 constexpr int kTcMaxCodeStages = 14;         // code stages in shared memory (4 KB each)
 constexpr int kTcDequantWarps = 4 * kTcGroups;
 constexpr int kTcThreads = (3 + kTcDequantWarps) * 32;
 constexpr uint32_t kTcCodeStage = 4096;      // 128 rows x 64 inputs, one byte per input pair
 constexpr uint32_t kTcWait = 1u << 22;
-constexpr uint32_t kTcACol = 256;            // TMEM columns [0, BN) accumulator, [256, 256 + 32*stages) A operand
+// TMEM columns: [0, BN) accumulator; A stages of 128 columns (256 inputs) from column 128 (BN <= 128: three stages)
+// or 256 (two stages).
+constexpr uint32_t kTcAStageCols = 128;
+constexpr int kTcMaxSplit = 8;               // K slices = blocks per cluster (8 is the portable limit)
 
 __device__ __forceinline__ uint32_t t_lds32(uint32_t a) { uint32_t v; asm("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(a)); return v; }
 __device__ __forceinline__ uint4 t_lds128(uint32_t a) {
@@ -66,29 +83,42 @@ __device__ __forceinline__ void t_mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void t_mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("{ .reg .b64 st; mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1; }" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ uint32_t t_mbar_try(uint32_t bar, uint32_t parity) {
+// Bounded wait, 1 when the phase completed, 0 when `limit` polls ran out.  The loop lives inside one asm statement and
+// callers never branch on the result inside their main loops (they OR the failures into a flag and shrink the limit
+// of later waits to one poll): a data-dependent exit from the loop that issues tcgen05.mma or bulk copies makes
+// every such instruction several times more expensive to issue (measured: 16 -> 50 cycles per MMA).
+__device__ __forceinline__ uint32_t t_wait(uint32_t bar, uint32_t parity, uint32_t limit) {
     uint32_t ok;
-    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .u32 n;\n\tmov.u32 n, 0;\n\t"
+                 "T_WAIT_LOOP:\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "@p bra T_WAIT_DONE;\n\t"
+                 "add.u32 n, n, 1;\n\t"
+                 "setp.lt.u32 p, n, %3;\n\t"
+                 "@p bra T_WAIT_LOOP;\n\t"
+                 "setp.ne.u32 p, n, n;\n\t"
+                 "T_WAIT_DONE:\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity), "r"(limit) : "memory");
     return ok;
 }
-// Bounded wait: false when the block is aborting or this wait ran out (then it raises the abort flag and the status).
-__device__ __forceinline__ bool t_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    for (uint32_t it = 0;; ++it) {
-        if (t_mbar_try(bar, parity)) return true;
-        if ((it & 63u) == 63u) {
-            if (*abort_flag) return false;
-            if (it > kTcWait) {
-                *abort_flag = 1;
-                atomicExch(&g_tc_status, (int)HIGGS_ERR_TIMEOUT);
-                return false;
-            }
-        }
+__device__ __forceinline__ uint32_t t_limit(uint32_t bad) { return bad ? 1u : kTcWait; }
+// A role whose wait ran out reports it: the block's abort flag (read by the K-split reduction) and the status word.
+__device__ __forceinline__ void t_report(uint32_t bad, volatile int* abort_flag) {
+    if (bad) {
+        *abort_flag = 1;
+        atomicExch(&g_tc_status, (int)HIGGS_ERR_TIMEOUT);
     }
 }
 __device__ __forceinline__ void t_bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                  "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// true in exactly one lane of the (converged) warp
+__device__ __forceinline__ bool elect_one() {
+    uint32_t is_elected;
+    asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(is_elected));
+    return is_elected != 0;
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -130,6 +160,9 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         : "r"(taddr) : "memory");
 }
 
+// FB = 64-input steps per activation-tile stage (4, 2, 1 for BN <= 64, <= 128, <= 256: a stage is at most 32 KB).  It is a
+// template parameter so that the MMA warp's loop body is straight-line code.
+template <int FB>
 __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams prm) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -139,8 +172,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
     //   [base+2 KB, lut)     code stages (CS x 4 KB): deep, because the codes are the HBM stream
     //   [lut, lut+64 KB)     lookup table, 256-byte rows (bytes 0..127 = the entry replicated per lane)
     //   [lut+64 KB, end)     activation-tile stages (3 x at most 32 KB; they come from L2)
-    // Three rings: codes (freed when the four dequant warps of a stage have read them), activation tiles and the
-    // A operand in TMEM (both freed by tcgen05.commit when the stage's MMAs are done).
+    //   after the main loop, K-split only: [base+2 KB, +BN x 512 B) the block's partial tile, [token][row] fp32
+    // Three rings: codes (freed when the four dequant warps of a step have read them), activation tiles and the
+    // A operand in TMEM (both freed by tcgen05.commit when the MMAs that read them are done).
     const uint32_t base = (uint32_t)__cvta_generic_to_shared(smem_raw);
     const uint32_t lut = (base + 2048u + 0xffffu) & ~0xffffu;
     const uint32_t bars = base;
@@ -149,7 +183,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
     auto b_full = [&](int s) { return bars + 8u * (uint32_t)(32 + s); };
     auto b_free = [&](int s) { return bars + 8u * (uint32_t)(36 + s); };
     auto a_full = [&](int s) { return bars + 8u * (uint32_t)(40 + s); };
-    auto a_free = [&](int s) { return bars + 8u * (uint32_t)(48 + s); };
+    auto a_free = [&](int s) { return bars + 8u * (uint32_t)(44 + s); };
     const uint32_t d_full = bars + 8u * 56u;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_raw + 1024);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + 1032);
@@ -160,16 +194,24 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
     auto b_stage = [&](int s) { return lut + 65536u + (uint32_t)s * 32768u; };
 
     const int BN = prm.BN;
-    const int ksteps = (int)(prm.K / 64);
+    const int ksplit = prm.ksplit;
+    const int kz = blockIdx.z;                               // K slice = rank in the cluster (cluster dims 1 x 1 x ksplit)
+    const int ksteps_all = (int)(prm.K / 64);
+    const int ksteps = ksteps_all / ksplit;                  // 64-input steps of this block, a multiple of 4
+    const int kstep0 = kz * ksteps;
+    const int nsuper = ksteps >> 2;                          // A stages (256 inputs) of this block
     const int64_t row0 = (int64_t)blockIdx.x * 128;
     const int bt = blockIdx.y;
-    const uint32_t b_bytes = (uint32_t)BN * 128u;
+    const uint32_t b_step_bytes = (uint32_t)BN * 128u;
+    const int AS = BN <= 128 ? 3 : 2;                        // A stages in TMEM
+    const uint32_t acol0 = BN <= 128 ? 128u : 256u;
 
     // ---- prologue ----
+    BTRACE(0);
     if (tid == 0) {
         for (int s = 0; s < 16; ++s) { t_mbar_init(code_full(s), 1); t_mbar_init(code_empty(s), 4); }
         for (int s = 0; s < 4; ++s) { t_mbar_init(b_full(s), 1); t_mbar_init(b_free(s), 1); }
-        for (int s = 0; s < kTcAStages; ++s) { t_mbar_init(a_full(s), 4); t_mbar_init(a_free(s), 1); }
+        for (int s = 0; s < 4; ++s) { t_mbar_init(a_full(s), kTcDequantWarps); t_mbar_init(a_free(s), 1); }
         t_mbar_init(d_full, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -210,18 +252,27 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    // The code ring needs one stage per warp group; the block's shared-memory window always leaves room for more, but
+    // a window that did not would be reported, not run.
+    int role = warp;
+    if (CS < kTcGroups) {
+        if (tid == 0) { *abort_flag = 1; atomicExch(&g_tc_status, (int)HIGGS_ERR_TIMEOUT); }
+        role = -1;
+    }
 
-    if (warp == 0) {
+    if (role == 0) {
         // =============================== code producer (weights: no dependency on earlier kernels) ===============
         // (whole warp in the loop, one elected lane issues: bulk copies take warp-uniform operands)
         uint32_t elected;
         asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(elected));
         int issued = 0;
-        const uint8_t* src0 = prm.packed + (row0 / 16) * (prm.K / 64) * 512;
-        const int64_t tile_stride = (prm.K / 64) * 512;            // bytes between consecutive 16-row tiles
+        const int64_t tile_stride = (int64_t)ksteps_all * 512;     // bytes between consecutive 16-row tiles
+        const uint8_t* src0 = prm.packed + (row0 / 16) * tile_stride + (int64_t)kstep0 * 512;
+        int s = 0, it = 0;
+        uint32_t bad = 0;
         for (int j = 0; j < ksteps; ++j) {
-            const int s = j % CS, it = j / CS;
-            if (it >= 1 && !t_wait(code_empty(s), (uint32_t)((it - 1) & 1), abort_flag)) break;
+            // (the first pass waits for the phase before the first one, which counts as complete)
+            bad |= t_wait(code_empty(s), (uint32_t)((it & 1) ^ 1), t_limit(bad)) ^ 1u;
             if (elected) {
                 t_mbar_expect_tx(code_full(s), kTcCodeStage);
 #pragma unroll
@@ -229,62 +280,96 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
                     t_bulk_load(code_stage(s) + rtl * 512, src0 + rtl * tile_stride + (int64_t)j * 512, 512u, code_full(s));
             }
             ++issued;
+            const bool wrap = s + 1 == CS;
+            s = wrap ? 0 : s + 1;
+            it += wrap ? 1 : 0;
             __syncwarp();
         }
         // never leave with copies in flight: wait (bounded) for the last stages issued
         for (int j = issued > CS ? issued - CS : 0; j < issued; ++j)
-            for (uint32_t it = 0; it < kTcWait && !t_mbar_try(code_full(j % CS), (uint32_t)((j / CS) & 1)); ++it) {}
-    } else if (warp == 2) {
+            bad |= t_wait(code_full(j % CS), (uint32_t)((j / CS) & 1), t_limit(bad)) ^ 1u;
+        t_report(bad, abort_flag);
+    } else if (role == 2) {
         // =============================== activation-tile producer ===============================
         uint32_t elected;
         asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(elected));
         pdl_wait();            // the rotated activations are the previous kernel's output
         int issued = 0;
-        const __half* xsrc = prm.xdag + (int64_t)bt * ksteps * BN * 64;
-        for (int j = 0; j < ksteps; ++j) {
-            const int s = j % kTcBStages, it = j / kTcBStages;
-            if (it >= 1 && !t_wait(b_free(s), (uint32_t)((it - 1) & 1), abort_flag)) break;
+        const int nb = ksteps / FB;
+        const uint32_t bytes = b_step_bytes * (uint32_t)FB;
+        const __half* xsrc = prm.xdag + ((int64_t)bt * ksteps_all + kstep0) * BN * 64;
+        int s = 0, it = 0;
+        uint32_t bad = 0;
+        for (int t = 0; t < nb; ++t) {
+            bad |= t_wait(b_free(s), (uint32_t)((it & 1) ^ 1), t_limit(bad)) ^ 1u;
             if (elected) {
-                t_mbar_expect_tx(b_full(s), b_bytes);
-                t_bulk_load(b_stage(s), xsrc + (int64_t)j * BN * 64, b_bytes, b_full(s));
+                t_mbar_expect_tx(b_full(s), bytes);
+                t_bulk_load(b_stage(s), xsrc + (int64_t)t * FB * BN * 64, bytes, b_full(s));
             }
             ++issued;
+            const bool wrap = s + 1 == kTcBStages;
+            s = wrap ? 0 : s + 1;
+            it += wrap ? 1 : 0;
             __syncwarp();
         }
-        for (int j = issued > kTcBStages ? issued - kTcBStages : 0; j < issued; ++j)
-            for (uint32_t it = 0; it < kTcWait && !t_mbar_try(b_full(j % kTcBStages), (uint32_t)((j / kTcBStages) & 1)); ++it) {}
-    } else if (warp == 1) {
+        for (int t = issued > kTcBStages ? issued - kTcBStages : 0; t < issued; ++t)
+            bad |= t_wait(b_full(t % kTcBStages), (uint32_t)((t / kTcBStages) & 1), t_limit(bad)) ^ 1u;
+        t_report(bad, abort_flag);
+    } else if (role == 1) {
         // =============================== MMA issuer ===============================
         // The whole warp runs the loop so that addresses and descriptors stay warp-uniform (tcgen05.mma takes its
-        // operands from uniform registers); one elected lane issues.
+        // operands from uniform registers); one elected lane issues.  Per A stage (256 inputs): one wait for the
+        // sixteen dequant warps, one wait per activation-tile stage, sixteen MMAs.
         const uint32_t idesc = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | (8u << 24);   // f32 accumulate, f16 x f16, K-major, M=128
         uint32_t elected;
         asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(elected));
-        for (int j = 0; j < ksteps; ++j) {
-            const int sb = j % kTcBStages, sa = j % kTcAStages;
-            TTRACE(1, 3 * j);
-            if (!t_wait(b_full(sb), (uint32_t)((j / kTcBStages) & 1), abort_flag)) break;
-            TTRACE(1, 3 * j + 1);
-            if (!t_wait(a_full(sa), (uint32_t)((j / kTcAStages) & 1), abort_flag)) break;
-            TTRACE(1, 3 * j + 2);
+        int sa = 0, ua = 0;            // A stage and its use count
+        int sb = 0, ub = 0;            // activation-tile stage and its use count
+        uint32_t bad = 0;
+        const uint64_t b_desc0 = smem_desc(b_stage(0), 128u, 1024u);
+        for (int S = 0; S < nsuper; ++S) {
+            TTRACE(1, 3 * S);
+            bad |= t_wait(a_full(sa), (uint32_t)(ua & 1), t_limit(bad)) ^ 1u;
+            TTRACE(1, 3 * S + 1);
+            if (S == 0 && lane == 0 && blockIdx.y == 0 && blockIdx.z == 0 && blockIdx.x < 512) { BTRACE_FIRST(); }
             tc_fence_after();
-            if (elected) {
+            const uint32_t a_stage = tmem + acol0 + kTcAStageCols * (uint32_t)sa;
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    tc_mma(tmem, tmem + kTcACol + 32u * sa + 8u * c, smem_desc(b_stage(sb) + 256u * c, 128u, 1024u), idesc,
-                           (uint32_t)((j | c) != 0));
-                TTRACE(2, 2 * j);
-                tc_commit(a_free(sa));        // both arrive when the MMAs issued so far are done
-                tc_commit(b_free(sb));
-                TTRACE(2, 2 * j + 1);
+            for (int h = 0; h < 4; ++h) {
+                if (h % FB == 0) {
+                    bad |= t_wait(b_full(sb), (uint32_t)(ub & 1), t_limit(bad)) ^ 1u;
+                    tc_fence_after();
+                }
+                // addresses and descriptors are computed by the whole warp; only the instruction is issued by one lane
+                const uint32_t a_addr = a_stage + 32u * (uint32_t)h;
+                const uint64_t b_desc = b_desc0 + (uint64_t)(((uint32_t)sb * 32768u + (uint32_t)(h % FB) * b_step_bytes) >> 4);
+                const uint32_t acc = (uint32_t)((S | h) != 0);
+                if (elected) {
+                    tc_mma(tmem, a_addr, b_desc, idesc, acc);
+                    tc_mma(tmem, a_addr + 8u, b_desc + 16u, idesc, 1u);      // + 256 bytes in the address field
+                    tc_mma(tmem, a_addr + 16u, b_desc + 32u, idesc, 1u);
+                    tc_mma(tmem, a_addr + 24u, b_desc + 48u, idesc, 1u);
+                    if (h % FB == FB - 1) tc_commit(b_free(sb));      // arrives when the MMAs issued so far are done
+                }
+                if (h % FB == FB - 1) {
+                    const bool wrap = sb + 1 == kTcBStages;
+                    sb = wrap ? 0 : sb + 1;
+                    ub += wrap ? 1 : 0;
+                }
             }
+            if (elected) tc_commit(a_free(sa));
+            TTRACE(1, 3 * S + 2);
+            const bool wrap = sa + 1 == AS;
+            sa = wrap ? 0 : sa + 1;
+            ua += wrap ? 1 : 0;
             __syncwarp();
         }
         if (elected) tc_commit(d_full);       // -> the accumulator is final
-    } else {
+        t_report(bad, abort_flag);
+    } else if (role >= 3) {
         // =============================== dequant warps (then epilogue) ===============================
-        // A warp may touch only the TMEM lanes 32 (warp % 4) .. +31; the four warps sharing a quadrant take the
-        // stages s = 0..3 in turn (warp group sg works on ring slot sg).
+        // A warp may touch only the TMEM lanes 32 (warp % 4) .. +31; the four warps sharing a quadrant (warp groups
+        // sg = 0..3) take the four 64-input quarters of each A stage.
         const int q = warp & 3, sg = (warp - 3) >> 2;
         const int i = 32 * q + lane;               // row of the tile = TMEM lane
         const int rtl = i >> 4, g = i & 7, h = (i >> 3) & 1;
@@ -294,28 +379,33 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
         const int groups = (int)(prm.K / kGroup);
         const __half* sc_row = prm.scales + ((row0 / 16 + rtl) * groups) * 16 + (i & 15);
         const uint32_t t_lane = tmem + ((uint32_t)(32 * q) << 16);
+        const uint32_t code_off = (uint32_t)(rtl * 512 + g * 64);
         int cur_group = -1;
         uint32_t sc2 = 0;
-        bool ok = true;
-        for (int j = sg; j < ksteps; j += kTcGroups) {
-            const int sa = j % kTcAStages, ua = j / kTcAStages, cs = j % CS;
-            if (warp == 3) TTRACE(0, 4 * (j / kTcGroups));
-            if (!t_wait(code_full(cs), (uint32_t)((j / CS) & 1), abort_flag)) { ok = false; break; }
-            if (warp == 3) TTRACE(0, 4 * (j / kTcGroups) + 1);
-            if ((j >> 4) != cur_group) {           // new group of 1024 inputs: this row's scale
-                cur_group = j >> 4;
+        uint32_t bad = 0;
+        int sa = 0, ua = 0;
+        int cs = sg % CS, ucs = 0;                 // code stage of step 4 S + sg and its use count (CS >= 4)
+        for (int S = 0; S < nsuper; ++S) {
+            const int jg = kstep0 + 4 * S + sg;    // 64-input step of the layer
+            if (warp == 3) TTRACE(0, 4 * S);
+            bad |= t_wait(code_full(cs), (uint32_t)(ucs & 1), t_limit(bad)) ^ 1u;
+            if (warp == 3) TTRACE(0, 4 * S + 1);
+            if ((jg >> 4) != cur_group) {          // new group of 1024 inputs: this row's scale
+                cur_group = jg >> 4;
                 const __half sc = sc_row[cur_group * 16];
                 const __half2 s2 = __half2half2(sc);
                 sc2 = *reinterpret_cast<const uint32_t*>(&s2);
             }
-            // the row's codes of this stage: the 16-byte chunks of lanes (g, t = 0..3) of row tile rtl; instruction jj
+            // the row's codes of this step: the 16-byte chunks of lanes (g, t = 0..3) of row tile rtl; instruction jj
             // reads chunk (jj + rot) & 3 so that the eight g of a warp hit eight different bank groups
             uint4 c4[4];
 #pragma unroll
             for (int jj = 0; jj < 4; ++jj)
-                c4[jj] = t_lds128(code_stage(cs) + (uint32_t)(rtl * 512 + (g * 4 + ((jj + rot) & 3)) * 16));
+                c4[jj] = t_lds128(code_stage(cs) + code_off + (uint32_t)(((jj + rot) & 3) * 16));
             __syncwarp();
             if (lane == 0) t_mbar_arrive(code_empty(cs));     // the code words are in registers: hand the stage back
+            cs += 4;
+            if (cs >= CS) { cs -= CS; ++ucs; }
             // undo the rotation: chunk t was loaded by instruction (t - rot) & 3
             if (rot & 1) { const uint4 t0 = c4[0]; c4[0] = c4[3]; c4[3] = c4[2]; c4[2] = c4[1]; c4[1] = t0; }
             if (rot & 2) { uint4 t0 = c4[0]; c4[0] = c4[2]; c4[2] = t0; t0 = c4[1]; c4[1] = c4[3]; c4[3] = t0; }
@@ -335,22 +425,29 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
                 }
             }
             // the A stage must have been consumed by the MMAs that used it last
-            if (warp == 3 && a[31] != 0x12345u) TTRACE(0, 4 * (j / kTcGroups) + 2);
-            if (ua >= 1 && !t_wait(a_free(sa), (uint32_t)((ua - 1) & 1), abort_flag)) { ok = false; break; }
-            if (warp == 3) TTRACE(0, 4 * (j / kTcGroups) + 3);
+            if (warp == 3 && a[31] != 0x12345u) TTRACE(0, 4 * S + 2);
+            bad |= t_wait(a_free(sa), (uint32_t)((ua & 1) ^ 1), t_limit(bad)) ^ 1u;   // (first use: the phase before the first)
+            if (warp == 3) TTRACE(0, 4 * S + 3);
             tc_fence_after();
-            tc_st32(t_lane + kTcACol + 32u * sa, a);         // columns 8m + jj of the stage = input pair 8m + jj
+            tc_st32(t_lane + acol0 + kTcAStageCols * (uint32_t)sa + 32u * (uint32_t)sg, a);   // column 8m + jj = input pair 8m + jj
             asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
             tc_fence_before();
             __syncwarp();
             if (lane == 0) t_mbar_arrive(a_full(sa));
+            if (++sa == AS) { sa = 0; ++ua; }
         }
-        if (sg == 0 && ok) {
-            // epilogue: accumulator row i, 32 token columns at a time
-            if (t_wait(d_full, 0u, abort_flag)) {
-                tc_fence_after();
-                const int64_t row = row0 + i;
-                for (int c0 = 0; c0 < BN; c0 += 32) {
+        if (warp == 3) TTRACE(3, 0);
+        bad |= t_wait(d_full, 0u, t_limit(bad)) ^ 1u;
+        if (warp == 3) TTRACE(3, 1);
+        BTRACE(2);
+        t_report(bad, abort_flag);
+        if (!bad) {
+            tc_fence_after();
+            const int64_t row = row0 + i;
+            if (ksplit == 1) {
+                // epilogue: accumulator row i, 32 token columns at a time, the column chunks dealt over the warp groups
+                pdl_wait();        // y may still be read by the kernel before this one
+                for (int c0 = 32 * sg; c0 < BN; c0 += 32 * kTcGroups) {
                     uint32_t d[32];
                     tc_ld32(t_lane + (uint32_t)c0, d);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
@@ -364,15 +461,61 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
                         }
                     }
                 }
+            } else {
+                // K-split: park the partial tile in shared memory as [token][row] (all rings are idle: every MMA
+                // has completed, so every copy has landed and every lookup has been done)
+                for (int c0 = 32 * sg; c0 < BN; c0 += 32 * kTcGroups) {
+                    uint32_t d[32];
+                    tc_ld32(t_lane + (uint32_t)c0, d);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                    for (int r = 0; r < 32; ++r)
+                        if (c0 + r < BN)
+                            asm volatile("st.shared.b32 [%0], %1;" ::"r"(code0 + (uint32_t)(((c0 + r) * 128 + i) * 4)), "r"(d[r]) : "memory");
+                }
             }
         }
     }
 
     // ---- every role ends here, aborted or not: TMEM must be handed back ----
+    if (warp == 3) TTRACE(3, 2);
     tc_fence_before();
     __syncthreads();
+    if (warp == 3) TTRACE(3, 3);
+    BTRACE(3);
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+    }
+    if (ksplit > 1) {
+        // Cluster reduction in a fixed order: block kz owns the token columns [kz, kz+1) * BN / ksplit and sums the
+        // partial tiles of all blocks of the cluster for them through distributed shared memory.
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        const int cols = BN / ksplit;
+        if (tid < 512 && !*abort_flag) {
+            pdl_wait();            // y may still be read by the kernel before this one
+            const int rrow = tid & 127;
+            for (int cc = tid >> 7; cc < cols; cc += 4) {
+                const int c = kz * cols + cc;
+                const uint32_t local = code0 + (uint32_t)((c * 128 + rrow) * 4);
+                float acc = 0.f;
+                for (int r = 0; r < ksplit; ++r) {
+                    uint32_t remote;
+                    float v;
+                    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(r));
+                    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+                    acc += v;
+                }
+                const int b = bt * BN + c;
+                if (b < prm.B) {
+                    if (prm.y_mode == 0) static_cast<float*>(prm.y)[(int64_t)b * prm.N + row0 + rrow] = acc;
+                    else static_cast<__nv_bfloat16*>(prm.y)[(int64_t)b * prm.N + row0 + rrow] = __float2bfloat16_rn(acc);
+                }
+            }
+        }
+        // nobody leaves while its shared memory may still be read
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
     }
 }
 
@@ -449,6 +592,16 @@ int launch_rht_tc(const higgs_desc& d, const void* x, int64_t B, __half* xdag_tc
                                   static_cast<const __nv_bfloat16*>(x), xdag_tc, B, d.K, d.rht_seed, BN));
 }
 
+// K slices of the tensor-core product: as many (a power of two, at most 8) as keep the grid within one wave of
+// clusters, every slice a multiple of 256 inputs and at least 512.
+int tc_k_split(const higgs_desc& d, int64_t B) {
+    const int BN = tc_batch_tile(B);
+    const int64_t tiles = (d.N / 128) * ((B + BN - 1) / BN);
+    int ks = 1;
+    while (ks < kTcMaxSplit && tiles * (ks * 2) <= 128 && d.K % (256 * ks * 2) == 0 && d.K / (ks * 2) >= 512) ks *= 2;
+    return ks;
+}
+
 // D2-D5 on the tensor cores, from activations rotated by launch_rht_tc for the same B.
 int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, const void* packed, const void* scales,
                      const float* grid, void* y, int y_mode, cudaStream_t st) {
@@ -458,7 +611,9 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        if (cudaFuncSetAttribute(linear_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem) != cudaSuccess)
+        if (cudaFuncSetAttribute(linear_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem) != cudaSuccess ||
+            cudaFuncSetAttribute(linear_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem) != cudaSuccess ||
+            cudaFuncSetAttribute(linear_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem) != cudaSuccess)
             return HIGGS_ERR_CUDA;
         configured[dev] = true;
     }
@@ -470,10 +625,31 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
     prm.y = y;
     prm.N = d.N; prm.K = d.K;
     prm.B = (int)B; prm.BN = BN; prm.n = d.n; prm.p = d.p; prm.y_mode = y_mode;
-    return cuda_status(launch_pdl(linear_tc_kernel, dim3((unsigned)(d.N / 128), (unsigned)tiles), dim3(kTcThreads), kTcSmem, st, prm));
+    prm.ksplit = tc_k_split(d, B);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(d.N / 128), (unsigned)tiles, (unsigned)prm.ksplit);
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = kTcSmem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.numAttrs = 1;
+    if (prm.ksplit > 1) {      // the K slices of a tile form one thread-block cluster
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = 1;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = (unsigned)prm.ksplit;
+        cfg.numAttrs = 2;
+    }
+    cfg.attrs = attr;
+    if (BN <= 64) return cuda_status(cudaLaunchKernelEx(&cfg, linear_tc_kernel<4>, prm));
+    if (BN <= 128) return cuda_status(cudaLaunchKernelEx(&cfg, linear_tc_kernel<2>, prm));
+    return cuda_status(cudaLaunchKernelEx(&cfg, linear_tc_kernel<1>, prm));
 }
 
 #ifdef HIGGS_TRACE
+extern "C" int higgs_tc_blocks_read(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_tc_blocks, sizeof(unsigned long long) * 4 * 512); }
 extern "C" int higgs_tc_trace_read(long long* out) { return (int)cudaMemcpyFromSymbol(out, g_tc_trace, sizeof(long long) * 4 * 256); }
 #endif
 

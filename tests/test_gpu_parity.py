@@ -218,6 +218,8 @@ def test_make_grid_is_a_lloyd_fixed_point_at_the_oracle_mse(p, n):
     (1, 16, 128, 2048, 48),
     (2, 256, 128, 8192, 256),    # full 256-token tile, long K
     (2, 256, 256, 1024, 300),    # two token tiles
+    (2, 256, 8448, 1024, 40),    # 66 row tiles: K is not split
+    (2, 256, 4096, 3072, 24),    # two K slices of 1536 inputs: the boundary falls inside a scale group
 ])
 def test_linear_tensor_core_path_matches_oracle(p, n, N, K, B):
     y, y_ref = run_linear_case(p, n, N, K, B, xi=inputs.rht_seed(3), wseed=300 + N, xseed=400 + B, lognormal=(B == 64))
@@ -240,6 +242,20 @@ def test_tensor_core_rotate_then_product_equals_one_call():
     y2 = hb.higgs_linear_prerotated(d, xd, packed, scales, gt, B=B)
     assert hb.higgs_device_status() == hb.HIGGS_OK
     assert torch.equal(y1, y2)
+
+
+def test_tensor_core_k_split_is_deterministic():
+    """The K slices of a tile are summed in a fixed order inside a cluster: two runs agree bit for bit."""
+    p, n, N, K, B = 2, 256, 256, 4096, 96
+    d = hb.make_desc(p, n, N, K, 3)
+    assert hb.higgs_linear_k_splits(d, B) == 8 and hb.higgs_linear_k_splits(hb.make_desc(p, n, 16384, K, 3), B) == 1
+    W = inputs.make_weights(N, K, seed=5, bf16=True)
+    _, gt = U.grid32(p, n)
+    packed, scales, _ = hb.higgs_quantize(d, U.bf16_tensor(W), gt)
+    x = U.bf16_tensor(inputs.make_activations(B, K, seed=6))
+    ys = [hb.higgs_linear(d, x, packed, scales, gt).clone() for _ in range(3)]
+    assert hb.higgs_device_status() == hb.HIGGS_OK
+    assert torch.equal(ys[0], ys[1]) and torch.equal(ys[0], ys[2])
 
 
 def test_linear_tensor_core_path_bf16_output():
