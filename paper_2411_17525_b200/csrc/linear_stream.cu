@@ -33,9 +33,12 @@ __device__ int g_device_status = 0;
 #ifdef HIGGS_TRACE
 __device__ long long g_trace[17][64];
 __device__ __forceinline__ long long trace_now() { return clock64(); }   // SM cycles (cheap); one block only, so one clock domain
+__device__ long long g_trace_pro[17][16];
+#define TRACEP(warp_, slot_) do { if (blockIdx.x == 7 && (threadIdx.x & 31) == 0) g_trace_pro[warp_][slot_] = trace_now(); } while (0)
 #define TRACE(warp_, slot_) do { if (blockIdx.x == 7 && (threadIdx.x & 31) == 0 && (slot_) < 64) g_trace[warp_][slot_] = trace_now(); } while (0)
 #else
 #define TRACE(warp_, slot_) do { } while (0)
+#define TRACEP(warp_, slot_) do { } while (0)
 #endif
 
 namespace {
@@ -51,6 +54,15 @@ struct StreamParams {
     int B, n, p;
     int ck;                // inputs per item
     int y_mode;            // 0: store fp32, 1: store bf16, 2: atomicAdd fp32
+    // Planned on the host so that the kernel's prologue has no divisions before its first copies are in flight:
+    int parts;             // blocks per K-chunk
+    unsigned long long parts_magic;   // x / parts == (x * parts_magic) >> (32 + parts_shift) for x < 2^31
+    int parts_shift;
+    int log_ns;            // log2 of NS = ck / KS (slices per item)
+    int tile_pieces;       // 128-byte pieces of one partial tile
+    int acc_slots, acc_shift;   // items whose partial tiles may be parked at once (a power of two) and its log2
+    int depth, warps_in_a; // ring depth and warps whose slots lie below the table, valid when the dynamic
+                           // shared-memory window starts at offset kAssumedBase (else recomputed on the device)
 };
 
 constexpr uint32_t kLutBytes = 65536;   // 256 entries x 256-byte row (32 lanes x 4 B; upper row halves hold accumulators)
@@ -60,6 +72,20 @@ constexpr int kWarps = 16;
 constexpr int kMaxDepth = 8;            // ring slots per warp
 constexpr int kMaxAccSlots = 32;        // items whose partial tiles may be parked at once
 constexpr uint32_t kWaitLimit = 1u << 22;
+constexpr uint32_t kAssumedBase = 1024; // offset of the dynamic shared-memory window the host plans the rings for
+
+// Ring layout for a window starting at `base`: table position, depth D and the number of warps whose D slots fit
+// below the table (the others' lie above it).
+__host__ __device__ inline void ring_layout(uint32_t base, uint32_t slot_bytes, uint32_t* lut_out, int* depth_out, int* warps_in_a_out) {
+    const uint32_t lut = (base + kSmallBytes + 0xffffu) & ~0xffffu;
+    const int nA = (int)((lut - (base + kSmallBytes)) / slot_bytes);
+    const int nB = (int)((base + kMaxDynSmem - (lut + kLutBytes)) / slot_bytes);
+    int D = kMaxDepth;
+    while (D > 1 && nA / D + nB / D < kWarps) --D;
+    *lut_out = lut;
+    *depth_out = D;
+    *warps_in_a_out = nA / D;
+}
 
 // ---- PTX helpers ------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t lds32(uint32_t addr) {
@@ -197,22 +223,46 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     //   [lut, lut+64 KB)     table rows of 256 B: bytes 0..127 = the entry replicated per lane,
     //                        bytes 128..255 = one 32-float piece of an accumulator tile
     //   [lut+64 KB, end)     ring slots, region B
+    TRACEP(warp, 0);
+    // ---- the table's source first: the grid loads are in flight while everything below is set up ----
+    // Table: entry(idx) replicated once per lane (bank = lane): conflict-free gathers.  Warp w fills rows
+    // w, w+17, ...; all lanes of a warp read the same grid entry (one broadcast transaction), and the 16 loads of
+    // a warp are independent, so the whole build costs one global round trip.  (The grid is a constant of the layer.)
+    constexpr int kRowsPerWarp = (256 + kWarps) / (kWarps + 1);     // 16 rows for 17 warps (last one partly idle)
+    float ent_lo[kRowsPerWarp], ent_hi[kRowsPerWarp];
+#pragma unroll
+    for (int r = 0; r < kRowsPerWarp; ++r) {
+        const int idx = warp + r * (kWarps + 1);
+        ent_lo[r] = 0.f; ent_hi[r] = 0.f;
+        if (idx < 256) {
+            if (prm.p == 2) {
+                const float2 gp = __ldg(reinterpret_cast<const float2*>(prm.grid) + (idx & (prm.n - 1)));
+                ent_lo[r] = gp.x; ent_hi[r] = gp.y;
+            } else {
+                ent_lo[r] = __ldg(prm.grid + (idx & 15));
+                ent_hi[r] = __ldg(prm.grid + (idx >> 4));
+            }
+        }
+    }
+
+    // ---- shared memory map (all offsets derived from the runtime base address) ----
+    //   [base, base+4 KB)    ring mbarriers (0..1023), item mbarriers and
+    //                        recycle counters of the partial-tile slots (2048..2559), abort flag (2560)
+    //   [base+4 KB, lut)     ring slots, region A
+    //   [lut, lut+64 KB)     table rows of 256 B: bytes 0..127 = the entry replicated per lane,
+    //                        bytes 128..255 = one 32-float piece of an accumulator tile
+    //   [lut+64 KB, end)     ring slots, region B
     const uint32_t base = (uint32_t)__cvta_generic_to_shared(smem_raw);
-    const uint32_t dyn_end = base + kMaxDynSmem;
-    const uint32_t lut = (base + kSmallBytes + 0xffffu) & ~0xffffu;   // 64 KB aligned: byte 1 of an address is free for the code
+    constexpr uint32_t kSlotBytes = Codes::kBytes + 64u;       // codes + 16 fp16 scales (padded)
+    uint32_t lut = (kAssumedBase + kSmallBytes + 0xffffu) & ~0xffffu;   // 64 KB aligned: byte 1 of an address is free for the code
+    int D = prm.depth, warps_in_A = prm.warps_in_a;
+    if (base != kAssumedBase) ring_layout(base, kSlotBytes, &lut, &D, &warps_in_A);
     const uint32_t bars = base;
     const uint32_t item_bars = base + 2048u;                                        // [kMaxAccSlots] mbarriers, NS arrivals each
     volatile int* recycled = reinterpret_cast<volatile int*>(smem_raw + 2048 + 8 * kMaxAccSlots);   // [kMaxAccSlots] generations
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + 2560);
-
-    constexpr uint32_t kSlotBytes = Codes::kBytes + 64u;       // codes + 16 fp16 scales (padded)
     const uint32_t ringA = base + kSmallBytes, ringB = lut + kLutBytes;
     // Every warp's D slots are contiguous and lie entirely in one region, so slot d is one multiply-add away.
-    const int nA = (int)((lut - ringA) / kSlotBytes);
-    const int nB = (int)((dyn_end - ringB) / kSlotBytes);
-    int D = kMaxDepth;
-    while (D > 1 && nA / D + nB / D < kWarps) --D;
-    const int warps_in_A = nA / D;
     const uint32_t slot0 = warp < warps_in_A ? ringA + (uint32_t)(warp * D) * kSlotBytes
                                              : ringB + (uint32_t)((warp - warps_in_A) * D) * kSlotBytes;
     const uint32_t bar0 = bars + 8u * (uint32_t)(warp * kMaxDepth);
@@ -220,32 +270,36 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     auto full_bar = [&](int d) { return bar0 + 8u * (uint32_t)d; };
 
     // ---- this block's items and this warp's share of them ----
-    // (all per-task bookkeeping below is incremental 32-bit arithmetic)
-    const int tiles = (int)(prm.N / kRowTile);
-    const int parts = (int)gridDim.x / prm.chunks;
-    const int chunk_begin = (int)blockIdx.x / parts, part = (int)blockIdx.x % parts;   // this block's K-chunk
-    const int rt_begin = (int)((int64_t)tiles * part / parts);
-    const int n_items = (int)((int64_t)tiles * (part + 1) / parts) - rt_begin;          // its row tiles
-    const int groups = (int)(prm.K / kGroup);
-    const int NS = prm.ck / KS;                // slices per item = warps per item
-    const int PG = kWarps / NS;                // warps sharing a slice take every PG-th item
+    // (32-bit arithmetic; NS and PG are powers of two)
+    const uint32_t tiles = (uint32_t)(prm.N / kRowTile);
+    const uint32_t parts = (uint32_t)prm.parts;
+    auto div_parts = [&](uint32_t x) { return (uint32_t)(((unsigned long long)x * prm.parts_magic) >> (32 + prm.parts_shift)); };
+    const uint32_t chunk_begin_u = div_parts(blockIdx.x), part = blockIdx.x - chunk_begin_u * parts;   // this block's K-chunk
+    const int chunk_begin = (int)chunk_begin_u;
+    const int rt_begin = (int)div_parts(tiles * part);
+    const int n_items = (int)div_parts(tiles * (part + 1)) - rt_begin;                                 // its row tiles
+    const int groups = (int)(prm.K >> 10);
+    const int log_ns = prm.log_ns;
+    const int NS = 1 << log_ns;                // slices per item = warps per item
+    const int log_pg = 4 - log_ns;             // kWarps = 16
+    const int PG = 1 << log_pg;                // warps sharing a slice take every PG-th item
     const bool flusher = warp == kWarps;
-    const int slice = warp % NS, phase = warp / NS;
-    const int n_tasks = (!flusher && n_items > phase) ? (n_items - phase + PG - 1) / PG : 0;
+    const int slice = warp & (NS - 1), phase = warp >> log_ns;
+    const int n_tasks = (!flusher && n_items > phase) ? (n_items - phase + PG - 1) >> log_pg : 0;
     const int gl = (slice * KS) >> 10;         // group of this slice inside the item
     const int ng = prm.ck >> 10;               // groups per item
     // Partial tiles live in the upper halves of the table rows: 256 pieces of 32 floats (128 B), piece i at
     // lut + 128 + 256 i.  A tile holds B columns of 16 rows ([col][row]) in tile_pieces whole pieces; the tile of
     // (item slot q, slice ns) is tile q * NS + ns.  Element (col, row) of a tile sits in piece (col*16+row) >> 5.
-    const int tile_pieces = (16 * prm.B + 31) >> 5;
-    int acc_slots = 256 / (NS * tile_pieces);
-    { int p2 = 1; while (p2 * 2 <= acc_slots && p2 < kMaxAccSlots) p2 *= 2; acc_slots = p2; }
-    const int acc_shift = 31 - __clz(acc_slots);
+    const int tile_pieces = prm.tile_pieces;
+    const int acc_slots = prm.acc_slots;
+    const int acc_shift = prm.acc_shift;
     const uint32_t part0 = lut + 128u;
     const uint32_t tile_stride = (uint32_t)tile_pieces * 256u;         // bytes between consecutive tiles
-    const uint32_t q_stride = (uint32_t)NS * tile_stride;              // bytes between consecutive item slots
+    const uint32_t q_stride = tile_stride << log_ns;                   // bytes between consecutive item slots
 
-    // ---- prologue ----
+    // ---- ring barriers, then the first copies ----
+    TRACEP(warp, 1);
     if (lane == 0 && !flusher) {
         for (int d = 0; d < kMaxDepth; ++d) mbar_init(full_bar(d), 1);
     }
@@ -263,8 +317,8 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     // one K-chunk, so source addresses advance by constant strides.
     const int64_t kslice = (int64_t)chunk_begin * prm.ck + (int64_t)slice * KS;
     const int64_t rt_first = rt_begin + phase;
-    const uint8_t* src_next = prm.packed + (SIX ? ((rt_first * (prm.K / 128) + kslice / 128) * 768)
-                                                : ((rt_first * (prm.K / 64) + kslice / 64) * 512));
+    const uint8_t* src_next = prm.packed + (SIX ? ((rt_first * (prm.K >> 7) + (kslice >> 7)) * 768)
+                                                : ((rt_first * (prm.K >> 6) + (kslice >> 6)) * 512));
     const __half* ssrc_next = prm.scales + (rt_first * groups + chunk_begin * ng + gl) * 16;
     const int64_t src_stride = (int64_t)PG * (SIX ? prm.K * 6 : prm.K * 8);
     const int64_t ssrc_stride = (int64_t)PG * groups * 16;
@@ -284,46 +338,19 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     // (every lane runs the loop so that addresses stay warp-uniform - bulk copies take uniform operands - and one
     // elected lane issues)
     int issued = 0;
-    if (!flusher) {
-        for (; issued < n_tasks && issued < D; ++issued) issue(issued);
-    }
+    TRACEP(warp, 2);
+    for (; issued < n_tasks && issued < D; ++issued) issue(issued);
+    TRACEP(warp, 3);
 
     TRACE(warp, 0);
     pdl_trigger();
-    // Table: entry(idx) replicated once per lane (bank = lane): conflict-free gathers.  Warp w fills rows
-    // w, w+17, ...; all lanes of a warp read the same grid entry (one broadcast transaction), and the 16 loads of
-    // a warp are independent, so the whole build costs one global round trip.  (The grid is a constant of the layer.)
-    {
-        constexpr int kRowsPerWarp = (256 + kWarps) / (kWarps + 1);     // 16 rows for 17 warps (last one partly idle)
-        uint32_t ent[kRowsPerWarp];
-#pragma unroll
-        for (int r = 0; r < kRowsPerWarp; ++r) {
-            const int idx = warp + r * (kWarps + 1);
-            float lo = 0.f, hi = 0.f;
-            if (idx < 256) {
-                if (prm.p == 2) {
-                    const float2 gp = __ldg(reinterpret_cast<const float2*>(prm.grid) + (idx & (prm.n - 1)));
-                    lo = gp.x; hi = gp.y;
-                } else {
-                    lo = __ldg(prm.grid + (idx & 15));
-                    hi = __ldg(prm.grid + (idx >> 4));
-                }
-            }
-            __half2 h = __floats2half2_rn(lo, hi);
-            ent[r] = *reinterpret_cast<uint32_t*>(&h);
-        }
-#pragma unroll
-        for (int r = 0; r < kRowsPerWarp; ++r) {
-            const int idx = warp + r * (kWarps + 1);
-            if (idx < 256) *reinterpret_cast<uint32_t*>(smem_raw + (lut - base) + idx * 256 + lane * 4) = ent[r];
-        }
-    }
     // Everything above depends only on the weights.  The activations (and y, which the previous kernel in the
     // stream may still be reading or clearing) are touched only after the previous kernel has completed.
     pdl_wait();
     TRACE(warp, 1);
+    TRACEP(warp, 6);
 
-    // B fragments of this warp's K-slice for the first chunk (global loads, overlapped with the table build)
+    // B fragments of this warp's K-slice (global loads; their latency overlaps the table build below)
     uint32_t bfrag[KS / 16][NB][2];
     int cur_chunk = -1;
     auto load_bfrag = [&](int chunk) {
@@ -345,14 +372,30 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
         }
     };
     int c_chunk = chunk_begin, c_rt = rt_begin + phase, c_item = phase;   // compute cursor
-    while (c_rt >= tiles) { c_rt -= tiles; ++c_chunk; }
     if (n_tasks > 0) {
         cur_chunk = c_chunk;
         load_bfrag(cur_chunk);
     }
 
+    {
+        uint32_t ent[kRowsPerWarp];
+#pragma unroll
+        for (int r = 0; r < kRowsPerWarp; ++r) {
+            __half2 h = __floats2half2_rn(ent_lo[r], ent_hi[r]);
+            ent[r] = *reinterpret_cast<uint32_t*>(&h);
+        }
+        if (ent[0] != 0x12345678u) TRACEP(warp, 4);
+#pragma unroll
+        for (int r = 0; r < kRowsPerWarp; ++r) {
+            const int idx = warp + r * (kWarps + 1);
+            if (idx < 256) *reinterpret_cast<uint32_t*>(smem_raw + (lut - base) + idx * 256 + lane * 4) = ent[r];
+        }
+    }
+    TRACEP(warp, 5);
+    if (n_tasks > 0 && bfrag[0][0][0] != 0x12345678u) TRACEP(warp, 7);
     __syncthreads();     // table and barriers visible to every warp
     TRACE(warp, 2);
+    TRACEP(warp, 8);
     // ---- flusher warp: one item after the other, in item order ----
     if (flusher) {
         int f_chunk = chunk_begin, f_rt = rt_begin;
@@ -412,7 +455,7 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
                 }
             }
             TRACE(16, 5 + 2 * j);
-            if (++f_rt == tiles) { f_rt = 0; ++f_chunk; }
+            if (++f_rt == (int)tiles) { f_rt = 0; ++f_chunk; }
         }
         return;
     }
@@ -500,7 +543,7 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
         }
         c_item += PG;
         c_rt += PG;
-        while (c_rt >= tiles) { c_rt -= tiles; ++c_chunk; }
+        while (c_rt >= (int)tiles) { c_rt -= (int)tiles; ++c_chunk; }
     }
     if (!ok && lane == 0) {
         // aborting: never leave the block with this warp's copies in flight (bounded wait on its armed slots)
@@ -605,6 +648,21 @@ int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const 
     prm.ck = pl.ck;
     prm.y_mode = y_mode;
     const bool six = format_of(d.p, d.n) == Format::kSixBit;
+    prm.parts = pl.parts;
+    prm.parts_shift = 0;
+    while ((1 << prm.parts_shift) < pl.parts) ++prm.parts_shift;
+    prm.parts_magic = ((1ull << (32 + prm.parts_shift)) + (unsigned long long)pl.parts - 1ull) / (unsigned long long)pl.parts;
+    const int ns = pl.ck / pl.ks;
+    prm.log_ns = 0;
+    while ((1 << prm.log_ns) < ns) ++prm.log_ns;
+    prm.tile_pieces = (16 * (int)B + 31) >> 5;
+    int acc_slots = 256 / (ns * prm.tile_pieces), p2 = 1;
+    while (p2 * 2 <= acc_slots && p2 < kMaxAccSlots) p2 *= 2;
+    prm.acc_slots = p2;
+    prm.acc_shift = 0;
+    while ((1 << prm.acc_shift) < p2) ++prm.acc_shift;
+    uint32_t lut_unused;
+    ring_layout(kAssumedBase, (uint32_t)(six ? pl.ks * 6 : pl.ks * 8) + 64u, &lut_unused, &prm.depth, &prm.warps_in_a);
     if (pl.nb == 1 && !six) return launch_one<1, 256, false>(prm, pl.blocks, st);
     if (pl.nb == 2 && !six) return launch_one<2, 128, false>(prm, pl.blocks, st);
     if (pl.nb == 1 && six) return launch_one<1, 256, true>(prm, pl.blocks, st);
@@ -619,6 +677,7 @@ int launch_convert_out(const float* y32, void* y, int y_dtype, size_t count, cud
 }
 
 #ifdef HIGGS_TRACE
+extern "C" int higgs_trace_pro_read(long long* out) { return (int)cudaMemcpyFromSymbol(out, g_trace_pro, sizeof(long long) * 17 * 16); }
 extern "C" int higgs_trace_read(long long* out) { return (int)cudaMemcpyFromSymbol(out, g_trace, sizeof(long long) * 17 * 64); }
 #endif
 
