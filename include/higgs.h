@@ -165,9 +165,11 @@ int higgs_linear(const higgs_desc* desc, const void* x, int64_t B,
  * transform "can be fully isolated from the matrix multiplication itself").
  *   higgs_rotate_activations: x (device [B][K] bf16) -> xdag_out (device,
  *     higgs_rotated_bytes(desc, B) bytes of fp16) = (H / sqrt(g)) diag(sign) x
- *     per K-group.  The storage order is higgs_rotated_layout(desc, B): 0 = row
- *     major [B][K] (B <= 16, or layers the tensor-core path does not take),
- *     t > 0 = blocked operand tiles of t tokens for the tensor-core path.
+ *     per K-group.  The storage order is internal to the library and named by
+ *     higgs_rotated_layout(desc, B): 0 = [B][K] with the 32 input pairs of every
+ *     64-input block in the product kernel's fragment order (B <= 16, or layers
+ *     the tensor-core path does not take), t > 0 = blocked operand tiles of t
+ *     tokens for the tensor-core path.
  *   higgs_linear_prerotated: the product of Appendix F on already rotated
  *     activations; other arguments as higgs_linear.  xdag may be shared by
  *     layers with the same K, seed and higgs_rotated_layout (e.g. q, k, v).

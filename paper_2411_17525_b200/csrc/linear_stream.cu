@@ -34,11 +34,15 @@ __device__ int g_device_status = 0;
 __device__ long long g_trace[17][64];
 __device__ __forceinline__ long long trace_now() { return clock64(); }   // SM cycles (cheap); one block only, so one clock domain
 __device__ long long g_trace_pro[17][16];
+__device__ unsigned long long g_stream_blocks[4][256];
+__device__ __forceinline__ unsigned long long gtime_ns() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define BTRACE(row_) do { if ((threadIdx.x & 31) == 0 && blockIdx.x < 256) g_stream_blocks[row_][blockIdx.x] = gtime_ns(); } while (0)
 #define TRACEP(warp_, slot_) do { if (blockIdx.x == 7 && (threadIdx.x & 31) == 0) g_trace_pro[warp_][slot_] = trace_now(); } while (0)
 #define TRACE(warp_, slot_) do { if (blockIdx.x == 7 && (threadIdx.x & 31) == 0 && (slot_) < 64) g_trace[warp_][slot_] = trace_now(); } while (0)
 #else
 #define TRACE(warp_, slot_) do { } while (0)
 #define TRACEP(warp_, slot_) do { } while (0)
+#define BTRACE(row_) do { } while (0)
 #endif
 
 namespace {
@@ -224,15 +228,16 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     //                        bytes 128..255 = one 32-float piece of an accumulator tile
     //   [lut+64 KB, end)     ring slots, region B
     TRACEP(warp, 0);
+    if (warp == 0) BTRACE(0);
     // ---- the table's source first: the grid loads are in flight while everything below is set up ----
     // Table: entry(idx) replicated once per lane (bank = lane): conflict-free gathers.  Warp w fills rows
-    // w, w+17, ...; all lanes of a warp read the same grid entry (one broadcast transaction), and the 16 loads of
-    // a warp are independent, so the whole build costs one global round trip.  (The grid is a constant of the layer.)
-    constexpr int kRowsPerWarp = (256 + kWarps) / (kWarps + 1);     // 16 rows for 17 warps (last one partly idle)
-    float ent_lo[kRowsPerWarp], ent_hi[kRowsPerWarp];
+    // 4 (w + 17 r) .. + 3; a row's 128 bytes are written by eight lanes with one 16-byte store each, and the loads
+    // of a warp are independent, so the whole build costs one global round trip.  (The grid is a constant of the layer.)
+    constexpr int kQuadsPerWarp = (64 + kWarps) / (kWarps + 1);     // 4 groups of four rows for 17 warps
+    float ent_lo[kQuadsPerWarp], ent_hi[kQuadsPerWarp];
 #pragma unroll
-    for (int r = 0; r < kRowsPerWarp; ++r) {
-        const int idx = warp + r * (kWarps + 1);
+    for (int r = 0; r < kQuadsPerWarp; ++r) {
+        const int idx = 4 * (warp + r * (kWarps + 1)) + (lane >> 3);      // this lane's row: 8 lanes x 16 B fill one
         ent_lo[r] = 0.f; ent_hi[r] = 0.f;
         if (idx < 256) {
             if (prm.p == 2) {
@@ -337,11 +342,6 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     // the weight stream depends on nothing this kernel computes: start it before anything else
     // (every lane runs the loop so that addresses stay warp-uniform - bulk copies take uniform operands - and one
     // elected lane issues)
-    int issued = 0;
-    TRACEP(warp, 2);
-    for (; issued < n_tasks && issued < D; ++issued) issue(issued);
-    TRACEP(warp, 3);
-
     TRACE(warp, 0);
     pdl_trigger();
     // Everything above depends only on the weights.  The activations (and y, which the previous kernel in the
@@ -349,51 +349,54 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     pdl_wait();
     TRACE(warp, 1);
     TRACEP(warp, 6);
+    if (warp == 0) BTRACE(1);
 
     // B fragments of this warp's K-slice (global loads; their latency overlaps the table build below)
     uint32_t bfrag[KS / 16][NB][2];
-    int cur_chunk = -1;
     auto load_bfrag = [&](int chunk) {
+        // The rotation kernel stores x+ in fragment order: the eight words this lane needs from a 64-input block
+        // (steps m = 0..3, halves 0..1) are 32 contiguous bytes at offset 32 t of the block.
         const int64_t k0 = (int64_t)chunk * prm.ck + (int64_t)slice * KS;
 #pragma unroll
-        for (int s = 0; s < KS / 16; ++s) {
+        for (int nb = 0; nb < NB; ++nb) {
+            const int col = nb * 8 + g;
 #pragma unroll
-            for (int nb = 0; nb < NB; ++nb) {
-                const int col = nb * 8 + g;
-                uint32_t b0 = 0u, b1 = 0u;
+            for (int jb = 0; jb < KS / 64; ++jb) {
+                uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = make_uint4(0u, 0u, 0u, 0u);
                 if (col < prm.B) {
-                    const __half* src = prm.xdag + (int64_t)col * prm.K + k0 + s * 16 + 2 * t;
-                    b0 = *reinterpret_cast<const uint32_t*>(src);
-                    b1 = *reinterpret_cast<const uint32_t*>(src + 8);
+                    const uint4* src = reinterpret_cast<const uint4*>(prm.xdag + (int64_t)col * prm.K + k0 + jb * 64 + t * 16);
+                    lo = src[0];
+                    hi = src[1];
                 }
-                bfrag[s][nb][0] = b0;
-                bfrag[s][nb][1] = b1;
+                bfrag[jb * 4 + 0][nb][0] = lo.x; bfrag[jb * 4 + 0][nb][1] = lo.y;
+                bfrag[jb * 4 + 1][nb][0] = lo.z; bfrag[jb * 4 + 1][nb][1] = lo.w;
+                bfrag[jb * 4 + 2][nb][0] = hi.x; bfrag[jb * 4 + 2][nb][1] = hi.y;
+                bfrag[jb * 4 + 3][nb][0] = hi.z; bfrag[jb * 4 + 3][nb][1] = hi.w;
             }
         }
     };
-    int c_chunk = chunk_begin, c_rt = rt_begin + phase, c_item = phase;   // compute cursor
-    if (n_tasks > 0) {
-        cur_chunk = c_chunk;
-        load_bfrag(cur_chunk);
-    }
+    int c_item = phase;                  // compute cursor: this warp's next item of the block
+    if (n_tasks > 0) load_bfrag(chunk_begin);
+
+    int issued = 0;
+    TRACEP(warp, 2);
+    for (; issued < n_tasks && issued < D; ++issued) issue(issued);
+    TRACEP(warp, 3);
 
     {
-        uint32_t ent[kRowsPerWarp];
 #pragma unroll
-        for (int r = 0; r < kRowsPerWarp; ++r) {
+        for (int r = 0; r < kQuadsPerWarp; ++r) {
+            const int idx = 4 * (warp + r * (kWarps + 1)) + (lane >> 3);
             __half2 h = __floats2half2_rn(ent_lo[r], ent_hi[r]);
-            ent[r] = *reinterpret_cast<uint32_t*>(&h);
-        }
-        if (ent[0] != 0x12345678u) TRACEP(warp, 4);
-#pragma unroll
-        for (int r = 0; r < kRowsPerWarp; ++r) {
-            const int idx = warp + r * (kWarps + 1);
-            if (idx < 256) *reinterpret_cast<uint32_t*>(smem_raw + (lut - base) + idx * 256 + lane * 4) = ent[r];
+            const uint32_t e = *reinterpret_cast<uint32_t*>(&h);
+            if (idx < 256)
+                *reinterpret_cast<uint4*>(smem_raw + (lut - base) + idx * 256 + (lane & 7) * 16) = make_uint4(e, e, e, e);
         }
     }
     TRACEP(warp, 5);
     if (n_tasks > 0 && bfrag[0][0][0] != 0x12345678u) TRACEP(warp, 7);
     __syncthreads();     // table and barriers visible to every warp
+    if (warp == 0) BTRACE(2);
     TRACE(warp, 2);
     TRACEP(warp, 8);
     // ---- flusher warp: one item after the other, in item order ----
@@ -457,6 +460,7 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
             TRACE(16, 5 + 2 * j);
             if (++f_rt == (int)tiles) { f_rt = 0; ++f_chunk; }
         }
+        BTRACE(3);
         return;
     }
 
@@ -542,8 +546,6 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
             asm volatile("{ .reg .b64 st; mbarrier.arrive.shared::cta.b64 st, [%0]; }" ::"r"(item_bars + 8u * q) : "memory");
         }
         c_item += PG;
-        c_rt += PG;
-        while (c_rt >= (int)tiles) { c_rt -= (int)tiles; ++c_chunk; }
     }
     if (!ok && lane == 0) {
         // aborting: never leave the block with this warp's copies in flight (bounded wait on its armed slots)
@@ -677,6 +679,7 @@ int launch_convert_out(const float* y32, void* y, int y_dtype, size_t count, cud
 }
 
 #ifdef HIGGS_TRACE
+extern "C" int higgs_stream_blocks_read(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_stream_blocks, sizeof(unsigned long long) * 4 * 256); }
 extern "C" int higgs_trace_pro_read(long long* out) { return (int)cudaMemcpyFromSymbol(out, g_trace_pro, sizeof(long long) * 17 * 16); }
 extern "C" int higgs_trace_read(long long* out) { return (int)cudaMemcpyFromSymbol(out, g_trace, sizeof(long long) * 17 * 64); }
 #endif

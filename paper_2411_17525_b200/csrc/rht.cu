@@ -37,8 +37,10 @@ __device__ __forceinline__ void load_group<float>(const float* __restrict__ src,
     }
 }
 
-// One warp per (token, group): x+ = (H/32) diag(sign) x, written as fp16 in natural
-// order.  Extra threads beyond the transform work clear `zero_ptr` (the fp32
+// One warp per (token, group): x+ = (H/32) diag(sign) x, written as fp16 in "fragment order": inside every block of
+// 64 inputs the 32 input pairs are permuted so that the eight pairs one lane of the product kernel needs as
+// m16n8k16 B-fragment registers (steps m = 0..3, halves h = 0..1 of its column pair t) are 32 contiguous bytes:
+// position t*8 + m*2 + h holds pair 8m + t + 4h.  Extra threads beyond the transform work clear `zero_ptr` (the fp32
 // accumulation target of a K-split product) so no separate memset launch is needed.
 template <typename T>
 __global__ void __launch_bounds__(256) rht_activations_kernel(const T* __restrict__ x, __half* __restrict__ xdag,
@@ -58,16 +60,18 @@ __global__ void __launch_bounds__(256) rht_activations_kernel(const T* __restric
     load_group<T>(x + b * K + gi * kGroup, lane, v);
     apply_signs1024(v, xi, gi * kGroup, lane);
     fwht1024_warp(v, lane);
-    __half* dst = xdag + b * K + gi * kGroup;
+    uint32_t* dst = reinterpret_cast<uint32_t*>(xdag + b * K + gi * kGroup);
+    // this lane's chunk c holds inputs c*256 + lane*8 .. +7: pairs 4j + i (i = 0..3) of 64-input block c*4 + lane/8,
+    // j = lane % 8, i.e. m = j >> 1, h = j & 1, t = i  ->  position i*8 + j
+    const int j = lane & 7;
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
-        uint32_t w[4];
+        uint32_t* blk = dst + (c * 4 + (lane >> 3)) * 32;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             __half2 h = __floats2half2_rn(v[c * 8 + 2 * e] * 0.03125f, v[c * 8 + 2 * e + 1] * 0.03125f);
-            w[e] = *reinterpret_cast<uint32_t*>(&h);
+            blk[e * 8 + j] = *reinterpret_cast<uint32_t*>(&h);
         }
-        *reinterpret_cast<uint4*>(dst + c * 256 + lane * 8) = make_uint4(w[0], w[1], w[2], w[3]);
     }
 }
 
