@@ -23,8 +23,6 @@
 // a status word instead of hanging.
 #include "common.cuh"
 
-#include <cstdlib>
-
 namespace higgs {
 
 __device__ int g_device_status = 0;
@@ -71,7 +69,7 @@ struct StreamParams {
 
 constexpr uint32_t kLutBytes = 65536;   // 256 entries x 256-byte row (32 lanes x 4 B; upper row halves hold accumulators)
 constexpr uint32_t kMaxDynSmem = 232448;
-constexpr uint32_t kSmallBytes = 4096;  // barriers, table seed, counters
+constexpr uint32_t kSmallBytes = 4096;  // barriers, recycle counters, abort flag
 constexpr int kWarps = 16;
 constexpr int kMaxDepth = 8;            // ring slots per warp
 constexpr int kMaxAccSlots = 32;        // items whose partial tiles may be parked at once
@@ -591,11 +589,9 @@ Plan make_plan(const higgs_desc& d, int64_t B) {
     const int sms = sm_count();
     const int64_t tiles = d.N / kRowTile;
     double best_score = -1.0;
-    const char* force = getenv("HIGGS_CK");
     for (int ck = 4096; ck >= 1024; ck >>= 1) {
         if (d.K % ck) continue;
         if (ck / ks > kWarps) continue;
-        if (force && atoi(force) != ck) continue;
         const int chunks = (int)(d.K / ck);
         int64_t parts = sms / chunks;
         if (parts < 1) parts = 1;
