@@ -246,6 +246,17 @@ int higgs_linear_launch_count(const higgs_desc* desc, int64_t B, int y_dtype);
 
 /* ---- validation helpers (not on the hot path) --------------------------- */
 
+/* Dequantisation to the original space (Appendix F, "Dequantization"):
+ *   W_out[r][group i] = diag(sign) (H / sqrt(g)) ( scale[r][i] * G[codes of (r, i)] ),
+ * the matrix the quantised layer stands for, so that y == x W_out^T up to rounding.
+ *   packed, scales, grid : device, as written by higgs_quantize / passed to higgs_linear
+ *   W_out                : device [N][K] row-major, w_dtype in {HIGGS_F32, HIGGS_BF16}
+ *   workspace            : device, higgs_workspace_bytes(desc, HIGGS_OP_QUANTIZE, 0) bytes
+ *                          (the canonical codes), 256-byte aligned
+ * Errors as higgs_quantize.  Asynchronous on `stream`.                        */
+int higgs_dequantize(const higgs_desc* desc, const void* packed, const void* scales, const float* grid,
+                     void* W_out, int w_dtype, void* workspace, size_t workspace_bytes, void* stream);
+
 /* The transform alone on `rows` rows of length K: out[r] = RHT of x[r] per
  * group (Algorithm 1 / Appendix F).  x_dtype in {HIGGS_F32, HIGGS_BF16};
  * out is device [rows][K] fp32; normalised != 0 divides by sqrt(g).        */

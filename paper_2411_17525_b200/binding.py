@@ -25,7 +25,7 @@ EXPORTS = [
     "higgs_pack_codes", "higgs_unpack_codes", "higgs_rotate_activations", "higgs_linear_prerotated",
     "higgs_linear_host", "higgs_linear_host_workspace_bytes", "higgs_linear_launch_count", "higgs_device_status",
     "higgs_linear_static", "higgs_linear_static_capacity", "higgs_linear_k_splits", "higgs_rotated_bytes",
-    "higgs_rotated_layout",
+    "higgs_rotated_layout", "higgs_dequantize",
 ]
 
 
@@ -92,6 +92,8 @@ def _load() -> ctypes.CDLL:
     lib.higgs_pack_codes.argtypes = [P, vp, vp, vp]
     lib.higgs_unpack_codes.restype = i32
     lib.higgs_unpack_codes.argtypes = [P, vp, vp, vp]
+    lib.higgs_dequantize.restype = i32
+    lib.higgs_dequantize.argtypes = [P, vp, vp, vp, vp, i32, vp, sz, vp]
     return lib
 
 
@@ -302,6 +304,16 @@ def higgs_pack_codes(desc: higgs_desc, canonical: torch.Tensor) -> torch.Tensor:
     packed = torch.empty(max(higgs_packed_bytes(desc), 16), dtype=torch.uint8, device=canonical.device)
     _check(lib.higgs_pack_codes(ctypes.byref(desc), _ptr(canonical), _ptr(packed), _stream()), "higgs_pack_codes")
     return packed
+
+
+def higgs_dequantize(desc: higgs_desc, packed: torch.Tensor, scales: torch.Tensor, grid: torch.Tensor,
+                     out_dtype: torch.dtype = torch.float32) -> torch.Tensor:
+    """packed codes + scales -> the matrix [N][K] the quantised layer stands for (Appendix F, 'Dequantization')."""
+    W = torch.empty((desc.N, desc.K), dtype=out_dtype, device=packed.device)
+    ws = _workspace(higgs_workspace_bytes(desc, HIGGS_OP_QUANTIZE, 0), packed.device)
+    _check(lib.higgs_dequantize(ctypes.byref(desc), _ptr(packed), _ptr(scales), _ptr(grid), _ptr(W), _dtype_code(W),
+                                _ptr(ws), ws.numel(), _stream()), "higgs_dequantize")
+    return W
 
 
 def higgs_unpack_codes(desc: higgs_desc, packed: torch.Tensor) -> torch.Tensor:

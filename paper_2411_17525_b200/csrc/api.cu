@@ -103,6 +103,22 @@ int higgs_quantize(const higgs_desc* d, const void* W, int w_dtype, const float*
     return launch_pack(*d, canonical, packed_out, st);
 }
 
+int higgs_dequantize(const higgs_desc* d, const void* packed, const void* scales, const float* grid, void* W_out,
+                     int w_dtype, void* workspace, size_t workspace_bytes, void* stream) {
+    int rc = check_desc(d);
+    if (rc != HIGGS_OK) return rc;
+    if (w_dtype != HIGGS_F32 && w_dtype != HIGGS_BF16) return HIGGS_ERR_UNSUPPORTED;
+    if (d->N == 0 || d->K == 0) return HIGGS_OK;
+    if (!packed || !scales || !grid || !W_out || !workspace) return HIGGS_ERR_INVALID_ARG;
+    if (!aligned(packed, 16) || !aligned(scales, 16) || !aligned(W_out, 16) || !aligned(workspace, 256)) return HIGGS_ERR_INVALID_ARG;
+    if (workspace_bytes < higgs_workspace_bytes(d, HIGGS_OP_QUANTIZE, 0)) return HIGGS_ERR_WORKSPACE;
+    cudaStream_t st = as_stream(stream);
+    uint8_t* canonical = static_cast<uint8_t*>(workspace);
+    rc = launch_unpack(*d, packed, canonical, st);
+    if (rc != HIGGS_OK) return rc;
+    return launch_dequantize(*d, canonical, scales, grid, W_out, w_dtype, st);
+}
+
 int higgs_rotate_activations(const higgs_desc* d, const void* x, int64_t B, void* xdag_out, void* stream) {
     int rc = check_desc(d);
     if (rc != HIGGS_OK) return rc;

@@ -129,6 +129,8 @@ int launch_encode(const higgs_desc& d, const void* W, int w_dtype, const float* 
                   void* scales, cudaStream_t st);
 int launch_pack(const higgs_desc& d, const uint8_t* canonical, void* packed, cudaStream_t st);
 int launch_unpack(const higgs_desc& d, const void* packed, uint8_t* canonical, cudaStream_t st);
+int launch_dequantize(const higgs_desc& d, const uint8_t* canonical, const void* scales, const float* grid, void* W_out,
+                      int w_dtype, cudaStream_t st);
 int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const void* packed, const void* scales,
                       const float* grid, void* y, int64_t ldy, int y_mode, cudaStream_t st);
 int launch_convert_out(const float* y32, void* y, int y_dtype, size_t count, cudaStream_t st);

@@ -210,6 +210,28 @@ def test_make_grid_is_a_lloyd_fixed_point_at_the_oracle_mse(p, n):
     assert abs(m_dev - m_ref) <= 0.01 * m_ref
 
 
+# ----------------------------------------------------------------------------- dequantisation to the original space
+@pytest.mark.parametrize("p,n,N,K", [(2, 256, 48, 2048), (2, 64, 32, 3072), (1, 16, 16, 1024)])
+def test_dequantize_matches_oracle(p, n, N, K):
+    """Appendix F 'Dequantization': LUT restore, inverse rotation, unscale; element by element against the oracle."""
+    xi = inputs.rht_seed(2)
+    W = inputs.make_weights(N, K, seed=900 + n, bf16=True)
+    g64, gt = U.grid32(p, n)
+    q, sc16 = U.oracle_encode(W, G, g64, xi)
+    d = hb.make_desc(p, n, N, K, xi)
+    packed = hb.higgs_pack_codes(d, torch.from_numpy(q.codes.astype(np.uint8)).to(U.dev()))
+    scales = hb.scales_to_tile_major(torch.from_numpy(sc16).to(U.dev()))
+    W_ref = oracle.dequantize(q.codes, sc16.astype(np.float64), G, g64, xi)
+    W_gpu = hb.higgs_dequantize(d, packed, scales, gt).cpu().numpy().astype(np.float64)
+    assert W_gpu.shape == (N, K)
+    assert np.max(np.abs(W_gpu - W_ref)) <= 2e-6 * np.max(np.abs(W_ref))      # fp32 butterflies over 10 stages
+    # and it is the matrix the layer stands for: relative error against W equals the grid's MSE level (Appendix E)
+    rel = np.sum((W_gpu - W) ** 2) / np.sum(W.astype(np.float64) ** 2)
+    assert rel < 0.25 if n == 16 else rel < 0.05
+    W_bf = hb.higgs_dequantize(d, packed, scales, gt, out_dtype=torch.bfloat16).float().cpu().numpy()
+    assert np.max(np.abs(W_bf - W_ref)) <= 2.0 ** -8 * np.max(np.abs(W_ref))
+
+
 # ----------------------------------------------------------------------------- tensor-core path (B > 16, N % 128 == 0)
 @pytest.mark.parametrize("p,n,N,K,B", [
     (2, 256, 128, 1024, 17),     # smallest tile: one block, 16 stages, token tile of 32
