@@ -25,6 +25,8 @@
 // released.
 #include "common.cuh"
 
+#include <cuda.h>
+
 namespace higgs {
 
 __device__ int g_tc_status = 0;
@@ -58,7 +60,7 @@ struct TcParams {
 constexpr uint32_t kTcSmem = 232448;
 constexpr int kTcGroups = 4;                 // dequant warp groups (4 warps each, one per TMEM lane quadrant)
 constexpr int kTcBStages = 3;                // activation-tile stages in shared memory (at most 32 KB each)
-constexpr int kTcMaxCodeStages = 14;         // code stages in shared memory (4 KB each)
+constexpr int kTcMaxCodeStages = 32;         // code stages in shared memory (4 KB each), below and above the table
 constexpr int kTcDequantWarps = 4 * kTcGroups;
 constexpr int kTcThreads = (3 + kTcDequantWarps) * 32;
 constexpr uint32_t kTcCodeStage = 4096;      // 128 rows x 64 inputs, one byte per input pair
@@ -114,11 +116,11 @@ __device__ __forceinline__ void t_bulk_load(uint32_t dst, const void* src, uint3
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                  "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-// true in exactly one lane of the (converged) warp
-__device__ __forceinline__ bool elect_one() {
-    uint32_t is_elected;
-    asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(is_elected));
-    return is_elected != 0;
+// One tiled TMA copy: the box (64 x 8-byte elements = one 512-byte block, 8 row tiles) at element column x, row tile y
+// of the packed stream viewed as a 2-D tensor [N/16 row tiles][K x 8 bytes]; lands as [8][512 B] in shared memory.
+__device__ __forceinline__ void t_tensor_load(uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -163,15 +165,16 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 // FB = 64-input steps per activation-tile stage (4, 2, 1 for BN <= 64, <= 128, <= 256: a stage is at most 32 KB).  It is a
 // template parameter so that the MMA warp's loop body is straight-line code.
 template <int FB>
-__global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams prm) {
+__global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap code_map) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     // ---- shared memory map ----
     //   [base, base+2 KB)    mbarriers, TMEM base address, abort flag
-    //   [base+2 KB, lut)     code stages (CS x 4 KB): deep, because the codes are the HBM stream
+    //   [base+2 KB, lut)     code stages, region A (4 KB each): deep, because the codes are the HBM stream
     //   [lut, lut+64 KB)     lookup table, 256-byte rows (bytes 0..127 = the entry replicated per lane)
-    //   [lut+64 KB, end)     activation-tile stages (3 x at most 32 KB; they come from L2)
+    //   [lut+64 KB, ...)     three activation-tile stages (FB x BN x 128 bytes each; they come from L2)
+    //   [..., end)           code stages, region B (whatever the activation stages leave: 52 KB for BN <= 128)
     //   after the main loop, K-split only: [base+2 KB, +BN x 512 B) the block's partial tile, [token][row] fp32
     // Three rings: codes (freed when the four dequant warps of a step have read them), activation tiles and the
     // A operand in TMEM (both freed by tcgen05.commit when the MMAs that read them are done).
@@ -179,19 +182,24 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
     const uint32_t lut = (base + 2048u + 0xffffu) & ~0xffffu;
     const uint32_t bars = base;
     auto code_full = [&](int s) { return bars + 8u * (uint32_t)s; };
-    auto code_empty = [&](int s) { return bars + 8u * (uint32_t)(16 + s); };
-    auto b_full = [&](int s) { return bars + 8u * (uint32_t)(32 + s); };
-    auto b_free = [&](int s) { return bars + 8u * (uint32_t)(36 + s); };
-    auto a_full = [&](int s) { return bars + 8u * (uint32_t)(40 + s); };
-    auto a_free = [&](int s) { return bars + 8u * (uint32_t)(44 + s); };
-    const uint32_t d_full = bars + 8u * 56u;
+    auto code_empty = [&](int s) { return bars + 8u * (uint32_t)(32 + s); };
+    auto b_full = [&](int s) { return bars + 8u * (uint32_t)(64 + s); };
+    auto b_free = [&](int s) { return bars + 8u * (uint32_t)(68 + s); };
+    auto a_full = [&](int s) { return bars + 8u * (uint32_t)(72 + s); };
+    auto a_free = [&](int s) { return bars + 8u * (uint32_t)(76 + s); };
+    const uint32_t d_full = bars + 8u * 80u;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_raw + 1024);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + 1032);
     const uint32_t code0 = base + 2048u;
-    int CS = (int)((lut - code0) / kTcCodeStage);
-    if (CS > kTcMaxCodeStages) CS = kTcMaxCodeStages;
-    auto code_stage = [&](int s) { return code0 + (uint32_t)s * kTcCodeStage; };
-    auto b_stage = [&](int s) { return lut + 65536u + (uint32_t)s * 32768u; };
+    const uint32_t b_stage_bytes = (uint32_t)FB * (uint32_t)prm.BN * 128u;
+    const uint32_t code1 = lut + 65536u + (uint32_t)kTcBStages * b_stage_bytes;      // region B
+    int nA = (int)((lut - code0) / kTcCodeStage);
+    if (nA > 16) nA = 16;
+    int nB = (int)((base + kTcSmem - code1) / kTcCodeStage);
+    if (nB > kTcMaxCodeStages - nA) nB = kTcMaxCodeStages - nA;
+    const int CS = nA + nB;
+    auto code_stage = [&](int s) { return s < nA ? code0 + (uint32_t)s * kTcCodeStage : code1 + (uint32_t)(s - nA) * kTcCodeStage; };
+    auto b_stage = [&](int s) { return lut + 65536u + (uint32_t)s * b_stage_bytes; };
 
     const int BN = prm.BN;
     const int ksplit = prm.ksplit;
@@ -203,81 +211,101 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
     const int64_t row0 = (int64_t)blockIdx.x * 128;
     const int bt = blockIdx.y;
     const uint32_t b_step_bytes = (uint32_t)BN * 128u;
+    const int tile0 = (int)(row0 / 16);                      // first 16-row tile of this block
     const int AS = BN <= 128 ? 3 : 2;                        // A stages in TMEM
     const uint32_t acol0 = BN <= 128 ? 128u : 256u;
 
     // ---- prologue ----
     BTRACE(0);
-    if (tid == 0) {
-        for (int s = 0; s < 16; ++s) { t_mbar_init(code_full(s), 1); t_mbar_init(code_empty(s), 4); }
-        for (int s = 0; s < 4; ++s) { t_mbar_init(b_full(s), 1); t_mbar_init(b_free(s), 1); }
-        for (int s = 0; s < 4; ++s) { t_mbar_init(a_full(s), kTcDequantWarps); t_mbar_init(a_free(s), 1); }
-        t_mbar_init(d_full, 1);
-        *abort_flag = 0;
+    // (1) the table's source: the grid loads are in flight while everything else is set up.  Warp w fills rows
+    //     4 (w + 19 r) .. + 3; a row's 128 bytes are written by eight lanes with one 16-byte store each.
+    constexpr int kW = kTcThreads / 32;
+    constexpr int kQuads = (64 + kW - 1) / kW;
+    float ent_lo[kQuads], ent_hi[kQuads];
+#pragma unroll
+    for (int r = 0; r < kQuads; ++r) {
+        const int idx = 4 * (warp + r * kW) + (lane >> 3);
+        ent_lo[r] = 0.f; ent_hi[r] = 0.f;
+        if (idx < 256) {
+            if (prm.p == 2) {
+                const float2 gp = __ldg(reinterpret_cast<const float2*>(prm.grid) + (idx & (prm.n - 1)));
+                ent_lo[r] = gp.x; ent_hi[r] = gp.y;
+            } else {
+                ent_lo[r] = __ldg(prm.grid + (idx & 15));
+                ent_hi[r] = __ldg(prm.grid + (idx >> 4));
+            }
+        }
+    }
+    // The code ring needs one stage per warp group; the block's shared-memory window always leaves room for more, but
+    // a window that did not would be reported, not run.
+    int role = warp;
+    if (CS < kTcGroups) role = -1;
+    // (2) barriers, each ring by the warp that produces into it; the code producer starts the weight stream (which
+    //     depends on nothing) before the block-wide barrier: the first CS stages need no wait.
+    int code_issued = 0;
+    uint32_t elected;
+    asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(elected));
+    if (warp == 0) {
+        t_mbar_init(code_full(lane), 1);
+        t_mbar_init(code_empty(lane), 4);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (role == 0) {
+            const int n0 = ksteps < CS ? ksteps : CS;
+            for (int j = 0; j < n0; ++j) {
+                if (elected) {
+                    t_mbar_expect_tx(code_full(j), kTcCodeStage);
+                    t_tensor_load(code_stage(j), &code_map, (kstep0 + j) * 64, tile0, code_full(j));
+                }
+                __syncwarp();
+            }
+            code_issued = n0;
+        }
+    } else if (warp == 1) {
+        if (lane < 4) { t_mbar_init(a_full(lane), kTcDequantWarps); t_mbar_init(a_free(lane), 1); }
+        if (lane == 4) t_mbar_init(d_full, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        // one warp allocates all 512 TMEM columns (one block per SM, so nobody else wants them)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + 1024u), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    } else if (warp == 2) {
+        if (lane < 4) { t_mbar_init(b_full(lane), 1); t_mbar_init(b_free(lane), 1); }
+        if (lane == 4) {
+            *abort_flag = 0;
+            if (role < 0) { *abort_flag = 1; atomicExch(&g_tc_status, (int)HIGGS_ERR_TIMEOUT); }
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) {   // one warp allocates all 512 TMEM columns (one block per SM, so nobody else wants them)
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + 1024u), "r"(512u) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
     pdl_trigger();
-    {   // lookup table: warp w fills rows w, w+19, ...; the grid is a constant of the layer
-        constexpr int kW = kTcThreads / 32;
-        constexpr int kRows = (256 + kW - 1) / kW;
-        uint32_t ent[kRows];
+    // (3) the table
 #pragma unroll
-        for (int r = 0; r < kRows; ++r) {
-            const int idx = warp + r * kW;
-            float lo = 0.f, hi = 0.f;
-            if (idx < 256) {
-                if (prm.p == 2) {
-                    const float2 gp = __ldg(reinterpret_cast<const float2*>(prm.grid) + (idx & (prm.n - 1)));
-                    lo = gp.x; hi = gp.y;
-                } else {
-                    lo = __ldg(prm.grid + (idx & 15));
-                    hi = __ldg(prm.grid + (idx >> 4));
-                }
-            }
-            __half2 h = __floats2half2_rn(lo, hi);
-            ent[r] = *reinterpret_cast<uint32_t*>(&h);
-        }
-#pragma unroll
-        for (int r = 0; r < kRows; ++r) {
-            const int idx = warp + r * kW;
-            if (idx < 256) *reinterpret_cast<uint32_t*>(smem_raw + (lut - base) + idx * 256 + lane * 4) = ent[r];
-        }
+    for (int r = 0; r < kQuads; ++r) {
+        const int idx = 4 * (warp + r * kW) + (lane >> 3);
+        __half2 h = __floats2half2_rn(ent_lo[r], ent_hi[r]);
+        const uint32_t e = *reinterpret_cast<uint32_t*>(&h);
+        if (idx < 256) *reinterpret_cast<uint4*>(smem_raw + (lut - base) + idx * 256 + (lane & 7) * 16) = make_uint4(e, e, e, e);
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
-    // The code ring needs one stage per warp group; the block's shared-memory window always leaves room for more, but
-    // a window that did not would be reported, not run.
-    int role = warp;
-    if (CS < kTcGroups) {
-        if (tid == 0) { *abort_flag = 1; atomicExch(&g_tc_status, (int)HIGGS_ERR_TIMEOUT); }
-        role = -1;
-    }
 
     if (role == 0) {
         // =============================== code producer (weights: no dependency on earlier kernels) ===============
-        // (whole warp in the loop, one elected lane issues: bulk copies take warp-uniform operands)
-        uint32_t elected;
-        asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(elected));
-        int issued = 0;
-        const int64_t tile_stride = (int64_t)ksteps_all * 512;     // bytes between consecutive 16-row tiles
-        const uint8_t* src0 = prm.packed + (row0 / 16) * tile_stride + (int64_t)kstep0 * 512;
-        int s = 0, it = 0;
+        // (whole warp in the loop, one elected lane issues: bulk copies take warp-uniform operands; the first stages
+        // were issued in the prologue)
+        int issued = code_issued;
+        int s = issued == CS ? 0 : issued, it = issued == CS ? 1 : 0;
         uint32_t bad = 0;
-        for (int j = 0; j < ksteps; ++j) {
-            // (the first pass waits for the phase before the first one, which counts as complete)
+        for (int j = issued; j < ksteps; ++j) {
             bad |= t_wait(code_empty(s), (uint32_t)((it & 1) ^ 1), t_limit(bad)) ^ 1u;
             if (elected) {
                 t_mbar_expect_tx(code_full(s), kTcCodeStage);
-#pragma unroll
-                for (int rtl = 0; rtl < 8; ++rtl)
-                    t_bulk_load(code_stage(s) + rtl * 512, src0 + rtl * tile_stride + (int64_t)j * 512, 512u, code_full(s));
+                t_tensor_load(code_stage(s), &code_map, (kstep0 + j) * 64, tile0, code_full(s));
             }
             ++issued;
             const bool wrap = s + 1 == CS;
@@ -291,8 +319,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
         t_report(bad, abort_flag);
     } else if (role == 2) {
         // =============================== activation-tile producer ===============================
-        uint32_t elected;
-        asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(elected));
         pdl_wait();            // the rotated activations are the previous kernel's output
         int issued = 0;
         const int nb = ksteps / FB;
@@ -321,8 +347,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
         // operands from uniform registers); one elected lane issues.  Per A stage (256 inputs): one wait for the
         // sixteen dequant warps, one wait per activation-tile stage, sixteen MMAs.
         const uint32_t idesc = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | (8u << 24);   // f32 accumulate, f16 x f16, K-major, M=128
-        uint32_t elected;
-        asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(elected));
         int sa = 0, ua = 0;            // A stage and its use count
         int sb = 0, ub = 0;            // activation-tile stage and its use count
         uint32_t bad = 0;
@@ -342,7 +366,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
                 }
                 // addresses and descriptors are computed by the whole warp; only the instruction is issued by one lane
                 const uint32_t a_addr = a_stage + 32u * (uint32_t)h;
-                const uint64_t b_desc = b_desc0 + (uint64_t)(((uint32_t)sb * 32768u + (uint32_t)(h % FB) * b_step_bytes) >> 4);
+                const uint64_t b_desc = b_desc0 + (uint64_t)(((uint32_t)sb * b_stage_bytes + (uint32_t)(h % FB) * b_step_bytes) >> 4);
                 const uint32_t acc = (uint32_t)((S | h) != 0);
                 if (elected) {
                     tc_mma(tmem, a_addr, b_desc, idesc, acc);
@@ -602,6 +626,42 @@ int tc_k_split(const higgs_desc& d, int64_t B) {
     return ks;
 }
 
+namespace {
+
+// cuTensorMapEncodeTiled through the runtime's driver-entry-point query (the library does not link libcuda).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
+            qr == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// The packed byte stream of a layer as a 2-D tensor of 8-byte elements: row = 16-row tile (K x 8 bytes: K/64 blocks
+// of 512 bytes), box = one block column of eight consecutive row tiles (the 128 rows of a thread block).
+bool make_code_map(const higgs_desc& d, const void* packed, CUtensorMap* map) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)d.K, (cuuint64_t)(d.N / 16)};
+    const cuuint64_t strides[1] = {(cuuint64_t)d.K * 8};
+    const cuuint32_t box[2] = {64, 8};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_INT64, 2, const_cast<void*>(packed), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
 // D2-D5 on the tensor cores, from activations rotated by launch_rht_tc for the same B.
 int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, const void* packed, const void* scales,
                      const float* grid, void* y, int y_mode, cudaStream_t st) {
@@ -617,6 +677,8 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
             return HIGGS_ERR_CUDA;
         configured[dev] = true;
     }
+    CUtensorMap code_map;
+    if (!make_code_map(d, packed, &code_map)) return HIGGS_ERR_CUDA;
     TcParams prm;
     prm.packed = static_cast<const uint8_t*>(packed);
     prm.scales = static_cast<const __half*>(scales);
@@ -643,9 +705,11 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
         cfg.numAttrs = 2;
     }
     cfg.attrs = attr;
-    if (BN <= 64) return cuda_status(cudaLaunchKernelEx(&cfg, linear_tc_kernel<4>, prm));
-    if (BN <= 128) return cuda_status(cudaLaunchKernelEx(&cfg, linear_tc_kernel<2>, prm));
-    return cuda_status(cudaLaunchKernelEx(&cfg, linear_tc_kernel<1>, prm));
+    // activation-tile stage = FB steps of BN x 128 bytes, at most 16 KB for BN <= 128 (so that the code ring gets the
+    // rest of shared memory) and 32 KB for wider tiles
+    if (BN <= 32) return cuda_status(cudaLaunchKernelEx(&cfg, linear_tc_kernel<4>, prm, code_map));
+    if (BN <= 64) return cuda_status(cudaLaunchKernelEx(&cfg, linear_tc_kernel<2>, prm, code_map));
+    return cuda_status(cudaLaunchKernelEx(&cfg, linear_tc_kernel<1>, prm, code_map));
 }
 
 #ifdef HIGGS_TRACE
