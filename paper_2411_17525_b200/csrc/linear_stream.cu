@@ -598,7 +598,8 @@ Plan make_plan(const higgs_desc& d, int64_t B) {
         if (parts > tiles) parts = tiles;
         const int64_t per = (tiles + parts - 1) / parts;          // row tiles of the busiest block
         const double eff = (double)tiles * chunks / (double)(per * sms);
-        const double score = eff * (chunks == 1 ? 1.0 : 0.45);
+        // every extra K-chunk adds a pass of atomics over y and shortens the items (more bookkeeping per byte)
+        const double score = eff * (chunks == 1 ? 1.0 : 0.45 / (1.0 + 0.04 * (chunks - 2)));
         if (score > best_score) {
             best_score = score;
             best.nb = nb; best.ks = ks; best.ck = ck; best.chunks = chunks;

@@ -597,9 +597,12 @@ int tc_batch_tile(int64_t B) {
     return (int)((per + 15) / 16 * 16);
 }
 
-// The tensor-core path takes batches above 16 of byte-coded layers whose row count is a multiple of 128.
+// The tensor-core path takes byte-coded layers whose row count is a multiple of 128: every batch above 16, and batches
+// 9..16 of large layers (there the small-batch kernel is limited by the legacy mma.sync rate, two per lookup group;
+// measured cross-over near 32 M weights).
 bool tc_eligible(const higgs_desc& d, int64_t B) {
-    return B > 16 && d.N % 128 == 0 && d.N > 0 && format_of(d.p, d.n) == Format::kByteLut;
+    if (!(d.N % 128 == 0 && d.N > 0 && format_of(d.p, d.n) == Format::kByteLut)) return false;
+    return B > 16 || (B > 8 && d.N * d.K >= ((int64_t)1 << 25));
 }
 
 size_t tc_workspace_bytes(const higgs_desc& d, int64_t B) {
