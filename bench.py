@@ -43,7 +43,9 @@ def parse_args():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="llama-3.2-1b", choices=list(inputs.LAYER_SETS))
     ap.add_argument("--batch", type=int, default=1)
-    ap.add_argument("--grid", default="2,256", help="p,n")
+    ap.add_argument("--grid", default="2,256",
+                    help="p,n for every layer, or 'mixed': 3 or 4 bits per matrix (p=2 n=64 / n=256) from the seeded assignment "
+                         "averaging 3.5 bits (the Llama-3.1-70B configuration)")
     ap.add_argument("--no-graph", action="store_true", help="launch kernels directly instead of replaying CUDA graphs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-detail", action="store_true", help="skip the per-layer / other-batch detail measurements")
@@ -53,6 +55,19 @@ def parse_args():
 def layer_bytes(N, K, p, n):
     bits = {(2, 256): 4, (1, 16): 4, (2, 64): 3}[(p, n)]
     return N * K * bits // 8 + N * (K // G) * 2
+
+
+def layer_grids(args, layers, cfg):
+    """(p, n) per layer: one grid for all, or the block of the seeded 3/4-bit assignment closest to 3.5 bits."""
+    if args.grid != "mixed":
+        p, n = (int(v) for v in args.grid.split(","))
+        return [(p, n)] * len(layers), f"p={p} n={n}"
+    blocks = inputs.bitwidth_assignment(7000 + cfg, layers)
+    sizes = np.array([N * K for _, N, K in layers], dtype=np.float64)
+    best = min(blocks, key=lambda b: abs(float((np.array(b) * sizes).sum() / sizes.sum()) - 3.5))
+    mean = float((np.array(best) * sizes).sum() / sizes.sum())
+    pn = [(2, 64) if b == 3 else (2, 256) for b in best]
+    return pn, "mixed " + ",".join(f"{nm}:{b}" for (nm, _, _), b in zip(layers, best)) + f" bits ({mean:.2f} bits/weight)"
 
 
 def algorithmic_bytes(N, K, p, n, B):
@@ -143,26 +158,26 @@ def run_reference(args):
     import oracle
     from tests.golden import make_grids
 
-    p, n = (int(v) for v in args.grid.split(","))
     layers = inputs.LAYER_SETS[args.workload]
     cfg = inputs.CONFIG_OF_SET[args.workload]
+    pn, grid_text = layer_grids(args, layers, cfg)
     xi = inputs.rht_seed(cfg)
-    grid = make_grids.load(p, n)
+    grids = {k: make_grids.load(*k) for k in set(pn)}
     B = args.batch
     rows = 64  # rows of every layer per step: rows are independent, so this is a plain sample of the layer set
     sample = []
     for li, (name, N, K) in enumerate(layers):
         r = min(rows, N)
         W = inputs.make_weights(r, K, inputs.weight_seed(cfg, li), bf16=True).astype(np.float64)
-        q = oracle.quantize(W, G, grid, xi)
+        q = oracle.quantize(W, G, grids[pn[li]], xi)
         sc = oracle.round_scales_fp16(q.scales).astype(np.float64)
         x = inputs.make_activations(B, K, inputs.activation_seed(cfg, B) + li).astype(np.float64)
-        sample.append((q.codes, sc, x, r, K))
-    nbytes = sum(layer_bytes(r, K, p, n) for _, _, _, r, K in sample)
+        sample.append((q.codes, sc, x, r, K, pn[li]))
+    nbytes = sum(layer_bytes(r, K, *k) for _, _, _, r, K, k in sample)
 
     def step():
-        for codes, sc, x, r, K in sample:
-            oracle.linear_dense(x, codes, sc, G, grid, xi)
+        for codes, sc, x, r, K, k in sample:
+            oracle.linear_dense(x, codes, sc, G, grids[k], xi)
 
     for _ in range(args.warmup):
         step()
@@ -176,7 +191,7 @@ def run_reference(args):
         "impl": "reference", "metric": "higgs_linear_effective_weight_bandwidth", "value": value, "unit": "GB/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{args.workload} layer set, grid p={p} n={n}, g=1024, batch {B}", "sample": desc},
+        "config": {"workload": f"{args.workload} layer set, grid {grid_text}, g=1024, batch {B}", "sample": desc},
         "cpu_baseline": {"value": value, "unit": "GB/s", "cores": oracle.threads(), "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -201,9 +216,9 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    p, n = (int(v) for v in args.grid.split(","))
     layers = inputs.LAYER_SETS[args.workload]
     cfg = inputs.CONFIG_OF_SET[args.workload]
+    pn, grid_text = layer_grids(args, layers, cfg)
     xi = inputs.rht_seed(cfg)
     B = args.batch
 
@@ -211,27 +226,29 @@ def run_ours(args):
         return torch.cuda.Event(enable_timing=True)
 
     # ---- E0: grid fit on the device (Algorithm 2), 2^18 seeded Gaussian samples
-    samples = torch.from_numpy(inputs.gaussian_samples(p, inputs.grid_sample_seed(p, n)).astype(np.float32)).to(dev)
-    e0, e1 = ev(), ev()
-    e0.record()
-    grid, grid_mse, grid_iters = hb.higgs_make_grid(p, n, samples, max_iters=3000)
-    e1.record()
-    torch.cuda.synchronize()
-    grid_ms = e0.elapsed_time(e1)
-    del samples
+    grids, grid_ms, grid_iters, grid_mse = {}, 0.0, 0, 0.0
+    for (p, n) in sorted(set(pn)):
+        samples = torch.from_numpy(inputs.gaussian_samples(p, inputs.grid_sample_seed(p, n)).astype(np.float32)).to(dev)
+        e0, e1 = ev(), ev()
+        e0.record()
+        grids[(p, n)], grid_mse, grid_iters = hb.higgs_make_grid(p, n, samples, max_iters=3000)
+        e1.record()
+        torch.cuda.synchronize()
+        grid_ms += e0.elapsed_time(e1)
+        del samples
 
     # ---- E1-E4: encode every layer once on the device (Algorithm 1)
-    set_bytes = sum(layer_bytes(N, K, p, n) for _, N, K in layers)
+    set_bytes = sum(layer_bytes(N, K, *pn[li]) for li, (_, N, K) in enumerate(layers))
     copies = max(2, -(-2 * L2_BYTES // set_bytes))          # rotating copies so that no step finds its codes in L2
     copies = min(copies, 64)
     descs, packed, scales, xs, xs_host, ws, ys = [], [], [], [], [], [], []
     enc_ms, enc_weights = 0.0, 0
     for li, (name, N, K) in enumerate(layers):
-        d = hb.make_desc(p, n, N, K, xi)
+        d = hb.make_desc(pn[li][0], pn[li][1], N, K, xi)
         W = torch.from_numpy(inputs.make_weights(N, K, inputs.weight_seed(cfg, li), bf16=True)).to(dev).to(torch.bfloat16)
         e0, e1 = ev(), ev()
         e0.record()
-        pk, sc, _ = hb.higgs_quantize(d, W, grid)
+        pk, sc, _ = hb.higgs_quantize(d, W, grids[pn[li]])
         e1.record()
         torch.cuda.synchronize()
         enc_ms += e0.elapsed_time(e1)
@@ -270,16 +287,16 @@ def run_ours(args):
             if len(lis) > 1:
                 hb.higgs_rotate_activations(descs[lis[0]], xs[lis[0]], out=xdags[key])
                 for li in lis:
-                    hb.higgs_linear_prerotated(descs[li], xdags[key], packed[li][c], scales[li][c], grid, workspace=ws[li],
+                    hb.higgs_linear_prerotated(descs[li], xdags[key], packed[li][c], scales[li][c], grids[pn[li]], workspace=ws[li],
                                                y=ys[li], B=B)
             else:
                 li = lis[0]
-                hb.higgs_linear(descs[li], xs[li], packed[li][c], scales[li][c], grid, workspace=ws[li], y=ys[li])
+                hb.higgs_linear(descs[li], xs[li], packed[li][c], scales[li][c], grids[pn[li]], workspace=ws[li], y=ys[li])
 
     def step_host(i):
         c = i % copies
         for li, d in enumerate(descs):
-            hb.higgs_linear_host(d, xs_host[li], packed[li][c], scales[li][c], grid, ys_host[li], ws[li])
+            hb.higgs_linear_host(d, xs_host[li], packed[li][c], scales[li][c], grids[pn[li]], ys_host[li], ws[li])
         torch.cuda.current_stream().synchronize()   # the step's results are read on the host
 
     # ---- graphs: one per weight copy, replayed in rotation
@@ -348,7 +365,8 @@ def run_ours(args):
                                            torch.from_numpy(inputs.make_activations(Bk, d.K, 1)).to(torch.bfloat16).to(dev))
         yk = torch.empty((Bk, d.N), dtype=torch.float32, device=dev)
         wk = torch.empty(hb.higgs_workspace_bytes(d, hb.HIGGS_OP_LINEAR, Bk), dtype=torch.uint8, device=dev)
-        per_launch_bytes = layer_bytes(d.N, d.K, p, n)
+        per_launch_bytes = layer_bytes(d.N, d.K, d.p, d.n)
+        grid = grids[(d.p, d.n)]
         need = max(2, -(-2 * L2_BYTES // per_launch_bytes))
         pks = list(packed[li])
         scs = list(scales[li])
@@ -376,6 +394,7 @@ def run_ours(args):
         return a.elapsed_time(b) * 1e3 / (rounds * len(pks)), nodes   # microseconds per call
 
     us_big, nodes_big = kernel_time(big, db, B)
+    p, n = pn[big]
     alg = algorithmic_bytes(Nb, Kb, p, n, B)
     achieved = alg / (us_big * 1e-6) / 1e9
     traffic = None
@@ -405,11 +424,11 @@ def run_ours(args):
     if not args.no_detail and rank == 0:
         detail = {"layers": []}
         for li, (name, N, K) in enumerate(layers):
-            if any(l["shape"] == f"{N}x{K}" for l in detail["layers"]):
+            if any(l["shape"] == f"{N}x{K}" and l["grid"] == f"p={pn[li][0]} n={pn[li][1]}" for l in detail["layers"]):
                 continue
             us, _ = kernel_time(li, descs[li], B)
-            wb = layer_bytes(N, K, p, n)
-            detail["layers"].append({"name": name, "shape": f"{N}x{K}", "B": B, "us": round(us, 3),
+            wb = layer_bytes(N, K, *pn[li])
+            detail["layers"].append({"name": name, "shape": f"{N}x{K}", "grid": f"p={pn[li][0]} n={pn[li][1]}", "B": B, "us": round(us, 3),
                                      "weight_GBps": round(wb / us / 1e3, 1), "frac_of_measured": round(wb / us / 1e3 / peak, 4)})
         if B != 16:
             us16, _ = kernel_time(big, db, 16)
@@ -420,7 +439,8 @@ def run_ours(args):
     # ---- the same block with q/k/v and gate/up stored row-concatenated (rows are independent and the packed stream is
     # ordered by row tile, so the concatenation of the packed buffers IS the packed concatenated matrix): 4 products
     # and 4 rotations per block instead of 7 and 4.  Reported beside the per-layer launches, not instead of them.
-    if detail is not None and all(nm in names for nm in ("q", "k", "v", "gate", "up")):
+    if detail is not None and all(nm in names for nm in ("q", "k", "v", "gate", "up")) and len(set(pn)) == 1:
+        grid = grids[pn[0]]
         idx = {nm: names.index(nm) for nm in names}
         merged = [("qkv", [idx["q"], idx["k"], idx["v"]]), ("o", [idx["o"]]), ("gate_up", [idx["gate"], idx["up"]]),
                   ("down", [idx["down"]])]
@@ -473,13 +493,13 @@ def run_ours(args):
         for li, (name, N, K) in enumerate(layers):
             r = min(rows, N)
             W = inputs.make_weights(r, K, inputs.weight_seed(cfg, li), bf16=True).astype(np.float64)
-            g64 = grid.cpu().numpy().astype(np.float64)
+            g64 = grids[pn[li]].cpu().numpy().astype(np.float64)
             q = oracle.quantize(W, G, g64, xi)
-            smp.append((q.codes, oracle.round_scales_fp16(q.scales).astype(np.float64), xs_host[li].float().numpy().astype(np.float64), r, K))
-        nb = sum(layer_bytes(r, K, p, n) for *_, r, K in smp)
+            smp.append((q.codes, oracle.round_scales_fp16(q.scales).astype(np.float64), xs_host[li].float().numpy().astype(np.float64), g64, r, K, pn[li]))
+        nb = sum(layer_bytes(r, K, *k) for *_, r, K, k in smp)
         reps, t0 = 0, time.perf_counter()
         while reps < 3 or time.perf_counter() - t0 < 10.0:
-            for codes, sc, x, r, K in smp:
+            for codes, sc, x, g64, r, K, k in smp:
                 oracle.linear_dense(x, codes, sc, G, g64, xi)
             reps += 1
             if time.perf_counter() - t0 > 30.0:
@@ -493,7 +513,7 @@ def run_ours(args):
             "metric": "higgs_linear_effective_weight_bandwidth", "value": value, "unit": "GB/s", "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f16xf16->f32", "data": "synthetic",
-            "config": {"workload": f"{args.workload} layer set ({len(layers)} matrices), grid p={p} n={n}, g=1024, batch {B}",
+            "config": {"workload": f"{args.workload} layer set ({len(layers)} matrices), grid {grid_text}, g=1024, batch {B}",
                        "global_batch": B * world, "parallelism": f"replicas x{world}",
                        "l2": f"rotating {copies} weight copies ({copies * set_bytes / 1e6:.0f} MB > 126 MB L2)",
                        "launch": "direct" if graphs is None else "one CUDA graph per weight copy",

@@ -708,6 +708,19 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
         cfg.numAttrs = 2;
     }
     cfg.attrs = attr;
+    if (prm.ksplit > 1) {
+        // a cluster of `ksplit` blocks with this much shared memory must fit the device (it does on a full B200; a
+        // partitioned one may not): checked once per device and cluster size
+        static int cluster_ok[64][kTcMaxSplit + 1] = {};
+        if (dev >= 0 && dev < 64 && cluster_ok[dev][prm.ksplit] == 0) {
+            int n_clusters = 0;
+            const cudaError_t e = BN <= 32 ? cudaOccupancyMaxActiveClusters(&n_clusters, linear_tc_kernel<4>, &cfg)
+                                : BN <= 64 ? cudaOccupancyMaxActiveClusters(&n_clusters, linear_tc_kernel<2>, &cfg)
+                                           : cudaOccupancyMaxActiveClusters(&n_clusters, linear_tc_kernel<1>, &cfg);
+            cluster_ok[dev][prm.ksplit] = (e == cudaSuccess && n_clusters > 0) ? 1 : -1;
+        }
+        if (dev >= 0 && dev < 64 && cluster_ok[dev][prm.ksplit] < 0) return HIGGS_ERR_UNSUPPORTED;
+    }
     // activation-tile stage = FB steps of BN x 128 bytes, at most 16 KB for BN <= 128 (so that the code ring gets the
     // rest of shared memory) and 32 KB for wider tiles
     if (BN <= 32) return cuda_status(cudaLaunchKernelEx(&cfg, linear_tc_kernel<4>, prm, code_map));
