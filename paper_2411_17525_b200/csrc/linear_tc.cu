@@ -710,7 +710,7 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
     cfg.attrs = attr;
     if (prm.ksplit > 1) {
         // a cluster of `ksplit` blocks with this much shared memory must fit the device (it does on a full B200; a
-        // partitioned one may not): checked once per device and cluster size
+        // partitioned one may not, and then K is not split): checked once per device and cluster size
         static int cluster_ok[64][kTcMaxSplit + 1] = {};
         if (dev >= 0 && dev < 64 && cluster_ok[dev][prm.ksplit] == 0) {
             int n_clusters = 0;
@@ -719,7 +719,11 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
                                            : cudaOccupancyMaxActiveClusters(&n_clusters, linear_tc_kernel<1>, &cfg);
             cluster_ok[dev][prm.ksplit] = (e == cudaSuccess && n_clusters > 0) ? 1 : -1;
         }
-        if (dev >= 0 && dev < 64 && cluster_ok[dev][prm.ksplit] < 0) return HIGGS_ERR_UNSUPPORTED;
+        if (dev >= 0 && dev < 64 && cluster_ok[dev][prm.ksplit] < 0) {      // fall back to one block per tile
+            prm.ksplit = 1;
+            cfg.gridDim.z = 1;
+            cfg.numAttrs = 1;
+        }
     }
     // activation-tile stage = FB steps of BN x 128 bytes, at most 16 KB for BN <= 128 (so that the code ring gets the
     // rest of shared memory) and 32 KB for wider tiles
