@@ -63,7 +63,8 @@ constexpr int kTcBStages = 3;                // activation-tile stages in shared
 constexpr int kTcMaxCodeStages = 32;         // code stages in shared memory (4 KB each), below and above the table
 constexpr int kTcDequantWarps = 4 * kTcGroups;
 constexpr int kTcThreads = (3 + kTcDequantWarps) * 32;
-constexpr uint32_t kTcCodeStage = 4096;      // 128 rows x 64 inputs, one byte per input pair
+// a code stage: byte formats 128 rows x 64 inputs (4 KB, one step); six-bit format 128 rows x 128 inputs (6 KB, two steps:
+// its three bit planes cover two neighbouring 64-input blocks)
 constexpr uint32_t kTcWait = 1u << 22;
 // TMEM columns: [0, BN) accumulator; A stages of 128 columns (256 inputs) from column 128 (BN <= 128: three stages)
 // or 256 (two stages).
@@ -164,7 +165,7 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 
 // FB = 64-input steps per activation-tile stage (4, 2, 1 for BN <= 64, <= 128, <= 256: a stage is at most 32 KB).  It is a
 // template parameter so that the MMA warp's loop body is straight-line code.
-template <int FB>
+template <int FB, bool SIX>
 __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap code_map) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -190,6 +191,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
     const uint32_t d_full = bars + 8u * 80u;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_raw + 1024);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + 1032);
+    constexpr uint32_t kTcCodeStage = SIX ? 6144u : 4096u;
+    constexpr int SPS = SIX ? 2 : 1;                         // 64-input steps per code stage
     const uint32_t code0 = base + 2048u;
     const uint32_t b_stage_bytes = (uint32_t)FB * (uint32_t)prm.BN * 128u;
     const uint32_t code1 = lut + 65536u + (uint32_t)kTcBStages * b_stage_bytes;      // region B
@@ -247,16 +250,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
     asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(elected));
     if (warp == 0) {
         t_mbar_init(code_full(lane), 1);
-        t_mbar_init(code_empty(lane), 4);
+        t_mbar_init(code_empty(lane), 4 * SPS);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
         if (role == 0) {
-            const int n0 = ksteps < CS ? ksteps : CS;
+            const int nstage = ksteps / SPS;
+            const int n0 = nstage < CS ? nstage : CS;
             for (int j = 0; j < n0; ++j) {
                 if (elected) {
                     t_mbar_expect_tx(code_full(j), kTcCodeStage);
-                    t_tensor_load(code_stage(j), &code_map, (kstep0 + j) * 64, tile0, code_full(j));
+                    t_tensor_load(code_stage(j), &code_map, (kstep0 / SPS + j) * (int)(kTcCodeStage / 64u), tile0, code_full(j));
                 }
                 __syncwarp();
             }
@@ -301,11 +305,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
         int issued = code_issued;
         int s = issued == CS ? 0 : issued, it = issued == CS ? 1 : 0;
         uint32_t bad = 0;
-        for (int j = issued; j < ksteps; ++j) {
+        for (int j = issued; j < ksteps / SPS; ++j) {
             bad |= t_wait(code_empty(s), (uint32_t)((it & 1) ^ 1), t_limit(bad)) ^ 1u;
             if (elected) {
                 t_mbar_expect_tx(code_full(s), kTcCodeStage);
-                t_tensor_load(code_stage(s), &code_map, (kstep0 + j) * 64, tile0, code_full(s));
+                t_tensor_load(code_stage(s), &code_map, (kstep0 / SPS + j) * (int)(kTcCodeStage / 64u), tile0, code_full(s));
             }
             ++issued;
             const bool wrap = s + 1 == CS;
@@ -403,12 +407,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
         const int groups = (int)(prm.K / kGroup);
         const __half* sc_row = prm.scales + ((row0 / 16 + rtl) * groups) * 16 + (i & 15);
         const uint32_t t_lane = tmem + ((uint32_t)(32 * q) << 16);
-        const uint32_t code_off = (uint32_t)(rtl * 512 + g * 64);
+        // byte formats: this row's words are the 16-byte chunks of lanes (g, t) of its row tile; six-bit: word 2 (4g + t) +
+        // (step & 1) of each of the tile's three 256-byte planes
+        const uint32_t code_off = SIX ? (uint32_t)(rtl * 768 + g * 32 + (sg & 1) * 4) : (uint32_t)(rtl * 512 + g * 64);
+        const int tx = rtl & 1;                    // six-bit: odd row tiles visit the lanes t in the order t ^ 1 (bank conflicts)
         int cur_group = -1;
         uint32_t sc2 = 0;
         uint32_t bad = 0;
         int sa = 0, ua = 0;
-        int cs = sg % CS, ucs = 0;                 // code stage of step 4 S + sg and its use count (CS >= 4)
+        int cs = (sg / SPS) % CS, ucs = 0;         // code stage of step 4 S + sg and its use count (CS >= 4)
         for (int S = 0; S < nsuper; ++S) {
             const int jg = kstep0 + 4 * S + sg;    // 64-input step of the layer
             if (warp == 3) TTRACE(0, 4 * S);
@@ -420,19 +427,44 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
                 const __half2 s2 = __half2half2(sc);
                 sc2 = *reinterpret_cast<const uint32_t*>(&s2);
             }
-            // the row's codes of this step: the 16-byte chunks of lanes (g, t = 0..3) of row tile rtl; instruction jj
-            // reads chunk (jj + rot) & 3 so that the eight g of a warp hit eight different bank groups
-            uint4 c4[4];
+            uint4 c4[4];                           // c4[t] = the four index words (steps m = 0..3) of lane (g, t)
+            if (!SIX) {
+                // the 16-byte chunks of lanes (g, t = 0..3) of row tile rtl; instruction jj reads chunk (jj + rot) & 3
+                // so that the eight g of a warp hit eight different bank groups
 #pragma unroll
-            for (int jj = 0; jj < 4; ++jj)
-                c4[jj] = t_lds128(code_stage(cs) + code_off + (uint32_t)(((jj + rot) & 3) * 16));
+                for (int jj = 0; jj < 4; ++jj)
+                    c4[jj] = t_lds128(code_stage(cs) + code_off + (uint32_t)(((jj + rot) & 3) * 16));
+            } else {
+                uint32_t w0[4], w1[4], w2[4];
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const uint32_t addr = code_stage(cs) + code_off + (uint32_t)((t ^ tx) * 8);
+                    w0[t] = t_lds32(addr);
+                    w1[t] = t_lds32(addr + 256u);
+                    w2[t] = t_lds32(addr + 512u);
+                }
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    // low nibbles: slot 4m + a at bit 8a + 4(m & 1) of word m >> 1; high bit pairs: bit 8a + 2m of word 2.
+                    // (x & 0x0f0f0f0f) | (y & 0xf0f0f0f0): bits 6-7 of every byte are don't-care (the table repeats)
+                    uint32_t r0, r1, r2, r3;
+                    asm("lop3.b32 %0, %1, %2, 0x0f0f0f0f, 0xe4;" : "=r"(r0) : "r"(w0[t]), "r"(w2[t] << 4));
+                    asm("lop3.b32 %0, %1, %2, 0x0f0f0f0f, 0xe4;" : "=r"(r1) : "r"(w0[t] >> 4), "r"(w2[t] << 2));
+                    asm("lop3.b32 %0, %1, %2, 0x0f0f0f0f, 0xe4;" : "=r"(r2) : "r"(w1[t]), "r"(w2[t]));
+                    asm("lop3.b32 %0, %1, %2, 0x0f0f0f0f, 0xe4;" : "=r"(r3) : "r"(w1[t] >> 4), "r"(w2[t] >> 2));
+                    c4[t] = make_uint4(r0, r1, r2, r3);
+                }
+                if (tx) { uint4 t0 = c4[0]; c4[0] = c4[1]; c4[1] = t0; t0 = c4[2]; c4[2] = c4[3]; c4[3] = t0; }
+            }
             __syncwarp();
             if (lane == 0) t_mbar_arrive(code_empty(cs));     // the code words are in registers: hand the stage back
-            cs += 4;
+            cs += 4 / SPS;
             if (cs >= CS) { cs -= CS; ++ucs; }
             // undo the rotation: chunk t was loaded by instruction (t - rot) & 3
-            if (rot & 1) { const uint4 t0 = c4[0]; c4[0] = c4[3]; c4[3] = c4[2]; c4[2] = c4[1]; c4[1] = t0; }
-            if (rot & 2) { uint4 t0 = c4[0]; c4[0] = c4[2]; c4[2] = t0; t0 = c4[1]; c4[1] = c4[3]; c4[3] = t0; }
+            if (!SIX) {
+                if (rot & 1) { const uint4 t0 = c4[0]; c4[0] = c4[3]; c4[3] = c4[2]; c4[2] = c4[1]; c4[1] = t0; }
+                if (rot & 2) { uint4 t0 = c4[0]; c4[0] = c4[2]; c4[2] = t0; t0 = c4[1]; c4[1] = c4[3]; c4[3] = t0; }
+            }
             uint32_t a[32];
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
@@ -597,11 +629,11 @@ int tc_batch_tile(int64_t B) {
     return (int)((per + 15) / 16 * 16);
 }
 
-// The tensor-core path takes byte-coded layers whose row count is a multiple of 128: every batch above 16, and batches
+// The tensor-core path takes layers whose row count is a multiple of 128: every batch above 16, and batches
 // 9..16 of large layers (there the small-batch kernel is limited by the legacy mma.sync rate, two per lookup group;
 // measured cross-over near 32 M weights).
 bool tc_eligible(const higgs_desc& d, int64_t B) {
-    if (!(d.N % 128 == 0 && d.N > 0 && format_of(d.p, d.n) == Format::kByteLut)) return false;
+    if (!(d.N % 128 == 0 && d.N > 0 && format_of(d.p, d.n) != Format::kNone)) return false;
     return B > 16 || (B > 8 && d.N * d.K >= ((int64_t)1 << 25));
 }
 
@@ -654,9 +686,12 @@ EncodeTiledFn encode_tiled_fn() {
 bool make_code_map(const higgs_desc& d, const void* packed, CUtensorMap* map) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)d.K, (cuuint64_t)(d.N / 16)};
-    const cuuint64_t strides[1] = {(cuuint64_t)d.K * 8};
-    const cuuint32_t box[2] = {64, 8};
+    // byte formats: K x 8 bytes per row tile, a stage is one 512-byte block; six-bit: K x 6 bytes, a stage is one 768-byte
+    // super-block (three bit planes of two neighbouring blocks)
+    const bool six = format_of(d.p, d.n) == Format::kSixBit;
+    const cuuint64_t dims[2] = {(cuuint64_t)(six ? d.K * 6 / 8 : d.K), (cuuint64_t)(d.N / 16)};
+    const cuuint64_t strides[1] = {(cuuint64_t)(six ? d.K * 6 : d.K * 8)};
+    const cuuint32_t box[2] = {six ? 96u : 64u, 8};
     const cuuint32_t estr[2] = {1, 1};
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_INT64, 2, const_cast<void*>(packed), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -674,10 +709,11 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        if (cudaFuncSetAttribute(linear_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem) != cudaSuccess ||
-            cudaFuncSetAttribute(linear_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem) != cudaSuccess ||
-            cudaFuncSetAttribute(linear_tc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem) != cudaSuccess)
-            return HIGGS_ERR_CUDA;
+        const void* kernels[6] = {(const void*)linear_tc_kernel<1, false>, (const void*)linear_tc_kernel<2, false>,
+                                  (const void*)linear_tc_kernel<4, false>, (const void*)linear_tc_kernel<1, true>,
+                                  (const void*)linear_tc_kernel<2, true>, (const void*)linear_tc_kernel<4, true>};
+        for (const void* k : kernels)
+            if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem) != cudaSuccess) return HIGGS_ERR_CUDA;
         configured[dev] = true;
     }
     CUtensorMap code_map;
@@ -708,15 +744,20 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
         cfg.numAttrs = 2;
     }
     cfg.attrs = attr;
+    // activation-tile stage = FB steps of BN x 128 bytes, at most 16 KB for BN <= 128 (so that the code ring gets the
+    // rest of shared memory) and 32 KB for wider tiles
+    const bool six = format_of(d.p, d.n) == Format::kSixBit;
+    void (*kernel)(const TcParams, const CUtensorMap) =
+        BN <= 32 ? (six ? linear_tc_kernel<4, true> : linear_tc_kernel<4, false>)
+      : BN <= 64 ? (six ? linear_tc_kernel<2, true> : linear_tc_kernel<2, false>)
+                 : (six ? linear_tc_kernel<1, true> : linear_tc_kernel<1, false>);
     if (prm.ksplit > 1) {
         // a cluster of `ksplit` blocks with this much shared memory must fit the device (it does on a full B200; a
         // partitioned one may not, and then K is not split): checked once per device and cluster size
         static int cluster_ok[64][kTcMaxSplit + 1] = {};
         if (dev >= 0 && dev < 64 && cluster_ok[dev][prm.ksplit] == 0) {
             int n_clusters = 0;
-            const cudaError_t e = BN <= 32 ? cudaOccupancyMaxActiveClusters(&n_clusters, linear_tc_kernel<4>, &cfg)
-                                : BN <= 64 ? cudaOccupancyMaxActiveClusters(&n_clusters, linear_tc_kernel<2>, &cfg)
-                                           : cudaOccupancyMaxActiveClusters(&n_clusters, linear_tc_kernel<1>, &cfg);
+            const cudaError_t e = cudaOccupancyMaxActiveClusters(&n_clusters, kernel, &cfg);
             cluster_ok[dev][prm.ksplit] = (e == cudaSuccess && n_clusters > 0) ? 1 : -1;
         }
         if (dev >= 0 && dev < 64 && cluster_ok[dev][prm.ksplit] < 0) {      // fall back to one block per tile
@@ -725,11 +766,7 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
             cfg.numAttrs = 1;
         }
     }
-    // activation-tile stage = FB steps of BN x 128 bytes, at most 16 KB for BN <= 128 (so that the code ring gets the
-    // rest of shared memory) and 32 KB for wider tiles
-    if (BN <= 32) return cuda_status(cudaLaunchKernelEx(&cfg, linear_tc_kernel<4>, prm, code_map));
-    if (BN <= 64) return cuda_status(cudaLaunchKernelEx(&cfg, linear_tc_kernel<2>, prm, code_map));
-    return cuda_status(cudaLaunchKernelEx(&cfg, linear_tc_kernel<1>, prm, code_map));
+    return cuda_status(cudaLaunchKernelEx(&cfg, kernel, prm, code_map));
 }
 
 #ifdef HIGGS_TRACE

@@ -242,6 +242,10 @@ def test_dequantize_matches_oracle(p, n, N, K):
     (2, 256, 256, 1024, 300),    # two token tiles
     (2, 256, 8448, 1024, 40),    # 66 row tiles: K is not split
     (2, 256, 4096, 3072, 24),    # two K slices of 1536 inputs: the boundary falls inside a scale group
+    (2, 64, 128, 2048, 20),      # six-bit format: bit planes rebuilt into index words by the dequant warps
+    (2, 64, 384, 4096, 100),
+    (2, 64, 8448, 1024, 40),     # six-bit, K not split
+    (2, 64, 256, 1024, 300),
 ])
 def test_linear_tensor_core_path_matches_oracle(p, n, N, K, B):
     y, y_ref = run_linear_case(p, n, N, K, B, xi=inputs.rht_seed(3), wseed=300 + N, xseed=400 + B, lognormal=(B == 64))
