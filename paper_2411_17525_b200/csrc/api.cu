@@ -40,7 +40,8 @@ int higgs_sign(uint64_t rht_seed, int64_t j) { return sign_bit(rht_seed, j) ? -1
 size_t higgs_packed_bytes(const higgs_desc* d) {
     if (check_desc(d) != HIGGS_OK) return 0;
     const size_t pairs = (size_t)d->N * (size_t)d->K / 2;
-    return format_of(d->p, d->n) == Format::kSixBit ? pairs / 4 * 3 : pairs;
+    const Format f = format_of(d->p, d->n);
+    return f == Format::kSixBit ? pairs / 4 * 3 : f == Format::kNibble ? pairs / 2 : pairs;
 }
 
 size_t higgs_scales_bytes(const higgs_desc* d) {

@@ -31,13 +31,16 @@ __host__ __device__ __forceinline__ uint32_t sign_bit(uint64_t xi, int64_t j) {
 //              p=2,n=256: the byte is the code.  p=1,n=16: the byte holds the
 //              codes of k (low nibble) and k+1 (high nibble).
 //   kSixBit  : p=2,n=64: 6-bit codes, low nibbles and high bit-pairs in
-//              separate planes (bit slices), see pack.cu.
-enum class Format : int { kNone = 0, kByteLut = 1, kSixBit = 2 };
+//              separate planes (bit slices), see quantize.cu.
+//   kNibble  : p=2,n=16: 4-bit codes, two per byte; the byte looks up an 8-byte
+//              table entry (the fp16 pairs of both codes = two A-fragment registers).
+enum class Format : int { kNone = 0, kByteLut = 1, kSixBit = 2, kNibble = 3 };
 
 __host__ __device__ inline Format format_of(int p, int n) {
     if (p == 2 && n == 256) return Format::kByteLut;
     if (p == 1 && n == 16) return Format::kByteLut;
     if (p == 2 && n == 64) return Format::kSixBit;
+    if (p == 2 && n == 16) return Format::kNibble;
     return Format::kNone;
 }
 

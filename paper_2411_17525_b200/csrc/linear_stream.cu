@@ -74,14 +74,16 @@ constexpr int kWarps = 16;
 constexpr int kMaxDepth = 8;            // ring slots per warp
 constexpr int kMaxAccSlots = 32;        // items whose partial tiles may be parked at once
 constexpr uint32_t kWaitLimit = 1u << 22;
+constexpr uint32_t kNibbleTileBytes = 32768; // nibble format: the table rows are full, the partial tiles live at the end of shared memory
 constexpr uint32_t kAssumedBase = 1024; // offset of the dynamic shared-memory window the host plans the rings for
 
 // Ring layout for a window starting at `base`: table position, depth D and the number of warps whose D slots fit
 // below the table (the others' lie above it).
-__host__ __device__ inline void ring_layout(uint32_t base, uint32_t slot_bytes, uint32_t* lut_out, int* depth_out, int* warps_in_a_out) {
+__host__ __device__ inline void ring_layout(uint32_t base, uint32_t slot_bytes, uint32_t tail_reserve, uint32_t* lut_out, int* depth_out,
+                                            int* warps_in_a_out) {
     const uint32_t lut = (base + kSmallBytes + 0xffffu) & ~0xffffu;
     const int nA = (int)((lut - (base + kSmallBytes)) / slot_bytes);
-    const int nB = (int)((base + kMaxDynSmem - (lut + kLutBytes)) / slot_bytes);
+    const int nB = (int)((base + kMaxDynSmem - tail_reserve - (lut + kLutBytes)) / slot_bytes);
     int D = kMaxDepth;
     while (D > 1 && nA / D + nB / D < kWarps) --D;
     *lut_out = lut;
@@ -98,6 +100,11 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr) {
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
     asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint2 lds64_table(uint32_t addr) {
+    uint2 v;
+    asm("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));   // table is read-only after the prologue
     return v;
 }
 __device__ __forceinline__ uint2 lds64(uint32_t addr) {
@@ -172,10 +179,13 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 }
 
 // Code words of one task (16 rows x KS inputs) for this lane, read from a ring slot.
-template <int KS, bool SIX>
+// FMT: 0 = byte format (one byte = one table index = one A-fragment register), 1 = six-bit planes, 2 = nibble pairs
+// (p=2 n=16: one byte = two 4-bit codes = an 8-byte table entry = two A-fragment registers).
+template <int KS, int FMT>
 struct TaskCodes {
-    static constexpr int kWords = SIX ? (KS / 128) * 6 : (KS / 64) * 4;
-    static constexpr uint32_t kBytes = SIX ? KS * 6 : KS * 8;   // bytes of one task in the packed stream
+    static constexpr bool SIX = FMT == 1, NIB = FMT == 2;
+    static constexpr int kWords = SIX ? (KS / 128) * 6 : NIB ? (KS / 64) * 2 : (KS / 64) * 4;
+    static constexpr uint32_t kBytes = SIX ? KS * 6 : NIB ? KS * 4 : KS * 8;   // bytes of one task in the packed stream
     uint32_t w[kWords];
     __device__ __forceinline__ void load(uint32_t slot, int lane) {
         if (SIX) {
@@ -188,6 +198,12 @@ struct TaskCodes {
                     w[sb * 6 + pl * 2 + 1] = q.y;
                 }
             }
+        } else if (NIB) {
+#pragma unroll
+            for (int j = 0; j < KS / 64; ++j) {
+                uint2 q = lds64(slot + (uint32_t)(j * 256 + lane * 8));
+                w[j * 2] = q.x; w[j * 2 + 1] = q.y;
+            }
         } else {
 #pragma unroll
             for (int j = 0; j < KS / 64; ++j) {
@@ -196,8 +212,10 @@ struct TaskCodes {
             }
         }
     }
-    // four byte-aligned table indices (slots 4m..4m+3) of 64-input block j, step m
+    // four byte-aligned table indices (slots 4m..4m+3) of 64-input block j, step m.  Nibble format: the word holding
+    // the two bytes of step m (bytes 2(m&1) and 2(m&1)+1 of word m >> 1).
     __device__ __forceinline__ uint32_t index_word(int j, int m) const {
+        if (NIB) return w[j * 2 + (m >> 1)];
         if (!SIX) return w[j * 4 + m];
         const int sb = j >> 1, h = j & 1;
         const uint32_t lo = w[sb * 6 + (m >> 1) * 2 + h];
@@ -211,34 +229,38 @@ struct TaskCodes {
     }
 };
 
-template <int NB, int KS, bool SIX>
+template <int NB, int KS, int FMT>
 __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(const StreamParams prm) {
+    constexpr bool SIX = FMT == 1, NIB = FMT == 2;
+    constexpr uint32_t kPieceStride = NIB ? 128u : 256u;     // bytes between consecutive 128-byte pieces of the partial tiles
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3;
-    using Codes = TaskCodes<KS, SIX>;
+    using Codes = TaskCodes<KS, FMT>;
 
-    // ---- shared memory map (all offsets derived from the runtime base address) ----
-    //   [base, base+4 KB)    ring mbarriers (0..1023), item mbarriers and
-    //                        recycle counters of the partial-tile slots (2048..2559), abort flag (2560)
-    //   [base+4 KB, lut)     ring slots, region A
-    //   [lut, lut+64 KB)     table rows of 256 B: bytes 0..127 = the entry replicated per lane,
-    //                        bytes 128..255 = one 32-float piece of an accumulator tile
-    //   [lut+64 KB, end)     ring slots, region B
     TRACEP(warp, 0);
     if (warp == 0) BTRACE(0);
     // ---- the table's source first: the grid loads are in flight while everything below is set up ----
     // Table: entry(idx) replicated once per lane (bank = lane): conflict-free gathers.  Warp w fills rows
     // 4 (w + 17 r) .. + 3; a row's 128 bytes are written by eight lanes with one 16-byte store each, and the loads
     // of a warp are independent, so the whole build costs one global round trip.  (The grid is a constant of the layer.)
-    constexpr int kQuadsPerWarp = (64 + kWarps) / (kWarps + 1);     // 4 groups of four rows for 17 warps
-    float ent_lo[kQuadsPerWarp], ent_hi[kQuadsPerWarp];
+    // Nibble format: an entry is 8 bytes (the pairs of the low and the high nibble), a row is 32 lanes x 8 B = 256 B,
+    // and one 16-byte store per lane covers two rows.
+    constexpr int kRowsPerStore = NIB ? 2 : 4;
+    constexpr int kStoresPerWarp = (256 / kRowsPerStore + kWarps) / (kWarps + 1);     // 4 (8 for the nibble format) for 17 warps
+    float ent_lo[kStoresPerWarp], ent_hi[kStoresPerWarp], ent_lo2[NIB ? kStoresPerWarp : 1], ent_hi2[NIB ? kStoresPerWarp : 1];
 #pragma unroll
-    for (int r = 0; r < kQuadsPerWarp; ++r) {
-        const int idx = 4 * (warp + r * (kWarps + 1)) + (lane >> 3);      // this lane's row: 8 lanes x 16 B fill one
+    for (int r = 0; r < kStoresPerWarp; ++r) {
+        // this lane's row: 8 (16) lanes x 16 B fill one
+        const int idx = kRowsPerStore * (warp + r * (kWarps + 1)) + (NIB ? (lane >> 4) : (lane >> 3));
         ent_lo[r] = 0.f; ent_hi[r] = 0.f;
+        if (NIB) { ent_lo2[r] = 0.f; ent_hi2[r] = 0.f; }
         if (idx < 256) {
-            if (prm.p == 2) {
+            if (NIB) {
+                const float2 g0 = __ldg(reinterpret_cast<const float2*>(prm.grid) + (idx & 15));
+                const float2 g1 = __ldg(reinterpret_cast<const float2*>(prm.grid) + (idx >> 4));
+                ent_lo[r] = g0.x; ent_hi[r] = g0.y; ent_lo2[r] = g1.x; ent_hi2[r] = g1.y;
+            } else if (prm.p == 2) {
                 const float2 gp = __ldg(reinterpret_cast<const float2*>(prm.grid) + (idx & (prm.n - 1)));
                 ent_lo[r] = gp.x; ent_hi[r] = gp.y;
             } else {
@@ -259,7 +281,8 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     constexpr uint32_t kSlotBytes = Codes::kBytes + 64u;       // codes + 16 fp16 scales (padded)
     uint32_t lut = (kAssumedBase + kSmallBytes + 0xffffu) & ~0xffffu;   // 64 KB aligned: byte 1 of an address is free for the code
     int D = prm.depth, warps_in_A = prm.warps_in_a;
-    if (base != kAssumedBase) ring_layout(base, kSlotBytes, &lut, &D, &warps_in_A);
+    constexpr uint32_t kTailReserve = NIB ? kNibbleTileBytes : 0u;
+    if (base != kAssumedBase) ring_layout(base, kSlotBytes, kTailReserve, &lut, &D, &warps_in_A);
     const uint32_t bars = base;
     const uint32_t item_bars = base + 2048u;                                        // [kMaxAccSlots] mbarriers, NS arrivals each
     volatile int* recycled = reinterpret_cast<volatile int*>(smem_raw + 2048 + 8 * kMaxAccSlots);   // [kMaxAccSlots] generations
@@ -297,8 +320,8 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     const int tile_pieces = prm.tile_pieces;
     const int acc_slots = prm.acc_slots;
     const int acc_shift = prm.acc_shift;
-    const uint32_t part0 = lut + 128u;
-    const uint32_t tile_stride = (uint32_t)tile_pieces * 256u;         // bytes between consecutive tiles
+    const uint32_t part0 = NIB ? base + kMaxDynSmem - kNibbleTileBytes : lut + 128u;
+    const uint32_t tile_stride = (uint32_t)tile_pieces * kPieceStride; // bytes between consecutive tiles
     const uint32_t q_stride = tile_stride << log_ns;                   // bytes between consecutive item slots
 
     // ---- ring barriers, then the first copies ----
@@ -321,9 +344,9 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     const int64_t kslice = (int64_t)chunk_begin * prm.ck + (int64_t)slice * KS;
     const int64_t rt_first = rt_begin + phase;
     const uint8_t* src_next = prm.packed + (SIX ? ((rt_first * (prm.K >> 7) + (kslice >> 7)) * 768)
-                                                : ((rt_first * (prm.K >> 6) + (kslice >> 6)) * 512));
+                                                : ((rt_first * (prm.K >> 6) + (kslice >> 6)) * (NIB ? 256 : 512)));
     const __half* ssrc_next = prm.scales + (rt_first * groups + chunk_begin * ng + gl) * 16;
-    const int64_t src_stride = (int64_t)PG * (SIX ? prm.K * 6 : prm.K * 8);
+    const int64_t src_stride = (int64_t)PG * (SIX ? prm.K * 6 : NIB ? prm.K * 4 : prm.K * 8);
     const int64_t ssrc_stride = (int64_t)PG * groups * 16;
     uint32_t elected;
     asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(elected));
@@ -383,12 +406,18 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
 
     {
 #pragma unroll
-        for (int r = 0; r < kQuadsPerWarp; ++r) {
-            const int idx = 4 * (warp + r * (kWarps + 1)) + (lane >> 3);
+        for (int r = 0; r < kStoresPerWarp; ++r) {
+            const int idx = kRowsPerStore * (warp + r * (kWarps + 1)) + (NIB ? (lane >> 4) : (lane >> 3));
             __half2 h = __floats2half2_rn(ent_lo[r], ent_hi[r]);
             const uint32_t e = *reinterpret_cast<uint32_t*>(&h);
-            if (idx < 256)
+            if (NIB) {
+                __half2 h2 = __floats2half2_rn(ent_lo2[r], ent_hi2[r]);
+                const uint32_t e2 = *reinterpret_cast<uint32_t*>(&h2);
+                if (idx < 256)
+                    *reinterpret_cast<uint4*>(smem_raw + (lut - base) + idx * 256 + (lane & 15) * 16) = make_uint4(e, e2, e, e2);
+            } else if (idx < 256) {
                 *reinterpret_cast<uint4*>(smem_raw + (lut - base) + idx * 256 + (lane & 7) * 16) = make_uint4(e, e, e, e);
+            }
         }
     }
     TRACEP(warp, 5);
@@ -416,7 +445,7 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
 #pragma unroll
                     for (int ns = 0; ns < 16; ++ns)
                         raw[ns] = lds128(part0 + (uint32_t)q * q_stride + (uint32_t)(ns < NS ? ns : 0) * tile_stride +
-                                         (uint32_t)((e >> 5) * 256 + (e & 31) * 4));
+                                         (uint32_t)(e >> 5) * kPieceStride + (uint32_t)((e & 31) * 4));
                     float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                     for (int ns = 0; ns < 16; ++ns) {
@@ -463,8 +492,8 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     }
 
     // ---- main loop: this warp's tasks ----
-    const uint32_t lut_lane = lut + lane * 4;
-    const uint32_t part_lane = part0 + (uint32_t)slice * tile_stride + (uint32_t)(t * 256 + g * 4);
+    const uint32_t lut_lane = lut + lane * (NIB ? 8 : 4);
+    const uint32_t part_lane = part0 + (uint32_t)slice * tile_stride + (uint32_t)t * kPieceStride + (uint32_t)(g * 4);
     int d = 0;
     uint32_t ph = 0;
     bool ok = true;
@@ -496,10 +525,18 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
                 const uint32_t iw = codes.index_word(jb, m);
-                const uint32_t a0 = lds32(__byte_perm(iw, lut_lane, 0x7604));
-                const uint32_t a1 = lds32(__byte_perm(iw, lut_lane, 0x7614));
-                const uint32_t a2 = lds32(__byte_perm(iw, lut_lane, 0x7624));
-                const uint32_t a3 = lds32(__byte_perm(iw, lut_lane, 0x7634));
+                uint32_t a0, a1, a2, a3;
+                if (NIB) {
+                    // one byte = the codes of registers (a0, a1) resp. (a2, a3): one 8-byte lookup each
+                    const uint2 p01 = lds64_table(__byte_perm(iw, lut_lane, (m & 1) ? 0x7624 : 0x7604));
+                    const uint2 p23 = lds64_table(__byte_perm(iw, lut_lane, (m & 1) ? 0x7634 : 0x7614));
+                    a0 = p01.x; a1 = p01.y; a2 = p23.x; a3 = p23.y;
+                } else {
+                    a0 = lds32(__byte_perm(iw, lut_lane, 0x7604));
+                    a1 = lds32(__byte_perm(iw, lut_lane, 0x7614));
+                    a2 = lds32(__byte_perm(iw, lut_lane, 0x7624));
+                    a3 = lds32(__byte_perm(iw, lut_lane, 0x7634));
+                }
 #pragma unroll
                 for (int nb = 0; nb < NB; ++nb) {
                     if (jb == 0) mma16816_first(acc4[m][nb], a0, a1, a2, a3, bfrag[m][nb][0], bfrag[m][nb][1]);
@@ -530,12 +567,12 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
             const float v2 = (acc4[0][nb][2] + acc4[1][nb][2]) + (acc4[2][nb][2] + acc4[3][nb][2]);
             const float v3 = (acc4[0][nb][3] + acc4[1][nb][3]) + (acc4[2][nb][3] + acc4[3][nb][3]);
             if (c0 < prm.B) {                        // only the B valid columns exist
-                asm volatile("st.shared.f32 [%0], %1;" ::"r"(pa + (uint32_t)(nb * 1024)), "f"(v0 * s_lo) : "memory");
-                asm volatile("st.shared.f32 [%0], %1;" ::"r"(pa + (uint32_t)(nb * 1024 + 32)), "f"(v2 * s_hi) : "memory");
+                asm volatile("st.shared.f32 [%0], %1;" ::"r"(pa + (uint32_t)(nb * 4) * kPieceStride), "f"(v0 * s_lo) : "memory");
+                asm volatile("st.shared.f32 [%0], %1;" ::"r"(pa + (uint32_t)(nb * 4) * kPieceStride + 32u), "f"(v2 * s_hi) : "memory");
             }
             if (c0 + 1 < prm.B) {
-                asm volatile("st.shared.f32 [%0], %1;" ::"r"(pa + (uint32_t)(nb * 1024 + 64)), "f"(v1 * s_lo) : "memory");
-                asm volatile("st.shared.f32 [%0], %1;" ::"r"(pa + (uint32_t)(nb * 1024 + 96)), "f"(v3 * s_hi) : "memory");
+                asm volatile("st.shared.f32 [%0], %1;" ::"r"(pa + (uint32_t)(nb * 4) * kPieceStride + 64u), "f"(v1 * s_lo) : "memory");
+                asm volatile("st.shared.f32 [%0], %1;" ::"r"(pa + (uint32_t)(nb * 4) * kPieceStride + 96u), "f"(v3 * s_hi) : "memory");
             }
         }
         __syncwarp();
@@ -609,18 +646,18 @@ Plan make_plan(const higgs_desc& d, int64_t B) {
     return best;
 }
 
-template <int NB, int KS, bool SIX>
+template <int NB, int KS, int FMT>
 int launch_one(const StreamParams& prm, int blocks, cudaStream_t st) {
     static bool configured[64] = {false};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(linear_stream_kernel<NB, KS, SIX>,
+        cudaError_t e = cudaFuncSetAttribute(linear_stream_kernel<NB, KS, FMT>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem);
         if (e != cudaSuccess) return HIGGS_ERR_CUDA;
         configured[dev] = true;
     }
-    return cuda_status(launch_pdl(linear_stream_kernel<NB, KS, SIX>, dim3((unsigned)blocks), dim3((kWarps + 1) * 32),
+    return cuda_status(launch_pdl(linear_stream_kernel<NB, KS, FMT>, dim3((unsigned)blocks), dim3((kWarps + 1) * 32),
                                   kMaxDynSmem, st, prm));
 }
 
@@ -646,7 +683,8 @@ int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const 
     prm.n = d.n; prm.p = d.p;
     prm.ck = pl.ck;
     prm.y_mode = y_mode;
-    const bool six = format_of(d.p, d.n) == Format::kSixBit;
+    const Format fmt = format_of(d.p, d.n);
+    const bool six = fmt == Format::kSixBit, nib = fmt == Format::kNibble;
     prm.parts = pl.parts;
     prm.parts_shift = 0;
     while ((1 << prm.parts_shift) < pl.parts) ++prm.parts_shift;
@@ -661,11 +699,12 @@ int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const 
     prm.acc_shift = 0;
     while ((1 << prm.acc_shift) < p2) ++prm.acc_shift;
     uint32_t lut_unused;
-    ring_layout(kAssumedBase, (uint32_t)(six ? pl.ks * 6 : pl.ks * 8) + 64u, &lut_unused, &prm.depth, &prm.warps_in_a);
-    if (pl.nb == 1 && !six) return launch_one<1, 256, false>(prm, pl.blocks, st);
-    if (pl.nb == 2 && !six) return launch_one<2, 128, false>(prm, pl.blocks, st);
-    if (pl.nb == 1 && six) return launch_one<1, 256, true>(prm, pl.blocks, st);
-    return launch_one<2, 128, true>(prm, pl.blocks, st);
+    ring_layout(kAssumedBase, (uint32_t)(six ? pl.ks * 6 : nib ? pl.ks * 4 : pl.ks * 8) + 64u, nib ? kNibbleTileBytes : 0u, &lut_unused,
+                &prm.depth, &prm.warps_in_a);
+    if (pl.nb == 1) return six ? launch_one<1, 256, 1>(prm, pl.blocks, st) : nib ? launch_one<1, 256, 2>(prm, pl.blocks, st)
+                                                                               : launch_one<1, 256, 0>(prm, pl.blocks, st);
+    return six ? launch_one<2, 128, 1>(prm, pl.blocks, st) : nib ? launch_one<2, 128, 2>(prm, pl.blocks, st)
+                                                               : launch_one<2, 128, 0>(prm, pl.blocks, st);
 }
 
 int launch_convert_out(const float* y32, void* y, int y_dtype, size_t count, cudaStream_t st) {

@@ -633,7 +633,8 @@ int tc_batch_tile(int64_t B) {
 // 9..16 of large layers (there the small-batch kernel is limited by the legacy mma.sync rate, two per lookup group;
 // measured cross-over near 32 M weights).
 bool tc_eligible(const higgs_desc& d, int64_t B) {
-    if (!(d.N % 128 == 0 && d.N > 0 && format_of(d.p, d.n) != Format::kNone)) return false;
+    const Format f = format_of(d.p, d.n);
+    if (!(d.N % 128 == 0 && d.N > 0 && (f == Format::kByteLut || f == Format::kSixBit))) return false;
     return B > 16 || (B > 8 && d.N * d.K >= ((int64_t)1 << 25));
 }
 

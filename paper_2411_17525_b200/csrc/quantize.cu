@@ -138,6 +138,9 @@ __global__ void __launch_bounds__(128) encode_kernel(const T* __restrict__ W, co
 //                    Word 2 holds the high bit-pairs: slot 4m+a at bit 8a + 2m.
 //                    (The consumer rebuilds four byte-aligned indices with one shift
 //                    and one three-input logic operation each, see linear_mma.cu.)
+//   nibble format  : (n = 16) two 32-bit words per lane and block, 256 bytes per block, lane L at
+//                    byte offset 8 L.  Byte 2m + h of the lane holds the slots 4m + 2h (low
+//                    nibble) and 4m + 2h + 1 (high nibble): the two registers of one row pair.
 //                    Two neighbouring blocks (2j, 2j+1 along K) form a 768-byte
 //                    super-block of three 256-byte planes; plane w stores word w of
 //                    lane L, block half h at 32-bit index 2L + h, so a warp reads
@@ -173,7 +176,7 @@ __device__ __forceinline__ int64_t six_bit_word(int64_t rt, int64_t kb, int64_t 
     return ((rt * (kblocks >> 1) + (kb >> 1)) * 3 + w) * 64 + 2 * L + (kb & 1);
 }
 
-template <int P, bool SIX>
+template <int P, int FMT>
 __global__ void __launch_bounds__(256) pack_kernel(const uint8_t* __restrict__ canonical, uint32_t* __restrict__ packed,
                                                    int64_t N, int64_t K) {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -182,6 +185,7 @@ __global__ void __launch_bounds__(256) pack_kernel(const uint8_t* __restrict__ c
     if (t >= total) return;
     const int L = (int)(t & 31);
     const int64_t blk = t >> 5, rt = blk / kblocks, kb = blk % kblocks;
+    constexpr bool SIX = FMT == 1, NIB = FMT == 2;
     if (SIX) {
         uint32_t w[3] = {0u, 0u, 0u};
         for (int s = 0; s < 16; ++s) {
@@ -190,6 +194,15 @@ __global__ void __launch_bounds__(256) pack_kernel(const uint8_t* __restrict__ c
             six_bit_store(w, s, pair_index<P>(canonical, K, row, pair) & 63u);
         }
         for (int i = 0; i < 3; ++i) packed[six_bit_word(rt, kb, kblocks, L, i)] = w[i];
+    } else if (NIB) {
+        uint32_t w[2] = {0u, 0u};
+        for (int s = 0; s < 16; ++s) {
+            int64_t row, pair;
+            slot_coords(rt, kb, L, s, row, pair);
+            const int m = s >> 2, a = s & 3, byte = 2 * m + (a >> 1);
+            w[byte >> 2] |= (pair_index<P>(canonical, K, row, pair) & 15u) << (8 * (byte & 3) + 4 * (a & 1));
+        }
+        reinterpret_cast<uint2*>(packed)[t] = make_uint2(w[0], w[1]);
     } else {
         uint32_t w[4] = {0u, 0u, 0u, 0u};
         for (int s = 0; s < 16; ++s) {
@@ -201,7 +214,7 @@ __global__ void __launch_bounds__(256) pack_kernel(const uint8_t* __restrict__ c
     }
 }
 
-template <int P, bool SIX>
+template <int P, int FMT>
 __global__ void __launch_bounds__(256) unpack_kernel(const uint32_t* __restrict__ packed, uint8_t* __restrict__ canonical,
                                                      int64_t N, int64_t K) {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -210,10 +223,14 @@ __global__ void __launch_bounds__(256) unpack_kernel(const uint32_t* __restrict_
     if (t >= total) return;
     const int L = (int)(t & 31);
     const int64_t blk = t >> 5, rt = blk / kblocks, kb = blk % kblocks;
+    constexpr bool SIX = FMT == 1, NIB = FMT == 2;
     uint32_t w6[3] = {0u, 0u, 0u};
     uint32_t w8[4] = {0u, 0u, 0u, 0u};
     if (SIX) {
         for (int i = 0; i < 3; ++i) w6[i] = packed[six_bit_word(rt, kb, kblocks, L, i)];
+    } else if (NIB) {
+        uint2 q = reinterpret_cast<const uint2*>(packed)[t];
+        w8[0] = q.x; w8[1] = q.y;
     } else {
         uint4 q = reinterpret_cast<const uint4*>(packed)[t];
         w8[0] = q.x; w8[1] = q.y; w8[2] = q.z; w8[3] = q.w;
@@ -221,7 +238,10 @@ __global__ void __launch_bounds__(256) unpack_kernel(const uint32_t* __restrict_
     for (int s = 0; s < 16; ++s) {
         int64_t row, pair;
         slot_coords(rt, kb, L, s, row, pair);
-        const uint32_t idx = SIX ? six_bit_load(w6, s) : ((w8[s >> 2] >> (8 * (s & 3))) & 255u);
+        const int nbyte = 2 * (s >> 2) + ((s & 3) >> 1);       // nibble format: byte of the lane holding slot s
+        const uint32_t idx = SIX ? six_bit_load(w6, s)
+                           : NIB ? ((w8[nbyte >> 2] >> (8 * (nbyte & 3) + 4 * (s & 1))) & 15u)
+                                 : ((w8[s >> 2] >> (8 * (s & 3))) & 255u);
         if (P == 2) {
             canonical[row * (K / 2) + pair] = (uint8_t)idx;
         } else {
@@ -256,9 +276,10 @@ int launch_pack(const higgs_desc& d, const uint8_t* canonical, void* packed, cud
     const unsigned blocks = (unsigned)((total + 255) / 256);
     uint32_t* out = static_cast<uint32_t*>(packed);
     const Format f = format_of(d.p, d.n);
-    if (f == Format::kByteLut && d.p == 2) pack_kernel<2, false><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K);
-    else if (f == Format::kByteLut && d.p == 1) pack_kernel<1, false><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K);
-    else if (f == Format::kSixBit) pack_kernel<2, true><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K);
+    if (f == Format::kByteLut && d.p == 2) pack_kernel<2, 0><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K);
+    else if (f == Format::kByteLut && d.p == 1) pack_kernel<1, 0><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K);
+    else if (f == Format::kSixBit) pack_kernel<2, 1><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K);
+    else if (f == Format::kNibble) pack_kernel<2, 2><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K);
     else return HIGGS_ERR_UNSUPPORTED;
     return cuda_status(cudaGetLastError());
 }
@@ -269,9 +290,10 @@ int launch_unpack(const higgs_desc& d, const void* packed, uint8_t* canonical, c
     const unsigned blocks = (unsigned)((total + 255) / 256);
     const uint32_t* in = static_cast<const uint32_t*>(packed);
     const Format f = format_of(d.p, d.n);
-    if (f == Format::kByteLut && d.p == 2) unpack_kernel<2, false><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K);
-    else if (f == Format::kByteLut && d.p == 1) unpack_kernel<1, false><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K);
-    else if (f == Format::kSixBit) unpack_kernel<2, true><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K);
+    if (f == Format::kByteLut && d.p == 2) unpack_kernel<2, 0><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K);
+    else if (f == Format::kByteLut && d.p == 1) unpack_kernel<1, 0><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K);
+    else if (f == Format::kSixBit) unpack_kernel<2, 1><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K);
+    else if (f == Format::kNibble) unpack_kernel<2, 2><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K);
     else return HIGGS_ERR_UNSUPPORTED;
     return cuda_status(cudaGetLastError());
 }

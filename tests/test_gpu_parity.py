@@ -55,6 +55,7 @@ def run_quantize(W32, p, n, xi, bf16):
     (2, 256, 48, 3072, True),       # several groups per row, ragged against any block size
     (2, 64, 80, 2048, True),
     (1, 16, 64, 2048, True),
+    (2, 16, 80, 2048, True),        # 2 bits per weight: two codes per byte
     (2, 256, 16, 1024, False),      # smallest supported matrix
 ])
 def test_quantize_codes_and_scales(p, n, N, K, bf16):
@@ -129,6 +130,12 @@ def run_linear_case(p, n, N, K, B, xi, wseed, xseed, out_dtype=torch.float32, lo
     (2, 64, 32, 1024, 12),
     (1, 16, 48, 2048, 1),
     (1, 16, 64, 4096, 16),
+    (2, 16, 48, 2048, 1),        # nibble format: one byte looks up the fp16 pairs of two codes
+    (2, 16, 272, 4096, 5),
+    (2, 16, 272, 4096, 8),
+    (2, 16, 64, 8192, 16),
+    (2, 16, 32, 14336, 2),
+    (2, 16, 128, 1024, 40),      # more tokens than one launch takes (no tensor-core path for this format)
     (2, 256, 16, 1024, 17),      # more tokens than one launch takes
     (2, 256, 32, 2048, 40),
 ])
@@ -184,7 +191,7 @@ def test_empty_inputs():
 
 
 # ----------------------------------------------------------------------------- grid fit
-@pytest.mark.parametrize("p,n", [(2, 64), (1, 16)])
+@pytest.mark.parametrize("p,n", [(2, 64), (1, 16), (2, 16)])
 def test_make_grid_is_a_lloyd_fixed_point_at_the_oracle_mse(p, n):
     s = inputs.gaussian_samples(p, inputs.grid_sample_seed(p, n), log2_count=16)
     st = U.f32_tensor(s)
@@ -211,7 +218,7 @@ def test_make_grid_is_a_lloyd_fixed_point_at_the_oracle_mse(p, n):
 
 
 # ----------------------------------------------------------------------------- dequantisation to the original space
-@pytest.mark.parametrize("p,n,N,K", [(2, 256, 48, 2048), (2, 64, 32, 3072), (1, 16, 16, 1024)])
+@pytest.mark.parametrize("p,n,N,K", [(2, 256, 48, 2048), (2, 64, 32, 3072), (1, 16, 16, 1024), (2, 16, 32, 2048)])
 def test_dequantize_matches_oracle(p, n, N, K):
     """Appendix F 'Dequantization': LUT restore, inverse rotation, unscale; element by element against the oracle."""
     xi = inputs.rht_seed(2)
