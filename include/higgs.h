@@ -67,8 +67,8 @@ typedef enum higgs_op { HIGGS_OP_QUANTIZE = 0, HIGGS_OP_LINEAR = 1, HIGGS_OP_MAK
 
 /*
  * Description of one quantized matrix.  Supported: g = 1024; (p, n) in
- * {(2,256), (2,64), (2,16), (1,16)} - the 4-, 3- and 2-bit vector grids and
- * the 4-bit scalar grid; N a multiple of 16, K a multiple of g.
+ * {(2,256), (2,64), (2,16), (1,16), (1,8), (1,4)} - the 4-, 3- and 2-bit vector
+ * and scalar grids; N a multiple of 16, K a multiple of g.
  * Anything else returns HIGGS_ERR_UNSUPPORTED (never padded silently).
  * scale_dtype must be HIGGS_F16: one 16-bit scale per (row, group), which is
  * what the paper's bit counts imply (4.02 = 4 + 16/1024 in the appendix on

@@ -37,12 +37,18 @@ __host__ __device__ __forceinline__ uint32_t sign_bit(uint64_t xi, int64_t j) {
 enum class Format : int { kNone = 0, kByteLut = 1, kSixBit = 2, kNibble = 3 };
 
 __host__ __device__ inline Format format_of(int p, int n) {
+    // a table index always covers two consecutive inputs: one p=2 code or two p=1 codes
     if (p == 2 && n == 256) return Format::kByteLut;
     if (p == 1 && n == 16) return Format::kByteLut;
     if (p == 2 && n == 64) return Format::kSixBit;
+    if (p == 1 && n == 8) return Format::kSixBit;
     if (p == 2 && n == 16) return Format::kNibble;
+    if (p == 1 && n == 4) return Format::kNibble;
     return Format::kNone;
 }
+
+// log2 of the grid size (bits per code)
+__host__ __device__ inline int code_bits(int n) { int b = 0; while ((1 << b) < n) ++b; return b; }
 
 // Validates the descriptor; returns HIGGS_OK or the error to hand back.
 int check_desc(const higgs_desc* d);

@@ -54,6 +54,7 @@ struct StreamParams {
     int64_t N, K, ldy;
     int chunks;            // K / ck; the grid is chunks x parts blocks
     int B, n, p;
+    int bits;              // log2(n): bits per code
     int ck;                // inputs per item
     int y_mode;            // 0: store fp32, 1: store bf16, 2: atomicAdd fp32
     // Planned on the host so that the kernel's prologue has no divisions before its first copies are in flight:
@@ -256,16 +257,22 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
         ent_lo[r] = 0.f; ent_hi[r] = 0.f;
         if (NIB) { ent_lo2[r] = 0.f; ent_hi2[r] = 0.f; }
         if (idx < 256) {
-            if (NIB) {
+            // a table index stands for two consecutive inputs: one p=2 code, or two p=1 codes of prm.bits bits each
+            if (NIB && prm.p == 2) {
                 const float2 g0 = __ldg(reinterpret_cast<const float2*>(prm.grid) + (idx & 15));
                 const float2 g1 = __ldg(reinterpret_cast<const float2*>(prm.grid) + (idx >> 4));
                 ent_lo[r] = g0.x; ent_hi[r] = g0.y; ent_lo2[r] = g1.x; ent_hi2[r] = g1.y;
+            } else if (NIB) {
+                ent_lo[r] = __ldg(prm.grid + (idx & 3));
+                ent_hi[r] = __ldg(prm.grid + ((idx >> 2) & 3));
+                ent_lo2[r] = __ldg(prm.grid + ((idx >> 4) & 3));
+                ent_hi2[r] = __ldg(prm.grid + (idx >> 6));
             } else if (prm.p == 2) {
                 const float2 gp = __ldg(reinterpret_cast<const float2*>(prm.grid) + (idx & (prm.n - 1)));
                 ent_lo[r] = gp.x; ent_hi[r] = gp.y;
             } else {
-                ent_lo[r] = __ldg(prm.grid + (idx & 15));
-                ent_hi[r] = __ldg(prm.grid + (idx >> 4));
+                ent_lo[r] = __ldg(prm.grid + (idx & (prm.n - 1)));
+                ent_hi[r] = __ldg(prm.grid + ((idx >> prm.bits) & (prm.n - 1)));
             }
         }
     }
@@ -681,6 +688,7 @@ int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const 
     prm.chunks = pl.chunks;
     prm.B = (int)B;
     prm.n = d.n; prm.p = d.p;
+    prm.bits = code_bits(d.n);
     prm.ck = pl.ck;
     prm.y_mode = y_mode;
     const Format fmt = format_of(d.p, d.n);

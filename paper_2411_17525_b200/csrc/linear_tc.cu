@@ -54,6 +54,7 @@ struct TcParams {
     void* y;                 // [B][N]
     int64_t N, K;
     int B, BN, n, p, y_mode; // y_mode 0: fp32, 1: bf16
+    int bits;                // log2(n)
     int ksplit;              // K slices (= cluster size along z); each a multiple of 256 inputs
 };
 
@@ -234,8 +235,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
                 const float2 gp = __ldg(reinterpret_cast<const float2*>(prm.grid) + (idx & (prm.n - 1)));
                 ent_lo[r] = gp.x; ent_hi[r] = gp.y;
             } else {
-                ent_lo[r] = __ldg(prm.grid + (idx & 15));
-                ent_hi[r] = __ldg(prm.grid + (idx >> 4));
+                ent_lo[r] = __ldg(prm.grid + (idx & (prm.n - 1)));          // two p=1 codes per table index
+                ent_hi[r] = __ldg(prm.grid + ((idx >> prm.bits) & (prm.n - 1)));
             }
         }
     }
@@ -727,6 +728,7 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
     prm.y = y;
     prm.N = d.N; prm.K = d.K;
     prm.B = (int)B; prm.BN = BN; prm.n = d.n; prm.p = d.p; prm.y_mode = y_mode;
+    prm.bits = code_bits(d.n);
     prm.ksplit = tc_k_split(d, B);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(d.N / 128), (unsigned)tiles, (unsigned)prm.ksplit);

@@ -154,10 +154,11 @@ __device__ __forceinline__ void slot_coords(int64_t rt, int64_t kb, int L, int s
 // table index of a pair of inputs (2 consecutive k) from the canonical codes
 template <int P>
 __device__ __forceinline__ uint32_t pair_index(const uint8_t* __restrict__ canonical, int64_t K, int64_t row,
-                                               int64_t pair) {
+                                               int64_t pair, int bits) {
     if (P == 2) return canonical[row * (K / 2) + pair];
-    const uint8_t* q = canonical + row * K + 2 * pair;
-    return (uint32_t)(q[0] & 15) | ((uint32_t)(q[1] & 15) << 4);
+    const uint8_t* q = canonical + row * K + 2 * pair;       // two scalar codes of `bits` bits each
+    const uint32_t mask = (1u << bits) - 1u;
+    return (uint32_t)(q[0] & mask) | ((uint32_t)(q[1] & mask) << bits);
 }
 
 __device__ __forceinline__ void six_bit_store(uint32_t (&w)[3], int s, uint32_t code) {
@@ -178,7 +179,7 @@ __device__ __forceinline__ int64_t six_bit_word(int64_t rt, int64_t kb, int64_t 
 
 template <int P, int FMT>
 __global__ void __launch_bounds__(256) pack_kernel(const uint8_t* __restrict__ canonical, uint32_t* __restrict__ packed,
-                                                   int64_t N, int64_t K) {
+                                                   int64_t N, int64_t K, int bits) {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t kblocks = K / kBlockK;
     const int64_t total = (N / 16) * kblocks * 32;
@@ -191,7 +192,7 @@ __global__ void __launch_bounds__(256) pack_kernel(const uint8_t* __restrict__ c
         for (int s = 0; s < 16; ++s) {
             int64_t row, pair;
             slot_coords(rt, kb, L, s, row, pair);
-            six_bit_store(w, s, pair_index<P>(canonical, K, row, pair) & 63u);
+            six_bit_store(w, s, pair_index<P>(canonical, K, row, pair, bits) & 63u);
         }
         for (int i = 0; i < 3; ++i) packed[six_bit_word(rt, kb, kblocks, L, i)] = w[i];
     } else if (NIB) {
@@ -200,7 +201,7 @@ __global__ void __launch_bounds__(256) pack_kernel(const uint8_t* __restrict__ c
             int64_t row, pair;
             slot_coords(rt, kb, L, s, row, pair);
             const int m = s >> 2, a = s & 3, byte = 2 * m + (a >> 1);
-            w[byte >> 2] |= (pair_index<P>(canonical, K, row, pair) & 15u) << (8 * (byte & 3) + 4 * (a & 1));
+            w[byte >> 2] |= (pair_index<P>(canonical, K, row, pair, bits) & 15u) << (8 * (byte & 3) + 4 * (a & 1));
         }
         reinterpret_cast<uint2*>(packed)[t] = make_uint2(w[0], w[1]);
     } else {
@@ -208,7 +209,7 @@ __global__ void __launch_bounds__(256) pack_kernel(const uint8_t* __restrict__ c
         for (int s = 0; s < 16; ++s) {
             int64_t row, pair;
             slot_coords(rt, kb, L, s, row, pair);
-            w[s >> 2] |= pair_index<P>(canonical, K, row, pair) << (8 * (s & 3));
+            w[s >> 2] |= pair_index<P>(canonical, K, row, pair, bits) << (8 * (s & 3));
         }
         reinterpret_cast<uint4*>(packed)[t] = make_uint4(w[0], w[1], w[2], w[3]);
     }
@@ -216,7 +217,7 @@ __global__ void __launch_bounds__(256) pack_kernel(const uint8_t* __restrict__ c
 
 template <int P, int FMT>
 __global__ void __launch_bounds__(256) unpack_kernel(const uint32_t* __restrict__ packed, uint8_t* __restrict__ canonical,
-                                                     int64_t N, int64_t K) {
+                                                     int64_t N, int64_t K, int bits) {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t kblocks = K / kBlockK;
     const int64_t total = (N / 16) * kblocks * 32;
@@ -245,8 +246,8 @@ __global__ void __launch_bounds__(256) unpack_kernel(const uint32_t* __restrict_
         if (P == 2) {
             canonical[row * (K / 2) + pair] = (uint8_t)idx;
         } else {
-            canonical[row * K + 2 * pair] = (uint8_t)(idx & 15u);
-            canonical[row * K + 2 * pair + 1] = (uint8_t)(idx >> 4);
+            canonical[row * K + 2 * pair] = (uint8_t)(idx & ((1u << bits) - 1u));
+            canonical[row * K + 2 * pair + 1] = (uint8_t)((idx >> bits) & ((1u << bits) - 1u));
         }
     }
 }
@@ -276,10 +277,13 @@ int launch_pack(const higgs_desc& d, const uint8_t* canonical, void* packed, cud
     const unsigned blocks = (unsigned)((total + 255) / 256);
     uint32_t* out = static_cast<uint32_t*>(packed);
     const Format f = format_of(d.p, d.n);
-    if (f == Format::kByteLut && d.p == 2) pack_kernel<2, 0><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K);
-    else if (f == Format::kByteLut && d.p == 1) pack_kernel<1, 0><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K);
-    else if (f == Format::kSixBit) pack_kernel<2, 1><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K);
-    else if (f == Format::kNibble) pack_kernel<2, 2><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K);
+    const int bits = code_bits(d.n);
+    if (f == Format::kByteLut && d.p == 2) pack_kernel<2, 0><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K, bits);
+    else if (f == Format::kByteLut && d.p == 1) pack_kernel<1, 0><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K, bits);
+    else if (f == Format::kSixBit && d.p == 2) pack_kernel<2, 1><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K, bits);
+    else if (f == Format::kSixBit) pack_kernel<1, 1><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K, bits);
+    else if (f == Format::kNibble && d.p == 2) pack_kernel<2, 2><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K, bits);
+    else if (f == Format::kNibble) pack_kernel<1, 2><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K, bits);
     else return HIGGS_ERR_UNSUPPORTED;
     return cuda_status(cudaGetLastError());
 }
@@ -290,10 +294,13 @@ int launch_unpack(const higgs_desc& d, const void* packed, uint8_t* canonical, c
     const unsigned blocks = (unsigned)((total + 255) / 256);
     const uint32_t* in = static_cast<const uint32_t*>(packed);
     const Format f = format_of(d.p, d.n);
-    if (f == Format::kByteLut && d.p == 2) unpack_kernel<2, 0><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K);
-    else if (f == Format::kByteLut && d.p == 1) unpack_kernel<1, 0><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K);
-    else if (f == Format::kSixBit) unpack_kernel<2, 1><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K);
-    else if (f == Format::kNibble) unpack_kernel<2, 2><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K);
+    const int bits = code_bits(d.n);
+    if (f == Format::kByteLut && d.p == 2) unpack_kernel<2, 0><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K, bits);
+    else if (f == Format::kByteLut && d.p == 1) unpack_kernel<1, 0><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K, bits);
+    else if (f == Format::kSixBit && d.p == 2) unpack_kernel<2, 1><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K, bits);
+    else if (f == Format::kSixBit) unpack_kernel<1, 1><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K, bits);
+    else if (f == Format::kNibble && d.p == 2) unpack_kernel<2, 2><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K, bits);
+    else if (f == Format::kNibble) unpack_kernel<1, 2><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K, bits);
     else return HIGGS_ERR_UNSUPPORTED;
     return cuda_status(cudaGetLastError());
 }

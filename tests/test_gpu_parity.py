@@ -56,6 +56,8 @@ def run_quantize(W32, p, n, xi, bf16):
     (2, 64, 80, 2048, True),
     (1, 16, 64, 2048, True),
     (2, 16, 80, 2048, True),        # 2 bits per weight: two codes per byte
+    (1, 8, 48, 2048, True),         # scalar grids: two codes per table index
+    (1, 4, 48, 2048, True),
     (2, 256, 16, 1024, False),      # smallest supported matrix
 ])
 def test_quantize_codes_and_scales(p, n, N, K, bf16):
@@ -136,6 +138,10 @@ def run_linear_case(p, n, N, K, B, xi, wseed, xseed, out_dtype=torch.float32, lo
     (2, 16, 64, 8192, 16),
     (2, 16, 32, 14336, 2),
     (2, 16, 128, 1024, 40),      # more tokens than one launch takes (no tensor-core path for this format)
+    (1, 8, 272, 4096, 4),        # scalar 3-bit grid: six-bit format, two codes per index
+    (1, 8, 64, 8192, 16),
+    (1, 4, 272, 4096, 8),        # scalar 2-bit grid: nibble format, four codes per byte
+    (1, 4, 48, 2048, 1),
     (2, 256, 16, 1024, 17),      # more tokens than one launch takes
     (2, 256, 32, 2048, 40),
 ])
@@ -218,7 +224,8 @@ def test_make_grid_is_a_lloyd_fixed_point_at_the_oracle_mse(p, n):
 
 
 # ----------------------------------------------------------------------------- dequantisation to the original space
-@pytest.mark.parametrize("p,n,N,K", [(2, 256, 48, 2048), (2, 64, 32, 3072), (1, 16, 16, 1024), (2, 16, 32, 2048)])
+@pytest.mark.parametrize("p,n,N,K", [(2, 256, 48, 2048), (2, 64, 32, 3072), (1, 16, 16, 1024), (2, 16, 32, 2048),
+                                     (1, 8, 16, 2048), (1, 4, 16, 1024)])
 def test_dequantize_matches_oracle(p, n, N, K):
     """Appendix F 'Dequantization': LUT restore, inverse rotation, unscale; element by element against the oracle."""
     xi = inputs.rht_seed(2)
@@ -234,7 +241,7 @@ def test_dequantize_matches_oracle(p, n, N, K):
     assert np.max(np.abs(W_gpu - W_ref)) <= 2e-6 * np.max(np.abs(W_ref))      # fp32 butterflies over 10 stages
     # and it is the matrix the layer stands for: relative error against W equals the grid's MSE level (Appendix E)
     rel = np.sum((W_gpu - W) ** 2) / np.sum(W.astype(np.float64) ** 2)
-    assert rel < 0.25 if n == 16 else rel < 0.05
+    assert rel < 0.25 if n <= 16 else rel < 0.05
     W_bf = hb.higgs_dequantize(d, packed, scales, gt, out_dtype=torch.bfloat16).float().cpu().numpy()
     assert np.max(np.abs(W_bf - W_ref)) <= 2.0 ** -8 * np.max(np.abs(W_ref))
 
@@ -253,6 +260,7 @@ def test_dequantize_matches_oracle(p, n, N, K):
     (2, 64, 384, 4096, 100),
     (2, 64, 8448, 1024, 40),     # six-bit, K not split
     (2, 64, 256, 1024, 300),
+    (1, 8, 256, 2048, 64),       # scalar 3-bit grid on the six-bit path
 ])
 def test_linear_tensor_core_path_matches_oracle(p, n, N, K, B):
     y, y_ref = run_linear_case(p, n, N, K, B, xi=inputs.rht_seed(3), wseed=300 + N, xseed=400 + B, lognormal=(B == 64))
