@@ -28,6 +28,9 @@ def sampled_rows(N, count, seed):
     ("1b-kv", 512, 2048, 2, 256, (1,)),
     ("8b-gate-3bit", 14336, 4096, 2, 64, (1, 4)),
     ("8b-q-p1", 4096, 4096, 1, 16, (16,)),
+    ("8b-gate-tensor", 14336, 4096, 2, 256, (64, 256)),   # tensor-core regime, outlier channels (log-normal scales)
+    ("8b-down-tensor", 4096, 14336, 2, 256, (64,)),       # K split over a thread-block cluster
+    ("8b-gate-2bit", 14336, 4096, 2, 16, (1,)),
 ])
 def test_full_size_layer_on_sampled_rows(name, N, K, p, n, batches):
     cfg = 1
@@ -52,7 +55,7 @@ def test_full_size_layer_on_sampled_rows(name, N, K, p, n, batches):
     packed2 = hb.higgs_pack_codes(d, canon)
     scales2 = hb.scales_to_tile_major(sc_rows)
     for B in batches:
-        x = inputs.make_activations(B, K, inputs.activation_seed(cfg, B))
+        x = inputs.make_activations(B, K, inputs.activation_seed(cfg, B), lognormal_channels=B >= 64)
         y = hb.higgs_linear(d, U.bf16_tensor(x), packed2, scales2, gt)
         assert hb.higgs_device_status() == hb.HIGGS_OK
         y_ref = oracle.linear_dense(x.astype(np.float64), q.codes, sc16.astype(np.float64), G, g64, xi)
@@ -63,5 +66,5 @@ def test_full_size_layer_on_sampled_rows(name, N, K, p, n, batches):
         assert bool(torch.isfinite(y).all())
         # the split rotation + product entry points give the same result as the one-call form
         xd = hb.higgs_rotate_activations(d, U.bf16_tensor(x))
-        y2 = hb.higgs_linear_prerotated(d, xd, packed2, scales2, gt)
+        y2 = hb.higgs_linear_prerotated(d, xd, packed2, scales2, gt, B=B)
         assert float((y2 - y).abs().max()) <= 1e-5 * float(y.abs().max())
