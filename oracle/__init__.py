@@ -140,6 +140,29 @@ def gauss_mse_1d(levels) -> float:
     return float(_load().higgs_oracle_gauss_mse_1d(_pd(lv), lv.shape[0]))
 
 
+def uniform_grid(n: int, iters: int = 200):
+    """Constrained HIGGS ("CH", Section 4.3): the uniform n-level grid, symmetric about 0, whose step minimises the
+    expected squared error of rounding N(0,1).  Golden-section search on the step over the closed-form MSE.
+    Returns (levels[n][1], step, mse)."""
+    k = np.arange(n, dtype=np.float64) - 0.5 * (n - 1)
+    f = lambda step: gauss_mse_1d(k * step)
+    lo, hi = 1e-4, 8.0 / n + 2.0
+    r = 0.5 * (np.sqrt(5.0) - 1.0)
+    a, b = hi - r * (hi - lo), lo + r * (hi - lo)
+    fa, fb = f(a), f(b)
+    for _ in range(iters):
+        if fa < fb:
+            hi, b, fb = b, a, fa
+            a = hi - r * (hi - lo)
+            fa = f(a)
+        else:
+            lo, a, fa = a, b, fb
+            b = lo + r * (hi - lo)
+            fb = f(b)
+    step = 0.5 * (lo + hi)
+    return (k * step).reshape(n, 1), float(step), float(f(step))
+
+
 def grid_mse(grid, pts) -> float:
     """Per-dimension MSE of rounding pts[m][p] to grid[n][p] (the t^2 of Appendix E)."""
     g = _d(grid)

@@ -23,6 +23,24 @@ def test_1d_lloyd_max_closed_form_matches_published_table(n, golden):
     assert abs(quad - mse) < 1e-8
 
 
+@pytest.mark.parametrize("n", [2, 4, 8, 16, 32])
+def test_uniform_grid_matches_published_table(n, golden):
+    """Constrained (uniform) grids: the MSE-optimal step and its error against Max's table of equally spaced levels."""
+    tab = golden("uniform_max_gaussian.txt")
+    levels, step, mse = oracle.uniform_grid(n)
+    assert abs(step - tab[f"step_n{n}"][0]) <= 1e-3 * tab[f"step_n{n}"][0]
+    assert abs(mse - tab[f"mse_n{n}"][0]) <= 2e-3 * tab[f"mse_n{n}"][0]
+    lv = levels.ravel()
+    assert np.allclose(np.diff(lv), step) and np.allclose(lv, -lv[::-1])
+    # a uniform grid can never beat the unconstrained Lloyd-Max grid of the same size, and n = 2 coincides with it
+    assert mse >= oracle.lloyd_max_1d(n)[1] - 1e-12
+    if n == 2:
+        assert abs(mse - (1 - 2 / np.pi)) < 1e-9
+    # stationarity in the step
+    k = np.arange(n) - 0.5 * (n - 1)
+    assert oracle.gauss_mse_1d(k * step * 1.01) > mse and oracle.gauss_mse_1d(k * step * 0.99) > mse
+
+
 def test_gauss_mse_1d_special_cases():
     # one level at 0: MSE = Var = 1; two levels +-sqrt(2/pi): 1 - 2/pi
     assert abs(oracle.gauss_mse_1d([0.0]) - 1.0) < 1e-12
