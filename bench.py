@@ -53,7 +53,7 @@ def parse_args():
 
 
 def layer_bytes(N, K, p, n):
-    bits = {(2, 256): 4, (1, 16): 4, (2, 64): 3, (2, 16): 2, (1, 8): 3, (1, 4): 2}[(p, n)]
+    bits = {(2, 256): 4, (1, 16): 4, (2, 64): 3, (2, 16): 2, (1, 8): 3, (1, 4): 2, (1, 256): 8}[(p, n)]
     return N * K * bits // 8 + N * (K // G) * 2
 
 

@@ -67,8 +67,8 @@ typedef enum higgs_op { HIGGS_OP_QUANTIZE = 0, HIGGS_OP_LINEAR = 1, HIGGS_OP_MAK
 
 /*
  * Description of one quantized matrix.  Supported: g = 1024; (p, n) in
- * {(2,256), (2,64), (2,16), (1,16), (1,8), (1,4)} - the 4-, 3- and 2-bit vector
- * and scalar grids; N a multiple of 16, K a multiple of g.
+ * {(2,256), (2,64), (2,16), (1,16), (1,8), (1,4), (1,256)} - the 4-, 3- and 2-bit
+ * vector and scalar grids and the 8-bit scalar one; N a multiple of 16, K a multiple of g.
  * Anything else returns HIGGS_ERR_UNSUPPORTED (never padded silently).
  * scale_dtype must be HIGGS_F16: one 16-bit scale per (row, group), which is
  * what the paper's bit counts imply (4.02 = 4 + 16/1024 in the appendix on
@@ -102,6 +102,17 @@ size_t higgs_canonical_bytes(const higgs_desc* desc);
  * samples and desc->p, desc->n the grid).  Workspaces must be 256-byte
  * aligned.  Contents need not be initialised and are undefined afterwards.  */
 size_t higgs_workspace_bytes(const higgs_desc* desc, int op, int64_t B);
+
+/*
+ * Section 4.3, "Constrained HIGGS": the uniform n-level scalar grid, symmetric about zero, whose step minimises
+ * the expected squared error of rounding N(0,1) (closed-form MSE, golden-section search in fp64 on the device).
+ * With n = 256 this is the paper's 8-bit option ("CH8"); use it with p = 1.
+ *   grid_out   device, [n] fp32 (= [n][1])
+ *   step_out   device, optional: the step
+ *   mse_out    device, optional: the expected squared error per weight
+ * 2 <= n <= 256, else HIGGS_ERR_UNSUPPORTED.  Asynchronous on `stream`.
+ */
+int higgs_make_uniform_grid(int n, float* grid_out, float* step_out, float* mse_out, void* stream);
 
 /*
  * Algorithm 2, first line: the Gaussian-MSE-optimal grid.  The paper names the

@@ -25,7 +25,7 @@ EXPORTS = [
     "higgs_pack_codes", "higgs_unpack_codes", "higgs_rotate_activations", "higgs_linear_prerotated",
     "higgs_linear_host", "higgs_linear_host_workspace_bytes", "higgs_linear_launch_count", "higgs_device_status",
     "higgs_linear_static", "higgs_linear_static_capacity", "higgs_linear_k_splits", "higgs_rotated_bytes",
-    "higgs_rotated_layout", "higgs_dequantize",
+    "higgs_rotated_layout", "higgs_dequantize", "higgs_make_uniform_grid",
 ]
 
 
@@ -92,6 +92,8 @@ def _load() -> ctypes.CDLL:
     lib.higgs_pack_codes.argtypes = [P, vp, vp, vp]
     lib.higgs_unpack_codes.restype = i32
     lib.higgs_unpack_codes.argtypes = [P, vp, vp, vp]
+    lib.higgs_make_uniform_grid.restype = i32
+    lib.higgs_make_uniform_grid.argtypes = [i32, vp, vp, vp, vp]
     lib.higgs_dequantize.restype = i32
     lib.higgs_dequantize.argtypes = [P, vp, vp, vp, vp, i32, vp, sz, vp]
     return lib
@@ -304,6 +306,15 @@ def higgs_pack_codes(desc: higgs_desc, canonical: torch.Tensor) -> torch.Tensor:
     packed = torch.empty(max(higgs_packed_bytes(desc), 16), dtype=torch.uint8, device=canonical.device)
     _check(lib.higgs_pack_codes(ctypes.byref(desc), _ptr(canonical), _ptr(packed), _stream()), "higgs_pack_codes")
     return packed
+
+
+def higgs_make_uniform_grid(n: int, device=None):
+    """The MSE-optimal uniform n-level grid (constrained HIGGS; n = 256 is 'CH8').  Returns (grid [n][1], step, mse)."""
+    device = device or torch.device("cuda", torch.cuda.current_device())
+    grid = torch.empty((n, 1), dtype=torch.float32, device=device)
+    out = torch.zeros(2, dtype=torch.float32, device=device)
+    _check(lib.higgs_make_uniform_grid(int(n), _ptr(grid), out.data_ptr(), out.data_ptr() + 4, _stream()), "higgs_make_uniform_grid")
+    return grid, out[0], out[1]
 
 
 def higgs_dequantize(desc: higgs_desc, packed: torch.Tensor, scales: torch.Tensor, grid: torch.Tensor,

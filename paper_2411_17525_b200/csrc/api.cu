@@ -41,7 +41,7 @@ size_t higgs_packed_bytes(const higgs_desc* d) {
     if (check_desc(d) != HIGGS_OK) return 0;
     const size_t pairs = (size_t)d->N * (size_t)d->K / 2;
     const Format f = format_of(d->p, d->n);
-    return f == Format::kSixBit ? pairs / 4 * 3 : f == Format::kNibble ? pairs / 2 : pairs;
+    return f == Format::kSixBit ? pairs / 4 * 3 : f == Format::kNibble ? pairs / 2 : f == Format::kByte8 ? pairs * 2 : pairs;
 }
 
 size_t higgs_scales_bytes(const higgs_desc* d) {
@@ -80,6 +80,12 @@ int higgs_make_grid(int p, int n, const float* samples, int64_t num_samples, int
     if (workspace_bytes < make_grid_workspace(p, n, num_samples)) return HIGGS_ERR_WORKSPACE;
     return launch_make_grid(p, n, samples, num_samples, max_iters, grid_out, mse_out, iters_out, workspace,
                             as_stream(stream));
+}
+
+int higgs_make_uniform_grid(int n, float* grid_out, float* step_out, float* mse_out, void* stream) {
+    if (!grid_out) return HIGGS_ERR_INVALID_ARG;
+    if (n < 2 || n > 256) return HIGGS_ERR_UNSUPPORTED;
+    return launch_uniform_grid(n, grid_out, step_out, mse_out, as_stream(stream));
 }
 
 int higgs_quantize(const higgs_desc* d, const void* W, int w_dtype, const float* grid, void* packed_out,

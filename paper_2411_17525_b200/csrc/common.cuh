@@ -34,7 +34,8 @@ __host__ __device__ __forceinline__ uint32_t sign_bit(uint64_t xi, int64_t j) {
 //              separate planes (bit slices), see quantize.cu.
 //   kNibble  : p=2,n=16: 4-bit codes, two per byte; the byte looks up an 8-byte
 //              table entry (the fp16 pairs of both codes = two A-fragment registers).
-enum class Format : int { kNone = 0, kByteLut = 1, kSixBit = 2, kNibble = 3 };
+//   kByte8   : p=1,n=256 (the constrained 8-bit grid): one byte = one input, a register takes two lookups.
+enum class Format : int { kNone = 0, kByteLut = 1, kSixBit = 2, kNibble = 3, kByte8 = 4 };
 
 __host__ __device__ inline Format format_of(int p, int n) {
     // a table index always covers two consecutive inputs: one p=2 code or two p=1 codes
@@ -44,6 +45,7 @@ __host__ __device__ inline Format format_of(int p, int n) {
     if (p == 1 && n == 8) return Format::kSixBit;
     if (p == 2 && n == 16) return Format::kNibble;
     if (p == 1 && n == 4) return Format::kNibble;
+    if (p == 1 && n == 256) return Format::kByte8;
     return Format::kNone;
 }
 
@@ -146,6 +148,7 @@ int launch_convert_out(const float* y32, void* y, int y_dtype, size_t count, cud
 size_t make_grid_workspace(int p, int n, int64_t m);
 int launch_make_grid(int p, int n, const float* samples, int64_t m, int max_iters, float* grid_out, float* mse_out,
                      int32_t* iters_out, void* ws, cudaStream_t st);
+int launch_uniform_grid(int n, float* grid_out, float* step_out, float* mse_out, cudaStream_t st);
 int linear_k_chunks(const higgs_desc& d, int64_t B);
 // tensor-core path (B > 16)
 bool tc_eligible(const higgs_desc& d, int64_t B);

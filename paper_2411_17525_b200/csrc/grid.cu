@@ -127,7 +127,69 @@ __global__ void grid_finalize_kernel(GridWs w, int p, int n, int64_t m, float* _
     }
 }
 
+// ---- constrained (uniform) grid, Section 4.3 "Constrained HIGGS" ------------------------------------------
+// n equally spaced levels (k - (n-1)/2) * step, symmetric about 0 (the Gaussian is); the step minimises the expected
+// squared error of rounding N(0,1):  MSE(step) = sum over cells of  M2 - 2 c M1 + c^2 P  with the cell's probability
+// P, first moment M1 = phi(a) - phi(b) and second moment M2 = P + a phi(a) - b phi(b)  (a, b the cell's thresholds,
+// the outer cells unbounded).  One block; thread i owns cell i; golden-section search on the step in fp64.
+__device__ __forceinline__ double d_phi(double x) { return 0.3989422804014327 * exp(-0.5 * x * x); }
+__device__ __forceinline__ double d_Phi(double x) { return 0.5 * erfc(-x * 0.7071067811865476); }
+
+__device__ double uniform_mse_block(int n, double step, double* red) {
+    double term = 0.0;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const double c = ((double)i - 0.5 * (double)(n - 1)) * step;
+        const bool lo_inf = i == 0, hi_inf = i == n - 1;
+        const double a = c - 0.5 * step, b = c + 0.5 * step;
+        const double Pa = lo_inf ? 0.0 : d_Phi(a), Pb = hi_inf ? 1.0 : d_Phi(b);
+        const double fa = lo_inf ? 0.0 : d_phi(a), fb = hi_inf ? 0.0 : d_phi(b);
+        const double P = Pb - Pa, M1 = fa - fb, M2 = P + (lo_inf ? 0.0 : a * fa) - (hi_inf ? 0.0 : b * fb);
+        term += M2 - 2.0 * c * M1 + c * c * P;
+    }
+    red[threadIdx.x] = term;
+    __syncthreads();
+    for (int s = blockDim.x / 2; s > 0; s >>= 1) {
+        if ((int)threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
+        __syncthreads();
+    }
+    const double v = red[0];
+    __syncthreads();
+    return v;
+}
+
+__global__ void __launch_bounds__(256) uniform_grid_kernel(int n, float* __restrict__ grid_out, float* __restrict__ step_out,
+                                                           float* __restrict__ mse_out) {
+    __shared__ double red[256];
+    double lo = 1e-4, hi = 8.0 / n + 2.0;
+    const double r = 0.6180339887498949;
+    double a = hi - r * (hi - lo), b = lo + r * (hi - lo);
+    double fa = uniform_mse_block(n, a, red), fb = uniform_mse_block(n, b, red);
+    for (int it = 0; it < 120; ++it) {         // every thread follows the same path: the values are block-uniform
+        if (fa < fb) {
+            hi = b; b = a; fb = fa;
+            a = hi - r * (hi - lo);
+            fa = uniform_mse_block(n, a, red);
+        } else {
+            lo = a; a = b; fa = fb;
+            b = lo + r * (hi - lo);
+            fb = uniform_mse_block(n, b, red);
+        }
+    }
+    const double step = 0.5 * (lo + hi);
+    const double mse = uniform_mse_block(n, step, red);
+    for (int i = threadIdx.x; i < n; i += blockDim.x) grid_out[i] = (float)(((double)i - 0.5 * (double)(n - 1)) * step);
+    if (threadIdx.x == 0) {
+        if (step_out) *step_out = (float)step;
+        if (mse_out) *mse_out = (float)mse;
+    }
+}
+
 }  // namespace
+
+int launch_uniform_grid(int n, float* grid_out, float* step_out, float* mse_out, cudaStream_t st) {
+    uniform_grid_kernel<<<1, 256, 0, st>>>(n, grid_out, step_out, mse_out);
+    return cuda_status(cudaGetLastError());
+}
 
 size_t make_grid_workspace(int p, int n, int64_t m) {
     return up256(sizeof(float) * n * p) + up256(sizeof(double) * n * p) + up256(sizeof(unsigned long long) * n) + 512 +

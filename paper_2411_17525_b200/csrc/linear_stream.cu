@@ -181,12 +181,13 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 
 // Code words of one task (16 rows x KS inputs) for this lane, read from a ring slot.
 // FMT: 0 = byte format (one byte = one table index = one A-fragment register), 1 = six-bit planes, 2 = nibble pairs
-// (p=2 n=16: one byte = two 4-bit codes = an 8-byte table entry = two A-fragment registers).
+// (p=2 n=16: one byte = two 4-bit codes = an 8-byte table entry = two A-fragment registers), 3 = 8-bit scalar codes
+// (p=1 n=256: one byte = one input; a register is put together from two lookups).
 template <int KS, int FMT>
 struct TaskCodes {
-    static constexpr bool SIX = FMT == 1, NIB = FMT == 2;
-    static constexpr int kWords = SIX ? (KS / 128) * 6 : NIB ? (KS / 64) * 2 : (KS / 64) * 4;
-    static constexpr uint32_t kBytes = SIX ? KS * 6 : NIB ? KS * 4 : KS * 8;   // bytes of one task in the packed stream
+    static constexpr bool SIX = FMT == 1, NIB = FMT == 2, B8 = FMT == 3;
+    static constexpr int kWords = SIX ? (KS / 128) * 6 : NIB ? (KS / 64) * 2 : B8 ? (KS / 64) * 8 : (KS / 64) * 4;
+    static constexpr uint32_t kBytes = SIX ? KS * 6 : NIB ? KS * 4 : B8 ? KS * 16 : KS * 8;   // bytes of one task in the packed stream
     uint32_t w[kWords];
     __device__ __forceinline__ void load(uint32_t slot, int lane) {
         if (SIX) {
@@ -204,6 +205,14 @@ struct TaskCodes {
             for (int j = 0; j < KS / 64; ++j) {
                 uint2 q = lds64(slot + (uint32_t)(j * 256 + lane * 8));
                 w[j * 2] = q.x; w[j * 2 + 1] = q.y;
+            }
+        } else if (B8) {
+#pragma unroll
+            for (int j = 0; j < KS / 64; ++j) {      // a 1 KB block = two 512-byte halves of 16 bytes per lane (words 0..3, 4..7)
+                uint4 q0 = lds128(slot + (uint32_t)(j * 1024 + lane * 16));
+                uint4 q1 = lds128(slot + (uint32_t)(j * 1024 + 512 + lane * 16));
+                w[j * 8] = q0.x; w[j * 8 + 1] = q0.y; w[j * 8 + 2] = q0.z; w[j * 8 + 3] = q0.w;
+                w[j * 8 + 4] = q1.x; w[j * 8 + 5] = q1.y; w[j * 8 + 6] = q1.z; w[j * 8 + 7] = q1.w;
             }
         } else {
 #pragma unroll
@@ -232,7 +241,7 @@ struct TaskCodes {
 
 template <int NB, int KS, int FMT>
 __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(const StreamParams prm) {
-    constexpr bool SIX = FMT == 1, NIB = FMT == 2;
+    constexpr bool SIX = FMT == 1, NIB = FMT == 2, B8 = FMT == 3;
     constexpr uint32_t kPieceStride = NIB ? 128u : 256u;     // bytes between consecutive 128-byte pieces of the partial tiles
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -267,6 +276,8 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
                 ent_hi[r] = __ldg(prm.grid + ((idx >> 2) & 3));
                 ent_lo2[r] = __ldg(prm.grid + ((idx >> 4) & 3));
                 ent_hi2[r] = __ldg(prm.grid + (idx >> 6));
+            } else if (B8) {
+                ent_lo[r] = ent_hi[r] = __ldg(prm.grid + idx);       // one input per index: the value in both halves
             } else if (prm.p == 2) {
                 const float2 gp = __ldg(reinterpret_cast<const float2*>(prm.grid) + (idx & (prm.n - 1)));
                 ent_lo[r] = gp.x; ent_hi[r] = gp.y;
@@ -351,9 +362,9 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     const int64_t kslice = (int64_t)chunk_begin * prm.ck + (int64_t)slice * KS;
     const int64_t rt_first = rt_begin + phase;
     const uint8_t* src_next = prm.packed + (SIX ? ((rt_first * (prm.K >> 7) + (kslice >> 7)) * 768)
-                                                : ((rt_first * (prm.K >> 6) + (kslice >> 6)) * (NIB ? 256 : 512)));
+                                                : ((rt_first * (prm.K >> 6) + (kslice >> 6)) * (NIB ? 256 : B8 ? 1024 : 512)));
     const __half* ssrc_next = prm.scales + (rt_first * groups + chunk_begin * ng + gl) * 16;
-    const int64_t src_stride = (int64_t)PG * (SIX ? prm.K * 6 : NIB ? prm.K * 4 : prm.K * 8);
+    const int64_t src_stride = (int64_t)PG * (SIX ? prm.K * 6 : NIB ? prm.K * 4 : B8 ? prm.K * 16 : prm.K * 8);
     const int64_t ssrc_stride = (int64_t)PG * groups * 16;
     uint32_t elected;
     asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(elected));
@@ -531,9 +542,17 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
         for (int jb = 0; jb < KS / 64; ++jb) {
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
-                const uint32_t iw = codes.index_word(jb, m);
+                const uint32_t iw = B8 ? 0u : codes.index_word(jb, m);
                 uint32_t a0, a1, a2, a3;
-                if (NIB) {
+                if (B8) {
+                    // words 2m and 2m+1 of the block hold the input bytes of (a0, a1) and (a2, a3); a table entry carries
+                    // its value in both halves, so a register is the low half of one lookup and the high half of the next
+                    const uint32_t w0 = codes.w[jb * 8 + 2 * m], w1 = codes.w[jb * 8 + 2 * m + 1];
+                    a0 = __byte_perm(lds32(__byte_perm(w0, lut_lane, 0x7604)), lds32(__byte_perm(w0, lut_lane, 0x7614)), 0x7610);
+                    a1 = __byte_perm(lds32(__byte_perm(w0, lut_lane, 0x7624)), lds32(__byte_perm(w0, lut_lane, 0x7634)), 0x7610);
+                    a2 = __byte_perm(lds32(__byte_perm(w1, lut_lane, 0x7604)), lds32(__byte_perm(w1, lut_lane, 0x7614)), 0x7610);
+                    a3 = __byte_perm(lds32(__byte_perm(w1, lut_lane, 0x7624)), lds32(__byte_perm(w1, lut_lane, 0x7634)), 0x7610);
+                } else if (NIB) {
                     // one byte = the codes of registers (a0, a1) resp. (a2, a3): one 8-byte lookup each
                     const uint2 p01 = lds64_table(__byte_perm(iw, lut_lane, (m & 1) ? 0x7624 : 0x7604));
                     const uint2 p23 = lds64_table(__byte_perm(iw, lut_lane, (m & 1) ? 0x7634 : 0x7614));
@@ -692,7 +711,7 @@ int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const 
     prm.ck = pl.ck;
     prm.y_mode = y_mode;
     const Format fmt = format_of(d.p, d.n);
-    const bool six = fmt == Format::kSixBit, nib = fmt == Format::kNibble;
+    const bool six = fmt == Format::kSixBit, nib = fmt == Format::kNibble, b8 = fmt == Format::kByte8;
     prm.parts = pl.parts;
     prm.parts_shift = 0;
     while ((1 << prm.parts_shift) < pl.parts) ++prm.parts_shift;
@@ -707,12 +726,13 @@ int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const 
     prm.acc_shift = 0;
     while ((1 << prm.acc_shift) < p2) ++prm.acc_shift;
     uint32_t lut_unused;
-    ring_layout(kAssumedBase, (uint32_t)(six ? pl.ks * 6 : nib ? pl.ks * 4 : pl.ks * 8) + 64u, nib ? kNibbleTileBytes : 0u, &lut_unused,
-                &prm.depth, &prm.warps_in_a);
-    if (pl.nb == 1) return six ? launch_one<1, 256, 1>(prm, pl.blocks, st) : nib ? launch_one<1, 256, 2>(prm, pl.blocks, st)
-                                                                               : launch_one<1, 256, 0>(prm, pl.blocks, st);
+    ring_layout(kAssumedBase, (uint32_t)(six ? pl.ks * 6 : nib ? pl.ks * 4 : b8 ? pl.ks * 16 : pl.ks * 8) + 64u,
+                nib ? kNibbleTileBytes : 0u, &lut_unused, &prm.depth, &prm.warps_in_a);
+    if (pl.nb == 1)
+        return six ? launch_one<1, 256, 1>(prm, pl.blocks, st) : nib ? launch_one<1, 256, 2>(prm, pl.blocks, st)
+             : b8 ? launch_one<1, 256, 3>(prm, pl.blocks, st) : launch_one<1, 256, 0>(prm, pl.blocks, st);
     return six ? launch_one<2, 128, 1>(prm, pl.blocks, st) : nib ? launch_one<2, 128, 2>(prm, pl.blocks, st)
-                                                               : launch_one<2, 128, 0>(prm, pl.blocks, st);
+         : b8 ? launch_one<2, 128, 3>(prm, pl.blocks, st) : launch_one<2, 128, 0>(prm, pl.blocks, st);
 }
 
 int launch_convert_out(const float* y32, void* y, int y_dtype, size_t count, cudaStream_t st) {

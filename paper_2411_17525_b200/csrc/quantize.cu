@@ -141,6 +141,9 @@ __global__ void __launch_bounds__(128) encode_kernel(const T* __restrict__ W, co
 //   nibble format  : (n = 16) two 32-bit words per lane and block, 256 bytes per block, lane L at
 //                    byte offset 8 L.  Byte 2m + h of the lane holds the slots 4m + 2h (low
 //                    nibble) and 4m + 2h + 1 (high nibble): the two registers of one row pair.
+//   8-bit format   : (p = 1, n = 256) one byte per input: slot 4m + a is the halfword a & 1 of the lane's
+//                    word 2m + (a >> 1) (low byte = first input of the pair); a block is 1024 bytes, two
+//                    512-byte halves holding words 0..3 and 4..7 of every lane (16 bytes per lane each).
 //                    Two neighbouring blocks (2j, 2j+1 along K) form a 768-byte
 //                    super-block of three 256-byte planes; plane w stores word w of
 //                    lane L, block half h at 32-bit index 2L + h, so a warp reads
@@ -186,8 +189,19 @@ __global__ void __launch_bounds__(256) pack_kernel(const uint8_t* __restrict__ c
     if (t >= total) return;
     const int L = (int)(t & 31);
     const int64_t blk = t >> 5, rt = blk / kblocks, kb = blk % kblocks;
-    constexpr bool SIX = FMT == 1, NIB = FMT == 2;
-    if (SIX) {
+    constexpr bool SIX = FMT == 1, NIB = FMT == 2, B8 = FMT == 3;
+    if (B8) {
+        uint32_t w[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+        for (int s = 0; s < 16; ++s) {
+            int64_t row, pair;
+            slot_coords(rt, kb, L, s, row, pair);
+            const uint8_t* q = canonical + row * K + 2 * pair;
+            w[2 * (s >> 2) + ((s & 3) >> 1)] |= ((uint32_t)q[0] | ((uint32_t)q[1] << 8)) << (16 * (s & 1));
+        }
+        uint4* out = reinterpret_cast<uint4*>(packed) + blk * 64;      // 1024-byte block = 64 uint4
+        out[L] = make_uint4(w[0], w[1], w[2], w[3]);
+        out[32 + L] = make_uint4(w[4], w[5], w[6], w[7]);
+    } else if (SIX) {
         uint32_t w[3] = {0u, 0u, 0u};
         for (int s = 0; s < 16; ++s) {
             int64_t row, pair;
@@ -224,7 +238,20 @@ __global__ void __launch_bounds__(256) unpack_kernel(const uint32_t* __restrict_
     if (t >= total) return;
     const int L = (int)(t & 31);
     const int64_t blk = t >> 5, rt = blk / kblocks, kb = blk % kblocks;
-    constexpr bool SIX = FMT == 1, NIB = FMT == 2;
+    constexpr bool SIX = FMT == 1, NIB = FMT == 2, B8 = FMT == 3;
+    if (B8) {
+        const uint4* in = reinterpret_cast<const uint4*>(packed) + blk * 64;
+        const uint4 q0 = in[L], q1 = in[32 + L];
+        const uint32_t w[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+        for (int s = 0; s < 16; ++s) {
+            int64_t row, pair;
+            slot_coords(rt, kb, L, s, row, pair);
+            const uint32_t hw = (w[2 * (s >> 2) + ((s & 3) >> 1)] >> (16 * (s & 1))) & 0xffffu;
+            canonical[row * K + 2 * pair] = (uint8_t)(hw & 255u);
+            canonical[row * K + 2 * pair + 1] = (uint8_t)(hw >> 8);
+        }
+        return;
+    }
     uint32_t w6[3] = {0u, 0u, 0u};
     uint32_t w8[4] = {0u, 0u, 0u, 0u};
     if (SIX) {
@@ -284,6 +311,7 @@ int launch_pack(const higgs_desc& d, const uint8_t* canonical, void* packed, cud
     else if (f == Format::kSixBit) pack_kernel<1, 1><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K, bits);
     else if (f == Format::kNibble && d.p == 2) pack_kernel<2, 2><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K, bits);
     else if (f == Format::kNibble) pack_kernel<1, 2><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K, bits);
+    else if (f == Format::kByte8) pack_kernel<1, 3><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K, bits);
     else return HIGGS_ERR_UNSUPPORTED;
     return cuda_status(cudaGetLastError());
 }
@@ -301,6 +329,7 @@ int launch_unpack(const higgs_desc& d, const void* packed, uint8_t* canonical, c
     else if (f == Format::kSixBit) unpack_kernel<1, 1><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K, bits);
     else if (f == Format::kNibble && d.p == 2) unpack_kernel<2, 2><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K, bits);
     else if (f == Format::kNibble) unpack_kernel<1, 2><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K, bits);
+    else if (f == Format::kByte8) unpack_kernel<1, 3><<<blocks, 256, 0, st>>>(in, canonical, d.N, d.K, bits);
     else return HIGGS_ERR_UNSUPPORTED;
     return cuda_status(cudaGetLastError());
 }

@@ -12,7 +12,8 @@ import sys
 import numpy as np
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-GRIDS = [(2, 256), (2, 64), (1, 16), (2, 16), (1, 8), (1, 4)]
+GRIDS = [(2, 256), (2, 64), (1, 16), (2, 16), (1, 8), (1, 4), (1, 256)]
+UNIFORM = {(1, 256)}      # constrained (equally spaced) grids: closed-form optimum of the step, no samples
 
 
 def path(p, n):
@@ -32,6 +33,13 @@ def main():
     for p, n in GRIDS:
         if os.path.exists(path(p, n)) and "--all" not in sys.argv:
             continue        # stored tables are never rewritten silently
+        if (p, n) in UNIFORM:
+            levels, step, mse = oracle.uniform_grid(n)
+            hdr = (f"MSE-optimal uniform grid (Section 4.3, constrained HIGGS), p={p} n={n}, step {step:.9g}, expected "
+                   f"squared error {mse:.6g}; written by tests/golden/make_grids.py from the fp64 oracle; values are fp32-exact")
+            np.savetxt(path(p, n), levels.astype(np.float32).astype(np.float64), fmt="%.9g", header=hdr)
+            print(p, n, "uniform", step, mse)
+            continue
         s = inputs.gaussian_samples(p, inputs.grid_sample_seed(p, n))
         res = oracle.make_grid_lloyd(p, n, s, max_iters=6000)
         g32 = res.grid.astype(np.float32)

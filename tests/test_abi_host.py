@@ -60,7 +60,7 @@ def test_size_queries():
 
 
 @pytest.mark.parametrize("p,n,g,N,K", [(2, 100, 1024, 16, 1024), (3, 256, 1024, 16, 1024), (2, 256, 512, 16, 1024),
-                                       (2, 256, 1024, 15, 1024), (2, 256, 1024, 16, 1000), (1, 256, 1024, 16, 1024)])
+                                       (2, 256, 1024, 15, 1024), (2, 256, 1024, 16, 1000), (1, 64, 1024, 16, 1024)])
 def test_unsupported_descriptors_are_refused(p, n, g, N, K):
     d = hb.make_desc(p, n, N, K, 1, g=g)
     assert hb.higgs_packed_bytes(d) == 0

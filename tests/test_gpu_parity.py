@@ -56,6 +56,7 @@ def run_quantize(W32, p, n, xi, bf16):
     (2, 64, 80, 2048, True),
     (1, 16, 64, 2048, True),
     (2, 16, 80, 2048, True),        # 2 bits per weight: two codes per byte
+    (1, 256, 32, 2048, True),       # constrained 8-bit grid: one byte per input
     (1, 8, 48, 2048, True),         # scalar grids: two codes per table index
     (1, 4, 48, 2048, True),
     (2, 256, 16, 1024, False),      # smallest supported matrix
@@ -142,6 +143,10 @@ def run_linear_case(p, n, N, K, B, xi, wseed, xseed, out_dtype=torch.float32, lo
     (1, 8, 64, 8192, 16),
     (1, 4, 272, 4096, 8),        # scalar 2-bit grid: nibble format, four codes per byte
     (1, 4, 48, 2048, 1),
+    (1, 256, 48, 2048, 1),       # 8-bit scalar codes: a register is put together from two lookups
+    (1, 256, 272, 4096, 7),
+    (1, 256, 64, 8192, 16),
+    (1, 256, 128, 1024, 33),
     (2, 256, 16, 1024, 17),      # more tokens than one launch takes
     (2, 256, 32, 2048, 40),
 ])
@@ -223,9 +228,19 @@ def test_make_grid_is_a_lloyd_fixed_point_at_the_oracle_mse(p, n):
     assert abs(m_dev - m_ref) <= 0.01 * m_ref
 
 
+def test_uniform_grid_fit_matches_oracle():
+    """Constrained HIGGS: the device's golden-section search lands on the oracle's step and MSE."""
+    for n in (16, 256):
+        grid, step, mse = hb.higgs_make_uniform_grid(n)
+        levels, step_ref, mse_ref = oracle.uniform_grid(n)
+        assert abs(float(step) - step_ref) <= 1e-5 * step_ref
+        assert abs(float(mse) - mse_ref) <= 1e-5 * mse_ref
+        assert np.allclose(grid.cpu().numpy().astype(np.float64), levels, rtol=1e-5, atol=1e-7)
+
+
 # ----------------------------------------------------------------------------- dequantisation to the original space
 @pytest.mark.parametrize("p,n,N,K", [(2, 256, 48, 2048), (2, 64, 32, 3072), (1, 16, 16, 1024), (2, 16, 32, 2048),
-                                     (1, 8, 16, 2048), (1, 4, 16, 1024)])
+                                     (1, 8, 16, 2048), (1, 4, 16, 1024), (1, 256, 16, 2048)])
 def test_dequantize_matches_oracle(p, n, N, K):
     """Appendix F 'Dequantization': LUT restore, inverse rotation, unscale; element by element against the oracle."""
     xi = inputs.rht_seed(2)
