@@ -269,6 +269,31 @@ int higgs_linear_launch_count(const higgs_desc* desc, int64_t B, int y_dtype);
 int higgs_dequantize(const higgs_desc* desc, const void* packed, const void* scales, const float* grid,
                      void* W_out, int w_dtype, void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---- dynamic bit widths (Section 5) ------------------------------------------------------------------------ */
+
+/* "Measuring Grid Parameters": one entry of the database of per-layer errors.  For the layer W quantised as
+ * (packed, scales, grid) it accumulates, without materialising the dequantised matrix,
+ *   sums_out[0] = || W^ - W ||_F^2,   sums_out[1] = || W ||_F^2        (device, two doubles, 8-byte aligned),
+ * so that t^2 = sums_out[0] / sums_out[1] is the relative error of the linearity theorem (Appendix E shows it
+ * equals the grid's expected squared error for Gaussian-like rotated weights).
+ * W: device [N][K], w_dtype in {HIGGS_F32, HIGGS_BF16}; workspace as for higgs_dequantize.  Asynchronous.    */
+int higgs_layer_error(const higgs_desc* desc, const void* W, int w_dtype, const void* packed, const void* scales,
+                      const float* grid, double* sums_out, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Eq. 4: choose option j_l in [0, num_options) for every layer l, minimising  sum_l alpha[l] * t2[l][j_l]  subject
+ * to  sum_l bits(j_l) * sizes[l] <= budget * sum_l sizes[l].  Exact (dynamic programming over the integer budget;
+ * ties: lowest option index, then lowest total size).  HOST function, host pointers, no GPU involved.
+ *   alpha[num_layers], t2[num_layers][num_options]  (row-major)
+ *   bits64[num_options] : bits per weight of every option in units of 1/64 bit (a 16-bit scale per 1024 weights
+ *                         is exactly 1/64 bit, so "4.02 bits" is 257); budget64: the target in the same unit
+ *   sizes[num_layers]   : number of weights of every layer
+ *   choice_out[num_layers], objective_out (optional)
+ * HIGGS_ERR_UNSUPPORTED if no assignment fits the budget, HIGGS_ERR_WORKSPACE if the table
+ * (num_layers x budget in reduced units) would exceed 2e9 entries.                                             */
+int higgs_allocate_bits(int32_t num_layers, int32_t num_options, const double* alpha, const double* t2,
+                        const int32_t* bits64, const int64_t* sizes, int64_t budget64, int32_t* choice_out,
+                        double* objective_out);
+
 /* The transform alone on `rows` rows of length K: out[r] = RHT of x[r] per
  * group (Algorithm 1 / Appendix F).  x_dtype in {HIGGS_F32, HIGGS_BF16};
  * out is device [rows][K] fp32; normalised != 0 divides by sqrt(g).        */

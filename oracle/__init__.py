@@ -215,6 +215,33 @@ def dequantize(codes, scales, g: int, grid, xi: int) -> np.ndarray:
     return out
 
 
+def layer_error(W, codes, scales, g: int, grid, xi: int) -> float:
+    """Section 5, 'Measuring Grid Parameters': t^2 = ||W^ - W||_F^2 / ||W||_F^2 with W^ the dequantised layer."""
+    Wd = _d(W)
+    What = dequantize(codes, scales, g, grid, xi)
+    return float(np.sum((What - Wd) ** 2) / np.sum(Wd ** 2))
+
+
+def allocate_bits_bruteforce(alpha, t2, bits, sizes, budget):
+    """Eq. 4 by exhaustive enumeration (tiny instances only): argmin over all J^L assignments of sum_l alpha_l t2[l][j_l]
+    subject to sum_l bits[j_l] sizes[l] <= budget * sum_l sizes[l].  Returns (choice, objective) or (None, inf)."""
+    import itertools
+    a = np.asarray(alpha, dtype=np.float64)
+    t = np.asarray(t2, dtype=np.float64)
+    b = np.asarray(bits, dtype=np.float64)
+    d = np.asarray(sizes, dtype=np.float64)
+    L, J = t.shape
+    best, arg = np.inf, None
+    for js in itertools.product(range(J), repeat=L):
+        idx = np.array(js)
+        if float(np.dot(b[idx], d)) > budget * float(d.sum()) * (1 + 1e-12):
+            continue
+        v = float(np.sum(a * t[np.arange(L), idx]))
+        if v < best - 1e-15:
+            best, arg = v, idx
+    return arg, best
+
+
 def matmul_nt(x, What) -> np.ndarray:
     x = _d(x)
     What = _d(What)

@@ -25,7 +25,8 @@ EXPORTS = [
     "higgs_pack_codes", "higgs_unpack_codes", "higgs_rotate_activations", "higgs_linear_prerotated",
     "higgs_linear_host", "higgs_linear_host_workspace_bytes", "higgs_linear_launch_count", "higgs_device_status",
     "higgs_linear_static", "higgs_linear_static_capacity", "higgs_linear_k_splits", "higgs_rotated_bytes",
-    "higgs_rotated_layout", "higgs_dequantize", "higgs_make_uniform_grid",
+    "higgs_rotated_layout", "higgs_dequantize", "higgs_make_uniform_grid", "higgs_layer_error",
+    "higgs_allocate_bits",
 ]
 
 
@@ -94,6 +95,10 @@ def _load() -> ctypes.CDLL:
     lib.higgs_unpack_codes.argtypes = [P, vp, vp, vp]
     lib.higgs_make_uniform_grid.restype = i32
     lib.higgs_make_uniform_grid.argtypes = [i32, vp, vp, vp, vp]
+    lib.higgs_layer_error.restype = i32
+    lib.higgs_layer_error.argtypes = [P, vp, i32, vp, vp, vp, vp, vp, sz, vp]
+    lib.higgs_allocate_bits.restype = i32
+    lib.higgs_allocate_bits.argtypes = [i32, i32, vp, vp, vp, vp, i64, vp, vp]
     lib.higgs_dequantize.restype = i32
     lib.higgs_dequantize.argtypes = [P, vp, vp, vp, vp, i32, vp, sz, vp]
     return lib
@@ -315,6 +320,33 @@ def higgs_make_uniform_grid(n: int, device=None):
     out = torch.zeros(2, dtype=torch.float32, device=device)
     _check(lib.higgs_make_uniform_grid(int(n), _ptr(grid), out.data_ptr(), out.data_ptr() + 4, _stream()), "higgs_make_uniform_grid")
     return grid, out[0], out[1]
+
+
+def higgs_layer_error(desc: higgs_desc, W: torch.Tensor, packed: torch.Tensor, scales: torch.Tensor, grid: torch.Tensor) -> float:
+    """Relative quantisation error t^2 = ||W^ - W||^2 / ||W||^2 of the layer (Section 5, 'Measuring Grid Parameters')."""
+    assert W.is_cuda and W.is_contiguous() and W.dtype in (torch.float32, torch.bfloat16)
+    sums = torch.zeros(2, dtype=torch.float64, device=W.device)
+    ws = _workspace(higgs_workspace_bytes(desc, HIGGS_OP_QUANTIZE, 0), W.device)
+    _check(lib.higgs_layer_error(ctypes.byref(desc), _ptr(W), _dtype_code(W), _ptr(packed), _ptr(scales), _ptr(grid), _ptr(sums),
+                                 _ptr(ws), ws.numel(), _stream()), "higgs_layer_error")
+    s = sums.cpu()
+    return float(s[0] / s[1]) if float(s[1]) > 0 else 0.0
+
+
+def higgs_allocate_bits(alpha, t2, bits64, sizes, budget64: int):
+    """Eq. 4 on the host: returns (choice per layer, objective).  bits64 / budget64 in units of 1/64 bit per weight."""
+    import numpy as np
+    a = np.ascontiguousarray(alpha, dtype=np.float64)
+    t = np.ascontiguousarray(t2, dtype=np.float64)
+    b = np.ascontiguousarray(bits64, dtype=np.int32)
+    d = np.ascontiguousarray(sizes, dtype=np.int64)
+    L, J = t.shape
+    assert a.shape == (L,) and b.shape == (J,) and d.shape == (L,)
+    choice = np.zeros(L, dtype=np.int32)
+    obj = ctypes.c_double(0.0)
+    _check(lib.higgs_allocate_bits(L, J, a.ctypes.data, t.ctypes.data, b.ctypes.data, d.ctypes.data, int(budget64),
+                                   choice.ctypes.data, ctypes.addressof(obj)), "higgs_allocate_bits")
+    return choice, float(obj.value)
 
 
 def higgs_dequantize(desc: higgs_desc, packed: torch.Tensor, scales: torch.Tensor, grid: torch.Tensor,

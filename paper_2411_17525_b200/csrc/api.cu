@@ -126,6 +126,28 @@ int higgs_dequantize(const higgs_desc* d, const void* packed, const void* scales
     return launch_dequantize(*d, canonical, scales, grid, W_out, w_dtype, st);
 }
 
+int higgs_layer_error(const higgs_desc* d, const void* W, int w_dtype, const void* packed, const void* scales,
+                      const float* grid, double* sums_out, void* workspace, size_t workspace_bytes, void* stream) {
+    int rc = check_desc(d);
+    if (rc != HIGGS_OK) return rc;
+    if (w_dtype != HIGGS_F32 && w_dtype != HIGGS_BF16) return HIGGS_ERR_UNSUPPORTED;
+    if (!sums_out || !aligned(sums_out, 8)) return HIGGS_ERR_INVALID_ARG;
+    if (d->N == 0 || d->K == 0) return cuda_status(cudaMemsetAsync(sums_out, 0, 2 * sizeof(double), as_stream(stream)));
+    if (!W || !packed || !scales || !grid || !workspace) return HIGGS_ERR_INVALID_ARG;
+    if (!aligned(W, 16) || !aligned(packed, 16) || !aligned(scales, 16) || !aligned(workspace, 256)) return HIGGS_ERR_INVALID_ARG;
+    if (workspace_bytes < higgs_workspace_bytes(d, HIGGS_OP_QUANTIZE, 0)) return HIGGS_ERR_WORKSPACE;
+    cudaStream_t st = as_stream(stream);
+    uint8_t* canonical = static_cast<uint8_t*>(workspace);
+    rc = launch_unpack(*d, packed, canonical, st);
+    if (rc != HIGGS_OK) return rc;
+    return launch_layer_error(*d, canonical, scales, grid, W, w_dtype, sums_out, st);
+}
+
+int higgs_allocate_bits(int32_t num_layers, int32_t num_options, const double* alpha, const double* t2, const int32_t* bits64,
+                        const int64_t* sizes, int64_t budget64, int32_t* choice_out, double* objective_out) {
+    return allocate_bits(num_layers, num_options, alpha, t2, bits64, sizes, budget64, choice_out, objective_out);
+}
+
 int higgs_rotate_activations(const higgs_desc* d, const void* x, int64_t B, void* xdag_out, void* stream) {
     int rc = check_desc(d);
     if (rc != HIGGS_OK) return rc;

@@ -148,6 +148,10 @@ int launch_convert_out(const float* y32, void* y, int y_dtype, size_t count, cud
 size_t make_grid_workspace(int p, int n, int64_t m);
 int launch_make_grid(int p, int n, const float* samples, int64_t m, int max_iters, float* grid_out, float* mse_out,
                      int32_t* iters_out, void* ws, cudaStream_t st);
+int launch_layer_error(const higgs_desc& d, const uint8_t* canonical, const void* scales, const float* grid, const void* W,
+                       int w_dtype, double* sums, cudaStream_t st);
+int allocate_bits(int L, int J, const double* alpha, const double* t2, const int32_t* bits64, const int64_t* sizes,
+                  int64_t budget64, int32_t* choice_out, double* objective_out);
 int launch_uniform_grid(int n, float* grid_out, float* step_out, float* mse_out, cudaStream_t st);
 int linear_k_chunks(const higgs_desc& d, int64_t B);
 // tensor-core path (B > 16)

@@ -261,6 +261,24 @@ def test_dequantize_matches_oracle(p, n, N, K):
     assert np.max(np.abs(W_bf - W_ref)) <= 2.0 ** -8 * np.max(np.abs(W_ref))
 
 
+@pytest.mark.parametrize("p,n,N,K", [(2, 256, 64, 2048), (2, 16, 32, 2048), (1, 256, 32, 1024)])
+def test_layer_error_matches_oracle(p, n, N, K):
+    """Section 5, 'Measuring Grid Parameters': the relative layer error t^2 against the oracle's, and against the
+    grid's own expected squared error (Appendix E: they agree for Gaussian-like rotated weights)."""
+    xi = inputs.rht_seed(3)
+    W = inputs.make_weights(N, K, seed=1200 + n, bf16=True)
+    g64, gt = U.grid32(p, n)
+    q, sc16 = U.oracle_encode(W, G, g64, xi)
+    d = hb.make_desc(p, n, N, K, xi)
+    packed = hb.higgs_pack_codes(d, torch.from_numpy(q.codes.astype(np.uint8)).to(U.dev()))
+    scales = hb.scales_to_tile_major(torch.from_numpy(sc16).to(U.dev()))
+    t2 = hb.higgs_layer_error(d, U.bf16_tensor(W), packed, scales, gt)
+    t2_ref = oracle.layer_error(W, q.codes, sc16.astype(np.float64), G, g64, xi)
+    assert abs(t2 - t2_ref) <= 2e-4 * t2_ref, (t2, t2_ref)
+    mse = oracle.grid_mse(g64, inputs.gaussian_samples(p, 99, log2_count=18))
+    assert abs(t2 - mse) <= (0.08 if n < 256 or p == 2 else 0.25) * mse, (t2, mse)
+
+
 # ----------------------------------------------------------------------------- tensor-core path (B > 16, N % 128 == 0)
 @pytest.mark.parametrize("p,n,N,K,B", [
     (2, 256, 128, 1024, 17),     # smallest tile: one block, 16 stages, token tile of 32
