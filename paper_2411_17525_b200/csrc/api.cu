@@ -105,7 +105,8 @@ int higgs_quantize(const higgs_desc* d, const void* W, int w_dtype, const float*
         return HIGGS_ERR_INVALID_ARG;
     }
     cudaStream_t st = as_stream(stream);
-    rc = launch_encode(*d, W, w_dtype, grid, canonical, scales_out, st);
+    // (the packed output is written by the pack kernel only: until then it lends the encoder its scratch space)
+    rc = launch_encode(*d, W, w_dtype, grid, canonical, scales_out, packed_out, higgs_packed_bytes(d), st);
     if (rc != HIGGS_OK) return rc;
     return launch_pack(*d, canonical, packed_out, st);
 }

@@ -137,7 +137,7 @@ int launch_rht_activations(const higgs_desc& d, const void* x, int64_t B, __half
 int launch_rht_debug(const higgs_desc& d, const void* x, int x_dtype, int64_t rows, float* out, int normalised,
                      cudaStream_t st);
 int launch_encode(const higgs_desc& d, const void* W, int w_dtype, const float* grid, uint8_t* canonical,
-                  void* scales, cudaStream_t st);
+                  void* scales, void* scratch, size_t scratch_bytes, cudaStream_t st);
 int launch_pack(const higgs_desc& d, const uint8_t* canonical, void* packed, cudaStream_t st);
 int launch_unpack(const higgs_desc& d, const void* packed, uint8_t* canonical, cudaStream_t st);
 int launch_dequantize(const higgs_desc& d, const uint8_t* canonical, const void* scales, const float* grid, void* W_out,

@@ -121,6 +121,139 @@ __global__ void __launch_bounds__(128) encode_kernel(const T* __restrict__ W, co
     }
 }
 
+// ---- exact pruned search ---------------------------------------------------------------------------------------
+// The same nearest-point rule as above, evaluated only on the grid points that can win.  The plane (the line for
+// p = 1) is cut into square cells over [-R, R)^p; for a cell, U = min over grid points of the distance to the cell's
+// farthest corner bounds the distance of the winner from any point of the cell, so only points whose distance to the
+// cell is at most U (+ a slack far above fp32 rounding) can be nearest.  Their indices are listed in ascending order,
+// so the strict '<' of the scan keeps the lowest index on ties exactly like the exhaustive scan.  Cells with more
+// than kMaxCand candidates, and inputs outside [-R, R)^p, fall back to the exhaustive scan.  The table is built once
+// by a small kernel (into scratch memory the caller lends: the packed-code output buffer, which is written only after
+// the encoder has finished) and copied into shared memory by every persistent encoder block.
+constexpr int kCells2 = 32;            // p = 2: 32 x 32 cells
+constexpr int kCells1 = 1024;          // p = 1
+constexpr int kMaxCand = 16;
+constexpr float kCellR = 4.0f;
+constexpr float kCandSlack = 1e-3f;
+
+template <int P>
+__global__ void __launch_bounds__(256) build_cells_kernel(const float* __restrict__ grid, int n, uint8_t* __restrict__ table) {
+    constexpr int NC = P == 2 ? kCells2 * kCells2 : kCells1;
+    __shared__ float sgrid[256 * 2];
+    for (int i = threadIdx.x; i < n * P; i += blockDim.x) sgrid[i] = grid[i];
+    __syncthreads();
+    uint8_t* cand = table;                       // [NC][kMaxCand]
+    uint8_t* cnt = table + NC * kMaxCand;        // [NC]
+    const float w = 2.0f * kCellR / (P == 2 ? kCells2 : kCells1);
+    for (int cell = blockIdx.x * blockDim.x + threadIdx.x; cell < NC; cell += gridDim.x * blockDim.x) {
+        const float x0 = -kCellR + w * (P == 2 ? (cell % kCells2) : cell), x1 = x0 + w;
+        const float y0 = P == 2 ? -kCellR + w * (cell / kCells2) : 0.f, y1 = y0 + w;
+        float U = INFINITY;
+        for (int c = 0; c < n; ++c) {
+            const float gx = sgrid[P * c], gy = P == 2 ? sgrid[2 * c + 1] : 0.f;
+            const float fx = fmaxf(fabsf(gx - x0), fabsf(gx - x1));
+            const float fy = P == 2 ? fmaxf(fabsf(gy - y0), fabsf(gy - y1)) : 0.f;
+            U = fminf(U, sqrtf(fx * fx + fy * fy));
+        }
+        int k = 0;
+        for (int c = 0; c < n; ++c) {
+            const float gx = sgrid[P * c], gy = P == 2 ? sgrid[2 * c + 1] : 0.f;
+            const float nx = fmaxf(fmaxf(x0 - gx, gx - x1), 0.f);
+            const float ny = P == 2 ? fmaxf(fmaxf(y0 - gy, gy - y1), 0.f) : 0.f;
+            if (sqrtf(nx * nx + ny * ny) <= U + kCandSlack) {
+                if (k < kMaxCand) cand[cell * kMaxCand + k] = (uint8_t)c;
+                ++k;
+            }
+        }
+        cnt[cell] = k <= kMaxCand ? (uint8_t)k : (uint8_t)255;
+    }
+}
+
+template <typename T, int P>
+__global__ void __launch_bounds__(256) encode_pruned_kernel(const T* __restrict__ W, const float* __restrict__ grid, int n,
+                                                            const uint8_t* __restrict__ table,
+                                                            uint8_t* __restrict__ canonical, __half* __restrict__ scales,
+                                                            int64_t N, int64_t K, uint64_t xi) {
+    constexpr int NC = P == 2 ? kCells2 * kCells2 : kCells1;
+    __shared__ float sgrid[256 * 2];
+    __shared__ __align__(16) uint8_t cand[NC * kMaxCand + NC];
+    const uint8_t* cnt = cand + NC * kMaxCand;
+    for (int i = threadIdx.x; i < n * P; i += blockDim.x) sgrid[i] = grid[i];
+    for (int i = threadIdx.x; i < (NC * kMaxCand + NC) / 16; i += blockDim.x)
+        reinterpret_cast<uint4*>(cand)[i] = reinterpret_cast<const uint4*>(table)[i];
+    __syncthreads();
+
+    const int lane = threadIdx.x & 31;
+    const int64_t groups = K / kGroup;
+    const int64_t tasks = N * groups;
+    const int64_t warps_total = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const float inv_w = (P == 2 ? kCells2 : kCells1) / (2.0f * kCellR);
+    for (int64_t task = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); task < tasks; task += warps_total) {
+        const int64_t row = task / groups, gi = task % groups;
+        float v[32];
+        load32<T>(W + row * K + gi * kGroup, lane, v);
+        float ss = 0.0f;
+#pragma unroll
+        for (int r = 0; r < 32; ++r) ss = fmaf(v[r], v[r], ss);
+#pragma unroll
+        for (int m = 16; m >= 1; m >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, m);
+        const float s = sqrtf(ss);
+        const float inv = s > 0.0f ? 1.0f / s : 0.0f;
+#pragma unroll
+        for (int r = 0; r < 32; ++r) v[r] *= inv;
+        apply_signs1024(v, xi, gi * kGroup, lane);
+        fwht1024_warp(v, lane);
+        if (lane == 0) scales[((row >> 4) * groups + gi) * 16 + (row & 15)] = __float2half_rn(s * 0.03125f);
+
+        int bi[32 / P];
+#pragma unroll
+        for (int t = 0; t < 32 / P; ++t) {
+            const float x = v[P * t], y = P == 2 ? v[2 * t + 1] : 0.f;
+            const float cx = (x + kCellR) * inv_w, cy = P == 2 ? (y + kCellR) * inv_w : 0.f;
+            const bool inside = cx >= 0.f && cx < (float)(P == 2 ? kCells2 : kCells1) &&
+                                (P == 1 || (cy >= 0.f && cy < (float)kCells2));
+            const int cell = inside ? (P == 2 ? (int)cy * kCells2 + (int)cx : (int)cx) : 0;
+            const int k = inside ? cnt[cell] : 255;
+            float best = INFINITY;
+            int b = 0;
+            if (k != 255) {
+                for (int i = 0; i < k; ++i) {
+                    const int c = cand[cell * kMaxCand + i];
+                    const float dx = x - sgrid[P * c], dy = P == 2 ? y - sgrid[2 * c + 1] : 0.f;
+                    const float d = P == 2 ? fmaf(dy, dy, dx * dx) : dx * dx;
+                    if (d < best) { best = d; b = c; }
+                }
+            } else {
+                for (int c = 0; c < n; ++c) {
+                    const float dx = x - sgrid[P * c], dy = P == 2 ? y - sgrid[2 * c + 1] : 0.f;
+                    const float d = P == 2 ? fmaf(dy, dy, dx * dx) : dx * dx;
+                    if (d < best) { best = d; b = c; }
+                }
+            }
+            bi[t] = b;
+        }
+        if (P == 2) {
+            uint8_t* dst = canonical + row * (K / 2) + gi * (kGroup / 2);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t w = (uint32_t)bi[c * 4] | ((uint32_t)bi[c * 4 + 1] << 8) | ((uint32_t)bi[c * 4 + 2] << 16) |
+                             ((uint32_t)bi[c * 4 + 3] << 24);
+                *reinterpret_cast<uint32_t*>(dst + c * 128 + lane * 4) = w;
+            }
+        } else {
+            uint8_t* dst = canonical + row * K + gi * kGroup;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t w0 = (uint32_t)bi[c * 8] | ((uint32_t)bi[c * 8 + 1] << 8) | ((uint32_t)bi[c * 8 + 2] << 16) |
+                              ((uint32_t)bi[c * 8 + 3] << 24);
+                uint32_t w1 = (uint32_t)bi[c * 8 + 4] | ((uint32_t)bi[c * 8 + 5] << 8) | ((uint32_t)bi[c * 8 + 6] << 16) |
+                              ((uint32_t)bi[c * 8 + 7] << 24);
+                *reinterpret_cast<uint2*>(dst + c * 256 + lane * 8) = make_uint2(w0, w1);
+            }
+        }
+    }
+}
+
 // ---- packed layout -----------------------------------------------------------
 // The packed stream is a sequence of blocks, block (rt, kb) covering rows
 // [16 rt, 16 rt + 16) and inputs [64 kb, 64 kb + 64), stored at block index
@@ -282,17 +415,29 @@ __global__ void __launch_bounds__(256) unpack_kernel(const uint32_t* __restrict_
 }  // namespace
 
 int launch_encode(const higgs_desc& d, const void* W, int w_dtype, const float* grid, uint8_t* canonical, void* scales,
-                  cudaStream_t st) {
+                  void* scratch, size_t scratch_bytes, cudaStream_t st) {
     const int64_t warps = d.N * (d.K / kGroup);
     if (warps == 0) return HIGGS_OK;
     const unsigned blocks = (unsigned)((warps + 3) / 4);
     __half* sc = static_cast<__half*>(scales);
+    // Large grids on large layers: the exact pruned search (persistent blocks that build their candidate table once);
+    // otherwise the exhaustive scan, whose cost is small there.
+    constexpr size_t kTableBytes = (size_t)(kCells1 > kCells2 * kCells2 ? kCells1 : kCells2 * kCells2) * (kMaxCand + 1);
+    const bool pruned = d.n >= 64 && warps >= 2048 && scratch && scratch_bytes >= kTableBytes &&
+                        (reinterpret_cast<uintptr_t>(scratch) % 16) == 0;
+    const unsigned pblocks = 592;          // 4 blocks of 8 warps per SM on a 148-SM part; any count is correct
+    uint8_t* table = static_cast<uint8_t*>(scratch);
+    if (pruned) {
+        if (d.p == 2) build_cells_kernel<2><<<4, 256, 0, st>>>(grid, d.n, table);
+        else build_cells_kernel<1><<<4, 256, 0, st>>>(grid, d.n, table);
+    }
 #define HIGGS_ENC(T, P) \
-    encode_kernel<T, P><<<blocks, 128, 0, st>>>(static_cast<const T*>(W), grid, d.n, canonical, sc, d.N, d.K, d.rht_seed)
-    if (w_dtype == HIGGS_F32 && d.p == 2) HIGGS_ENC(float, 2);
-    else if (w_dtype == HIGGS_F32 && d.p == 1) HIGGS_ENC(float, 1);
-    else if (w_dtype == HIGGS_BF16 && d.p == 2) HIGGS_ENC(__nv_bfloat16, 2);
-    else if (w_dtype == HIGGS_BF16 && d.p == 1) HIGGS_ENC(__nv_bfloat16, 1);
+    if (pruned) encode_pruned_kernel<T, P><<<pblocks, 256, 0, st>>>(static_cast<const T*>(W), grid, d.n, table, canonical, sc, d.N, d.K, d.rht_seed); \
+    else encode_kernel<T, P><<<blocks, 128, 0, st>>>(static_cast<const T*>(W), grid, d.n, canonical, sc, d.N, d.K, d.rht_seed)
+    if (w_dtype == HIGGS_F32 && d.p == 2) { HIGGS_ENC(float, 2); }
+    else if (w_dtype == HIGGS_F32 && d.p == 1) { HIGGS_ENC(float, 1); }
+    else if (w_dtype == HIGGS_BF16 && d.p == 2) { HIGGS_ENC(__nv_bfloat16, 2); }
+    else if (w_dtype == HIGGS_BF16 && d.p == 1) { HIGGS_ENC(__nv_bfloat16, 1); }
     else return HIGGS_ERR_UNSUPPORTED;
 #undef HIGGS_ENC
     return cuda_status(cudaGetLastError());

@@ -68,3 +68,23 @@ def test_full_size_layer_on_sampled_rows(name, N, K, p, n, batches):
         xd = hb.higgs_rotate_activations(d, U.bf16_tensor(x))
         y2 = hb.higgs_linear_prerotated(d, xd, packed2, scales2, gt, B=B)
         assert float((y2 - y).abs().max()) <= 1e-5 * float(y.abs().max())
+
+
+@pytest.mark.parametrize("p,n,N,K", [(2, 256, 8192, 2048), (2, 64, 4096, 4096), (1, 256, 8192, 1024)])
+def test_pruned_search_equals_exhaustive_scan(p, n, N, K):
+    """Large layers are encoded with the exact pruned nearest-point search, small ones with the exhaustive scan: rows are
+    independent, so re-encoding a slice of the rows as a small matrix must give the very same codes and scales."""
+    cfg = 2
+    xi = inputs.rht_seed(cfg)
+    W = inputs.make_weights(N, K, inputs.weight_seed(cfg, 5), bf16=True)
+    W[7, :] *= 40.0                                     # a row of large values changes nothing (groups are normalised)
+    W[9, 100:110] = 3.0                                 # a few huge entries: rotated values beyond the cell table's range
+    W = inputs.bf16_round(W)
+    _, gt = U.grid32(p, n)
+    d = hb.make_desc(p, n, N, K, xi)
+    packed, scales, canon = hb.higgs_quantize(d, U.bf16_tensor(W), gt, want_canonical=True)
+    rows = 64
+    ds = hb.make_desc(p, n, rows, K, xi)
+    packed_s, scales_s, canon_s = hb.higgs_quantize(ds, U.bf16_tensor(W[:rows]), gt, want_canonical=True)
+    assert torch.equal(canon[:rows], canon_s)
+    assert torch.equal(hb.scales_from_tile_major(scales, N)[:rows], hb.scales_from_tile_major(scales_s, rows))
