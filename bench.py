@@ -257,7 +257,10 @@ def run_ours(args):
         descs.append(d)
         packed.append([pk] + [pk.clone() for _ in range(copies - 1)])
         scales.append([sc] + [sc.clone() for _ in range(copies - 1)])
-        xh = torch.from_numpy(inputs.make_activations(B, K, inputs.activation_seed(cfg, B) + li)).to(torch.bfloat16)
+        # q/k/v read the same block input, so do gate/up
+        xi_of = {"k": "q", "v": "q", "up": "gate"}.get(name, name)
+        x_seed = inputs.activation_seed(cfg, B) + [nm for nm, _, _ in layers].index(xi_of)
+        xh = torch.from_numpy(inputs.make_activations(B, K, x_seed)).to(torch.bfloat16)
         xs_host.append(xh.pin_memory())
         xs.append(xh.to(dev))
         ws.append(torch.empty(hb.higgs_linear_host_workspace_bytes(d, B), dtype=torch.uint8, device=dev))
@@ -278,8 +281,10 @@ def run_ours(args):
              for k, v in groups_of.items() if len(v) > 1}
     launches_per_step = 0
     for k, v in groups_of.items():
-        launches_per_step += (1 + sum(hb.higgs_linear_launch_count(descs[li], B) - 1 for li in v)) if len(v) > 1 \
-            else hb.higgs_linear_launch_count(descs[v[0]], B)
+        if len(v) > 1:      # one rotation, then one product launch per layer (per 16 tokens on the small-batch path)
+            launches_per_step += 1 + sum(1 if hb.higgs_rotated_layout(descs[li], B) > 0 else -(-B // 16) for li in v)
+        else:
+            launches_per_step += hb.higgs_linear_launch_count(descs[v[0]], B)
 
     def step(i):
         c = i % copies
@@ -517,7 +522,7 @@ def run_ours(args):
                        "global_batch": B * world, "parallelism": f"replicas x{world}",
                        "l2": f"rotating {copies} weight copies ({copies * set_bytes / 1e6:.0f} MB > 126 MB L2)",
                        "launch": "direct" if graphs is None else "one CUDA graph per weight copy",
-                       "step": "one transformer block: activation rotations (q/k/v and gate/up share theirs where the layout allows) + 7 products"},
+                       "step": "one transformer block: activation rotations (q/k/v and gate/up share theirs where the layout allows; a layer with its own rotation has it fused into the product kernel for 1-2 tokens when K is not split) + 7 products"},
             "us_per_layer": ms_per_step * 1e3 / len(layers),
             "weight_bytes_per_step": set_bytes,
             "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

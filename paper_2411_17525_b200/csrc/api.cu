@@ -209,6 +209,11 @@ int higgs_linear(const higgs_desc* d, const void* x, int64_t B, const void* pack
         return launch_linear_tc(*d, static_cast<const __half*>(workspace), B, packed, scales, grid, y,
                                 y_dtype == HIGGS_F32 ? 0 : 1, st);
     }
+    if (linear_fused_eligible(*d, B)) {
+        // one or two tokens, K not split: the product kernel rotates the activations itself (D1 fused into D2-D5)
+        void* yo = y;
+        return launch_linear_mma(*d, nullptr, B, packed, scales, grid, yo, d->N, y_dtype == HIGGS_F32 ? 0 : 1, st, x);
+    }
     __half* xdag = static_cast<__half*>(workspace);
     float* y32 = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up((size_t)B * d->K * 2, 256));
     const bool split = linear_k_chunks(*d, B) > 1;
@@ -285,6 +290,7 @@ int higgs_linear_k_splits(const higgs_desc* d, int64_t B) {
 int higgs_linear_launch_count(const higgs_desc* d, int64_t B, int y_dtype) {
     if (check_desc(d) != HIGGS_OK || B < 1 || d->N == 0) return 0;
     if (tc_eligible(*d, B)) return 2;
+    if (linear_fused_eligible(*d, B)) return 1;
     const bool split = linear_k_chunks(*d, B) > 1;
     return 1 + (int)((B + 15) / 16) + ((split && y_dtype == HIGGS_BF16) ? 1 : 0);
 }

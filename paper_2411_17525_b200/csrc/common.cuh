@@ -142,8 +142,10 @@ int launch_pack(const higgs_desc& d, const uint8_t* canonical, void* packed, cud
 int launch_unpack(const higgs_desc& d, const void* packed, uint8_t* canonical, cudaStream_t st);
 int launch_dequantize(const higgs_desc& d, const uint8_t* canonical, const void* scales, const float* grid, void* W_out,
                       int w_dtype, cudaStream_t st);
+// x_raw != nullptr: the activations as given (bf16); the kernel rotates them itself (only if linear_fused_eligible)
 int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const void* packed, const void* scales,
-                      const float* grid, void* y, int64_t ldy, int y_mode, cudaStream_t st);
+                      const float* grid, void* y, int64_t ldy, int y_mode, cudaStream_t st, const void* x_raw = nullptr);
+bool linear_fused_eligible(const higgs_desc& d, int64_t B);
 int launch_convert_out(const float* y32, void* y, int y_dtype, size_t count, cudaStream_t st);
 size_t make_grid_workspace(int p, int n, int64_t m);
 int launch_make_grid(int p, int n, const float* samples, int64_t m, int max_iters, float* grid_out, float* mse_out,

@@ -46,6 +46,8 @@ __device__ __forceinline__ unsigned long long gtime_ns() { unsigned long long t;
 namespace {
 
 struct StreamParams {
+    const __nv_bfloat16* x;   // fused-rotation kernels only: [B][K] activations as the caller gave them
+    unsigned long long xi;    // ... and the seed of the sign sequence
     const __half* xdag;    // [B][K] rotated activations, fp16
     const uint8_t* packed; // packed code stream
     const __half* scales;  // tile-major scales [N/16][K/g][16]
@@ -239,9 +241,14 @@ struct TaskCodes {
     }
 };
 
-template <int NB, int KS, int FMT>
+// FUSED (NB = 1, B <= 2, K not split): the kernel takes the activations as given and rotates them itself (Appendix F's
+// x+ = (H / sqrt(g)) diag(sign) x) - the four warps that own the four 256-input slices of a 1024-group transform it
+// together: butterflies over a lane's 8 values in registers, over the 32 lanes by shuffles, over the 4 warps through
+// shared memory - so that no rotation kernel (and no hand-over between two dependent launches) precedes the product.
+template <int NB, int KS, int FMT, bool FUSED>
 __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(const StreamParams prm) {
     constexpr bool SIX = FMT == 1, NIB = FMT == 2, B8 = FMT == 3;
+    static_assert(!FUSED || (NB == 1 && KS == 256), "the fused rotation maps one warp to one 256-input slice");
     constexpr uint32_t kPieceStride = NIB ? 128u : 256u;     // bytes between consecutive 128-byte pieces of the partial tiles
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -415,12 +422,100 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
         }
     };
     int c_item = phase;                  // compute cursor: this warp's next item of the block
-    if (n_tasks > 0) load_bfrag(chunk_begin);
-
+    // (fused rotation: the activations are requested first, then the ring is armed, then they are transformed while
+    // the first weights are on their way)
+    uint4 xraw[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
+    const int64_t kbase = (int64_t)chunk_begin * prm.ck + (int64_t)slice * KS;
+    if (!FUSED) {
+        if (n_tasks > 0) load_bfrag(chunk_begin);
+    } else if (!flusher) {
+#pragma unroll
+        for (int b = 0; b < 2; ++b)
+            if (b < prm.B) xraw[b] = *reinterpret_cast<const uint4*>(prm.x + (int64_t)b * prm.K + kbase + lane * 8);
+    }
     int issued = 0;
     TRACEP(warp, 2);
     for (; issued < n_tasks && issued < D; ++issued) issue(issued);
     TRACEP(warp, 3);
+    if (FUSED && !flusher) {
+        // Scratch in the (still unused) partial-tile area, addressed in 128-byte pieces: bytes [0, 16 KB) exchange
+        // buffers of the four warp units, then 512 bytes per (warp, token) for the slice in fragment order.
+        auto scratch = [&](uint32_t off) { return part0 + (off >> 7) * kPieceStride + (off & 127u); };
+        const int unit = warp >> 2, quarter = warp & 3;       // the unit's four warps hold the four slices of one group
+#pragma unroll
+        for (int b = 0; b < 2; ++b) {
+            if (b >= prm.B) break;
+            float v[8];
+            {
+                const uint4 q4 = xraw[b];
+                const uint32_t w4[4] = {q4.x, q4.y, q4.z, q4.w};
+                const uint64_t j0 = (uint64_t)kbase + (uint64_t)(lane * 8);
+                const uint32_t bits = (uint32_t)(sign_word(prm.xi, j0 >> 6) >> (j0 & 63ull)) & 0xffu;
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    v[2 * e] = __uint_as_float((w4[e] << 16) ^ (((bits >> (2 * e)) & 1u) << 31));
+                    v[2 * e + 1] = __uint_as_float((w4[e] & 0xffff0000u) ^ (((bits >> (2 * e + 1)) & 1u) << 31));
+                }
+            }
+#pragma unroll
+            for (int h = 1; h < 8; h <<= 1) {
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    if ((r & h) == 0) { const float a = v[r], c = v[r | h]; v[r] = a + c; v[r | h] = a - c; }
+                }
+            }
+#pragma unroll
+            for (int m = 1; m < 32; m <<= 1) {
+                const bool upper = (lane & m) != 0;
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    const float o = __shfl_xor_sync(0xffffffffu, v[r], m);
+                    v[r] = upper ? (o - v[r]) : (v[r] + o);
+                }
+            }
+            // the last two stages run over the unit's four warps
+            const uint32_t ex = (uint32_t)(unit * 4096 + lane * 32);
+            asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(scratch(ex + quarter * 1024)), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]) : "memory");
+            asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(scratch(ex + quarter * 1024 + 16)), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]) : "memory");
+            asm volatile("bar.sync %0, 128;" ::"r"(1 + unit) : "memory");
+            float o[8];
+#pragma unroll
+            for (int r = 0; r < 8; ++r) o[r] = 0.f;
+#pragma unroll
+            for (int qq = 0; qq < 4; ++qq) {
+                const uint4 u0 = lds128(scratch(ex + qq * 1024)), u1 = lds128(scratch(ex + qq * 1024 + 16));
+                const float sgn = (__popc(quarter & qq) & 1) ? -1.f : 1.f;
+                o[0] = fmaf(sgn, __uint_as_float(u0.x), o[0]); o[1] = fmaf(sgn, __uint_as_float(u0.y), o[1]);
+                o[2] = fmaf(sgn, __uint_as_float(u0.z), o[2]); o[3] = fmaf(sgn, __uint_as_float(u0.w), o[3]);
+                o[4] = fmaf(sgn, __uint_as_float(u1.x), o[4]); o[5] = fmaf(sgn, __uint_as_float(u1.y), o[5]);
+                o[6] = fmaf(sgn, __uint_as_float(u1.z), o[6]); o[7] = fmaf(sgn, __uint_as_float(u1.w), o[7]);
+            }
+            asm volatile("bar.sync %0, 128;" ::"r"(1 + unit) : "memory");      // the exchange buffer is reused by the next token
+            // this lane holds inputs 8 lane .. + 7 of the slice: pairs 4 j + i (j = lane & 7) of 64-input block lane >> 3
+            // -> fragment-order position i * 8 + j
+            const uint32_t st = (uint32_t)(16384 + (warp * 2 + b) * 512 + (lane >> 3) * 128 + (lane & 7) * 4);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const __half2 hh = __floats2half2_rn(o[2 * i] * 0.03125f, o[2 * i + 1] * 0.03125f);
+                asm volatile("st.shared.b32 [%0], %1;" ::"r"(scratch(st + i * 32)), "r"(*reinterpret_cast<const uint32_t*>(&hh)) : "memory");
+            }
+        }
+        __syncwarp();
+#pragma unroll
+        for (int jb = 0; jb < KS / 64; ++jb) {
+            uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = make_uint4(0u, 0u, 0u, 0u);
+            if (g < prm.B) {
+                const uint32_t a = (uint32_t)(16384 + (warp * 2 + g) * 512 + jb * 128 + t * 32);
+                lo = lds128(scratch(a));
+                hi = lds128(scratch(a + 16));
+            }
+            bfrag[jb * 4 + 0][0][0] = lo.x; bfrag[jb * 4 + 0][0][1] = lo.y;
+            bfrag[jb * 4 + 1][0][0] = lo.z; bfrag[jb * 4 + 1][0][1] = lo.w;
+            bfrag[jb * 4 + 2][0][0] = hi.x; bfrag[jb * 4 + 2][0][1] = hi.y;
+            bfrag[jb * 4 + 3][0][0] = hi.z; bfrag[jb * 4 + 3][0][1] = hi.w;
+        }
+    }
+
 
     {
 #pragma unroll
@@ -672,18 +767,18 @@ Plan make_plan(const higgs_desc& d, int64_t B) {
     return best;
 }
 
-template <int NB, int KS, int FMT>
+template <int NB, int KS, int FMT, bool FUSED = false>
 int launch_one(const StreamParams& prm, int blocks, cudaStream_t st) {
     static bool configured[64] = {false};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(linear_stream_kernel<NB, KS, FMT>,
+        cudaError_t e = cudaFuncSetAttribute(linear_stream_kernel<NB, KS, FMT, FUSED>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem);
         if (e != cudaSuccess) return HIGGS_ERR_CUDA;
         configured[dev] = true;
     }
-    return cuda_status(launch_pdl(linear_stream_kernel<NB, KS, FMT>, dim3((unsigned)blocks), dim3((kWarps + 1) * 32),
+    return cuda_status(launch_pdl(linear_stream_kernel<NB, KS, FMT, FUSED>, dim3((unsigned)blocks), dim3((kWarps + 1) * 32),
                                   kMaxDynSmem, st, prm));
 }
 
@@ -691,13 +786,22 @@ int launch_one(const StreamParams& prm, int blocks, cudaStream_t st) {
 
 int linear_k_chunks(const higgs_desc& d, int64_t B) { return make_plan(d, B > 16 ? 16 : B).chunks; }
 
+// The rotation can be fused into the product kernel for one or two tokens when K is not split over thread blocks.
+bool linear_fused_eligible(const higgs_desc& d, int64_t B) {
+    return B >= 1 && B <= 2 && d.N > 0 && make_plan(d, B).chunks == 1;
+}
+
 // y_mode: 0 store fp32, 1 store bf16, 2 atomicAdd fp32 (target must be zero).  B <= 16.
 int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const void* packed, const void* scales,
-                      const float* grid, void* y, int64_t ldy, int y_mode, cudaStream_t st) {
+                      const float* grid, void* y, int64_t ldy, int y_mode, cudaStream_t st, const void* x_raw) {
     if (d.N == 0) return HIGGS_OK;
     const Plan pl = make_plan(d, B);
     if (pl.items == 0) return HIGGS_ERR_UNSUPPORTED;
+    const bool fused = x_raw != nullptr;
+    if (fused && !linear_fused_eligible(d, B)) return HIGGS_ERR_INVALID_ARG;
     StreamParams prm;
+    prm.x = static_cast<const __nv_bfloat16*>(x_raw);
+    prm.xi = d.rht_seed;
     prm.xdag = xdag;
     prm.packed = static_cast<const uint8_t*>(packed);
     prm.scales = static_cast<const __half*>(scales);
@@ -728,6 +832,9 @@ int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const 
     uint32_t lut_unused;
     ring_layout(kAssumedBase, (uint32_t)(six ? pl.ks * 6 : nib ? pl.ks * 4 : b8 ? pl.ks * 16 : pl.ks * 8) + 64u,
                 nib ? kNibbleTileBytes : 0u, &lut_unused, &prm.depth, &prm.warps_in_a);
+    if (fused)
+        return six ? launch_one<1, 256, 1, true>(prm, pl.blocks, st) : nib ? launch_one<1, 256, 2, true>(prm, pl.blocks, st)
+             : b8 ? launch_one<1, 256, 3, true>(prm, pl.blocks, st) : launch_one<1, 256, 0, true>(prm, pl.blocks, st);
     if (pl.nb == 1)
         return six ? launch_one<1, 256, 1>(prm, pl.blocks, st) : nib ? launch_one<1, 256, 2>(prm, pl.blocks, st)
              : b8 ? launch_one<1, 256, 3>(prm, pl.blocks, st) : launch_one<1, 256, 0>(prm, pl.blocks, st);
