@@ -164,8 +164,15 @@ int higgs_quantize(const higgs_desc* desc, const void* W, int w_dtype, const flo
  *   scales   device, tile-major fp16 scales as written by higgs_quantize
  *   grid     device, [n][p] fp32
  *   y        device, [B][N] row-major, y_dtype in {HIGGS_F32, HIGGS_BF16}
- * When K is split over several thread blocks the partial sums meet in fp32
- * atomics, so the last bits of y may differ from run to run.
+ * Kernels behind the call: for one or two tokens (K not split) a single kernel
+ * that rotates the activations in its prologue; up to 16 tokens a rotation
+ * kernel and the small-batch product kernel; above that (and from 9 tokens
+ * for layers above 32 M weights) a rotation kernel and the tcgen05 kernel.
+ * When the small-batch kernel splits K over several thread blocks the partial
+ * sums meet in fp32 atomics, so the last bits of y may differ from run to run;
+ * every other path is bit-reproducible.  The one-call form and the two-call
+ * form below agree to fp16 rounding of x+ (the fused prologue orders the
+ * butterflies differently), not bit for bit.
  */
 int higgs_linear(const higgs_desc* desc, const void* x, int64_t B,
                  const void* packed, const void* scales, const float* grid,
@@ -185,7 +192,7 @@ int higgs_linear(const higgs_desc* desc, const void* x, int64_t B,
  *   higgs_linear_prerotated: the product of Appendix F on already rotated
  *     activations; other arguments as higgs_linear.  xdag may be shared by
  *     layers with the same K, seed and higgs_rotated_layout (e.g. q, k, v).
- * higgs_linear(x) == higgs_linear_prerotated(higgs_rotate_activations(x)).
+ * higgs_linear(x) computes what higgs_linear_prerotated(higgs_rotate_activations(x)) does.
  */
 int higgs_rotate_activations(const higgs_desc* desc, const void* x, int64_t B, void* xdag_out, void* stream);
 size_t higgs_rotated_bytes(const higgs_desc* desc, int64_t B);
