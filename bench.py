@@ -246,9 +246,11 @@ def run_ours(args):
     for li, (name, N, K) in enumerate(layers):
         d = hb.make_desc(pn[li][0], pn[li][1], N, K, xi)
         W = torch.from_numpy(inputs.make_weights(N, K, inputs.weight_seed(cfg, li), bf16=True)).to(dev).to(torch.bfloat16)
+        pk, sc, _ = hb.higgs_quantize(d, W, grids[pn[li]])       # first call: the allocator fetches the output buffers
+        torch.cuda.synchronize()
         e0, e1 = ev(), ev()
         e0.record()
-        pk, sc, _ = hb.higgs_quantize(d, W, grids[pn[li]])
+        pk, sc, _ = hb.higgs_quantize(d, W, grids[pn[li]])       # timed: encode + pack kernels of the whole layer
         e1.record()
         torch.cuda.synchronize()
         enc_ms += e0.elapsed_time(e1)
