@@ -47,6 +47,9 @@ def parse_args():
                     help="p,n for every layer, or 'mixed': 3 or 4 bits per matrix (p=2 n=64 / n=256) from the seeded assignment "
                          "averaging 3.5 bits (the Llama-3.1-70B configuration)")
     ap.add_argument("--no-graph", action="store_true", help="launch kernels directly instead of replaying CUDA graphs")
+    ap.add_argument("--steps-per-graph", type=int, default=8,
+                    help="consecutive steps (over rotating weight copies) captured in one CUDA graph; a remainder of --steps runs "
+                         "from one-step graphs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-detail", action="store_true", help="skip the per-layer / other-batch detail measurements")
     return ap.parse_args()
@@ -312,6 +315,8 @@ def run_ours(args):
     with torch.cuda.stream(stream):
         step(0)
         stream.synchronize()
+        spg = max(1, args.steps_per_graph)
+        graphs_multi = None
         if not args.no_graph:
             graphs = []
             for c in range(copies):
@@ -319,12 +324,34 @@ def run_ours(args):
                 with torch.cuda.graph(g, stream=stream):
                     step(c)
                 graphs.append(g)
+            if spg > 1:          # the same steps, spg of them per graph: a graph boundary costs about 2 us on the device
+                graphs_multi = []
+                for c in range(copies):
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=stream):
+                        for k in range(spg):
+                            step(c * spg + k)
+                    graphs_multi.append(g)
 
-    def run_step(i):
-        if graphs is not None:
-            graphs[i % copies].replay()
-        else:
-            step(i)
+    def run_steps(first, count):      # exactly `count` steps, starting with step number `first`
+        i = first
+        while count > 0:
+            if graphs_multi is not None and count >= spg:
+                graphs_multi[(i // spg) % copies].replay()
+                i += spg
+                count -= spg
+            elif graphs is not None:
+                graphs[i % copies].replay()
+                i += 1
+                count -= 1
+            else:
+                step(i)
+                i += 1
+                count -= 1
+
+    def run_steps_host(first, count):
+        for i in range(first, first + count):
+            step_host(i)
 
     def barrier():
         if world > 1:
@@ -332,15 +359,13 @@ def run_ours(args):
 
     def timed(fn, steps, warmup):
         with torch.cuda.stream(stream):
-            for i in range(warmup):
-                fn(i)
+            fn(0, warmup)
             stream.synchronize()
             barrier()
             torch.cuda.synchronize()
             a, b = ev(), ev()
             a.record(stream)
-            for i in range(steps):
-                fn(warmup + i)
+            fn(warmup, steps)
             b.record(stream)
             torch.cuda.synchronize()
             barrier()
@@ -350,8 +375,8 @@ def run_ours(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    ms = timed(run_step, args.steps, max(args.warmup, 3))
-    ms_e2e = timed(step_host, args.steps, max(args.warmup, 3))
+    ms = timed(run_steps, args.steps, max(args.warmup, 3))
+    ms_e2e = timed(run_steps_host, args.steps, max(args.warmup, 3))
     clocks = sampler.stop() if rank == 0 else None
 
     ms_per_step = ms / args.steps
@@ -476,7 +501,11 @@ def run_ours(args):
                 with torch.cuda.graph(g, stream=stream):
                     fused_step(c)
                 fgraphs.append(g)
-        ms_f = timed(lambda i: fgraphs[i % copies].replay(), args.steps, max(args.warmup, 3))
+        def run_fused(first, count):
+            for i in range(first, first + count):
+                fgraphs[i % copies].replay()
+
+        ms_f = timed(run_fused, args.steps, max(args.warmup, 3))
         # the concatenated launch computes the same rows: compare with the per-layer outputs of the last plain step
         with torch.cuda.stream(stream):
             step(0)
@@ -523,7 +552,8 @@ def run_ours(args):
             "config": {"workload": f"{args.workload} layer set ({len(layers)} matrices), grid {grid_text}, g=1024, batch {B}",
                        "global_batch": B * world, "parallelism": f"replicas x{world}",
                        "l2": f"rotating {copies} weight copies ({copies * set_bytes / 1e6:.0f} MB > 126 MB L2)",
-                       "launch": "direct" if graphs is None else "one CUDA graph per weight copy",
+                       "launch": "direct" if graphs is None else (f"CUDA graphs of {spg} consecutive steps (rotating weight copies), remainder from one-step graphs"
+                                                                  if graphs_multi is not None else "one CUDA graph per step"),
                        "step": "one transformer block: activation rotations (q/k/v and gate/up share theirs where the layout allows; a layer with its own rotation has it fused into the product kernel for 1-2 tokens when K is not split) + 7 products"},
             "us_per_layer": ms_per_step * 1e3 / len(layers),
             "weight_bytes_per_step": set_bytes,
