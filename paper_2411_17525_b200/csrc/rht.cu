@@ -37,41 +37,86 @@ __device__ __forceinline__ void load_group<float>(const float* __restrict__ src,
     }
 }
 
-// One warp per (token, group): x+ = (H/32) diag(sign) x, written as fp16 in "fragment order": inside every block of
-// 64 inputs the 32 input pairs are permuted so that the eight pairs one lane of the product kernel needs as
-// m16n8k16 B-fragment registers (steps m = 0..3, halves h = 0..1 of its column pair t) are 32 contiguous bytes:
-// position t*8 + m*2 + h holds pair 8m + t + 4h.  Extra threads beyond the transform work clear `zero_ptr` (the fp32
-// accumulation target of a K-split product) so no separate memset launch is needed.
+// Four warps per (token, group), one block of 128 threads each: x+ = (H/32) diag(sign) x, written as fp16 in "fragment
+// order": inside every block of 64 inputs the 32 input pairs are permuted so that the eight pairs one lane of the
+// product kernel needs as m16n8k16 B-fragment registers (steps m = 0..3, halves h = 0..1 of its column pair t) are 32
+// contiguous bytes: position t*8 + m*2 + h holds pair 8m + t + 4h.  Warp q of the block owns inputs 256 q .. + 255 of
+// the group, 8 per lane: butterflies over those 8 in registers, over the 32 lanes by shuffles, over the 4 warps
+// through shared memory (the transform is on the latency path between two dependent product launches, so it is
+// spread over four warps instead of one).  Threads also clear `zero_ptr` (the fp32 accumulation target of a K-split
+// product) so that no separate memset launch is needed.
 template <typename T>
-__global__ void __launch_bounds__(256) rht_activations_kernel(const T* __restrict__ x, __half* __restrict__ xdag,
+__global__ void __launch_bounds__(128) rht_activations_kernel(const T* __restrict__ x, __half* __restrict__ xdag,
                                                               int64_t B, int64_t K, uint64_t xi,
                                                               float* __restrict__ zero_ptr, size_t zero_floats) {
-    const int lane = threadIdx.x & 31;
-    const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    __shared__ __align__(16) float ex[4][256];
+    const int lane = threadIdx.x & 31, q = threadIdx.x >> 5;
     const int64_t groups = K / kGroup;
     const size_t gtid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     const size_t gthreads = (size_t)gridDim.x * blockDim.x;
     pdl_trigger();     // the product kernel may start its table build and weight prefetch now
     pdl_wait();        // x may be the previous kernel's output; the buffers written below may still be read by it
     for (size_t i = gtid; i < zero_floats; i += gthreads) zero_ptr[i] = 0.0f;
-    if (warp >= B * groups) return;
-    const int64_t b = warp / groups, gi = warp % groups;
-    float v[32];
-    load_group<T>(x + b * K + gi * kGroup, lane, v);
-    apply_signs1024(v, xi, gi * kGroup, lane);
-    fwht1024_warp(v, lane);
-    uint32_t* dst = reinterpret_cast<uint32_t*>(xdag + b * K + gi * kGroup);
-    // this lane's chunk c holds inputs c*256 + lane*8 .. +7: pairs 4j + i (i = 0..3) of 64-input block c*4 + lane/8,
-    // j = lane % 8, i.e. m = j >> 1, h = j & 1, t = i  ->  position i*8 + j
+    if ((int64_t)blockIdx.x >= B * groups) return;           // (blocks beyond the transform work only clear)
+    const int64_t b = blockIdx.x / groups, gi = blockIdx.x % groups;
+    const int64_t k0 = gi * kGroup + q * 256 + lane * 8;     // this lane's 8 consecutive inputs
+    float v[8];
+    {
+        const T* src = x + b * K + k0;
+        if (sizeof(T) == 2) {
+            const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(src));
+            const uint32_t w4[4] = {q4.x, q4.y, q4.z, q4.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                v[2 * e] = __uint_as_float(w4[e] << 16);
+                v[2 * e + 1] = __uint_as_float(w4[e] & 0xffff0000u);
+            }
+        } else {
+            const float4 a = __ldg(reinterpret_cast<const float4*>(src)), c = __ldg(reinterpret_cast<const float4*>(src) + 1);
+            v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = c.x; v[5] = c.y; v[6] = c.z; v[7] = c.w;
+        }
+        const uint32_t bits = (uint32_t)(sign_word(xi, (uint64_t)k0 >> 6) >> ((uint64_t)k0 & 63ull)) & 0xffu;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(__float_as_uint(v[e]) ^ (((bits >> e) & 1u) << 31));
+    }
+#pragma unroll
+    for (int h = 1; h < 8; h <<= 1) {
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            if ((r & h) == 0) { const float a = v[r], c = v[r | h]; v[r] = a + c; v[r | h] = a - c; }
+        }
+    }
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+        const bool upper = (lane & m) != 0;
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            const float o = __shfl_xor_sync(0xffffffffu, v[r], m);
+            v[r] = upper ? (o - v[r]) : (v[r] + o);
+        }
+    }
+    *reinterpret_cast<float4*>(&ex[q][lane * 8]) = make_float4(v[0], v[1], v[2], v[3]);
+    *reinterpret_cast<float4*>(&ex[q][lane * 8 + 4]) = make_float4(v[4], v[5], v[6], v[7]);
+    __syncthreads();
+    float o[8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r) o[r] = 0.f;
+#pragma unroll
+    for (int qq = 0; qq < 4; ++qq) {
+        const float4 u0 = *reinterpret_cast<const float4*>(&ex[qq][lane * 8]);
+        const float4 u1 = *reinterpret_cast<const float4*>(&ex[qq][lane * 8 + 4]);
+        const float sgn = (__popc(q & qq) & 1) ? -1.f : 1.f;
+        o[0] = fmaf(sgn, u0.x, o[0]); o[1] = fmaf(sgn, u0.y, o[1]); o[2] = fmaf(sgn, u0.z, o[2]); o[3] = fmaf(sgn, u0.w, o[3]);
+        o[4] = fmaf(sgn, u1.x, o[4]); o[5] = fmaf(sgn, u1.y, o[5]); o[6] = fmaf(sgn, u1.z, o[6]); o[7] = fmaf(sgn, u1.w, o[7]);
+    }
+    // this lane holds pairs 4 j + i (i = 0..3, j = lane % 8) of 64-input block q*4 + lane/8 of the group, i.e.
+    // m = j >> 1, h = j & 1, t = i  ->  position i*8 + j
+    uint32_t* blk = reinterpret_cast<uint32_t*>(xdag + b * K + gi * kGroup) + (q * 4 + (lane >> 3)) * 32;
     const int j = lane & 7;
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        uint32_t* blk = dst + (c * 4 + (lane >> 3)) * 32;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            __half2 h = __floats2half2_rn(v[c * 8 + 2 * e] * 0.03125f, v[c * 8 + 2 * e + 1] * 0.03125f);
-            blk[e * 8 + j] = *reinterpret_cast<uint32_t*>(&h);
-        }
+    for (int e = 0; e < 4; ++e) {
+        const __half2 hh = __floats2half2_rn(o[2 * e] * 0.03125f, o[2 * e + 1] * 0.03125f);
+        blk[e * 8 + j] = *reinterpret_cast<const uint32_t*>(&hh);
     }
 }
 
@@ -101,14 +146,13 @@ __global__ void __launch_bounds__(256) rht_debug_kernel(const T* __restrict__ x,
 
 int launch_rht_activations(const higgs_desc& d, const void* x, int64_t B, __half* xdag, float* zero_ptr,
                            size_t zero_floats, cudaStream_t st) {
-    const int64_t warps = B * (d.K / kGroup);
-    int64_t blocks = (warps + 7) / 8;
+    int64_t blocks = B * (d.K / kGroup);                   // one block of four warps per (token, group)
     if (zero_floats) {
-        int64_t zb = (int64_t)((zero_floats + 256 * 8 - 1) / (256 * 8));
+        int64_t zb = (int64_t)((zero_floats + 128 * 8 - 1) / (128 * 8));
         if (zb > 1184) zb = 1184;
         if (zb > blocks) blocks = zb;
     }
-    return cuda_status(launch_pdl(rht_activations_kernel<__nv_bfloat16>, dim3((unsigned)blocks), dim3(256), 0, st,
+    return cuda_status(launch_pdl(rht_activations_kernel<__nv_bfloat16>, dim3((unsigned)blocks), dim3(128), 0, st,
                                   static_cast<const __nv_bfloat16*>(x), xdag, B, d.K, d.rht_seed, zero_ptr, zero_floats));
 }
 
