@@ -145,27 +145,37 @@ __global__ void __launch_bounds__(256) build_cells_kernel(const float* __restric
     uint8_t* cand = table;                       // [NC][kMaxCand]
     uint8_t* cnt = table + NC * kMaxCand;        // [NC]
     const float w = 2.0f * kCellR / (P == 2 ? kCells2 : kCells1);
-    for (int cell = blockIdx.x * blockDim.x + threadIdx.x; cell < NC; cell += gridDim.x * blockDim.x) {
+    const int lane = threadIdx.x & 31;
+    const int warps = (gridDim.x * blockDim.x) >> 5;
+    // one warp per cell; lane l looks at grid points l, l + 32, ... (rounds keep the candidate list in index order)
+    for (int cell = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; cell < NC; cell += warps) {
         const float x0 = -kCellR + w * (P == 2 ? (cell % kCells2) : cell), x1 = x0 + w;
         const float y0 = P == 2 ? -kCellR + w * (cell / kCells2) : 0.f, y1 = y0 + w;
         float U = INFINITY;
-        for (int c = 0; c < n; ++c) {
+        for (int c = lane; c < n; c += 32) {
             const float gx = sgrid[P * c], gy = P == 2 ? sgrid[2 * c + 1] : 0.f;
             const float fx = fmaxf(fabsf(gx - x0), fabsf(gx - x1));
             const float fy = P == 2 ? fmaxf(fabsf(gy - y0), fabsf(gy - y1)) : 0.f;
             U = fminf(U, sqrtf(fx * fx + fy * fy));
         }
+#pragma unroll
+        for (int m = 16; m >= 1; m >>= 1) U = fminf(U, __shfl_xor_sync(0xffffffffu, U, m));
         int k = 0;
-        for (int c = 0; c < n; ++c) {
-            const float gx = sgrid[P * c], gy = P == 2 ? sgrid[2 * c + 1] : 0.f;
-            const float nx = fmaxf(fmaxf(x0 - gx, gx - x1), 0.f);
-            const float ny = P == 2 ? fmaxf(fmaxf(y0 - gy, gy - y1), 0.f) : 0.f;
-            if (sqrtf(nx * nx + ny * ny) <= U + kCandSlack) {
-                if (k < kMaxCand) cand[cell * kMaxCand + k] = (uint8_t)c;
-                ++k;
+        for (int c0 = 0; c0 < n; c0 += 32) {
+            const int c = c0 + lane;
+            bool in = false;
+            if (c < n) {
+                const float gx = sgrid[P * c], gy = P == 2 ? sgrid[2 * c + 1] : 0.f;
+                const float nx = fmaxf(fmaxf(x0 - gx, gx - x1), 0.f);
+                const float ny = P == 2 ? fmaxf(fmaxf(y0 - gy, gy - y1), 0.f) : 0.f;
+                in = sqrtf(nx * nx + ny * ny) <= U + kCandSlack;
             }
+            const unsigned m = __ballot_sync(0xffffffffu, in);
+            const int pos = k + __popc(m & ((1u << lane) - 1u));
+            if (in && pos < kMaxCand) cand[cell * kMaxCand + pos] = (uint8_t)c;
+            k += __popc(m);
         }
-        cnt[cell] = k <= kMaxCand ? (uint8_t)k : (uint8_t)255;
+        if (lane == 0) cnt[cell] = k <= kMaxCand ? (uint8_t)k : (uint8_t)255;
     }
 }
 
@@ -428,8 +438,8 @@ int launch_encode(const higgs_desc& d, const void* W, int w_dtype, const float* 
     const unsigned pblocks = 592;          // 4 blocks of 8 warps per SM on a 148-SM part; any count is correct
     uint8_t* table = static_cast<uint8_t*>(scratch);
     if (pruned) {
-        if (d.p == 2) build_cells_kernel<2><<<4, 256, 0, st>>>(grid, d.n, table);
-        else build_cells_kernel<1><<<4, 256, 0, st>>>(grid, d.n, table);
+        if (d.p == 2) build_cells_kernel<2><<<128, 256, 0, st>>>(grid, d.n, table);      // one warp per cell
+        else build_cells_kernel<1><<<128, 256, 0, st>>>(grid, d.n, table);
     }
 #define HIGGS_ENC(T, P) \
     if (pruned) encode_pruned_kernel<T, P><<<pblocks, 256, 0, st>>>(static_cast<const T*>(W), grid, d.n, table, canonical, sc, d.N, d.K, d.rht_seed); \
