@@ -797,6 +797,8 @@ int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const 
     if (d.N == 0) return HIGGS_OK;
     const Plan pl = make_plan(d, B);
     if (pl.items == 0) return HIGGS_ERR_UNSUPPORTED;
+    // the kernel's work split is 32-bit arithmetic: (row tiles) x (blocks per K-chunk) must stay below 2^31
+    if ((d.N / kRowTile) * (int64_t)(pl.parts + 1) >= ((int64_t)1 << 31)) return HIGGS_ERR_UNSUPPORTED;
     const bool fused = x_raw != nullptr;
     if (fused && !linear_fused_eligible(d, B)) return HIGGS_ERR_INVALID_ARG;
     StreamParams prm;

@@ -504,10 +504,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
             if (ksplit == 1) {
                 // epilogue: accumulator row i, 32 token columns at a time, the column chunks dealt over the warp groups
                 pdl_wait();        // y may still be read by the kernel before this one
+                if (warp == 3) TTRACE(3, 4);
                 for (int c0 = 32 * sg; c0 < BN; c0 += 32 * kTcGroups) {
                     uint32_t d[32];
                     tc_ld32(t_lane + (uint32_t)c0, d);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (warp == 3 && c0 == 0) TTRACE(3, 5);
 #pragma unroll
                     for (int r = 0; r < 32; ++r) {
                         const int b = bt * BN + c0 + r;
@@ -517,6 +519,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
                             else static_cast<__nv_bfloat16*>(prm.y)[(int64_t)b * prm.N + row] = __float2bfloat16_rn(v);
                         }
                     }
+                    if (warp == 3 && c0 == 0) TTRACE(3, 6);
                 }
             } else {
                 // K-split: park the partial tile in shared memory as [token][row] (all rings are idle: every MMA
