@@ -131,6 +131,8 @@ int higgs_make_uniform_grid(int n, float* grid_out, float* step_out, float* mse_
  *                max_iters was reached without convergence
  * Distances are fp32, sums fp64; the result is a fixed point of the same
  * iteration the fp64 definition runs but need not be bit-identical to it.
+ * 1 <= p <= 4 and 1 <= n <= 4096 (n need not be a power of two), else
+ * HIGGS_ERR_UNSUPPORTED.
  */
 int higgs_make_grid(int p, int n, const float* samples, int64_t num_samples, int max_iters,
                     float* grid_out, float* mse_out, int32_t* iters_out,
@@ -286,6 +288,23 @@ int higgs_dequantize(const higgs_desc* desc, const void* packed, const void* sca
  * W: device [N][K], w_dtype in {HIGGS_F32, HIGGS_BF16}; workspace as for higgs_dequantize.  Asynchronous.    */
 int higgs_layer_error(const higgs_desc* desc, const void* W, int w_dtype, const void* packed, const void* scales,
                       const float* grid, double* sums_out, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Algorithm 1 for ANY grid (1 <= p <= 4, 1 <= n <= 4096, n need not be a power of two): the encoder for the grids
+ * the paper evaluates beside the kernel-supported ones, e.g. (p, n) = (3, 830), (2, 88), (2, 361), (1, 19)
+ * ("Experiment Configurations"), and the error-database entry of such a grid in the same pass.  No product
+ * kernel reads this output.
+ *   W          : device [N][K] row-major, w_dtype in {HIGGS_F32, HIGGS_BF16}; K a multiple of 1024 (the group size)
+ *   grid       : device [n][p] fp32
+ *   codes_out  : device [N][K/1024][T] uint16, T = higgs_general_tuples(p) = ceil(1024 / p); code t of a group covers
+ *                rotated coordinates [t p, (t+1) p).  When p does not divide 1024 the last tuple is completed with
+ *                zeros and matched on all p coordinates; its completed coordinates are dropped on reconstruction.
+ *   scales_out : device [N][K/1024] fp16, ROW-major (not the product kernels' tile-major order): ||w|| / sqrt(1024)
+ *   sums_out   : device, two doubles, optional: || W^ - W ||_F^2 (with the fp16 scale) and || W ||_F^2, so that
+ *                t^2 = sums_out[0] / sums_out[1]; cleared by the call.
+ * HIGGS_ERR_UNSUPPORTED for p, n or K outside the above; HIGGS_ERR_INVALID_ARG for null pointers.  Asynchronous.  */
+int higgs_general_tuples(int p);
+int higgs_quantize_general(int p, int n, int64_t N, int64_t K, uint64_t rht_seed, const void* W, int w_dtype,
+                           const float* grid, uint16_t* codes_out, void* scales_out, double* sums_out, void* stream);
 
 /* Eq. 4: choose option j_l in [0, num_options) for every layer l, minimising  sum_l alpha[l] * t2[l][j_l]  subject
  * to  sum_l bits(j_l) * sizes[l] <= budget * sum_l sizes[l].  Exact (dynamic programming over the integer budget;

@@ -171,10 +171,17 @@ def grid_mse(grid, pts) -> float:
     return float(_load().higgs_oracle_grid_mse(p, n, _pd(g), _pd(x), x.shape[0]))
 
 
+def tuples_per_group(g: int, p: int) -> int:
+    """Number of p-tuples a group of g rotated values is cut into.  When p does not divide g (the paper's p = 3 grids
+    with g = 1024; it does not say how) the last tuple is completed with zeros, matched on all p coordinates, and its
+    completed coordinates are dropped on reconstruction."""
+    return (g + p - 1) // p
+
+
 class Quantized(NamedTuple):
-    codes: np.ndarray  # int32 [N][K/p], 0-based
-    runner: np.ndarray  # int32 [N][K/p], second-nearest point
-    margin: np.ndarray  # float64 [N][K/p], distance to the winner/runner-up bisector
+    codes: np.ndarray  # int32 [N][(K/g) * tuples_per_group] (= [N][K/p] when p divides g), 0-based
+    runner: np.ndarray  # int32, same shape, second-nearest point
+    margin: np.ndarray  # float64, same shape, distance to the winner/runner-up bisector
     scales: np.ndarray  # float64 [N][K/g] = ||w||/sqrt(g), unrounded
 
 
@@ -184,9 +191,10 @@ def quantize(W, g: int, grid, xi: int) -> Quantized:
     N, K = W.shape
     gr = _d(grid)
     n, p = gr.shape
-    codes = np.zeros((N, K // p), dtype=np.int32)
-    runner = np.zeros((N, K // p), dtype=np.int32)
-    margin = np.zeros((N, K // p), dtype=np.float64)
+    cols = (K // g) * tuples_per_group(g, p)
+    codes = np.zeros((N, cols), dtype=np.int32)
+    runner = np.zeros((N, cols), dtype=np.int32)
+    margin = np.zeros((N, cols), dtype=np.float64)
     scales = np.zeros((N, K // g), dtype=np.float64)
     rc = _load().higgs_oracle_quantize(_pd(W), N, K, g, p, n, _pd(gr), ctypes.c_uint64(xi & (2**64 - 1)), _pi(codes), _pi(runner), _pd(margin), _pd(scales))
     if rc != 0:
@@ -205,9 +213,9 @@ def dequantize(codes, scales, g: int, grid, xi: int) -> np.ndarray:
     gr = _d(grid)
     n, p = gr.shape
     N = codes.shape[0]
-    K = codes.shape[1] * p
+    K = codes.shape[1] // tuples_per_group(g, p) * g
     sc = _d(scales)
-    assert sc.shape == (N, K // g)
+    assert sc.shape == (N, K // g) and codes.shape[1] == (K // g) * tuples_per_group(g, p)
     out = np.zeros((N, K), dtype=np.float64)
     rc = _load().higgs_oracle_dequantize(_pi(codes), _pd(sc), N, K, g, p, n, _pd(gr), ctypes.c_uint64(xi & (2**64 - 1)), _pd(out))
     if rc != 0:

@@ -267,24 +267,28 @@ double higgs_oracle_grid_mse(int p, int n, const double* grid, const double* pts
 /* output row and g consecutive inputs).  Per (row, group):                   */
 /*   s  = ||w||_2                                                             */
 /*   w+ = H diag(sign(xi, .)) (w / s)        (H unnormalised: entries ~N(0,1)) */
-/*   code_t = argmin_c || w+[tp:(t+1)p] - G[c] ||^2,  t = 0..g/p-1             */
+/*   code_t = argmin_c || w+[tp:(t+1)p] - G[c] ||^2,  t = 0..ceil(g/p)-1       */
 /*   stored scale = s / sqrt(g)                                               */
+/* When p does not divide g (the paper's p = 3 grids with g = 1024; it does    */
+/* not say how) the last tuple is completed with zeros and matched on all p   */
+/* coordinates; reconstruction drops the completed coordinates.               */
 /* A group of all zeros gets scale 0 and the code of the point nearest the    */
 /* origin (the paper divides by zero there; this reading keeps it finite).    */
-/* Outputs: codes/runner[N][K/p] (int32), margin[N][K/p], scales[N][K/g]      */
+/* Outputs: codes/runner/margin [N][K/g][ceil(g/p)] (= [N][K/p] when p        */
+/* divides g; int32 / double), scales[N][K/g]                                 */
 /* (double, NOT yet rounded to the 16-bit storage type; the caller rounds).   */
 int higgs_oracle_quantize(const double* W, int64_t N, int64_t K, int g, int p, int n,
                           const double* grid, uint64_t xi,
                           int32_t* codes, int32_t* runner, double* margin, double* scales) {
-    if (g < 1 || (g & (g - 1)) || K % g || g % p) return -1;
-    int64_t groups = K / g, tup = g / p;
+    if (g < 1 || (g & (g - 1)) || K % g || p < 1 || p > 16) return -1;
+    int64_t groups = K / g, tup = (g + p - 1) / p;
     double* signs = (double*)malloc((size_t)K * sizeof(double));
     if (!signs) return -1;
     for (int64_t j = 0; j < K; ++j) signs[j] = higgs_oracle_sign(xi, j);
     int fail = 0;
 #pragma omp parallel for schedule(dynamic, 1)
     for (int64_t r = 0; r < N; ++r) {
-        double* v = (double*)malloc((size_t)g * sizeof(double));
+        double* v = (double*)calloc((size_t)g + 16, sizeof(double));   /* zeros behind the group complete a short tuple */
         if (!v) { fail = 1; continue; }
         for (int64_t i = 0; i < groups; ++i) {
             const double* w = W + r * K + i * g;
@@ -297,7 +301,7 @@ int higgs_oracle_quantize(const double* W, int64_t N, int64_t K, int g, int p, i
                 int c1, c2;
                 double mg;
                 nearest_point(v + t * p, p, n, grid, &c1, &c2, &mg);
-                int64_t o = r * (K / p) + i * tup + t;
+                int64_t o = (r * groups + i) * tup + t;
                 codes[o] = c1;
                 if (runner) runner[o] = c2;
                 if (margin) margin[o] = mg;
@@ -317,9 +321,9 @@ int higgs_oracle_quantize(const double* W, int64_t N, int64_t K, int g, int p, i
 /* scales[N][K/g] are the stored (already rounded) scales, widened to double.  */
 int higgs_oracle_dequantize(const int32_t* codes, const double* scales, int64_t N, int64_t K,
                             int g, int p, int n, const double* grid, uint64_t xi, double* What) {
-    if (g < 1 || (g & (g - 1)) || K % g || g % p) return -1;
+    if (g < 1 || (g & (g - 1)) || K % g || p < 1 || p > 16) return -1;
     (void)n;
-    int64_t groups = K / g, tup = g / p;
+    int64_t groups = K / g, tup = (g + p - 1) / p;
     double* ones = (double*)malloc((size_t)g * sizeof(double));
     if (!ones) return -1;
     for (int j = 0; j < g; ++j) ones[j] = 1.0;
@@ -329,8 +333,8 @@ int higgs_oracle_dequantize(const int32_t* codes, const double* scales, int64_t 
             double* v = What + r * K + i * g;
             double sc = scales[r * groups + i];
             for (int64_t t = 0; t < tup; ++t) {
-                int c = codes[r * (K / p) + i * tup + t];
-                for (int k = 0; k < p; ++k) v[t * p + k] = sc * grid[(int64_t)c * p + k];
+                int c = codes[(r * groups + i) * tup + t];
+                for (int k = 0; k < p && t * p + k < g; ++k) v[t * p + k] = sc * grid[(int64_t)c * p + k];
             }
             higgs_oracle_rht(v, g, ones, 1);                 /* Hn r            */
             for (int j = 0; j < g; ++j) v[j] *= higgs_oracle_sign(xi, i * g + j); /* diag(sign) */

@@ -26,7 +26,7 @@ EXPORTS = [
     "higgs_linear_host", "higgs_linear_host_workspace_bytes", "higgs_linear_launch_count", "higgs_device_status",
     "higgs_linear_static", "higgs_linear_static_capacity", "higgs_linear_k_splits", "higgs_rotated_bytes",
     "higgs_rotated_layout", "higgs_dequantize", "higgs_make_uniform_grid", "higgs_layer_error",
-    "higgs_allocate_bits",
+    "higgs_allocate_bits", "higgs_general_tuples", "higgs_quantize_general",
 ]
 
 
@@ -99,6 +99,10 @@ def _load() -> ctypes.CDLL:
     lib.higgs_layer_error.argtypes = [P, vp, i32, vp, vp, vp, vp, vp, sz, vp]
     lib.higgs_allocate_bits.restype = i32
     lib.higgs_allocate_bits.argtypes = [i32, i32, vp, vp, vp, vp, i64, vp, vp]
+    lib.higgs_general_tuples.restype = i32
+    lib.higgs_general_tuples.argtypes = [i32]
+    lib.higgs_quantize_general.restype = i32
+    lib.higgs_quantize_general.argtypes = [i32, i32, i64, i64, u64, vp, i32, vp, vp, vp, vp, vp]
     lib.higgs_dequantize.restype = i32
     lib.higgs_dequantize.argtypes = [P, vp, vp, vp, vp, i32, vp, sz, vp]
     return lib
@@ -331,6 +335,25 @@ def higgs_layer_error(desc: higgs_desc, W: torch.Tensor, packed: torch.Tensor, s
                                  _ptr(ws), ws.numel(), _stream()), "higgs_layer_error")
     s = sums.cpu()
     return float(s[0] / s[1]) if float(s[1]) > 0 else 0.0
+
+
+def higgs_quantize_general(p: int, n: int, W: torch.Tensor, grid: torch.Tensor, rht_seed: int, want_error: bool = True):
+    """Algorithm 1 for any grid (p <= 4, n <= 4096).  Returns (codes int16-as-uint16 [N][K/1024][ceil(1024/p)],
+    scales fp16 [N][K/1024] row-major, t^2 or None)."""
+    assert W.is_cuda and W.is_contiguous() and W.dtype in (torch.float32, torch.bfloat16)
+    assert grid.is_cuda and grid.dtype == torch.float32 and grid.is_contiguous() and tuple(grid.shape) == (n, p)
+    N, K = W.shape
+    tuples = lib.higgs_general_tuples(p)
+    codes = torch.empty((N, K // 1024, max(tuples, 1)), dtype=torch.uint16, device=W.device)
+    scales = torch.empty((N, K // 1024), dtype=torch.float16, device=W.device)
+    sums = torch.zeros(2, dtype=torch.float64, device=W.device) if want_error else None
+    _check(lib.higgs_quantize_general(p, n, N, K, rht_seed, _ptr(W), _dtype_code(W), _ptr(grid), _ptr(codes), _ptr(scales),
+                                      _ptr(sums), _stream()), "higgs_quantize_general")
+    t2 = None
+    if want_error:
+        s = sums.cpu()
+        t2 = float(s[0] / s[1]) if float(s[1]) > 0 else 0.0
+    return codes, scales, t2
 
 
 def higgs_allocate_bits(alpha, t2, bits64, sizes, budget64: int):

@@ -57,7 +57,7 @@ size_t higgs_canonical_bytes(const higgs_desc* d) {
 size_t higgs_workspace_bytes(const higgs_desc* d, int op, int64_t B) {
     if (!d) return 0;
     if (op == HIGGS_OP_MAKE_GRID) {
-        if (!((d->p == 1 || d->p == 2) && d->n >= 1 && d->n <= 256 && d->K >= d->n)) return 0;
+        if (!(d->p >= 1 && d->p <= kMaxGridDim && d->n >= 1 && d->n <= kMaxGridPoints && d->K >= d->n)) return 0;
         return make_grid_workspace(d->p, d->n, d->K);
     }
     if (check_desc(d) != HIGGS_OK) return 0;
@@ -74,12 +74,28 @@ size_t higgs_workspace_bytes(const higgs_desc* d, int op, int64_t B) {
 int higgs_make_grid(int p, int n, const float* samples, int64_t num_samples, int max_iters, float* grid_out,
                     float* mse_out, int32_t* iters_out, void* workspace, size_t workspace_bytes, void* stream) {
     if (!samples || !grid_out || !workspace || max_iters < 1) return HIGGS_ERR_INVALID_ARG;
-    if (!(p == 1 || p == 2) || n < 1 || n > 256) return HIGGS_ERR_UNSUPPORTED;
+    if (p < 1 || p > kMaxGridDim || n < 1 || n > kMaxGridPoints) return HIGGS_ERR_UNSUPPORTED;
     if (num_samples < n || num_samples > ((int64_t)1 << 31) - 1) return HIGGS_ERR_INVALID_ARG;
     if (!aligned(workspace, 256)) return HIGGS_ERR_INVALID_ARG;
     if (workspace_bytes < make_grid_workspace(p, n, num_samples)) return HIGGS_ERR_WORKSPACE;
     return launch_make_grid(p, n, samples, num_samples, max_iters, grid_out, mse_out, iters_out, workspace,
                             as_stream(stream));
+}
+
+int higgs_general_tuples(int p) { return p >= 1 && p <= kMaxGridDim ? (kGroup + p - 1) / p : 0; }
+
+int higgs_quantize_general(int p, int n, int64_t N, int64_t K, uint64_t rht_seed, const void* W, int w_dtype,
+                           const float* grid, uint16_t* codes_out, void* scales_out, double* sums_out, void* stream) {
+    if (p < 1 || p > kMaxGridDim || n < 1 || n > kMaxGridPoints) return HIGGS_ERR_UNSUPPORTED;
+    if (w_dtype != HIGGS_F32 && w_dtype != HIGGS_BF16) return HIGGS_ERR_UNSUPPORTED;
+    if (N < 0 || K < 0) return HIGGS_ERR_INVALID_ARG;
+    if (K % kGroup) return HIGGS_ERR_UNSUPPORTED;
+    if (N == 0 || K == 0) return HIGGS_OK;
+    if (!W || !grid || !codes_out || !scales_out) return HIGGS_ERR_INVALID_ARG;
+    if (!aligned(W, 16) || !aligned(codes_out, 2) || !aligned(scales_out, 2) || (sums_out && !aligned(sums_out, 8)))
+        return HIGGS_ERR_INVALID_ARG;
+    return launch_encode_general(p, n, N, K, rht_seed, W, w_dtype, grid, codes_out, scales_out, sums_out,
+                                 as_stream(stream));
 }
 
 int higgs_make_uniform_grid(int n, float* grid_out, float* step_out, float* mse_out, void* stream) {

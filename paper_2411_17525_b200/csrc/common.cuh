@@ -13,6 +13,8 @@ namespace higgs {
 constexpr int kGroup = 1024;     // the only supported group size g
 constexpr int kRowTile = 16;     // rows of W per mma tile (m16n8k16) and per scale tile
 constexpr int kBlockK = 64;      // k-extent of one 512-byte packed block
+constexpr int kMaxGridDim = 4;        // grid fit and general encoder: 1 <= p <= 4
+constexpr int kMaxGridPoints = 4096;  //                               n <= 4096 (64 KB of fp32 at p = 4)
 
 // Output number m of the splitmix64 stream seeded with xi: 64 sign bits, for inputs 64 m .. 64 m + 63.
 __host__ __device__ __forceinline__ uint64_t sign_word(uint64_t xi, uint64_t m) {
@@ -154,6 +156,8 @@ int launch_layer_error(const higgs_desc& d, const uint8_t* canonical, const void
                        int w_dtype, double* sums, cudaStream_t st);
 int allocate_bits(int L, int J, const double* alpha, const double* t2, const int32_t* bits64, const int64_t* sizes,
                   int64_t budget64, int32_t* choice_out, double* objective_out);
+int launch_encode_general(int p, int n, int64_t N, int64_t K, uint64_t xi, const void* W, int w_dtype, const float* grid,
+                          uint16_t* codes, void* scales, double* sums, cudaStream_t st);
 int launch_uniform_grid(int n, float* grid_out, float* step_out, float* mse_out, cudaStream_t st);
 int linear_k_chunks(const higgs_desc& d, int64_t B);
 // tensor-core path (B > 16)

@@ -40,48 +40,65 @@ __global__ void grid_init_kernel(GridWs w, const float* __restrict__ samples, in
     if (i < 3) w.flags[i] = 0;
 }
 
-template <int P>
+// Assignment step.  The centres sit in dynamic shared memory ([n][P] floats, at most 64 KB).  SMALL (n <= 256): the
+// per-cell sums are first collected in shared memory and then added to the global ones; otherwise every sample adds
+// to the global sums directly (with thousands of cells the atomics rarely collide).  Distances are the plain
+// sum of (x_k - c_k)^2 in coordinate order, fp32, strict '<' (lowest index wins a tie) - the encoder's rule.
+template <int P, bool SMALL>
 __global__ void __launch_bounds__(256) grid_assign_kernel(GridWs w, const float* __restrict__ samples, int n, int64_t m) {
-    __shared__ float sc[256 * 2];
-    __shared__ double ssum[256 * 2];
-    __shared__ unsigned int scnt[256];
+    extern __shared__ __align__(16) unsigned char grid_smem[];
+    float* sc = reinterpret_cast<float*>(grid_smem);
+    double* ssum = reinterpret_cast<double*>(grid_smem + up256(sizeof(float) * n * P));
+    unsigned int* scnt = reinterpret_cast<unsigned int*>(ssum + (SMALL ? n * P : 0));
     __shared__ double serr;
     __shared__ int schanged;
     if (w.flags[1]) return;
-    for (int i = threadIdx.x; i < n * P; i += blockDim.x) { sc[i] = w.centres[i]; ssum[i] = 0.0; }
-    for (int i = threadIdx.x; i < n; i += blockDim.x) scnt[i] = 0u;
+    for (int i = threadIdx.x; i < n * P; i += blockDim.x) {
+        sc[i] = w.centres[i];
+        if (SMALL) ssum[i] = 0.0;
+    }
+    if (SMALL)
+        for (int i = threadIdx.x; i < n; i += blockDim.x) scnt[i] = 0u;
     if (threadIdx.x == 0) { serr = 0.0; schanged = 0; }
     __syncthreads();
     double err = 0.0;
     int changed = 0;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < m; i += (int64_t)gridDim.x * blockDim.x) {
-        float x0 = samples[i * P], x1 = P == 2 ? samples[i * P + 1] : 0.f;
+        float x[P];
+#pragma unroll
+        for (int k = 0; k < P; ++k) x[k] = samples[i * P + k];
         float best = INFINITY;
         int bi = 0;
         for (int c = 0; c < n; ++c) {
-            float d;
-            if (P == 2) {
-                const float dx = x0 - sc[2 * c], dy = x1 - sc[2 * c + 1];
-                d = fmaf(dy, dy, dx * dx);
-            } else {
-                const float dx = x0 - sc[c];
-                d = dx * dx;
+            float d = 0.f;
+#pragma unroll
+            for (int k = 0; k < P; ++k) {
+                const float e = x[k] - sc[c * P + k];
+                d = k == 0 ? e * e : fmaf(e, e, d);
             }
             if (d < best) { best = d; bi = c; }
         }
         if (w.assign[i] != bi) { w.assign[i] = bi; ++changed; }
         err += (double)best;
-        atomicAdd(&ssum[bi * P], (double)x0);
-        if (P == 2) atomicAdd(&ssum[bi * P + 1], (double)x1);
-        atomicAdd(&scnt[bi], 1u);
+        if (SMALL) {
+#pragma unroll
+            for (int k = 0; k < P; ++k) atomicAdd(&ssum[bi * P + k], (double)x[k]);
+            atomicAdd(&scnt[bi], 1u);
+        } else {
+#pragma unroll
+            for (int k = 0; k < P; ++k) atomicAdd(&w.sums[bi * P + k], (double)x[k]);
+            atomicAdd(&w.counts[bi], 1ull);
+        }
     }
     atomicAdd(&serr, err);
     if (changed) atomicAdd(&schanged, changed);
     __syncthreads();
-    for (int i = threadIdx.x; i < n * P; i += blockDim.x)
-        if (ssum[i] != 0.0) atomicAdd(&w.sums[i], ssum[i]);
-    for (int i = threadIdx.x; i < n; i += blockDim.x)
-        if (scnt[i]) atomicAdd(&w.counts[i], (unsigned long long)scnt[i]);
+    if (SMALL) {
+        for (int i = threadIdx.x; i < n * P; i += blockDim.x)
+            if (ssum[i] != 0.0) atomicAdd(&w.sums[i], ssum[i]);
+        for (int i = threadIdx.x; i < n; i += blockDim.x)
+            if (scnt[i]) atomicAdd(&w.counts[i], (unsigned long long)scnt[i]);
+    }
     if (threadIdx.x == 0) {
         atomicAdd(&w.err[0], serr);
         if (schanged) atomicAdd(&w.flags[0], schanged);
@@ -110,16 +127,18 @@ __global__ void grid_update_kernel(GridWs w, int p, int n) {
 
 __global__ void grid_finalize_kernel(GridWs w, int p, int n, int64_t m, float* __restrict__ grid_out,
                                      float* __restrict__ mse_out, int32_t* __restrict__ iters_out) {
+    // lexicographic sort by rank counting (coordinate 0 first; equal points keep their index order)
     for (int c = threadIdx.x; c < n; c += blockDim.x) {
-        const float a0 = w.centres[c * p], a1 = p == 2 ? w.centres[c * p + 1] : 0.f;
         int rank = 0;
         for (int o = 0; o < n; ++o) {
-            const float b0 = w.centres[o * p], b1 = p == 2 ? w.centres[o * p + 1] : 0.f;
-            const bool less = (b0 < a0) || (b0 == a0 && (b1 < a1 || (b1 == a1 && o < c)));
-            rank += less ? 1 : 0;
+            int cmp = 0;                                   // sign of (centre o) - (centre c)
+            for (int k = 0; k < p && cmp == 0; ++k) {
+                const float a = w.centres[c * p + k], b = w.centres[o * p + k];
+                cmp = b < a ? -1 : (b > a ? 1 : 0);
+            }
+            rank += (cmp < 0 || (cmp == 0 && o < c)) ? 1 : 0;
         }
-        grid_out[rank * p] = a0;
-        if (p == 2) grid_out[rank * p + 1] = a1;
+        for (int k = 0; k < p; ++k) grid_out[rank * p + k] = w.centres[c * p + k];
     }
     if (threadIdx.x == 0) {
         if (mse_out) *mse_out = (float)(w.err[1] / ((double)m * p));
@@ -196,6 +215,20 @@ size_t make_grid_workspace(int p, int n, int64_t m) {
            up256(sizeof(int32_t) * (size_t)m);
 }
 
+template <int P, bool SMALL>
+static int assign_step(GridWs w, const float* samples, int n, int64_t m, unsigned blocks, cudaStream_t st) {
+    const size_t smem = up256(sizeof(float) * n * P) + (SMALL ? sizeof(double) * n * P + sizeof(unsigned int) * n : 0);
+    static bool opted = false;                             // per instantiation
+    if (!opted && smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(grid_assign_kernel<P, SMALL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)(up256(sizeof(float) * kMaxGridPoints * P)));
+        if (e != cudaSuccess) return cuda_status(e);
+        opted = true;
+    }
+    grid_assign_kernel<P, SMALL><<<blocks, 256, smem, st>>>(w, samples, n, m);
+    return HIGGS_OK;
+}
+
 int launch_make_grid(int p, int n, const float* samples, int64_t m, int max_iters, float* grid_out, float* mse_out,
                      int32_t* iters_out, void* ws, cudaStream_t st) {
     GridWs w = carve(ws, p, n, m);
@@ -203,9 +236,21 @@ int launch_make_grid(int p, int n, const float* samples, int64_t m, int max_iter
     grid_init_kernel<<<(unsigned)((init_threads + 255) / 256), 256, 0, st>>>(w, samples, p, n, m);
     int64_t blocks = (m + 255) / 256;
     if (blocks > 592) blocks = 592;
+    const bool small = n <= 256;
     for (int it = 0; it < max_iters; ++it) {
-        if (p == 2) grid_assign_kernel<2><<<(unsigned)blocks, 256, 0, st>>>(w, samples, n, m);
-        else grid_assign_kernel<1><<<(unsigned)blocks, 256, 0, st>>>(w, samples, n, m);
+        int rc;
+        switch (p * 2 + (small ? 1 : 0)) {
+            case 3: rc = assign_step<1, true>(w, samples, n, m, (unsigned)blocks, st); break;
+            case 2: rc = assign_step<1, false>(w, samples, n, m, (unsigned)blocks, st); break;
+            case 5: rc = assign_step<2, true>(w, samples, n, m, (unsigned)blocks, st); break;
+            case 4: rc = assign_step<2, false>(w, samples, n, m, (unsigned)blocks, st); break;
+            case 7: rc = assign_step<3, true>(w, samples, n, m, (unsigned)blocks, st); break;
+            case 6: rc = assign_step<3, false>(w, samples, n, m, (unsigned)blocks, st); break;
+            case 9: rc = assign_step<4, true>(w, samples, n, m, (unsigned)blocks, st); break;
+            case 8: rc = assign_step<4, false>(w, samples, n, m, (unsigned)blocks, st); break;
+            default: return HIGGS_ERR_UNSUPPORTED;
+        }
+        if (rc != HIGGS_OK) return rc;
         grid_update_kernel<<<1, 256, 0, st>>>(w, p, n);
     }
     grid_finalize_kernel<<<1, 256, 0, st>>>(w, p, n, m, grid_out, mse_out, iters_out);

@@ -86,7 +86,14 @@ def test_invalid_arguments_are_refused_before_any_cuda_call():
     assert L.higgs_linear(ctypes.byref(d), a, 1, a, a, a, a, 0, a, 16, None) == hb.HIGGS_ERR_WORKSPACE
     assert L.higgs_quantize(ctypes.byref(d), a, 0, a, a, a, None, a, 16, None) == hb.HIGGS_ERR_WORKSPACE
     assert L.higgs_make_grid(2, 256, a, 100, 10, a, None, None, a, 1 << 30, None) == hb.HIGGS_ERR_INVALID_ARG  # fewer samples than points
-    assert L.higgs_make_grid(3, 256, a, 1000, 10, a, None, None, a, 1 << 30, None) == hb.HIGGS_ERR_UNSUPPORTED
+    assert L.higgs_make_grid(5, 256, a, 1000, 10, a, None, None, a, 1 << 30, None) == hb.HIGGS_ERR_UNSUPPORTED
+    assert L.higgs_make_grid(2, 4097, a, 10000, 10, a, None, None, a, 1 << 30, None) == hb.HIGGS_ERR_UNSUPPORTED
+    # general-grid encoder
+    assert L.higgs_general_tuples(3) == 342 and L.higgs_general_tuples(2) == 512 and L.higgs_general_tuples(5) == 0
+    assert L.higgs_quantize_general(5, 16, 16, 1024, 1, a, 0, a, a, a, None, None) == hb.HIGGS_ERR_UNSUPPORTED
+    assert L.higgs_quantize_general(3, 830, 16, 1000, 1, a, 0, a, a, a, None, None) == hb.HIGGS_ERR_UNSUPPORTED
+    assert L.higgs_quantize_general(3, 830, 16, 1024, 1, None, 0, a, a, a, None, None) == hb.HIGGS_ERR_INVALID_ARG
+    assert L.higgs_quantize_general(3, 830, 0, 1024, 1, None, 0, None, None, None, None, None) == hb.HIGGS_OK
     assert L.higgs_make_grid(2, 256, a, 1000, 10, a, None, None, a, 16, None) == hb.HIGGS_ERR_WORKSPACE
     empty = hb.make_desc(2, 256, 0, 1024, 1)
     assert L.higgs_quantize(ctypes.byref(empty), None, 0, None, None, None, None, None, 0, None) == hb.HIGGS_OK

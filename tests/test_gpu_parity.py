@@ -279,6 +279,106 @@ def test_layer_error_matches_oracle(p, n, N, K):
     assert abs(t2 - mse) <= (0.08 if n < 256 or p == 2 else 0.25) * mse, (t2, mse)
 
 
+# ----------------------------------------------------------------------------- general grids (evaluation encoder)
+def _random_grid(p, n, seed):
+    """n points of N(0, I_p), fp32-exact, sorted lexicographically: a valid grid for encoder parity (the encoder
+    does not care whether the grid is optimal)."""
+    g = np.random.default_rng(seed).standard_normal((n, p)).astype(np.float32).astype(np.float64)
+    return g[np.lexsort(g.T[::-1])]
+
+
+@pytest.mark.parametrize("p,n,N,K,bf16", [
+    (3, 830, 12, 2048, True),     # the paper's 3.25-bit grid: 342 tuples per group, the last one completed with zeros
+    (2, 88, 16, 1024, True),      # 3.25 bits, p = 2
+    (2, 361, 9, 3072, False),     # 4.25 bits
+    (1, 19, 16, 2048, True),      # 4.25 bits, scalar
+    (4, 256, 8, 2048, True),      # 2 bits, p = 4
+    (4, 4096, 5, 1024, False),    # the largest supported grid (64 KB of fp32)
+    (3, 9, 300, 1024, True),      # smallest n of the paper's sweep; more items than one wave of warps
+    (2, 256, 16, 2048, True),     # a kernel-supported grid through the general encoder
+])
+def test_quantize_general_matches_oracle(p, n, N, K, bf16):
+    """Algorithm 1 with any grid: codes against the oracle (near-ties counted), scales, and the layer error t^2 the
+    same pass accumulates against the oracle's dequantise-and-subtract in the original space."""
+    xi = inputs.rht_seed(4)
+    W = inputs.make_weights(N, K, seed=3000 + n, bf16=bf16)
+    g64 = _random_grid(p, n, 50 + n)
+    gt = U.f32_tensor(g64)
+    Wt = U.bf16_tensor(W) if bf16 else U.f32_tensor(W)
+    codes, scales, t2 = hb.higgs_quantize_general(p, n, Wt, gt, xi)
+    torch.cuda.synchronize()
+    q, sc16 = U.oracle_encode(W, G, g64, xi)
+    T = oracle.tuples_per_group(G, p)
+    gc = codes.cpu().numpy().astype(np.int64).reshape(N, (K // G) * T)
+    assert gc.min() >= 0 and gc.max() < n
+    U.compare_codes(gc, q, max_frac=max(1e-4, 1.5 / gc.size))
+    # stored scale: the oracle's value rounded once to fp16, up to one unit in the last place (fp32 norm on the device)
+    sg = scales.cpu().numpy()
+    assert sg.shape == sc16.shape
+    assert np.max(np.abs(sg.astype(np.float64) - sc16.astype(np.float64)) / sc16.astype(np.float64)) <= 2.0 ** -10
+    # t^2 from the device's own codes and scales, evaluated by the oracle in the original space
+    t2_ref = oracle.layer_error(W, gc.astype(np.int32), sg.astype(np.float64), G, g64, xi)
+    assert abs(t2 - t2_ref) <= 2e-4 * t2_ref, (t2, t2_ref)
+    if (p, n) == (2, 256):
+        d = hb.make_desc(p, n, N, K, xi)
+        _, _, canon = hb.higgs_quantize(d, Wt, gt, want_canonical=True)
+        assert np.array_equal(canon.cpu().numpy().astype(np.int64), gc)
+
+
+def test_quantize_general_edge_cases():
+    xi = inputs.rht_seed(4)
+    g64 = _random_grid(3, 17, 1)
+    gt = U.f32_tensor(g64)
+    # a zero group: scale 0, finite codes (the point nearest the origin), error 0
+    W = np.zeros((2, 1024), dtype=np.float32)
+    codes, scales, t2 = hb.higgs_quantize_general(3, 17, U.f32_tensor(W), gt, xi)
+    q, _ = U.oracle_encode(W, G, g64, xi)
+    assert np.array_equal(codes.cpu().numpy().astype(np.int64).reshape(2, -1), q.codes)
+    assert float(scales.abs().max()) == 0.0 and t2 == 0.0
+    # empty matrix
+    codes, scales, t2 = hb.higgs_quantize_general(3, 17, torch.empty((0, 1024), dtype=torch.float32, device=U.dev()), gt, xi)
+    assert codes.numel() == 0 and t2 == 0.0
+    # unsupported shapes are refused
+    for (pp, nn) in [(5, 16), (2, 4097)]:
+        with pytest.raises(hb.HiggsError) as e:
+            hb.higgs_quantize_general(pp, nn, U.f32_tensor(np.zeros((1, 1024))), torch.zeros((nn, pp), device=U.dev()), xi)
+        assert e.value.status == hb.HIGGS_ERR_UNSUPPORTED
+    with pytest.raises(hb.HiggsError) as e:                       # K must be a multiple of the group size
+        hb.higgs_quantize_general(3, 17, U.f32_tensor(np.zeros((1, 512))), gt, xi)
+    assert e.value.status == hb.HIGGS_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("p,n,log2m", [(3, 830, 15), (2, 88, 15), (1, 19, 16), (4, 300, 14), (2, 361, 15)])
+def test_make_grid_general_is_a_lloyd_fixed_point(p, n, log2m):
+    """Algorithm 2 for the grids outside the kernel family: the device's fit is a fixed point of the oracle's Lloyd
+    step on the same samples, sorted, with the MSE the oracle computes for it; t^2 of a layer encoded with it agrees
+    with that MSE on fresh Gaussian samples (Appendix 'Proof of Expected Error')."""
+    s = inputs.gaussian_samples(p, 4000 + n, log2_count=log2m)
+    grid, mse, iters = hb.higgs_make_grid(p, n, U.f32_tensor(s), max_iters=3000)
+    torch.cuda.synchronize()
+    g = grid.cpu().numpy().astype(np.float64)
+    assert int(iters) > 3, int(iters)
+    keys = [tuple(r) for r in g]
+    assert keys == sorted(keys)
+    s32 = s.astype(np.float32).astype(np.float64)
+    assert abs(float(mse) - oracle.grid_mse(g, s32)) <= 1e-5 * float(mse)
+    a = np.concatenate([((c[:, None, :] - g[None, :, :]) ** 2).sum(-1).argmin(1) for c in np.array_split(s32, 64)])
+    sums = np.zeros((n, p))
+    np.add.at(sums, a, s32)
+    cnt = np.bincount(a, minlength=n)
+    occupied = cnt > 0
+    assert np.max(np.abs(sums[occupied] / cnt[occupied, None] - g[occupied])) < 5e-6
+    # rate-distortion sanity: below the scalar Lloyd-Max error at the next lower integer rate, above Shannon's bound
+    rate = np.log2(n) / p
+    assert 2.0 ** (-2 * rate) < float(mse)
+    # the layer error of weights encoded with this grid is the grid's error on fresh samples
+    xi = inputs.rht_seed(5)
+    W = inputs.make_weights(48, 2048, seed=77 + n, bf16=True)
+    _, _, t2 = hb.higgs_quantize_general(p, n, U.bf16_tensor(W), grid, xi)
+    fresh = oracle.grid_mse(g, inputs.gaussian_samples(p, 778, log2_count=18))
+    assert abs(t2 - fresh) <= 0.06 * fresh, (t2, fresh)
+
+
 # ----------------------------------------------------------------------------- tensor-core path (B > 16, N % 128 == 0)
 @pytest.mark.parametrize("p,n,N,K,B", [
     (2, 256, 128, 1024, 17),     # smallest tile: one block, 16 stages, token tile of 32

@@ -72,6 +72,40 @@ def test_matches_brute_force(g, p, n):
     assert np.all(q.runner != q.codes)
 
 
+@pytest.mark.parametrize("g,p,n", [(16, 3, 7), (64, 3, 40), (1024, 3, 830), (8, 4, 9), (32, 3, 5)])
+def test_ragged_tuples_match_brute_force(g, p, n):
+    """p need not divide g (the paper's (p, n) = (3, 830) with g = 1024): the last tuple is completed with zeros and
+    matched on all p coordinates; reconstruction drops the completed coordinates.  Independent restatement with an
+    explicit Hadamard matrix."""
+    rng = np.random.default_rng(7 * g + n)
+    grid = rng.standard_normal((n, p))
+    grid = grid[np.lexsort(grid.T[::-1])]
+    N, K = (4, 2 * g) if g < 1024 else (2, 1024)
+    W = rng.standard_normal((N, K)) * 0.02
+    xi = 1234 + g
+    sg = oracle.signs(xi, K)
+    H = scipy.linalg.hadamard(g).astype(np.float64)
+    T = -(-g // p)
+    assert oracle.tuples_per_group(g, p) == T
+    q = oracle.quantize(W, g, grid, xi)
+    assert q.codes.shape == (N, (K // g) * T)
+    What = np.zeros_like(W)
+    for r in range(N):
+        for i in range(K // g):
+            w = W[r, i * g:(i + 1) * g]
+            s = np.sqrt((w * w).sum())
+            wd = np.concatenate([H @ (sg[i * g:(i + 1) * g] * w / s), np.zeros(T * p - g)]).reshape(T, p)
+            d = ((wd[:, None, :] - grid[None, :, :]) ** 2).sum(-1)
+            sl = slice((r * 0) + i * T, i * T + T)
+            clear = q.margin[r, sl] > 1e-9
+            assert np.array_equal(q.codes[r, sl][clear], d.argmin(1)[clear]) and clear.mean() > 0.98
+            rec = (s / np.sqrt(g)) * grid[q.codes[r, sl]].reshape(-1)[:g]
+            What[r, i * g:(i + 1) * g] = sg[i * g:(i + 1) * g] * (H @ rec) / np.sqrt(g)
+    assert np.allclose(oracle.dequantize(q.codes, q.scales, g, grid, xi), What, atol=1e-13)
+    # the paper's bit count for this grid: ceil(1024/3) codes of log2(830) bits plus a 16-bit scale per 1024 weights
+    assert round(np.log2(830) / 3 + 16 / 1024, 2) == 3.25 and round(342 * np.log2(830) / 1024 + 16 / 1024, 2) == 3.25
+
+
 def test_margin_is_distance_to_bisector():
     grid = np.array([[0.0, 0.0], [2.0, 0.0], [0.0, 5.0]])
     # g=2 group whose rotated tuple is (0.6, 0.1)*: choose w so that H2 (w/s) = t
