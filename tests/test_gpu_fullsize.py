@@ -88,3 +88,25 @@ def test_pruned_search_equals_exhaustive_scan(p, n, N, K):
     packed_s, scales_s, canon_s = hb.higgs_quantize(ds, U.bf16_tensor(W[:rows]), gt, want_canonical=True)
     assert torch.equal(canon[:rows], canon_s)
     assert torch.equal(hb.scales_from_tile_major(scales, N)[:rows], hb.scales_from_tile_major(scales_s, rows))
+
+
+def test_general_grid_encoder_full_size_on_sampled_rows():
+    """The 3.25-bit grid (p, n) = (3, 830) of the paper's experiment configurations on the 8B q/o matrix: the whole
+    matrix is encoded on the device, sampled rows are compared with the oracle code by code, and the device's t^2 for
+    the whole layer is bracketed by the oracle's t^2 on the sample."""
+    p, n, N, K = 3, 830, 4096, 4096
+    xi = inputs.rht_seed(1)
+    W = inputs.make_weights(N, K, inputs.weight_seed(1, 5), bf16=True)
+    s = inputs.gaussian_samples(p, inputs.grid_sample_seed(p, n), log2_count=16)
+    grid, _, _ = hb.higgs_make_grid(p, n, U.f32_tensor(s), max_iters=500)
+    g64 = grid.cpu().numpy().astype(np.float64)
+    codes, scales, t2 = hb.higgs_quantize_general(p, n, U.bf16_tensor(W), grid, xi)
+    rows = sampled_rows(N, 16, seed=9)
+    q, sc16 = U.oracle_encode(W[rows], G, g64, xi)
+    gc = codes.cpu().numpy().astype(np.int64)[rows].reshape(len(rows), -1)
+    U.compare_codes(gc, q, max_frac=2e-4)
+    sg = scales.cpu().numpy()[rows]
+    ulp = np.abs(sg.view(np.int16).astype(np.int64) - sc16.view(np.int16).astype(np.int64))
+    assert ulp.max() <= 1
+    t2_rows = oracle.layer_error(W[rows], q.codes, sc16.astype(np.float64), G, g64, xi)
+    assert abs(t2 - t2_rows) <= 0.03 * t2_rows, (t2, t2_rows)
