@@ -127,12 +127,14 @@ __global__ void __launch_bounds__(128) encode_kernel(const T* __restrict__ W, co
 // farthest corner bounds the distance of the winner from any point of the cell, so only points whose distance to the
 // cell is at most U (+ a slack far above fp32 rounding) can be nearest.  Their indices are listed in ascending order,
 // so the strict '<' of the scan keeps the lowest index on ties exactly like the exhaustive scan.  Cells with more
-// than kMaxCand candidates, and inputs outside [-R, R)^p, fall back to the exhaustive scan.  The table is built once
+// than kMaxCand candidates, and inputs outside [-R, R)^p, fall back to the exhaustive scan (done by the whole warp for
+// one such point at a time: same distances, lowest index on ties).  The table is built once
 // by a small kernel (into scratch memory the caller lends: the packed-code output buffer, which is written only after
 // the encoder has finished) and copied into shared memory by every persistent encoder block.
-constexpr int kCells2 = 32;            // p = 2: 32 x 32 cells
+constexpr int kCells2 = 64;            // p = 2: 64 x 64 cells of width 1/8 (n = 256: 3 candidates on average, 5 for the
+                                       // slowest of a warp's 32 lanes; 32 x 32 cells had 8 and 13)
 constexpr int kCells1 = 1024;          // p = 1
-constexpr int kMaxCand = 16;
+constexpr int kMaxCand = 8;            // a cell's list is one 8-byte word
 constexpr float kCellR = 4.0f;
 constexpr float kCandSlack = 1e-3f;
 
@@ -219,26 +221,45 @@ __global__ void __launch_bounds__(256) encode_pruned_kernel(const T* __restrict_
 #pragma unroll
         for (int t = 0; t < 32 / P; ++t) {
             const float x = v[P * t], y = P == 2 ? v[2 * t + 1] : 0.f;
-            const float cx = (x + kCellR) * inv_w, cy = P == 2 ? (y + kCellR) * inv_w : 0.f;
-            const bool inside = cx >= 0.f && cx < (float)(P == 2 ? kCells2 : kCells1) &&
-                                (P == 1 || (cy >= 0.f && cy < (float)kCells2));
-            const int cell = inside ? (P == 2 ? (int)cy * kCells2 + (int)cx : (int)cx) : 0;
+            // cell coordinates by rounding down; negative, huge or NaN inputs fail the unsigned comparison
+            const int ix = __float2int_rd((x + kCellR) * inv_w), iy = P == 2 ? __float2int_rd((y + kCellR) * inv_w) : 0;
+            const bool inside = (unsigned)ix < (unsigned)(P == 2 ? kCells2 : kCells1) && (P == 1 || (unsigned)iy < (unsigned)kCells2);
+            const int cell = inside ? (P == 2 ? iy * kCells2 + ix : ix) : 0;
             const int k = inside ? cnt[cell] : 255;
             float best = INFINITY;
             int b = 0;
+            // lanes whose point has no candidate list (a crowded outer cell, or outside the table): the warp scans the
+            // whole grid for them together, one such lane at a time - left to the lane itself the scan would hold up
+            // the other 31 for n iterations whenever any lane needs it
+            unsigned full_scan = __ballot_sync(0xffffffffu, k == 255);
             if (k != 255) {
+                const uint2 l2 = *reinterpret_cast<const uint2*>(&cand[cell * kMaxCand]);     // the whole list
                 for (int i = 0; i < k; ++i) {
-                    const int c = cand[cell * kMaxCand + i];
+                    const int c = (int)(__byte_perm(l2.x, l2.y, (uint32_t)i) & 0xffu);   // byte i of the list
                     const float dx = x - sgrid[P * c], dy = P == 2 ? y - sgrid[2 * c + 1] : 0.f;
                     const float d = P == 2 ? fmaf(dy, dy, dx * dx) : dx * dx;
                     if (d < best) { best = d; b = c; }
                 }
-            } else {
-                for (int c = 0; c < n; ++c) {
-                    const float dx = x - sgrid[P * c], dy = P == 2 ? y - sgrid[2 * c + 1] : 0.f;
+            }
+            __syncwarp();
+            while (full_scan) {
+                const int src = __ffs(full_scan) - 1;
+                full_scan &= full_scan - 1;
+                const float px = __shfl_sync(0xffffffffu, x, src), py = __shfl_sync(0xffffffffu, y, src);
+                float bd = INFINITY;
+                int bc = 0x7fffffff;
+                for (int c = lane; c < n; c += 32) {           // ascending within the lane: '<' keeps its lowest index
+                    const float dx = px - sgrid[P * c], dy = P == 2 ? py - sgrid[2 * c + 1] : 0.f;
                     const float d = P == 2 ? fmaf(dy, dy, dx * dx) : dx * dx;
-                    if (d < best) { best = d; b = c; }
+                    if (d < bd) { bd = d; bc = c; }
                 }
+#pragma unroll
+                for (int m = 16; m >= 1; m >>= 1) {             // across lanes: smaller distance, then lower index
+                    const float od = __shfl_xor_sync(0xffffffffu, bd, m);
+                    const int oc = __shfl_xor_sync(0xffffffffu, bc, m);
+                    if (od < bd || (od == bd && oc < bc)) { bd = od; bc = oc; }
+                }
+                if (lane == src) b = bc;
             }
             bi[t] = b;
         }
