@@ -15,7 +15,8 @@
 //                    shared-memory descriptor) per A stage - one barrier wait per 256 inputs keeps the issuing
 //                    warp's serial bookkeeping off the critical path - and commits them to the mbarriers that free
 //                    the stages;
-//   epilogue         all dequant warps read the fp32 accumulator with tcgen05.ld and store y.
+//   epilogue         all dequant warps read the fp32 accumulator with tcgen05.ld and park it in shared memory, from
+//                    where y is written in 512-byte runs (or the cluster sums the K slices).
 // Layers with few row tiles split K over the blocks of a thread-block cluster (grid z): every block parks its
 // partial tile in its own shared memory, and after a cluster barrier block z sums the partials of "its" token
 // columns through distributed shared memory in a fixed order and writes them - no atomics, no zeroing, and the
@@ -177,7 +178,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
     //   [lut, lut+64 KB)     lookup table, 256-byte rows (bytes 0..127 = the entry replicated per lane)
     //   [lut+64 KB, ...)     three activation-tile stages (FB x BN x 128 bytes each; they come from L2)
     //   [..., end)           code stages, region B (whatever the activation stages leave: 52 KB for BN <= 128)
-    //   after the main loop, K-split only: [base+2 KB, +BN x 512 B) the block's partial tile, [token][row] fp32
+    //   after the main loop: [base+2 KB, +BN x 512 B) the block's (partial) output tile, [token][row] fp32
     // Three rings: codes (freed when the four dequant warps of a step have read them), activation tiles and the
     // A operand in TMEM (both freed by tcgen05.commit when the MMAs that read them are done).
     const uint32_t base = (uint32_t)__cvta_generic_to_shared(smem_raw);
@@ -500,39 +501,20 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
         t_report(bad, abort_flag);
         if (!bad) {
             tc_fence_after();
-            const int64_t row = row0 + i;
-            if (ksplit == 1) {
-                // epilogue: accumulator row i, 32 token columns at a time, the column chunks dealt over the warp groups
-                pdl_wait();        // y may still be read by the kernel before this one
-                if (warp == 3) TTRACE(3, 4);
-                for (int c0 = 32 * sg; c0 < BN; c0 += 32 * kTcGroups) {
-                    uint32_t d[32];
-                    tc_ld32(t_lane + (uint32_t)c0, d);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                    if (warp == 3 && c0 == 0) TTRACE(3, 5);
+            // Park the fp32 tile in shared memory as [token][row] (all rings are idle: every MMA has completed, so
+            // every copy has landed and every lookup has been done).  Without a K split it is written out from there in
+            // 512-byte runs (one token's 128 rows per store instruction of a warp): storing straight from the
+            // accumulator registers - 128 bytes per instruction, 32 instructions per thread - took 1.5-1.8 us per 32
+            // token columns.  With a K split the cluster sums the parked tiles.
+            for (int c0 = 32 * sg; c0 < BN; c0 += 32 * kTcGroups) {
+                uint32_t d[32];
+                tc_ld32(t_lane + (uint32_t)c0, d);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (warp == 3 && c0 == 0) TTRACE(3, 5);
 #pragma unroll
-                    for (int r = 0; r < 32; ++r) {
-                        const int b = bt * BN + c0 + r;
-                        if (c0 + r < BN && b < prm.B) {
-                            const float v = __uint_as_float(d[r]);
-                            if (prm.y_mode == 0) static_cast<float*>(prm.y)[(int64_t)b * prm.N + row] = v;
-                            else static_cast<__nv_bfloat16*>(prm.y)[(int64_t)b * prm.N + row] = __float2bfloat16_rn(v);
-                        }
-                    }
-                    if (warp == 3 && c0 == 0) TTRACE(3, 6);
-                }
-            } else {
-                // K-split: park the partial tile in shared memory as [token][row] (all rings are idle: every MMA
-                // has completed, so every copy has landed and every lookup has been done)
-                for (int c0 = 32 * sg; c0 < BN; c0 += 32 * kTcGroups) {
-                    uint32_t d[32];
-                    tc_ld32(t_lane + (uint32_t)c0, d);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-                    for (int r = 0; r < 32; ++r)
-                        if (c0 + r < BN)
-                            asm volatile("st.shared.b32 [%0], %1;" ::"r"(code0 + (uint32_t)(((c0 + r) * 128 + i) * 4)), "r"(d[r]) : "memory");
-                }
+                for (int r = 0; r < 32; ++r)
+                    if (c0 + r < BN)
+                        asm volatile("st.shared.b32 [%0], %1;" ::"r"(code0 + (uint32_t)(((c0 + r) * 128 + i) * 4)), "r"(d[r]) : "memory");
             }
         }
     }
@@ -546,7 +528,30 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
     }
-    if (ksplit > 1) {
+    if (ksplit == 1) {
+        // the parked tile -> y: warp w writes token columns w, w + 16, ...; a lane holds four consecutive rows
+        if (tid < 512 && !*abort_flag) {
+            pdl_wait();            // y may still be read by the kernel before this one
+            if (warp == 3) TTRACE(3, 4);
+            for (int c = warp; c < BN; c += 16) {
+                const int b = bt * BN + c;
+                if (b >= prm.B) break;
+                uint32_t v0, v1, v2, v3;
+                asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3)
+                             : "r"(code0 + (uint32_t)((c * 128 + lane * 4) * 4)) : "memory");
+                const int64_t o = (int64_t)b * prm.N + row0 + lane * 4;
+                if (prm.y_mode == 0) {
+                    *reinterpret_cast<uint4*>(static_cast<float*>(prm.y) + o) = make_uint4(v0, v1, v2, v3);
+                } else {
+                    const __nv_bfloat162 lo = __floats2bfloat162_rn(__uint_as_float(v0), __uint_as_float(v1));
+                    const __nv_bfloat162 hi = __floats2bfloat162_rn(__uint_as_float(v2), __uint_as_float(v3));
+                    *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(prm.y) + o) =
+                        make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+                }
+            }
+            if (warp == 3) TTRACE(3, 6);
+        }
+    } else {
         // Cluster reduction in a fixed order: block kz owns the token columns [kz, kz+1) * BN / ksplit and sums the
         // partial tiles of all blocks of the cluster for them through distributed shared memory.
         asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
@@ -554,22 +559,37 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
         const int cols = BN / ksplit;
         if (tid < 512 && !*abort_flag) {
             pdl_wait();            // y may still be read by the kernel before this one
-            const int rrow = tid & 127;
-            for (int cc = tid >> 7; cc < cols; cc += 4) {
+            // warp w sums token columns w, w + 16, ... of this block's share; a lane holds four consecutive rows, so a
+            // warp reads 512 contiguous bytes of every slice's tile and writes 512 contiguous bytes of y
+            for (int cc = warp; cc < cols; cc += 16) {
                 const int c = kz * cols + cc;
-                const uint32_t local = code0 + (uint32_t)((c * 128 + rrow) * 4);
-                float acc = 0.f;
-                for (int r = 0; r < ksplit; ++r) {
-                    uint32_t remote;
-                    float v;
-                    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(r));
-                    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
-                    acc += v;
+                const uint32_t local = code0 + (uint32_t)((c * 128 + lane * 4) * 4);
+                float4 part[8];
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    part[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (r < ksplit) {
+                        uint32_t remote;
+                        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(r));
+                        asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];"
+                                     : "=f"(part[r].x), "=f"(part[r].y), "=f"(part[r].z), "=f"(part[r].w) : "r"(remote) : "memory");
+                    }
+                }
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {            // slice order: fixed, so the sum is reproducible
+                    if (r < ksplit) { acc.x += part[r].x; acc.y += part[r].y; acc.z += part[r].z; acc.w += part[r].w; }
                 }
                 const int b = bt * BN + c;
                 if (b < prm.B) {
-                    if (prm.y_mode == 0) static_cast<float*>(prm.y)[(int64_t)b * prm.N + row0 + rrow] = acc;
-                    else static_cast<__nv_bfloat16*>(prm.y)[(int64_t)b * prm.N + row0 + rrow] = __float2bfloat16_rn(acc);
+                    const int64_t o = (int64_t)b * prm.N + row0 + lane * 4;
+                    if (prm.y_mode == 0) {
+                        *reinterpret_cast<float4*>(static_cast<float*>(prm.y) + o) = acc;
+                    } else {
+                        const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+                        *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(prm.y) + o) =
+                            make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+                    }
                 }
             }
         }
