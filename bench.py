@@ -383,9 +383,9 @@ def run_ours(args):
     if rank == 0:
         t_probe = time.perf_counter()
         with torch.cuda.stream(stream):
-            while time.perf_counter() - t_probe < 0.5:
-                run_steps(0, 64)
-                extra_steps += 64
+            while time.perf_counter() - t_probe < 0.5:      # small batches: under a profiler every launch is slow
+                run_steps(0, 8)
+                extra_steps += 8
                 stream.synchronize()
     clocks = sampler.stop() if rank == 0 else None
     if clocks is not None:

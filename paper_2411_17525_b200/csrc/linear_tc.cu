@@ -603,45 +603,71 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
 
 namespace {
 
-// Rotation of the activations (Appendix F) for the tensor-core path: one warp per (token, group), output written in
-// the blocked order the MMA's shared-memory descriptor expects, so that one stage (BN tokens x 64 inputs) is one
-// contiguous run:  [batch tile][K/64][BN/8 token blocks][8 input cores][8 tokens][8 inputs] fp16.
-__global__ void __launch_bounds__(256) rht_activations_tc_kernel(const __nv_bfloat16* __restrict__ x, __half* __restrict__ xdag,
+// Rotation of the activations (Appendix F) for the tensor-core path: four warps per (token, group) - the transform sits
+// on the latency path between dependent launches -, output written in the blocked order the MMA's shared-memory
+// descriptor expects, so that one stage (BN tokens x 64 inputs) is one contiguous run:
+//   [batch tile][K/64][BN/8 token blocks][8 input cores][8 tokens][8 inputs] fp16.
+// Warp q of the block owns inputs 256 q .. + 255 of the group, 8 consecutive ones per lane (one core-matrix row):
+// butterflies over those 8 in registers, over the 32 lanes by shuffles, over the 4 warps through shared memory.
+__global__ void __launch_bounds__(128) rht_activations_tc_kernel(const __nv_bfloat16* __restrict__ x, __half* __restrict__ xdag,
                                                                  int64_t B, int64_t K, uint64_t xi, int BN) {
-    const int lane = threadIdx.x & 31;
-    const int64_t warp = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    __shared__ __align__(16) float ex[4][256];
+    const int lane = threadIdx.x & 31, q = threadIdx.x >> 5;
     const int64_t groups = K / kGroup;
     pdl_trigger();
     pdl_wait();
-    if (warp >= B * groups) return;
-    const int64_t b = warp / groups, gi = warp % groups;
-    const __nv_bfloat16* src = x + b * K + gi * kGroup;
-    float v[32];
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(src + c * 256 + lane * 8));
+    const int64_t b = blockIdx.x / groups, gi = blockIdx.x % groups;       // grid = B * groups blocks
+    const int64_t k0 = gi * kGroup + q * 256 + lane * 8;
+    float v[8];
+    {
+        const uint4 q4 = __ldg(reinterpret_cast<const uint4*>(x + b * K + k0));
         const uint32_t w4[4] = {q4.x, q4.y, q4.z, q4.w};
+        const uint32_t bits = (uint32_t)(sign_word(xi, (uint64_t)k0 >> 6) >> ((uint64_t)k0 & 63ull)) & 0xffu;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            v[c * 8 + 2 * e] = __uint_as_float(w4[e] << 16);
-            v[c * 8 + 2 * e + 1] = __uint_as_float(w4[e] & 0xffff0000u);
+            v[2 * e] = __uint_as_float((w4[e] << 16) ^ (((bits >> (2 * e)) & 1u) << 31));
+            v[2 * e + 1] = __uint_as_float((w4[e] & 0xffff0000u) ^ (((bits >> (2 * e + 1)) & 1u) << 31));
         }
     }
-    apply_signs1024(v, xi, gi * kGroup, lane);
-    fwht1024_warp(v, lane);
+#pragma unroll
+    for (int h = 1; h < 8; h <<= 1) {
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            if ((r & h) == 0) { const float a = v[r], c = v[r | h]; v[r] = a + c; v[r | h] = a - c; }
+        }
+    }
+#pragma unroll
+    for (int m = 1; m < 32; m <<= 1) {
+        const bool upper = (lane & m) != 0;
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            const float o = __shfl_xor_sync(0xffffffffu, v[r], m);
+            v[r] = upper ? (o - v[r]) : (v[r] + o);
+        }
+    }
+    *reinterpret_cast<float4*>(&ex[q][lane * 8]) = make_float4(v[0], v[1], v[2], v[3]);
+    *reinterpret_cast<float4*>(&ex[q][lane * 8 + 4]) = make_float4(v[4], v[5], v[6], v[7]);
+    __syncthreads();
+    float o[8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r) o[r] = 0.f;
+#pragma unroll
+    for (int qq = 0; qq < 4; ++qq) {
+        const float4 u0 = *reinterpret_cast<const float4*>(&ex[qq][lane * 8]);
+        const float4 u1 = *reinterpret_cast<const float4*>(&ex[qq][lane * 8 + 4]);
+        const float sgn = (__popc(q & qq) & 1) ? -1.f : 1.f;
+        o[0] = fmaf(sgn, u0.x, o[0]); o[1] = fmaf(sgn, u0.y, o[1]); o[2] = fmaf(sgn, u0.z, o[2]); o[3] = fmaf(sgn, u0.w, o[3]);
+        o[4] = fmaf(sgn, u1.x, o[4]); o[5] = fmaf(sgn, u1.y, o[5]); o[6] = fmaf(sgn, u1.z, o[6]); o[7] = fmaf(sgn, u1.w, o[7]);
+    }
+    uint32_t w4[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const __half2 hh = __floats2half2_rn(o[2 * e] * 0.03125f, o[2 * e + 1] * 0.03125f);
+        w4[e] = *reinterpret_cast<const uint32_t*>(&hh);
+    }
     const int64_t bt = b / BN, nloc = b % BN;
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        uint32_t w4[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            __half2 h = __floats2half2_rn(v[c * 8 + 2 * e] * 0.03125f, v[c * 8 + 2 * e + 1] * 0.03125f);
-            w4[e] = *reinterpret_cast<uint32_t*>(&h);
-        }
-        const int64_t k = gi * kGroup + c * 256 + lane * 8;        // 8 consecutive inputs = one core-matrix row
-        const int64_t off = ((bt * (K / 64) + k / 64) * BN * 64) + (nloc / 8) * 512 + ((k % 64) / 8) * 64 + (nloc % 8) * 8;
-        *reinterpret_cast<uint4*>(xdag + off) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
-    }
+    const int64_t off = ((bt * (K / 64) + k0 / 64) * BN * 64) + (nloc / 8) * 512 + ((k0 % 64) / 8) * 64 + (nloc % 8) * 8;
+    *reinterpret_cast<uint4*>(xdag + off) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
 }
 
 }  // namespace
@@ -671,8 +697,9 @@ size_t tc_workspace_bytes(const higgs_desc& d, int64_t B) {
 // D1 for the tensor-core path: rotated activations in the blocked operand layout (tc_workspace_bytes() bytes).
 int launch_rht_tc(const higgs_desc& d, const void* x, int64_t B, __half* xdag_tc, cudaStream_t st) {
     const int BN = tc_batch_tile(B);
-    const int64_t warps = B * (d.K / kGroup);
-    return cuda_status(launch_pdl(rht_activations_tc_kernel, dim3((unsigned)((warps + 7) / 8)), dim3(256), 0, st,
+    const int64_t blocks = B * (d.K / kGroup);              // four warps per (token, group)
+    if (blocks > 0x7fffffff) return HIGGS_ERR_UNSUPPORTED;
+    return cuda_status(launch_pdl(rht_activations_tc_kernel, dim3((unsigned)blocks), dim3(128), 0, st,
                                   static_cast<const __nv_bfloat16*>(x), xdag_tc, B, d.K, d.rht_seed, BN));
 }
 
