@@ -384,7 +384,7 @@ def run_ours(args):
         t_probe = time.perf_counter()
         with torch.cuda.stream(stream):
             while time.perf_counter() - t_probe < 0.5:      # small batches: under a profiler every launch is slow
-                run_steps(0, 8)
+                run_steps(extra_steps, 8)               # keeps rotating over the weight copies like the timed steps
                 extra_steps += 8
                 stream.synchronize()
     clocks = sampler.stop() if rank == 0 else None
