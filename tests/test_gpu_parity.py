@@ -432,7 +432,10 @@ def test_tensor_core_k_split_is_deterministic():
     assert torch.equal(ys[0], ys[1]) and torch.equal(ys[0], ys[2])
 
 
-def test_linear_tensor_core_path_bf16_output():
-    y, y_ref = run_linear_case(2, 256, 128, 2048, 32, xi=5, wseed=9, xseed=10, out_dtype=torch.bfloat16)
+@pytest.mark.parametrize("N,K,B", [(128, 2048, 32),      # K split over a cluster: the reduction writes bf16
+                                   (8448, 1024, 40),     # no K split: the parked tile is written out as bf16
+                                   (8448, 1024, 300)])   # two token tiles, the second one ragged
+def test_linear_tensor_core_path_bf16_output(N, K, B):
+    y, y_ref = run_linear_case(2, 256, N, K, B, xi=5, wseed=9, xseed=10, out_dtype=torch.bfloat16)
     assert y.dtype == torch.bfloat16
     assert U.linear_error(y.float().cpu().numpy(), y_ref) <= Y_TOL + 2.0 ** -8
