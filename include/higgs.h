@@ -219,6 +219,20 @@ int higgs_linear_host(const higgs_desc* desc, const void* x_host, int64_t B,
 size_t higgs_linear_host_workspace_bytes(const higgs_desc* desc, int64_t B, int y_dtype);
 
 /*
+ * `count` higgs_linear_host calls enqueued by ONE call - the products of a transformer block, say - so that the
+ * host spends one library call, not `count`, per step.  Argument i of every array belongs to layer i
+ * (descs[i], x_hosts[i], packed[i], scales[i], grids[i], y_hosts[i], workspaces[i], workspace_bytes[i]); B and
+ * y_dtype are common.  Layers that name the SAME x_hosts pointer and have the same K (q/k/v; gate/up) share one
+ * host-to-device copy: the later layer reads the staged copy in the earlier layer's workspace, so those workspaces
+ * must stay untouched until the stream has passed this call.  Returns the first error and enqueues nothing further
+ * after it.  Asynchronous on `stream`; the caller synchronises before reading any y_hosts[i].
+ */
+int higgs_linear_host_batch(int32_t count, const higgs_desc* const* descs, const void* const* x_hosts, int64_t B,
+                            const void* const* packed, const void* const* scales, const float* const* grids,
+                            void* const* y_hosts, int y_dtype, void* const* workspaces,
+                            const size_t* workspace_bytes, void* stream);
+
+/*
  * higgs_linear without a workspace argument, for callers that cannot allocate
  * device memory (code running where cudaMalloc is off limits, plugins that are
  * only handed their input and output buffers, processes whose memory pool

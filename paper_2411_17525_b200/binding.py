@@ -26,7 +26,7 @@ EXPORTS = [
     "higgs_linear_host", "higgs_linear_host_workspace_bytes", "higgs_linear_launch_count", "higgs_device_status",
     "higgs_linear_static", "higgs_linear_static_capacity", "higgs_linear_k_splits", "higgs_rotated_bytes",
     "higgs_rotated_layout", "higgs_dequantize", "higgs_make_uniform_grid", "higgs_layer_error",
-    "higgs_allocate_bits", "higgs_general_tuples", "higgs_quantize_general",
+    "higgs_allocate_bits", "higgs_general_tuples", "higgs_quantize_general", "higgs_linear_host_batch",
 ]
 
 
@@ -71,6 +71,8 @@ def _load() -> ctypes.CDLL:
     lib.higgs_linear_prerotated.argtypes = [P, vp, i64, vp, vp, vp, vp, i32, vp, sz, vp]
     lib.higgs_linear_host.restype = i32
     lib.higgs_linear_host.argtypes = [P, vp, i64, vp, vp, vp, vp, i32, vp, sz, vp]
+    lib.higgs_linear_host_batch.restype = i32
+    lib.higgs_linear_host_batch.argtypes = [i32, vp, vp, i64, vp, vp, vp, vp, i32, vp, vp, vp]
     lib.higgs_linear_host_workspace_bytes.restype = sz
     lib.higgs_linear_host_workspace_bytes.argtypes = [P, i64, i32]
     lib.higgs_rotated_bytes.restype = sz
@@ -250,6 +252,45 @@ def higgs_linear_host(desc: higgs_desc, x_host: torch.Tensor, packed: torch.Tens
                                  _ptr(y_host), _dtype_code(y_host), _ptr(workspace), workspace.numel(), _stream()),
            "higgs_linear_host")
     return y_host
+
+
+class HostBatch:
+    """Argument arrays of higgs_linear_host_batch, marshalled once: `count` layers of one step.  x_hosts may name the
+    same pinned tensor for layers that read the same activations (they then share one host-to-device copy)."""
+
+    def __init__(self, descs, x_hosts, packed, scales, grids, y_hosts, workspaces):
+        n = len(descs)
+        assert all(len(a) == n for a in (x_hosts, packed, scales, grids, y_hosts, workspaces))
+        for x, y, w in zip(x_hosts, y_hosts, workspaces):
+            assert (not x.is_cuda) and x.dtype == torch.bfloat16 and x.is_contiguous()
+            assert (not y.is_cuda) and y.is_contiguous() and y.dtype == y_hosts[0].dtype and w.is_cuda
+        self.keep = (list(descs), list(x_hosts), list(packed), list(scales), list(grids), list(y_hosts), list(workspaces))
+        self.count = n
+        self.B = int(x_hosts[0].shape[0]) if n else 0
+        self.y_dtype = _dtype_code(y_hosts[0]) if n else HIGGS_F32
+        arr = ctypes.c_void_p * max(n, 1)
+        self.descs = arr(*[ctypes.addressof(d) for d in descs])
+        self.x = arr(*[t.data_ptr() for t in x_hosts])
+        self.y = arr(*[t.data_ptr() for t in y_hosts])
+        self.ws = arr(*[t.data_ptr() for t in workspaces])
+        self.ws_bytes = (ctypes.c_size_t * max(n, 1))(*[t.numel() for t in workspaces])
+        self.packed = arr(*[t.data_ptr() for t in packed])
+        self.scales = arr(*[t.data_ptr() for t in scales])
+        self.grids = arr(*[t.data_ptr() for t in grids])
+
+    def set_weights(self, packed, scales):
+        """Point the batch at another copy of the packed weights (same shapes)."""
+        self.keep = self.keep[:2] + (list(packed), list(scales)) + self.keep[4:]
+        for i, (p, s) in enumerate(zip(packed, scales)):
+            self.packed[i] = p.data_ptr()
+            self.scales[i] = s.data_ptr()
+
+
+def higgs_linear_host_batch(batch: HostBatch) -> None:
+    """Enqueues copy-in, the layers and copy-out of every layer of `batch` on the current stream with one library call;
+    synchronise before reading the y_hosts."""
+    _check(lib.higgs_linear_host_batch(batch.count, batch.descs, batch.x, batch.B, batch.packed, batch.scales, batch.grids,
+                                       batch.y, batch.y_dtype, batch.ws, batch.ws_bytes, _stream()), "higgs_linear_host_batch")
 
 
 def higgs_linear_static_capacity() -> int:

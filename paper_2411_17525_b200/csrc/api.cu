@@ -281,6 +281,46 @@ int higgs_linear_host(const higgs_desc* d, const void* x_host, int64_t B, const 
     return HIGGS_OK;
 }
 
+int higgs_linear_host_batch(int32_t count, const higgs_desc* const* descs, const void* const* x_hosts, int64_t B,
+                            const void* const* packed, const void* const* scales, const float* const* grids,
+                            void* const* y_hosts, int y_dtype, void* const* workspaces,
+                            const size_t* workspace_bytes, void* stream) {
+    if (count < 0) return HIGGS_ERR_INVALID_ARG;
+    if (count == 0) return HIGGS_OK;
+    if (!descs || !x_hosts || !packed || !scales || !grids || !y_hosts || !workspaces || !workspace_bytes)
+        return HIGGS_ERR_INVALID_ARG;
+    if (y_dtype != HIGGS_F32 && y_dtype != HIGGS_BF16) return HIGGS_ERR_UNSUPPORTED;
+    if (B < 0) return HIGGS_ERR_INVALID_ARG;
+    cudaStream_t st = as_stream(stream);
+    for (int i = 0; i < count; ++i) {
+        const higgs_desc* d = descs[i];
+        int rc = check_desc(d);
+        if (rc != HIGGS_OK) return rc;
+        if (B == 0 || d->N == 0) continue;
+        if (!x_hosts[i] || !y_hosts[i] || !workspaces[i] || !aligned(workspaces[i], 256)) return HIGGS_ERR_INVALID_ARG;
+        const size_t inner = higgs_workspace_bytes(d, HIGGS_OP_LINEAR, B);
+        const size_t xb = align_up((size_t)B * d->K * 2, 256);
+        const size_t ybytes = (size_t)B * d->N * (y_dtype == HIGGS_F32 ? 4 : 2);
+        if (workspace_bytes[i] < inner + xb + align_up(ybytes, 256)) return HIGGS_ERR_WORKSPACE;
+        uint8_t* ws = static_cast<uint8_t*>(workspaces[i]);
+        const void* x_dev = nullptr;
+        for (int j = 0; j < i && !x_dev; ++j) {       // an earlier layer staged the same activations
+            if (x_hosts[j] == x_hosts[i] && descs[j]->K == d->K && descs[j]->N != 0)
+                x_dev = static_cast<const uint8_t*>(workspaces[j]) + higgs_workspace_bytes(descs[j], HIGGS_OP_LINEAR, B);
+        }
+        if (!x_dev) {
+            if (cudaMemcpyAsync(ws + inner, x_hosts[i], (size_t)B * d->K * 2, cudaMemcpyHostToDevice, st) != cudaSuccess)
+                return HIGGS_ERR_CUDA;
+            x_dev = ws + inner;
+        }
+        void* y_dev = ws + inner + xb;
+        rc = higgs_linear(d, x_dev, B, packed[i], scales[i], grids[i], y_dev, y_dtype, ws, inner, stream);
+        if (rc != HIGGS_OK) return rc;
+        if (cudaMemcpyAsync(y_hosts[i], y_dev, ybytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return HIGGS_ERR_CUDA;
+    }
+    return HIGGS_OK;
+}
+
 size_t higgs_linear_host_workspace_bytes(const higgs_desc* d, int64_t B, int y_dtype) {
     const size_t inner = higgs_workspace_bytes(d, HIGGS_OP_LINEAR, B);
     if (inner == 0) return 0;

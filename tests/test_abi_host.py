@@ -88,6 +88,10 @@ def test_invalid_arguments_are_refused_before_any_cuda_call():
     assert L.higgs_make_grid(2, 256, a, 100, 10, a, None, None, a, 1 << 30, None) == hb.HIGGS_ERR_INVALID_ARG  # fewer samples than points
     assert L.higgs_make_grid(5, 256, a, 1000, 10, a, None, None, a, 1 << 30, None) == hb.HIGGS_ERR_UNSUPPORTED
     assert L.higgs_make_grid(2, 4097, a, 10000, 10, a, None, None, a, 1 << 30, None) == hb.HIGGS_ERR_UNSUPPORTED
+    # batched host call
+    assert L.higgs_linear_host_batch(-1, None, None, 1, None, None, None, None, 0, None, None, None) == hb.HIGGS_ERR_INVALID_ARG
+    assert L.higgs_linear_host_batch(0, None, None, 1, None, None, None, None, 0, None, None, None) == hb.HIGGS_OK
+    assert L.higgs_linear_host_batch(2, None, None, 1, None, None, None, None, 0, None, None, None) == hb.HIGGS_ERR_INVALID_ARG
     # general-grid encoder
     assert L.higgs_general_tuples(3) == 342 and L.higgs_general_tuples(2) == 512 and L.higgs_general_tuples(5) == 0
     assert L.higgs_quantize_general(5, 16, 16, 1024, 1, a, 0, a, a, a, None, None) == hb.HIGGS_ERR_UNSUPPORTED

@@ -279,6 +279,44 @@ def test_layer_error_matches_oracle(p, n, N, K):
     assert abs(t2 - mse) <= (0.08 if n < 256 or p == 2 else 0.25) * mse, (t2, mse)
 
 
+# ----------------------------------------------------------------------------- host-buffer entry points
+@pytest.mark.parametrize("B", [1, 4, 40])
+def test_linear_host_and_host_batch_match_device_path(B):
+    """higgs_linear_host / higgs_linear_host_batch (host activations in, host outputs out) give exactly what
+    higgs_linear gives on device buffers; layers naming the same host tensor share one copy."""
+    xi = inputs.rht_seed(6)
+    shapes = [(2, 256, 256, 2048), (2, 256, 128, 2048), (2, 64, 128, 1024)]
+    descs, packed, scales, grids, xs, ys_dev = [], [], [], [], [], []
+    x_shared = torch.from_numpy(inputs.make_activations(B, 2048, seed=31)).to(torch.bfloat16).pin_memory()
+    x_other = torch.from_numpy(inputs.make_activations(B, 1024, seed=32)).to(torch.bfloat16).pin_memory()
+    for li, (p, n, N, K) in enumerate(shapes):
+        d = hb.make_desc(p, n, N, K, xi)
+        # bit-for-bit comparison: the small-batch path must not split K (atomics); the cluster split of the tensor-core
+        # path sums in a fixed order
+        assert hb.higgs_linear_k_splits(d, B) == 1 or hb.higgs_rotated_layout(d, B) > 0
+        _, gt = U.grid32(p, n)
+        W = inputs.make_weights(N, K, seed=40 + li, bf16=True)
+        pk, sc, _ = hb.higgs_quantize(d, U.bf16_tensor(W), gt)
+        xh = x_shared if K == 2048 else x_other
+        descs.append(d); packed.append(pk); scales.append(sc); grids.append(gt); xs.append(xh)
+        ys_dev.append(hb.higgs_linear(d, xh.to(U.dev()), pk, sc, gt).cpu())
+    ws = [torch.empty(hb.higgs_linear_host_workspace_bytes(d, B), dtype=torch.uint8, device=U.dev()) for d in descs]
+    # one call per layer
+    for li, d in enumerate(descs):
+        yh = torch.empty((B, d.N), dtype=torch.float32).pin_memory()
+        hb.higgs_linear_host(d, xs[li], packed[li], scales[li], grids[li], yh, ws[li])
+        torch.cuda.synchronize()
+        assert torch.equal(yh, ys_dev[li])
+    # one call for all
+    ys_host = [torch.zeros((B, d.N), dtype=torch.float32).pin_memory() for d in descs]
+    batch = hb.HostBatch(descs, xs, packed, scales, grids, ys_host, ws)
+    hb.higgs_linear_host_batch(batch)
+    torch.cuda.synchronize()
+    assert hb.higgs_device_status() == hb.HIGGS_OK
+    for li in range(len(descs)):
+        assert torch.equal(ys_host[li], ys_dev[li])
+
+
 # ----------------------------------------------------------------------------- general grids (evaluation encoder)
 def _random_grid(p, n, seed):
     """n points of N(0, I_p), fp32-exact, sorted lexicographically: a valid grid for encoder parity (the encoder
