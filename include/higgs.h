@@ -205,6 +205,25 @@ int higgs_linear_prerotated(const higgs_desc* desc, const void* xdag, int64_t B,
                             void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Row-sharded layer with the all-gather fused into the product's epilogue (Appendix F's product is independent per
+ * output row, and the rotation is local to a 1024-group of inputs, so a layer splits over devices by rows with no
+ * exchange of weights): this device holds rows [row_offset, row_offset + desc->N) of a layer with `ld` rows in all
+ * (desc, packed, scales describe the SHARD), every device holds the full activations x, and the shard's outputs are
+ * written straight into columns [row_offset, row_offset + desc->N) of EVERY destination
+ *   y_dsts[i] : device-accessible [B][ld] of y_dtype, i < n_dst <= 8 - this device's own output buffer first, then the
+ *               peer-mapped pointers of the other devices' buffers (cudaDeviceEnablePeerAccess / IPC / symmetric
+ *               memory; plain stores over NVLink, no multicast).
+ * The kernels store to all destinations from their epilogue (a K-split small-batch product sums into the workspace
+ * first and a copy kernel spreads the result).  The call neither waits for nor signals other devices: the caller
+ * orders "all shards written" before any reader (e.g. a barrier on the participating streams), and no two shards
+ * overlap in columns.  row_offset a multiple of 16, ld a multiple of 8, ld >= row_offset + desc->N; y_dsts is a HOST
+ * array.  Other arguments, errors and workspace as higgs_linear.
+ */
+int higgs_linear_gather(const higgs_desc* desc, const void* x, int64_t B, const void* packed, const void* scales,
+                        const float* grid, void* const* y_dsts, int32_t n_dst, int64_t ld, int64_t row_offset,
+                        int y_dtype, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * higgs_linear with HOST activations and HOST output (Appendix F product; the
  * weights stay resident on the device): copies x_host ([B][K] bf16, ideally
  * pinned) to the device, runs higgs_linear, copies y ([B][N] of y_dtype) back to

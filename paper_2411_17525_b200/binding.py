@@ -27,6 +27,7 @@ EXPORTS = [
     "higgs_linear_static", "higgs_linear_static_capacity", "higgs_linear_k_splits", "higgs_rotated_bytes",
     "higgs_rotated_layout", "higgs_dequantize", "higgs_make_uniform_grid", "higgs_layer_error",
     "higgs_allocate_bits", "higgs_general_tuples", "higgs_quantize_general", "higgs_linear_host_batch",
+    "higgs_linear_gather",
 ]
 
 
@@ -71,6 +72,8 @@ def _load() -> ctypes.CDLL:
     lib.higgs_linear_prerotated.argtypes = [P, vp, i64, vp, vp, vp, vp, i32, vp, sz, vp]
     lib.higgs_linear_host.restype = i32
     lib.higgs_linear_host.argtypes = [P, vp, i64, vp, vp, vp, vp, i32, vp, sz, vp]
+    lib.higgs_linear_gather.restype = i32
+    lib.higgs_linear_gather.argtypes = [P, vp, i64, vp, vp, vp, vp, i32, i64, i64, i32, vp, sz, vp]
     lib.higgs_linear_host_batch.restype = i32
     lib.higgs_linear_host_batch.argtypes = [i32, vp, vp, i64, vp, vp, vp, vp, i32, vp, vp, vp]
     lib.higgs_linear_host_workspace_bytes.restype = sz
@@ -252,6 +255,35 @@ def higgs_linear_host(desc: higgs_desc, x_host: torch.Tensor, packed: torch.Tens
                                  _ptr(y_host), _dtype_code(y_host), _ptr(workspace), workspace.numel(), _stream()),
            "higgs_linear_host")
     return y_host
+
+
+def shard_rows(N: int, world: int, rank: int, multiple: int = 128):
+    """Rows [begin, end) of an N-row layer that rank `rank` of `world` holds: contiguous, multiples of `multiple` rows
+    (128 keeps every shard eligible for the tensor-core path; at least the 16-row tile), the remainder spread over the
+    first ranks."""
+    assert N % multiple == 0 and 0 <= rank < world
+    units = N // multiple
+    base, extra = divmod(units, world)
+    begin = rank * base + min(rank, extra)
+    return begin * multiple, (begin + base + (1 if rank < extra else 0)) * multiple
+
+
+def higgs_linear_gather(desc: higgs_desc, x: torch.Tensor, packed: torch.Tensor, scales: torch.Tensor, grid: torch.Tensor,
+                        y_dsts, row_offset: int, workspace: Optional[torch.Tensor] = None) -> None:
+    """Row-sharded layer: this device's shard (desc, packed, scales) times x, written into columns
+    [row_offset, row_offset + desc.N) of every tensor of y_dsts ([B][ld] each; this device's own first, then
+    peer-mapped tensors of the other devices).  The caller orders the ranks (see include/higgs.h)."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous()
+    B = x.shape[0]
+    ld = y_dsts[0].shape[1]
+    for t in y_dsts:
+        assert t.is_contiguous() and t.dtype == y_dsts[0].dtype and tuple(t.shape) == (B, ld)
+    if workspace is None:
+        workspace = _workspace(higgs_workspace_bytes(desc, HIGGS_OP_LINEAR, B), x.device)
+    ptrs = (ctypes.c_void_p * len(y_dsts))(*[t.data_ptr() for t in y_dsts])
+    _check(lib.higgs_linear_gather(ctypes.byref(desc), _ptr(x), B, _ptr(packed), _ptr(scales), _ptr(grid), ptrs, len(y_dsts),
+                                   ld, int(row_offset), _dtype_code(y_dsts[0]), _ptr(workspace), workspace.numel(), _stream()),
+           "higgs_linear_gather")
 
 
 class HostBatch:

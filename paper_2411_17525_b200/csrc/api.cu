@@ -241,6 +241,54 @@ int higgs_linear(const higgs_desc* d, const void* x, int64_t B, const void* pack
     return linear_tail(d, xdag, B, packed, scales, grid, y, y_dtype, y32, true, st);
 }
 
+int higgs_linear_gather(const higgs_desc* d, const void* x, int64_t B, const void* packed, const void* scales,
+                        const float* grid, void* const* y_dsts, int32_t n_dst, int64_t ld, int64_t row_offset, int y_dtype,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+    if (!y_dsts || n_dst < 1 || n_dst > kMaxGather) return HIGGS_ERR_INVALID_ARG;
+    int rc = linear_args(d, B, x, packed, scales, grid, y_dsts[0], y_dtype, workspace, workspace_bytes);
+    if (rc != HIGGS_OK) return rc < 0 ? HIGGS_OK : rc;
+    if (row_offset < 0 || row_offset % kRowTile || ld < row_offset + d->N || ld % 8) return HIGGS_ERR_INVALID_ARG;
+    const size_t esz = y_dtype == HIGGS_F32 ? 4 : 2;
+    void* dst[kMaxGather];
+    for (int i = 0; i < n_dst; ++i) {
+        if (!y_dsts[i] || !aligned(y_dsts[i], 16)) return HIGGS_ERR_INVALID_ARG;
+        dst[i] = static_cast<uint8_t*>(y_dsts[i]) + (size_t)row_offset * esz;       // this shard's columns of [B][ld]
+    }
+    GatherTargets more;
+    more.count = n_dst - 1;
+    for (int i = 0; i < kMaxGather - 1; ++i) more.y[i] = i + 1 < n_dst ? dst[i + 1] : nullptr;
+    cudaStream_t st = as_stream(stream);
+    const int mode = y_dtype == HIGGS_F32 ? 0 : 1;
+    if (tc_eligible(*d, B)) {
+        rc = launch_rht_tc(*d, x, B, static_cast<__half*>(workspace), st);
+        if (rc != HIGGS_OK) return rc;
+        return launch_linear_tc(*d, static_cast<const __half*>(workspace), B, packed, scales, grid, dst[0], mode, st, ld, &more);
+    }
+    if (linear_fused_eligible(*d, B))
+        return launch_linear_mma(*d, nullptr, B, packed, scales, grid, dst[0], ld, mode, st, x, &more);
+    __half* xdag = static_cast<__half*>(workspace);
+    float* y32 = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up((size_t)B * d->K * 2, 256));
+    const bool split = linear_k_chunks(*d, B) > 1;
+    // D1 (and, for a K-split product, the cleared contiguous fp32 accumulator in the workspace)
+    rc = launch_rht_activations(*d, x, B, xdag, split ? y32 : nullptr, split ? (size_t)B * d->N : 0, st);
+    if (rc != HIGGS_OK) return rc;
+    for (int64_t b0 = 0; b0 < B; b0 += 16) {
+        const int64_t bn = B - b0 < 16 ? B - b0 : 16;
+        if (split) {
+            rc = launch_linear_mma(*d, xdag + b0 * d->K, bn, packed, scales, grid, y32 + b0 * d->N, d->N, 2, st);
+        } else {
+            GatherTargets m2 = more;
+            for (int i = 0; i < more.count; ++i) m2.y[i] = static_cast<uint8_t*>(more.y[i]) + (size_t)b0 * ld * esz;
+            rc = launch_linear_mma(*d, xdag + b0 * d->K, bn, packed, scales, grid,
+                                   static_cast<uint8_t*>(dst[0]) + (size_t)b0 * ld * esz, ld, mode, st, nullptr, &m2);
+        }
+        if (rc != HIGGS_OK) return rc;
+    }
+    // a K-split product sums with atomics into its own contiguous buffer; one small kernel spreads the result
+    if (split) return launch_scatter_out(y32, B, d->N, dst, n_dst, ld, y_dtype, st);
+    return HIGGS_OK;
+}
+
 int higgs_linear_prerotated(const higgs_desc* d, const void* xdag, int64_t B, const void* packed, const void* scales,
                             const float* grid, void* y, int y_dtype, void* workspace, size_t workspace_bytes,
                             void* stream) {

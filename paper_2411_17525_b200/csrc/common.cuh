@@ -13,6 +13,7 @@ namespace higgs {
 constexpr int kGroup = 1024;     // the only supported group size g
 constexpr int kRowTile = 16;     // rows of W per mma tile (m16n8k16) and per scale tile
 constexpr int kBlockK = 64;      // k-extent of one 512-byte packed block
+constexpr int kMaxGather = 8;          // destinations of a gathered output (this device's own among them)
 constexpr int kMaxGridDim = 4;        // grid fit and general encoder: 1 <= p <= 4
 constexpr int kMaxGridPoints = 4096;  //                               n <= 4096 (64 KB of fp32 at p = 4)
 
@@ -144,9 +145,18 @@ int launch_pack(const higgs_desc& d, const uint8_t* canonical, void* packed, cud
 int launch_unpack(const higgs_desc& d, const void* packed, uint8_t* canonical, cudaStream_t st);
 int launch_dequantize(const higgs_desc& d, const uint8_t* canonical, const void* scales, const float* grid, void* W_out,
                       int w_dtype, cudaStream_t st);
+// Further destinations of a product's output - the all-gather of a row-sharded layer fused into the epilogue: the same
+// [B][ldy] window in the memory of other devices (peer-mapped pointers), written with plain stores.
+struct GatherTargets {
+    void* y[kMaxGather - 1];
+    int count;
+};
 // x_raw != nullptr: the activations as given (bf16); the kernel rotates them itself (only if linear_fused_eligible)
 int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const void* packed, const void* scales,
-                      const float* grid, void* y, int64_t ldy, int y_mode, cudaStream_t st, const void* x_raw = nullptr);
+                      const float* grid, void* y, int64_t ldy, int y_mode, cudaStream_t st, const void* x_raw = nullptr,
+                      const GatherTargets* more = nullptr);
+int launch_scatter_out(const float* y32, int64_t B, int64_t N, void* const* dsts, int n_dst, int64_t ldy, int y_dtype,
+                       cudaStream_t st);
 bool linear_fused_eligible(const higgs_desc& d, int64_t B);
 int launch_convert_out(const float* y32, void* y, int y_dtype, size_t count, cudaStream_t st);
 size_t make_grid_workspace(int p, int n, int64_t m);
@@ -167,7 +177,8 @@ int tc_batch_tile(int64_t B);
 int tc_k_split(const higgs_desc& d, int64_t B);
 int launch_rht_tc(const higgs_desc& d, const void* x, int64_t B, __half* xdag_tc, cudaStream_t st);
 int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, const void* packed, const void* scales,
-                     const float* grid, void* y, int y_mode, cudaStream_t st);
+                     const float* grid, void* y, int y_mode, cudaStream_t st, int64_t ldy = 0,
+                     const GatherTargets* more = nullptr);
 int read_tc_status(int clear);
 int read_device_status(cudaStream_t st, int clear);
 

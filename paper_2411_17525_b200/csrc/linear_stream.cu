@@ -53,6 +53,8 @@ struct StreamParams {
     const __half* scales;  // tile-major scales [N/16][K/g][16]
     const float* grid;     // [n][p]
     void* y;               // [B][ldy]
+    void* y_more[kMaxGather - 1];   // the same window on other devices (gathered output), n_more of them
+    int n_more;
     int64_t N, K, ldy;
     int chunks;            // K / ck; the grid is chunks x parts blocks
     int B, n, p;
@@ -241,12 +243,26 @@ struct TaskCodes {
     }
 };
 
+// The flusher's stores to the other devices of a gathered output.  Kept out of line: the common case (no gathering)
+// must not pay for it in registers.
+__device__ __noinline__ void gather_store(const StreamParams* prm, int64_t o, float4 sum) {
+    for (int pd = 0; pd < prm->n_more; ++pd) {
+        if (prm->y_mode == 0) {
+            *reinterpret_cast<float4*>(static_cast<float*>(prm->y_more[pd]) + o) = sum;
+        } else {
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(sum.x, sum.y), hi = __floats2bfloat162_rn(sum.z, sum.w);
+            *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(prm->y_more[pd]) + o) =
+                make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+        }
+    }
+}
+
 // FUSED (NB = 1, B <= 2, K not split): the kernel takes the activations as given and rotates them itself (Appendix F's
 // x+ = (H / sqrt(g)) diag(sign) x) - the four warps that own the four 256-input slices of a 1024-group transform it
 // together: butterflies over a lane's 8 values in registers, over the 32 lanes by shuffles, over the 4 warps through
 // shared memory - so that no rotation kernel (and no hand-over between two dependent launches) precedes the product.
 template <int NB, int KS, int FMT, bool FUSED>
-__global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(const StreamParams prm) {
+__global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(const __grid_constant__ StreamParams prm) {
     constexpr bool SIX = FMT == 1, NIB = FMT == 2, B8 = FMT == 3;
     static_assert(!FUSED || (NB == 1 && KS == 256), "the fused rotation maps one warp to one 256-input slice");
     constexpr uint32_t kPieceStride = NIB ? 128u : 256u;     // bytes between consecutive 128-byte pieces of the partial tiles
@@ -586,10 +602,12 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
                     const int64_t o = (int64_t)col * prm.ldy + (int64_t)f_rt * 16 + row;
                     if (prm.y_mode == 0) {
                         *reinterpret_cast<float4*>(static_cast<float*>(prm.y) + o) = sum;
+                        if (prm.n_more) gather_store(&prm, o, sum);   // gathered output: the other devices' copies
                     } else if (prm.y_mode == 1) {
                         __nv_bfloat162 lo = __floats2bfloat162_rn(sum.x, sum.y), hi = __floats2bfloat162_rn(sum.z, sum.w);
                         uint2 pk = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
                         *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(prm.y) + o) = pk;
+                        if (prm.n_more) gather_store(&prm, o, sum);
                     } else {
                         asm volatile("red.global.add.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(static_cast<float*>(prm.y) + o),
                                      "f"(sum.x), "f"(sum.y), "f"(sum.z), "f"(sum.w)
@@ -793,8 +811,10 @@ bool linear_fused_eligible(const higgs_desc& d, int64_t B) {
 
 // y_mode: 0 store fp32, 1 store bf16, 2 atomicAdd fp32 (target must be zero).  B <= 16.
 int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const void* packed, const void* scales,
-                      const float* grid, void* y, int64_t ldy, int y_mode, cudaStream_t st, const void* x_raw) {
+                      const float* grid, void* y, int64_t ldy, int y_mode, cudaStream_t st, const void* x_raw,
+                      const GatherTargets* more) {
     if (d.N == 0) return HIGGS_OK;
+    if (more && more->count > 0 && (y_mode == 2 || more->count > kMaxGather - 1)) return HIGGS_ERR_INVALID_ARG;
     const Plan pl = make_plan(d, B);
     if (pl.items == 0) return HIGGS_ERR_UNSUPPORTED;
     // the kernel's work split is 32-bit arithmetic: (row tiles) x (blocks per K-chunk) must stay below 2^31
@@ -809,6 +829,8 @@ int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const 
     prm.scales = static_cast<const __half*>(scales);
     prm.grid = grid;
     prm.y = y;
+    prm.n_more = more ? more->count : 0;
+    for (int i = 0; i < kMaxGather - 1; ++i) prm.y_more[i] = (more && i < more->count) ? more->y[i] : nullptr;
     prm.N = d.N; prm.K = d.K; prm.ldy = ldy;
     prm.chunks = pl.chunks;
     prm.B = (int)B;
@@ -842,6 +864,40 @@ int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const 
              : b8 ? launch_one<1, 256, 3>(prm, pl.blocks, st) : launch_one<1, 256, 0>(prm, pl.blocks, st);
     return six ? launch_one<2, 128, 1>(prm, pl.blocks, st) : nib ? launch_one<2, 128, 2>(prm, pl.blocks, st)
          : b8 ? launch_one<2, 128, 3>(prm, pl.blocks, st) : launch_one<2, 128, 0>(prm, pl.blocks, st);
+}
+
+// A K-split product accumulates into a contiguous fp32 [B][N]; this spreads it to the gathered destinations.
+struct ScatterDst { void* y[kMaxGather]; int n; };
+__global__ void scatter_out_kernel(const float* __restrict__ src, int64_t B, int64_t N, ScatterDst dst, int64_t ldy, int bf16) {
+    pdl_trigger();
+    pdl_wait();
+    const int64_t quads = N / 4;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < B * quads; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t b = i / quads, c = (i % quads) * 4;
+        const float4 v = *reinterpret_cast<const float4*>(src + b * N + c);
+        for (int pd = 0; pd < dst.n; ++pd) {
+            if (bf16) {
+                const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+                *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(dst.y[pd]) + b * ldy + c) =
+                    make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+            } else {
+                *reinterpret_cast<float4*>(static_cast<float*>(dst.y[pd]) + b * ldy + c) = v;
+            }
+        }
+    }
+}
+
+int launch_scatter_out(const float* y32, int64_t B, int64_t N, void* const* dsts, int n_dst, int64_t ldy, int y_dtype,
+                       cudaStream_t st) {
+    if (n_dst < 1 || n_dst > kMaxGather) return HIGGS_ERR_INVALID_ARG;
+    if (B == 0 || N == 0) return HIGGS_OK;
+    ScatterDst dst;
+    dst.n = n_dst;
+    for (int i = 0; i < kMaxGather; ++i) dst.y[i] = i < n_dst ? dsts[i] : nullptr;
+    int64_t blocks = (B * (N / 4) + 255) / 256;
+    if (blocks > 1184) blocks = 1184;
+    return cuda_status(launch_pdl(scatter_out_kernel, dim3((unsigned)blocks), dim3(256), 0, st, y32, B, N, dst, ldy,
+                                  y_dtype == HIGGS_BF16 ? 1 : 0));
 }
 
 int launch_convert_out(const float* y32, void* y, int y_dtype, size_t count, cudaStream_t st) {

@@ -52,8 +52,10 @@ struct TcParams {
     const __half* scales;    // tile-major scales [N/16][K/g][16]
     const float* grid;       // [n][p]
     const __half* xdag;      // rotated activations, blocked: [batch tile][K/64][BN/8][8 k-cores][8 tokens][8 inputs]
-    void* y;                 // [B][N]
-    int64_t N, K;
+    void* y;                 // [B][ldy]
+    void* y_more[kMaxGather - 1];   // the same window on other devices (gathered output), n_more of them
+    int n_more;
+    int64_t N, K, ldy;
     int B, BN, n, p, y_mode; // y_mode 0: fp32, 1: bf16
     int bits;                // log2(n)
     int ksplit;              // K slices (= cluster size along z); each a multiple of 256 inputs
@@ -539,14 +541,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
                 uint32_t v0, v1, v2, v3;
                 asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3)
                              : "r"(code0 + (uint32_t)((c * 128 + lane * 4) * 4)) : "memory");
-                const int64_t o = (int64_t)b * prm.N + row0 + lane * 4;
+                const int64_t o = (int64_t)b * prm.ldy + row0 + lane * 4;
                 if (prm.y_mode == 0) {
-                    *reinterpret_cast<uint4*>(static_cast<float*>(prm.y) + o) = make_uint4(v0, v1, v2, v3);
+                    const uint4 v = make_uint4(v0, v1, v2, v3);
+                    *reinterpret_cast<uint4*>(static_cast<float*>(prm.y) + o) = v;
+                    for (int pd = 0; pd < prm.n_more; ++pd)       // gathered output: the other devices' copies
+                        *reinterpret_cast<uint4*>(static_cast<float*>(prm.y_more[pd]) + o) = v;
                 } else {
                     const __nv_bfloat162 lo = __floats2bfloat162_rn(__uint_as_float(v0), __uint_as_float(v1));
                     const __nv_bfloat162 hi = __floats2bfloat162_rn(__uint_as_float(v2), __uint_as_float(v3));
-                    *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(prm.y) + o) =
-                        make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+                    const uint2 v = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+                    *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(prm.y) + o) = v;
+                    for (int pd = 0; pd < prm.n_more; ++pd)
+                        *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(prm.y_more[pd]) + o) = v;
                 }
             }
             if (warp == 3) TTRACE(3, 6);
@@ -582,13 +589,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
                 }
                 const int b = bt * BN + c;
                 if (b < prm.B) {
-                    const int64_t o = (int64_t)b * prm.N + row0 + lane * 4;
+                    const int64_t o = (int64_t)b * prm.ldy + row0 + lane * 4;
                     if (prm.y_mode == 0) {
                         *reinterpret_cast<float4*>(static_cast<float*>(prm.y) + o) = acc;
+                        for (int pd = 0; pd < prm.n_more; ++pd)
+                            *reinterpret_cast<float4*>(static_cast<float*>(prm.y_more[pd]) + o) = acc;
                     } else {
                         const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
-                        *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(prm.y) + o) =
-                            make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+                        const uint2 v = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+                        *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(prm.y) + o) = v;
+                        for (int pd = 0; pd < prm.n_more; ++pd)
+                            *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(prm.y_more[pd]) + o) = v;
                     }
                 }
             }
@@ -754,7 +765,8 @@ bool make_code_map(const higgs_desc& d, const void* packed, CUtensorMap* map) {
 
 // D2-D5 on the tensor cores, from activations rotated by launch_rht_tc for the same B.
 int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, const void* packed, const void* scales,
-                     const float* grid, void* y, int y_mode, cudaStream_t st) {
+                     const float* grid, void* y, int y_mode, cudaStream_t st, int64_t ldy, const GatherTargets* more) {
+    if (more && more->count > kMaxGather - 1) return HIGGS_ERR_INVALID_ARG;
     const int BN = tc_batch_tile(B);
     const int64_t tiles = (B + BN - 1) / BN;
     static bool configured[64] = {false};
@@ -776,7 +788,9 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
     prm.grid = grid;
     prm.xdag = xdag_tc;
     prm.y = y;
-    prm.N = d.N; prm.K = d.K;
+    prm.n_more = more ? more->count : 0;
+    for (int i = 0; i < kMaxGather - 1; ++i) prm.y_more[i] = (more && i < more->count) ? more->y[i] : nullptr;
+    prm.N = d.N; prm.K = d.K; prm.ldy = ldy > 0 ? ldy : d.N;
     prm.B = (int)B; prm.BN = BN; prm.n = d.n; prm.p = d.p; prm.y_mode = y_mode;
     prm.bits = code_bits(d.n);
     prm.ksplit = tc_k_split(d, B);

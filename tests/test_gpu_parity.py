@@ -279,6 +279,66 @@ def test_layer_error_matches_oracle(p, n, N, K):
     assert abs(t2 - mse) <= (0.08 if n < 256 or p == 2 else 0.25) * mse, (t2, mse)
 
 
+# ----------------------------------------------------------------------------- row-sharded layer, gathered output
+@pytest.mark.parametrize("p,n,N,K,B,world,dtype", [
+    (2, 256, 512, 2048, 1, 2, torch.float32),       # fused rotation, stores from the flusher warp
+    (2, 256, 384, 2048, 8, 3, torch.float32),       # three uneven shards (128-row units)
+    (2, 256, 256, 8192, 4, 2, torch.float32),       # K split in the small-batch kernel: workspace sum + copy kernel
+    (2, 64, 512, 2048, 16, 2, torch.bfloat16),      # six-bit grid, bf16 output
+    (2, 256, 512, 2048, 40, 2, torch.float32),      # tensor-core kernel, cluster K split
+    (2, 256, 16896, 1024, 24, 2, torch.bfloat16),   # tensor-core kernel without a K split (66 row tiles per shard)
+])
+def test_linear_gather_writes_every_destination(p, n, N, K, B, world, dtype):
+    """A layer split by rows over `world` shards; each shard's product writes its columns into every destination
+    buffer.  One GPU stands in for all devices: the shards' launches run one after the other (they never wait on one
+    another) and the destination buffers are separate allocations of this GPU.  Every destination must hold the whole
+    [B][N] output, equal to the oracle's."""
+    xi = inputs.rht_seed(7)
+    W = inputs.make_weights(N, K, seed=70 + n, bf16=True)
+    x = inputs.make_activations(B, K, seed=71)
+    g64, gt = U.grid32(p, n)
+    q, sc16 = U.oracle_encode(W, G, g64, xi)
+    y_ref = oracle.linear_dense(x.astype(np.float64), q.codes, sc16.astype(np.float64), G, g64, xi)
+    dsts = [torch.full((B, N), float("nan"), dtype=dtype, device=U.dev()) for _ in range(world)]
+    xt = U.bf16_tensor(x)
+    covered = 0
+    for rank in range(world):
+        r0, r1 = hb.shard_rows(N, world, rank)
+        assert r0 == covered and r1 > r0
+        covered = r1
+        d = hb.make_desc(p, n, r1 - r0, K, xi)
+        codes = torch.from_numpy(q.codes[r0:r1].astype(np.uint8)).to(U.dev())
+        packed = hb.higgs_pack_codes(d, codes)
+        scales = hb.scales_to_tile_major(torch.from_numpy(sc16[r0:r1]).to(U.dev()))
+        # "own buffer first, then the peers'": rank r's own buffer is dsts[r]
+        order = [dsts[rank]] + [dsts[o] for o in range(world) if o != rank]
+        hb.higgs_linear_gather(d, xt, packed, scales, gt, order, r0)
+    torch.cuda.synchronize()
+    assert covered == N and hb.higgs_device_status() == hb.HIGGS_OK
+    tol = Y_TOL + (2.0 ** -8 if dtype == torch.bfloat16 else 0.0)
+    for t in dsts:
+        y = t.float().cpu().numpy()
+        assert np.isfinite(y).all()
+        assert U.linear_error(y, y_ref) <= tol
+    for t in dsts[1:]:
+        assert torch.equal(t, dsts[0]) or hb.higgs_linear_k_splits(hb.make_desc(p, n, hb.shard_rows(N, world, 0)[1], K, xi), B) > 1
+
+
+def test_linear_gather_argument_checks():
+    d = hb.make_desc(2, 256, 128, 1024, 1)
+    _, gt = U.grid32(2, 256)
+    x = torch.zeros((1, 1024), dtype=torch.bfloat16, device=U.dev())
+    packed = torch.zeros(hb.higgs_packed_bytes(d), dtype=torch.uint8, device=U.dev())
+    scales = torch.zeros((8, 1, 16), dtype=torch.float16, device=U.dev())
+    y = torch.zeros((1, 256), dtype=torch.float32, device=U.dev())
+    for off in (8, 144, -16):                       # not a row-tile multiple / beyond the row count / negative
+        with pytest.raises(hb.HiggsError) as e:
+            hb.higgs_linear_gather(d, x, packed, scales, gt, [y], off)
+        assert e.value.status == hb.HIGGS_ERR_INVALID_ARG
+    with pytest.raises(hb.HiggsError):
+        hb.higgs_linear_gather(d, x, packed, scales, gt, [y] * 9, 0)
+
+
 # ----------------------------------------------------------------------------- host-buffer entry points
 @pytest.mark.parametrize("B", [1, 4, 40])
 def test_linear_host_and_host_batch_match_device_path(B):

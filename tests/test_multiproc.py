@@ -48,3 +48,69 @@ def test_max_over_ranks_and_aggregate_value():
 def test_single_rank_is_identity():
     assert bench.max_over_ranks(3.5, torch.device("cpu"), 1) == 3.5
     assert abs(bench.aggregate_value(2_000_000, 2, 4.0, 1) - 1.0) < 1e-12
+
+
+# ---- row-sharded layer: the host-side protocol of higgs_linear_gather on two CPU ranks --------------------------------
+def _gather_worker(rank, world, port, out):
+    import numpy as np
+
+    import oracle
+    from paper_2411_17525_b200 import binding
+    from synth import inputs
+    from tests.golden import make_grids
+
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        N, K, B, g, xi = 384, 1024, 3, 1024, 5
+        grid = make_grids.load(2, 64)
+        W = inputs.make_weights(N, K, seed=9, bf16=True).astype(np.float64)      # every rank can draw the full matrix...
+        x = inputs.make_activations(B, K, seed=10).astype(np.float64)
+        r0, r1 = binding.shard_rows(N, world, rank)                               # ...but encodes and multiplies only its rows
+        q = oracle.quantize(W[r0:r1], g, grid, xi)
+        sc = oracle.round_scales_fp16(q.scales).astype(np.float64)
+        y_shard = oracle.linear_dense(x, q.codes, sc, g, grid, xi)              # [B][r1 - r0]
+        # what the fused epilogue does over peer memory: this shard's columns land in every rank's [B][N] buffer
+        spans = [None] * world
+        dist.all_gather_object(spans, (r0, r1))
+        blocks = [None] * world
+        dist.all_gather_object(blocks, y_shard)
+        y = np.full((B, N), np.nan)
+        for (a, b), blk in zip(spans, blocks):
+            y[:, a:b] = blk
+        dist.barrier()                                                            # "all shards written" before any reader
+        q_all = oracle.quantize(W, g, grid, xi)
+        y_ref = oracle.linear_dense(x, q_all.codes, oracle.round_scales_fp16(q_all.scales).astype(np.float64), g, grid, xi)
+        out.put((rank, spans, float(np.max(np.abs(y - y_ref)))))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_row_sharded_layer_protocol_on_two_ranks():
+    """Rows are independent in Algorithm 1 and in the product of Appendix F, so shards encoded and multiplied separately
+    and gathered by column blocks reproduce the unsharded layer exactly; the shard spans tile [0, N) in 128-row units."""
+    world = 2
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_gather_worker, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = sorted(out.get(timeout=300) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, spans, err in res:
+        assert spans == [(0, 256), (256, 384)]          # three 128-row units over two ranks: 2 + 1
+        assert err == 0.0
+
+
+def test_shard_rows_tiles_the_layer():
+    from paper_2411_17525_b200 import binding
+    for N, world in [(4096, 8), (14336, 8), (1024, 3), (128, 2), (8192, 5)]:
+        spans = [binding.shard_rows(N, world, r) for r in range(world)]
+        assert spans[0][0] == 0 and spans[-1][1] == N
+        assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))
+        assert all(s[0] % 128 == 0 and s[1] % 128 == 0 for s in spans)
+        sizes = [s[1] - s[0] for s in spans]
+        assert max(sizes) - min(sizes) <= 128
