@@ -31,6 +31,7 @@ def sampled_rows(N, count, seed):
     ("8b-gate-tensor", 14336, 4096, 2, 256, (64, 256)),   # tensor-core regime, outlier channels (log-normal scales)
     ("8b-down-tensor", 4096, 14336, 2, 256, (64,)),       # K split over a thread-block cluster
     ("8b-gate-2bit", 14336, 4096, 2, 16, (1,)),
+    ("70b-gate-3bit", 28672, 8192, 2, 64, (1, 32)),       # the largest matrix of the benchmark's configurations
 ])
 def test_full_size_layer_on_sampled_rows(name, N, K, p, n, batches):
     cfg = 1
