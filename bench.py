@@ -89,6 +89,25 @@ def measured_peaks():
         return 6650.0, 1590.0, "fallback"
 
 
+# The encoder is bound by instruction issue (profiles/encode_pruned_kernel_...): 3748 warp instructions per
+# (row, group) task of 1024 weights for p=2 n=256 (ncu, smsp__inst_executed.sum / tasks), against a peak of
+# 148 SMs x 4 schedulers x 1 warp instruction per clock at the SM clock.
+ENCODER_WARP_INSTR_PER_WEIGHT = {(2, 256): 3748.0 / 1024.0}
+
+
+def encoder_roofline(weights_per_s, pn, clocks):
+    grids = set(pn)
+    if len(grids) != 1 or next(iter(grids)) not in ENCODER_WARP_INSTR_PER_WEIGHT:
+        return None
+    ipw = ENCODER_WARP_INSTR_PER_WEIGHT[next(iter(grids))]
+    mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
+    peak = 148 * 4 * mhz * 1e6 / 1e9                    # G warp instructions / s
+    achieved = weights_per_s * ipw / 1e9
+    return {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "G warp-instr/s", "frac": achieved / peak,
+            "warp_instr_per_weight": ipw,
+            "note": "whole higgs_quantize calls (search, pack and table build) against the issue rate of 148 SMs x 4 schedulers"}
+
+
 def max_over_ranks(ms: float, device, world: int) -> float:
     """Duration of the timed region as the slowest rank saw it (replicas run independently; no data-path collective)."""
     if world <= 1:
@@ -581,7 +600,8 @@ def run_ours(args):
             "roofline": roofline,
             "cpu_baseline": cpu,
             "quantize": {"weights_per_s": enc_weights / (enc_ms * 1e-3), "ms": enc_ms, "weights": enc_weights,
-                         "grid_fit_ms": grid_ms, "grid_fit_iters": int(grid_iters), "grid_mse": float(grid_mse)},
+                         "grid_fit_ms": grid_ms, "grid_fit_iters": int(grid_iters), "grid_mse": float(grid_mse),
+                         "roofline": encoder_roofline(enc_weights / (enc_ms * 1e-3), pn, clocks)},
             "detail": detail,
         }
         print(json.dumps(line))
