@@ -402,12 +402,12 @@ def run_ours(args):
     ms = timed(run_steps, args.steps, max(args.warmup, 3))
     ms_e2e = timed(run_steps_host, args.steps, max(args.warmup, 3))
     # nvidia-smi samples every 100 ms and the timed regions above last tens of milliseconds: keep the same load running
-    # (untimed) for half a second more so that the clock record has samples taken under it
+    # (untimed) for a second more so that the clock record has samples taken under it
     extra_steps = 0
     if rank == 0:
         t_probe = time.perf_counter()
         with torch.cuda.stream(stream):
-            while time.perf_counter() - t_probe < 0.5:      # small batches: under a profiler every launch is slow
+            while time.perf_counter() - t_probe < 1.0:      # small batches: under a profiler every launch is slow
                 run_steps(extra_steps, 8)               # keeps rotating over the weight copies like the timed steps
                 extra_steps += 8
                 stream.synchronize()
