@@ -114,3 +114,25 @@ def test_shard_rows_tiles_the_layer():
         assert all(s[0] % 128 == 0 and s[1] % 128 == 0 for s in spans)
         sizes = [s[1] - s[0] for s in spans]
         assert max(sizes) - min(sizes) <= 128
+
+
+def test_reference_arm_prints_the_contract_line():
+    """`bench.py --impl reference` (the oracle timed on the host cores) runs without a GPU and prints one JSON line with
+    the keys of the benchmark contract, on the same metric, unit and workload name as the CUDA arm."""
+    import json
+    import subprocess
+    import sys
+
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--impl", "reference", "--steps", "2", "--warmup", "1"],
+                         capture_output=True, text=True, timeout=600, cwd=root)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    for key in ("impl", "metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better", "scaling",
+                "vs_baseline", "dtype", "data", "config", "cpu_baseline", "e2e"):
+        assert key in line, key
+    assert line["impl"] == "reference" and line["metric"] == "higgs_linear_effective_weight_bandwidth" and line["unit"] == "GB/s"
+    assert line["steps"] == 2 and line["value"] > 0 and line["dtype"] == "f64" and line["vs_baseline"] is None
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["value"] == line["value"]
+    assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
+    assert "llama-3.2-1b layer set (7 matrices), grid p=2 n=256, g=1024, batch 1" == line["config"]["workload"]
