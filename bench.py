@@ -306,9 +306,13 @@ def run_ours(args):
     xdags = {k: torch.empty(hb.higgs_rotated_bytes(descs[v[0]], B) // 2, dtype=torch.float16, device=dev)
              for k, v in groups_of.items() if len(v) > 1}
     launches_per_step = 0
+    share_first = True     # the first layer of a group goes through higgs_linear_share
     for k, v in groups_of.items():
-        if len(v) > 1:      # one rotation, then one product launch per layer (per 16 tokens on the small-batch path)
-            launches_per_step += 1 + sum(1 if hb.higgs_rotated_layout(descs[li], B) > 0 else -(-B // 16) for li in v)
+        if len(v) > 1:      # one rotation, then one product launch per layer (per 16 tokens on the small-batch path);
+                            # for 1-2 tokens the first product rotates x itself and leaves the result for the others
+            first_is_one_launch = share_first and hb.higgs_linear_launch_count(descs[v[0]], B) == 1
+            launches_per_step += (0 if first_is_one_launch else 1) + \
+                sum(1 if hb.higgs_rotated_layout(descs[li], B) > 0 else -(-B // 16) for li in v)
         else:
             launches_per_step += hb.higgs_linear_launch_count(descs[v[0]], B)
 
@@ -316,8 +320,15 @@ def run_ours(args):
         c = i % copies
         for key, lis in groups_of.items():
             if len(lis) > 1:
-                hb.higgs_rotate_activations(descs[lis[0]], xs[lis[0]], out=xdags[key])
-                for li in lis:
+                rest = lis
+                if share_first:       # the first layer of the group also produces the rotated activations of the others
+                    li = lis[0]
+                    hb.higgs_linear_share(descs[li], xs[li], packed[li][c], scales[li][c], grids[pn[li]], xdag_out=xdags[key],
+                                          workspace=ws[li], y=ys[li])
+                    rest = lis[1:]
+                else:
+                    hb.higgs_rotate_activations(descs[lis[0]], xs[lis[0]], out=xdags[key])
+                for li in rest:
                     hb.higgs_linear_prerotated(descs[li], xdags[key], packed[li][c], scales[li][c], grids[pn[li]], workspace=ws[li],
                                                y=ys[li], B=B)
             else:
@@ -590,7 +601,7 @@ def run_ours(args):
                        "l2": f"rotating {copies} weight copies ({copies * set_bytes / 1e6:.0f} MB > 126 MB L2)",
                        "launch": "direct" if graphs is None else (f"CUDA graphs of {spg} consecutive steps (rotating weight copies), remainder from one-step graphs"
                                                                   if graphs_multi is not None else "one CUDA graph per step"),
-                       "step": "one transformer block: activation rotations (q/k/v and gate/up share theirs where the layout allows; a layer with its own rotation has it fused into the product kernel for 1-2 tokens when K is not split) + 7 products"},
+                       "step": "one transformer block: activation rotations (q/k/v and gate/up share theirs where the layout allows: the first layer of the group goes through higgs_linear_share, which for 1-2 tokens rotates inside its product kernel and leaves the result for the others; a layer with its own rotation has it fused likewise when K is not split) + 7 products"},
             "us_per_layer": ms_per_step * 1e3 / len(layers),
             "weight_bytes_per_step": set_bytes,
             "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

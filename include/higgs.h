@@ -205,6 +205,19 @@ int higgs_linear_prerotated(const higgs_desc* desc, const void* xdag, int64_t B,
                             void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * higgs_linear that also leaves the rotated activations behind, for the first of several layers that read the same
+ * x (q before k and v; gate before up): y as higgs_linear, and xdag_out (device, higgs_rotated_bytes(desc, B) bytes,
+ * 16-byte aligned) receives what higgs_rotate_activations(desc, x, B) writes, to be passed to
+ * higgs_linear_prerotated for the other layers (same K, seed and higgs_rotated_layout).  For one or two tokens on a
+ * layer whose K is not split this is ONE launch - the product kernel rotates x itself and one of its blocks stores
+ * the result - instead of a rotation launch followed by a product launch; otherwise it is those two launches.
+ * xdag_out is complete when the call's last kernel has completed (stream order).
+ */
+int higgs_linear_share(const higgs_desc* desc, const void* x, int64_t B, const void* packed, const void* scales,
+                       const float* grid, void* y, int y_dtype, void* xdag_out, void* workspace,
+                       size_t workspace_bytes, void* stream);
+
+/*
  * Row-sharded layer with the all-gather fused into the product's epilogue (Appendix F's product is independent per
  * output row, and the rotation is local to a 1024-group of inputs, so a layer splits over devices by rows with no
  * exchange of weights): this device holds rows [row_offset, row_offset + desc->N) of a layer with `ld` rows in all

@@ -27,7 +27,7 @@ EXPORTS = [
     "higgs_linear_static", "higgs_linear_static_capacity", "higgs_linear_k_splits", "higgs_rotated_bytes",
     "higgs_rotated_layout", "higgs_dequantize", "higgs_make_uniform_grid", "higgs_layer_error",
     "higgs_allocate_bits", "higgs_general_tuples", "higgs_quantize_general", "higgs_linear_host_batch",
-    "higgs_linear_gather",
+    "higgs_linear_gather", "higgs_linear_share",
 ]
 
 
@@ -72,6 +72,8 @@ def _load() -> ctypes.CDLL:
     lib.higgs_linear_prerotated.argtypes = [P, vp, i64, vp, vp, vp, vp, i32, vp, sz, vp]
     lib.higgs_linear_host.restype = i32
     lib.higgs_linear_host.argtypes = [P, vp, i64, vp, vp, vp, vp, i32, vp, sz, vp]
+    lib.higgs_linear_share.restype = i32
+    lib.higgs_linear_share.argtypes = [P, vp, i64, vp, vp, vp, vp, i32, vp, vp, sz, vp]
     lib.higgs_linear_gather.restype = i32
     lib.higgs_linear_gather.argtypes = [P, vp, i64, vp, vp, vp, vp, i32, i64, i64, i32, vp, sz, vp]
     lib.higgs_linear_host_batch.restype = i32
@@ -208,6 +210,26 @@ def higgs_linear(desc: higgs_desc, x: torch.Tensor, packed: torch.Tensor, scales
     _check(lib.higgs_linear(ctypes.byref(desc), _ptr(x), B, _ptr(packed), _ptr(scales), _ptr(grid), _ptr(y),
                             _dtype_code(y), _ptr(workspace), workspace.numel(), _stream()), "higgs_linear")
     return y
+
+
+def higgs_linear_share(desc: higgs_desc, x: torch.Tensor, packed: torch.Tensor, scales: torch.Tensor, grid: torch.Tensor,
+                       xdag_out: Optional[torch.Tensor] = None, out_dtype: torch.dtype = torch.float32,
+                       workspace: Optional[torch.Tensor] = None, y: Optional[torch.Tensor] = None):
+    """higgs_linear that also leaves the rotated activations in xdag_out for the other layers reading the same x
+    (pass it to higgs_linear_prerotated).  Returns (y, xdag_out)."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous()
+    B = x.shape[0]
+    if y is None:
+        y = torch.empty((B, desc.N), dtype=out_dtype, device=x.device)
+    if xdag_out is None:
+        nb = higgs_rotated_bytes(desc, B)
+        xdag_out = torch.empty(x.shape if nb == x.numel() * 2 else (nb // 2,), dtype=torch.float16, device=x.device)
+    if workspace is None:
+        workspace = _workspace(higgs_workspace_bytes(desc, HIGGS_OP_LINEAR, B), x.device)
+    _check(lib.higgs_linear_share(ctypes.byref(desc), _ptr(x), B, _ptr(packed), _ptr(scales), _ptr(grid), _ptr(y),
+                                  _dtype_code(y), _ptr(xdag_out), _ptr(workspace), workspace.numel(), _stream()),
+           "higgs_linear_share")
+    return y, xdag_out
 
 
 def higgs_rotate_activations(desc: higgs_desc, x: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:

@@ -241,6 +241,22 @@ int higgs_linear(const higgs_desc* d, const void* x, int64_t B, const void* pack
     return linear_tail(d, xdag, B, packed, scales, grid, y, y_dtype, y32, true, st);
 }
 
+int higgs_linear_share(const higgs_desc* d, const void* x, int64_t B, const void* packed, const void* scales,
+                       const float* grid, void* y, int y_dtype, void* xdag_out, void* workspace, size_t workspace_bytes,
+                       void* stream) {
+    int rc = linear_args(d, B, x, packed, scales, grid, y, y_dtype, workspace, workspace_bytes);
+    if (rc != HIGGS_OK) return rc < 0 ? HIGGS_OK : rc;
+    if (!xdag_out || !aligned(xdag_out, 16)) return HIGGS_ERR_INVALID_ARG;
+    cudaStream_t st = as_stream(stream);
+    if (!tc_eligible(*d, B) && linear_fused_eligible(*d, B))
+        // one launch: the product kernel rotates x itself and its first block leaves x+ behind for the other layers
+        return launch_linear_mma(*d, nullptr, B, packed, scales, grid, y, d->N, y_dtype == HIGGS_F32 ? 0 : 1, st, x, nullptr,
+                                 static_cast<__half*>(xdag_out));
+    rc = higgs_rotate_activations(d, x, B, xdag_out, stream);
+    if (rc != HIGGS_OK) return rc;
+    return higgs_linear_prerotated(d, xdag_out, B, packed, scales, grid, y, y_dtype, workspace, workspace_bytes, stream);
+}
+
 int higgs_linear_gather(const higgs_desc* d, const void* x, int64_t B, const void* packed, const void* scales,
                         const float* grid, void* const* y_dsts, int32_t n_dst, int64_t ld, int64_t row_offset, int y_dtype,
                         void* workspace, size_t workspace_bytes, void* stream) {

@@ -49,6 +49,7 @@ struct StreamParams {
     const __nv_bfloat16* x;   // fused-rotation kernels only: [B][K] activations as the caller gave them
     unsigned long long xi;    // ... and the seed of the sign sequence
     const __half* xdag;    // [B][K] rotated activations, fp16
+    __half* xdag_emit;     // fused-rotation kernels only, optional: block 0 also writes the rotated activations here
     const uint8_t* packed; // packed code stream
     const __half* scales;  // tile-major scales [N/16][K/g][16]
     const float* grid;     // [n][p]
@@ -517,6 +518,17 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
             }
         }
         __syncwarp();
+        // Other layers that read the same x (k and v after q, up after gate) can skip their rotation: one warp per slice
+        // of block 0 leaves the slice, already in the rotation kernel's fragment order, in global memory.
+        if (prm.xdag_emit != nullptr && blockIdx.x == 0 && warp < NS) {
+#pragma unroll
+            for (int b = 0; b < 2; ++b) {
+                if (b < prm.B) {
+                    const uint4 v = lds128(scratch((uint32_t)(16384 + (warp * 2 + b) * 512 + lane * 16)));
+                    *reinterpret_cast<uint4*>(prm.xdag_emit + (int64_t)b * prm.K + kbase + lane * 8) = v;
+                }
+            }
+        }
 #pragma unroll
         for (int jb = 0; jb < KS / 64; ++jb) {
             uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = make_uint4(0u, 0u, 0u, 0u);
@@ -812,7 +824,7 @@ bool linear_fused_eligible(const higgs_desc& d, int64_t B) {
 // y_mode: 0 store fp32, 1 store bf16, 2 atomicAdd fp32 (target must be zero).  B <= 16.
 int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const void* packed, const void* scales,
                       const float* grid, void* y, int64_t ldy, int y_mode, cudaStream_t st, const void* x_raw,
-                      const GatherTargets* more) {
+                      const GatherTargets* more, __half* xdag_emit) {
     if (d.N == 0) return HIGGS_OK;
     if (more && more->count > 0 && (y_mode == 2 || more->count > kMaxGather - 1)) return HIGGS_ERR_INVALID_ARG;
     const Plan pl = make_plan(d, B);
@@ -825,6 +837,7 @@ int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const 
     prm.x = static_cast<const __nv_bfloat16*>(x_raw);
     prm.xi = d.rht_seed;
     prm.xdag = xdag;
+    prm.xdag_emit = fused ? xdag_emit : nullptr;
     prm.packed = static_cast<const uint8_t*>(packed);
     prm.scales = static_cast<const __half*>(scales);
     prm.grid = grid;

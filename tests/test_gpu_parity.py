@@ -279,6 +279,41 @@ def test_layer_error_matches_oracle(p, n, N, K):
     assert abs(t2 - mse) <= (0.08 if n < 256 or p == 2 else 0.25) * mse, (t2, mse)
 
 
+# ----------------------------------------------------------------------------- shared rotation from the first layer
+@pytest.mark.parametrize("N,K,B", [(512, 2048, 1), (256, 4096, 2), (128, 1024, 1), (256, 8192, 1), (256, 2048, 8), (256, 2048, 40)])
+def test_linear_share_leaves_the_rotated_activations(N, K, B):
+    """higgs_linear_share: y equals higgs_linear's, and the rotated activations it leaves behind equal what
+    higgs_rotate_activations writes, bit for bit - whether the product kernel emitted them (1-2 tokens, K not split) or a
+    rotation kernel did."""
+    xi = inputs.rht_seed(8)
+    p, n = 2, 256
+    d = hb.make_desc(p, n, N, K, xi)
+    _, gt = U.grid32(p, n)
+    W = inputs.make_weights(N, K, seed=81, bf16=True)
+    packed, scales, _ = hb.higgs_quantize(d, U.bf16_tensor(W), gt)
+    x = U.bf16_tensor(inputs.make_activations(B, K, seed=82))
+    y_ref = hb.higgs_linear(d, x, packed, scales, gt)
+    xd_ref = hb.higgs_rotate_activations(d, x)
+    xd = torch.full_like(xd_ref, float("nan"))
+    y, xd = hb.higgs_linear_share(d, x, packed, scales, gt, xdag_out=xd)
+    torch.cuda.synchronize()
+    assert hb.higgs_device_status() == hb.HIGGS_OK
+    if hb.higgs_rotated_layout(d, B) == 0:            # (the blocked tensor-core layout has padding tokens nobody writes)
+        assert torch.equal(xd.view(torch.int16), xd_ref.view(torch.int16))
+    if hb.higgs_linear_k_splits(d, B) == 1 or hb.higgs_rotated_layout(d, B) > 0:
+        assert torch.equal(y, y_ref)
+    else:
+        assert U.linear_error(y.cpu().numpy(), y_ref.cpu().numpy().astype(np.float64)) <= 1e-5
+    # and a second layer on the shared activations
+    d2 = hb.make_desc(p, n, 128, K, xi)
+    W2 = inputs.make_weights(128, K, seed=83, bf16=True)
+    pk2, sc2, _ = hb.higgs_quantize(d2, U.bf16_tensor(W2), gt)
+    if hb.higgs_rotated_layout(d2, B) == hb.higgs_rotated_layout(d, B):
+        y2 = hb.higgs_linear_prerotated(d2, xd, pk2, sc2, gt, B=B)
+        y2_ref = hb.higgs_linear(d2, x, pk2, sc2, gt)
+        assert U.linear_error(y2.cpu().numpy(), y2_ref.cpu().numpy().astype(np.float64)) <= 1e-5
+
+
 # ----------------------------------------------------------------------------- row-sharded layer, gathered output
 @pytest.mark.parametrize("p,n,N,K,B,world,dtype", [
     (2, 256, 512, 2048, 1, 2, torch.float32),       # fused rotation, stores from the flusher warp
