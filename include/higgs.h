@@ -206,7 +206,8 @@ int higgs_linear_prerotated(const higgs_desc* desc, const void* xdag, int64_t B,
 
 /*
  * higgs_linear that also leaves the rotated activations behind, for the first of several layers that read the same
- * x (q before k and v; gate before up): y as higgs_linear, and xdag_out (device, higgs_rotated_bytes(desc, B) bytes,
+ * x (q before k and v; gate before up) - Section 4.3 notes that the transform of the activations can be isolated from
+ * the product of Appendix F, so layers with a common input need it once: y as higgs_linear, and xdag_out (device, higgs_rotated_bytes(desc, B) bytes,
  * 16-byte aligned) receives what higgs_rotate_activations(desc, x, B) writes, to be passed to
  * higgs_linear_prerotated for the other layers (same K, seed and higgs_rotated_layout).  For one or two tokens on a
  * layer whose K is not split this is ONE launch - the product kernel rotates x itself and one of its blocks stores
@@ -251,7 +252,8 @@ int higgs_linear_host(const higgs_desc* desc, const void* x_host, int64_t B,
 size_t higgs_linear_host_workspace_bytes(const higgs_desc* desc, int64_t B, int y_dtype);
 
 /*
- * `count` higgs_linear_host calls enqueued by ONE call - the products of a transformer block, say - so that the
+ * `count` higgs_linear_host calls (each the rotated-space product of Appendix F from host activations to a host
+ * output) enqueued by ONE call - the products of a transformer block, say - so that the
  * host spends one library call, not `count`, per step.  Argument i of every array belongs to layer i
  * (descs[i], x_hosts[i], packed[i], scales[i], grids[i], y_hosts[i], workspaces[i], workspace_bytes[i]); B and
  * y_dtype are common.  Layers that name the SAME x_hosts pointer and have the same K (q/k/v; gate/up) share one
