@@ -445,7 +445,7 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     const int64_t kbase = (int64_t)chunk_begin * prm.ck + (int64_t)slice * KS;
     if (!FUSED) {
         if (n_tasks > 0) load_bfrag(chunk_begin);
-    } else if (!flusher) {
+    } else if (!flusher && warp < NS) {
 #pragma unroll
         for (int b = 0; b < 2; ++b)
             if (b < prm.B) xraw[b] = *reinterpret_cast<const uint4*>(prm.x + (int64_t)b * prm.K + kbase + lane * 8);
@@ -454,10 +454,12 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     TRACEP(warp, 2);
     for (; issued < n_tasks && issued < D; ++issued) issue(issued);
     TRACEP(warp, 3);
-    if (FUSED && !flusher) {
+    auto scratch = [&](uint32_t off) { return part0 + (off >> 7) * kPieceStride + (off & 127u); };
+    // (when K < 4096 several units own the same 1024-group: only the first of them transforms it - every warp of the
+    // block would otherwise spend the same issue slots on the same butterflies - and the others read the result)
+    if (FUSED && !flusher && warp < NS) {
         // Scratch in the (still unused) partial-tile area, addressed in 128-byte pieces: bytes [0, 16 KB) exchange
         // buffers of the four warp units, then 512 bytes per (warp, token) for the slice in fragment order.
-        auto scratch = [&](uint32_t off) { return part0 + (off >> 7) * kPieceStride + (off & 127u); };
         const int unit = warp >> 2, quarter = warp & 3;       // the unit's four warps hold the four slices of one group
 #pragma unroll
         for (int b = 0; b < 2; ++b) {
@@ -520,7 +522,7 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
         __syncwarp();
         // Other layers that read the same x (k and v after q, up after gate) can skip their rotation: one warp per slice
         // of block 0 leaves the slice, already in the rotation kernel's fragment order, in global memory.
-        if (prm.xdag_emit != nullptr && blockIdx.x == 0 && warp < NS) {
+        if (prm.xdag_emit != nullptr && blockIdx.x == 0) {
 #pragma unroll
             for (int b = 0; b < 2; ++b) {
                 if (b < prm.B) {
@@ -528,19 +530,6 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
                     *reinterpret_cast<uint4*>(prm.xdag_emit + (int64_t)b * prm.K + kbase + lane * 8) = v;
                 }
             }
-        }
-#pragma unroll
-        for (int jb = 0; jb < KS / 64; ++jb) {
-            uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = make_uint4(0u, 0u, 0u, 0u);
-            if (g < prm.B) {
-                const uint32_t a = (uint32_t)(16384 + (warp * 2 + g) * 512 + jb * 128 + t * 32);
-                lo = lds128(scratch(a));
-                hi = lds128(scratch(a + 16));
-            }
-            bfrag[jb * 4 + 0][0][0] = lo.x; bfrag[jb * 4 + 0][0][1] = lo.y;
-            bfrag[jb * 4 + 1][0][0] = lo.z; bfrag[jb * 4 + 1][0][1] = lo.w;
-            bfrag[jb * 4 + 2][0][0] = hi.x; bfrag[jb * 4 + 2][0][1] = hi.y;
-            bfrag[jb * 4 + 3][0][0] = hi.z; bfrag[jb * 4 + 3][0][1] = hi.w;
         }
     }
 
@@ -563,7 +552,25 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     }
     TRACEP(warp, 5);
     if (n_tasks > 0 && bfrag[0][0][0] != 0x12345678u) TRACEP(warp, 7);
-    __syncthreads();     // table and barriers visible to every warp
+    __syncthreads();     // table and barriers visible to every warp (fused rotation: also the rotated slices)
+    if (FUSED) {
+        if (!flusher) {
+#pragma unroll
+            for (int jb = 0; jb < KS / 64; ++jb) {
+                uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = make_uint4(0u, 0u, 0u, 0u);
+                if (g < prm.B) {
+                    const uint32_t a = (uint32_t)(16384 + (slice * 2 + g) * 512 + jb * 128 + t * 32);
+                    lo = lds128(scratch(a));
+                    hi = lds128(scratch(a + 16));
+                }
+                bfrag[jb * 4 + 0][0][0] = lo.x; bfrag[jb * 4 + 0][0][1] = lo.y;
+                bfrag[jb * 4 + 1][0][0] = lo.z; bfrag[jb * 4 + 1][0][1] = lo.w;
+                bfrag[jb * 4 + 2][0][0] = hi.x; bfrag[jb * 4 + 2][0][1] = hi.y;
+                bfrag[jb * 4 + 3][0][0] = hi.z; bfrag[jb * 4 + 3][0][1] = hi.w;
+            }
+        }
+        __syncthreads();     // every warp has its B fragments: the scratch area may now take partial tiles
+    }
     if (warp == 0) BTRACE(2);
     TRACE(warp, 2);
     TRACEP(warp, 8);
