@@ -485,25 +485,29 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
             }
 #pragma unroll
             for (int m = 1; m < 32; m <<= 1) {
-                const bool upper = (lane & m) != 0;
+                const float sg = (lane & m) != 0 ? -1.f : 1.f;       // upper lane of a pair: other - own (one rounding either way)
 #pragma unroll
                 for (int r = 0; r < 8; ++r) {
                     const float o = __shfl_xor_sync(0xffffffffu, v[r], m);
-                    v[r] = upper ? (o - v[r]) : (v[r] + o);
+                    v[r] = fmaf(sg, v[r], o);
                 }
             }
-            // the last two stages run over the unit's four warps
-            const uint32_t ex = (uint32_t)(unit * 4096 + lane * 32);
-            asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(scratch(ex + quarter * 1024)), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]) : "memory");
-            asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(scratch(ex + quarter * 1024 + 16)), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]) : "memory");
+            // the last two stages run over the unit's four warps: exchange buffer of the unit at scratch bytes
+            // [4096 unit, + 4096), 32 bytes per lane and quarter (byte 4096 unit + 1024 quarter + 32 lane), i.e. piece
+            // 32 unit + 8 quarter + lane / 4, offset 32 (lane % 4)
+            const uint32_t ex0 = part0 + (uint32_t)(unit * 32 + (lane >> 2)) * kPieceStride + (uint32_t)((lane & 3) * 32);
+            const uint32_t exq = ex0 + (uint32_t)quarter * 8u * kPieceStride;
+            asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(exq), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]) : "memory");
+            asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(exq + 16u), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]) : "memory");
             asm volatile("bar.sync %0, 128;" ::"r"(1 + unit) : "memory");
             float o[8];
 #pragma unroll
             for (int r = 0; r < 8; ++r) o[r] = 0.f;
 #pragma unroll
             for (int qq = 0; qq < 4; ++qq) {
-                const uint4 u0 = lds128(scratch(ex + qq * 1024)), u1 = lds128(scratch(ex + qq * 1024 + 16));
-                const float sgn = (__popc(quarter & qq) & 1) ? -1.f : 1.f;
+                const uint4 u0 = lds128(ex0 + (uint32_t)qq * 8u * kPieceStride), u1 = lds128(ex0 + (uint32_t)qq * 8u * kPieceStride + 16u);
+                // the orthonormal transform's 1/32 rides on the sign (a power of two: the sums are the same, scaled)
+                const float sgn = (__popc(quarter & qq) & 1) ? -0.03125f : 0.03125f;
                 o[0] = fmaf(sgn, __uint_as_float(u0.x), o[0]); o[1] = fmaf(sgn, __uint_as_float(u0.y), o[1]);
                 o[2] = fmaf(sgn, __uint_as_float(u0.z), o[2]); o[3] = fmaf(sgn, __uint_as_float(u0.w), o[3]);
                 o[4] = fmaf(sgn, __uint_as_float(u1.x), o[4]); o[5] = fmaf(sgn, __uint_as_float(u1.y), o[5]);
@@ -512,11 +516,12 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
             asm volatile("bar.sync %0, 128;" ::"r"(1 + unit) : "memory");      // the exchange buffer is reused by the next token
             // this lane holds inputs 8 lane .. + 7 of the slice: pairs 4 j + i (j = lane & 7) of 64-input block lane >> 3
             // -> fragment-order position i * 8 + j
-            const uint32_t st = (uint32_t)(16384 + (warp * 2 + b) * 512 + (lane >> 3) * 128 + (lane & 7) * 4);
+            // (scratch byte 16384 + 512 (2 warp + b) + 128 (lane / 8) + 4 (lane % 8) + 32 i: piece 128 + 4 (2 warp + b) + lane / 8)
+            const uint32_t st = part0 + (uint32_t)(128 + (warp * 2 + b) * 4 + (lane >> 3)) * kPieceStride + (uint32_t)((lane & 7) * 4);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const __half2 hh = __floats2half2_rn(o[2 * i] * 0.03125f, o[2 * i + 1] * 0.03125f);
-                asm volatile("st.shared.b32 [%0], %1;" ::"r"(scratch(st + i * 32)), "r"(*reinterpret_cast<const uint32_t*>(&hh)) : "memory");
+                const __half2 hh = __floats2half2_rn(o[2 * i], o[2 * i + 1]);
+                asm volatile("st.shared.b32 [%0], %1;" ::"r"(st + (uint32_t)(i * 32)), "r"(*reinterpret_cast<const uint32_t*>(&hh)) : "memory");
             }
         }
         __syncwarp();
