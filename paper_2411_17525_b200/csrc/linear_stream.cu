@@ -27,22 +27,6 @@ namespace higgs {
 
 __device__ int g_device_status = 0;
 
-// Optional timeline tracing of one block (build with -DHIGGS_TRACE): SM cycle stamps per warp and event.
-#ifdef HIGGS_TRACE
-__device__ long long g_trace[17][64];
-__device__ __forceinline__ long long trace_now() { return clock64(); }   // SM cycles (cheap); one block only, so one clock domain
-__device__ long long g_trace_pro[17][16];
-__device__ unsigned long long g_stream_blocks[4][256];
-__device__ __forceinline__ unsigned long long gtime_ns() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define BTRACE(row_) do { if ((threadIdx.x & 31) == 0 && blockIdx.x < 256) g_stream_blocks[row_][blockIdx.x] = gtime_ns(); } while (0)
-#define TRACEP(warp_, slot_) do { if (blockIdx.x == 7 && (threadIdx.x & 31) == 0) g_trace_pro[warp_][slot_] = trace_now(); } while (0)
-#define TRACE(warp_, slot_) do { if (blockIdx.x == 7 && (threadIdx.x & 31) == 0 && (slot_) < 64) g_trace[warp_][slot_] = trace_now(); } while (0)
-#else
-#define TRACE(warp_, slot_) do { } while (0)
-#define TRACEP(warp_, slot_) do { } while (0)
-#define BTRACE(row_) do { } while (0)
-#endif
-
 namespace {
 
 struct StreamParams {
@@ -258,6 +242,13 @@ __device__ __noinline__ void gather_store(const StreamParams* prm, int64_t o, fl
     }
 }
 
+__device__ __noinline__ void gather_store1(const StreamParams* prm, int64_t o, float sum) {
+    for (int pd = 0; pd < prm->n_more; ++pd) {
+        if (prm->y_mode == 0) static_cast<float*>(prm->y_more[pd])[o] = sum;
+        else static_cast<__nv_bfloat16*>(prm->y_more[pd])[o] = __float2bfloat16_rn(sum);
+    }
+}
+
 // FUSED (NB = 1, B <= 2, K not split): the kernel takes the activations as given and rotates them itself (Appendix F's
 // x+ = (H / sqrt(g)) diag(sign) x) - the four warps that own the four 256-input slices of a 1024-group transform it
 // together: butterflies over a lane's 8 values in registers, over the 32 lanes by shuffles, over the 4 warps through
@@ -272,8 +263,6 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     const int g = lane >> 2, t = lane & 3;
     using Codes = TaskCodes<KS, FMT>;
 
-    TRACEP(warp, 0);
-    if (warp == 0) BTRACE(0);
     // ---- the table's source first: the grid loads are in flight while everything below is set up ----
     // Table: entry(idx) replicated once per lane (bank = lane): conflict-free gathers.  Warp w fills rows
     // 4 (w + 17 r) .. + 3; a row's 128 bytes are written by eight lanes with one 16-byte store each, and the loads
@@ -367,7 +356,6 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     const uint32_t q_stride = tile_stride << log_ns;                   // bytes between consecutive item slots
 
     // ---- ring barriers, then the first copies ----
-    TRACEP(warp, 1);
     if (lane == 0 && !flusher) {
         for (int d = 0; d < kMaxDepth; ++d) mbar_init(full_bar(d), 1);
     }
@@ -405,14 +393,10 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     // the weight stream depends on nothing this kernel computes: start it before anything else
     // (every lane runs the loop so that addresses stay warp-uniform - bulk copies take uniform operands - and one
     // elected lane issues)
-    TRACE(warp, 0);
     pdl_trigger();
     // Everything above depends only on the weights.  The activations (and y, which the previous kernel in the
     // stream may still be reading or clearing) are touched only after the previous kernel has completed.
     pdl_wait();
-    TRACE(warp, 1);
-    TRACEP(warp, 6);
-    if (warp == 0) BTRACE(1);
 
     // B fragments of this warp's K-slice (global loads; their latency overlaps the table build below)
     uint32_t bfrag[KS / 16][NB][2];
@@ -451,9 +435,7 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
             if (b < prm.B) xraw[b] = *reinterpret_cast<const uint4*>(prm.x + (int64_t)b * prm.K + kbase + lane * 8);
     }
     int issued = 0;
-    TRACEP(warp, 2);
     for (; issued < n_tasks && issued < D; ++issued) issue(issued);
-    TRACEP(warp, 3);
     auto scratch = [&](uint32_t off) { return part0 + (off >> 7) * kPieceStride + (off & 127u); };
     // (when K < 4096 several units own the same 1024-group: only the first of them transforms it - every warp of the
     // block would otherwise spend the same issue slots on the same butterflies - and the others read the result)
@@ -555,8 +537,6 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
             }
         }
     }
-    TRACEP(warp, 5);
-    if (n_tasks > 0 && bfrag[0][0][0] != 0x12345678u) TRACEP(warp, 7);
     __syncthreads();     // table and barriers visible to every warp (fused rotation: also the rotated slices)
     if (FUSED) {
         if (!flusher) {
@@ -576,17 +556,44 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
         }
         __syncthreads();     // every warp has its B fragments: the scratch area may now take partial tiles
     }
-    if (warp == 0) BTRACE(2);
-    TRACE(warp, 2);
-    TRACEP(warp, 8);
     // ---- flusher warp: one item after the other, in item order ----
     if (flusher) {
-        int f_chunk = chunk_begin, f_rt = rt_begin;
-        (void)f_chunk;
+        int f_rt = rt_begin;
         for (int j = 0; j < n_items; ++j) {
             const int q = j & (acc_slots - 1), gen = j >> acc_shift;
             if (!mbar_wait_relaxed(item_bars + 8u * q, (uint32_t)(gen & 1), abort_flag)) return;
-            TRACE(16, 4 + 2 * j);
+            if (prm.B <= 2) {
+                // one or two tokens: a tile is one 128-byte piece and lane = column * 16 + row owns one output: the NS
+                // partial values of its element are summed in slice order
+                const uint32_t a0 = part0 + (uint32_t)q * q_stride + (uint32_t)(lane * 4);
+                float part[16];
+#pragma unroll
+                for (int ns = 0; ns < 16; ++ns) {
+                    uint32_t v;
+                    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(a0 + (uint32_t)(ns < NS ? ns : 0) * tile_stride));
+                    part[ns] = __uint_as_float(v);
+                }
+                float sum = 0.f;
+#pragma unroll
+                for (int ns = 0; ns < 16; ++ns) sum += ns < NS ? part[ns] : 0.f;
+                __syncwarp();
+                if (lane == 0) recycled[q] = gen + 1;
+                const int col = lane >> 4, row = lane & 15;
+                if (col < prm.B) {
+                    const int64_t o = (int64_t)col * prm.ldy + (int64_t)f_rt * 16 + row;
+                    if (prm.y_mode == 0) {
+                        static_cast<float*>(prm.y)[o] = sum;
+                        if (prm.n_more) gather_store1(&prm, o, sum);
+                    } else if (prm.y_mode == 1) {
+                        static_cast<__nv_bfloat16*>(prm.y)[o] = __float2bfloat16_rn(sum);
+                        if (prm.n_more) gather_store1(&prm, o, sum);
+                    } else {
+                        asm volatile("red.global.add.f32 [%0], %1;" ::"l"(static_cast<float*>(prm.y) + o), "f"(sum) : "memory");
+                    }
+                }
+                ++f_rt;
+                continue;
+            }
             float4 sums[NB];
 #pragma unroll
             for (int qq = 0; qq < NB; ++qq) {
@@ -613,10 +620,8 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
             }
             // The partial tiles are in registers (the sums above consumed every load): hand the slot back first,
             // then write y.  No fence follows the global write, so the warp never waits for its round trip.
-            if (sums[0].x != 1.2345e-30f) TRACE(16, 30 + 3 * j);
             __syncwarp();
             if (lane == 0) recycled[q] = gen + 1;
-            TRACE(16, 31 + 3 * j);
 #pragma unroll
             for (int qq = 0; qq < NB; ++qq) {
                 const int e = (qq * 32 + lane) * 4;
@@ -639,10 +644,8 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
                     }
                 }
             }
-            TRACE(16, 5 + 2 * j);
-            if (++f_rt == (int)tiles) { f_rt = 0; ++f_chunk; }
+            ++f_rt;
         }
-        BTRACE(3);
         return;
     }
 
@@ -654,9 +657,7 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     bool ok = true;
     int done = 0;                                // tasks whose slot has been consumed
     for (int i = 0; i < n_tasks; ++i) {
-        TRACE(warp, 4 + 3 * i);
         if (!mbar_wait(full_bar(d), ph, abort_flag)) { ok = false; break; }
-        TRACE(warp, 5 + 3 * i);
         const uint32_t slot = slot_addr(d);
         Codes codes;
         codes.load(slot, lane);
@@ -739,7 +740,6 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
             }
         }
         __syncwarp();
-        TRACE(warp, 6 + 3 * i);
         if (lane == 0) {                         // release: the partial tile is visible before the arrival counts
             asm volatile("{ .reg .b64 st; mbarrier.arrive.shared::cta.b64 st, [%0]; }" ::"r"(item_bars + 8u * q) : "memory");
         }
@@ -931,12 +931,6 @@ int launch_convert_out(const float* y32, void* y, int y_dtype, size_t count, cud
     return cuda_status(launch_pdl(convert_out_kernel, dim3((unsigned)((count + 255) / 256)), dim3(256), 0, st, y32,
                                   static_cast<__nv_bfloat16*>(y), count));
 }
-
-#ifdef HIGGS_TRACE
-extern "C" int higgs_stream_blocks_read(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_stream_blocks, sizeof(unsigned long long) * 4 * 256); }
-extern "C" int higgs_trace_pro_read(long long* out) { return (int)cudaMemcpyFromSymbol(out, g_trace_pro, sizeof(long long) * 17 * 16); }
-extern "C" int higgs_trace_read(long long* out) { return (int)cudaMemcpyFromSymbol(out, g_trace, sizeof(long long) * 17 * 64); }
-#endif
 
 int read_device_status(cudaStream_t st, int clear) {
     int v = 0;
