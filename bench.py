@@ -178,7 +178,7 @@ def run_reference(args):
     if rank != 0:
         return
     import oracle
-    from tests.golden import make_grids
+    from synth import grids as make_grids
 
     layers = inputs.LAYER_SETS[args.workload]
     cfg = inputs.CONFIG_OF_SET[args.workload]

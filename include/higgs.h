@@ -32,14 +32,27 @@
  *   i.e. output number m of the splitmix64 stream seeded with xi, and
  *   sign(xi, j) = -1 if bit (j mod 64) of out(xi, floor(j / 64)) is set, else +1.
  * One sign per input index j in [0, K), shared by every row of W and every
- * token, so that the activations are rotated once (Appendix F: "same xi ...
- * same groups").
+ * token, so that the activations are rotated once (Appendix F, "Rotating
+ * Activations": activations and weights are transformed with one seed over
+ * identical groups).
  *
  * The transform itself: RHT(v) = H * diag(sign) * v on each group of g values,
  * H the Sylvester-ordered Hadamard matrix H[i][j] = (-1)^popcount(i & j).
  * The encoder uses H unnormalised (Algorithm 1: entries of the rotated unit
- * vector are approximately N(0,1)); the activations use H / sqrt(g) (Appendix
- * F: "additional scale 1/sqrt(g) ... making it a random rotation").
+ * vector are approximately N(0,1)); the activations use H / sqrt(g), which is
+ * orthonormal, i.e. a random rotation (Appendix F).
+ *
+ * Ordering of producers and consumers on a stream.  The product kernels are
+ * launched so that they may begin (table build, first weight copies) before
+ * the previous kernel of the stream has finished; they wait for it before
+ * they touch x, y or the workspace.  packed, scales and grid are therefore
+ * read early: they must not be written by work that is still running when a
+ * higgs_linear* call is enqueued behind it.  The library's own producers
+ * (higgs_quantize, higgs_pack_codes, higgs_make_grid*, higgs_make_uniform_grid)
+ * end with a kernel that is launched without that early-start permission, so
+ * calling them and a product back to back on one stream is safe; a caller
+ * who fills these buffers with kernels of their own must leave one ordinary
+ * kernel launch or event between those kernels and the product.
  */
 #ifndef HIGGS_H_
 #define HIGGS_H_
@@ -63,7 +76,10 @@ typedef enum higgs_status {
 
 typedef enum higgs_dtype { HIGGS_F32 = 0, HIGGS_F16 = 1, HIGGS_BF16 = 2 } higgs_dtype;
 
-typedef enum higgs_op { HIGGS_OP_QUANTIZE = 0, HIGGS_OP_LINEAR = 1, HIGGS_OP_MAKE_GRID = 2 } higgs_op;
+typedef enum higgs_op { HIGGS_OP_QUANTIZE = 0, HIGGS_OP_LINEAR = 1, HIGGS_OP_MAKE_GRID = 2, HIGGS_OP_MAKE_GRID_SEEDED = 3 } higgs_op;
+
+/* Version of the packed code stream and scale layouts this library writes and reads (higgs_desc.layout_version). */
+#define HIGGS_LAYOUT_VERSION 1
 
 /*
  * Description of one quantized matrix.  Supported: g = 1024; (p, n) in
@@ -72,7 +88,9 @@ typedef enum higgs_op { HIGGS_OP_QUANTIZE = 0, HIGGS_OP_LINEAR = 1, HIGGS_OP_MAK
  * Anything else returns HIGGS_ERR_UNSUPPORTED (never padded silently).
  * scale_dtype must be HIGGS_F16: one 16-bit scale per (row, group), which is
  * what the paper's bit counts imply (4.02 = 4 + 16/1024 in the appendix on
- * experiment configurations).
+ * experiment configurations).  layout_version must be HIGGS_LAYOUT_VERSION: packed
+ * buffers are only meaningful to the library version that wrote them, and a
+ * descriptor saved beside them says which that was.
  */
 typedef struct higgs_desc {
     int32_t p;
@@ -82,6 +100,8 @@ typedef struct higgs_desc {
     uint64_t rht_seed; /* xi */
     int64_t N;
     int64_t K;
+    int32_t layout_version; /* HIGGS_LAYOUT_VERSION */
+    int32_t reserved;       /* 0 */
 } higgs_desc;
 
 /* Text for a status code (static storage, never NULL). */
@@ -98,8 +118,9 @@ size_t higgs_scales_bytes(const higgs_desc* desc);
 size_t higgs_canonical_bytes(const higgs_desc* desc);
 
 /* Scratch bytes the given operation needs for batch B (B ignored unless
- * op == HIGGS_OP_LINEAR; for HIGGS_OP_MAKE_GRID desc->K holds the number of
- * samples and desc->p, desc->n the grid).  Workspaces must be 256-byte
+ * op == HIGGS_OP_LINEAR; for HIGGS_OP_MAKE_GRID and HIGGS_OP_MAKE_GRID_SEEDED
+ * desc->K holds the number of samples and desc->p, desc->n the grid; the other
+ * descriptor fields are ignored for these two).  Workspaces must be 256-byte
  * aligned.  Contents need not be initialised and are undefined afterwards.  */
 size_t higgs_workspace_bytes(const higgs_desc* desc, int op, int64_t B);
 
@@ -137,6 +158,19 @@ int higgs_make_uniform_grid(int n, float* grid_out, float* step_out, float* mse_
 int higgs_make_grid(int p, int n, const float* samples, int64_t num_samples, int max_iters,
                     float* grid_out, float* mse_out, int32_t* iters_out,
                     void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Algorithm 2's grid with the samples drawn by the library: 2^log2_samples points of N(0, I_p) from sample_seed, then
+ * the iteration of higgs_make_grid on them.  Sample i, coordinate k is sqrt(-2 ln u1) cos(2 pi u2) with
+ * u1 = (bits 40..63 of z + 0.5) / 2^24, u2 = (bits 16..39 of z + 0.5) / 2^24, z = out(sample_seed, i p + k) of the
+ * splitmix64 stream defined above (fp32 arithmetic).  workspace: higgs_workspace_bytes(desc, HIGGS_OP_MAKE_GRID_SEEDED,
+ * 0) bytes with desc->K = 2^log2_samples (it holds the samples too).  1 <= log2_samples <= 24.  Other arguments and
+ * errors as higgs_make_grid.  higgs_gaussian_samples writes the same samples ([num_samples][p] fp32, device) alone.
+ */
+int higgs_make_grid_seeded(int p, int n, uint64_t sample_seed, int log2_samples, int max_iters,
+                           float* grid_out, float* mse_out, int32_t* iters_out,
+                           void* workspace, size_t workspace_bytes, void* stream);
+int higgs_gaussian_samples(int p, uint64_t sample_seed, int64_t num_samples, float* samples_out, void* stream);
 
 /*
  * Algorithm 1 (RHT-VQ) on every row of W.  Per (row r, group i):
@@ -182,8 +216,8 @@ int higgs_linear(const higgs_desc* desc, const void* x, int64_t B,
                  void* workspace, size_t workspace_bytes, void* stream);
 
 /*
- * The two halves of higgs_linear as separate calls (Section 4.3: the Hadamard
- * transform "can be fully isolated from the matrix multiplication itself").
+ * The two halves of higgs_linear as separate calls (Section 4.3 observes that
+ * the Hadamard transform does not have to be part of the matrix product).
  *   higgs_rotate_activations: x (device [B][K] bf16) -> xdag_out (device,
  *     higgs_rotated_bytes(desc, B) bytes of fp16) = (H / sqrt(g)) diag(sign) x
  *     per K-group.  The storage order is internal to the library and named by
@@ -236,6 +270,15 @@ int higgs_linear_share(const higgs_desc* desc, const void* x, int64_t B, const v
 int higgs_linear_gather(const higgs_desc* desc, const void* x, int64_t B, const void* packed, const void* scales,
                         const float* grid, void* const* y_dsts, int32_t n_dst, int64_t ld, int64_t row_offset,
                         int y_dtype, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The row range of a layer with N rows that rank `rank` of `world` devices holds when the layer is sharded by rows
+ * for higgs_linear_gather (rows are independent in Algorithm 1 and in Appendix F's product): contiguous ranges of
+ * whole units of `multiple` rows (a multiple of 16; 128 keeps every shard on the tensor-core path), the remainder
+ * units going to the first ranks.  HOST function.  *begin_out = first row, *count_out = rows of the shard.
+ * HIGGS_ERR_UNSUPPORTED if N is not a multiple of `multiple`.
+ */
+int higgs_shard_rows(int64_t N, int32_t world, int32_t rank, int32_t multiple, int64_t* begin_out, int64_t* count_out);
 
 /*
  * higgs_linear with HOST activations and HOST output (Appendix F product; the
@@ -302,6 +345,19 @@ size_t higgs_linear_static_capacity(void);
  * timed out are undefined.
  */
 int higgs_device_status(void* stream, int clear);
+
+/*
+ * Measurement and self-check helpers (the paper has no counterpart).
+ * higgs_launch_floor enqueues one kernel that does nothing, launched exactly like the product kernels (early start
+ * permitted, `blocks` x `threads`, `shared_bytes` of dynamic shared memory <= 232448): a chain of them measures what a
+ * chain of product launches costs before a byte moves.
+ * higgs_selftest_wait runs the bounded wait of the small-batch kernel (which = 0) or of the tensor-core kernel
+ * (which = 1) on a barrier that nothing arrives at, with no copy in flight, giving up after about `polls` polls
+ * (<= 2^20): the kernel returns, result_out[0..1] (device int32[2]) is 0 for every wait that ran out, and
+ * higgs_device_status() then reports HIGGS_ERR_TIMEOUT until cleared.  Nothing traps, faults or hangs.
+ */
+int higgs_launch_floor(int32_t blocks, int32_t threads, size_t shared_bytes, void* stream);
+int higgs_selftest_wait(int32_t which, uint32_t polls, int32_t* result_out, void* stream);
 
 /* Number of K ranges the product kernel assigns to different thread blocks for this shape and
  * batch (1 = not split).  For batches up to 16 a split product accumulates with fp32 atomics into a

@@ -17,7 +17,8 @@ LIB_PATH = os.path.join(_PKG, "libhiggs_b200.so")
 
 HIGGS_OK, HIGGS_ERR_INVALID_ARG, HIGGS_ERR_UNSUPPORTED, HIGGS_ERR_WORKSPACE, HIGGS_ERR_CUDA, HIGGS_ERR_TIMEOUT, HIGGS_ERR_STATIC_SCRATCH = range(7)
 HIGGS_F32, HIGGS_F16, HIGGS_BF16 = 0, 1, 2
-HIGGS_OP_QUANTIZE, HIGGS_OP_LINEAR, HIGGS_OP_MAKE_GRID = 0, 1, 2
+HIGGS_OP_QUANTIZE, HIGGS_OP_LINEAR, HIGGS_OP_MAKE_GRID, HIGGS_OP_MAKE_GRID_SEEDED = 0, 1, 2, 3
+HIGGS_LAYOUT_VERSION = 1
 
 EXPORTS = [
     "higgs_status_string", "higgs_sign", "higgs_packed_bytes", "higgs_scales_bytes", "higgs_canonical_bytes",
@@ -27,7 +28,8 @@ EXPORTS = [
     "higgs_linear_static", "higgs_linear_static_capacity", "higgs_linear_k_splits", "higgs_rotated_bytes",
     "higgs_rotated_layout", "higgs_dequantize", "higgs_make_uniform_grid", "higgs_layer_error",
     "higgs_allocate_bits", "higgs_general_tuples", "higgs_quantize_general", "higgs_linear_host_batch",
-    "higgs_linear_gather", "higgs_linear_share",
+    "higgs_linear_gather", "higgs_linear_share", "higgs_make_grid_seeded", "higgs_gaussian_samples", "higgs_shard_rows",
+    "higgs_launch_floor", "higgs_selftest_wait",
 ]
 
 
@@ -35,6 +37,7 @@ class higgs_desc(ctypes.Structure):
     _fields_ = [
         ("p", ctypes.c_int32), ("n", ctypes.c_int32), ("g", ctypes.c_int32), ("scale_dtype", ctypes.c_int32),
         ("rht_seed", ctypes.c_uint64), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+        ("layout_version", ctypes.c_int32), ("reserved", ctypes.c_int32),
     ]
 
 
@@ -112,6 +115,16 @@ def _load() -> ctypes.CDLL:
     lib.higgs_quantize_general.argtypes = [i32, i32, i64, i64, u64, vp, i32, vp, vp, vp, vp, vp]
     lib.higgs_dequantize.restype = i32
     lib.higgs_dequantize.argtypes = [P, vp, vp, vp, vp, i32, vp, sz, vp]
+    lib.higgs_make_grid_seeded.restype = i32
+    lib.higgs_make_grid_seeded.argtypes = [i32, i32, u64, i32, i32, vp, vp, vp, vp, sz, vp]
+    lib.higgs_gaussian_samples.restype = i32
+    lib.higgs_gaussian_samples.argtypes = [i32, u64, i64, vp, vp]
+    lib.higgs_shard_rows.restype = i32
+    lib.higgs_shard_rows.argtypes = [i64, i32, i32, i32, ctypes.POINTER(i64), ctypes.POINTER(i64)]
+    lib.higgs_launch_floor.restype = i32
+    lib.higgs_launch_floor.argtypes = [i32, i32, sz, vp]
+    lib.higgs_selftest_wait.restype = i32
+    lib.higgs_selftest_wait.argtypes = [i32, ctypes.c_uint32, vp, vp]
     return lib
 
 
@@ -119,7 +132,7 @@ lib = _load()
 
 
 def make_desc(p: int, n: int, N: int, K: int, rht_seed: int, g: int = 1024) -> higgs_desc:
-    return higgs_desc(p, n, g, HIGGS_F16, rht_seed & (2**64 - 1), N, K)
+    return higgs_desc(p, n, g, HIGGS_F16, rht_seed & (2**64 - 1), N, K, HIGGS_LAYOUT_VERSION, 0)
 
 
 def status_string(status: int) -> str:
@@ -171,7 +184,7 @@ def higgs_make_grid(p: int, n: int, samples: torch.Tensor, max_iters: int = 4000
     """samples: cuda fp32 [m][p].  Returns (grid [n][p] fp32, mse fp32 scalar tensor, iters int32 scalar tensor)."""
     assert samples.is_cuda and samples.dtype == torch.float32 and samples.is_contiguous()
     m = samples.numel() // p
-    d = higgs_desc(p, n, 0, HIGGS_F16, 0, 0, m)
+    d = higgs_desc(p, n, 0, HIGGS_F16, 0, 0, m, HIGGS_LAYOUT_VERSION, 0)
     if workspace is None:
         workspace = _workspace(higgs_workspace_bytes(d, HIGGS_OP_MAKE_GRID), samples.device)
     grid = torch.empty((n, p), dtype=torch.float32, device=samples.device)
@@ -180,6 +193,38 @@ def higgs_make_grid(p: int, n: int, samples: torch.Tensor, max_iters: int = 4000
     _check(lib.higgs_make_grid(p, n, _ptr(samples), m, int(max_iters), _ptr(grid), _ptr(mse), _ptr(iters),
                                _ptr(workspace), workspace.numel(), _stream()), "higgs_make_grid")
     return grid, mse, iters
+
+
+def higgs_make_grid_seeded(p: int, n: int, sample_seed: int, log2_samples: int = 18, max_iters: int = 4000, device=None):
+    """Grid fit on samples the library draws from the seed.  Returns (grid, mse, iters) like higgs_make_grid."""
+    device = device or torch.device("cuda")
+    d = higgs_desc(p, n, 0, HIGGS_F16, 0, 0, 1 << log2_samples, HIGGS_LAYOUT_VERSION, 0)
+    workspace = _workspace(higgs_workspace_bytes(d, HIGGS_OP_MAKE_GRID_SEEDED), device)
+    grid = torch.empty((n, p), dtype=torch.float32, device=device)
+    mse = torch.empty((), dtype=torch.float32, device=device)
+    iters = torch.empty((), dtype=torch.int32, device=device)
+    _check(lib.higgs_make_grid_seeded(p, n, sample_seed & (2**64 - 1), log2_samples, int(max_iters), _ptr(grid), _ptr(mse),
+                                      _ptr(iters), _ptr(workspace), workspace.numel(), _stream()), "higgs_make_grid_seeded")
+    return grid, mse, iters
+
+
+def higgs_gaussian_samples(p: int, sample_seed: int, num_samples: int, device=None) -> torch.Tensor:
+    device = device or torch.device("cuda")
+    out = torch.empty((num_samples, p), dtype=torch.float32, device=device)
+    _check(lib.higgs_gaussian_samples(p, sample_seed & (2**64 - 1), num_samples, _ptr(out), _stream()), "higgs_gaussian_samples")
+    return out
+
+
+def higgs_launch_floor(blocks: int, threads: int, shared_bytes: int) -> None:
+    _check(lib.higgs_launch_floor(blocks, threads, shared_bytes, _stream()), "higgs_launch_floor")
+
+
+def higgs_selftest_wait(which: int, polls: int, device=None) -> torch.Tensor:
+    """Runs the bounded-wait self-check; returns the device int32[2] result (0 = that wait ran out)."""
+    device = device or torch.device("cuda")
+    out = torch.full((2,), -1, dtype=torch.int32, device=device)
+    _check(lib.higgs_selftest_wait(which, polls, _ptr(out), _stream()), "higgs_selftest_wait")
+    return out
 
 
 def higgs_quantize(desc: higgs_desc, W: torch.Tensor, grid: torch.Tensor, want_canonical: bool = False,
@@ -280,14 +325,12 @@ def higgs_linear_host(desc: higgs_desc, x_host: torch.Tensor, packed: torch.Tens
 
 
 def shard_rows(N: int, world: int, rank: int, multiple: int = 128):
-    """Rows [begin, end) of an N-row layer that rank `rank` of `world` holds: contiguous, multiples of `multiple` rows
-    (128 keeps every shard eligible for the tensor-core path; at least the 16-row tile), the remainder spread over the
-    first ranks."""
-    assert N % multiple == 0 and 0 <= rank < world
-    units = N // multiple
-    base, extra = divmod(units, world)
-    begin = rank * base + min(rank, extra)
-    return begin * multiple, (begin + base + (1 if rank < extra else 0)) * multiple
+    """Rows [begin, end) of an N-row layer that rank `rank` of `world` holds (higgs_shard_rows: contiguous ranges of whole
+    units of `multiple` rows, the remainder spread over the first ranks)."""
+    begin, count = ctypes.c_int64(0), ctypes.c_int64(0)
+    _check(lib.higgs_shard_rows(int(N), int(world), int(rank), int(multiple), ctypes.byref(begin), ctypes.byref(count)),
+           "higgs_shard_rows")
+    return begin.value, begin.value + count.value
 
 
 def higgs_linear_gather(desc: higgs_desc, x: torch.Tensor, packed: torch.Tensor, scales: torch.Tensor, grid: torch.Tensor,

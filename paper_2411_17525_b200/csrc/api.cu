@@ -9,6 +9,7 @@ int check_desc(const higgs_desc* d) {
     if (d->g != kGroup) return HIGGS_ERR_UNSUPPORTED;
     if (format_of(d->p, d->n) == Format::kNone) return HIGGS_ERR_UNSUPPORTED;
     if (d->scale_dtype != HIGGS_F16) return HIGGS_ERR_UNSUPPORTED;
+    if (d->layout_version != HIGGS_LAYOUT_VERSION) return HIGGS_ERR_UNSUPPORTED;
     if (d->N % kRowTile || d->K % kGroup) return HIGGS_ERR_UNSUPPORTED;
     if (d->N > (int64_t)1 << 30 || d->K > (int64_t)1 << 30) return HIGGS_ERR_UNSUPPORTED;
     return HIGGS_OK;
@@ -60,6 +61,10 @@ size_t higgs_workspace_bytes(const higgs_desc* d, int op, int64_t B) {
         if (!(d->p >= 1 && d->p <= kMaxGridDim && d->n >= 1 && d->n <= kMaxGridPoints && d->K >= d->n)) return 0;
         return make_grid_workspace(d->p, d->n, d->K);
     }
+    if (op == HIGGS_OP_MAKE_GRID_SEEDED) {
+        if (!(d->p >= 1 && d->p <= kMaxGridDim && d->n >= 1 && d->n <= kMaxGridPoints && d->K >= d->n)) return 0;
+        return align_up(make_grid_workspace(d->p, d->n, d->K), 256) + (size_t)d->K * d->p * sizeof(float);
+    }
     if (check_desc(d) != HIGGS_OK) return 0;
     if (op == HIGGS_OP_QUANTIZE) return align_up(higgs_canonical_bytes(d), 256) + 256;
     if (op == HIGGS_OP_LINEAR) {
@@ -78,8 +83,55 @@ int higgs_make_grid(int p, int n, const float* samples, int64_t num_samples, int
     if (num_samples < n || num_samples > ((int64_t)1 << 31) - 1) return HIGGS_ERR_INVALID_ARG;
     if (!aligned(workspace, 256)) return HIGGS_ERR_INVALID_ARG;
     if (workspace_bytes < make_grid_workspace(p, n, num_samples)) return HIGGS_ERR_WORKSPACE;
-    return launch_make_grid(p, n, samples, num_samples, max_iters, grid_out, mse_out, iters_out, workspace,
-                            as_stream(stream));
+    const int rc = launch_make_grid(p, n, samples, num_samples, max_iters, grid_out, mse_out, iters_out, workspace,
+                                    as_stream(stream));
+    return rc != HIGGS_OK ? rc : launch_stream_fence(as_stream(stream));
+}
+
+int higgs_make_grid_seeded(int p, int n, uint64_t sample_seed, int log2_samples, int max_iters, float* grid_out,
+                            float* mse_out, int32_t* iters_out, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!grid_out || !workspace || max_iters < 1) return HIGGS_ERR_INVALID_ARG;
+    if (p < 1 || p > kMaxGridDim || n < 1 || n > kMaxGridPoints) return HIGGS_ERR_UNSUPPORTED;
+    if (log2_samples < 1 || log2_samples > 24 || ((int64_t)1 << log2_samples) < n) return HIGGS_ERR_INVALID_ARG;
+    if (!aligned(workspace, 256)) return HIGGS_ERR_INVALID_ARG;
+    const int64_t m = (int64_t)1 << log2_samples;
+    const size_t fit = align_up(make_grid_workspace(p, n, m), 256);
+    if (workspace_bytes < fit + (size_t)m * p * sizeof(float)) return HIGGS_ERR_WORKSPACE;
+    float* samples = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + fit);
+    const int rc = launch_gaussian_samples(p, sample_seed, m, samples, as_stream(stream));
+    if (rc != HIGGS_OK) return rc;
+    const int rc2 = launch_make_grid(p, n, samples, m, max_iters, grid_out, mse_out, iters_out, workspace, as_stream(stream));
+    return rc2 != HIGGS_OK ? rc2 : launch_stream_fence(as_stream(stream));
+}
+
+int higgs_gaussian_samples(int p, uint64_t sample_seed, int64_t num_samples, float* samples_out, void* stream) {
+    if (p < 1 || p > kMaxGridDim || num_samples < 0 || num_samples > ((int64_t)1 << 28)) return HIGGS_ERR_INVALID_ARG;
+    if (num_samples == 0) return HIGGS_OK;
+    if (!samples_out) return HIGGS_ERR_INVALID_ARG;
+    return launch_gaussian_samples(p, sample_seed, num_samples, samples_out, as_stream(stream));
+}
+
+int higgs_shard_rows(int64_t N, int32_t world, int32_t rank, int32_t multiple, int64_t* begin_out, int64_t* count_out) {
+    if (!begin_out || !count_out || world < 1 || rank < 0 || rank >= world || multiple < kRowTile || multiple % kRowTile)
+        return HIGGS_ERR_INVALID_ARG;
+    if (N < 0 || N % multiple) return HIGGS_ERR_UNSUPPORTED;
+    const int64_t units = N / multiple, base = units / world, extra = units % world;
+    const int64_t begin = rank * base + (rank < extra ? rank : extra);
+    *begin_out = begin * multiple;
+    *count_out = (base + (rank < extra ? 1 : 0)) * multiple;
+    return HIGGS_OK;
+}
+
+int higgs_launch_floor(int32_t blocks, int32_t threads, size_t shared_bytes, void* stream) {
+    if (blocks < 1 || threads < 1 || threads > 1024 || shared_bytes > 232448) return HIGGS_ERR_INVALID_ARG;
+    return launch_floor(blocks, threads, shared_bytes, as_stream(stream));
+}
+
+int higgs_selftest_wait(int32_t which, uint32_t polls, int32_t* result_out, void* stream) {
+    if (!result_out || polls > (1u << 20)) return HIGGS_ERR_INVALID_ARG;
+    if (which == 0) return launch_wait_selftest(polls, result_out, as_stream(stream));
+    if (which == 1) return launch_tc_wait_selftest(polls, result_out, as_stream(stream));
+    return HIGGS_ERR_INVALID_ARG;
 }
 
 int higgs_general_tuples(int p) { return p >= 1 && p <= kMaxGridDim ? (kGroup + p - 1) / p : 0; }
@@ -101,7 +153,8 @@ int higgs_quantize_general(int p, int n, int64_t N, int64_t K, uint64_t rht_seed
 int higgs_make_uniform_grid(int n, float* grid_out, float* step_out, float* mse_out, void* stream) {
     if (!grid_out) return HIGGS_ERR_INVALID_ARG;
     if (n < 2 || n > 256) return HIGGS_ERR_UNSUPPORTED;
-    return launch_uniform_grid(n, grid_out, step_out, mse_out, as_stream(stream));
+    const int rc = launch_uniform_grid(n, grid_out, step_out, mse_out, as_stream(stream));
+    return rc != HIGGS_OK ? rc : launch_stream_fence(as_stream(stream));
 }
 
 int higgs_quantize(const higgs_desc* d, const void* W, int w_dtype, const float* grid, void* packed_out,
@@ -124,7 +177,8 @@ int higgs_quantize(const higgs_desc* d, const void* W, int w_dtype, const float*
     // (the packed output is written by the pack kernel only: until then it lends the encoder its scratch space)
     rc = launch_encode(*d, W, w_dtype, grid, canonical, scales_out, packed_out, higgs_packed_bytes(d), st);
     if (rc != HIGGS_OK) return rc;
-    return launch_pack(*d, canonical, packed_out, st);
+    rc = launch_pack(*d, canonical, packed_out, st);
+    return rc != HIGGS_OK ? rc : launch_stream_fence(st);
 }
 
 int higgs_dequantize(const higgs_desc* d, const void* packed, const void* scales, const float* grid, void* W_out,
@@ -431,7 +485,8 @@ int higgs_pack_codes(const higgs_desc* d, const uint8_t* canonical, void* packed
     if (rc != HIGGS_OK) return rc;
     if (d->N == 0 || d->K == 0) return HIGGS_OK;
     if (!canonical || !packed_out || !aligned(packed_out, 16)) return HIGGS_ERR_INVALID_ARG;
-    return launch_pack(*d, canonical, packed_out, as_stream(stream));
+    rc = launch_pack(*d, canonical, packed_out, as_stream(stream));
+    return rc != HIGGS_OK ? rc : launch_stream_fence(as_stream(stream));
 }
 
 int higgs_unpack_codes(const higgs_desc* d, const void* packed, uint8_t* canonical_out, void* stream) {

@@ -9,6 +9,7 @@
 #include <cmath>
 #include <cstdlib>
 #include <limits>
+#include <new>
 #include <vector>
 
 namespace higgs {
@@ -20,6 +21,9 @@ int64_t gcd64(int64_t a, int64_t b) { while (b) { const int64_t t = a % b; a = b
 int allocate_bits(int L, int J, const double* alpha, const double* t2, const int32_t* bits64, const int64_t* sizes,
                   int64_t budget64, int32_t* choice_out, double* objective_out) {
     if (L < 1 || J < 1 || !alpha || !t2 || !bits64 || !sizes || !choice_out) return HIGGS_ERR_INVALID_ARG;
+    if (J > 255) return HIGGS_ERR_UNSUPPORTED;                  // the choice table stores one byte per state (255 = unset)
+    if (budget64 < 0) return HIGGS_ERR_INVALID_ARG;
+    try {
     int64_t g = 0, total = 0;
     for (int l = 0; l < L; ++l) {
         if (sizes[l] <= 0) return HIGGS_ERR_INVALID_ARG;
@@ -30,8 +34,8 @@ int allocate_bits(int L, int J, const double* alpha, const double* t2, const int
     std::vector<int64_t> unit(L);
     for (int l = 0; l < L; ++l) { unit[l] = sizes[l] / g; total += unit[l]; }
     // budget: sum_l bits64[j_l] * unit_l <= budget64 * total
+    if (budget64 > std::numeric_limits<int64_t>::max() / total) return HIGGS_ERR_WORKSPACE;   // the product below would overflow
     const int64_t cap = budget64 * total;
-    if (cap < 0) return HIGGS_ERR_INVALID_ARG;
     int64_t min_cost = 0;
     int minb = bits64[0];
     for (int j = 1; j < J; ++j) if (bits64[j] < minb) minb = bits64[j];
@@ -70,6 +74,9 @@ int allocate_bits(int L, int J, const double* alpha, const double* t2, const int
     }
     if (objective_out) *objective_out = bv;
     return HIGGS_OK;
+    } catch (const std::bad_alloc&) {
+        return HIGGS_ERR_WORKSPACE;                              // never let an exception cross the C boundary
+    }
 }
 
 }  // namespace higgs

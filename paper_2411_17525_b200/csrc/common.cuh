@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "higgs.h"
 
 namespace higgs {
@@ -63,6 +65,18 @@ inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s
 inline int cuda_status(cudaError_t e) { return e == cudaSuccess ? HIGGS_OK : HIGGS_ERR_CUDA; }
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// One-time set-up per device (function attributes, occupancy queries) that several host threads may reach at once:
+// `state[dev]` is read and written under one process-wide mutex.  Returns the stored value (0 = not yet set).
+inline std::mutex& device_setup_mutex() { static std::mutex m; return m; }
+template <typename F>
+inline int device_once(int (&state)[64], F&& setup) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return setup();
+    std::lock_guard<std::mutex> lock(device_setup_mutex());
+    if (state[dev] == 0) state[dev] = setup();
+    return state[dev];
+}
 
 // ---- programmatic dependent launch -----------------------------------------------------------
 // Every kernel of the decode path is launched with the programmatic-stream-serialization
@@ -180,6 +194,11 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
                      const float* grid, void* y, int y_mode, cudaStream_t st, int64_t ldy = 0,
                      const GatherTargets* more = nullptr);
 int read_tc_status(int clear);
+int launch_wait_selftest(uint32_t limit, int* result, cudaStream_t st);
+int launch_tc_wait_selftest(uint32_t limit, int* result, cudaStream_t st);
+int launch_stream_fence(cudaStream_t st);
+int launch_floor(int blocks, int threads, size_t smem, cudaStream_t st);
+int launch_gaussian_samples(int p, uint64_t seed, int64_t m, float* out, cudaStream_t st);
 int read_device_status(cudaStream_t st, int clear);
 
 }  // namespace higgs

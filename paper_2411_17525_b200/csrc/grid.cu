@@ -218,14 +218,13 @@ size_t make_grid_workspace(int p, int n, int64_t m) {
 template <int P, bool SMALL>
 static int assign_step(GridWs w, const float* samples, int n, int64_t m, unsigned blocks, cudaStream_t st) {
     const size_t smem = up256(sizeof(float) * n * P) + (SMALL ? sizeof(double) * n * P + sizeof(unsigned int) * n : 0);
-    static bool opted[64] = {false};                       // per instantiation and device
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = -1;
-    if (smem > 48 * 1024 && (dev < 0 || !opted[dev])) {
-        cudaError_t e = cudaFuncSetAttribute(grid_assign_kernel<P, SMALL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)(up256(sizeof(float) * kMaxGridPoints * P)));
-        if (e != cudaSuccess) return cuda_status(e);
-        if (dev >= 0) opted[dev] = true;
+    if (smem > 48 * 1024) {
+        static int opted[64] = {0};                        // per instantiation and device: 1 = done, -1 = failed
+        const int ok = device_once(opted, [] {
+            return cudaFuncSetAttribute(grid_assign_kernel<P, SMALL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)(up256(sizeof(float) * kMaxGridPoints * P))) == cudaSuccess ? 1 : -1;
+        });
+        if (ok < 0) return HIGGS_ERR_CUDA;
     }
     grid_assign_kernel<P, SMALL><<<blocks, 256, smem, st>>>(w, samples, n, m);
     return HIGGS_OK;

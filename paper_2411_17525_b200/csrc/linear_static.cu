@@ -1,7 +1,7 @@
 // higgs_linear for callers that cannot hand the library a workspace.
 //
-// Some callers cannot allocate device memory: code that runs inside a stream capture or a
-// real-time loop where cudaMalloc is forbidden, plugins that only receive input and output
+// Some callers cannot allocate device memory: code that runs in a real-time loop or another
+// context where cudaMalloc is forbidden, plugins that only receive input and output
 // tensors from their host framework, and processes whose memory pool is owned by someone
 // else.  For them the scratch that higgs_linear needs (the rotated activations and, for some
 // shapes, an fp32 staging copy of the output) lives in one fixed array inside the library

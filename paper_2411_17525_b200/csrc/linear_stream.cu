@@ -133,12 +133,12 @@ __device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false when the block is aborting (another wait ran out) or this
 // wait ran out itself, in which case it raises the abort flag and the status word.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t limit = kWaitLimit) {
     for (uint32_t it = 0;; ++it) {
         if (mbar_try(bar, parity)) return true;
         if ((it & 63u) == 63u) {
             if (*abort_flag) return false;
-            if (it > kWaitLimit) {
+            if (it > limit) {
                 *abort_flag = 1;
                 atomicExch(&g_device_status, (int)HIGGS_ERR_TIMEOUT);
                 return false;
@@ -148,13 +148,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 }
 // Same for a warp that is not on the critical path: sleeps between polls so that its spinning does not take
 // issue slots from the compute warps of its scheduler.
-__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t limit = kWaitLimit) {
     for (uint32_t it = 0;; ++it) {
         if (mbar_try(bar, parity)) return true;
         __nanosleep(64);
         if ((it & 63u) == 63u) {
             if (*abort_flag) return false;
-            if (it > kWaitLimit) {
+            if (it > limit) {
                 *abort_flag = 1;
                 atomicExch(&g_device_status, (int)HIGGS_ERR_TIMEOUT);
                 return false;
@@ -754,6 +754,22 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     }
 }
 
+// Failure-path check: the product kernel's bounded waits on a barrier nothing ever arrives at (no copy is in flight,
+// nothing else runs): warp 0 uses the compute warps' wait, warp 1 the flusher's.  Both give up after `limit` polls,
+// raise the block's abort flag and the status word, and the kernel returns.
+__global__ void wait_selftest_kernel(uint32_t limit, int* result) {
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int abort_flag;
+    const uint32_t b = (uint32_t)__cvta_generic_to_shared(&bar);
+    if (threadIdx.x == 0) { mbar_init(b, 1); abort_flag = 0; }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+    bool ok;
+    if ((threadIdx.x >> 5) == 0) ok = mbar_wait(b, 0, &abort_flag, limit);
+    else ok = mbar_wait_relaxed(b, 0, &abort_flag, limit);
+    if ((threadIdx.x & 31) == 0) result[threadIdx.x >> 5] = ok ? 1 : 0;
+}
+
 __global__ void convert_out_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, size_t count) {
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     pdl_trigger();
@@ -763,14 +779,12 @@ __global__ void convert_out_kernel(const float* __restrict__ src, __nv_bfloat16*
 
 int sm_count() {
     static int cached[64] = {0};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
-    if (cached[dev] == 0) {
-        int v = 0;
-        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
-        cached[dev] = v;
-    }
-    return cached[dev];
+    return device_once(cached, [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0)
+            v = 148;
+        return v;
+    });
 }
 
 struct Plan {
@@ -811,15 +825,12 @@ Plan make_plan(const higgs_desc& d, int64_t B) {
 
 template <int NB, int KS, int FMT, bool FUSED = false>
 int launch_one(const StreamParams& prm, int blocks, cudaStream_t st) {
-    static bool configured[64] = {false};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(linear_stream_kernel<NB, KS, FMT, FUSED>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem);
-        if (e != cudaSuccess) return HIGGS_ERR_CUDA;
-        configured[dev] = true;
-    }
+    static int configured[64] = {0};       // 1 = attribute set, -1 = failed (per instantiation and device)
+    const int ok = device_once(configured, [] {
+        return cudaFuncSetAttribute(linear_stream_kernel<NB, KS, FMT, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)kMaxDynSmem) == cudaSuccess ? 1 : -1;
+    });
+    if (ok < 0) return HIGGS_ERR_CUDA;
     return cuda_status(launch_pdl(linear_stream_kernel<NB, KS, FMT, FUSED>, dim3((unsigned)blocks), dim3((kWarps + 1) * 32),
                                   kMaxDynSmem, st, prm));
 }
@@ -930,6 +941,11 @@ int launch_convert_out(const float* y32, void* y, int y_dtype, size_t count, cud
     if (count == 0) return HIGGS_OK;
     return cuda_status(launch_pdl(convert_out_kernel, dim3((unsigned)((count + 255) / 256)), dim3(256), 0, st, y32,
                                   static_cast<__nv_bfloat16*>(y), count));
+}
+
+int launch_wait_selftest(uint32_t limit, int* result, cudaStream_t st) {
+    wait_selftest_kernel<<<1, 64, 0, st>>>(limit, result);
+    return cuda_status(cudaGetLastError());
 }
 
 int read_device_status(cudaStream_t st, int clear) {

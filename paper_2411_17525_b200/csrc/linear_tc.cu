@@ -32,18 +32,6 @@ namespace higgs {
 
 __device__ int g_tc_status = 0;
 
-#ifdef HIGGS_TRACE
-__device__ long long g_tc_trace[4][256];
-__device__ unsigned long long g_tc_blocks[4][512];
-__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define BTRACE(row_) do { if (threadIdx.x == 96 && blockIdx.y == 0 && blockIdx.z == 0 && blockIdx.x < 512) g_tc_blocks[row_][blockIdx.x] = gtime(); } while (0)
-#define BTRACE_FIRST() do { g_tc_blocks[1][blockIdx.x] = gtime(); } while (0)
-#define TTRACE(row_, slot_) do { if (blockIdx.x == 3 && blockIdx.y == 0 && (threadIdx.x & 31) == 0 && (slot_) < 256) g_tc_trace[row_][slot_] = clock64(); } while (0)
-#else
-#define TTRACE(row_, slot_) do { } while (0)
-#define BTRACE(row_) do { } while (0)
-#define BTRACE_FIRST() do { } while (0)
-#endif
 
 namespace {
 
@@ -223,7 +211,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
     const uint32_t acol0 = BN <= 128 ? 128u : 256u;
 
     // ---- prologue ----
-    BTRACE(0);
     // (1) the table's source: the grid loads are in flight while everything else is set up.  Warp w fills rows
     //     4 (w + 19 r) .. + 3; a row's 128 bytes are written by eight lanes with one 16-byte store each.
     constexpr int kW = kTcThreads / 32;
@@ -360,10 +347,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
         uint32_t bad = 0;
         const uint64_t b_desc0 = smem_desc(b_stage(0), 128u, 1024u);
         for (int S = 0; S < nsuper; ++S) {
-            TTRACE(1, 3 * S);
             bad |= t_wait(a_full(sa), (uint32_t)(ua & 1), t_limit(bad)) ^ 1u;
-            TTRACE(1, 3 * S + 1);
-            if (S == 0 && lane == 0 && blockIdx.y == 0 && blockIdx.z == 0 && blockIdx.x < 512) { BTRACE_FIRST(); }
             tc_fence_after();
             const uint32_t a_stage = tmem + acol0 + kTcAStageCols * (uint32_t)sa;
 #pragma unroll
@@ -390,7 +374,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
                 }
             }
             if (elected) tc_commit(a_free(sa));
-            TTRACE(1, 3 * S + 2);
             const bool wrap = sa + 1 == AS;
             sa = wrap ? 0 : sa + 1;
             ua += wrap ? 1 : 0;
@@ -422,9 +405,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
         int cs = (sg / SPS) % CS, ucs = 0;         // code stage of step 4 S + sg and its use count (CS >= 4)
         for (int S = 0; S < nsuper; ++S) {
             const int jg = kstep0 + 4 * S + sg;    // 64-input step of the layer
-            if (warp == 3) TTRACE(0, 4 * S);
             bad |= t_wait(code_full(cs), (uint32_t)(ucs & 1), t_limit(bad)) ^ 1u;
-            if (warp == 3) TTRACE(0, 4 * S + 1);
             if ((jg >> 4) != cur_group) {          // new group of 1024 inputs: this row's scale
                 cur_group = jg >> 4;
                 const __half sc = sc_row[cur_group * 16];
@@ -485,9 +466,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
                 }
             }
             // the A stage must have been consumed by the MMAs that used it last
-            if (warp == 3 && a[31] != 0x12345u) TTRACE(0, 4 * S + 2);
             bad |= t_wait(a_free(sa), (uint32_t)((ua & 1) ^ 1), t_limit(bad)) ^ 1u;   // (first use: the phase before the first)
-            if (warp == 3) TTRACE(0, 4 * S + 3);
             tc_fence_after();
             tc_st32(t_lane + acol0 + kTcAStageCols * (uint32_t)sa + 32u * (uint32_t)sg, a);   // column 8m + jj = input pair 8m + jj
             asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
@@ -496,10 +475,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
             if (lane == 0) t_mbar_arrive(a_full(sa));
             if (++sa == AS) { sa = 0; ++ua; }
         }
-        if (warp == 3) TTRACE(3, 0);
         bad |= t_wait(d_full, 0u, t_limit(bad)) ^ 1u;
-        if (warp == 3) TTRACE(3, 1);
-        BTRACE(2);
         t_report(bad, abort_flag);
         if (!bad) {
             tc_fence_after();
@@ -512,7 +488,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
                 uint32_t d[32];
                 tc_ld32(t_lane + (uint32_t)c0, d);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (warp == 3 && c0 == 0) TTRACE(3, 5);
 #pragma unroll
                 for (int r = 0; r < 32; ++r)
                     if (c0 + r < BN)
@@ -522,11 +497,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
     }
 
     // ---- every role ends here, aborted or not: TMEM must be handed back ----
-    if (warp == 3) TTRACE(3, 2);
     tc_fence_before();
     __syncthreads();
-    if (warp == 3) TTRACE(3, 3);
-    BTRACE(3);
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
     }
@@ -534,7 +506,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
         // the parked tile -> y: warp w writes token columns w, w + 16, ...; a lane holds four consecutive rows
         if (tid < 512 && !*abort_flag) {
             pdl_wait();            // y may still be read by the kernel before this one
-            if (warp == 3) TTRACE(3, 4);
             for (int c = warp; c < BN; c += 16) {
                 const int b = bt * BN + c;
                 if (b >= prm.B) break;
@@ -556,7 +527,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
                         *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(prm.y_more[pd]) + o) = v;
                 }
             }
-            if (warp == 3) TTRACE(3, 6);
         }
     } else {
         // Cluster reduction in a fixed order: block kz owns the token columns [kz, kz+1) * BN / ksplit and sums the
@@ -731,16 +701,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn encode_tiled_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
+    static const EncodeTiledFn fn = [] {       // initialised once (thread-safe)
         void* p = nullptr;
         cudaDriverEntryPointQueryResult qr;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess &&
             qr == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-    }
+            return reinterpret_cast<EncodeTiledFn>(p);
+        return static_cast<EncodeTiledFn>(nullptr);
+    }();
     return fn;
 }
 
@@ -769,17 +737,16 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
     if (more && more->count > kMaxGather - 1) return HIGGS_ERR_INVALID_ARG;
     const int BN = tc_batch_tile(B);
     const int64_t tiles = (B + BN - 1) / BN;
-    static bool configured[64] = {false};
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !configured[dev]) {
+    static int configured[64] = {0};
+    const int conf = device_once(configured, [] {
         const void* kernels[6] = {(const void*)linear_tc_kernel<1, false>, (const void*)linear_tc_kernel<2, false>,
                                   (const void*)linear_tc_kernel<4, false>, (const void*)linear_tc_kernel<1, true>,
                                   (const void*)linear_tc_kernel<2, true>, (const void*)linear_tc_kernel<4, true>};
         for (const void* k : kernels)
-            if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem) != cudaSuccess) return HIGGS_ERR_CUDA;
-        configured[dev] = true;
-    }
+            if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem) != cudaSuccess) return -1;
+        return 1;
+    });
+    if (conf < 0) return HIGGS_ERR_CUDA;
     CUtensorMap code_map;
     if (!make_code_map(d, packed, &code_map)) return HIGGS_ERR_CUDA;
     TcParams prm;
@@ -821,13 +788,13 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
     if (prm.ksplit > 1) {
         // a cluster of `ksplit` blocks with this much shared memory must fit the device (it does on a full B200; a
         // partitioned one may not, and then K is not split): checked once per device and cluster size
-        static int cluster_ok[64][kTcMaxSplit + 1] = {};
-        if (dev >= 0 && dev < 64 && cluster_ok[dev][prm.ksplit] == 0) {
+        static int cluster_ok[kTcMaxSplit + 1][64] = {};
+        const int fits = device_once(cluster_ok[prm.ksplit], [&] {
             int n_clusters = 0;
             const cudaError_t e = cudaOccupancyMaxActiveClusters(&n_clusters, kernel, &cfg);
-            cluster_ok[dev][prm.ksplit] = (e == cudaSuccess && n_clusters > 0) ? 1 : -1;
-        }
-        if (dev >= 0 && dev < 64 && cluster_ok[dev][prm.ksplit] < 0) {      // fall back to one block per tile
+            return (e == cudaSuccess && n_clusters > 0) ? 1 : -1;
+        });
+        if (fits < 0) {      // fall back to one block per tile
             prm.ksplit = 1;
             cfg.gridDim.z = 1;
             cfg.numAttrs = 1;
@@ -836,10 +803,26 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
     return cuda_status(cudaLaunchKernelEx(&cfg, kernel, prm, code_map));
 }
 
-#ifdef HIGGS_TRACE
-extern "C" int higgs_tc_blocks_read(unsigned long long* out) { return (int)cudaMemcpyFromSymbol(out, g_tc_blocks, sizeof(unsigned long long) * 4 * 512); }
-extern "C" int higgs_tc_trace_read(long long* out) { return (int)cudaMemcpyFromSymbol(out, g_tc_trace, sizeof(long long) * 4 * 256); }
-#endif
+// Failure-path check for the tensor-core kernel's wait helper: a barrier nothing arrives at, no copy or MMA in flight.
+__global__ void tc_wait_selftest_kernel(uint32_t limit, int* result) {
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int abort_flag;
+    const uint32_t b = (uint32_t)__cvta_generic_to_shared(&bar);
+    if (threadIdx.x == 0) { t_mbar_init(b, 1); abort_flag = 0; }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+    uint32_t bad = 0;
+    bad |= t_wait(b, 0, limit) ^ 1u;          // runs out
+    bad |= t_wait(b, 0, t_limit(bad)) ^ 1u;   // a later wait of the same role polls once
+    t_report(bad, &abort_flag);
+    __syncthreads();
+    if (threadIdx.x == 0) result[0] = bad ? 0 : 1;
+}
+
+int launch_tc_wait_selftest(uint32_t limit, int* result, cudaStream_t st) {
+    tc_wait_selftest_kernel<<<1, 32, 0, st>>>(limit, result);
+    return cuda_status(cudaGetLastError());
+}
 
 int read_tc_status(int clear) {
     int v = 0;

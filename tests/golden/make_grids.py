@@ -11,19 +11,11 @@ import sys
 
 import numpy as np
 
-HERE = os.path.dirname(os.path.abspath(__file__))
-GRIDS = [(2, 256), (2, 64), (1, 16), (2, 16), (1, 8), (1, 4), (1, 256)]
+sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.dirname(os.path.abspath(__file__)))))
+
+from synth.grids import GRIDS, load, path  # noqa: F401  (tests import the loader from here or from synth.grids)
+
 UNIFORM = {(1, 256)}      # constrained (equally spaced) grids: closed-form optimum of the step, no samples
-
-
-def path(p, n):
-    return os.path.join(HERE, f"grid_p{p}_n{n}.txt")
-
-
-def load(p, n):
-    """The stored table as float64 holding exactly the fp32 values (9 printed digits identify an fp32)."""
-    g = np.loadtxt(path(p, n), dtype=np.float64, comments="#", ndmin=2)
-    return g.astype(np.float32).astype(np.float64).reshape(n, p)
 
 
 def main():

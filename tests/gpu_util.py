@@ -4,7 +4,7 @@ import torch
 
 import oracle
 import paper_2411_17525_b200 as hb
-from tests.golden import make_grids
+from synth import grids as make_grids
 
 
 def dev():
@@ -52,3 +52,8 @@ def compare_codes(gpu_codes: np.ndarray, q, max_margin=1e-5, max_frac=1e-4):
 def linear_error(y_gpu: np.ndarray, y_ref: np.ndarray) -> float:
     """max |y - y_ref| / max |y_ref| over the whole call (the layer-level relative error)."""
     return float(np.max(np.abs(y_gpu.astype(np.float64) - y_ref)) / np.max(np.abs(y_ref)))
+
+
+def linear_error_rms(y_gpu: np.ndarray, y_ref: np.ndarray) -> float:
+    """max |y - y_ref| / rms(y_ref): the same deviation against the typical output size instead of the largest."""
+    return float(np.max(np.abs(y_gpu.astype(np.float64) - y_ref)) / np.sqrt(np.mean(np.square(y_ref))))

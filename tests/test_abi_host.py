@@ -103,3 +103,45 @@ def test_invalid_arguments_are_refused_before_any_cuda_call():
     assert L.higgs_quantize(ctypes.byref(empty), None, 0, None, None, None, None, None, 0, None) == hb.HIGGS_OK
     for s in range(7):
         assert isinstance(hb.status_string(s), str) and hb.status_string(s)
+
+
+def test_layout_version_is_checked():
+    d = hb.make_desc(2, 256, 16, 1024, 1)
+    assert d.layout_version == hb.HIGGS_LAYOUT_VERSION and hb.higgs_packed_bytes(d) > 0
+    d.layout_version = hb.HIGGS_LAYOUT_VERSION + 1          # a stream written by some other version of the layouts
+    assert hb.higgs_packed_bytes(d) == 0
+    assert binding.lib.higgs_linear(ctypes.byref(d), None, 1, None, None, None, None, 0, None, 0, None) == hb.HIGGS_ERR_UNSUPPORTED
+
+
+def test_shard_rows_partitions_the_rows():
+    for N, world, mult in ((28672, 8, 128), (4096, 3, 128), (1024, 8, 128), (512, 5, 16), (14336, 7, 128)):
+        spans = [hb.shard_rows(N, world, r, mult) for r in range(world)]
+        assert spans[0][0] == 0 and spans[-1][1] == N
+        for (b0, e0), (b1, e1) in zip(spans, spans[1:]):
+            assert e0 == b1                                                      # contiguous, in rank order
+        sizes = [e - b for b, e in spans]
+        assert all(s % mult == 0 for s in sizes) and max(sizes) - min(sizes) <= mult
+        assert sizes == sorted(sizes, reverse=True)                              # the remainder goes to the first ranks
+    b, c = ctypes.c_int64(), ctypes.c_int64()
+    L = binding.lib
+    assert L.higgs_shard_rows(1000, 4, 0, 128, ctypes.byref(b), ctypes.byref(c)) == hb.HIGGS_ERR_UNSUPPORTED
+    assert L.higgs_shard_rows(1024, 4, 4, 128, ctypes.byref(b), ctypes.byref(c)) == hb.HIGGS_ERR_INVALID_ARG
+    assert L.higgs_shard_rows(1024, 4, 0, 24, ctypes.byref(b), ctypes.byref(c)) == hb.HIGGS_ERR_INVALID_ARG
+    assert L.higgs_shard_rows(1024, 4, 0, 128, None, ctypes.byref(c)) == hb.HIGGS_ERR_INVALID_ARG
+
+
+def test_seeded_grid_and_helper_arguments():
+    a = ctypes.c_void_p(0x1000)
+    L = binding.lib
+    assert L.higgs_make_grid_seeded(2, 256, 1, 5, 10, a, None, None, a, 1 << 30, None) == hb.HIGGS_ERR_INVALID_ARG   # 32 samples < 256 points
+    assert L.higgs_make_grid_seeded(2, 256, 1, 30, 10, a, None, None, a, 1 << 30, None) == hb.HIGGS_ERR_INVALID_ARG
+    assert L.higgs_make_grid_seeded(5, 256, 1, 18, 10, a, None, None, a, 1 << 30, None) == hb.HIGGS_ERR_UNSUPPORTED
+    assert L.higgs_make_grid_seeded(2, 256, 1, 18, 10, a, None, None, a, 1024, None) == hb.HIGGS_ERR_WORKSPACE
+    d = hb.make_desc(2, 256, 0, 1 << 18, 0)
+    assert hb.higgs_workspace_bytes(d, hb.HIGGS_OP_MAKE_GRID_SEEDED) >= hb.higgs_workspace_bytes(d, hb.HIGGS_OP_MAKE_GRID) + (1 << 18) * 2 * 4
+    assert L.higgs_gaussian_samples(2, 1, 0, None, None) == hb.HIGGS_OK
+    assert L.higgs_gaussian_samples(2, 1, 16, None, None) == hb.HIGGS_ERR_INVALID_ARG
+    assert L.higgs_launch_floor(0, 32, 0, None) == hb.HIGGS_ERR_INVALID_ARG
+    assert L.higgs_launch_floor(148, 2048, 0, None) == hb.HIGGS_ERR_INVALID_ARG
+    assert L.higgs_selftest_wait(0, 100, None, None) == hb.HIGGS_ERR_INVALID_ARG
+    assert L.higgs_selftest_wait(2, 100, a, None) == hb.HIGGS_ERR_INVALID_ARG

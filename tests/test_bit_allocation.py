@@ -28,6 +28,44 @@ def test_solver_matches_exhaustive_enumeration(L, J, budget64, seed):
     assert abs(float(np.sum(alpha * t2[np.arange(L), choice])) - obj) <= 1e-12
 
 
+def test_enumeration_and_solver_on_the_hand_solved_instance(golden):
+    """Two layers, two options, solved on paper in tests/golden/allocate_2x2.txt: pins the oracle's enumeration (which
+    pins the solver everywhere else) and the solver itself."""
+    ref = golden("allocate_2x2.txt")
+    sizes = np.array(ref["sizes"], dtype=np.int64)
+    bits = np.array(ref["bits"])
+    alpha = np.array(ref["alpha"])
+    t2 = np.array([ref["t2_layer0"], ref["t2_layer1"]])
+    for key, budget in (("budget_3", 3.0), ("budget_3p5", 3.5), ("budget_2", 2.0)):
+        j0, j1, obj = ref[key]
+        choice, got = oracle.allocate_bits_bruteforce(alpha, t2, bits, sizes, budget)
+        assert choice.tolist() == [int(j0), int(j1)] and abs(got - obj) < 1e-12
+        c2, o2 = hb.higgs_allocate_bits(alpha, t2, (bits * 64).astype(np.int32), sizes, int(budget * 64))
+        assert list(c2) == [int(j0), int(j1)] and abs(o2 - obj) < 1e-12
+    choice, got = oracle.allocate_bits_bruteforce(alpha, t2, bits, sizes, 1.9)
+    assert choice is None and got == np.inf
+
+
+def test_argument_limits_are_reported_not_wrapped():
+    import ctypes
+    from paper_2411_17525_b200 import binding
+    L, J = 2, 300                                                          # more options than the choice table can index
+    alpha = np.ones(L); t2 = np.ones((L, J)); bits = np.arange(1, J + 1, dtype=np.int32); sizes = np.ones(L, dtype=np.int64)
+    with pytest.raises(RuntimeError) as e:
+        hb.higgs_allocate_bits(alpha, t2, bits, sizes, 64)
+    assert e.value.status == hb.HIGGS_ERR_UNSUPPORTED
+    alpha, t2, bits64, sizes = instance(4, 3, 1)
+    with pytest.raises(RuntimeError) as e:                                 # budget * total would overflow 64 bits
+        hb.higgs_allocate_bits(alpha, t2, bits64, sizes, 2 ** 62)
+    assert e.value.status == hb.HIGGS_ERR_WORKSPACE
+    with pytest.raises(RuntimeError) as e:                                 # a table of more than 2e9 states is refused
+        hb.higgs_allocate_bits(np.ones(50), np.ones((50, 3)), bits64, np.arange(1, 51, dtype=np.int64) * 1000003, 10 ** 6)
+    assert e.value.status == hb.HIGGS_ERR_WORKSPACE
+    with pytest.raises(RuntimeError) as e:
+        hb.higgs_allocate_bits(alpha, t2, bits64, sizes, -5)
+    assert e.value.status == hb.HIGGS_ERR_INVALID_ARG
+
+
 def test_budget_extremes_and_monotonicity():
     alpha, t2, bits64, sizes = instance(40, 4, 9)
     lo, _ = hb.higgs_allocate_bits(alpha, t2, bits64, sizes, 129)        # only the smallest option fits everywhere

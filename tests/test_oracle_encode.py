@@ -47,9 +47,32 @@ def test_hand_worked_example(golden):
     assert np.allclose(What[0], ref["what"], atol=1e-6)
     rel = ((What - W) ** 2).sum() / (W ** 2).sum()
     assert abs(rel - ref["relerr"][0]) < 1e-6
+    # the error-database helper itself on the same instance (its W carries the seed's signs, like quantize's input)
+    assert abs(oracle.layer_error(W * sg[None, :], q.codes, q.scales, 4, grid, xi) - ref["relerr"][0]) < 1e-6
     x = np.ones((1, 4)) * sg[None, :]
     assert abs(oracle.linear_dense(x, q.codes, q.scales, 4, grid, xi)[0, 0] - ref["y"][0]) < 1e-6
     assert abs(oracle.linear_rotated(x, q.codes, q.scales, 4, grid, xi)[0, 0] - ref["y"][0]) < 1e-6
+
+
+def test_layer_error_divides_by_the_norm_of_w_not_of_its_reconstruction():
+    """Section 5, 'Measuring Grid Parameters': t^2 = ||W^ - W||^2 / ||W||^2.  One group of g = 2 with a one-point grid
+    at the origin makes W^ = 0 whatever W is, so t^2 = 1 exactly (dividing by ||W^||^2 would divide by zero); a
+    one-point grid at (1, 1) with w = (3, 4), all by hand: s = 5, stored scale 5 / sqrt 2, rotated reconstruction
+    r = (5 / sqrt 2) (1, 1), w^ = diag(sign) (H2 / sqrt 2) r = diag(sign) (5, 0); with signs (+, +):
+    ||w^ - w||^2 = 4 + 16 = 20, ||w||^2 = 25, t^2 = 0.8 (and ||w^||^2 = 25 too, so a second case with ||w^|| != ||w||:
+    two rows w = (3, 4) and (0, 1) -> w^ rows (5, 0) and (1, 0): errors 20 + 2 = 22 over 25 + 1 = 26)."""
+    xi = 4242
+    sg = oracle.signs(xi, 2)
+    W = np.array([[3.0, 4.0]]) * sg[None, :]
+    zero = np.zeros((1, 2))
+    q0 = oracle.quantize(W, 2, zero, xi)
+    assert abs(oracle.layer_error(W, q0.codes, q0.scales, 2, zero, xi) - 1.0) < 1e-12
+    one = np.ones((1, 2))
+    q1 = oracle.quantize(W, 2, one, xi)
+    assert abs(oracle.layer_error(W, q1.codes, q1.scales, 2, one, xi) - 0.8) < 1e-12
+    W2 = np.array([[3.0, 4.0], [0.0, 1.0]]) * sg[None, :]
+    q2 = oracle.quantize(W2, 2, one, xi)
+    assert abs(oracle.layer_error(W2, q2.codes, q2.scales, 2, one, xi) - 22.0 / 26.0) < 1e-12
 
 
 @pytest.mark.parametrize("g,p,n", [(2, 1, 2), (4, 1, 4), (4, 2, 4), (8, 2, 16), (64, 2, 64), (64, 1, 16), (1024, 2, 256)])
