@@ -7,7 +7,13 @@ in the block: q, k, v read one input (rotated once), o its own, gate and up one 
 effective weight bandwidth (packed codes + scales bytes of the layer set / time per step).  The encoder
 (Algorithm 1) and the grid fit (Algorithm 2) run once during set-up, on the GPU, and are reported separately.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama-3.2-1b] [--batch 1] [--grid 2,256]
+The default workload is the largest single-GPU configuration: the Llama-3.1-70B layer shapes with the seeded 3/4-bit
+assignment (3.5 bits per weight on average), batch 1.  The same run reports, under "detail", one row per layer, grid
+and batch of the other configurations (8B shapes at three grids and batches 1/4/16, and at batches 64/256 with
+log-normal channel scales; 1B shapes at batches 1/16), each with its share of the roofline and a parity check of the
+timed output against the fp64 oracle on sampled rows.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama-3.1-70b] [--batch 1] [--grid mixed]
     python bench.py --impl reference ...      # the fp64 CPU oracle timed on the host cores (reported baseline)
 
 Under torchrun (N > 1) every rank runs an independent replica of the same layer set on its own GPU (the layer
@@ -41,18 +47,21 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", default="llama-3.2-1b", choices=list(inputs.LAYER_SETS))
+    ap.add_argument("--workload", default="llama-3.1-70b", choices=list(inputs.LAYER_SETS))
     ap.add_argument("--batch", type=int, default=1)
-    ap.add_argument("--grid", default="2,256",
+    ap.add_argument("--grid", default=None,
                     help="p,n for every layer, or 'mixed': 3 or 4 bits per matrix (p=2 n=64 / n=256) from the seeded assignment "
-                         "averaging 3.5 bits (the Llama-3.1-70B configuration)")
+                         "averaging 3.5 bits (the default for the Llama-3.1-70B shapes; the other sets default to 2,256)")
     ap.add_argument("--no-graph", action="store_true", help="launch kernels directly instead of replaying CUDA graphs")
     ap.add_argument("--steps-per-graph", type=int, default=8,
-                    help="consecutive steps (over rotating weight copies) captured in one CUDA graph; a remainder of --steps runs "
-                         "from one-step graphs")
+                    help="at most this many consecutive steps (over rotating weight copies) per CUDA graph; the largest divisor "
+                         "of --steps not above it is used, so that exactly --steps steps run from equal graphs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-detail", action="store_true", help="skip the per-layer / other-batch detail measurements")
-    return ap.parse_args()
+    ap.add_argument("--no-detail", action="store_true", help="skip the per-layer rows and the rows of the other configurations")
+    args = ap.parse_args()
+    if args.grid is None:
+        args.grid = "mixed" if args.workload == "llama-3.1-70b" else "2,256"
+    return args
 
 
 def layer_bytes(N, K, p, n):
@@ -89,23 +98,34 @@ def measured_peaks():
         return 6650.0, 1590.0, "fallback"
 
 
-# The encoder is bound by instruction issue (profiles/encode_pruned_kernel_...): 3748 warp instructions per
-# (row, group) task of 1024 weights for p=2 n=256 (ncu, smsp__inst_executed.sum / tasks), against a peak of
-# 148 SMs x 4 schedulers x 1 warp instruction per clock at the SM clock.
+# Encoder rooflines.  ALU: the pruned search is bound by instruction issue (profiles/encode_pruned_kernel_...): ncu
+# counted 3748 warp instructions per (row, group) task of 1024 weights for p=2 n=256 (smsp__inst_executed.sum / tasks);
+# achieved = weights/s x that count, against 148 SMs x 4 schedulers x 1 warp instruction per clock.  It is derived from
+# the measured weights/s and a counted constant, not read from a counter in this run.  HBM: what the encoder must move
+# per weight - the bf16 weight in, log2(n)/p bits of code and 16/1024 bits of scale out - against the copy peak; this
+# is the floor an exact pruned search approaches.
 ENCODER_WARP_INSTR_PER_WEIGHT = {(2, 256): 3748.0 / 1024.0}
 
 
-def encoder_roofline(weights_per_s, pn, clocks):
+def encoder_rooflines(weights_per_s, pn, sizes, clocks, hbm_peak, peak_src):
+    out = []
+    bits = {(2, 256): 4, (1, 16): 4, (2, 64): 3, (2, 16): 2, (1, 8): 3, (1, 4): 2, (1, 256): 8}
+    total = float(sum(sizes))
+    bytes_per_weight = sum(s * (2.0 + bits[k] / 8.0 + 2.0 / G) for s, k in zip(sizes, pn)) / total
+    gbs = weights_per_s * bytes_per_weight / 1e9
+    out.append({"bound": "hbm", "achieved": gbs, "peak": hbm_peak, "unit": "GB/s", "frac": gbs / hbm_peak,
+                "bytes_per_weight": bytes_per_weight, "peak_source": f"of {peak_src}"})
     grids = set(pn)
-    if len(grids) != 1 or next(iter(grids)) not in ENCODER_WARP_INSTR_PER_WEIGHT:
-        return None
-    ipw = ENCODER_WARP_INSTR_PER_WEIGHT[next(iter(grids))]
-    mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
-    peak = 148 * 4 * mhz * 1e6 / 1e9                    # G warp instructions / s
-    achieved = weights_per_s * ipw / 1e9
-    return {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "G warp-instr/s", "frac": achieved / peak,
-            "warp_instr_per_weight": ipw,
-            "note": "whole higgs_quantize calls (search, pack and table build) against the issue rate of 148 SMs x 4 schedulers"}
+    if len(grids) == 1 and next(iter(grids)) in ENCODER_WARP_INSTR_PER_WEIGHT:
+        ipw = ENCODER_WARP_INSTR_PER_WEIGHT[next(iter(grids))]
+        mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
+        peak = 148 * 4 * mhz * 1e6 / 1e9                    # G warp instructions / s
+        achieved = weights_per_s * ipw / 1e9
+        out.append({"bound": "alu", "achieved": achieved, "peak": peak, "unit": "G warp-instr/s", "frac": achieved / peak,
+                    "warp_instr_per_weight": ipw,
+                    "note": "derived: measured weights/s of whole higgs_quantize calls x warp instructions per weight "
+                            "counted by ncu in the committed capture, against the issue rate of 148 SMs x 4 schedulers"})
+    return out
 
 
 def max_over_ranks(ms: float, device, world: int) -> float:
@@ -172,34 +192,41 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------------------------- reference arm
+def oracle_sample(layers, pn, cfg, xi, grids64, B, rows):
+    """`rows` rows of every layer, encoded by the oracle (rows are independent, so this is a plain sample of the set)."""
+    import oracle
+    sample = []
+    for li, (name, N, K) in enumerate(layers):
+        r = min(rows, N)
+        W = inputs.make_weights(r, K, inputs.weight_seed(cfg, li), bf16=True).astype(np.float64)
+        q = oracle.quantize(W, G, grids64[pn[li]], xi)
+        sc = oracle.round_scales_fp16(q.scales).astype(np.float64)
+        x = inputs.make_activations(B, K, inputs.activation_seed(cfg, B) + li).astype(np.float64)
+        sample.append((W, q.codes, sc, x, r, K, pn[li]))
+    return sample
+
+
 def run_reference(args):
     """The fp64 oracle (as it stands) on the host cores: the same metric on a bounded sample of the workload."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     import oracle
-    from synth import grids as make_grids
+    from synth import grids as stored_grids
 
     layers = inputs.LAYER_SETS[args.workload]
     cfg = inputs.CONFIG_OF_SET[args.workload]
     pn, grid_text = layer_grids(args, layers, cfg)
     xi = inputs.rht_seed(cfg)
-    grids = {k: make_grids.load(*k) for k in set(pn)}
+    grids64 = {k: stored_grids.load(*k) for k in set(pn)}
     B = args.batch
-    rows = 64  # rows of every layer per step: rows are independent, so this is a plain sample of the layer set
-    sample = []
-    for li, (name, N, K) in enumerate(layers):
-        r = min(rows, N)
-        W = inputs.make_weights(r, K, inputs.weight_seed(cfg, li), bf16=True).astype(np.float64)
-        q = oracle.quantize(W, G, grids[pn[li]], xi)
-        sc = oracle.round_scales_fp16(q.scales).astype(np.float64)
-        x = inputs.make_activations(B, K, inputs.activation_seed(cfg, B) + li).astype(np.float64)
-        sample.append((q.codes, sc, x, r, K, pn[li]))
-    nbytes = sum(layer_bytes(r, K, *k) for _, _, _, r, K, k in sample)
+    rows = 16 if args.workload == "llama-3.1-70b" else 64
+    sample = oracle_sample(layers, pn, cfg, xi, grids64, B, rows)
+    nbytes = sum(layer_bytes(r, K, *k) for *_, r, K, k in sample)
 
     def step():
-        for codes, sc, x, r, K, k in sample:
-            oracle.linear_dense(x, codes, sc, G, grids[k], xi)
+        for _, codes, sc, x, r, K, k in sample:
+            oracle.linear_dense(x, codes, sc, G, grids64[k], xi)
 
     for _ in range(args.warmup):
         step()
@@ -221,6 +248,220 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def cpu_baseline(layers, pn, cfg, xi, grids64, B):
+    """The oracle as it stands on this machine's cores, on a bounded row sample: the product (dequantise + fp64 matmul) on
+    all cores and on one, and the encoder (Algorithm 1) likewise.  About 25 s in all."""
+    import oracle
+    cores = oracle.threads()
+    rows = 64 if sum(N * K for _, N, K in layers) > 5e8 else 256
+    smp = oracle_sample(layers, pn, cfg, xi, grids64, B, rows)
+    nb = sum(layer_bytes(r, K, *k) for *_, r, K, k in smp)
+    nw = sum(r * K for *_, r, K, k in smp)
+
+    def product():
+        for _, codes, sc, x, r, K, k in smp:
+            oracle.linear_dense(x, codes, sc, G, grids64[k], xi)
+
+    def encode():
+        for W, _, _, _, r, K, k in smp:
+            oracle.quantize(W, G, grids64[k], xi)
+
+    def timed(fn, budget):
+        reps, t0 = 0, time.perf_counter()
+        while reps < 1 or time.perf_counter() - t0 < budget:
+            fn()
+            reps += 1
+        return (time.perf_counter() - t0) / reps, reps
+
+    dt_all, reps = timed(product, 8.0)
+    dtq_all, _ = timed(encode, 4.0)
+    oracle.set_threads(1)
+    try:
+        dt_one, _ = timed(product, 5.0)
+        dtq_one, _ = timed(encode, 4.0)
+    finally:
+        oracle.set_threads(cores)
+    return {"value": nb / dt_all / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
+            "sample": f"{rows} rows of each of the {len(layers)} layers (rows are independent), dequantise + fp64 matmul, {reps} passes",
+            "single_thread_value": nb / dt_one / 1e9,
+            "quantize_weights_per_s": nw / dtq_all, "quantize_weights_per_s_single_thread": nw / dtq_one}
+
+
+# --------------------------------------------------------------------------------------------- our arm: helpers
+def divisor_at_most(steps: int, cap: int) -> int:
+    """Largest divisor of `steps` that is <= cap (>= 1): `steps` steps then run from steps / d equal graphs."""
+    for d in range(max(1, min(cap, steps)), 0, -1):
+        if steps % d == 0:
+            return d
+    return 1
+
+
+class Quantized:
+    """One layer encoded on the device (Algorithm 1) with everything a timed product or a parity check needs."""
+
+    def __init__(self, hb, torch, dev, name, N, K, pn, xi, grid, W, time_it=False):
+        self.name, self.N, self.K, self.pn = name, N, K, pn
+        self.desc = hb.make_desc(pn[0], pn[1], N, K, xi)
+        self.grid = grid
+        self.enc_ms = None
+        pk, sc, _ = hb.higgs_quantize(self.desc, W, grid)
+        if time_it:      # second call: the allocator already holds the output buffers
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            pk, sc, _ = hb.higgs_quantize(self.desc, W, grid)
+            e1.record()
+            torch.cuda.synchronize()
+            self.enc_ms = e0.elapsed_time(e1)
+        self.packed, self.scales = [pk], [sc]
+        self.bytes = layer_bytes(N, K, *pn)
+
+    @classmethod
+    def from_buffers(cls, name, desc, grid, packed, scales):
+        """A layer whose packed buffers exist already (row-concatenated layers)."""
+        q = cls.__new__(cls)
+        q.name, q.N, q.K, q.pn, q.desc, q.grid = name, desc.N, desc.K, (desc.p, desc.n), desc, grid
+        q.packed, q.scales, q.bytes, q.enc_ms = list(packed), list(scales), layer_bytes(desc.N, desc.K, desc.p, desc.n), None
+        return q
+
+    def ensure_copies(self, count):
+        while len(self.packed) < count:
+            self.packed.append(self.packed[0].clone())
+            self.scales.append(self.scales[0].clone())
+
+
+def parity_on_sampled_rows(hb, oracle, q, x_host32, y, xi, grid64, rows=16, seed=1):
+    """The timed output against the fp64 oracle on `rows` sampled rows, given the device's own codes and stored scales:
+    (max |dy| / max |y^|, max |dy| / rms(y^)) over the sample."""
+    rng = np.random.default_rng(seed + q.N)
+    ridx = np.sort(rng.choice(q.N, size=min(rows, q.N), replace=False))
+    canon = hb.higgs_unpack_codes(q.desc, q.packed[0])
+    codes = canon[ridx.tolist()].cpu().numpy().astype(np.int64)
+    sc = hb.scales_from_tile_major(q.scales[0], q.N)[ridx.tolist()].float().cpu().numpy().astype(np.float64)
+    del canon
+    y_ref = oracle.linear_dense(x_host32.astype(np.float64), codes, sc, G, grid64, xi)
+    got = y.float()[:, ridx.tolist()].cpu().numpy().astype(np.float64)
+    err = np.max(np.abs(got - y_ref))
+    return float(err / np.max(np.abs(y_ref))), float(err / np.sqrt(np.mean(y_ref ** 2)))
+
+
+def time_product(hb, torch, stream, q, B, x_dev, reps=200, copies_bytes=2 * L2_BYTES):
+    """One launch of the product kernel (D2-D5 on already rotated activations) of layer `q` at batch B, timed with CUDA
+    events on the launching stream: a CUDA graph of back-to-back launches over rotating weight copies (>= 2 x L2, so no
+    launch finds its codes in L2), every replay timed separately.  Returns mean / median / min microseconds per launch
+    over the replays, the kernels per call and the output of the last launch."""
+    d = q.desc
+    xdag = hb.higgs_rotate_activations(d, x_dev)
+    yk = torch.empty((B, d.N), dtype=torch.float32, device=x_dev.device)
+    wk = torch.empty(hb.higgs_workspace_bytes(d, hb.HIGGS_OP_LINEAR, B), dtype=torch.uint8, device=x_dev.device)
+    q.ensure_copies(min(64, max(2, -(-copies_bytes // q.bytes))))
+    n = len(q.packed)
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        hb.higgs_linear_prerotated(d, xdag, q.packed[0], q.scales[0], q.grid, workspace=wk, y=yk, B=B)
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for c in range(n):
+                hb.higgs_linear_prerotated(d, xdag, q.packed[c], q.scales[c], q.grid, workspace=wk, y=yk, B=B)
+        rounds = max(3, reps // n)
+        for _ in range(3):
+            g.replay()
+        stream.synchronize()
+        marks = [ev() for _ in range(rounds + 1)]
+        marks[0].record(stream)
+        for r in range(rounds):
+            g.replay()
+            marks[r + 1].record(stream)
+        stream.synchronize()
+    per = [marks[r].elapsed_time(marks[r + 1]) * 1e3 / n for r in range(rounds)]
+    total = marks[0].elapsed_time(marks[rounds]) * 1e3 / (rounds * n)
+    return {"us": total, "us_median": statistics.median(per), "us_min": min(per), "launches": rounds * n,
+            "kernels_per_call": hb.higgs_linear_launch_count(d, B) - 1, "y": yk}
+
+
+def product_row(hb, q, B, t, peak, peak_tf, parity=None):
+    """A detail row: time, weight bandwidth and the roofline share of one layer at one batch."""
+    p, n = q.pn
+    tiled = hb.higgs_rotated_layout(q.desc, B) > 0
+    alg = algorithmic_bytes(q.N, q.K, p, n, B)
+    row = {"layer": q.name, "shape": f"{q.N}x{q.K}", "grid": f"p={p} n={n}", "B": B,
+           "kernel": "linear_tc_kernel" if tiled else "linear_stream_kernel",
+           "us": round(t["us"], 3), "us_median": round(t["us_median"], 3), "us_min": round(t["us_min"], 3),
+           "weight_GBps": round(q.bytes / t["us"] / 1e3, 1)}
+    if B >= 64 and tiled:
+        tf = 2.0 * B * q.N * q.K / (t["us"] * 1e-6) / 1e12
+        row["roofline"] = {"bound": "tensor", "achieved": round(tf, 1), "peak": peak_tf, "unit": "TFLOP/s", "frac": round(tf / peak_tf, 4)}
+    else:
+        gb = alg / (t["us"] * 1e-6) / 1e9
+        row["roofline"] = {"bound": "hbm", "achieved": round(gb, 1), "peak": peak, "unit": "GB/s", "frac": round(gb / peak, 4)}
+    if parity is not None:
+        row["parity_max_rel"], row["parity_max_over_rms"] = (float(f"{v:.3g}") for v in parity)
+    return row
+
+
+def launch_floor(hb, torch, stream, blocks, threads, smem, reps=2000):
+    """Microseconds per launch of a chain of kernels that do nothing, launched like the product kernels."""
+    with torch.cuda.stream(stream):
+        hb.higgs_launch_floor(blocks, threads, smem)
+        stream.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
+            for _ in range(50):
+                hb.higgs_launch_floor(blocks, threads, smem)
+        g.replay()
+        stream.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(reps // 50):
+            g.replay()
+        b.record(stream)
+        stream.synchronize()
+    return a.elapsed_time(b) * 1e3 / (reps // 50 * 50)
+
+
+def other_configurations(hb, torch, oracle, dev, stream, peak, peak_tf, fit_grid):
+    """Rows for the configurations that are not the headline workload: the distinct layer shapes of the 8B set at three
+    grids and batches 1, 4, 16; the same shapes at p=2 n=256 and batches 64, 256 with one log-normal scale per input
+    channel; the 1B shapes at batches 1 and 16.  Every row carries the parity of its timed output on sampled rows."""
+    rows = []
+    plan = [("llama-3.1-8b", [(2, 256), (2, 64), (1, 16)], [1, 4, 16], False),
+            ("llama-3.1-8b", [(2, 256)], [64, 256], True),
+            ("llama-3.2-1b", [(2, 256)], [1, 16], False)]
+    cache = {}
+    for workload, grid_list, batches, lognormal in plan:
+        cfg = inputs.CONFIG_OF_SET[workload] + (1 if lognormal else 0)      # configs[3] is the 8B set in the tensor regime
+        xi = inputs.rht_seed(cfg)
+        layers = inputs.LAYER_SETS[workload]
+        seen = set()
+        for li, (name, N, K) in enumerate(layers):
+            if (N, K) in seen:
+                continue
+            seen.add((N, K))
+            key = (workload, N, K)
+            if key not in cache:
+                cache[key] = torch.from_numpy(inputs.make_weights(N, K, inputs.weight_seed(inputs.CONFIG_OF_SET[workload], li),
+                                                                  bf16=True)).to(dev).to(torch.bfloat16)
+            W = cache[key]
+            for pn in grid_list:
+                grid = fit_grid(pn)
+                q = Quantized(hb, torch, dev, name, N, K, pn, xi, grid, W)
+                g64 = grid.cpu().numpy().astype(np.float64)
+                for B in batches:
+                    x32 = inputs.make_activations(B, K, inputs.activation_seed(cfg, B) + li, lognormal_channels=lognormal)
+                    x = torch.from_numpy(x32).to(dev).to(torch.bfloat16)
+                    t = time_product(hb, torch, stream, q, B, x, reps=100)
+                    par = parity_on_sampled_rows(hb, oracle, q, x32, t["y"], xi, g64)
+                    row = product_row(hb, q, B, t, peak, peak_tf, par)
+                    row["workload"] = workload + (" (log-normal channel scales)" if lognormal else "")
+                    rows.append(row)
+                del q
+        if workload == "llama-3.1-8b" and not lognormal:
+            continue            # the 8B weights are used again by the next entry
+        cache.clear()
+    return rows
+
+
 # --------------------------------------------------------------------------------------------- our arm
 def run_ours(args):
     import torch
@@ -239,63 +480,63 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
 
     layers = inputs.LAYER_SETS[args.workload]
+    names = [nm for nm, _, _ in layers]
     cfg = inputs.CONFIG_OF_SET[args.workload]
     pn, grid_text = layer_grids(args, layers, cfg)
     xi = inputs.rht_seed(cfg)
     B = args.batch
+    peak, peak_tf, peak_src = measured_peaks()
 
     def ev():
         return torch.cuda.Event(enable_timing=True)
 
-    # ---- E0: grid fit on the device (Algorithm 2), 2^18 seeded Gaussian samples
-    grids, grid_ms, grid_iters, grid_mse = {}, 0.0, 0, 0.0
-    for (p, n) in sorted(set(pn)):
-        samples = torch.from_numpy(inputs.gaussian_samples(p, inputs.grid_sample_seed(p, n)).astype(np.float32)).to(dev)
-        e0, e1 = ev(), ev()
-        e0.record()
-        grids[(p, n)], grid_mse, grid_iters = hb.higgs_make_grid(p, n, samples, max_iters=3000)
-        e1.record()
-        torch.cuda.synchronize()
-        grid_ms += e0.elapsed_time(e1)
-        del samples
+    # ---- E0: grid fit on the device (Algorithm 2), 2^18 seeded Gaussian samples (the host recipe both arms share)
+    grids, grid_info = {}, {}
+
+    def fit_grid(key):
+        if key not in grids:
+            p, n = key
+            samples = torch.from_numpy(inputs.gaussian_samples(p, inputs.grid_sample_seed(p, n)).astype(np.float32)).to(dev)
+            e0, e1 = ev(), ev()
+            e0.record()
+            grids[key], mse, iters = hb.higgs_make_grid(p, n, samples, max_iters=3000)
+            e1.record()
+            torch.cuda.synchronize()
+            grid_info[f"p={p} n={n}"] = {"ms": e0.elapsed_time(e1), "iters": int(iters), "mse": float(mse)}
+        return grids[key]
+
+    for key in sorted(set(pn)):
+        fit_grid(key)
 
     # ---- E1-E4: encode every layer once on the device (Algorithm 1)
     set_bytes = sum(layer_bytes(N, K, *pn[li]) for li, (_, N, K) in enumerate(layers))
-    copies = max(2, -(-2 * L2_BYTES // set_bytes))          # rotating copies so that no step finds its codes in L2
-    copies = min(copies, 64)
-    descs, packed, scales, xs, xs_host, ws, ys = [], [], [], [], [], [], []
-    enc_ms, enc_weights = 0.0, 0
+    copies = min(64, max(2, -(-2 * L2_BYTES // set_bytes)))      # rotating copies so that no step finds its codes in L2
+    qs, xs, xs_host, xs32, ws, ys = [], [], [], [], [], []
     for li, (name, N, K) in enumerate(layers):
-        d = hb.make_desc(pn[li][0], pn[li][1], N, K, xi)
         W = torch.from_numpy(inputs.make_weights(N, K, inputs.weight_seed(cfg, li), bf16=True)).to(dev).to(torch.bfloat16)
-        pk, sc, _ = hb.higgs_quantize(d, W, grids[pn[li]])       # first call: the allocator fetches the output buffers
-        torch.cuda.synchronize()
-        e0, e1 = ev(), ev()
-        e0.record()
-        pk, sc, _ = hb.higgs_quantize(d, W, grids[pn[li]])       # timed: encode + pack kernels of the whole layer
-        e1.record()
-        torch.cuda.synchronize()
-        enc_ms += e0.elapsed_time(e1)
-        enc_weights += N * K
+        q = Quantized(hb, torch, dev, name, N, K, pn[li], xi, grids[pn[li]], W, time_it=True)
         del W
-        descs.append(d)
-        packed.append([pk] + [pk.clone() for _ in range(copies - 1)])
-        scales.append([sc] + [sc.clone() for _ in range(copies - 1)])
+        q.ensure_copies(copies)
+        qs.append(q)
         # q/k/v read the same block input, so do gate/up
         xi_of = {"k": "q", "v": "q", "up": "gate"}.get(name, name)
-        x_seed = inputs.activation_seed(cfg, B) + [nm for nm, _, _ in layers].index(xi_of)
         if xi_of != name:                  # the same pinned tensor: the block input is one buffer on the host too
-            xs_host.append(xs_host[[nm for nm, _, _ in layers].index(xi_of)])
+            j = names.index(xi_of)
+            xs_host.append(xs_host[j])
+            xs32.append(xs32[j])
         else:
-            xs_host.append(torch.from_numpy(inputs.make_activations(B, K, x_seed)).to(torch.bfloat16).pin_memory())
+            xs32.append(inputs.make_activations(B, K, inputs.activation_seed(cfg, B) + names.index(xi_of)))
+            xs_host.append(torch.from_numpy(xs32[-1]).to(torch.bfloat16).pin_memory())
         xs.append(xs_host[-1].to(dev))
-        ws.append(torch.empty(hb.higgs_linear_host_workspace_bytes(d, B), dtype=torch.uint8, device=dev))
+        ws.append(torch.empty(hb.higgs_linear_host_workspace_bytes(q.desc, B), dtype=torch.uint8, device=dev))
         ys.append(torch.empty((B, N), dtype=torch.float32, device=dev))
+    descs = [q.desc for q in qs]
+    enc_ms = sum(q.enc_ms for q in qs)
+    enc_weights = sum(N * K for _, N, K in layers)
     ys_host = [torch.empty((B, N), dtype=torch.float32).pin_memory() for _, N, _ in layers]
 
     # layers that read the same block input share one rotation (the transform is isolated from the product, Sec. 4.3);
     # a layer whose K is split across thread blocks goes through higgs_linear, whose rotation kernel also clears y
-    names = [nm for nm, _, _ in layers]
     share = {"q": "attn", "k": "attn", "v": "attn", "gate": "mlp", "up": "mlp"}
     groups_of = {}
     for li, nm in enumerate(names):
@@ -306,11 +547,10 @@ def run_ours(args):
     xdags = {k: torch.empty(hb.higgs_rotated_bytes(descs[v[0]], B) // 2, dtype=torch.float16, device=dev)
              for k, v in groups_of.items() if len(v) > 1}
     launches_per_step = 0
-    share_first = True     # the first layer of a group goes through higgs_linear_share
     for k, v in groups_of.items():
         if len(v) > 1:      # one rotation, then one product launch per layer (per 16 tokens on the small-batch path);
                             # for 1-2 tokens the first product rotates x itself and leaves the result for the others
-            first_is_one_launch = share_first and hb.higgs_linear_launch_count(descs[v[0]], B) == 1
+            first_is_one_launch = hb.higgs_linear_launch_count(descs[v[0]], B) == 1
             launches_per_step += (0 if first_is_one_launch else 1) + \
                 sum(1 if hb.higgs_rotated_layout(descs[li], B) > 0 else -(-B // 16) for li in v)
         else:
@@ -319,66 +559,53 @@ def run_ours(args):
     def step(i):
         c = i % copies
         for key, lis in groups_of.items():
-            if len(lis) > 1:
-                rest = lis
-                if share_first:       # the first layer of the group also produces the rotated activations of the others
-                    li = lis[0]
-                    hb.higgs_linear_share(descs[li], xs[li], packed[li][c], scales[li][c], grids[pn[li]], xdag_out=xdags[key],
-                                          workspace=ws[li], y=ys[li])
-                    rest = lis[1:]
-                else:
-                    hb.higgs_rotate_activations(descs[lis[0]], xs[lis[0]], out=xdags[key])
-                for li in rest:
-                    hb.higgs_linear_prerotated(descs[li], xdags[key], packed[li][c], scales[li][c], grids[pn[li]], workspace=ws[li],
-                                               y=ys[li], B=B)
+            if len(lis) > 1:      # the first layer of the group also produces the rotated activations of the others
+                li = lis[0]
+                hb.higgs_linear_share(descs[li], xs[li], qs[li].packed[c], qs[li].scales[c], qs[li].grid, xdag_out=xdags[key],
+                                      workspace=ws[li], y=ys[li])
+                for li in lis[1:]:
+                    hb.higgs_linear_prerotated(descs[li], xdags[key], qs[li].packed[c], qs[li].scales[c], qs[li].grid,
+                                               workspace=ws[li], y=ys[li], B=B)
             else:
                 li = lis[0]
-                hb.higgs_linear(descs[li], xs[li], packed[li][c], scales[li][c], grids[pn[li]], workspace=ws[li], y=ys[li])
+                hb.higgs_linear(descs[li], xs[li], qs[li].packed[c], qs[li].scales[c], qs[li].grid, workspace=ws[li], y=ys[li])
 
     # end to end: host activations in, host outputs out, one library call per step (higgs_linear_host_batch)
-    host_batches = [hb.HostBatch(descs, xs_host, [packed[li][c] for li in range(len(descs))],
-                                 [scales[li][c] for li in range(len(descs))], [grids[pn[li]] for li in range(len(descs))],
+    host_batches = [hb.HostBatch(descs, xs_host, [q.packed[c] for q in qs], [q.scales[c] for q in qs], [q.grid for q in qs],
                                  ys_host, ws) for c in range(copies)]
 
     def step_host(i):
         hb.higgs_linear_host_batch(host_batches[i % copies])
         torch.cuda.current_stream().synchronize()   # the step's results are read on the host
 
-    # ---- graphs: one per weight copy, replayed in rotation
+    # ---- graphs of spg consecutive steps (over rotating weight copies); spg divides --steps, so exactly --steps steps
+    # run from equal graphs (a graph boundary costs about 2 us on the device)
     stream = torch.cuda.Stream()
+    spg = divisor_at_most(args.steps, max(1, args.steps_per_graph))
+    spg_w = divisor_at_most(max(args.warmup, 3), spg)
     graphs = None
     with torch.cuda.stream(stream):
         step(0)
         stream.synchronize()
-        spg = max(1, args.steps_per_graph)
-        graphs_multi = None
         if not args.no_graph:
-            graphs = []
-            for c in range(copies):
-                g = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g, stream=stream):
-                    step(c)
-                graphs.append(g)
-            if spg > 1:          # the same steps, spg of them per graph: a graph boundary costs about 2 us on the device
-                graphs_multi = []
+            graphs = {}
+            for length in {spg, spg_w}:
+                graphs[length] = []
                 for c in range(copies):
                     g = torch.cuda.CUDAGraph()
                     with torch.cuda.graph(g, stream=stream):
-                        for k in range(spg):
-                            step(c * spg + k)
-                    graphs_multi.append(g)
+                        for k in range(length):
+                            step(c * length + k)
+                    graphs[length].append(g)
 
     def run_steps(first, count):      # exactly `count` steps, starting with step number `first`
+        length = spg if count % spg == 0 else spg_w
         i = first
         while count > 0:
-            if graphs_multi is not None and count >= spg:
-                graphs_multi[(i // spg) % copies].replay()
-                i += spg
-                count -= spg
-            elif graphs is not None:
-                graphs[i % copies].replay()
-                i += 1
-                count -= 1
+            if graphs is not None and count >= length:
+                graphs[length][(i // length) % copies].replay()
+                i += length
+                count -= length
             else:
                 step(i)
                 i += 1
@@ -407,20 +634,21 @@ def run_ours(args):
             ms = a.elapsed_time(b)
         return max_over_ranks(ms, dev, world)
 
+    warm = max(args.warmup, 3)
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    ms = timed(run_steps, args.steps, max(args.warmup, 3))
-    ms_e2e = timed(run_steps_host, args.steps, max(args.warmup, 3))
+    ms = timed(run_steps, args.steps, warm)
+    ms_e2e = timed(run_steps_host, args.steps, warm)
     # nvidia-smi samples every 100 ms and the timed regions above last tens of milliseconds: keep the same load running
     # (untimed) for a second more so that the clock record has samples taken under it
     extra_steps = 0
     if rank == 0:
         t_probe = time.perf_counter()
         with torch.cuda.stream(stream):
-            while time.perf_counter() - t_probe < 1.0:      # small batches: under a profiler every launch is slow
-                run_steps(extra_steps, 8)               # keeps rotating over the weight copies like the timed steps
-                extra_steps += 8
+            while time.perf_counter() - t_probe < 1.0:
+                run_steps(extra_steps, spg)
+                extra_steps += spg
                 stream.synchronize()
     clocks = sampler.stop() if rank == 0 else None
     if clocks is not None:
@@ -432,111 +660,112 @@ def run_ours(args):
     h2d = sum(t.numel() * 2 for t in {id(t): t for t in xs_host}.values())       # layers that share their input copy it once
     d2h = sum(B * N * 4 for _, N, _ in layers)
 
-    # ---- dominant kernel: the product kernel on the largest layer, timed alone with CUDA events
-    peak, peak_tf, peak_src = measured_peaks()
-    big = max(range(len(layers)), key=lambda i: layers[i][1] * layers[i][2])
-    _, Nb, Kb = layers[big]
-    db = descs[big]
-
-    def kernel_time(li, d, Bk, reps=200):
-        """Average duration of one launch of the product kernel (pre-rotated activations), rotating weight copies."""
-        xdag = hb.higgs_rotate_activations(d, xs[li] if Bk == B else
-                                           torch.from_numpy(inputs.make_activations(Bk, d.K, 1)).to(torch.bfloat16).to(dev))
-        yk = torch.empty((Bk, d.N), dtype=torch.float32, device=dev)
-        wk = torch.empty(hb.higgs_workspace_bytes(d, hb.HIGGS_OP_LINEAR, Bk), dtype=torch.uint8, device=dev)
-        per_launch_bytes = layer_bytes(d.N, d.K, d.p, d.n)
-        grid = grids[(d.p, d.n)]
-        need = max(2, -(-2 * L2_BYTES // per_launch_bytes))
-        pks = list(packed[li])
-        scs = list(scales[li])
-        while len(pks) < min(need, 64):
-            pks.append(pks[0].clone())
-            scs.append(scs[0].clone())
-        with torch.cuda.stream(stream):
-            g = torch.cuda.CUDAGraph()
-            hb.higgs_linear_prerotated(d, xdag, pks[0], scs[0], grid, workspace=wk, y=yk, B=Bk)
-            stream.synchronize()
-            with torch.cuda.graph(g, stream=stream):
-                for c in range(len(pks)):
-                    hb.higgs_linear_prerotated(d, xdag, pks[c], scs[c], grid, workspace=wk, y=yk, B=Bk)
-            rounds = max(1, reps // len(pks))
-            for _ in range(2):
-                g.replay()
-            stream.synchronize()
-            a, b = ev(), ev()
-            a.record(stream)
-            for _ in range(rounds):
-                g.replay()
-            b.record(stream)
-            stream.synchronize()
-        nodes = hb.higgs_linear_launch_count(d, Bk) - 1
-        return a.elapsed_time(b) * 1e3 / (rounds * len(pks)), nodes   # microseconds per call
-
-    us_big, nodes_big = kernel_time(big, db, B)
-    p, n = pn[big]
-    alg = algorithmic_bytes(Nb, Kb, p, n, B)
-    achieved = alg / (us_big * 1e-6) / 1e9
+    # ---- dominant kernel: the product kernel on the largest layer (most code bytes), timed alone with CUDA events
+    import oracle
+    grids64 = {k: g.cpu().numpy().astype(np.float64) for k, g in grids.items()}
+    big = max(range(len(layers)), key=lambda i: qs[i].bytes)
+    qb = qs[big]
+    tb = time_product(hb, torch, stream, qb, B, xs[big])
+    p, n = qb.pn
+    alg = algorithmic_bytes(qb.N, qb.K, p, n, B)
+    achieved = alg / (tb["us"] * 1e-6) / 1e9
     traffic = None
     tpath = os.path.join(ROOT, "profiles", "traffic.json")
     if os.path.exists(tpath):
         try:
             with open(tpath) as f:
-                traffic = json.load(f).get(f"{args.workload}:{layers[big][0]}:p{p}n{n}:B{B}")
+                traffic = json.load(f).get(f"{args.workload}:{qb.name}:p{p}n{n}:B{B}")
         except Exception:
             traffic = None
-    tiled_big = hb.higgs_rotated_layout(db, B) > 0
+    tiled_big = hb.higgs_rotated_layout(qb.desc, B) > 0
     kname = "linear_tc_kernel" if tiled_big else "linear_stream_kernel"
+    common = {"traffic": traffic, "kernel": kname, "layer": f"{qb.name} {qb.N}x{qb.K} p={p} n={n}", "us_per_launch": tb["us"],
+              "us_per_launch_median": tb["us_median"], "us_per_launch_min": tb["us_min"], "launches_timed": tb["launches"]}
     if B >= 64 and tiled_big:
         # dense-contraction regime: tensor roofline (fp16 operands; nominal fp16 peak = bf16 peak)
-        tf = 2.0 * B * Nb * Kb / (us_big * 1e-6) / 1e12
+        tf = 2.0 * B * qb.N * qb.K / (tb["us"] * 1e-6) / 1e12
         roofline = {"bound": "tensor", "achieved": tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": tf / peak_tf,
-                    "traffic": traffic, "peak_source": f"of {peak_src} (cuBLAS bf16 burst)", "kernel": kname,
-                    "layer": f"{layers[big][0]} {Nb}x{Kb}", "us_per_launch": us_big, "flops": 2.0 * B * Nb * Kb,
-                    "weight_GBps": layer_bytes(Nb, Kb, p, n) / us_big / 1e3}
+                    "peak_source": f"of {peak_src} (cuBLAS bf16 burst)", "flops": 2.0 * B * qb.N * qb.K,
+                    "weight_GBps": qb.bytes / tb["us"] / 1e3, **common}
     else:
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                    "traffic": traffic, "peak_source": f"of {peak_src}", "kernel": kname,
-                    "layer": f"{layers[big][0]} {Nb}x{Kb}", "us_per_launch": us_big, "algorithmic_bytes": alg,
-                    "frac_of_8TBps": achieved / 8000.0}
+                    "peak_source": f"of {peak_src}", "algorithmic_bytes": alg, "frac_of_8TBps": achieved / 8000.0, **common}
 
     detail = None
     if not args.no_detail and rank == 0:
         detail = {"layers": []}
-        for li, (name, N, K) in enumerate(layers):
-            if any(l["shape"] == f"{N}x{K}" and l["grid"] == f"p={pn[li][0]} n={pn[li][1]}" for l in detail["layers"]):
+        # one row per distinct (shape, grid) of the headline workload at its batch - and at the configuration's other
+        # batch (32 for the 70B shapes, 16 otherwise) - each with the parity of the timed output on sampled rows
+        other_B = 32 if args.workload == "llama-3.1-70b" else 16
+        seen = set()
+        for li, q in enumerate(qs):
+            if (q.N, q.K, q.pn) in seen:
                 continue
-            us, _ = kernel_time(li, descs[li], B)
-            wb = layer_bytes(N, K, *pn[li])
-            detail["layers"].append({"name": name, "shape": f"{N}x{K}", "grid": f"p={pn[li][0]} n={pn[li][1]}", "B": B, "us": round(us, 3),
-                                     "weight_GBps": round(wb / us / 1e3, 1), "frac_of_measured": round(wb / us / 1e3 / peak, 4)})
-        if B != 16:
-            us16, _ = kernel_time(big, db, 16)
-            wb = layer_bytes(Nb, Kb, p, n)
-            detail["batch16_largest_layer"] = {"us": round(us16, 3), "weight_GBps": round(wb / us16 / 1e3, 1),
-                                               "frac_of_measured": round(wb / us16 / 1e3 / peak, 4)}
+            seen.add((q.N, q.K, q.pn))
+            for Bk in sorted({B, other_B}):
+                if Bk == B:
+                    x32, xk = xs32[li], xs[li]
+                else:
+                    x32 = inputs.make_activations(Bk, q.K, inputs.activation_seed(cfg, Bk) + li)
+                    xk = torch.from_numpy(x32).to(dev).to(torch.bfloat16)
+                t = tb if (li == big and Bk == B) else time_product(hb, torch, stream, q, Bk, xk, reps=100)
+                par = parity_on_sampled_rows(hb, oracle, q, x32, t["y"], xi, grids64[q.pn])
+                detail["layers"].append(product_row(hb, q, Bk, t, peak, peak_tf, par))
+        detail["parity_bound"] = "max |y - y^| / max |y^| <= 2e-3 on 16 sampled rows of every timed layer, fp64 oracle on the device's codes"
+        worst = max(r["parity_max_rel"] for r in detail["layers"])
+        if worst > 2e-3:
+            raise SystemExit(f"parity re-check failed on a timed shape: {worst}")
+
+        # launch-latency floor: chains of kernels that do nothing, launched like the product kernels
+        detail["launch_floor_us"] = {
+            "one_block_per_sm_544_threads_227KB": round(launch_floor(hb, torch, stream, 148, 544, 232448), 3),
+            "one_small_block": round(launch_floor(hb, torch, stream, 1, 32, 0), 3)}
+        # the fit T = T0 + bytes / BW over the rows of the small-batch kernel at the headline batch
+        nbytes = {(f"{q.N}x{q.K}", f"p={q.pn[0]} n={q.pn[1]}"): q.bytes for q in qs}
+        pts = [(r["us"], nbytes[(r["shape"], r["grid"])]) for r in detail["layers"]
+               if r["B"] == B and r["kernel"] == "linear_stream_kernel"]
+        if len(pts) >= 3:
+            A = np.array([[1.0, b] for _, b in pts])
+            t0, slope = np.linalg.lstsq(A, np.array([u for u, _ in pts]), rcond=None)[0]
+            detail["fit"] = {"T0_us": round(float(t0), 3), "BW_GBps": round(1e-3 / float(slope), 1) if slope > 0 else None,
+                             "model": "us = T0 + bytes / BW over the layers of this set at the headline batch"}
 
     # ---- the same block with q/k/v and gate/up stored row-concatenated (rows are independent and the packed stream is
-    # ordered by row tile, so the concatenation of the packed buffers IS the packed concatenated matrix): 4 products
-    # and 4 rotations per block instead of 7 and 4.  Reported beside the per-layer launches, not instead of them.
-    if detail is not None and all(nm in names for nm in ("q", "k", "v", "gate", "up")) and len(set(pn)) == 1:
-        grid = grids[pn[0]]
+    # ordered by row tile, so the concatenation of the packed buffers IS the packed concatenated matrix): fewer, larger
+    # products per block.  Layers are merged only where they share a grid.  Reported beside the per-layer launches.
+    if detail is not None and all(nm in names for nm in ("q", "k", "v", "gate", "up")):
         idx = {nm: names.index(nm) for nm in names}
-        merged = [("qkv", [idx["q"], idx["k"], idx["v"]]), ("o", [idx["o"]]), ("gate_up", [idx["gate"], idx["up"]]),
-                  ("down", [idx["down"]])]
-        f_desc, f_packed, f_scales, f_y, f_ws, f_x = [], [], [], [], [], []
-        for nm, lis in merged:
+
+        def merge(group):
+            out = []
+            for li in group:
+                for m in out:
+                    if qs[m[0]].pn == qs[li].pn:
+                        m.append(li)
+                        break
+                else:
+                    out.append([li])
+            return out
+
+        merged = merge([idx["q"], idx["k"], idx["v"]]) + [[idx["o"]]] + merge([idx["gate"], idx["up"]]) + [[idx["down"]]]
+        f_q, f_packed, f_scales, f_y, f_ws, f_x = [], [], [], [], [], []
+        for lis in merged:
             Nf, Kf = sum(layers[li][1] for li in lis), layers[lis[0]][2]
-            d = hb.make_desc(p, n, Nf, Kf, xi)
-            f_desc.append(d)
-            f_packed.append([torch.cat([packed[li][c] for li in lis]) for c in range(copies)])
-            f_scales.append([torch.cat([scales[li][c] for li in lis]) for c in range(copies)])
+            d = hb.make_desc(qs[lis[0]].pn[0], qs[lis[0]].pn[1], Nf, Kf, xi)
+            f_q.append((d, qs[lis[0]].grid, "|".join(names[li] for li in lis)))
+            if len(lis) == 1:
+                f_packed.append(qs[lis[0]].packed[:copies])
+                f_scales.append(qs[lis[0]].scales[:copies])
+            else:
+                f_packed.append([torch.cat([qs[li].packed[c] for li in lis]) for c in range(copies)])
+                f_scales.append([torch.cat([qs[li].scales[c] for li in lis]) for c in range(copies)])
             f_y.append(torch.empty((B, Nf), dtype=torch.float32, device=dev))
             f_ws.append(torch.empty(hb.higgs_workspace_bytes(d, hb.HIGGS_OP_LINEAR, B), dtype=torch.uint8, device=dev))
             f_x.append(xs[lis[0]])
 
         def fused_step(i):
             c = i % copies
-            for j, d in enumerate(f_desc):
+            for j, (d, grid, _) in enumerate(f_q):
                 hb.higgs_linear(d, f_x[j], f_packed[j][c], f_scales[j][c], grid, workspace=f_ws[j], y=f_y[j])
 
         with torch.cuda.stream(stream):
@@ -546,61 +775,71 @@ def run_ours(args):
             for c in range(copies):
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g, stream=stream):
-                    fused_step(c)
+                    for k in range(spg):
+                        fused_step(c * spg + k)
                 fgraphs.append(g)
-        def run_fused(first, count):
-            for i in range(first, first + count):
-                fgraphs[i % copies].replay()
 
-        ms_f = timed(run_fused, args.steps, max(args.warmup, 3))
-        # the concatenated launch computes the same rows: compare with the per-layer outputs of the last plain step
+        def run_fused(first, count):
+            i = first
+            while count >= spg:
+                fgraphs[(i // spg) % copies].replay()
+                i += spg
+                count -= spg
+            for k in range(count):
+                fused_step(i + k)
+
+        ms_f = timed(run_fused, args.steps, warm)
+        # the concatenated launch computes the same rows: compare with the per-layer outputs of a plain step
         with torch.cuda.stream(stream):
             step(0)
             fused_step(0)
             stream.synchronize()
-        qkv = torch.cat([ys[idx["q"]], ys[idx["k"]], ys[idx["v"]]], dim=1)
-        err = float((f_y[0] - qkv).abs().max() / qkv.abs().max())
+        err = 0.0
+        for j, lis in enumerate(merged):
+            sep = torch.cat([ys[li] for li in lis], dim=1)
+            err = max(err, float((f_y[j] - sep).abs().max() / sep.abs().max()))
         detail["row_concatenated"] = {
             "ms_per_step": ms_f / args.steps, "value_GBps": aggregate_value(set_bytes, args.steps, ms_f, 1),
-            "launches_per_step": sum(hb.higgs_linear_launch_count(d, B) for d in f_desc),
-            "layers": [f"{nm} {d.N}x{d.K}" for (nm, _), d in zip(merged, f_desc)],
-            "qkv_vs_separate_max_rel": err}
+            "launches_per_step": sum(hb.higgs_linear_launch_count(d, B) for d, _, _ in f_q),
+            "layers": [f"{nm} {d.N}x{d.K} p={d.p} n={d.n}" for d, _, nm in f_q],
+            "max_rel_vs_separate_launches": err}
+        # the largest concatenated product alone
+        jbig = max(range(len(f_q)), key=lambda j: f_packed[j][0].numel())
+        if len(merged[jbig]) > 1:
+            d, grid, nm = f_q[jbig]
+            qcat = Quantized.from_buffers(nm, d, grid, f_packed[jbig], f_scales[jbig])
+            tcat = time_product(hb, torch, stream, qcat, B, f_x[jbig], reps=100)
+            detail["row_concatenated"]["largest"] = product_row(hb, qcat, B, tcat, peak, peak_tf)
+            del qcat
         del fgraphs, f_packed, f_scales
+
+    if detail is not None:
+        # free the headline workload's copies before the other configurations are encoded
+        for q in qs:
+            del q.packed[1:], q.scales[1:]
+        host_batches = None
+        graphs = None
+        torch.cuda.empty_cache()
+        detail["other_configurations"] = other_configurations(hb, torch, oracle, dev, stream, peak, peak_tf, fit_grid)
+        worst = max(r["parity_max_rel"] for r in detail["other_configurations"])
+        if worst > 2e-3:
+            raise SystemExit(f"parity re-check failed on a timed shape: {worst}")
 
     # ---- CPU baseline: the oracle as it stands on this machine's cores (rank 0, single-GPU runs only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        import oracle
-        rows = 256
-        smp = []
-        for li, (name, N, K) in enumerate(layers):
-            r = min(rows, N)
-            W = inputs.make_weights(r, K, inputs.weight_seed(cfg, li), bf16=True).astype(np.float64)
-            g64 = grids[pn[li]].cpu().numpy().astype(np.float64)
-            q = oracle.quantize(W, G, g64, xi)
-            smp.append((q.codes, oracle.round_scales_fp16(q.scales).astype(np.float64), xs_host[li].float().numpy().astype(np.float64), g64, r, K, pn[li]))
-        nb = sum(layer_bytes(r, K, *k) for *_, r, K, k in smp)
-        reps, t0 = 0, time.perf_counter()
-        while reps < 3 or time.perf_counter() - t0 < 10.0:
-            for codes, sc, x, g64, r, K, k in smp:
-                oracle.linear_dense(x, codes, sc, G, g64, xi)
-            reps += 1
-            if time.perf_counter() - t0 > 30.0:
-                break
-        dt = (time.perf_counter() - t0) / reps
-        cpu = {"value": nb / dt / 1e9, "unit": "GB/s", "cores": oracle.threads(), "kind": "oracle",
-               "sample": f"{rows} rows of each of the {len(layers)} layers (rows are independent), dequantise + fp64 matmul, {reps} passes"}
+        cpu = cpu_baseline(layers, pn, cfg, xi, grids64, B)
 
     if rank == 0:
+        wps = enc_weights / (enc_ms * 1e-3)
         line = {
             "metric": "higgs_linear_effective_weight_bandwidth", "value": value, "unit": "GB/s", "n_gpus": world,
-            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "steps": args.steps, "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f16xf16->f32", "data": "synthetic",
             "config": {"workload": f"{args.workload} layer set ({len(layers)} matrices), grid {grid_text}, g=1024, batch {B}",
                        "global_batch": B * world, "parallelism": f"replicas x{world}",
                        "l2": f"rotating {copies} weight copies ({copies * set_bytes / 1e6:.0f} MB > 126 MB L2)",
-                       "launch": "direct" if graphs is None else (f"CUDA graphs of {spg} consecutive steps (rotating weight copies), remainder from one-step graphs"
-                                                                  if graphs_multi is not None else "one CUDA graph per step"),
+                       "launch": "direct" if args.no_graph else f"CUDA graphs of {spg} consecutive steps over rotating weight copies ({args.steps // spg} replays timed)",
                        "step": "one transformer block: activation rotations (q/k/v and gate/up share theirs where the layout allows: the first layer of the group goes through higgs_linear_share, which for 1-2 tokens rotates inside its product kernel and leaves the result for the others; a layer with its own rotation has it fused likewise when K is not split) + 7 products"},
             "us_per_layer": ms_per_step * 1e3 / len(layers),
             "weight_bytes_per_step": set_bytes,
@@ -610,9 +849,8 @@ def run_ours(args):
             "clocks": clocks,
             "roofline": roofline,
             "cpu_baseline": cpu,
-            "quantize": {"weights_per_s": enc_weights / (enc_ms * 1e-3), "ms": enc_ms, "weights": enc_weights,
-                         "grid_fit_ms": grid_ms, "grid_fit_iters": int(grid_iters), "grid_mse": float(grid_mse),
-                         "roofline": encoder_roofline(enc_weights / (enc_ms * 1e-3), pn, clocks)},
+            "quantize": {"weights_per_s": wps, "ms": enc_ms, "weights": enc_weights, "grid_fit": grid_info,
+                         "rooflines": encoder_rooflines(wps, pn, [N * K for _, N, K in layers], clocks, peak, peak_src)},
             "detail": detail,
         }
         print(json.dumps(line))
