@@ -541,7 +541,7 @@ def run_ours(args):
     groups_of = {}
     for li, nm in enumerate(names):
         tiled = hb.higgs_rotated_layout(descs[li], B) > 0          # tensor-core path: never split
-        split = (not tiled) and hb.higgs_linear_k_splits(descs[li], B) > 1
+        split = (not tiled) and hb.higgs_linear_uses_atomics(descs[li], B)
         key = (share.get(nm) + f":{hb.higgs_rotated_layout(descs[li], B)}") if (share.get(nm) and not split) else None
         groups_of.setdefault(key if key else f"own{li}", []).append(li)
     xdags = {k: torch.empty(hb.higgs_rotated_bytes(descs[v[0]], B) // 2, dtype=torch.float16, device=dev)

@@ -200,13 +200,13 @@ int higgs_quantize(const higgs_desc* desc, const void* W, int w_dtype, const flo
  *   scales   device, tile-major fp16 scales as written by higgs_quantize
  *   grid     device, [n][p] fp32
  *   y        device, [B][N] row-major, y_dtype in {HIGGS_F32, HIGGS_BF16}
- * Kernels behind the call: for one or two tokens (K not split) a single kernel
+ * Kernels behind the call: for one or two tokens (K up to 8192) a single kernel
  * that rotates the activations in its prologue; up to 16 tokens a rotation
  * kernel and the small-batch product kernel; above that (and from 9 tokens
  * for layers above 32 M weights) a rotation kernel and the tcgen05 kernel.
- * When the small-batch kernel splits K over several thread blocks the partial
- * sums meet in fp32 atomics, so the last bits of y may differ from run to run;
- * every other path is bit-reproducible.  The one-call form and the two-call
+ * When the small-batch kernel splits K over more than two thread blocks the
+ * partial sums meet in fp32 atomics, so the last bits of y may differ from run
+ * to run (higgs_linear_uses_atomics); every other path is bit-reproducible.  The one-call form and the two-call
  * form below agree to fp16 rounding of x+ (the fused prologue orders the
  * butterflies differently), not bit for bit.
  */
@@ -360,10 +360,13 @@ int higgs_launch_floor(int32_t blocks, int32_t threads, size_t shared_bytes, voi
 int higgs_selftest_wait(int32_t which, uint32_t polls, int32_t* result_out, void* stream);
 
 /* Number of K ranges the product kernel assigns to different thread blocks for this shape and
- * batch (1 = not split).  For batches up to 16 a split product accumulates with fp32 atomics into a
- * cleared output (higgs_linear clears it inside its rotation kernel, higgs_linear_prerotated with a
- * memset), so its last bits depend on timing.  The tensor-core path (larger batches) sums the ranges
- * of a tile in a fixed order inside a thread-block cluster and needs no clearing. */
+ * batch (1 = not split), and whether those ranges meet in fp32 atomics.  For batches up to 16 two ranges are taken
+ * by the two blocks of a thread-block cluster, which sum their partial results in a fixed order through
+ * distributed shared memory; more than two accumulate with fp32 atomics into a cleared output (higgs_linear
+ * clears it inside its rotation kernel, higgs_linear_prerotated with a memset), so the last bits of such a
+ * result depend on timing: higgs_linear_uses_atomics returns 1 for exactly those calls.  The tensor-core path
+ * (larger batches) sums the ranges of a tile in a fixed order inside a cluster too. */
+int higgs_linear_uses_atomics(const higgs_desc* desc, int64_t B);
 int higgs_linear_k_splits(const higgs_desc* desc, int64_t B);
 
 /* Number of kernels one higgs_linear call enqueues for this shape and batch. */

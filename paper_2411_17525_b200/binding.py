@@ -29,7 +29,7 @@ EXPORTS = [
     "higgs_rotated_layout", "higgs_dequantize", "higgs_make_uniform_grid", "higgs_layer_error",
     "higgs_allocate_bits", "higgs_general_tuples", "higgs_quantize_general", "higgs_linear_host_batch",
     "higgs_linear_gather", "higgs_linear_share", "higgs_make_grid_seeded", "higgs_gaussian_samples", "higgs_shard_rows",
-    "higgs_launch_floor", "higgs_selftest_wait",
+    "higgs_launch_floor", "higgs_selftest_wait", "higgs_linear_uses_atomics",
 ]
 
 
@@ -89,6 +89,8 @@ def _load() -> ctypes.CDLL:
     lib.higgs_rotated_layout.argtypes = [P, i64]
     lib.higgs_linear_k_splits.restype = i32
     lib.higgs_linear_k_splits.argtypes = [P, i64]
+    lib.higgs_linear_uses_atomics.restype = i32
+    lib.higgs_linear_uses_atomics.argtypes = [P, i64]
     lib.higgs_linear_launch_count.restype = i32
     lib.higgs_linear_launch_count.argtypes = [P, i64, i32]
     lib.higgs_linear_static.restype = i32
@@ -433,6 +435,10 @@ def higgs_rotated_layout(desc: higgs_desc, B: int) -> int:
 
 def higgs_linear_k_splits(desc: higgs_desc, B: int) -> int:
     return int(lib.higgs_linear_k_splits(ctypes.byref(desc), int(B)))
+
+
+def higgs_linear_uses_atomics(desc: higgs_desc, B: int) -> bool:
+    return bool(lib.higgs_linear_uses_atomics(ctypes.byref(desc), B))
 
 
 def higgs_linear_launch_count(desc: higgs_desc, B: int, y_dtype: int = HIGGS_F32) -> int:

@@ -232,8 +232,7 @@ int higgs_rotate_activations(const higgs_desc* d, const void* x, int64_t B, void
 // Shared tail of higgs_linear / higgs_linear_prerotated: D2-D5 on rotated activations.
 static int linear_tail(const higgs_desc* d, const __half* xdag, int64_t B, const void* packed, const void* scales,
                        const float* grid, void* y, int y_dtype, float* y32, bool target_is_clear, cudaStream_t st) {
-    const int chunks = linear_k_chunks(*d, B);
-    const bool split = chunks > 1;
+    const bool split = linear_uses_atomics(*d, B);
     float* acc_target = split ? (y_dtype == HIGGS_F32 ? static_cast<float*>(y) : y32) : nullptr;
     if (split && !target_is_clear) {
         if (cudaMemsetAsync(acc_target, 0, (size_t)B * d->N * sizeof(float), st) != cudaSuccess) return HIGGS_ERR_CUDA;
@@ -286,7 +285,7 @@ int higgs_linear(const higgs_desc* d, const void* x, int64_t B, const void* pack
     }
     __half* xdag = static_cast<__half*>(workspace);
     float* y32 = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up((size_t)B * d->K * 2, 256));
-    const bool split = linear_k_chunks(*d, B) > 1;
+    const bool split = linear_uses_atomics(*d, B);
     float* acc_target = split ? (y_dtype == HIGGS_F32 ? static_cast<float*>(y) : y32) : nullptr;
     // D1: rotate the activations once (and clear the accumulation target of a K-split product)
     rc = launch_rht_activations(*d, x, B, xdag, acc_target, split ? (size_t)B * d->N : 0, st);
@@ -338,7 +337,7 @@ int higgs_linear_gather(const higgs_desc* d, const void* x, int64_t B, const voi
         return launch_linear_mma(*d, nullptr, B, packed, scales, grid, dst[0], ld, mode, st, x, &more);
     __half* xdag = static_cast<__half*>(workspace);
     float* y32 = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + align_up((size_t)B * d->K * 2, 256));
-    const bool split = linear_k_chunks(*d, B) > 1;
+    const bool split = linear_uses_atomics(*d, B);
     // D1 (and, for a K-split product, the cleared contiguous fp32 accumulator in the workspace)
     rc = launch_rht_activations(*d, x, B, xdag, split ? y32 : nullptr, split ? (size_t)B * d->N : 0, st);
     if (rc != HIGGS_OK) return rc;
@@ -461,11 +460,17 @@ int higgs_linear_k_splits(const higgs_desc* d, int64_t B) {
     return linear_k_chunks(*d, B);
 }
 
+int higgs_linear_uses_atomics(const higgs_desc* d, int64_t B) {
+    if (check_desc(d) != HIGGS_OK || B < 1 || d->N == 0 || d->K == 0) return 0;
+    if (tc_eligible(*d, B)) return 0;
+    return linear_uses_atomics(*d, B) ? 1 : 0;
+}
+
 int higgs_linear_launch_count(const higgs_desc* d, int64_t B, int y_dtype) {
     if (check_desc(d) != HIGGS_OK || B < 1 || d->N == 0) return 0;
     if (tc_eligible(*d, B)) return 2;
     if (linear_fused_eligible(*d, B)) return 1;
-    const bool split = linear_k_chunks(*d, B) > 1;
+    const bool split = linear_uses_atomics(*d, B);
     return 1 + (int)((B + 15) / 16) + ((split && y_dtype == HIGGS_BF16) ? 1 : 0);
 }
 

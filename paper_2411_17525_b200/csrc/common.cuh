@@ -102,6 +102,27 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// The same with the blocks grouped into thread-block clusters of `cluster_x` along x.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                      unsigned cluster_x, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = cluster_x;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---- in-register / warp-shuffle fast Walsh-Hadamard transform over 1024 ----
 // A warp owns one group.  Lane l holds 32 values v[r], r = c*8 + e, standing
 // for element index  idx = c*256 + l*8 + e  (c in 0..3, e in 0..7), so that a
@@ -184,6 +205,7 @@ int launch_encode_general(int p, int n, int64_t N, int64_t K, uint64_t xi, const
                           uint16_t* codes, void* scales, double* sums, cudaStream_t st);
 int launch_uniform_grid(int n, float* grid_out, float* step_out, float* mse_out, cudaStream_t st);
 int linear_k_chunks(const higgs_desc& d, int64_t B);
+bool linear_uses_atomics(const higgs_desc& d, int64_t B);   // K ranges meet in fp32 atomics: the output must be cleared first
 // tensor-core path (B > 16)
 bool tc_eligible(const higgs_desc& d, int64_t B);
 size_t tc_workspace_bytes(const higgs_desc& d, int64_t B);

@@ -253,9 +253,14 @@ __device__ __noinline__ void gather_store1(const StreamParams* prm, int64_t o, f
 // x+ = (H / sqrt(g)) diag(sign) x) - the four warps that own the four 256-input slices of a 1024-group transform it
 // together: butterflies over a lane's 8 values in registers, over the 32 lanes by shuffles, over the 4 warps through
 // shared memory - so that no rotation kernel (and no hand-over between two dependent launches) precedes the product.
-template <int NB, int KS, int FMT, bool FUSED>
+// PAIR: K is cut into two chunks that the two blocks of a thread-block cluster take (grid = 2 x parts, cluster = 2).
+// Both work on the same row tiles; the partial tiles of item j of both blocks go - through distributed shared memory -
+// to the block with rank j % 2, whose flusher sums the 2 NS of them in a fixed order and writes y: no atomics, no
+// cleared output, bit-reproducible, and the two flushers share the work.
+template <int NB, int KS, int FMT, bool FUSED, bool PAIR>
 __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(const __grid_constant__ StreamParams prm) {
     constexpr bool SIX = FMT == 1, NIB = FMT == 2, B8 = FMT == 3;
+    constexpr int kHomes = PAIR ? 2 : 1;          // blocks that sum and write items
     static_assert(!FUSED || (NB == 1 && KS == 256), "the fused rotation maps one warp to one 256-input slice");
     constexpr uint32_t kPieceStride = NIB ? 128u : 256u;     // bytes between consecutive 128-byte pieces of the partial tiles
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -303,7 +308,7 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
 
     // ---- shared memory map (all offsets derived from the runtime base address) ----
     //   [base, base+4 KB)    ring mbarriers (0..1023), item mbarriers and
-    //                        recycle counters of the partial-tile slots (2048..2559), abort flag (2560)
+    //                        recycle counters of the partial-tile slots (2048..2559), abort flag (2688)
     //   [base+4 KB, lut)     ring slots, region A
     //   [lut, lut+64 KB)     table rows of 256 B: bytes 0..127 = the entry replicated per lane,
     //                        bytes 128..255 = one 32-float piece of an accumulator tile
@@ -316,8 +321,8 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     if (base != kAssumedBase) ring_layout(base, kSlotBytes, kTailReserve, &lut, &D, &warps_in_A);
     const uint32_t bars = base;
     const uint32_t item_bars = base + 2048u;                                        // [kMaxAccSlots] mbarriers, NS arrivals each
-    volatile int* recycled = reinterpret_cast<volatile int*>(smem_raw + 2048 + 8 * kMaxAccSlots);   // [kMaxAccSlots] generations
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + 2560);
+    volatile int* recycled = reinterpret_cast<volatile int*>(smem_raw + 2048 + 8 * kMaxAccSlots);   // [kHomes][kMaxAccSlots] generations
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + 2688);
     const uint32_t ringA = base + kSmallBytes, ringB = lut + kLutBytes;
     // Every warp's D slots are contiguous and lie entirely in one region, so slot d is one multiply-add away.
     const uint32_t slot0 = warp < warps_in_A ? ringA + (uint32_t)(warp * D) * kSlotBytes
@@ -331,7 +336,9 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     const uint32_t tiles = (uint32_t)(prm.N / kRowTile);
     const uint32_t parts = (uint32_t)prm.parts;
     auto div_parts = [&](uint32_t x) { return (uint32_t)(((unsigned long long)x * prm.parts_magic) >> (32 + prm.parts_shift)); };
-    const uint32_t chunk_begin_u = div_parts(blockIdx.x), part = blockIdx.x - chunk_begin_u * parts;   // this block's K-chunk
+    // this block's K-chunk: in a cluster pair it is the block's rank in the cluster
+    const uint32_t chunk_begin_u = PAIR ? (blockIdx.x & 1u) : div_parts(blockIdx.x);
+    const uint32_t part = PAIR ? (blockIdx.x >> 1) : blockIdx.x - chunk_begin_u * parts;
     const int chunk_begin = (int)chunk_begin_u;
     const int rt_begin = (int)div_parts(tiles * part);
     const int n_items = (int)div_parts(tiles * (part + 1)) - rt_begin;                                 // its row tiles
@@ -353,7 +360,7 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     const int acc_shift = prm.acc_shift;
     const uint32_t part0 = NIB ? base + kMaxDynSmem - kNibbleTileBytes : lut + 128u;
     const uint32_t tile_stride = (uint32_t)tile_pieces * kPieceStride; // bytes between consecutive tiles
-    const uint32_t q_stride = tile_stride << log_ns;                   // bytes between consecutive item slots
+    const uint32_t q_stride = (tile_stride << log_ns) * (uint32_t)kHomes; // bytes between consecutive item slots (kHomes x NS tiles)
 
     // ---- ring barriers, then the first copies ----
     if (lane == 0 && !flusher) {
@@ -361,8 +368,9 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     }
     __syncwarp();
     if (flusher) {
-        mbar_init(item_bars + 8u * lane, (uint32_t)NS);
+        mbar_init(item_bars + 8u * lane, PAIR ? 1u : (uint32_t)NS);      // pair: the flusher's expect_tx; the tiles count as bytes
         recycled[lane] = 0;
+        if (PAIR) recycled[kMaxAccSlots + lane] = 0;
         if (lane == 0) *abort_flag = 0;
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -509,7 +517,7 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
         __syncwarp();
         // Other layers that read the same x (k and v after q, up after gate) can skip their rotation: one warp per slice
         // of block 0 leaves the slice, already in the rotation kernel's fragment order, in global memory.
-        if (prm.xdag_emit != nullptr && blockIdx.x == 0) {
+        if (prm.xdag_emit != nullptr && part == 0) {
 #pragma unroll
             for (int b = 0; b < 2; ++b) {
                 if (b < prm.B) {
@@ -556,28 +564,57 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
         }
         __syncthreads();     // every warp has its B fragments: the scratch area may now take partial tiles
     }
-    // ---- flusher warp: one item after the other, in item order ----
+    // (pair) bytes of the 2 NS partial tiles of an item: what the item's barrier waits for
+    const uint32_t item_tx = (uint32_t)(2 * NS * 16 * prm.B * 4);
+    if (PAIR) {
+        if (flusher) mbar_expect_tx(item_bars + 8u * lane, item_tx);      // first use of every slot
+        // the peer's barriers and counters are initialised and its scratch area is free before anything is sent to it
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    }
+    uint32_t my_rank = 0;
+    if (PAIR) asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(my_rank));
+    // ---- flusher warp: one item after the other, in item order (in a cluster pair: the items of this block's rank) ----
     if (flusher) {
-        int f_rt = rt_begin;
-        for (int j = 0; j < n_items; ++j) {
-            const int q = j & (acc_slots - 1), gen = j >> acc_shift;
-            if (!mbar_wait_relaxed(item_bars + 8u * q, (uint32_t)(gen & 1), abort_flag)) return;
-            if (prm.B <= 2) {
-                // one or two tokens: a tile is one 128-byte piece and lane = column * 16 + row owns one output: the NS
-                // partial values of its element are summed in slice order
-                const uint32_t a0 = part0 + (uint32_t)q * q_stride + (uint32_t)(lane * 4);
-                float part[16];
-#pragma unroll
-                for (int ns = 0; ns < 16; ++ns) {
-                    uint32_t v;
-                    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(a0 + (uint32_t)(ns < NS ? ns : 0) * tile_stride));
-                    part[ns] = __uint_as_float(v);
+        constexpr int kPasses = PAIR ? 2 : 1;          // 16 partial tiles per pass
+        const int NT = NS * kHomes;                    // partial tiles per item
+        for (int j = (int)my_rank; j < n_items; j += kHomes) {
+            const int jj = PAIR ? (j >> 1) : j;
+            const int q = jj & (acc_slots - 1), gen = jj >> acc_shift;
+            const int f_rt = rt_begin + j;
+            if (!mbar_wait_relaxed(item_bars + 8u * q, (uint32_t)(gen & 1), abort_flag)) break;
+            auto recycle = [&]() {      // the partial tiles are in registers: hand the slot back (to both blocks of a pair)
+                __syncwarp();
+                if (lane == 0) {
+                    if (PAIR) mbar_expect_tx(item_bars + 8u * q, item_tx);     // the slot's next use, before anybody may send to it
+                    recycled[my_rank * kMaxAccSlots + q] = gen + 1;
+                    if (PAIR) {
+                        const uint32_t local = base + 2048u + 8u * kMaxAccSlots + 4u * (my_rank * kMaxAccSlots + (uint32_t)q);
+                        uint32_t remote;
+                        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(my_rank ^ 1u));
+                        asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(remote), "r"((uint32_t)(gen + 1)) : "memory");
+                    }
                 }
+            };
+            if (prm.B <= 2) {
+                // one or two tokens: a tile is one 128-byte piece and lane = column * 16 + row owns one output: the
+                // partial values of its element are summed in tile order (chunk, then slice)
+                const uint32_t a0 = part0 + (uint32_t)q * q_stride + (uint32_t)(lane * 4);
                 float sum = 0.f;
 #pragma unroll
-                for (int ns = 0; ns < 16; ++ns) sum += ns < NS ? part[ns] : 0.f;
-                __syncwarp();
-                if (lane == 0) recycled[q] = gen + 1;
+                for (int pass = 0; pass < kPasses; ++pass) {
+                    float part[16];
+#pragma unroll
+                    for (int ns = 0; ns < 16; ++ns) {
+                        const int tile = pass * 16 + ns;
+                        uint32_t v;
+                        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(a0 + (uint32_t)(tile < NT ? tile : 0) * tile_stride));
+                        part[ns] = __uint_as_float(v);
+                    }
+#pragma unroll
+                    for (int ns = 0; ns < 16; ++ns) sum += pass * 16 + ns < NT ? part[ns] : 0.f;
+                }
+                recycle();
                 const int col = lane >> 4, row = lane & 15;
                 if (col < prm.B) {
                     const int64_t o = (int64_t)col * prm.ldy + (int64_t)f_rt * 16 + row;
@@ -591,7 +628,6 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
                         asm volatile("red.global.add.f32 [%0], %1;" ::"l"(static_cast<float*>(prm.y) + o), "f"(sum) : "memory");
                     }
                 }
-                ++f_rt;
                 continue;
             }
             float4 sums[NB];
@@ -600,28 +636,32 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
                 const int e = (qq * 32 + lane) * 4;      // 4 consecutive rows of one column
                 sums[qq] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if ((e >> 4) < prm.B) {
-                    // unconditional loads (clamped slice index), issued back to back; unused ones are dropped below
-                    uint4 raw[16];
-#pragma unroll
-                    for (int ns = 0; ns < 16; ++ns)
-                        raw[ns] = lds128(part0 + (uint32_t)q * q_stride + (uint32_t)(ns < NS ? ns : 0) * tile_stride +
-                                         (uint32_t)(e >> 5) * kPieceStride + (uint32_t)((e & 31) * 4));
                     float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-                    for (int ns = 0; ns < 16; ++ns) {
-                        const float m = ns < NS ? 1.f : 0.f;
-                        sum.x = fmaf(m, __uint_as_float(raw[ns].x), sum.x);
-                        sum.y = fmaf(m, __uint_as_float(raw[ns].y), sum.y);
-                        sum.z = fmaf(m, __uint_as_float(raw[ns].z), sum.z);
-                        sum.w = fmaf(m, __uint_as_float(raw[ns].w), sum.w);
+                    for (int pass = 0; pass < kPasses; ++pass) {
+                        // unconditional loads (clamped tile index), issued back to back; unused ones are dropped below
+                        uint4 raw[16];
+#pragma unroll
+                        for (int ns = 0; ns < 16; ++ns) {
+                            const int tile = pass * 16 + ns;
+                            raw[ns] = lds128(part0 + (uint32_t)q * q_stride + (uint32_t)(tile < NT ? tile : 0) * tile_stride +
+                                             (uint32_t)(e >> 5) * kPieceStride + (uint32_t)((e & 31) * 4));
+                        }
+#pragma unroll
+                        for (int ns = 0; ns < 16; ++ns) {
+                            const float m = pass * 16 + ns < NT ? 1.f : 0.f;
+                            sum.x = fmaf(m, __uint_as_float(raw[ns].x), sum.x);
+                            sum.y = fmaf(m, __uint_as_float(raw[ns].y), sum.y);
+                            sum.z = fmaf(m, __uint_as_float(raw[ns].z), sum.z);
+                            sum.w = fmaf(m, __uint_as_float(raw[ns].w), sum.w);
+                        }
                     }
                     sums[qq] = sum;
                 }
             }
             // The partial tiles are in registers (the sums above consumed every load): hand the slot back first,
             // then write y.  No fence follows the global write, so the warp never waits for its round trip.
-            __syncwarp();
-            if (lane == 0) recycled[q] = gen + 1;
+            recycle();
 #pragma unroll
             for (int qq = 0; qq < NB; ++qq) {
                 const int e = (qq * 32 + lane) * 4;
@@ -644,14 +684,11 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
                     }
                 }
             }
-            ++f_rt;
         }
-        return;
-    }
-
+    } else {
     // ---- main loop: this warp's tasks ----
     const uint32_t lut_lane = lut + lane * (NIB ? 8 : 4);
-    const uint32_t part_lane = part0 + (uint32_t)slice * tile_stride + (uint32_t)t * kPieceStride + (uint32_t)(g * 4);
+    const uint32_t part_lane = part0 + (uint32_t)((PAIR ? (chunk_begin << log_ns) : 0) + slice) * tile_stride + (uint32_t)t * kPieceStride + (uint32_t)(g * 4);
     int d = 0;
     uint32_t ph = 0;
     bool ok = true;
@@ -711,9 +748,12 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
         const float s_lo = __half2float(__ushort_as_half(slo16));
         const float s_hi = __half2float(__ushort_as_half(shi16));
 
-        // partial-tile slot of this item: slot q, generation gen; wait (rarely) until its previous user was flushed
-        const int q = c_item & (acc_slots - 1), gen = c_item >> acc_shift;
-        for (uint32_t it = 0; recycled[q] != gen; ++it) {
+        // partial-tile slot of this item: slot q, generation gen, in the block that flushes the item (in a cluster pair:
+        // the block of rank item % 2); wait (rarely) until its previous user was flushed
+        const uint32_t home = PAIR ? (uint32_t)(c_item & 1) : 0u;
+        const int cj = PAIR ? (c_item >> 1) : c_item;
+        const int q = cj & (acc_slots - 1), gen = cj >> acc_shift;
+        for (uint32_t it = 0; recycled[home * kMaxAccSlots + q] != gen; ++it) {
             if ((it & 63u) == 63u && (*abort_flag || it > kWaitLimit)) {
                 if (!*abort_flag) { *abort_flag = 1; atomicExch(&g_device_status, (int)HIGGS_ERR_TIMEOUT); }
                 ok = false;
@@ -722,7 +762,17 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
         }
         if (!ok) break;
         // this lane's elements of the tile: (col 2t, row g) at piece t, float g; the others at fixed offsets
-        const uint32_t pa = part_lane + (uint32_t)q * q_stride;
+        uint32_t pa = part_lane + (uint32_t)q * q_stride, ibar = item_bars + 8u * q;
+        if (PAIR) {       // the same offsets in the home block's shared memory (its own or the peer's)
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(pa) : "r"(pa), "r"(home));
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ibar) : "r"(ibar), "r"(home));
+        }
+        auto park = [&](uint32_t addr, float v) {
+            // pair: an asynchronous store into the home block's shared memory that counts its 4 bytes on the item's barrier
+            if (PAIR) asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
+                                   ::"r"(addr), "r"(__float_as_uint(v)), "r"(ibar) : "memory");
+            else asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+        };
 #pragma unroll
         for (int nb = 0; nb < NB; ++nb) {
             const int c0 = nb * 8 + 2 * t;           // this lane holds columns c0, c0+1 of rows g and g+8
@@ -731,17 +781,18 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
             const float v2 = (acc4[0][nb][2] + acc4[1][nb][2]) + (acc4[2][nb][2] + acc4[3][nb][2]);
             const float v3 = (acc4[0][nb][3] + acc4[1][nb][3]) + (acc4[2][nb][3] + acc4[3][nb][3]);
             if (c0 < prm.B) {                        // only the B valid columns exist
-                asm volatile("st.shared.f32 [%0], %1;" ::"r"(pa + (uint32_t)(nb * 4) * kPieceStride), "f"(v0 * s_lo) : "memory");
-                asm volatile("st.shared.f32 [%0], %1;" ::"r"(pa + (uint32_t)(nb * 4) * kPieceStride + 32u), "f"(v2 * s_hi) : "memory");
+                park(pa + (uint32_t)(nb * 4) * kPieceStride, v0 * s_lo);
+                park(pa + (uint32_t)(nb * 4) * kPieceStride + 32u, v2 * s_hi);
             }
             if (c0 + 1 < prm.B) {
-                asm volatile("st.shared.f32 [%0], %1;" ::"r"(pa + (uint32_t)(nb * 4) * kPieceStride + 64u), "f"(v1 * s_lo) : "memory");
-                asm volatile("st.shared.f32 [%0], %1;" ::"r"(pa + (uint32_t)(nb * 4) * kPieceStride + 96u), "f"(v3 * s_hi) : "memory");
+                park(pa + (uint32_t)(nb * 4) * kPieceStride + 64u, v1 * s_lo);
+                park(pa + (uint32_t)(nb * 4) * kPieceStride + 96u, v3 * s_hi);
             }
         }
-        __syncwarp();
-        if (lane == 0) {                         // release: the partial tile is visible before the arrival counts
-            asm volatile("{ .reg .b64 st; mbarrier.arrive.shared::cta.b64 st, [%0]; }" ::"r"(item_bars + 8u * q) : "memory");
+        if (!PAIR) {
+            __syncwarp();
+            if (lane == 0)                           // release: the partial tile is visible before the arrival counts
+                asm volatile("{ .reg .b64 st; mbarrier.arrive.shared::cta.b64 st, [%0]; }" ::"r"(ibar) : "memory");
         }
         c_item += PG;
     }
@@ -751,6 +802,13 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
             for (uint32_t it = 0; it < kWaitLimit && !mbar_try(full_bar(d), ph); ++it) {}
             if (++d == D) { d = 0; ph ^= 1u; }
         }
+    }
+    }   // compute warps
+    if (PAIR) {
+        // neither block of the pair leaves while the other may still write into its shared memory
+        __syncwarp();
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
     }
 }
 
@@ -789,13 +847,38 @@ int sm_count() {
 
 struct Plan {
     int nb, ks, ck, chunks, parts, blocks;
+    bool pair;           // two K-chunks taken by the two blocks of a cluster (fixed-order sum, no atomics)
     int64_t items;
 };
 
+// Cluster pairs of the product kernel that the device can hold at once (0 if clusters of two such blocks cannot be
+// scheduled, e.g. on a partitioned device); every instantiation has the same block shape and shared memory.
+int pair_capacity() {
+    static int cached[64] = {0};
+    const int v = device_once(cached, [] {
+        auto kernel = linear_stream_kernel<1, 256, 0, false, true>;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMaxDynSmem) != cudaSuccess) return -1;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * 74);
+        cfg.blockDim = dim3((kWarps + 1) * 32);
+        cfg.dynamicSmemBytes = kMaxDynSmem;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n < 1) return -1;
+        return n;
+    });
+    return v > 0 ? v : 0;
+}
+
 // Picks the item width CK (inputs per item).  A block never leaves its K-chunk (its B fragments are loaded
 // once), so the grid is chunks x parts with parts = floor(SMs / chunks).  The score is the fraction of the
-// busiest block's time that is useful; splitting K is penalised because the partial results then meet in global
-// atomics and the output must be cleared first.
+// busiest block's time that is useful.  Two chunks are taken by cluster pairs (a fixed-order sum through
+// distributed shared memory); more than two meet in global atomics, for which the output must be cleared first:
+// that is penalised.
 Plan make_plan(const higgs_desc& d, int64_t B) {
     Plan best{};
     const int nb = B <= 8 ? 1 : 2;
@@ -808,15 +891,17 @@ Plan make_plan(const higgs_desc& d, int64_t B) {
         if (ck / ks > kWarps) continue;
         const int chunks = (int)(d.K / ck);
         int64_t parts = sms / chunks;
+        const bool pair = chunks == 2 && d.K > (int64_t)kWarps * ks && pair_capacity() > 0;
+        if (pair && parts > pair_capacity()) parts = pair_capacity();
         if (parts < 1) parts = 1;
         if (parts > tiles) parts = tiles;
         const int64_t per = (tiles + parts - 1) / parts;          // row tiles of the busiest block
         const double eff = (double)tiles * chunks / (double)(per * sms);
         // every extra K-chunk adds a pass of atomics over y and shortens the items (more bookkeeping per byte)
-        const double score = eff * (chunks == 1 ? 1.0 : 0.45 / (1.0 + 0.04 * (chunks - 2)));
+        const double score = eff * (chunks == 1 ? 1.0 : pair ? 0.95 : 0.45 / (1.0 + 0.04 * (chunks - 2)));
         if (score > best_score) {
             best_score = score;
-            best.nb = nb; best.ks = ks; best.ck = ck; best.chunks = chunks;
+            best.nb = nb; best.ks = ks; best.ck = ck; best.chunks = chunks; best.pair = pair;
             best.parts = (int)parts; best.blocks = (int)(parts * chunks); best.items = tiles * chunks;
         }
     }
@@ -824,14 +909,19 @@ Plan make_plan(const higgs_desc& d, int64_t B) {
 }
 
 template <int NB, int KS, int FMT, bool FUSED = false>
-int launch_one(const StreamParams& prm, int blocks, cudaStream_t st) {
+int launch_one(const StreamParams& prm, int blocks, bool pair, cudaStream_t st) {
     static int configured[64] = {0};       // 1 = attribute set, -1 = failed (per instantiation and device)
     const int ok = device_once(configured, [] {
-        return cudaFuncSetAttribute(linear_stream_kernel<NB, KS, FMT, FUSED>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    (int)kMaxDynSmem) == cudaSuccess ? 1 : -1;
+        return (cudaFuncSetAttribute(linear_stream_kernel<NB, KS, FMT, FUSED, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)kMaxDynSmem) == cudaSuccess &&
+                cudaFuncSetAttribute(linear_stream_kernel<NB, KS, FMT, FUSED, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)kMaxDynSmem) == cudaSuccess) ? 1 : -1;
     });
     if (ok < 0) return HIGGS_ERR_CUDA;
-    return cuda_status(launch_pdl(linear_stream_kernel<NB, KS, FMT, FUSED>, dim3((unsigned)blocks), dim3((kWarps + 1) * 32),
+    if (pair)
+        return cuda_status(launch_pdl_cluster(linear_stream_kernel<NB, KS, FMT, FUSED, true>, dim3((unsigned)blocks),
+                                              dim3((kWarps + 1) * 32), kMaxDynSmem, st, 2u, prm));
+    return cuda_status(launch_pdl(linear_stream_kernel<NB, KS, FMT, FUSED, false>, dim3((unsigned)blocks), dim3((kWarps + 1) * 32),
                                   kMaxDynSmem, st, prm));
 }
 
@@ -839,9 +929,17 @@ int launch_one(const StreamParams& prm, int blocks, cudaStream_t st) {
 
 int linear_k_chunks(const higgs_desc& d, int64_t B) { return make_plan(d, B > 16 ? 16 : B).chunks; }
 
-// The rotation can be fused into the product kernel for one or two tokens when K is not split over thread blocks.
+bool linear_uses_atomics(const higgs_desc& d, int64_t B) {
+    const Plan pl = make_plan(d, B > 16 ? 16 : B);
+    return pl.chunks > 1 && !pl.pair;
+}
+
+// The rotation can be fused into the product kernel for one or two tokens when every block owns whole 1024-groups and
+// the K ranges do not meet in atomics (one chunk, or the two chunks of a cluster pair).
 bool linear_fused_eligible(const higgs_desc& d, int64_t B) {
-    return B >= 1 && B <= 2 && d.N > 0 && make_plan(d, B).chunks == 1;
+    if (!(B >= 1 && B <= 2 && d.N > 0)) return false;
+    const Plan pl = make_plan(d, B);
+    return pl.chunks == 1 || pl.pair;
 }
 
 // y_mode: 0 store fp32, 1 store bf16, 2 atomicAdd fp32 (target must be zero).  B <= 16.
@@ -851,6 +949,7 @@ int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const 
     if (d.N == 0) return HIGGS_OK;
     if (more && more->count > 0 && (y_mode == 2 || more->count > kMaxGather - 1)) return HIGGS_ERR_INVALID_ARG;
     const Plan pl = make_plan(d, B);
+    if (pl.pair && y_mode == 2) y_mode = 0;          // a cluster pair sums in shared memory and stores
     if (pl.items == 0) return HIGGS_ERR_UNSUPPORTED;
     // the kernel's work split is 32-bit arithmetic: (row tiles) x (blocks per K-chunk) must stay below 2^31
     if ((d.N / kRowTile) * (int64_t)(pl.parts + 1) >= ((int64_t)1 << 31)) return HIGGS_ERR_UNSUPPORTED;
@@ -884,7 +983,7 @@ int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const 
     prm.log_ns = 0;
     while ((1 << prm.log_ns) < ns) ++prm.log_ns;
     prm.tile_pieces = (16 * (int)B + 31) >> 5;
-    int acc_slots = 256 / (ns * prm.tile_pieces), p2 = 1;
+    int acc_slots = 256 / (ns * (pl.pair ? 2 : 1) * prm.tile_pieces), p2 = 1;
     while (p2 * 2 <= acc_slots && p2 < kMaxAccSlots) p2 *= 2;
     prm.acc_slots = p2;
     prm.acc_shift = 0;
@@ -893,13 +992,13 @@ int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const 
     ring_layout(kAssumedBase, (uint32_t)(six ? pl.ks * 6 : nib ? pl.ks * 4 : b8 ? pl.ks * 16 : pl.ks * 8) + 64u,
                 nib ? kNibbleTileBytes : 0u, &lut_unused, &prm.depth, &prm.warps_in_a);
     if (fused)
-        return six ? launch_one<1, 256, 1, true>(prm, pl.blocks, st) : nib ? launch_one<1, 256, 2, true>(prm, pl.blocks, st)
-             : b8 ? launch_one<1, 256, 3, true>(prm, pl.blocks, st) : launch_one<1, 256, 0, true>(prm, pl.blocks, st);
+        return six ? launch_one<1, 256, 1, true>(prm, pl.blocks, pl.pair, st) : nib ? launch_one<1, 256, 2, true>(prm, pl.blocks, pl.pair, st)
+             : b8 ? launch_one<1, 256, 3, true>(prm, pl.blocks, pl.pair, st) : launch_one<1, 256, 0, true>(prm, pl.blocks, pl.pair, st);
     if (pl.nb == 1)
-        return six ? launch_one<1, 256, 1>(prm, pl.blocks, st) : nib ? launch_one<1, 256, 2>(prm, pl.blocks, st)
-             : b8 ? launch_one<1, 256, 3>(prm, pl.blocks, st) : launch_one<1, 256, 0>(prm, pl.blocks, st);
-    return six ? launch_one<2, 128, 1>(prm, pl.blocks, st) : nib ? launch_one<2, 128, 2>(prm, pl.blocks, st)
-         : b8 ? launch_one<2, 128, 3>(prm, pl.blocks, st) : launch_one<2, 128, 0>(prm, pl.blocks, st);
+        return six ? launch_one<1, 256, 1>(prm, pl.blocks, pl.pair, st) : nib ? launch_one<1, 256, 2>(prm, pl.blocks, pl.pair, st)
+             : b8 ? launch_one<1, 256, 3>(prm, pl.blocks, pl.pair, st) : launch_one<1, 256, 0>(prm, pl.blocks, pl.pair, st);
+    return six ? launch_one<2, 128, 1>(prm, pl.blocks, pl.pair, st) : nib ? launch_one<2, 128, 2>(prm, pl.blocks, pl.pair, st)
+         : b8 ? launch_one<2, 128, 3>(prm, pl.blocks, pl.pair, st) : launch_one<2, 128, 0>(prm, pl.blocks, pl.pair, st);
 }
 
 // A K-split product accumulates into a contiguous fp32 [B][N]; this spreads it to the gathered destinations.

@@ -300,7 +300,7 @@ def test_linear_share_leaves_the_rotated_activations(N, K, B):
     assert hb.higgs_device_status() == hb.HIGGS_OK
     if hb.higgs_rotated_layout(d, B) == 0:            # (the blocked tensor-core layout has padding tokens nobody writes)
         assert torch.equal(xd.view(torch.int16), xd_ref.view(torch.int16))
-    if hb.higgs_linear_k_splits(d, B) == 1 or hb.higgs_rotated_layout(d, B) > 0:
+    if not hb.higgs_linear_uses_atomics(d, B):
         assert torch.equal(y, y_ref)
     else:
         assert U.linear_error(y.cpu().numpy(), y_ref.cpu().numpy().astype(np.float64)) <= 1e-5
@@ -356,7 +356,7 @@ def test_linear_gather_writes_every_destination(p, n, N, K, B, world, dtype):
         assert np.isfinite(y).all()
         assert U.linear_error(y, y_ref) <= tol
     for t in dsts[1:]:
-        assert torch.equal(t, dsts[0]) or hb.higgs_linear_k_splits(hb.make_desc(p, n, hb.shard_rows(N, world, 0)[1], K, xi), B) > 1
+        assert torch.equal(t, dsts[0]) or hb.higgs_linear_uses_atomics(hb.make_desc(p, n, hb.shard_rows(N, world, 0)[1], K, xi), B)
 
 
 def test_linear_gather_argument_checks():
@@ -388,7 +388,7 @@ def test_linear_host_and_host_batch_match_device_path(B):
         d = hb.make_desc(p, n, N, K, xi)
         # bit-for-bit comparison: the small-batch path must not split K (atomics); the cluster split of the tensor-core
         # path sums in a fixed order
-        assert hb.higgs_linear_k_splits(d, B) == 1 or hb.higgs_rotated_layout(d, B) > 0
+        assert not hb.higgs_linear_uses_atomics(d, B)
         _, gt = U.grid32(p, n)
         W = inputs.make_weights(N, K, seed=40 + li, bf16=True)
         pk, sc, _ = hb.higgs_quantize(d, U.bf16_tensor(W), gt)
@@ -572,3 +572,39 @@ def test_linear_tensor_core_path_bf16_output(N, K, B):
     y, y_ref = run_linear_case(2, 256, N, K, B, xi=5, wseed=9, xseed=10, out_dtype=torch.bfloat16)
     assert y.dtype == torch.bfloat16
     assert U.linear_error(y.float().cpu().numpy(), y_ref) <= Y_TOL + 2.0 ** -8
+
+
+@pytest.mark.parametrize("p,n,N,K,B,dtype", [
+    (2, 256, 512, 8192, 1, torch.float32),      # fused rotation, both halves of K in one cluster pair
+    (2, 256, 4096, 8192, 2, torch.float32),
+    (2, 64, 1040, 8192, 1, torch.bfloat16),     # six-bit planes, ragged row-tile split over the pairs
+    (2, 16, 2048, 8192, 2, torch.float32),      # nibble format: partial tiles behind the table
+    (1, 256, 2368, 8192, 3, torch.float32),     # 8-bit scalar codes
+    (2, 256, 2048, 8192, 5, torch.float32),     # rotation kernel + product, generic flusher
+    (2, 256, 768, 4096, 16, torch.float32),     # two token blocks per MMA step (128-input slices)
+    (1, 16, 1184, 8192, 8, torch.bfloat16),
+])
+def test_two_k_chunks_meet_in_a_cluster_pair_in_a_fixed_order(p, n, N, K, B, dtype):
+    """K ranges of 2 x 4096 inputs (2 x 2048 when nine or more tokens halve the slices): the two blocks of a thread-block
+    cluster take them, item j is summed by block j % 2 in a fixed order.  Checked against the oracle, bit for bit
+    between two runs, and the call must report that it uses no atomics."""
+    xi = 2024
+    g64, gt = U.grid32(p, n)
+    W = inputs.make_weights(N, K, seed=600 + N + B, bf16=True)
+    q, sc16 = U.oracle_encode(W, 1024, g64, xi)
+    d = hb.make_desc(p, n, N, K, xi)
+    assert hb.higgs_linear_k_splits(d, B) == 2 and not hb.higgs_linear_uses_atomics(d, B)
+    packed = hb.higgs_pack_codes(d, torch.from_numpy(q.codes.astype(np.uint8)).to(U.dev()))
+    sc = hb.scales_to_tile_major(torch.from_numpy(sc16).to(U.dev()))
+    x = inputs.make_activations(B, K, seed=601 + B)
+    xt = U.bf16_tensor(x)
+    y1 = hb.higgs_linear(d, xt, packed, sc, gt, out_dtype=dtype)
+    y2 = hb.higgs_linear(d, xt, packed, sc, gt, out_dtype=dtype)
+    y3 = hb.higgs_linear_prerotated(d, hb.higgs_rotate_activations(d, xt), packed, sc, gt, out_dtype=dtype)
+    torch.cuda.synchronize()
+    assert hb.higgs_device_status() == hb.HIGGS_OK
+    assert torch.equal(y1, y2)
+    y_ref = oracle.linear_dense(x.astype(np.float64), q.codes, sc16.astype(np.float64), 1024, g64, xi)
+    tol = Y_TOL + (2.0 ** -8 if dtype == torch.bfloat16 else 0.0)
+    assert U.linear_error(y1.float().cpu().numpy(), y_ref) <= tol
+    assert U.linear_error(y3.float().cpu().numpy(), y_ref) <= tol
