@@ -157,7 +157,8 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 
 // FB = 64-input steps per activation-tile stage (4, 2, 1 for BN <= 64, <= 128, <= 256: a stage is at most 32 KB).  It is a
 // template parameter so that the MMA warp's loop body is straight-line code.
-template <int FB, bool SIX>
+// FMT: 0 = byte format, 1 = six-bit planes, 2 = nibble pairs (p=2 n=16, p=1 n=4), 3 = 8-bit scalar codes (p=1 n=256).
+template <int FB, int FMT>
 __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams prm, const __grid_constant__ CUtensorMap code_map) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -183,7 +184,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
     const uint32_t d_full = bars + 8u * 80u;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_raw + 1024);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem_raw + 1032);
-    constexpr uint32_t kTcCodeStage = SIX ? 6144u : 4096u;
+    constexpr bool SIX = FMT == 1, NIB = FMT == 2, B8 = FMT == 3;
+    // bytes of the block's 128 rows in one code stage: 512 B per row tile and 64 inputs (byte format), 768 B per 128
+    // inputs (six-bit), 256 B (nibble), 1 KB (8-bit)
+    constexpr uint32_t kTcCodeStage = SIX ? 6144u : NIB ? 2048u : B8 ? 8192u : 4096u;
     constexpr int SPS = SIX ? 2 : 1;                         // 64-input steps per code stage
     const uint32_t code0 = base + 2048u;
     const uint32_t b_stage_bytes = (uint32_t)FB * (uint32_t)prm.BN * 128u;
@@ -221,7 +225,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
         const int idx = 4 * (warp + r * kW) + (lane >> 3);
         ent_lo[r] = 0.f; ent_hi[r] = 0.f;
         if (idx < 256) {
-            if (prm.p == 2) {
+            if (B8) {
+                ent_lo[r] = ent_hi[r] = __ldg(prm.grid + idx);              // one input per index: the value in both halves
+            } else if (prm.p == 2) {
                 const float2 gp = __ldg(reinterpret_cast<const float2*>(prm.grid) + (idx & (prm.n - 1)));
                 ent_lo[r] = gp.x; ent_hi[r] = gp.y;
             } else {
@@ -396,7 +402,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
         const uint32_t t_lane = tmem + ((uint32_t)(32 * q) << 16);
         // byte formats: this row's words are the 16-byte chunks of lanes (g, t) of its row tile; six-bit: word 2 (4g + t) +
         // (step & 1) of each of the tile's three 256-byte planes
-        const uint32_t code_off = SIX ? (uint32_t)(rtl * 768 + g * 32 + (sg & 1) * 4) : (uint32_t)(rtl * 512 + g * 64);
+        // nibble format: the 8-byte chunks of lanes (g, t = 0..3) are 32 contiguous bytes; 8-bit format: the 16-byte chunks
+        // of lanes (g, t) in each 512-byte half of the row tile's 1 KB block
+        const uint32_t code_off = SIX ? (uint32_t)(rtl * 768 + g * 32 + (sg & 1) * 4) : NIB ? (uint32_t)(rtl * 256 + g * 32)
+                                : B8 ? (uint32_t)(rtl * 1024 + g * 64) : (uint32_t)(rtl * 512 + g * 64);
         const int tx = rtl & 1;                    // six-bit: odd row tiles visit the lanes t in the order t ^ 1 (bank conflicts)
         int cur_group = -1;
         uint32_t sc2 = 0;
@@ -413,7 +422,54 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
                 sc2 = *reinterpret_cast<const uint32_t*>(&s2);
             }
             uint4 c4[4];                           // c4[t] = the four index words (steps m = 0..3) of lane (g, t)
-            if (!SIX) {
+            uint32_t a[32];
+            auto unrotate = [&]() {                // chunk t was loaded by instruction (t - rot) & 3
+                if (rot & 1) { const uint4 t0 = c4[0]; c4[0] = c4[3]; c4[3] = c4[2]; c4[2] = c4[1]; c4[1] = t0; }
+                if (rot & 2) { uint4 t0 = c4[0]; c4[0] = c4[2]; c4[2] = t0; t0 = c4[1]; c4[1] = c4[3]; c4[3] = t0; }
+            };
+            if (B8) {
+                // 8-bit scalar codes: a register (two consecutive inputs of the row) is halfword h of word 2m + kh of lane
+                // (g, t) - two code bytes, two lookups (a table entry carries its value in both halves).  Words 0..3 of
+                // every lane sit in the first 512-byte half of the row tile's block (steps m = 0, 1), words 4..7 in the second.
+                const uint32_t selA = 0x7604u + ((uint32_t)(2 * h) << 4), selB = 0x7604u + ((uint32_t)(2 * h + 1) << 4);
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj)
+                        c4[jj] = t_lds128(code_stage(cs) + code_off + (uint32_t)(hh * 512) + (uint32_t)(((jj + rot) & 3) * 16));
+                    unrotate();
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) {          // r = 2 (m & 1) + kh
+                            const uint32_t w = r == 0 ? c4[t].x : r == 1 ? c4[t].y : r == 2 ? c4[t].z : c4[t].w;
+                            const uint32_t l0 = t_lds32(__byte_perm(w, lut_lane, selA));
+                            const uint32_t l1 = t_lds32(__byte_perm(w, lut_lane, selB));
+                            const uint32_t e = __byte_perm(l0, l1, 0x7610);
+                            const __half2 pr = __hmul2(*reinterpret_cast<const __half2*>(&e), *reinterpret_cast<const __half2*>(&sc2));
+                            a[(2 * hh + (r >> 1)) * 8 + (r & 1) * 4 + t] = *reinterpret_cast<const uint32_t*>(&pr);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) t_mbar_arrive(code_empty(cs));     // every code word has been looked up: hand the stage back
+                cs += 4 / SPS;
+                if (cs >= CS) { cs -= CS; ++ucs; }
+            } else {
+            if (NIB) {
+                // nibble pairs: byte 2m + kh of lane (g, t) holds the codes of row halves 0 (low nibble) and 1 (high nibble);
+                // the row's eight nibbles per lane become the bytes of two index words.  The two 16-byte loads are issued in
+                // the order that keeps the eight g of a warp on different banks.
+                const bool swp = (g & 4) != 0;
+                const uint4 f0 = t_lds128(code_stage(cs) + code_off + (swp ? 16u : 0u));
+                const uint4 f1 = t_lds128(code_stage(cs) + code_off + (swp ? 0u : 16u));
+                const uint4 lo = swp ? f1 : f0, hi = swp ? f0 : f1;        // lanes t = 0, 1 and t = 2, 3
+                const uint32_t sh = (uint32_t)(4 * h);
+                c4[0] = make_uint4((lo.x >> sh) & 0x0f0f0f0fu, (lo.y >> sh) & 0x0f0f0f0fu, 0u, 0u);
+                c4[1] = make_uint4((lo.z >> sh) & 0x0f0f0f0fu, (lo.w >> sh) & 0x0f0f0f0fu, 0u, 0u);
+                c4[2] = make_uint4((hi.x >> sh) & 0x0f0f0f0fu, (hi.y >> sh) & 0x0f0f0f0fu, 0u, 0u);
+                c4[3] = make_uint4((hi.z >> sh) & 0x0f0f0f0fu, (hi.w >> sh) & 0x0f0f0f0fu, 0u, 0u);
+            } else if (!SIX) {
                 // the 16-byte chunks of lanes (g, t = 0..3) of row tile rtl; instruction jj reads chunk (jj + rot) & 3
                 // so that the eight g of a warp hit eight different bank groups
 #pragma unroll
@@ -445,25 +501,29 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
             if (lane == 0) t_mbar_arrive(code_empty(cs));     // the code words are in registers: hand the stage back
             cs += 4 / SPS;
             if (cs >= CS) { cs -= CS; ++ucs; }
-            // undo the rotation: chunk t was loaded by instruction (t - rot) & 3
-            if (!SIX) {
-                if (rot & 1) { const uint4 t0 = c4[0]; c4[0] = c4[3]; c4[3] = c4[2]; c4[2] = c4[1]; c4[1] = t0; }
-                if (rot & 2) { uint4 t0 = c4[0]; c4[0] = c4[2]; c4[2] = t0; t0 = c4[1]; c4[1] = c4[3]; c4[3] = t0; }
-            }
-            uint32_t a[32];
+            if (!SIX && !NIB) unrotate();
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
 #pragma unroll
                 for (int t = 0; t < 4; ++t) {
-                    const uint32_t w = m == 0 ? c4[t].x : m == 1 ? c4[t].y : m == 2 ? c4[t].z : c4[t].w;
-                    // input pairs 8m + t (byte h) and 8m + 4 + t (byte h + 2) of the 64-input block
-                    const uint32_t e0 = t_lds32(__byte_perm(w, lut_lane, sel0));
-                    const uint32_t e1 = t_lds32(__byte_perm(w, lut_lane, sel1));
+                    uint32_t e0, e1;
+                    if (NIB) {
+                        // bytes 2 (m & 1) and 2 (m & 1) + 1 of index word m >> 1: input pairs 8m + t and 8m + 4 + t
+                        const uint32_t w = (m >> 1) ? c4[t].y : c4[t].x;
+                        e0 = t_lds32(__byte_perm(w, lut_lane, (m & 1) ? 0x7624u : 0x7604u));
+                        e1 = t_lds32(__byte_perm(w, lut_lane, (m & 1) ? 0x7634u : 0x7614u));
+                    } else {
+                        const uint32_t w = m == 0 ? c4[t].x : m == 1 ? c4[t].y : m == 2 ? c4[t].z : c4[t].w;
+                        // input pairs 8m + t (byte h) and 8m + 4 + t (byte h + 2) of the 64-input block
+                        e0 = t_lds32(__byte_perm(w, lut_lane, sel0));
+                        e1 = t_lds32(__byte_perm(w, lut_lane, sel1));
+                    }
                     const __half2 p0 = __hmul2(*reinterpret_cast<const __half2*>(&e0), *reinterpret_cast<const __half2*>(&sc2));
                     const __half2 p1 = __hmul2(*reinterpret_cast<const __half2*>(&e1), *reinterpret_cast<const __half2*>(&sc2));
                     a[m * 8 + t] = *reinterpret_cast<const uint32_t*>(&p0);
                     a[m * 8 + 4 + t] = *reinterpret_cast<const uint32_t*>(&p1);
                 }
+            }
             }
             // the A stage must have been consumed by the MMAs that used it last
             bad |= t_wait(a_free(sa), (uint32_t)((ua & 1) ^ 1), t_limit(bad)) ^ 1u;   // (first use: the phase before the first)
@@ -665,7 +725,7 @@ int tc_batch_tile(int64_t B) {
 // measured cross-over near 32 M weights).
 bool tc_eligible(const higgs_desc& d, int64_t B) {
     const Format f = format_of(d.p, d.n);
-    if (!(d.N % 128 == 0 && d.N > 0 && (f == Format::kByteLut || f == Format::kSixBit))) return false;
+    if (!(d.N % 128 == 0 && d.N > 0 && f != Format::kNone)) return false;
     return B > 16 || (B > 8 && d.N * d.K >= ((int64_t)1 << 25));
 }
 
@@ -717,12 +777,14 @@ EncodeTiledFn encode_tiled_fn() {
 bool make_code_map(const higgs_desc& d, const void* packed, CUtensorMap* map) {
     EncodeTiledFn enc = encode_tiled_fn();
     if (!enc) return false;
-    // byte formats: K x 8 bytes per row tile, a stage is one 512-byte block; six-bit: K x 6 bytes, a stage is one 768-byte
-    // super-block (three bit planes of two neighbouring blocks)
-    const bool six = format_of(d.p, d.n) == Format::kSixBit;
-    const cuuint64_t dims[2] = {(cuuint64_t)(six ? d.K * 6 / 8 : d.K), (cuuint64_t)(d.N / 16)};
-    const cuuint64_t strides[1] = {(cuuint64_t)(six ? d.K * 6 : d.K * 8)};
-    const cuuint32_t box[2] = {six ? 96u : 64u, 8};
+    // per row tile (16 rows) an input takes 8 bytes (byte format), 6 (six-bit), 4 (nibble) or 16 (8-bit); a stage is
+    // one 64-input block of the eight row tiles - for the six-bit format one 768-byte super-block (three bit planes of
+    // two neighbouring blocks)
+    const Format f = format_of(d.p, d.n);
+    const cuuint64_t bpi = f == Format::kSixBit ? 6 : f == Format::kNibble ? 4 : f == Format::kByte8 ? 16 : 8;
+    const cuuint64_t dims[2] = {(cuuint64_t)d.K * bpi / 8, (cuuint64_t)(d.N / 16)};
+    const cuuint64_t strides[1] = {(cuuint64_t)d.K * bpi};
+    const cuuint32_t box[2] = {f == Format::kSixBit ? 96u : f == Format::kNibble ? 32u : f == Format::kByte8 ? 128u : 64u, 8};
     const cuuint32_t estr[2] = {1, 1};
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_INT64, 2, const_cast<void*>(packed), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -739,9 +801,11 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
     const int64_t tiles = (B + BN - 1) / BN;
     static int configured[64] = {0};
     const int conf = device_once(configured, [] {
-        const void* kernels[6] = {(const void*)linear_tc_kernel<1, false>, (const void*)linear_tc_kernel<2, false>,
-                                  (const void*)linear_tc_kernel<4, false>, (const void*)linear_tc_kernel<1, true>,
-                                  (const void*)linear_tc_kernel<2, true>, (const void*)linear_tc_kernel<4, true>};
+        const void* kernels[12] = {
+            (const void*)linear_tc_kernel<1, 0>, (const void*)linear_tc_kernel<2, 0>, (const void*)linear_tc_kernel<4, 0>,
+            (const void*)linear_tc_kernel<1, 1>, (const void*)linear_tc_kernel<2, 1>, (const void*)linear_tc_kernel<4, 1>,
+            (const void*)linear_tc_kernel<1, 2>, (const void*)linear_tc_kernel<2, 2>, (const void*)linear_tc_kernel<4, 2>,
+            (const void*)linear_tc_kernel<1, 3>, (const void*)linear_tc_kernel<2, 3>, (const void*)linear_tc_kernel<4, 3>};
         for (const void* k : kernels)
             if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTcSmem) != cudaSuccess) return -1;
         return 1;
@@ -780,11 +844,14 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
     cfg.attrs = attr;
     // activation-tile stage = FB steps of BN x 128 bytes, at most 16 KB for BN <= 128 (so that the code ring gets the
     // rest of shared memory) and 32 KB for wider tiles
-    const bool six = format_of(d.p, d.n) == Format::kSixBit;
-    void (*kernel)(const TcParams, const CUtensorMap) =
-        BN <= 32 ? (six ? linear_tc_kernel<4, true> : linear_tc_kernel<4, false>)
-      : BN <= 64 ? (six ? linear_tc_kernel<2, true> : linear_tc_kernel<2, false>)
-                 : (six ? linear_tc_kernel<1, true> : linear_tc_kernel<1, false>);
+    const Format fmt = format_of(d.p, d.n);
+    const int fi = fmt == Format::kSixBit ? 1 : fmt == Format::kNibble ? 2 : fmt == Format::kByte8 ? 3 : 0;
+    typedef void (*TcKernel)(const TcParams, const CUtensorMap);
+    static const TcKernel table[3][4] = {
+        {linear_tc_kernel<4, 0>, linear_tc_kernel<4, 1>, linear_tc_kernel<4, 2>, linear_tc_kernel<4, 3>},
+        {linear_tc_kernel<2, 0>, linear_tc_kernel<2, 1>, linear_tc_kernel<2, 2>, linear_tc_kernel<2, 3>},
+        {linear_tc_kernel<1, 0>, linear_tc_kernel<1, 1>, linear_tc_kernel<1, 2>, linear_tc_kernel<1, 3>}};
+    TcKernel kernel = table[BN <= 32 ? 0 : BN <= 64 ? 1 : 2][fi];
     if (prm.ksplit > 1) {
         // a cluster of `ksplit` blocks with this much shared memory must fit the device (it does on a full B200; a
         // partitioned one may not, and then K is not split): checked once per device and cluster size

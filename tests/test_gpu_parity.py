@@ -138,7 +138,7 @@ def run_linear_case(p, n, N, K, B, xi, wseed, xseed, out_dtype=torch.float32, lo
     (2, 16, 272, 4096, 8),
     (2, 16, 64, 8192, 16),
     (2, 16, 32, 14336, 2),
-    (2, 16, 128, 1024, 40),      # more tokens than one launch takes (no tensor-core path for this format)
+    (2, 16, 144, 1024, 40),      # more tokens than one launch takes (the row count keeps it off the tensor-core path)
     (1, 8, 272, 4096, 4),        # scalar 3-bit grid: six-bit format, two codes per index
     (1, 8, 64, 8192, 16),
     (1, 4, 272, 4096, 8),        # scalar 2-bit grid: nibble format, four codes per byte
@@ -146,7 +146,7 @@ def run_linear_case(p, n, N, K, B, xi, wseed, xseed, out_dtype=torch.float32, lo
     (1, 256, 48, 2048, 1),       # 8-bit scalar codes: a register is put together from two lookups
     (1, 256, 272, 4096, 7),
     (1, 256, 64, 8192, 16),
-    (1, 256, 128, 1024, 33),
+    (1, 256, 144, 1024, 33),
     (2, 256, 16, 1024, 17),      # more tokens than one launch takes
     (2, 256, 32, 2048, 40),
 ])
@@ -527,6 +527,18 @@ def test_make_grid_general_is_a_lloyd_fixed_point(p, n, log2m):
     (2, 64, 8448, 1024, 40),     # six-bit, K not split
     (2, 64, 256, 1024, 300),
     (1, 8, 256, 2048, 64),       # scalar 3-bit grid on the six-bit path
+    (2, 16, 128, 1024, 17),      # nibble format: the row's nibbles become the bytes of its index words
+    (2, 16, 256, 2048, 64),
+    (2, 16, 384, 4096, 100),
+    (2, 16, 8448, 1024, 40),     # K not split
+    (2, 16, 128, 8192, 256),
+    (1, 4, 256, 2048, 64),       # scalar 2-bit grid on the nibble path
+    (1, 256, 128, 1024, 17),     # 8-bit scalar codes: two lookups per operand register, 8 KB code stages
+    (1, 256, 256, 2048, 64),
+    (1, 256, 384, 4096, 100),
+    (1, 256, 8448, 1024, 40),
+    (1, 256, 128, 8192, 256),
+    (1, 256, 256, 1024, 300),
 ])
 def test_linear_tensor_core_path_matches_oracle(p, n, N, K, B):
     y, y_ref = run_linear_case(p, n, N, K, B, xi=inputs.rht_seed(3), wseed=300 + N, xseed=400 + B, lognormal=(B == 64))
