@@ -281,6 +281,28 @@ int higgs_linear_gather(const higgs_desc* desc, const void* x, int64_t B, const 
 int higgs_shard_rows(int64_t N, int32_t world, int32_t rank, int32_t multiple, int64_t* begin_out, int64_t* count_out);
 
 /*
+ * Layer sharded along K on group boundaries (Appendix F: the rotation acts inside a 1024-group, so a device that holds
+ * inputs [k0, k0 + K_r) of every row, k0 a multiple of 1024, can rotate its slice of x and multiply it on its own; the
+ * fp32 partial outputs of the devices are then summed).  A K-shard is an ordinary layer of K_r inputs whose sign
+ * sequence starts at input k0: higgs_shard_seed(xi, k0) is the seed that makes sign(seed', j) = sign(xi, k0 + j), so
+ * a shard encoded and multiplied with {N, K_r, seed'} carries exactly the codes and signs of columns [k0, k0 + K_r)
+ * of the unsharded layer.  (HOST function.)
+ *
+ * higgs_linear_kshard: this device's partial product, written from the kernels' epilogues (plain stores, own
+ * memory and peer-mapped memory alike, no multicast) into slot `rank` of EVERY device's slot buffer
+ *   slot_bufs[i] : device-accessible fp32 [world][B][N] of device i (i = rank: this device's own), a HOST array;
+ * desc/x_shard/packed/scales describe the shard (x_shard is [B][K_r] bf16).  It neither waits for nor signals other
+ * devices: the caller orders "all partials written" before higgs_reduce_slots (a barrier of the process group).
+ * higgs_reduce_slots: y[i] = slots[0][i] + slots[1][i] + ... in slot order (bit-reproducible), count = B * N values
+ * (a multiple of 4), y fp32 or bf16.  Both asynchronous on `stream`; errors and workspace as higgs_linear_gather.
+ */
+uint64_t higgs_shard_seed(uint64_t rht_seed, int64_t k_offset);
+int higgs_linear_kshard(const higgs_desc* desc, const void* x_shard, int64_t B, const void* packed, const void* scales,
+                        const float* grid, void* const* slot_bufs, int32_t world, int32_t rank,
+                        void* workspace, size_t workspace_bytes, void* stream);
+int higgs_reduce_slots(const float* slots, int32_t world, int64_t count, void* y, int y_dtype, void* stream);
+
+/*
  * higgs_linear with HOST activations and HOST output (Appendix F product; the
  * weights stay resident on the device): copies x_host ([B][K] bf16, ideally
  * pinned) to the device, runs higgs_linear, copies y ([B][N] of y_dtype) back to

@@ -29,7 +29,7 @@ EXPORTS = [
     "higgs_rotated_layout", "higgs_dequantize", "higgs_make_uniform_grid", "higgs_layer_error",
     "higgs_allocate_bits", "higgs_general_tuples", "higgs_quantize_general", "higgs_linear_host_batch",
     "higgs_linear_gather", "higgs_linear_share", "higgs_make_grid_seeded", "higgs_gaussian_samples", "higgs_shard_rows",
-    "higgs_launch_floor", "higgs_selftest_wait", "higgs_linear_uses_atomics",
+    "higgs_launch_floor", "higgs_selftest_wait", "higgs_linear_uses_atomics", "higgs_shard_seed", "higgs_linear_kshard", "higgs_reduce_slots",
 ]
 
 
@@ -123,6 +123,12 @@ def _load() -> ctypes.CDLL:
     lib.higgs_gaussian_samples.argtypes = [i32, u64, i64, vp, vp]
     lib.higgs_shard_rows.restype = i32
     lib.higgs_shard_rows.argtypes = [i64, i32, i32, i32, ctypes.POINTER(i64), ctypes.POINTER(i64)]
+    lib.higgs_shard_seed.restype = u64
+    lib.higgs_shard_seed.argtypes = [u64, i64]
+    lib.higgs_linear_kshard.restype = i32
+    lib.higgs_linear_kshard.argtypes = [P, vp, i64, vp, vp, vp, vp, i32, i32, vp, sz, vp]
+    lib.higgs_reduce_slots.restype = i32
+    lib.higgs_reduce_slots.argtypes = [vp, i32, i64, vp, i32, vp]
     lib.higgs_launch_floor.restype = i32
     lib.higgs_launch_floor.argtypes = [i32, i32, sz, vp]
     lib.higgs_selftest_wait.restype = i32
@@ -351,6 +357,34 @@ def higgs_linear_gather(desc: higgs_desc, x: torch.Tensor, packed: torch.Tensor,
     _check(lib.higgs_linear_gather(ctypes.byref(desc), _ptr(x), B, _ptr(packed), _ptr(scales), _ptr(grid), ptrs, len(y_dsts),
                                    ld, int(row_offset), _dtype_code(y_dsts[0]), _ptr(workspace), workspace.numel(), _stream()),
            "higgs_linear_gather")
+
+
+def higgs_shard_seed(rht_seed: int, k_offset: int) -> int:
+    return int(lib.higgs_shard_seed(rht_seed & (2**64 - 1), int(k_offset)))
+
+
+def higgs_linear_kshard(desc: higgs_desc, x_shard: torch.Tensor, packed: torch.Tensor, scales: torch.Tensor, grid: torch.Tensor,
+                        slot_bufs, rank: int, workspace: Optional[torch.Tensor] = None) -> None:
+    """K-sharded layer: this device's fp32 partial product into slot `rank` of every tensor of slot_bufs
+    ([world][B][N] fp32 each, slot_bufs[i] on device i or peer-mapped)."""
+    assert x_shard.is_cuda and x_shard.dtype == torch.bfloat16 and x_shard.is_contiguous()
+    B, world = x_shard.shape[0], len(slot_bufs)
+    for t in slot_bufs:
+        assert t.is_contiguous() and t.dtype == torch.float32 and tuple(t.shape) == (world, B, desc.N)
+    if workspace is None:
+        workspace = _workspace(higgs_workspace_bytes(desc, HIGGS_OP_LINEAR, B), x_shard.device)
+    ptrs = (ctypes.c_void_p * world)(*[t.data_ptr() for t in slot_bufs])
+    _check(lib.higgs_linear_kshard(ctypes.byref(desc), _ptr(x_shard), B, _ptr(packed), _ptr(scales), _ptr(grid), ptrs, world,
+                                   int(rank), _ptr(workspace), workspace.numel(), _stream()), "higgs_linear_kshard")
+
+
+def higgs_reduce_slots(slots: torch.Tensor, out_dtype: torch.dtype = torch.float32) -> torch.Tensor:
+    """slots: cuda fp32 [world][B][N] -> y [B][N] = the slots summed in slot order."""
+    assert slots.is_cuda and slots.dtype == torch.float32 and slots.is_contiguous() and slots.dim() == 3
+    world, B, N = slots.shape
+    y = torch.empty((B, N), dtype=out_dtype, device=slots.device)
+    _check(lib.higgs_reduce_slots(_ptr(slots), world, B * N, _ptr(y), _dtype_code(y), _stream()), "higgs_reduce_slots")
+    return y
 
 
 class HostBatch:

@@ -122,6 +122,39 @@ int higgs_shard_rows(int64_t N, int32_t world, int32_t rank, int32_t multiple, i
     return HIGGS_OK;
 }
 
+uint64_t higgs_shard_seed(uint64_t rht_seed, int64_t k_offset) {
+    // output number m + k_offset / 64 of the stream seeded with xi is output number m of the stream seeded with
+    // xi + (k_offset / 64) * golden-ratio increment: the sign function's state advances by that increment per output
+    return rht_seed + (uint64_t)(k_offset / 64) * 0x9E3779B97F4A7C15ull;
+}
+
+int higgs_linear_kshard(const higgs_desc* d, const void* x_shard, int64_t B, const void* packed, const void* scales,
+                        const float* grid, void* const* slot_bufs, int32_t world, int32_t rank, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+    if (!d || !slot_bufs || world < 1 || world > kMaxGather || rank < 0 || rank >= world || B < 0) return HIGGS_ERR_INVALID_ARG;
+    void* dst[kMaxGather];
+    for (int i = 0; i < world; ++i) {
+        if (!slot_bufs[i]) return HIGGS_ERR_INVALID_ARG;
+        dst[i] = static_cast<float*>(slot_bufs[i]) + (size_t)rank * (size_t)B * (size_t)d->N;    // slot `rank` of device i
+    }
+    // the own device's buffer first (slot_bufs[rank]), then the peers' in rank order
+    void* ordered[kMaxGather];
+    int n = 0;
+    ordered[n++] = dst[rank];
+    for (int i = 0; i < world; ++i)
+        if (i != rank) ordered[n++] = dst[i];
+    return higgs_linear_gather(d, x_shard, B, packed, scales, grid, ordered, world, d->N, 0, HIGGS_F32, workspace, workspace_bytes,
+                               stream);
+}
+
+int higgs_reduce_slots(const float* slots, int32_t world, int64_t count, void* y, int y_dtype, void* stream) {
+    if (world < 1 || world > kMaxGather || count < 0 || count % 4) return HIGGS_ERR_INVALID_ARG;
+    if (y_dtype != HIGGS_F32 && y_dtype != HIGGS_BF16) return HIGGS_ERR_UNSUPPORTED;
+    if (count == 0) return HIGGS_OK;
+    if (!slots || !y || !aligned(slots, 16) || !aligned(y, 16)) return HIGGS_ERR_INVALID_ARG;
+    return launch_reduce_slots(slots, world, count, y, y_dtype, as_stream(stream));
+}
+
 int higgs_launch_floor(int32_t blocks, int32_t threads, size_t shared_bytes, void* stream) {
     if (blocks < 1 || threads < 1 || threads > 1024 || shared_bytes > 232448) return HIGGS_ERR_INVALID_ARG;
     return launch_floor(blocks, threads, shared_bytes, as_stream(stream));

@@ -219,6 +219,7 @@ int read_tc_status(int clear);
 int launch_wait_selftest(uint32_t limit, int* result, cudaStream_t st);
 int launch_tc_wait_selftest(uint32_t limit, int* result, cudaStream_t st);
 int launch_stream_fence(cudaStream_t st);
+int launch_reduce_slots(const float* slots, int world, int64_t count, void* y, int y_dtype, cudaStream_t st);
 int launch_floor(int blocks, int threads, size_t smem, cudaStream_t st);
 int launch_gaussian_samples(int p, uint64_t seed, int64_t m, float* out, cudaStream_t st);
 int read_device_status(cudaStream_t st, int clear);

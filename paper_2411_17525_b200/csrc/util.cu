@@ -23,6 +23,26 @@ __global__ void gaussian_samples_kernel(int p, uint64_t seed, int64_t count, flo
     out[c] = sqrtf(-2.0f * logf(u1)) * cospif(2.0f * u2);
 }
 
+// Sums `world` fp32 slots of `count` values in slot order (a fixed order: the result is reproducible) into y.
+__global__ void reduce_slots_kernel(const float* __restrict__ slots, int world, int64_t count, void* __restrict__ y, int bf16) {
+    pdl_trigger();
+    pdl_wait();
+    const int64_t quads = count / 4;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < quads; i += (int64_t)gridDim.x * blockDim.x) {
+        float4 acc = *reinterpret_cast<const float4*>(slots + 4 * i);
+        for (int r = 1; r < world; ++r) {
+            const float4 v = *reinterpret_cast<const float4*>(slots + (int64_t)r * count + 4 * i);
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        if (bf16) {
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+            reinterpret_cast<uint2*>(y)[i] = make_uint2(*reinterpret_cast<const uint32_t*>(&lo), *reinterpret_cast<const uint32_t*>(&hi));
+        } else {
+            reinterpret_cast<float4*>(y)[i] = acc;
+        }
+    }
+}
+
 // Ordinary (fully stream-ordered) empty kernel: see launch_stream_fence.
 __global__ void fence_kernel() {}
 
@@ -34,6 +54,14 @@ __global__ void fence_kernel() {}
 int launch_stream_fence(cudaStream_t st) {
     fence_kernel<<<1, 32, 0, st>>>();
     return cuda_status(cudaGetLastError());
+}
+
+int launch_reduce_slots(const float* slots, int world, int64_t count, void* y, int y_dtype, cudaStream_t st) {
+    int64_t blocks = (count / 4 + 255) / 256;
+    if (blocks > 1184) blocks = 1184;
+    if (blocks < 1) blocks = 1;
+    return cuda_status(launch_pdl(reduce_slots_kernel, dim3((unsigned)blocks), dim3(256), 0, st, slots, world, count, y,
+                                  y_dtype == HIGGS_BF16 ? 1 : 0));
 }
 
 int launch_floor(int blocks, int threads, size_t smem, cudaStream_t st) {

@@ -620,3 +620,44 @@ def test_two_k_chunks_meet_in_a_cluster_pair_in_a_fixed_order(p, n, N, K, B, dty
     tol = Y_TOL + (2.0 ** -8 if dtype == torch.bfloat16 else 0.0)
     assert U.linear_error(y1.float().cpu().numpy(), y_ref) <= tol
     assert U.linear_error(y3.float().cpu().numpy(), y_ref) <= tol
+
+
+@pytest.mark.parametrize("p,n,N,K,B,world,dtype", [
+    (2, 256, 256, 8192, 1, 2, torch.float32),      # shards of 4096 inputs: fused rotation
+    (2, 256, 2048, 16384, 2, 2, torch.float32),    # shards of 8192 inputs: cluster pairs
+    (2, 64, 128, 4096, 5, 4, torch.bfloat16),      # shards of one group
+    (2, 256, 256, 8192, 40, 4, torch.float32),     # tensor-core path, K split inside a cluster
+    (2, 256, 64, 28672, 3, 2, torch.float32),      # shards of 14336 inputs: atomics inside a shard, copy kernel spreads
+])
+def test_k_sharded_layer_sums_to_the_unsharded_output(p, n, N, K, B, world, dtype):
+    """higgs_linear_kshard + higgs_reduce_slots with the `world` devices emulated on one GPU (the shards are launched
+    one after the other and never wait on one another; every "device" has its own slot buffer): each shard is the
+    layer's columns [k0, k0 + K / world) with the shifted seed, and every device's reduced output is the oracle's
+    output of the whole layer."""
+    xi = 4711
+    g64, gt = U.grid32(p, n)
+    W = inputs.make_weights(N, K, seed=700 + N, bf16=True)
+    q, sc16 = U.oracle_encode(W, 1024, g64, xi)
+    x = inputs.make_activations(B, K, seed=701 + B)
+    Kr = K // world
+    slot_bufs = [torch.full((world, B, N), float("nan"), dtype=torch.float32, device=U.dev()) for _ in range(world)]
+    for r in range(world):
+        k0 = r * Kr
+        d = hb.make_desc(p, n, N, Kr, hb.higgs_shard_seed(xi, k0))
+        codes = np.ascontiguousarray(q.codes[:, k0 // p:(k0 + Kr) // p]).astype(np.uint8)
+        packed = hb.higgs_pack_codes(d, torch.from_numpy(codes).to(U.dev()))
+        sc = hb.scales_to_tile_major(torch.from_numpy(np.ascontiguousarray(sc16[:, k0 // 1024:(k0 + Kr) // 1024])).to(U.dev()))
+        xs = U.bf16_tensor(np.ascontiguousarray(x[:, k0:k0 + Kr]))
+        # "device" r: its own buffer first in its call, the others as peers
+        hb.higgs_linear_kshard(d, xs, packed, sc, gt, slot_bufs, r)
+    torch.cuda.synchronize()
+    assert hb.higgs_device_status() == hb.HIGGS_OK
+    y_ref = oracle.linear_dense(x.astype(np.float64), q.codes, sc16.astype(np.float64), 1024, g64, xi)
+    tol = Y_TOL + (2.0 ** -8 if dtype == torch.bfloat16 else 0.0)
+    ys = [hb.higgs_reduce_slots(sb, out_dtype=dtype) for sb in slot_bufs]
+    for y in ys:
+        got = y.float().cpu().numpy()
+        assert np.isfinite(got).all()
+        assert U.linear_error(got, y_ref) <= tol
+    for y in ys[1:]:
+        assert torch.equal(y, ys[0])

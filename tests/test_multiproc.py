@@ -105,6 +105,71 @@ def test_row_sharded_layer_protocol_on_two_ranks():
         assert err == 0.0
 
 
+# ---- K-sharded layer: the host-side protocol of higgs_linear_kshard + higgs_reduce_slots on two CPU ranks ------------
+def _kshard_worker(rank, world, port, out):
+    import numpy as np
+
+    import oracle
+    from paper_2411_17525_b200 import binding
+    from synth import inputs
+    from synth import grids as stored
+
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        N, K, B, g, xi = 64, 4096, 2, 1024, 0x48494747
+        grid = stored.load(2, 64)
+        W = inputs.make_weights(N, K, seed=19, bf16=True).astype(np.float64)
+        x = inputs.make_activations(B, K, seed=20).astype(np.float64)
+        Kr = K // world
+        k0 = rank * Kr                                                            # a multiple of the group size
+        xi_r = binding.higgs_shard_seed(xi, k0)                                   # the shard's signs are the layer's, shifted
+        q = oracle.quantize(W[:, k0:k0 + Kr], g, grid, xi_r)
+        sc = oracle.round_scales_fp16(q.scales).astype(np.float64)
+        part = oracle.linear_dense(x[:, k0:k0 + Kr], q.codes, sc, g, grid, xi_r)  # this rank's fp partial [B][N]
+        slots = [None] * world                                                    # what the epilogues write into every rank's slot buffer
+        dist.all_gather_object(slots, part)
+        dist.barrier()                                                            # "all partials written" before the reduction
+        y = np.zeros((B, N))
+        for r in range(world):                                                    # higgs_reduce_slots: slot order
+            y = y + slots[r]
+        q_all = oracle.quantize(W, g, grid, xi)
+        same_codes = bool(np.array_equal(q_all.codes[:, k0 // 2:(k0 + Kr) // 2], q.codes))
+        y_ref = oracle.linear_dense(x, q_all.codes, oracle.round_scales_fp16(q_all.scales).astype(np.float64), g, grid, xi)
+        out.put((rank, same_codes, float(np.max(np.abs(y - y_ref)) / np.max(np.abs(y_ref)))))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_k_sharded_layer_protocol_on_two_ranks():
+    """The rotation is local to a 1024-group (Appendix F), so a layer cut along K on group boundaries is a sum of
+    independent layers; with the shifted seed each shard carries exactly the codes of its columns of the unsharded
+    layer, and the slot-ordered sum of the partial outputs is the unsharded output (up to fp64 summation order)."""
+    world = 2
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_kshard_worker, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = sorted(out.get(timeout=300) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, same_codes, err in res:
+        assert same_codes
+        assert err < 1e-12
+
+
+def test_shard_seed_shifts_the_sign_sequence():
+    import oracle
+    from paper_2411_17525_b200 import binding
+    for xi in (0, 7, 0x48494747, 2**64 - 5):
+        for k0 in (0, 1024, 4096, 28672 - 1024):
+            s = binding.higgs_shard_seed(xi, k0)
+            assert [oracle.sign(s, j) for j in range(0, 2048, 37)] == [oracle.sign(xi, k0 + j) for j in range(0, 2048, 37)]
+
+
 def test_shard_rows_tiles_the_layer():
     from paper_2411_17525_b200 import binding
     for N, world in [(4096, 8), (14336, 8), (1024, 3), (128, 2), (8192, 5)]:
@@ -135,4 +200,5 @@ def test_reference_arm_prints_the_contract_line():
     assert line["steps"] == 2 and line["value"] > 0 and line["dtype"] == "f64" and line["vs_baseline"] is None
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["value"] == line["value"]
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
-    assert "llama-3.2-1b layer set (7 matrices), grid p=2 n=256, g=1024, batch 1" == line["config"]["workload"]
+    assert line["config"]["workload"].startswith("llama-3.1-70b layer set (7 matrices), grid mixed ")
+    assert line["config"]["workload"].endswith("g=1024, batch 1")
