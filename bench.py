@@ -502,7 +502,9 @@ def run_ours(args):
             grids[key], mse, iters = hb.higgs_make_grid(p, n, samples, max_iters=3000)
             e1.record()
             torch.cuda.synchronize()
-            grid_info[f"p={p} n={n}"] = {"ms": e0.elapsed_time(e1), "iters": int(iters), "mse": float(mse)}
+            it = int(iters)         # negative: the iteration limit was reached before the assignment stopped changing
+            grid_info[f"p={p} n={n}"] = {"ms": e0.elapsed_time(e1), "iters": abs(it), "converged": it > 0, "max_iters": 3000,
+                                         "mse": float(mse)}
         return grids[key]
 
     for key in sorted(set(pn)):

@@ -13,7 +13,7 @@ struct GridWs {
     unsigned long long* counts;   // [n]
     int32_t* assign;              // [m]
     double* err;                  // [2]: running, last completed
-    int32_t* flags;               // [0] changed, [1] done, [2] iterations
+    int32_t* flags;               // [0] changed, [1] done, [2] iterations, [3] grid-barrier arrivals (persistent fit)
 };
 
 __host__ __device__ inline size_t up256(size_t v) { return (v + 255) / 256 * 256; }
@@ -37,7 +37,7 @@ __global__ void grid_init_kernel(GridWs w, const float* __restrict__ samples, in
     if (i < (int64_t)n * p) { w.centres[i] = samples[i]; w.sums[i] = 0.0; }
     if (i < n) w.counts[i] = 0ull;
     if (i < 2) w.err[i] = 0.0;
-    if (i < 3) w.flags[i] = 0;
+    if (i < 8) w.flags[i] = 0;
 }
 
 // Assignment step.  The centres sit in dynamic shared memory ([n][P] floats, at most 64 KB).  SMALL (n <= 256): the
@@ -45,16 +45,15 @@ __global__ void grid_init_kernel(GridWs w, const float* __restrict__ samples, in
 // to the global sums directly (with thousands of cells the atomics rarely collide).  Distances are the plain
 // sum of (x_k - c_k)^2 in coordinate order, fp32, strict '<' (lowest index wins a tie) - the encoder's rule.
 template <int P, bool SMALL>
-__global__ void __launch_bounds__(256) grid_assign_kernel(GridWs w, const float* __restrict__ samples, int n, int64_t m) {
-    extern __shared__ __align__(16) unsigned char grid_smem[];
+__device__ __forceinline__ void assign_body(const GridWs& w, const float* __restrict__ samples, int n, int64_t m,
+                                            unsigned char* grid_smem) {
     float* sc = reinterpret_cast<float*>(grid_smem);
     double* ssum = reinterpret_cast<double*>(grid_smem + up256(sizeof(float) * n * P));
     unsigned int* scnt = reinterpret_cast<unsigned int*>(ssum + (SMALL ? n * P : 0));
     __shared__ double serr;
     __shared__ int schanged;
-    if (w.flags[1]) return;
     for (int i = threadIdx.x; i < n * P; i += blockDim.x) {
-        sc[i] = w.centres[i];
+        sc[i] = __ldcg(&w.centres[i]);       // (bypasses L1: in the persistent fit another block rewrote the centres)
         if (SMALL) ssum[i] = 0.0;
     }
     if (SMALL)
@@ -105,23 +104,74 @@ __global__ void __launch_bounds__(256) grid_assign_kernel(GridWs w, const float*
     }
 }
 
-__global__ void grid_update_kernel(GridWs w, int p, int n) {
+template <int P, bool SMALL>
+__global__ void __launch_bounds__(256) grid_assign_kernel(GridWs w, const float* __restrict__ samples, int n, int64_t m) {
+    extern __shared__ __align__(16) unsigned char grid_smem[];
     if (w.flags[1]) return;
-    const int changed = w.flags[0];
+    assign_body<P, SMALL>(w, samples, n, m, grid_smem);
+}
+
+__device__ __forceinline__ void update_body(const GridWs& w, int p, int n) {
+    const int changed = __ldcg(&w.flags[0]);
     __syncthreads();
     for (int i = threadIdx.x; i < n * p; i += blockDim.x) {
-        const unsigned long long cnt = w.counts[i / p];
-        if (changed && cnt) w.centres[i] = (float)(w.sums[i] / (double)cnt);
+        const unsigned long long cnt = __ldcg(&w.counts[i / p]);
+        if (changed && cnt) w.centres[i] = (float)(__ldcg(&w.sums[i]) / (double)cnt);
     }
     __syncthreads();
     for (int i = threadIdx.x; i < n * p; i += blockDim.x) w.sums[i] = 0.0;
     for (int i = threadIdx.x; i < n; i += blockDim.x) w.counts[i] = 0ull;
     if (threadIdx.x == 0) {
-        w.err[1] = w.err[0];
+        w.err[1] = __ldcg(&w.err[0]);
         w.err[0] = 0.0;
-        w.flags[2] += 1;
+        w.flags[2] = __ldcg(&w.flags[2]) + 1;
         w.flags[0] = 0;
         if (!changed) w.flags[1] = 1;
+    }
+}
+
+__global__ void grid_update_kernel(GridWs w, int p, int n) {
+    if (w.flags[1]) return;
+    update_body(w, p, n);
+}
+
+// ---- the whole iteration in ONE cooperatively launched kernel ---------------------------------------------------
+// Every block is resident (the launch fails otherwise), so the blocks can meet at a barrier between the assignment and
+// the update step: a counter in the workspace that every block's first thread increments and then polls, with a limit
+// on the polls - a barrier that runs out raises the grid-fit status word and every block leaves.
+__device__ int g_grid_status = 0;
+constexpr unsigned kGridBarrierLimit = 1u << 22;
+
+__device__ __forceinline__ bool grid_barrier(int32_t* counter, int target) {
+    __syncthreads();
+    int ok = 1;
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(counter, 1);
+        unsigned it = 0;
+        for (;;) {
+            int v;
+            asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(counter) : "memory");
+            if (v >= target) break;
+            if (++it > kGridBarrierLimit) { ok = 0; atomicExch(&g_grid_status, (int)HIGGS_ERR_TIMEOUT); break; }
+            __nanosleep(64);
+        }
+        __threadfence();
+    }
+    return __syncthreads_and(ok) != 0;
+}
+
+template <int P, bool SMALL>
+__global__ void __launch_bounds__(256) grid_fit_kernel(GridWs w, const float* __restrict__ samples, int n, int64_t m, int max_iters) {
+    extern __shared__ __align__(16) unsigned char grid_smem[];
+    const int blocks = (int)gridDim.x;
+    int barrier_no = 0;
+    for (int it = 0; it < max_iters; ++it) {
+        assign_body<P, SMALL>(w, samples, n, m, grid_smem);
+        if (!grid_barrier(&w.flags[3], ++barrier_no * blocks)) return;
+        if (blockIdx.x == 0) update_body(w, P, n);
+        if (!grid_barrier(&w.flags[3], ++barrier_no * blocks)) return;
+        if (*reinterpret_cast<volatile int32_t*>(&w.flags[1])) return;       // no assignment changed: a fixed point
     }
 }
 
@@ -230,6 +280,38 @@ static int assign_step(GridWs w, const float* samples, int n, int64_t m, unsigne
     return HIGGS_OK;
 }
 
+// One cooperative launch for the whole iteration; returns HIGGS_ERR_UNSUPPORTED when the device or the shape does not
+// allow it (the caller then enqueues one pair of kernels per iteration).
+static int sm_count_of_device() {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v < 1) v = 1;
+    return v;
+}
+
+template <int P, bool SMALL>
+static int fit_persistent(GridWs w, const float* samples, int n, int64_t m, int max_iters, cudaStream_t st) {
+    const size_t smem = up256(sizeof(float) * n * P) + (SMALL ? sizeof(double) * n * P + sizeof(unsigned int) * n : 0);
+    static int per_sm[64] = {0};          // resident blocks per SM at the largest shared-memory size, -1 = not available
+    const int bps = device_once(per_sm, [] {
+        int dev = 0, coop = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess || !coop)
+            return -1;
+        const size_t max_smem = up256(sizeof(float) * kMaxGridPoints * P) + (SMALL ? (sizeof(double) * P + sizeof(unsigned int)) * 256 : 0);
+        if (cudaFuncSetAttribute(grid_fit_kernel<P, SMALL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)max_smem) != cudaSuccess) return -1;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&v, grid_fit_kernel<P, SMALL>, 256, max_smem) != cudaSuccess || v < 1) return -1;
+        return v;
+    });
+    if (bps < 1) return HIGGS_ERR_UNSUPPORTED;
+    int64_t blocks = (m + 255) / 256;
+    const int64_t cap = (int64_t)bps * sm_count_of_device();
+    if (blocks > cap) blocks = cap;
+    if (blocks > 592) blocks = 592;
+    void* args[] = {&w, &samples, &n, &m, &max_iters};
+    const cudaError_t e = cudaLaunchCooperativeKernel((const void*)grid_fit_kernel<P, SMALL>, dim3((unsigned)blocks), dim3(256), args, smem, st);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return HIGGS_ERR_UNSUPPORTED; }
+    return HIGGS_OK;
+}
+
 int launch_make_grid(int p, int n, const float* samples, int64_t m, int max_iters, float* grid_out, float* mse_out,
                      int32_t* iters_out, void* ws, cudaStream_t st) {
     GridWs w = carve(ws, p, n, m);
@@ -238,6 +320,24 @@ int launch_make_grid(int p, int n, const float* samples, int64_t m, int max_iter
     int64_t blocks = (m + 255) / 256;
     if (blocks > 592) blocks = 592;
     const bool small = n <= 256;
+    {
+        int rc = HIGGS_ERR_UNSUPPORTED;
+        switch (p * 2 + (small ? 1 : 0)) {
+            case 3: rc = fit_persistent<1, true>(w, samples, n, m, max_iters, st); break;
+            case 2: rc = fit_persistent<1, false>(w, samples, n, m, max_iters, st); break;
+            case 5: rc = fit_persistent<2, true>(w, samples, n, m, max_iters, st); break;
+            case 4: rc = fit_persistent<2, false>(w, samples, n, m, max_iters, st); break;
+            case 7: rc = fit_persistent<3, true>(w, samples, n, m, max_iters, st); break;
+            case 6: rc = fit_persistent<3, false>(w, samples, n, m, max_iters, st); break;
+            case 9: rc = fit_persistent<4, true>(w, samples, n, m, max_iters, st); break;
+            case 8: rc = fit_persistent<4, false>(w, samples, n, m, max_iters, st); break;
+            default: return HIGGS_ERR_UNSUPPORTED;
+        }
+        if (rc == HIGGS_OK) {
+            grid_finalize_kernel<<<1, 256, 0, st>>>(w, p, n, m, grid_out, mse_out, iters_out);
+            return cuda_status(cudaGetLastError());
+        }
+    }
     for (int it = 0; it < max_iters; ++it) {
         int rc;
         switch (p * 2 + (small ? 1 : 0)) {
@@ -256,6 +356,16 @@ int launch_make_grid(int p, int n, const float* samples, int64_t m, int max_iter
     }
     grid_finalize_kernel<<<1, 256, 0, st>>>(w, p, n, m, grid_out, mse_out, iters_out);
     return cuda_status(cudaGetLastError());
+}
+
+int read_grid_status(int clear) {
+    int v = 0;
+    if (cudaMemcpyFromSymbol(&v, g_grid_status, sizeof(int)) != cudaSuccess) return HIGGS_ERR_CUDA;
+    if (clear && v != 0) {
+        const int zero = 0;
+        if (cudaMemcpyToSymbol(g_grid_status, &zero, sizeof(int)) != cudaSuccess) return HIGGS_ERR_CUDA;
+    }
+    return v;
 }
 
 }  // namespace higgs

@@ -1056,7 +1056,8 @@ int read_device_status(cudaStream_t st, int clear) {
         if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)) != cudaSuccess) return HIGGS_ERR_CUDA;
     }
     const int tc = read_tc_status(clear);
-    return v != 0 ? v : tc;
+    const int gf = read_grid_status(clear);
+    return v != 0 ? v : tc != 0 ? tc : gf;
 }
 
 }  // namespace higgs
