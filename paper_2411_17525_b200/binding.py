@@ -236,12 +236,18 @@ def higgs_selftest_wait(which: int, polls: int, device=None) -> torch.Tensor:
 
 
 def higgs_quantize(desc: higgs_desc, W: torch.Tensor, grid: torch.Tensor, want_canonical: bool = False,
-                   workspace: Optional[torch.Tensor] = None):
-    """W: cuda [N][K] fp32 or bf16; grid: cuda [n][p] fp32.  Returns (packed u8, scales fp16 tile-major [N/16][K/g][16], canonical u8 or None)."""
+                   workspace: Optional[torch.Tensor] = None, out=None):
+    """W: cuda [N][K] fp32 or bf16; grid: cuda [n][p] fp32.  Returns (packed u8, scales fp16 tile-major [N/16][K/g][16], canonical u8 or None).
+    out = (packed, scales) reuses existing output tensors."""
     assert W.is_cuda and W.is_contiguous() and grid.is_cuda and grid.dtype == torch.float32 and grid.is_contiguous()
     dev = W.device
-    packed = torch.empty(max(higgs_packed_bytes(desc), 16), dtype=torch.uint8, device=dev)
-    scales = torch.empty((desc.N // 16, max(desc.K // desc.g, 0), 16), dtype=torch.float16, device=dev)
+    if out is not None:
+        packed, scales = out
+        assert packed.is_cuda and packed.dtype == torch.uint8 and packed.numel() >= higgs_packed_bytes(desc)
+        assert scales.is_cuda and scales.dtype == torch.float16 and scales.numel() * 2 >= higgs_scales_bytes(desc)
+    else:
+        packed = torch.empty(max(higgs_packed_bytes(desc), 16), dtype=torch.uint8, device=dev)
+        scales = torch.empty((desc.N // 16, max(desc.K // desc.g, 0), 16), dtype=torch.float16, device=dev)
     canonical = torch.empty((desc.N, desc.K // desc.p), dtype=torch.uint8, device=dev) if want_canonical else None
     if workspace is None:
         workspace = _workspace(higgs_workspace_bytes(desc, HIGGS_OP_QUANTIZE), dev)

@@ -891,7 +891,8 @@ Plan make_plan(const higgs_desc& d, int64_t B) {
         if (ck / ks > kWarps) continue;
         const int chunks = (int)(d.K / ck);
         int64_t parts = sms / chunks;
-        const bool pair = chunks == 2 && d.K > (int64_t)kWarps * ks && pair_capacity() > 0;
+        // (one token block only: with nine or more tokens the flush of twice sixteen larger tiles costs more than the atomics)
+        const bool pair = nb == 1 && chunks == 2 && d.K > (int64_t)kWarps * ks && pair_capacity() > 0;
         if (pair && parts > pair_capacity()) parts = pair_capacity();
         if (parts < 1) parts = 1;
         if (parts > tiles) parts = tiles;

@@ -593,11 +593,10 @@ def test_linear_tensor_core_path_bf16_output(N, K, B):
     (2, 16, 2048, 8192, 2, torch.float32),      # nibble format: partial tiles behind the table
     (1, 256, 2368, 8192, 3, torch.float32),     # 8-bit scalar codes
     (2, 256, 2048, 8192, 5, torch.float32),     # rotation kernel + product, generic flusher
-    (2, 256, 768, 4096, 16, torch.float32),     # two token blocks per MMA step (128-input slices)
     (1, 16, 1184, 8192, 8, torch.bfloat16),
 ])
 def test_two_k_chunks_meet_in_a_cluster_pair_in_a_fixed_order(p, n, N, K, B, dtype):
-    """K ranges of 2 x 4096 inputs (2 x 2048 when nine or more tokens halve the slices): the two blocks of a thread-block
+    """K ranges of 2 x 4096 inputs at up to eight tokens: the two blocks of a thread-block
     cluster take them, item j is summed by block j % 2 in a fixed order.  Checked against the oracle, bit for bit
     between two runs, and the call must report that it uses no atomics."""
     xi = 2024
