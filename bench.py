@@ -550,9 +550,19 @@ def run_ours(args):
         groups_of.setdefault(key if key else f"own{li}", []).append(li)
     xdags = {k: torch.empty(hb.higgs_rotated_bytes(descs[v[0]], B) // 2, dtype=torch.float16, device=dev)
              for k, v in groups_of.items() if len(v) > 1}
+    # a sharing group whose layers also share a grid runs as ONE product over the concatenated rows (higgs_linear_multi:
+    # rows are independent); otherwise the first layer rotates for the others (higgs_linear_share)
+    multis = {}
+    for k, v in groups_of.items():
+        if len(v) > 1 and len({qs[li].pn for li in v}) == 1:
+            multis[k] = [hb.MultiLinear([descs[li] for li in v], [qs[li].packed[c] for li in v], [qs[li].scales[c] for li in v],
+                                        qs[v[0]].grid, [ys[li] for li in v], B) for c in range(copies)]
+    merged_names = ", ".join("|".join(names[li] for li in groups_of[k]) for k in multis) or "none"
     launches_per_step = 0
     for k, v in groups_of.items():
-        if len(v) > 1:      # one rotation, then one product launch per layer (per 16 tokens on the small-batch path);
+        if k in multis:
+            launches_per_step += multis[k][0].launches
+        elif len(v) > 1:    # one rotation, then one product launch per layer (per 16 tokens on the small-batch path);
                             # for 1-2 tokens the first product rotates x itself and leaves the result for the others
             first_is_one_launch = hb.higgs_linear_launch_count(descs[v[0]], B) == 1
             launches_per_step += (0 if first_is_one_launch else 1) + \
@@ -563,7 +573,9 @@ def run_ours(args):
     def step(i):
         c = i % copies
         for key, lis in groups_of.items():
-            if len(lis) > 1:      # the first layer of the group also produces the rotated activations of the others
+            if key in multis:
+                hb.higgs_linear_multi(multis[key][c], xs[lis[0]])
+            elif len(lis) > 1:    # the first layer of the group also produces the rotated activations of the others
                 li = lis[0]
                 hb.higgs_linear_share(descs[li], xs[li], qs[li].packed[c], qs[li].scales[c], qs[li].grid, xdag_out=xdags[key],
                                       workspace=ws[li], y=ys[li])
@@ -822,6 +834,7 @@ def run_ours(args):
         for q in qs:
             del q.packed[1:], q.scales[1:]
         host_batches = None
+        multis = None
         graphs = None
         torch.cuda.empty_cache()
         detail["other_configurations"] = other_configurations(hb, torch, oracle, dev, stream, peak, peak_tf, fit_grid)
@@ -844,7 +857,7 @@ def run_ours(args):
                        "global_batch": B * world, "parallelism": f"replicas x{world}",
                        "l2": f"rotating {copies} weight copies ({copies * set_bytes / 1e6:.0f} MB > 126 MB L2)",
                        "launch": "direct" if args.no_graph else f"CUDA graphs of {spg} consecutive steps over rotating weight copies ({args.steps // spg} replays timed)",
-                       "step": "one transformer block: activation rotations (q/k/v and gate/up share theirs where the layout allows: the first layer of the group goes through higgs_linear_share, which for 1-2 tokens rotates inside its product kernel and leaves the result for the others; a layer with its own rotation has it fused likewise when K is not split) + 7 products"},
+                       "step": "one transformer block, 7 matrices: layers that read the same input and share a grid (here: " + merged_names + ") run as one product over their concatenated rows (higgs_linear_multi); other sharing layers share one rotation (higgs_linear_share + higgs_linear_prerotated); a layer with its own input goes through higgs_linear; for 1-2 tokens the rotation runs inside the product kernel"},
             "us_per_layer": ms_per_step * 1e3 / len(layers),
             "weight_bytes_per_step": set_bytes,
             "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

@@ -253,6 +253,24 @@ int higgs_linear_share(const higgs_desc* desc, const void* x, int64_t B, const v
                        size_t workspace_bytes, void* stream);
 
 /*
+ * Several layers that read the same activations (q, k, v; gate, up) as ONE product: Appendix F's product is
+ * independent per output row, so matrices with the same K, grid, group size and seed are one layer over their
+ * concatenated rows - the activations are rotated once and, for batches up to 16 (the small-batch kernel, K ranges
+ * not meeting in atomics), one kernel launch per 16 tokens streams all of them; for one or two tokens that launch also
+ * does the rotation.  Other shapes and batches run as one higgs_linear per matrix (same results, no gain).
+ *   count <= 4; descs[i], packed[i], scales[i], ys[i] (device [B][descs[i]->N] of y_dtype) belong to matrix i;
+ *   descs must agree in p, n, g, K, rht_seed (else HIGGS_ERR_INVALID_ARG); grid and x are common;
+ *   workspace: higgs_linear_multi_workspace_bytes(count, descs, B) bytes.  The arrays are HOST arrays.
+ * Results equal those of higgs_linear on each matrix (bit for bit where neither uses atomics).
+ * higgs_linear_multi_launch_count: kernels the call enqueues.
+ */
+int higgs_linear_multi(int32_t count, const higgs_desc* const* descs, const void* x, int64_t B,
+                       const void* const* packed, const void* const* scales, const float* grid,
+                       void* const* ys, int y_dtype, void* workspace, size_t workspace_bytes, void* stream);
+size_t higgs_linear_multi_workspace_bytes(int32_t count, const higgs_desc* const* descs, int64_t B);
+int higgs_linear_multi_launch_count(int32_t count, const higgs_desc* const* descs, int64_t B, int y_dtype);
+
+/*
  * Row-sharded layer with the all-gather fused into the product's epilogue (Appendix F's product is independent per
  * output row, and the rotation is local to a 1024-group of inputs, so a layer splits over devices by rows with no
  * exchange of weights): this device holds rows [row_offset, row_offset + desc->N) of a layer with `ld` rows in all

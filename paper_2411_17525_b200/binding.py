@@ -29,7 +29,8 @@ EXPORTS = [
     "higgs_rotated_layout", "higgs_dequantize", "higgs_make_uniform_grid", "higgs_layer_error",
     "higgs_allocate_bits", "higgs_general_tuples", "higgs_quantize_general", "higgs_linear_host_batch",
     "higgs_linear_gather", "higgs_linear_share", "higgs_make_grid_seeded", "higgs_gaussian_samples", "higgs_shard_rows",
-    "higgs_launch_floor", "higgs_selftest_wait", "higgs_linear_uses_atomics", "higgs_shard_seed", "higgs_linear_kshard", "higgs_reduce_slots",
+    "higgs_launch_floor", "higgs_selftest_wait", "higgs_linear_uses_atomics", "higgs_shard_seed", "higgs_linear_kshard", "higgs_reduce_slots", "higgs_linear_multi", "higgs_linear_multi_workspace_bytes",
+    "higgs_linear_multi_launch_count",
 ]
 
 
@@ -123,6 +124,12 @@ def _load() -> ctypes.CDLL:
     lib.higgs_gaussian_samples.argtypes = [i32, u64, i64, vp, vp]
     lib.higgs_shard_rows.restype = i32
     lib.higgs_shard_rows.argtypes = [i64, i32, i32, i32, ctypes.POINTER(i64), ctypes.POINTER(i64)]
+    lib.higgs_linear_multi.restype = i32
+    lib.higgs_linear_multi.argtypes = [i32, vp, vp, i64, vp, vp, vp, vp, i32, vp, sz, vp]
+    lib.higgs_linear_multi_workspace_bytes.restype = sz
+    lib.higgs_linear_multi_workspace_bytes.argtypes = [i32, vp, i64]
+    lib.higgs_linear_multi_launch_count.restype = i32
+    lib.higgs_linear_multi_launch_count.argtypes = [i32, vp, i64, i32]
     lib.higgs_shard_seed.restype = u64
     lib.higgs_shard_seed.argtypes = [u64, i64]
     lib.higgs_linear_kshard.restype = i32
@@ -363,6 +370,40 @@ def higgs_linear_gather(desc: higgs_desc, x: torch.Tensor, packed: torch.Tensor,
     _check(lib.higgs_linear_gather(ctypes.byref(desc), _ptr(x), B, _ptr(packed), _ptr(scales), _ptr(grid), ptrs, len(y_dsts),
                                    ld, int(row_offset), _dtype_code(y_dsts[0]), _ptr(workspace), workspace.numel(), _stream()),
            "higgs_linear_gather")
+
+
+class MultiLinear:
+    """Argument arrays of higgs_linear_multi, marshalled once: several matrices (same K, grid and seed) that read the
+    same activations and run as one product over their concatenated rows."""
+
+    def __init__(self, descs, packed, scales, grid, ys, B, workspace=None):
+        n = len(descs)
+        assert n == len(packed) == len(scales) == len(ys)
+        self.keep = (list(descs), list(packed), list(scales), grid, list(ys))
+        self.count, self.B, self.grid = n, int(B), grid
+        arr = ctypes.c_void_p * n
+        self.descs = arr(*[ctypes.addressof(d) for d in descs])
+        self.packed = arr(*[t.data_ptr() for t in packed])
+        self.scales = arr(*[t.data_ptr() for t in scales])
+        self.ys = arr(*[t.data_ptr() for t in ys])
+        self.y_dtype = _dtype_code(ys[0])
+        need = int(lib.higgs_linear_multi_workspace_bytes(n, self.descs, self.B))
+        self.workspace = workspace if workspace is not None else _workspace(need, ys[0].device)
+        assert self.workspace.numel() >= need
+        self.launches = int(lib.higgs_linear_multi_launch_count(n, self.descs, self.B, self.y_dtype))
+
+    def set_weights(self, packed, scales):
+        self.keep = (self.keep[0], list(packed), list(scales)) + self.keep[3:]
+        for i, (p, s) in enumerate(zip(packed, scales)):
+            self.packed[i] = p.data_ptr()
+            self.scales[i] = s.data_ptr()
+
+
+def higgs_linear_multi(m: MultiLinear, x: torch.Tensor) -> None:
+    """Enqueues the product of every matrix of `m` with x ([B][K] bf16) on the current stream; outputs land in m's ys."""
+    assert x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous() and x.shape[0] == m.B
+    _check(lib.higgs_linear_multi(m.count, m.descs, _ptr(x), m.B, m.packed, m.scales, _ptr(m.grid), m.ys, m.y_dtype,
+                                  _ptr(m.workspace), m.workspace.numel(), _stream()), "higgs_linear_multi")
 
 
 def higgs_shard_seed(rht_seed: int, k_offset: int) -> int:

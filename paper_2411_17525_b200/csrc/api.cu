@@ -343,6 +343,98 @@ int higgs_linear_share(const higgs_desc* d, const void* x, int64_t B, const void
     return higgs_linear_prerotated(d, xdag_out, B, packed, scales, grid, y, y_dtype, workspace, workspace_bytes, stream);
 }
 
+size_t higgs_linear_multi_workspace_bytes(int32_t count, const higgs_desc* const* descs, int64_t B) {
+    if (count < 1 || count > kMaxMulti || !descs || !descs[0]) return 0;
+    higgs_desc v = *descs[0];
+    size_t most = 0;
+    v.N = 0;
+    for (int i = 0; i < count; ++i) {
+        if (!descs[i]) return 0;
+        v.N += descs[i]->N;
+        const size_t one = higgs_workspace_bytes(descs[i], HIGGS_OP_LINEAR, B);
+        if (one == 0 && descs[i]->N != 0) return 0;
+        most = one > most ? one : most;
+    }
+    const size_t all = higgs_workspace_bytes(&v, HIGGS_OP_LINEAR, B);
+    return all > most ? all : most;
+}
+
+int higgs_linear_multi(int32_t count, const higgs_desc* const* descs, const void* x, int64_t B, const void* const* packed,
+                       const void* const* scales, const float* grid, void* const* ys, int y_dtype, void* workspace,
+                       size_t workspace_bytes, void* stream) {
+    if (count < 1 || count > kMaxMulti || !descs || !packed || !scales || !ys) return HIGGS_ERR_INVALID_ARG;
+    if (y_dtype != HIGGS_F32 && y_dtype != HIGGS_BF16) return HIGGS_ERR_UNSUPPORTED;
+    if (B < 0) return HIGGS_ERR_INVALID_ARG;
+    higgs_desc v;
+    MultiSegments segs;
+    segs.count = 0;
+    for (int i = 0; i < count; ++i) {
+        const higgs_desc* d = descs[i];
+        const int rc = check_desc(d);
+        if (rc != HIGGS_OK) return rc;
+        if (i == 0) { v = *d; v.N = 0; }
+        else if (d->p != v.p || d->n != v.n || d->g != v.g || d->K != v.K || d->rht_seed != v.rht_seed) return HIGGS_ERR_INVALID_ARG;
+        if (d->N == 0) continue;
+        if (!packed[i] || !scales[i] || !ys[i] || !aligned(packed[i], 16) || !aligned(scales[i], 16) || !aligned(ys[i], 16))
+            return HIGGS_ERR_INVALID_ARG;
+        segs.rows[segs.count] = d->N;
+        segs.packed[segs.count] = packed[i];
+        segs.scales[segs.count] = scales[i];
+        segs.y[segs.count] = ys[i];
+        ++segs.count;
+        v.N += d->N;
+    }
+    if (B == 0 || v.N == 0) return HIGGS_OK;
+    if (v.K == 0) return HIGGS_ERR_UNSUPPORTED;
+    if (!x || !grid || !workspace || !aligned(x, 16) || !aligned(workspace, 256)) return HIGGS_ERR_INVALID_ARG;
+    if (workspace_bytes < higgs_linear_multi_workspace_bytes(count, descs, B)) return HIGGS_ERR_WORKSPACE;
+    cudaStream_t st = as_stream(stream);
+    const int mode = y_dtype == HIGGS_F32 ? 0 : 1;
+    if (segs.count > 1 && B <= 16 && !tc_eligible(v, B) && !linear_uses_atomics(v, B)) {
+        // ONE launch of the small-batch kernel over the concatenated rows (per 16 tokens), the rotation done once
+        if (linear_fused_eligible(v, B))
+            return launch_linear_mma(v, nullptr, B, segs.packed[0], segs.scales[0], grid, segs.y[0], segs.rows[0], mode, st, x,
+                                     nullptr, nullptr, &segs);
+        __half* xdag = static_cast<__half*>(workspace);
+        int rc = launch_rht_activations(v, x, B, xdag, nullptr, 0, st);
+        if (rc != HIGGS_OK) return rc;
+        const size_t esz = y_dtype == HIGGS_F32 ? 4 : 2;
+        for (int64_t b0 = 0; b0 < B; b0 += 16) {
+            const int64_t bn = B - b0 < 16 ? B - b0 : 16;
+            MultiSegments part = segs;
+            for (int i = 0; i < segs.count; ++i) part.y[i] = static_cast<uint8_t*>(segs.y[i]) + (size_t)b0 * segs.rows[i] * esz;
+            rc = launch_linear_mma(v, xdag + b0 * v.K, bn, part.packed[0], part.scales[0], grid, part.y[0], part.rows[0], mode, st,
+                                   nullptr, nullptr, nullptr, &part);
+            if (rc != HIGGS_OK) return rc;
+        }
+        return HIGGS_OK;
+    }
+    // other shapes and batches (tensor-core path, K ranges that meet in atomics): one higgs_linear per matrix
+    for (int i = 0; i < count; ++i) {
+        if (descs[i]->N == 0) continue;
+        const int rc = higgs_linear(descs[i], x, B, packed[i], scales[i], grid, ys[i], y_dtype, workspace, workspace_bytes, stream);
+        if (rc != HIGGS_OK) return rc;
+    }
+    return HIGGS_OK;
+}
+
+int higgs_linear_multi_launch_count(int32_t count, const higgs_desc* const* descs, int64_t B, int y_dtype) {
+    if (count < 1 || count > kMaxMulti || !descs || B < 1) return 0;
+    higgs_desc v = *descs[0];
+    v.N = 0;
+    int live = 0, separate = 0;
+    for (int i = 0; i < count; ++i) {
+        if (check_desc(descs[i]) != HIGGS_OK) return 0;
+        if (descs[i]->N == 0) continue;
+        v.N += descs[i]->N;
+        ++live;
+        separate += higgs_linear_launch_count(descs[i], B, y_dtype);
+    }
+    if (live > 1 && B <= 16 && !tc_eligible(v, B) && !linear_uses_atomics(v, B))
+        return linear_fused_eligible(v, B) ? 1 : 1 + (int)((B + 15) / 16);
+    return separate;
+}
+
 int higgs_linear_gather(const higgs_desc* d, const void* x, int64_t B, const void* packed, const void* scales,
                         const float* grid, void* const* y_dsts, int32_t n_dst, int64_t ld, int64_t row_offset, int y_dtype,
                         void* workspace, size_t workspace_bytes, void* stream) {

@@ -186,10 +186,21 @@ struct GatherTargets {
     void* y[kMaxGather - 1];
     int count;
 };
+// Several matrices with the same K, grid and seed that read the same activations, run as one product over their
+// concatenated rows (rows are independent in Appendix F's product): matrix i has rows[i] rows, its own packed stream,
+// scales and output [B][rows[i]].
+constexpr int kMaxMulti = 4;
+struct MultiSegments {
+    int count;
+    int64_t rows[kMaxMulti];
+    const void* packed[kMaxMulti];
+    const void* scales[kMaxMulti];
+    void* y[kMaxMulti];
+};
 // x_raw != nullptr: the activations as given (bf16); the kernel rotates them itself (only if linear_fused_eligible)
 int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const void* packed, const void* scales,
                       const float* grid, void* y, int64_t ldy, int y_mode, cudaStream_t st, const void* x_raw = nullptr,
-                      const GatherTargets* more = nullptr, __half* xdag_emit = nullptr);
+                      const GatherTargets* more = nullptr, __half* xdag_emit = nullptr, const MultiSegments* segs = nullptr);
 int launch_scatter_out(const float* y32, int64_t B, int64_t N, void* const* dsts, int n_dst, int64_t ldy, int y_dtype,
                        cudaStream_t st);
 bool linear_fused_eligible(const higgs_desc& d, int64_t B);

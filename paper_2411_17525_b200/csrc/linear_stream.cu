@@ -29,6 +29,8 @@ __device__ int g_device_status = 0;
 
 namespace {
 
+constexpr int kMaxSegments = 4;      // matrices one multi-matrix product takes
+
 struct StreamParams {
     const __nv_bfloat16* x;   // fused-rotation kernels only: [B][K] activations as the caller gave them
     unsigned long long xi;    // ... and the seed of the sign sequence
@@ -53,6 +55,15 @@ struct StreamParams {
     int log_ns;            // log2 of NS = ck / KS (slices per item)
     int tile_pieces;       // 128-byte pieces of one partial tile
     int acc_slots, acc_shift;   // items whose partial tiles may be parked at once (a power of two) and its log2
+    // Several matrices that read the same activations (q|k|v, gate|up) as ONE product: segment s holds the row tiles
+    // [seg_tile[s], seg_tile[s+1]) of the concatenated row space, with its own packed stream, scales and output.
+    // nseg == 1: the plain case, the fields above apply.
+    int nseg;
+    int seg_tile[kMaxSegments + 1];
+    const uint8_t* seg_packed[kMaxSegments];
+    const __half* seg_scales[kMaxSegments];
+    void* seg_y[kMaxSegments];
+    int64_t seg_ldy[kMaxSegments];
     int depth, warps_in_a; // ring depth and warps whose slots lie below the table, valid when the dynamic
                            // shared-memory window starts at offset kAssumedBase (else recomputed on the device)
 };
@@ -381,14 +392,37 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     // one K-chunk, so source addresses advance by constant strides.
     const int64_t kslice = (int64_t)chunk_begin * prm.ck + (int64_t)slice * KS;
     const int64_t rt_first = rt_begin + phase;
-    const uint8_t* src_next = prm.packed + (SIX ? ((rt_first * (prm.K >> 7) + (kslice >> 7)) * 768)
-                                                : ((rt_first * (prm.K >> 6) + (kslice >> 6)) * (NIB ? 256 : B8 ? 1024 : 512)));
-    const __half* ssrc_next = prm.scales + (rt_first * groups + chunk_begin * ng + gl) * 16;
+    // source of the task (row tile rt of a matrix whose streams start at `packed` / `scales`, this warp's slice)
+    auto code_src = [&](const uint8_t* packed, int64_t rt) {
+        return packed + (SIX ? ((rt * (prm.K >> 7) + (kslice >> 7)) * 768)
+                             : ((rt * (prm.K >> 6) + (kslice >> 6)) * (NIB ? 256 : B8 ? 1024 : 512)));
+    };
+    auto scale_src = [&](const __half* scales, int64_t rt) { return scales + (rt * groups + chunk_begin * ng + gl) * 16; };
+    // multi-matrix product: segment of a row tile of the concatenated row space (explicit selects: indexing the
+    // parameter arrays with a run-time index would copy them to local memory)
+    auto seg_of = [&](int rt) { return (int)(rt >= prm.seg_tile[1]) + (int)(rt >= prm.seg_tile[2]) + (int)(rt >= prm.seg_tile[3]); };
+    auto seg_begin = [&](int sg) { return sg == 0 ? 0 : sg == 1 ? prm.seg_tile[1] : sg == 2 ? prm.seg_tile[2] : prm.seg_tile[3]; };
+    auto seg_end = [&](int sg) { return sg == 0 ? prm.seg_tile[1] : sg == 1 ? prm.seg_tile[2] : sg == 2 ? prm.seg_tile[3] : prm.seg_tile[4]; };
+    auto seg_pk = [&](int sg) { return sg == 0 ? prm.seg_packed[0] : sg == 1 ? prm.seg_packed[1] : sg == 2 ? prm.seg_packed[2] : prm.seg_packed[3]; };
+    auto seg_sc = [&](int sg) { return sg == 0 ? prm.seg_scales[0] : sg == 1 ? prm.seg_scales[1] : sg == 2 ? prm.seg_scales[2] : prm.seg_scales[3]; };
+    const bool multi = prm.nseg > 1;
+    int rt_issue = (int)rt_first;          // row tile of the next task to request
+    int issue_seg_end = 0x7fffffff;        // multi: first row tile beyond the segment the cursors below point into
+    const uint8_t* src_next = code_src(prm.packed, rt_first);
+    const __half* ssrc_next = scale_src(prm.scales, rt_first);
+    if (multi) issue_seg_end = 0;          // forces the first task to locate its segment
     const int64_t src_stride = (int64_t)PG * (SIX ? prm.K * 6 : NIB ? prm.K * 4 : B8 ? prm.K * 16 : prm.K * 8);
     const int64_t ssrc_stride = (int64_t)PG * groups * 16;
     uint32_t elected;
     asm volatile("{ .reg .pred p; elect.sync _|p, 0xffffffff; selp.u32 %0, 1, 0, p; }" : "=r"(elected));
     auto issue = [&](int d) {   // whole warp: start the copies of the next task into slot d (elected lane issues)
+        if (multi && rt_issue >= issue_seg_end) {       // the task is the first this warp takes from its matrix
+            const int sg = seg_of(rt_issue);
+            src_next = code_src(seg_pk(sg), rt_issue - seg_begin(sg));
+            ssrc_next = scale_src(seg_sc(sg), rt_issue - seg_begin(sg));
+            issue_seg_end = seg_end(sg);
+        }
+        rt_issue += PG;
         const uint32_t dst = slot_addr(d), bar = full_bar(d);
         if (elected) {
             mbar_expect_tx(bar, Codes::kBytes + 32u);
@@ -581,7 +615,15 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
         for (int j = (int)my_rank; j < n_items; j += kHomes) {
             const int jj = PAIR ? (j >> 1) : j;
             const int q = jj & (acc_slots - 1), gen = jj >> acc_shift;
-            const int f_rt = rt_begin + j;
+            int f_rt = rt_begin + j;
+            void* yb = prm.y;
+            int64_t ldy = prm.ldy;
+            if (multi) {          // this row tile's matrix: its output and the tile's index inside it
+                const int sg = seg_of(f_rt);
+                yb = sg == 0 ? prm.seg_y[0] : sg == 1 ? prm.seg_y[1] : sg == 2 ? prm.seg_y[2] : prm.seg_y[3];
+                ldy = sg == 0 ? prm.seg_ldy[0] : sg == 1 ? prm.seg_ldy[1] : sg == 2 ? prm.seg_ldy[2] : prm.seg_ldy[3];
+                f_rt -= seg_begin(sg);
+            }
             if (!mbar_wait_relaxed(item_bars + 8u * q, (uint32_t)(gen & 1), abort_flag)) break;
             auto recycle = [&]() {      // the partial tiles are in registers: hand the slot back (to both blocks of a pair)
                 __syncwarp();
@@ -617,15 +659,15 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
                 recycle();
                 const int col = lane >> 4, row = lane & 15;
                 if (col < prm.B) {
-                    const int64_t o = (int64_t)col * prm.ldy + (int64_t)f_rt * 16 + row;
+                    const int64_t o = (int64_t)col * ldy + (int64_t)f_rt * 16 + row;
                     if (prm.y_mode == 0) {
-                        static_cast<float*>(prm.y)[o] = sum;
+                        static_cast<float*>(yb)[o] = sum;
                         if (prm.n_more) gather_store1(&prm, o, sum);
                     } else if (prm.y_mode == 1) {
-                        static_cast<__nv_bfloat16*>(prm.y)[o] = __float2bfloat16_rn(sum);
+                        static_cast<__nv_bfloat16*>(yb)[o] = __float2bfloat16_rn(sum);
                         if (prm.n_more) gather_store1(&prm, o, sum);
                     } else {
-                        asm volatile("red.global.add.f32 [%0], %1;" ::"l"(static_cast<float*>(prm.y) + o), "f"(sum) : "memory");
+                        asm volatile("red.global.add.f32 [%0], %1;" ::"l"(static_cast<float*>(yb) + o), "f"(sum) : "memory");
                     }
                 }
                 continue;
@@ -668,17 +710,17 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
                 const int col = e >> 4, row = e & 15;
                 if (col < prm.B) {
                     const float4 sum = sums[qq];
-                    const int64_t o = (int64_t)col * prm.ldy + (int64_t)f_rt * 16 + row;
+                    const int64_t o = (int64_t)col * ldy + (int64_t)f_rt * 16 + row;
                     if (prm.y_mode == 0) {
-                        *reinterpret_cast<float4*>(static_cast<float*>(prm.y) + o) = sum;
+                        *reinterpret_cast<float4*>(static_cast<float*>(yb) + o) = sum;
                         if (prm.n_more) gather_store(&prm, o, sum);   // gathered output: the other devices' copies
                     } else if (prm.y_mode == 1) {
                         __nv_bfloat162 lo = __floats2bfloat162_rn(sum.x, sum.y), hi = __floats2bfloat162_rn(sum.z, sum.w);
                         uint2 pk = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
-                        *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(prm.y) + o) = pk;
+                        *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(yb) + o) = pk;
                         if (prm.n_more) gather_store(&prm, o, sum);
                     } else {
-                        asm volatile("red.global.add.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(static_cast<float*>(prm.y) + o),
+                        asm volatile("red.global.add.v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(static_cast<float*>(yb) + o),
                                      "f"(sum.x), "f"(sum.y), "f"(sum.z), "f"(sum.w)
                                      : "memory");
                     }
@@ -946,11 +988,12 @@ bool linear_fused_eligible(const higgs_desc& d, int64_t B) {
 // y_mode: 0 store fp32, 1 store bf16, 2 atomicAdd fp32 (target must be zero).  B <= 16.
 int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const void* packed, const void* scales,
                       const float* grid, void* y, int64_t ldy, int y_mode, cudaStream_t st, const void* x_raw,
-                      const GatherTargets* more, __half* xdag_emit) {
+                      const GatherTargets* more, __half* xdag_emit, const MultiSegments* segs) {
     if (d.N == 0) return HIGGS_OK;
     if (more && more->count > 0 && (y_mode == 2 || more->count > kMaxGather - 1)) return HIGGS_ERR_INVALID_ARG;
     const Plan pl = make_plan(d, B);
     if (pl.pair && y_mode == 2) y_mode = 0;          // a cluster pair sums in shared memory and stores
+    if (segs && (segs->count < 1 || segs->count > kMaxSegments || y_mode == 2 || (more && more->count > 0))) return HIGGS_ERR_INVALID_ARG;
     if (pl.items == 0) return HIGGS_ERR_UNSUPPORTED;
     // the kernel's work split is 32-bit arithmetic: (row tiles) x (blocks per K-chunk) must stay below 2^31
     if ((d.N / kRowTile) * (int64_t)(pl.parts + 1) >= ((int64_t)1 << 31)) return HIGGS_ERR_UNSUPPORTED;
@@ -974,6 +1017,27 @@ int launch_linear_mma(const higgs_desc& d, const __half* xdag, int64_t B, const 
     prm.bits = code_bits(d.n);
     prm.ck = pl.ck;
     prm.y_mode = y_mode;
+    prm.nseg = segs ? segs->count : 1;
+    {
+        int tile = 0;
+        for (int i = 0; i < kMaxSegments; ++i) {
+            const bool live = segs && i < segs->count;
+            prm.seg_tile[i] = live ? tile : 0x7fffffff;          // (segments beyond the last never match a row tile)
+            prm.seg_packed[i] = live ? static_cast<const uint8_t*>(segs->packed[i]) : nullptr;
+            prm.seg_scales[i] = live ? static_cast<const __half*>(segs->scales[i]) : nullptr;
+            prm.seg_y[i] = live ? segs->y[i] : nullptr;
+            prm.seg_ldy[i] = live ? segs->rows[i] : 0;
+            if (live) tile += (int)(segs->rows[i] / kRowTile);
+        }
+        prm.seg_tile[kMaxSegments] = 0x7fffffff;
+        if (segs) {
+            prm.seg_tile[segs->count] = tile;
+            if ((int64_t)tile * kRowTile != d.N) return HIGGS_ERR_INVALID_ARG;
+            prm.packed = prm.seg_packed[0];
+            prm.scales = prm.seg_scales[0];
+            prm.y = prm.seg_y[0];
+        }
+    }
     const Format fmt = format_of(d.p, d.n);
     const bool six = fmt == Format::kSixBit, nib = fmt == Format::kNibble, b8 = fmt == Format::kByte8;
     prm.parts = pl.parts;

@@ -660,3 +660,50 @@ def test_k_sharded_layer_sums_to_the_unsharded_output(p, n, N, K, B, world, dtyp
         assert U.linear_error(got, y_ref) <= tol
     for y in ys[1:]:
         assert torch.equal(y, ys[0])
+
+
+@pytest.mark.parametrize("p,n,Ns,K,B,dtype", [
+    (2, 256, (256, 64, 64), 4096, 1, torch.float32),        # q|k|v: one launch that also rotates
+    (2, 256, (1024, 1024), 8192, 2, torch.float32),         # gate|up over cluster pairs
+    (2, 64, (272, 48, 16, 528), 2048, 1, torch.bfloat16),   # four matrices, ragged sizes, six-bit planes
+    (2, 256, (512, 128, 128), 4096, 5, torch.float32),      # rotation kernel + one product launch
+    (1, 16, (320, 320), 4096, 16, torch.float32),           # two token blocks per MMA step
+    (2, 16, (256, 256), 2048, 40, torch.float32),           # more than 16 tokens: the tensor-core path per matrix
+    (2, 256, (32, 32), 14336, 3, torch.float32),            # few rows, long K: the K ranges meet in atomics, per matrix
+])
+def test_linear_multi_equals_the_separate_products(p, n, Ns, K, B, dtype):
+    """Matrices that read the same activations as one product over their concatenated rows (rows are independent):
+    every output equals what higgs_linear gives for that matrix alone - bit for bit where no atomics are involved - and
+    the oracle's."""
+    xi = 31337
+    g64, gt = U.grid32(p, n)
+    x = inputs.make_activations(B, K, seed=800 + B)
+    xt = U.bf16_tensor(x)
+    descs, packed, scales, refs, oracles = [], [], [], [], []
+    for i, N in enumerate(Ns):
+        W = inputs.make_weights(N, K, seed=810 + 7 * i + N, bf16=True)
+        q, sc16 = U.oracle_encode(W, 1024, g64, xi)
+        d = hb.make_desc(p, n, N, K, xi)
+        pk = hb.higgs_pack_codes(d, torch.from_numpy(q.codes.astype(np.uint8)).to(U.dev()))
+        sc = hb.scales_to_tile_major(torch.from_numpy(sc16).to(U.dev()))
+        descs.append(d); packed.append(pk); scales.append(sc)
+        refs.append(hb.higgs_linear(d, xt, pk, sc, gt, out_dtype=dtype))
+        oracles.append(oracle.linear_dense(x.astype(np.float64), q.codes, sc16.astype(np.float64), 1024, g64, xi))
+    ys = [torch.full((B, N), float("nan"), dtype=dtype, device=U.dev()) for N in Ns]
+    m = hb.MultiLinear(descs, packed, scales, gt, ys, B)
+    hb.higgs_linear_multi(m, xt)
+    hb.higgs_linear_multi(m, xt)                  # a second call into the same buffers
+    torch.cuda.synchronize()
+    assert hb.higgs_device_status() == hb.HIGGS_OK
+    total = hb.make_desc(p, n, sum(Ns), K, xi)
+    one_product = B <= 16 and hb.higgs_rotated_layout(total, B) == 0 and not hb.higgs_linear_uses_atomics(total, B)
+    assert m.launches == ((1 if B <= 2 else 1 + (B + 15) // 16) if one_product else sum(hb.higgs_linear_launch_count(d, B) for d in descs))
+    tol = Y_TOL + (2.0 ** -8 if dtype == torch.bfloat16 else 0.0)
+    for d, y, ref, y_or in zip(descs, ys, refs, oracles):
+        got = y.float().cpu().numpy()
+        assert np.isfinite(got).all()
+        assert U.linear_error(got, y_or) <= tol
+        if not hb.higgs_linear_uses_atomics(d, B) and one_product and B > 2:
+            assert torch.equal(y, ref)            # same rotation kernel, same fixed-order sums
+        else:
+            assert U.linear_error(got, ref.float().cpu().numpy().astype(np.float64)) <= 2e-3
