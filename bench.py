@@ -532,12 +532,11 @@ def run_ours(args):
             xs32.append(inputs.make_activations(B, K, inputs.activation_seed(cfg, B) + names.index(xi_of)))
             xs_host.append(torch.from_numpy(xs32[-1]).to(torch.bfloat16).pin_memory())
         xs.append(xs_host[-1].to(dev))
-        ws.append(torch.empty(hb.higgs_linear_host_workspace_bytes(q.desc, B), dtype=torch.uint8, device=dev))
+        ws.append(torch.empty(hb.higgs_workspace_bytes(q.desc, hb.HIGGS_OP_LINEAR, B), dtype=torch.uint8, device=dev))
         ys.append(torch.empty((B, N), dtype=torch.float32, device=dev))
     descs = [q.desc for q in qs]
     enc_ms = sum(q.enc_ms for q in qs)
     enc_weights = sum(N * K for _, N, K in layers)
-    ys_host = [torch.empty((B, N), dtype=torch.float32).pin_memory() for _, N, _ in layers]
 
     # layers that read the same block input share one rotation (the transform is isolated from the product, Sec. 4.3);
     # a layer whose K is split across thread blocks goes through higgs_linear, whose rotation kernel also clears y
@@ -586,12 +585,15 @@ def run_ours(args):
                 li = lis[0]
                 hb.higgs_linear(descs[li], xs[li], qs[li].packed[c], qs[li].scales[c], qs[li].grid, workspace=ws[li], y=ys[li])
 
-    # end to end: host activations in, host outputs out, one library call per step (higgs_linear_host_batch)
-    host_batches = [hb.HostBatch(descs, xs_host, [q.packed[c] for q in qs], [q.scales[c] for q in qs], [q.grid for q in qs],
-                                 ys_host, ws) for c in range(copies)]
+    # end to end: one pinned host block of activations in, one pinned host block of outputs out, one library call per
+    # step (higgs_linear_host_block: one copy each way, the block's products, layers with a common input and grid merged)
+    x_keys = [str(id(t)) for t in xs_host]
+    distinct = list({k: t for k, t in zip(x_keys, xs_host)}.items())
+    host_blocks = [hb.HostBlock(descs, x_keys, distinct, [q.packed[c] for q in qs], [q.scales[c] for q in qs],
+                                [q.grid for q in qs], B) for c in range(copies)]
 
     def step_host(i):
-        hb.higgs_linear_host_batch(host_batches[i % copies])
+        hb.higgs_linear_host_block(host_blocks[i % copies])
         torch.cuda.current_stream().synchronize()   # the step's results are read on the host
 
     # ---- graphs of spg consecutive steps (over rotating weight copies); spg divides --steps, so exactly --steps steps
@@ -673,8 +675,8 @@ def run_ours(args):
     ms_per_step = ms / args.steps
     value = aggregate_value(set_bytes, args.steps, ms, world)
     e2e_value = aggregate_value(set_bytes, args.steps, ms_e2e, world)
-    h2d = sum(t.numel() * 2 for t in {id(t): t for t in xs_host}.values())       # layers that share their input copy it once
-    d2h = sum(B * N * 4 for _, N, _ in layers)
+    h2d = host_blocks[0].x_block.numel()       # the copied blocks (inputs shared by layers are there once; 256-byte padding included)
+    d2h = host_blocks[0].y_block.numel()
 
     # ---- dominant kernel: the product kernel on the largest layer (most code bytes), timed alone with CUDA events
     import oracle
@@ -833,7 +835,7 @@ def run_ours(args):
         # free the headline workload's copies before the other configurations are encoded
         for q in qs:
             del q.packed[1:], q.scales[1:]
-        host_batches = None
+        host_blocks = None
         multis = None
         graphs = None
         torch.cuda.empty_cache()

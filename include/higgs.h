@@ -350,6 +350,24 @@ int higgs_linear_host_batch(int32_t count, const higgs_desc* const* descs, const
                             const size_t* workspace_bytes, void* stream);
 
 /*
+ * The same with ONE host block in and ONE host block out, so that a step costs two copies whatever the number of
+ * layers: x_host_block (ideally pinned) holds every distinct input of the step, layer i reads [B][K_i] bf16 at byte
+ * offset x_offsets[i] (layers with a common input name the same offset); y_host_block receives layer i's [B][N_i]
+ * output of y_dtype at byte offset y_offsets[i] (offsets multiples of 16, ranges inside the blocks, else
+ * HIGGS_ERR_INVALID_ARG).  Enqueued on `stream`: one host-to-device copy of the input block, the products of Appendix F
+ * in order - consecutive layers that name the same input offset, grid table, (p, n), K and seed run as one product
+ * (higgs_linear_multi) - and one device-to-host copy of the output block.  workspace: ONE device buffer of
+ * higgs_linear_host_block_workspace_bytes() bytes (inner scratch shared by the products, which run one after the
+ * other, plus the two staged blocks).  The caller synchronises before reading y_host_block.  Arrays are HOST arrays.
+ */
+int higgs_linear_host_block(int32_t count, const higgs_desc* const* descs, const void* x_host_block, size_t x_block_bytes,
+                            const size_t* x_offsets, int64_t B, const void* const* packed, const void* const* scales,
+                            const float* const* grids, void* y_host_block, size_t y_block_bytes, const size_t* y_offsets,
+                            int y_dtype, void* workspace, size_t workspace_bytes, void* stream);
+size_t higgs_linear_host_block_workspace_bytes(int32_t count, const higgs_desc* const* descs, int64_t B,
+                                               size_t x_block_bytes, size_t y_block_bytes);
+
+/*
  * higgs_linear without a workspace argument, for callers that cannot allocate
  * device memory (code running where cudaMalloc is off limits, plugins that are
  * only handed their input and output buffers, processes whose memory pool

@@ -30,7 +30,7 @@ EXPORTS = [
     "higgs_allocate_bits", "higgs_general_tuples", "higgs_quantize_general", "higgs_linear_host_batch",
     "higgs_linear_gather", "higgs_linear_share", "higgs_make_grid_seeded", "higgs_gaussian_samples", "higgs_shard_rows",
     "higgs_launch_floor", "higgs_selftest_wait", "higgs_linear_uses_atomics", "higgs_shard_seed", "higgs_linear_kshard", "higgs_reduce_slots", "higgs_linear_multi", "higgs_linear_multi_workspace_bytes",
-    "higgs_linear_multi_launch_count",
+    "higgs_linear_multi_launch_count", "higgs_linear_host_block", "higgs_linear_host_block_workspace_bytes",
 ]
 
 
@@ -130,6 +130,10 @@ def _load() -> ctypes.CDLL:
     lib.higgs_linear_multi_workspace_bytes.argtypes = [i32, vp, i64]
     lib.higgs_linear_multi_launch_count.restype = i32
     lib.higgs_linear_multi_launch_count.argtypes = [i32, vp, i64, i32]
+    lib.higgs_linear_host_block.restype = i32
+    lib.higgs_linear_host_block.argtypes = [i32, vp, vp, sz, vp, i64, vp, vp, vp, vp, sz, vp, i32, vp, sz, vp]
+    lib.higgs_linear_host_block_workspace_bytes.restype = sz
+    lib.higgs_linear_host_block_workspace_bytes.argtypes = [i32, vp, i64, sz, sz]
     lib.higgs_shard_seed.restype = u64
     lib.higgs_shard_seed.argtypes = [u64, i64]
     lib.higgs_linear_kshard.restype = i32
@@ -370,6 +374,63 @@ def higgs_linear_gather(desc: higgs_desc, x: torch.Tensor, packed: torch.Tensor,
     _check(lib.higgs_linear_gather(ctypes.byref(desc), _ptr(x), B, _ptr(packed), _ptr(scales), _ptr(grid), ptrs, len(y_dsts),
                                    ld, int(row_offset), _dtype_code(y_dsts[0]), _ptr(workspace), workspace.numel(), _stream()),
            "higgs_linear_gather")
+
+
+class HostBlock:
+    """Argument arrays of higgs_linear_host_block, marshalled once: the layers of one step with ONE pinned input block and
+    ONE pinned output block.  inputs: list of (key, x) with x a [B][K] bf16 host tensor per distinct input; layer i reads
+    the input named x_keys[i].  After the call and a stream synchronisation, self.y[i] is layer i's [B][N_i] output (a view
+    of the output block)."""
+
+    def __init__(self, descs, x_keys, inputs, packed, scales, grids, B, y_dtype=torch.float32, device=None):
+        n = len(descs)
+        assert n == len(x_keys) == len(packed) == len(scales) == len(grids)
+        device = device or packed[0].device
+        self.count, self.B = n, int(B)
+        off, pos = {}, 0
+        for key, x in inputs:
+            assert (not x.is_cuda) and x.dtype == torch.bfloat16 and x.is_contiguous() and x.shape[0] == B
+            off[key] = pos
+            pos += (x.numel() * 2 + 255) // 256 * 256
+        self.x_block = torch.empty(max(pos, 256), dtype=torch.uint8).pin_memory()
+        self.x_views = {}
+        for key, x in inputs:
+            v = self.x_block[off[key]: off[key] + x.numel() * 2].view(torch.bfloat16).view(x.shape)
+            v.copy_(x)
+            self.x_views[key] = v
+        esz = 4 if y_dtype == torch.float32 else 2
+        y_off, pos = [], 0
+        for d in descs:
+            y_off.append(pos)
+            pos += (B * d.N * esz + 255) // 256 * 256
+        self.y_block = torch.empty(max(pos, 256), dtype=torch.uint8).pin_memory()
+        self.y = [self.y_block[o: o + B * d.N * esz].view(y_dtype).view(B, d.N) for o, d in zip(y_off, descs)]
+        self.keep = (list(descs), list(packed), list(scales), list(grids))
+        arr = ctypes.c_void_p * n
+        szs = ctypes.c_size_t * n
+        self.descs = arr(*[ctypes.addressof(d) for d in descs])
+        self.x_offsets = szs(*[off[k] for k in x_keys])
+        self.y_offsets = szs(*y_off)
+        self.packed = arr(*[t.data_ptr() for t in packed])
+        self.scales = arr(*[t.data_ptr() for t in scales])
+        self.grids = arr(*[t.data_ptr() for t in grids])
+        self.y_dtype = HIGGS_F32 if y_dtype == torch.float32 else HIGGS_BF16
+        need = int(lib.higgs_linear_host_block_workspace_bytes(n, self.descs, self.B, self.x_block.numel(), self.y_block.numel()))
+        self.workspace = _workspace(need, device)
+
+    def set_weights(self, packed, scales):
+        self.keep = (self.keep[0], list(packed), list(scales), self.keep[3])
+        for i, (p, s) in enumerate(zip(packed, scales)):
+            self.packed[i] = p.data_ptr()
+            self.scales[i] = s.data_ptr()
+
+
+def higgs_linear_host_block(hbk: HostBlock) -> None:
+    """One host-to-device copy, the step's products, one device-to-host copy, enqueued with one library call."""
+    _check(lib.higgs_linear_host_block(hbk.count, hbk.descs, hbk.x_block.data_ptr(), hbk.x_block.numel(), hbk.x_offsets, hbk.B,
+                                       hbk.packed, hbk.scales, hbk.grids, hbk.y_block.data_ptr(), hbk.y_block.numel(),
+                                       hbk.y_offsets, hbk.y_dtype, _ptr(hbk.workspace), hbk.workspace.numel(), _stream()),
+           "higgs_linear_host_block")
 
 
 class MultiLinear:

@@ -563,6 +563,80 @@ int higgs_linear_host_batch(int32_t count, const higgs_desc* const* descs, const
     return HIGGS_OK;
 }
 
+// ---- one host block in, one host block out ---------------------------------------------------------------------
+static size_t host_block_inner(int32_t count, const higgs_desc* const* descs, int64_t B) {
+    // the products run one after the other on the stream and share one inner workspace: the largest any of them -
+    // or any run of up to four layers taken together by higgs_linear_multi - needs
+    size_t inner = 0;
+    for (int i = 0; i < count; ++i) {
+        for (int n = 1; n <= kMaxMulti && i + n <= count; ++n) {
+            const size_t w = n == 1 ? higgs_workspace_bytes(descs[i], HIGGS_OP_LINEAR, B)
+                                    : higgs_linear_multi_workspace_bytes(n, descs + i, B);
+            inner = w > inner ? w : inner;
+        }
+    }
+    return align_up(inner, 256);
+}
+
+size_t higgs_linear_host_block_workspace_bytes(int32_t count, const higgs_desc* const* descs, int64_t B, size_t x_block_bytes,
+                                               size_t y_block_bytes) {
+    if (count < 1 || !descs || B < 1) return 0;
+    for (int i = 0; i < count; ++i)
+        if (check_desc(descs[i]) != HIGGS_OK) return 0;
+    return host_block_inner(count, descs, B) + align_up(x_block_bytes, 256) + align_up(y_block_bytes, 256);
+}
+
+int higgs_linear_host_block(int32_t count, const higgs_desc* const* descs, const void* x_host_block, size_t x_block_bytes,
+                            const size_t* x_offsets, int64_t B, const void* const* packed, const void* const* scales,
+                            const float* const* grids, void* y_host_block, size_t y_block_bytes, const size_t* y_offsets,
+                            int y_dtype, void* workspace, size_t workspace_bytes, void* stream) {
+    if (count < 0) return HIGGS_ERR_INVALID_ARG;
+    if (count == 0) return HIGGS_OK;
+    if (!descs || !x_offsets || !y_offsets || !packed || !scales || !grids) return HIGGS_ERR_INVALID_ARG;
+    if (y_dtype != HIGGS_F32 && y_dtype != HIGGS_BF16) return HIGGS_ERR_UNSUPPORTED;
+    if (B < 0) return HIGGS_ERR_INVALID_ARG;
+    const size_t esz = y_dtype == HIGGS_F32 ? 4 : 2;
+    for (int i = 0; i < count; ++i) {
+        const int rc = check_desc(descs[i]);
+        if (rc != HIGGS_OK) return rc;
+        if (x_offsets[i] % 16 || y_offsets[i] % 16) return HIGGS_ERR_INVALID_ARG;
+        if (x_offsets[i] + (size_t)B * descs[i]->K * 2 > x_block_bytes) return HIGGS_ERR_INVALID_ARG;
+        if (y_offsets[i] + (size_t)B * descs[i]->N * esz > y_block_bytes) return HIGGS_ERR_INVALID_ARG;
+    }
+    if (B == 0) return HIGGS_OK;
+    if (!x_host_block || !y_host_block || !workspace || !aligned(workspace, 256)) return HIGGS_ERR_INVALID_ARG;
+    if (workspace_bytes < higgs_linear_host_block_workspace_bytes(count, descs, B, x_block_bytes, y_block_bytes)) return HIGGS_ERR_WORKSPACE;
+    const size_t inner = host_block_inner(count, descs, B);
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    uint8_t* x_dev = ws + inner;
+    uint8_t* y_dev = x_dev + align_up(x_block_bytes, 256);
+    cudaStream_t st = as_stream(stream);
+    if (cudaMemcpyAsync(x_dev, x_host_block, x_block_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return HIGGS_ERR_CUDA;
+    for (int i = 0; i < count;) {
+        // consecutive layers with the same input, grid table, grid, group size, K and seed run as one product
+        int n = 1;
+        while (i + n < count && n < kMaxMulti && x_offsets[i + n] == x_offsets[i] && grids[i + n] == grids[i] &&
+               descs[i + n]->p == descs[i]->p && descs[i + n]->n == descs[i]->n && descs[i + n]->K == descs[i]->K &&
+               descs[i + n]->rht_seed == descs[i]->rht_seed)
+            ++n;
+        int rc;
+        if (n == 1) {
+            rc = descs[i]->N == 0 ? HIGGS_OK
+                                  : higgs_linear(descs[i], x_dev + x_offsets[i], B, packed[i], scales[i], grids[i], y_dev + y_offsets[i],
+                                                 y_dtype, ws, inner, stream);
+        } else {
+            void* ys[kMaxMulti];
+            for (int j = 0; j < n; ++j) ys[j] = y_dev + y_offsets[i + j];
+            rc = higgs_linear_multi(n, descs + i, x_dev + x_offsets[i], B, packed + i, scales + i, grids[i], ys, y_dtype, ws, inner,
+                                    stream);
+        }
+        if (rc != HIGGS_OK) return rc;
+        i += n;
+    }
+    if (cudaMemcpyAsync(y_host_block, y_dev, y_block_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return HIGGS_ERR_CUDA;
+    return HIGGS_OK;
+}
+
 size_t higgs_linear_host_workspace_bytes(const higgs_desc* d, int64_t B, int y_dtype) {
     const size_t inner = higgs_workspace_bytes(d, HIGGS_OP_LINEAR, B);
     if (inner == 0) return 0;

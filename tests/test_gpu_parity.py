@@ -410,6 +410,20 @@ def test_linear_host_and_host_batch_match_device_path(B):
     assert hb.higgs_device_status() == hb.HIGGS_OK
     for li in range(len(descs)):
         assert torch.equal(ys_host[li], ys_dev[li])
+    # one pinned block in, one pinned block out (two copies per step); the first two layers share input and grid and run
+    # as one product over their concatenated rows
+    blk = hb.HostBlock(descs, ["a", "a", "b"], [("a", x_shared), ("b", x_other)], packed, scales, grids, B)
+    for _ in range(2):
+        for y in blk.y:
+            y.fill_(float("nan"))
+        hb.higgs_linear_host_block(blk)
+        torch.cuda.synchronize()
+        assert hb.higgs_device_status() == hb.HIGGS_OK
+        for li in range(len(descs)):
+            if B <= 2:      # one or two tokens: the merged product rotates in its own kernel; equal to fp16 rounding of x+
+                assert U.linear_error(blk.y[li].numpy(), ys_dev[li].numpy().astype(np.float64)) <= 2e-3
+            else:
+                assert torch.equal(blk.y[li], ys_dev[li])
 
 
 # ----------------------------------------------------------------------------- general grids (evaluation encoder)
