@@ -710,7 +710,7 @@ def run_ours(args):
                     "peak_source": f"of {peak_src}", "algorithmic_bytes": alg, "frac_of_8TBps": achieved / 8000.0, **common}
 
     detail = None
-    if not args.no_detail and rank == 0:
+    if not args.no_detail and rank == 0 and world == 1:      # (detail times more launches with collectives-free code paths: single-GPU runs only)
         detail = {"layers": []}
         # one row per distinct (shape, grid) of the headline workload at its batch - and at the configuration's other
         # batch (32 for the 70B shapes, 16 otherwise) - each with the parity of the timed output on sampled rows

@@ -721,12 +721,13 @@ int tc_batch_tile(int64_t B) {
 }
 
 // The tensor-core path takes layers whose row count is a multiple of 128: every batch above 16, and batches
-// 9..16 of large layers (there the small-batch kernel is limited by the legacy mma.sync rate, two per lookup group;
-// measured cross-over near 32 M weights).
+// 9..16 of layers with at least 4096 rows and 16 M weights (there the small-batch kernel is limited by the legacy
+// mma.sync rate, two per lookup group; measured at 16 tokens: 4096 x 4096 8.7 us here against 11.6 us there, 8192 x 2048
+// 7.9 against 7.6, while 2048 x 8192 - few row tiles, K split over a cluster - takes 12.9 us here against 9.3 us there).
 bool tc_eligible(const higgs_desc& d, int64_t B) {
     const Format f = format_of(d.p, d.n);
     if (!(d.N % 128 == 0 && d.N > 0 && f != Format::kNone)) return false;
-    return B > 16 || (B > 8 && d.N * d.K >= ((int64_t)1 << 25));
+    return B > 16 || (B > 8 && d.N >= 4096 && d.N * d.K >= ((int64_t)1 << 24));
 }
 
 size_t tc_workspace_bytes(const higgs_desc& d, int64_t B) {
