@@ -203,7 +203,7 @@ int higgs_quantize(const higgs_desc* desc, const void* W, int w_dtype, const flo
  * Kernels behind the call: for one or two tokens (K up to 8192) a single kernel
  * that rotates the activations in its prologue; up to 16 tokens a rotation
  * kernel and the small-batch product kernel; above that (and from 9 tokens
- * for layers with at least 4096 rows and 16 M weights) a rotation kernel and the tcgen05 kernel.
+ * for layers with at least 4096 rows, 4096 inputs and 16 M weights) a rotation kernel and the tcgen05 kernel.
  * When the small-batch kernel splits K over more than two thread blocks the
  * partial sums meet in fp32 atomics, so the last bits of y may differ from run
  * to run (higgs_linear_uses_atomics); every other path is bit-reproducible.  The one-call form and the two-call

@@ -421,7 +421,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) linear_tc_kernel(const TcParams
                 const __half2 s2 = __half2half2(sc);
                 sc2 = *reinterpret_cast<const uint32_t*>(&s2);
             }
-            uint4 c4[4];                           // c4[t] = the four index words (steps m = 0..3) of lane (g, t)
+            uint4 c4[4] = {};                      // c4[t] = the four index words (steps m = 0..3) of lane (g, t)
             uint32_t a[32];
             auto unrotate = [&]() {                // chunk t was loaded by instruction (t - rot) & 3
                 if (rot & 1) { const uint4 t0 = c4[0]; c4[0] = c4[3]; c4[3] = c4[2]; c4[2] = c4[1]; c4[1] = t0; }
@@ -721,13 +721,13 @@ int tc_batch_tile(int64_t B) {
 }
 
 // The tensor-core path takes layers whose row count is a multiple of 128: every batch above 16, and batches
-// 9..16 of layers with at least 4096 rows and 16 M weights (there the small-batch kernel is limited by the legacy
+// 9..16 of layers with at least 4096 rows, 4096 inputs and 16 M weights (there the small-batch kernel is limited by the legacy
 // mma.sync rate, two per lookup group; measured at 16 tokens: 4096 x 4096 8.7 us here against 11.6 us there, 8192 x 2048
-// 7.9 against 7.6, while 2048 x 8192 - few row tiles, K split over a cluster - takes 12.9 us here against 9.3 us there).
+// 8.1 against 7.6 (stays there), and 2048 x 8192 - few row tiles, K split over a cluster - takes 12.9 us here against 9.3 us there.
 bool tc_eligible(const higgs_desc& d, int64_t B) {
     const Format f = format_of(d.p, d.n);
     if (!(d.N % 128 == 0 && d.N > 0 && f != Format::kNone)) return false;
-    return B > 16 || (B > 8 && d.N >= 4096 && d.N * d.K >= ((int64_t)1 << 24));
+    return B > 16 || (B > 8 && d.N >= 4096 && d.K >= 4096 && d.N * d.K >= ((int64_t)1 << 24));
 }
 
 size_t tc_workspace_bytes(const higgs_desc& d, int64_t B) {
