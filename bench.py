@@ -56,6 +56,11 @@ def parse_args():
     ap.add_argument("--steps-per-graph", type=int, default=8,
                     help="at most this many consecutive steps (over rotating weight copies) per CUDA graph; the largest divisor "
                          "of --steps not above it is used, so that exactly --steps steps run from equal graphs")
+    ap.add_argument("--shard", choices=["none", "rows", "k"], default="none",
+                    help="none: every rank runs an independent replica (the default); rows / k: ONE layer set sharded over the "
+                         "ranks by rows (outputs written into every rank's buffer from the kernels' epilogues) or along K on "
+                         "group boundaries (partial outputs into every rank's slot buffer, then a slot-ordered sum), through "
+                         "peer-mapped symmetric memory")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-detail", action="store_true", help="skip the per-layer rows and the rows of the other configurations")
     args = ap.parse_args()
@@ -877,10 +882,168 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# --------------------------------------------------------------------------------------------- sharded layer set
+def split_units(total_units: int, world: int, rank: int):
+    """[begin, end) of `total_units` units for `rank`: contiguous, the remainder to the first ranks."""
+    base, extra = divmod(total_units, world)
+    begin = rank * base + min(rank, extra)
+    return begin, begin + base + (1 if rank < extra else 0)
+
+
+def run_sharded(args):
+    """ONE layer set sharded over the ranks (strong scaling): every rank encodes and multiplies its shard of every matrix
+    and the kernels' epilogues write into peer-mapped buffers of all ranks (plain stores over NVLink, no multicast, no
+    library kernel on peer memory).  rows: higgs_linear_gather, every rank ends a step holding the full outputs.  k:
+    higgs_linear_kshard into slot buffers, a barrier, higgs_reduce_slots.  Between a step's writes and its readers
+    stands the symmetric-memory barrier of the process group, enqueued on the timed stream."""
+    import torch
+    import torch.distributed as dist
+    import torch.distributed._symmetric_memory as symm_mem
+
+    import paper_2411_17525_b200 as hb
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the HIGGS kernels have no CPU fallback")
+    if world > 8:
+        raise SystemExit("a sharded layer writes into at most 8 devices' buffers")
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29517")
+    os.environ.setdefault("RANK", "0")
+    os.environ.setdefault("WORLD_SIZE", "1")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist.init_process_group("nccl", device_id=dev)
+
+    layers = inputs.LAYER_SETS[args.workload]
+    cfg = inputs.CONFIG_OF_SET[args.workload]
+    pn, grid_text = layer_grids(args, layers, cfg)
+    xi = inputs.rht_seed(cfg)
+    B = args.batch
+    peak, peak_tf, peak_src = measured_peaks()
+    grids = {}
+    for key in sorted(set(pn)):
+        p, n = key
+        samples = torch.from_numpy(inputs.gaussian_samples(p, inputs.grid_sample_seed(p, n)).astype(np.float32)).to(dev)
+        grids[key], _, _ = hb.higgs_make_grid(p, n, samples, max_iters=3000)
+    set_bytes = sum(layer_bytes(N, K, *pn[li]) for li, (_, N, K) in enumerate(layers))
+
+    shards = []      # per layer: (desc, packed, scales, x, workspace, symmetric buffer, peer tensors, extra)
+    for li, (name, N, K) in enumerate(layers):
+        grid = grids[pn[li]]
+        if args.shard == "rows":
+            mult = 128 if N % (128 * world) == 0 else 16
+            r0, r1 = hb.shard_rows(N, world, rank, mult)
+            Ns, Ks, seed, x_cols = r1 - r0, K, xi, (0, K)
+        else:
+            g0, g1 = split_units(K // G, world, rank)
+            Ns, Ks, seed, x_cols = N, (g1 - g0) * G, hb.higgs_shard_seed(xi, g0 * G), (g0 * G, g1 * G)
+            r0 = 0
+        d = hb.make_desc(pn[li][0], pn[li][1], Ns, Ks, seed)
+        if Ns == 0 or Ks == 0:
+            shards.append(None)
+            continue
+        # the shard's weights: the recipe's distribution, drawn per (layer, rank) - the sharded run is a throughput
+        # measurement, parity of sharded layers is covered by the tests
+        W = torch.from_numpy(inputs.make_weights(Ns, Ks, inputs.weight_seed(cfg, li) + 100 * (rank + 1), bf16=True)).to(dev).to(torch.bfloat16)
+        pk, sc, _ = hb.higgs_quantize(d, W, grid)
+        del W
+        x_full = inputs.make_activations(B, K, inputs.activation_seed(cfg, B) + li)
+        x = torch.from_numpy(np.ascontiguousarray(x_full[:, x_cols[0]:x_cols[1]])).to(dev).to(torch.bfloat16)
+        ws = torch.empty(hb.higgs_workspace_bytes(d, hb.HIGGS_OP_LINEAR, B), dtype=torch.uint8, device=dev)
+        shape = (B, N) if args.shard == "rows" else (world, B, N)
+        buf = symm_mem.empty(shape, dtype=torch.float32, device=dev)
+        hdl = symm_mem.rendezvous(buf, group=dist.group.WORLD)
+        peers = [buf if r == rank else hdl.get_buffer(r, shape, torch.float32) for r in range(world)]
+        shards.append((d, pk, sc, grid, x, ws, buf, hdl, peers, r0))
+    live = [s for s in shards if s is not None]
+    if not live:
+        raise SystemExit("this rank holds no shard")
+    barrier_hdl = live[0][7]
+
+    def step(_i):
+        for d, pk, sc, grid, x, ws, buf, hdl, peers, r0 in live:
+            if args.shard == "rows":
+                ordered = [peers[rank]] + [peers[r] for r in range(world) if r != rank]
+                hb.higgs_linear_gather(d, x, pk, sc, grid, ordered, r0, workspace=ws)
+            else:
+                hb.higgs_linear_kshard(d, x, pk, sc, grid, peers, rank, workspace=ws)
+        barrier_hdl.barrier()                      # all shards / partials of the step written, on every rank
+        if args.shard == "k":
+            for d, pk, sc, grid, x, ws, buf, hdl, peers, r0 in live:
+                hb.higgs_reduce_slots(buf)
+            barrier_hdl.barrier()                  # nobody overwrites a slot that is still being summed
+
+    stream = torch.cuda.Stream()
+    warm = max(args.warmup, 3)
+    spg = divisor_at_most(args.steps, max(1, args.steps_per_graph))
+    graph = None
+    with torch.cuda.stream(stream):
+        for i in range(warm):
+            step(i)
+        stream.synchronize()
+        if not args.no_graph:        # spg steps per replay: the host's launch cost leaves the timed region
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                for k in range(spg):
+                    step(k)
+            graph.replay()
+        stream.synchronize()
+        dist.barrier()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        if graph is not None:
+            for _ in range(args.steps // spg):
+                graph.replay()
+        else:
+            for i in range(args.steps):
+                step(i)
+        b.record(stream)
+        torch.cuda.synchronize()
+        dist.barrier()
+        ms = max_over_ranks(a.elapsed_time(b), dev, world)
+    # after the last step every rank holds every rank's contribution: this rank's own part must equal the plain product
+    # of its shard, and nothing may be left unwritten (the buffers were never cleared, so a NaN-filled start shows holes)
+    check = 0.0
+    for d, pk, sc, grid, x, ws, buf, hdl, peers, r0 in live[:2]:
+        y_own = hb.higgs_linear(d, x, pk, sc, grid)
+        if args.shard == "rows":
+            check = max(check, float((buf[:, r0:r0 + d.N] - y_own).abs().max() / y_own.abs().max()))
+        elif world == 1:
+            check = max(check, float((buf[0] - y_own).abs().max() / y_own.abs().max()))
+        if not bool(torch.isfinite(buf).all()):
+            check = float("inf")
+    check = max_over_ranks(check, dev, world)
+    status = hb.higgs_device_status()
+    if rank == 0:
+        value = set_bytes / (ms / args.steps * 1e-3) / 1e9          # the WHOLE layer set's weights per step: strong scaling
+        line = {
+            "metric": "higgs_linear_effective_weight_bandwidth", "value": value, "unit": "GB/s", "n_gpus": world,
+            "steps": args.steps, "warmup": warm, "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "f16xf16->f32", "data": "synthetic",
+            "config": {"workload": f"{args.workload} layer set ({len(layers)} matrices), grid {grid_text}, g=1024, batch {B}",
+                       "global_batch": B, "parallelism": f"{args.shard}-sharded x{world}",
+                       "l2": "one weight copy per rank (the sharded mode measures the exchange, not the L2-cold stream)",
+                       "launch": "direct" if graph is None else f"CUDA graphs of {spg} steps",
+                       "step": "every matrix of the block as a sharded layer: shard product with the exchange fused into the "
+                               "epilogues (peer stores), symmetric-memory barrier" + (", slot-ordered sum, barrier" if args.shard == "k" else "")},
+            "weight_bytes_per_step": set_bytes, "device_status": status, "own_shard_max_rel_dev": check,
+            "e2e": None, "gpu_launches": None, "clocks": None, "roofline": None, "cpu_baseline": None,
+            "frac_of_measured_hbm_per_gpu": value / world / peak,
+        }
+        print(json.dumps(line))
+    dist.destroy_process_group()
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.shard != "none":
+        run_sharded(args)
     else:
         run_ours(args)
 

@@ -94,3 +94,28 @@ def test_quantize_then_linear_back_to_back_on_one_stream():
         torch.cuda.synchronize()
         assert torch.equal(packed, packed0)
         assert torch.equal(y, y0)
+
+
+@pytest.mark.parametrize("mode", ["rows", "k"])
+def test_sharded_benchmark_mode_on_one_rank(mode):
+    """bench.py --shard runs the sharded-layer entry points on peer-mapped symmetric memory; with one rank the peer list
+    is this device alone, which still takes the whole path: symmetric allocation, rendezvous, the epilogue's stores into
+    the mapped buffer, the barrier, (k) the slot sum, all inside CUDA graphs.  Its own-shard check must agree with the
+    plain product."""
+    import json
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1", MASTER_PORT="29541", NCCL_NVLS_ENABLE="0")
+    for k in ("RANK", "WORLD_SIZE", "LOCAL_RANK"):
+        env.pop(k, None)
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--shard", mode, "--workload", "llama-3.2-1b",
+                          "--grid", "2,256", "--steps", "8", "--warmup", "3"], cwd=root, env=env, capture_output=True,
+                         text=True, timeout=600)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads([l for l in out.stdout.splitlines() if l.startswith("{")][-1])
+    assert line["scaling"] == "strong" and line["n_gpus"] == 1 and line["device_status"] == 0
+    assert line["config"]["parallelism"] == f"{mode}-sharded x1"
+    assert line["own_shard_max_rel_dev"] <= 1e-5
+    assert line["value"] > 0
