@@ -183,7 +183,7 @@ int higgs_gaussian_samples(int p, uint64_t sample_seed, int64_t num_samples, flo
  *   packed_out     device, higgs_packed_bytes() bytes, 16-byte aligned
  *   scales_out     device, higgs_scales_bytes() bytes, 16-byte aligned: fp16 scales stored
  *                  tile-major, element (r, i) at index ((r / 16) * (K/g) + i) * 16 + r % 16
- *   canonical_out  device, optional, [N][K/p] one byte per code (for checking)
+ *   canonical_out  device, optional, [N][K/p] one byte per code (for checking), 16-byte aligned
  */
 int higgs_quantize(const higgs_desc* desc, const void* W, int w_dtype, const float* grid,
                    void* packed_out, void* scales_out, uint8_t* canonical_out,
@@ -491,7 +491,7 @@ int higgs_allocate_bits(int32_t num_layers, int32_t num_options, const double* a
 int higgs_rht(const higgs_desc* desc, const void* x, int x_dtype, int64_t rows,
               float* out, int normalised, void* stream);
 
-/* Canonical codes ([N][K/p] bytes, device) -> packed stream, and back.  They
+/* Canonical codes ([N][K/p] bytes, device, 16-byte aligned) -> packed stream, and back.  They
  * let codes produced elsewhere (e.g. by a reference encoder) be fed to
  * higgs_linear, and the packed output of higgs_quantize be inspected.       */
 int higgs_pack_codes(const higgs_desc* desc, const uint8_t* canonical, void* packed_out, void* stream);

@@ -203,7 +203,7 @@ int higgs_quantize(const higgs_desc* d, const void* W, int w_dtype, const float*
         if (!workspace || !aligned(workspace, 256)) return HIGGS_ERR_INVALID_ARG;
         if (workspace_bytes < higgs_workspace_bytes(d, HIGGS_OP_QUANTIZE, 0)) return HIGGS_ERR_WORKSPACE;
         canonical = static_cast<uint8_t*>(workspace);
-    } else if (!aligned(canonical, 8)) {
+    } else if (!aligned(canonical, 16)) {
         return HIGGS_ERR_INVALID_ARG;
     }
     cudaStream_t st = as_stream(stream);
@@ -688,7 +688,7 @@ int higgs_pack_codes(const higgs_desc* d, const uint8_t* canonical, void* packed
     int rc = check_desc(d);
     if (rc != HIGGS_OK) return rc;
     if (d->N == 0 || d->K == 0) return HIGGS_OK;
-    if (!canonical || !packed_out || !aligned(packed_out, 16)) return HIGGS_ERR_INVALID_ARG;
+    if (!canonical || !packed_out || !aligned(packed_out, 16) || !aligned(canonical, 16)) return HIGGS_ERR_INVALID_ARG;
     rc = launch_pack(*d, canonical, packed_out, as_stream(stream));
     return rc != HIGGS_OK ? rc : launch_stream_fence(as_stream(stream));
 }

@@ -144,11 +144,13 @@ __device__ __forceinline__ void fwht1024_warp(float (&v)[32], int lane) {
     }
 #pragma unroll
     for (int m = 1; m < 32; m <<= 1) {
-        const bool upper = (lane & m) != 0;
+        // upper lane of a pair: other - own, lower lane: own + other - one fused multiply-add with +-1 (exact product,
+        // one rounding: the same value as the subtraction / addition)
+        const float sgn = (lane & m) != 0 ? -1.0f : 1.0f;
 #pragma unroll
         for (int r = 0; r < 32; ++r) {
             float o = __shfl_xor_sync(0xffffffffu, v[r], m);
-            v[r] = upper ? (o - v[r]) : (v[r] + o);
+            v[r] = fmaf(v[r], sgn, o);
         }
     }
 }
@@ -157,12 +159,17 @@ __device__ __forceinline__ void fwht1024_warp(float (&v)[32], int lane) {
 // of 1024): chunk c covers inputs k0 + c*256 + lane*8 .. +7, eight consecutive bits of one 64-bit sign word.
 __device__ __forceinline__ void apply_signs1024(float (&v)[32], uint64_t xi, int64_t k0, int lane) {
 #pragma unroll
+    // the group's 16 sign words: lane l computes word l & 15, chunk c of a lane needs word 4c + lane/8
+    const uint64_t word = sign_word(xi, ((uint64_t)k0 >> 6) + (uint64_t)(lane & 15));
+    const uint32_t lo = (uint32_t)word, hi = (uint32_t)(word >> 32);
+#pragma unroll
     for (int c = 0; c < 4; ++c) {
-        const uint64_t j0 = (uint64_t)k0 + (uint64_t)(c * 256 + lane * 8);
-        const uint32_t bits = (uint32_t)(sign_word(xi, j0 >> 6) >> (j0 & 63ull)) & 0xffu;
+        const int src = 4 * c + (lane >> 3);
+        const uint32_t from_lo = __shfl_sync(0xffffffffu, lo, src), from_hi = __shfl_sync(0xffffffffu, hi, src);
+        const uint32_t bits = ((lane & 4) ? from_hi : from_lo) >> ((lane & 3) * 8);
 #pragma unroll
         for (int e = 0; e < 8; ++e)
-            v[c * 8 + e] = __uint_as_float(__float_as_uint(v[c * 8 + e]) ^ (((bits >> e) & 1u) << 31));
+            v[c * 8 + e] = __uint_as_float(__float_as_uint(v[c * 8 + e]) ^ ((bits << (31 - e)) & 0x80000000u));
     }
 }
 

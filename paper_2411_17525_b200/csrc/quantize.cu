@@ -123,45 +123,55 @@ __global__ void __launch_bounds__(128) encode_kernel(const T* __restrict__ W, co
 
 // ---- exact pruned search ---------------------------------------------------------------------------------------
 // The same nearest-point rule as above, evaluated only on the grid points that can win.  The plane (the line for
-// p = 1) is cut into square cells over [-R, R)^p; for a cell, U = min over grid points of the distance to the cell's
-// farthest corner bounds the distance of the winner from any point of the cell, so only points whose distance to the
-// cell is at most U (+ a slack far above fp32 rounding) can be nearest.  Their indices are listed in ascending order,
-// so the strict '<' of the scan keeps the lowest index on ties exactly like the exhaustive scan.  Cells with more
-// than kMaxCand candidates, and inputs outside [-R, R)^p, fall back to the exhaustive scan (done by the whole warp for
-// one such point at a time: same distances, lowest index on ties).  The table is built once
-// by a small kernel (into scratch memory the caller lends: the packed-code output buffer, which is written only after
-// the encoder has finished) and copied into shared memory by every persistent encoder block.
-constexpr int kCells2 = 64;            // p = 2: 64 x 64 cells of width 1/8 (n = 256: 3 candidates on average, 5 for the
-                                       // slowest of a warp's 32 lanes; 32 x 32 cells had 8 and 13)
-constexpr int kCells1 = 1024;          // p = 1
-constexpr int kMaxCand = 8;            // a cell's list is one 8-byte word
+// p = 1) is cut into square cells; cell i of an axis covers the values whose scaled coordinate x * cells / 2R + cells / 2
+// rounds to i (found with one fused multiply-add onto 2^23: the integer is then the low bits of the float).  A cell's
+// candidate list is built in two steps.  (1) U = min over grid points of the distance to the cell's farthest corner
+// bounds the winner's distance from any point of the cell, so only points whose distance to the cell is at most U (+ a
+// slack far above fp32 rounding) can be nearest.  (2) Of those, c is dropped if another candidate c' is nearer at all
+// corners of the cell by a margin: |z - c|^2 - |z - c'|^2 is affine in z, so its minimum over the cell is at a corner,
+// and c wins nowhere in the cell.  The surviving indices (at most four, else the cell is marked) are stored in
+// ascending order, the last one repeated up to four: the encoder evaluates all four without a branch, and its strict
+// '<' keeps the lowest index on ties exactly like the exhaustive scan (a repeated candidate never replaces itself).
+// Marked cells and inputs outside the table take the exhaustive scan, done by the whole warp for one such point at a
+// time, after the warp's other points: same distances, lowest index on ties.  The table is built once per call by a
+// small kernel (into scratch memory the caller lends: the packed-code output buffer, which is written only after the
+// encoder has finished) and copied into shared memory by every persistent encoder block.
+constexpr int kCells2 = 128;           // p = 2: 128 x 128 cells of width 1/16 (n = 256: 1.6 candidates on average, at most 4)
+constexpr int kCells1 = 1024;          // p = 1: width 1/128, at most 2 candidates
+constexpr int kMaxCand = 4;            // a cell's list is one 32-bit word
+constexpr int kPrefilter = 32;         // candidates that step (1) may leave for step (2)
+constexpr uint32_t kCellScan = 1u;     // bytes (1, 0, 0, 0) are not an ascending list: the cell needs the exhaustive scan
 constexpr float kCellR = 4.0f;
 constexpr float kCandSlack = 1e-3f;
+constexpr float kDominance = 1e-3f;    // margin of step (2) on squared distances (fp32 rounding there is below 1e-5)
+constexpr size_t kCellTableBytes = (size_t)(kCells2 * kCells2 > kCells1 ? kCells2 * kCells2 : kCells1) * 4;
 
 template <int P>
-__global__ void __launch_bounds__(256) build_cells_kernel(const float* __restrict__ grid, int n, uint8_t* __restrict__ table) {
+__global__ void __launch_bounds__(256) build_cells_kernel(const float* __restrict__ grid, int n, uint32_t* __restrict__ table) {
     constexpr int NC = P == 2 ? kCells2 * kCells2 : kCells1;
+    constexpr int CELLS = P == 2 ? kCells2 : kCells1;
     __shared__ float sgrid[256 * 2];
+    __shared__ int slist[8][kPrefilter];
     for (int i = threadIdx.x; i < n * P; i += blockDim.x) sgrid[i] = grid[i];
     __syncthreads();
-    uint8_t* cand = table;                       // [NC][kMaxCand]
-    uint8_t* cnt = table + NC * kMaxCand;        // [NC]
-    const float w = 2.0f * kCellR / (P == 2 ? kCells2 : kCells1);
-    const int lane = threadIdx.x & 31;
+    const float w = 2.0f * kCellR / CELLS;
+    const int lane = threadIdx.x & 31, wi = threadIdx.x >> 5;
     const int warps = (gridDim.x * blockDim.x) >> 5;
     // one warp per cell; lane l looks at grid points l, l + 32, ... (rounds keep the candidate list in index order)
     for (int cell = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; cell < NC; cell += warps) {
-        const float x0 = -kCellR + w * (P == 2 ? (cell % kCells2) : cell), x1 = x0 + w;
-        const float y0 = P == 2 ? -kCellR + w * (cell / kCells2) : 0.f, y1 = y0 + w;
-        float U = INFINITY;
+        const int cx = P == 2 ? cell % kCells2 : cell, cy = P == 2 ? cell / kCells2 : 0;
+        const float x0 = w * ((float)cx - 0.5f - 0.5f * CELLS), x1 = x0 + w;
+        const float y0 = P == 2 ? w * ((float)cy - 0.5f - 0.5f * CELLS) : 0.f, y1 = y0 + w;
+        float U2 = INFINITY;
         for (int c = lane; c < n; c += 32) {
             const float gx = sgrid[P * c], gy = P == 2 ? sgrid[2 * c + 1] : 0.f;
             const float fx = fmaxf(fabsf(gx - x0), fabsf(gx - x1));
             const float fy = P == 2 ? fmaxf(fabsf(gy - y0), fabsf(gy - y1)) : 0.f;
-            U = fminf(U, sqrtf(fx * fx + fy * fy));
+            U2 = fminf(U2, fx * fx + fy * fy);
         }
 #pragma unroll
-        for (int m = 16; m >= 1; m >>= 1) U = fminf(U, __shfl_xor_sync(0xffffffffu, U, m));
+        for (int m = 16; m >= 1; m >>= 1) U2 = fminf(U2, __shfl_xor_sync(0xffffffffu, U2, m));
+        const float reach = sqrtf(U2) + kCandSlack, reach2 = reach * reach;
         int k = 0;
         for (int c0 = 0; c0 < n; c0 += 32) {
             const int c = c0 + lane;
@@ -170,36 +180,102 @@ __global__ void __launch_bounds__(256) build_cells_kernel(const float* __restric
                 const float gx = sgrid[P * c], gy = P == 2 ? sgrid[2 * c + 1] : 0.f;
                 const float nx = fmaxf(fmaxf(x0 - gx, gx - x1), 0.f);
                 const float ny = P == 2 ? fmaxf(fmaxf(y0 - gy, gy - y1), 0.f) : 0.f;
-                in = sqrtf(nx * nx + ny * ny) <= U + kCandSlack;
+                in = nx * nx + ny * ny <= reach2;
             }
             const unsigned m = __ballot_sync(0xffffffffu, in);
             const int pos = k + __popc(m & ((1u << lane) - 1u));
-            if (in && pos < kMaxCand) cand[cell * kMaxCand + pos] = (uint8_t)c;
+            if (in && pos < kPrefilter) slist[wi][pos] = c;
             k += __popc(m);
         }
-        if (lane == 0) cnt[cell] = k <= kMaxCand ? (uint8_t)k : (uint8_t)255;
+        __syncwarp();
+        uint32_t word = kCellScan;
+        if (k <= kPrefilter) {
+            // step (2): lane i judges candidate i against every candidate j
+            const bool have = lane < k;
+            const int mine = have ? slist[wi][lane] : 0;
+            const float mx = sgrid[P * mine], my = P == 2 ? sgrid[2 * mine + 1] : 0.f;
+            const float qx[2] = {x0, x1}, qy[2] = {y0, y1};
+            float dm[4];
+#pragma unroll
+            for (int q = 0; q < (P == 2 ? 4 : 2); ++q) {
+                const float dx = qx[q & 1] - mx, dy = P == 2 ? qy[q >> 1] - my : 0.f;
+                dm[q] = dx * dx + dy * dy;
+            }
+            bool dominated = false;
+            for (int j = 0; j < k; ++j) {
+                const int cj = slist[wi][j];
+                const float gx = sgrid[P * cj], gy = P == 2 ? sgrid[2 * cj + 1] : 0.f;
+                bool all = true;
+#pragma unroll
+                for (int q = 0; q < (P == 2 ? 4 : 2); ++q) {
+                    const float dx = qx[q & 1] - gx, dy = P == 2 ? qy[q >> 1] - gy : 0.f;
+                    all = all && (dx * dx + dy * dy + kDominance < dm[q]);
+                }
+                dominated = dominated || all;
+            }
+            const unsigned kept = __ballot_sync(0xffffffffu, have && !dominated);
+            const int cnt = __popc(kept);
+            if (cnt >= 1 && cnt <= kMaxCand) {
+                word = 0u;
+#pragma unroll
+                for (int r = 0; r < kMaxCand; ++r) {
+                    const int src = __fns(kept, 0, (r < cnt ? r : cnt - 1) + 1);
+                    word |= (uint32_t)__shfl_sync(0xffffffffu, mine, src) << (8 * r);
+                }
+            }
+        }
+        if (lane == 0) table[cell] = word;
+        __syncwarp();
     }
 }
 
+// the exhaustive scan of one point by the whole warp (lowest index among equal distances)
+template <int P>
+__device__ __noinline__ int warp_scan(const float* sgrid, int n, float px, float py, int lane) {
+    float bd = INFINITY;
+    int bc = 0x7fffffff;
+    for (int c = lane; c < n; c += 32) {           // ascending within the lane: '<' keeps its lowest index
+        const float dx = px - sgrid[P * c], dy = P == 2 ? py - sgrid[2 * c + 1] : 0.f;
+        const float d = P == 2 ? fmaf(dy, dy, dx * dx) : dx * dx;
+        if (d < bd) { bd = d; bc = c; }
+    }
+#pragma unroll
+    for (int m = 16; m >= 1; m >>= 1) {             // across lanes: smaller distance, then lower index
+        const float od = __shfl_xor_sync(0xffffffffu, bd, m);
+        const int oc = __shfl_xor_sync(0xffffffffu, bc, m);
+        if (od < bd || (od == bd && oc < bc)) { bd = od; bc = oc; }
+    }
+    return bc == 0x7fffffff ? 0 : bc;               // no distance compared below infinity (a NaN input): index 0, as the scan
+}
+
+// Persistent blocks of 16 warps, one (row, group) per warp and turn.  Shared memory: the cell table and the grid with
+// every point repeated across a 128-byte row (16 copies of an 8-byte point for p = 2, 32 copies of a float for p = 1), so
+// that a lane reads "its" copy and the 32 lookups of a warp never meet in a bank.
 template <typename T, int P>
-__global__ void __launch_bounds__(256) encode_pruned_kernel(const T* __restrict__ W, const float* __restrict__ grid, int n,
-                                                            const uint8_t* __restrict__ table,
-                                                            uint8_t* __restrict__ canonical, __half* __restrict__ scales,
-                                                            int64_t N, int64_t K, uint64_t xi) {
+__global__ void __launch_bounds__(512, 2) encode_pruned_kernel(const T* __restrict__ W, const float* __restrict__ grid, int n,
+                                                               const uint32_t* __restrict__ table,
+                                                               uint8_t* __restrict__ canonical, __half* __restrict__ scales,
+                                                               int64_t N, int64_t K, uint64_t xi) {
     constexpr int NC = P == 2 ? kCells2 * kCells2 : kCells1;
+    constexpr int CELLS = P == 2 ? kCells2 : kCells1;
+    extern __shared__ __align__(128) uint8_t enc_smem[];
     __shared__ float sgrid[256 * 2];
-    __shared__ __align__(16) uint8_t cand[NC * kMaxCand + NC];
-    const uint8_t* cnt = cand + NC * kMaxCand;
+    uint32_t* cells = reinterpret_cast<uint32_t*>(enc_smem);
+    uint8_t* rep = enc_smem + (size_t)NC * 4;
     for (int i = threadIdx.x; i < n * P; i += blockDim.x) sgrid[i] = grid[i];
-    for (int i = threadIdx.x; i < (NC * kMaxCand + NC) / 16; i += blockDim.x)
-        reinterpret_cast<uint4*>(cand)[i] = reinterpret_cast<const uint4*>(table)[i];
+    for (int i = threadIdx.x; i < NC / 4; i += blockDim.x)
+        reinterpret_cast<uint4*>(cells)[i] = reinterpret_cast<const uint4*>(table)[i];
+    for (int i = threadIdx.x; i < n * 32; i += blockDim.x)
+        reinterpret_cast<float*>(rep)[i] = grid[P == 2 ? 2 * (i >> 5) + (i & 1) : (i >> 5)];
     __syncthreads();
 
     const int lane = threadIdx.x & 31;
+    const uint8_t* rep_lane = rep + (P == 2 ? (lane & 15) * 8 : lane * 4);
     const int64_t groups = K / kGroup;
     const int64_t tasks = N * groups;
     const int64_t warps_total = (int64_t)gridDim.x * (blockDim.x >> 5);
-    const float inv_w = (P == 2 ? kCells2 : kCells1) / (2.0f * kCellR);
+    const float inv_w = CELLS / (2.0f * kCellR);
+    const float magic = 8388608.0f + 0.5f * CELLS;
     for (int64_t task = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); task < tasks; task += warps_total) {
         const int64_t row = task / groups, gi = task % groups;
         float v[32];
@@ -217,70 +293,59 @@ __global__ void __launch_bounds__(256) encode_pruned_kernel(const T* __restrict_
         fwht1024_warp(v, lane);
         if (lane == 0) scales[((row >> 4) * groups + gi) * 16 + (row & 15)] = __float2half_rn(s * 0.03125f);
 
-        int bi[32 / P];
+        uint32_t out[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};      // the lane's codes, one byte each, in storage order
+        uint32_t slow = 0u;                                       // bit t: tuple t needs the exhaustive scan
 #pragma unroll
         for (int t = 0; t < 32 / P; ++t) {
             const float x = v[P * t], y = P == 2 ? v[2 * t + 1] : 0.f;
-            // cell coordinates by rounding down; negative, huge or NaN inputs fail the unsigned comparison
-            const int ix = __float2int_rd((x + kCellR) * inv_w), iy = P == 2 ? __float2int_rd((y + kCellR) * inv_w) : 0;
-            const bool inside = (unsigned)ix < (unsigned)(P == 2 ? kCells2 : kCells1) && (P == 1 || (unsigned)iy < (unsigned)kCells2);
-            const int cell = inside ? (P == 2 ? iy * kCells2 + ix : ix) : 0;
-            const int k = inside ? cnt[cell] : 255;
-            float best = INFINITY;
-            int b = 0;
-            // lanes whose point has no candidate list (a crowded outer cell, or outside the table): the warp scans the
-            // whole grid for them together, one such lane at a time - left to the lane itself the scan would hold up
-            // the other 31 for n iterations whenever any lane needs it
-            unsigned full_scan = __ballot_sync(0xffffffffu, k == 255);
-            if (k != 255) {
-                const uint2 l2 = *reinterpret_cast<const uint2*>(&cand[cell * kMaxCand]);     // the whole list
-                for (int i = 0; i < k; ++i) {
-                    const int c = (int)(__byte_perm(l2.x, l2.y, (uint32_t)i) & 0xffu);   // byte i of the list
-                    const float dx = x - sgrid[P * c], dy = P == 2 ? y - sgrid[2 * c + 1] : 0.f;
-                    const float d = P == 2 ? fmaf(dy, dy, dx * dx) : dx * dx;
-                    if (d < best) { best = d; b = c; }
-                }
-            }
-            __syncwarp();
-            while (full_scan) {
-                const int src = __ffs(full_scan) - 1;
-                full_scan &= full_scan - 1;
-                const float px = __shfl_sync(0xffffffffu, x, src), py = __shfl_sync(0xffffffffu, y, src);
-                float bd = INFINITY;
-                int bc = 0x7fffffff;
-                for (int c = lane; c < n; c += 32) {           // ascending within the lane: '<' keeps its lowest index
-                    const float dx = px - sgrid[P * c], dy = P == 2 ? py - sgrid[2 * c + 1] : 0.f;
-                    const float d = P == 2 ? fmaf(dy, dy, dx * dx) : dx * dx;
-                    if (d < bd) { bd = d; bc = c; }
-                }
+            // the float 2^23 + i carries i in its low bits; anything else (outside the table, NaN) leaves other bits set
+            const uint32_t ix = __float_as_uint(fmaf(x, inv_w, magic)) ^ 0x4B000000u;
+            const uint32_t iy = P == 2 ? __float_as_uint(fmaf(y, inv_w, magic)) ^ 0x4B000000u : 0u;
+            const bool inside = (ix | iy) < (uint32_t)CELLS;
+            uint32_t list = kCellScan;
+            if (inside) list = cells[P == 2 ? iy * kCells2 + ix : ix];
+            if (list == kCellScan) { slow |= 1u << t; list = 0u; }
+            float best;
+            uint32_t b;
 #pragma unroll
-                for (int m = 16; m >= 1; m >>= 1) {             // across lanes: smaller distance, then lower index
-                    const float od = __shfl_xor_sync(0xffffffffu, bd, m);
-                    const int oc = __shfl_xor_sync(0xffffffffu, bc, m);
-                    if (od < bd || (od == bd && oc < bc)) { bd = od; bc = oc; }
+            for (int i = 0; i < (P == 2 ? kMaxCand : 2); ++i) {
+                const uint32_t c = __byte_perm(list, 0u, 0x4440u + i);
+                float d;
+                if (P == 2) {
+                    const float2 g = *reinterpret_cast<const float2*>(rep_lane + c * 128u);
+                    const float dx = x - g.x, dy = y - g.y;
+                    d = fmaf(dy, dy, dx * dx);
+                } else {
+                    const float dx = x - *reinterpret_cast<const float*>(rep_lane + c * 128u);
+                    d = dx * dx;
                 }
-                if (lane == src) b = bc;
+                if (i == 0 || d < best) { best = d; b = c; }
             }
-            bi[t] = b;
+            out[t >> 2] |= b << (8 * (t & 3));
+        }
+        if (__any_sync(0xffffffffu, slow != 0u)) {
+#pragma unroll
+            for (int t = 0; t < 32 / P; ++t) {
+                unsigned m = __ballot_sync(0xffffffffu, (slow >> t) & 1u);
+                while (m) {
+                    const int src = __ffs(m) - 1;
+                    m &= m - 1;
+                    const float px = __shfl_sync(0xffffffffu, v[P * t], src);
+                    const float py = P == 2 ? __shfl_sync(0xffffffffu, v[2 * t + 1], src) : 0.f;
+                    const int bc = warp_scan<P>(sgrid, n, px, py, lane);
+                    if (lane == src) out[t >> 2] = (out[t >> 2] & ~(0xffu << (8 * (t & 3)))) | ((uint32_t)bc << (8 * (t & 3)));
+                }
+            }
         }
         if (P == 2) {
+            // tuple t of chunk c sits at tuple index c*128 + lane*4 + (t&3): 4 consecutive bytes per chunk
             uint8_t* dst = canonical + row * (K / 2) + gi * (kGroup / 2);
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t w = (uint32_t)bi[c * 4] | ((uint32_t)bi[c * 4 + 1] << 8) | ((uint32_t)bi[c * 4 + 2] << 16) |
-                             ((uint32_t)bi[c * 4 + 3] << 24);
-                *reinterpret_cast<uint32_t*>(dst + c * 128 + lane * 4) = w;
-            }
+            for (int c = 0; c < 4; ++c) *reinterpret_cast<uint32_t*>(dst + c * 128 + lane * 4) = out[c];
         } else {
             uint8_t* dst = canonical + row * K + gi * kGroup;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t w0 = (uint32_t)bi[c * 8] | ((uint32_t)bi[c * 8 + 1] << 8) | ((uint32_t)bi[c * 8 + 2] << 16) |
-                              ((uint32_t)bi[c * 8 + 3] << 24);
-                uint32_t w1 = (uint32_t)bi[c * 8 + 4] | ((uint32_t)bi[c * 8 + 5] << 8) | ((uint32_t)bi[c * 8 + 6] << 16) |
-                              ((uint32_t)bi[c * 8 + 7] << 24);
-                *reinterpret_cast<uint2*>(dst + c * 256 + lane * 8) = make_uint2(w0, w1);
-            }
+            for (int c = 0; c < 4; ++c) *reinterpret_cast<uint2*>(dst + c * 256 + lane * 8) = make_uint2(out[2 * c], out[2 * c + 1]);
         }
     }
 }
@@ -318,16 +383,6 @@ __device__ __forceinline__ void slot_coords(int64_t rt, int64_t kb, int L, int s
     pair = kb * 32 + m * 8 + (L & 3) + 4 * (a >> 1);   // index of the 2-input pair along K
 }
 
-// table index of a pair of inputs (2 consecutive k) from the canonical codes
-template <int P>
-__device__ __forceinline__ uint32_t pair_index(const uint8_t* __restrict__ canonical, int64_t K, int64_t row,
-                                               int64_t pair, int bits) {
-    if (P == 2) return canonical[row * (K / 2) + pair];
-    const uint8_t* q = canonical + row * K + 2 * pair;       // two scalar codes of `bits` bits each
-    const uint32_t mask = (1u << bits) - 1u;
-    return (uint32_t)(q[0] & mask) | ((uint32_t)(q[1] & mask) << bits);
-}
-
 __device__ __forceinline__ void six_bit_store(uint32_t (&w)[3], int s, uint32_t code) {
     const int m = s >> 2, a = s & 3;
     w[m >> 1] |= (code & 15u) << (8 * a + 4 * (m & 1));
@@ -344,52 +399,64 @@ __device__ __forceinline__ int64_t six_bit_word(int64_t rt, int64_t kb, int64_t 
     return ((rt * (kblocks >> 1) + (kb >> 1)) * 3 + w) * 64 + 2 * L + (kb & 1);
 }
 
+// One block packs 16 rows x 1024 inputs: the canonical codes of the tile are staged in shared memory with coalesced
+// 16-byte loads (rows 16 bytes apart in bank position, so the byte gathers below meet no bank conflicts), then every
+// thread assembles the words of two (64-input block, lane) positions and stores them coalesced.
 template <int P, int FMT>
 __global__ void __launch_bounds__(256) pack_kernel(const uint8_t* __restrict__ canonical, uint32_t* __restrict__ packed,
                                                    int64_t N, int64_t K, int bits) {
-    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int64_t kblocks = K / kBlockK;
-    const int64_t total = (N / 16) * kblocks * 32;
-    if (t >= total) return;
-    const int L = (int)(t & 31);
-    const int64_t blk = t >> 5, rt = blk / kblocks, kb = blk % kblocks;
+    constexpr int RB = P == 2 ? 512 : 1024;          // canonical bytes of one row and 1024 inputs
+    constexpr int RS = RB + 16;
+    __shared__ __align__(16) uint8_t tile[16 * RS];
+    const int64_t kblocks = K / kBlockK, ktiles = K / kGroup;
+    const int64_t rt = blockIdx.x / ktiles, kt = blockIdx.x % ktiles;
+    for (int i = threadIdx.x; i < 16 * (RB / 16); i += 256) {
+        const int r = i / (RB / 16), c = i % (RB / 16);
+        *reinterpret_cast<uint4*>(tile + r * RS + c * 16) =
+            *reinterpret_cast<const uint4*>(canonical + ((rt * 16 + r) * ktiles + kt) * RB + c * 16);
+    }
+    __syncthreads();
     constexpr bool SIX = FMT == 1, NIB = FMT == 2, B8 = FMT == 3;
-    if (B8) {
-        uint32_t w[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
-        for (int s = 0; s < 16; ++s) {
-            int64_t row, pair;
-            slot_coords(rt, kb, L, s, row, pair);
-            const uint8_t* q = canonical + row * K + 2 * pair;
-            w[2 * (s >> 2) + ((s & 3) >> 1)] |= ((uint32_t)q[0] | ((uint32_t)q[1] << 8)) << (16 * (s & 1));
+    const uint32_t mask = (1u << bits) - 1u;
+    for (int item = threadIdx.x; item < 512; item += 256) {
+        const int L = item & 31, kbl = item >> 5;
+        const int64_t kb = kt * 16 + kbl, blk = rt * kblocks + kb, t = blk * 32 + L;
+        // table index of slot s = 4m + a of this lane (two consecutive inputs): row (L>>2) + 8(a&1) of the tile,
+        // pair kbl*32 + m*8 + (L&3) + 4(a>>1)
+        auto index_of = [&](int s) -> uint32_t {
+            const int m = s >> 2, a = s & 3;
+            const int row = (L >> 2) + 8 * (a & 1), pair = kbl * 32 + m * 8 + (L & 3) + 4 * (a >> 1);
+            if (P == 2) return tile[row * RS + pair];
+            const uint8_t* q = tile + row * RS + 2 * pair;       // two scalar codes of `bits` bits each
+            return B8 ? ((uint32_t)q[0] | ((uint32_t)q[1] << 8)) : ((uint32_t)(q[0] & mask) | ((uint32_t)(q[1] & mask) << bits));
+        };
+        if (B8) {
+            uint32_t w[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+#pragma unroll
+            for (int s = 0; s < 16; ++s) w[2 * (s >> 2) + ((s & 3) >> 1)] |= index_of(s) << (16 * (s & 1));
+            uint4* out = reinterpret_cast<uint4*>(packed) + blk * 64;      // 1024-byte block = 64 uint4
+            out[L] = make_uint4(w[0], w[1], w[2], w[3]);
+            out[32 + L] = make_uint4(w[4], w[5], w[6], w[7]);
+        } else if (SIX) {
+            uint32_t w[3] = {0u, 0u, 0u};
+#pragma unroll
+            for (int s = 0; s < 16; ++s) six_bit_store(w, s, index_of(s) & 63u);
+#pragma unroll
+            for (int i = 0; i < 3; ++i) packed[six_bit_word(rt, kb, kblocks, L, i)] = w[i];
+        } else if (NIB) {
+            uint32_t w[2] = {0u, 0u};
+#pragma unroll
+            for (int s = 0; s < 16; ++s) {
+                const int m = s >> 2, a = s & 3, byte = 2 * m + (a >> 1);
+                w[byte >> 2] |= (index_of(s) & 15u) << (8 * (byte & 3) + 4 * (a & 1));
+            }
+            reinterpret_cast<uint2*>(packed)[t] = make_uint2(w[0], w[1]);
+        } else {
+            uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+            for (int s = 0; s < 16; ++s) w[s >> 2] |= index_of(s) << (8 * (s & 3));
+            reinterpret_cast<uint4*>(packed)[t] = make_uint4(w[0], w[1], w[2], w[3]);
         }
-        uint4* out = reinterpret_cast<uint4*>(packed) + blk * 64;      // 1024-byte block = 64 uint4
-        out[L] = make_uint4(w[0], w[1], w[2], w[3]);
-        out[32 + L] = make_uint4(w[4], w[5], w[6], w[7]);
-    } else if (SIX) {
-        uint32_t w[3] = {0u, 0u, 0u};
-        for (int s = 0; s < 16; ++s) {
-            int64_t row, pair;
-            slot_coords(rt, kb, L, s, row, pair);
-            six_bit_store(w, s, pair_index<P>(canonical, K, row, pair, bits) & 63u);
-        }
-        for (int i = 0; i < 3; ++i) packed[six_bit_word(rt, kb, kblocks, L, i)] = w[i];
-    } else if (NIB) {
-        uint32_t w[2] = {0u, 0u};
-        for (int s = 0; s < 16; ++s) {
-            int64_t row, pair;
-            slot_coords(rt, kb, L, s, row, pair);
-            const int m = s >> 2, a = s & 3, byte = 2 * m + (a >> 1);
-            w[byte >> 2] |= (pair_index<P>(canonical, K, row, pair, bits) & 15u) << (8 * (byte & 3) + 4 * (a & 1));
-        }
-        reinterpret_cast<uint2*>(packed)[t] = make_uint2(w[0], w[1]);
-    } else {
-        uint32_t w[4] = {0u, 0u, 0u, 0u};
-        for (int s = 0; s < 16; ++s) {
-            int64_t row, pair;
-            slot_coords(rt, kb, L, s, row, pair);
-            w[s >> 2] |= pair_index<P>(canonical, K, row, pair, bits) << (8 * (s & 3));
-        }
-        reinterpret_cast<uint4*>(packed)[t] = make_uint4(w[0], w[1], w[2], w[3]);
     }
 }
 
@@ -443,6 +510,16 @@ __global__ void __launch_bounds__(256) unpack_kernel(const uint32_t* __restrict_
     }
 }
 
+int sm_count() {
+    static int cached[64] = {0};
+    return device_once(cached, [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0)
+            v = 148;
+        return v;
+    });
+}
+
 }  // namespace
 
 int launch_encode(const higgs_desc& d, const void* W, int w_dtype, const float* grid, uint8_t* canonical, void* scales,
@@ -451,19 +528,30 @@ int launch_encode(const higgs_desc& d, const void* W, int w_dtype, const float* 
     if (warps == 0) return HIGGS_OK;
     const unsigned blocks = (unsigned)((warps + 3) / 4);
     __half* sc = static_cast<__half*>(scales);
-    // Large grids on large layers: the exact pruned search (persistent blocks that build their candidate table once);
-    // otherwise the exhaustive scan, whose cost is small there.
-    constexpr size_t kTableBytes = (size_t)(kCells1 > kCells2 * kCells2 ? kCells1 : kCells2 * kCells2) * (kMaxCand + 1);
-    const bool pruned = d.n >= 64 && warps >= 2048 && scratch && scratch_bytes >= kTableBytes &&
+    // Large layers: the exact pruned search (persistent blocks that copy the candidate table once); otherwise the
+    // exhaustive scan, whose cost is small there.
+    const bool pruned = warps >= 2048 && scratch && scratch_bytes >= kCellTableBytes &&
                         (reinterpret_cast<uintptr_t>(scratch) % 16) == 0;
-    const unsigned pblocks = 592;          // 4 blocks of 8 warps per SM on a 148-SM part; any count is correct
-    uint8_t* table = static_cast<uint8_t*>(scratch);
+    uint32_t* table = static_cast<uint32_t*>(scratch);
+    const size_t smem = (size_t)(d.p == 2 ? kCells2 * kCells2 : kCells1) * 4 + (size_t)d.n * 128;
     if (pruned) {
-        if (d.p == 2) build_cells_kernel<2><<<128, 256, 0, st>>>(grid, d.n, table);      // one warp per cell
+        static int configured[64];
+        const int ok = device_once(configured, [] {
+            constexpr int kMax = kCells2 * kCells2 * 4 + 256 * 128;
+            bool good = true;
+            good = good && cudaFuncSetAttribute(encode_pruned_kernel<float, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMax) == cudaSuccess;
+            good = good && cudaFuncSetAttribute(encode_pruned_kernel<float, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMax) == cudaSuccess;
+            good = good && cudaFuncSetAttribute(encode_pruned_kernel<__nv_bfloat16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMax) == cudaSuccess;
+            good = good && cudaFuncSetAttribute(encode_pruned_kernel<__nv_bfloat16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMax) == cudaSuccess;
+            return good ? 1 : -1;
+        });
+        if (ok < 0) return HIGGS_ERR_CUDA;
+        if (d.p == 2) build_cells_kernel<2><<<592, 256, 0, st>>>(grid, d.n, table);      // one warp per cell and turn
         else build_cells_kernel<1><<<128, 256, 0, st>>>(grid, d.n, table);
     }
+    const unsigned pblocks = 2u * (unsigned)sm_count();     // two blocks of 16 warps per SM; any count is correct
 #define HIGGS_ENC(T, P) \
-    if (pruned) encode_pruned_kernel<T, P><<<pblocks, 256, 0, st>>>(static_cast<const T*>(W), grid, d.n, table, canonical, sc, d.N, d.K, d.rht_seed); \
+    if (pruned) encode_pruned_kernel<T, P><<<pblocks, 512, smem, st>>>(static_cast<const T*>(W), grid, d.n, table, canonical, sc, d.N, d.K, d.rht_seed); \
     else encode_kernel<T, P><<<blocks, 128, 0, st>>>(static_cast<const T*>(W), grid, d.n, canonical, sc, d.N, d.K, d.rht_seed)
     if (w_dtype == HIGGS_F32 && d.p == 2) { HIGGS_ENC(float, 2); }
     else if (w_dtype == HIGGS_F32 && d.p == 1) { HIGGS_ENC(float, 1); }
@@ -475,9 +563,11 @@ int launch_encode(const higgs_desc& d, const void* W, int w_dtype, const float* 
 }
 
 int launch_pack(const higgs_desc& d, const uint8_t* canonical, void* packed, cudaStream_t st) {
-    const int64_t total = (d.N / 16) * (d.K / kBlockK) * 32;
-    if (total == 0) return HIGGS_OK;
-    const unsigned blocks = (unsigned)((total + 255) / 256);
+    const int64_t tiles = (d.N / 16) * (d.K / kGroup);
+    if (tiles == 0) return HIGGS_OK;
+    if (tiles > 0x7fffffff) return HIGGS_ERR_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(canonical) % 16) return HIGGS_ERR_INVALID_ARG;
+    const unsigned blocks = (unsigned)tiles;
     uint32_t* out = static_cast<uint32_t*>(packed);
     const Format f = format_of(d.p, d.n);
     const int bits = code_bits(d.n);
