@@ -216,12 +216,11 @@ __global__ void __launch_bounds__(256) build_cells_kernel(const float* __restric
             const unsigned kept = __ballot_sync(0xffffffffu, have && !dominated);
             const int cnt = __popc(kept);
             if (cnt >= 1 && cnt <= kMaxCand) {
-                word = 0u;
-#pragma unroll
-                for (int r = 0; r < kMaxCand; ++r) {
-                    const int src = __fns(kept, 0, (r < cnt ? r : cnt - 1) + 1);
-                    word |= (uint32_t)__shfl_sync(0xffffffffu, mine, src) << (8 * r);
-                }
+                // the kept lane of rank r supplies byte r; the last one also fills the bytes above it
+                const int r = __popc(kept & ((1u << lane) - 1u));
+                const bool is_kept = (kept >> lane) & 1u;
+                const uint32_t part = !is_kept ? 0u : (r == cnt - 1 ? (uint32_t)mine * (0x01010101u << (8 * r)) : (uint32_t)mine << (8 * r));
+                word = __reduce_or_sync(0xffffffffu, part);
             }
         }
         if (lane == 0) table[cell] = word;
@@ -276,8 +275,12 @@ __global__ void __launch_bounds__(512, 2) encode_pruned_kernel(const T* __restri
     const int64_t warps_total = (int64_t)gridDim.x * (blockDim.x >> 5);
     const float inv_w = CELLS / (2.0f * kCellR);
     const float magic = 8388608.0f + 0.5f * CELLS;
-    for (int64_t task = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); task < tasks; task += warps_total) {
-        const int64_t row = task / groups, gi = task % groups;
+    // (row, group) of the warp's task, advanced by the grid's stride without a division per task
+    const int64_t first = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    int64_t row = first / groups, gi = first % groups;
+    const int64_t step_rows = warps_total / groups, step_groups = warps_total % groups;
+    for (int64_t task = first; task < tasks; task += warps_total, row += step_rows, gi += step_groups) {
+        if (gi >= groups) { gi -= groups; ++row; }
         float v[32];
         load32<T>(W + row * K + gi * kGroup, lane, v);
         float ss = 0.0f;
