@@ -189,6 +189,21 @@ int higgs_quantize(const higgs_desc* desc, const void* W, int w_dtype, const flo
                    void* packed_out, void* scales_out, uint8_t* canonical_out,
                    void* workspace, size_t workspace_bytes, void* stream);
 
+/* The search table of the encoder, built once per grid.  Layers of at least 2 M weights are encoded with an exact
+ * pruned nearest-point search (same codes as the exhaustive scan of Algorithm 1's rounding step, bit for bit) over a
+ * table of candidate lists that depends on the grid only; higgs_quantize builds it on every call (in its workspace),
+ * higgs_quantize_prepared takes one built beforehand - worthwhile when many layers share a grid, as the layers of a
+ * model do.  The paper does not describe the search; this is an implementation device with no counterpart there.
+ *   higgs_encoder_table_bytes  size of the table for (p, n); 0 if the pair has no kernel
+ *   higgs_make_encoder_table   grid: device [n][p] fp32; table_out: device, 16-byte aligned; asynchronous on `stream`
+ *   higgs_quantize_prepared    as higgs_quantize; table: device, from higgs_make_encoder_table for the same (p, n) and
+ *                              grid values, or NULL (then identical to higgs_quantize)                              */
+size_t higgs_encoder_table_bytes(int p, int n);
+int higgs_make_encoder_table(int p, int n, const float* grid, void* table_out, void* stream);
+int higgs_quantize_prepared(const higgs_desc* desc, const void* W, int w_dtype, const float* grid, const void* table,
+                            void* packed_out, void* scales_out, uint8_t* canonical_out,
+                            void* workspace, size_t workspace_bytes, void* stream);
+
 /*
  * Appendix F, "Rotating Activations": y = x W^T computed in the rotated space.
  *   x+ = (H / sqrt(g)) diag(sign) x per token and K-group (same xi as the

@@ -23,6 +23,7 @@ HIGGS_LAYOUT_VERSION = 1
 EXPORTS = [
     "higgs_status_string", "higgs_sign", "higgs_packed_bytes", "higgs_scales_bytes", "higgs_canonical_bytes",
     "higgs_workspace_bytes", "higgs_make_grid", "higgs_quantize", "higgs_linear", "higgs_rht",
+    "higgs_encoder_table_bytes", "higgs_make_encoder_table", "higgs_quantize_prepared",
     "higgs_pack_codes", "higgs_unpack_codes", "higgs_rotate_activations", "higgs_linear_prerotated",
     "higgs_linear_host", "higgs_linear_host_workspace_bytes", "higgs_linear_launch_count", "higgs_device_status",
     "higgs_linear_static", "higgs_linear_static_capacity", "higgs_linear_k_splits", "higgs_rotated_bytes",
@@ -68,6 +69,12 @@ def _load() -> ctypes.CDLL:
     lib.higgs_make_grid.argtypes = [i32, i32, vp, i64, i32, vp, vp, vp, vp, sz, vp]
     lib.higgs_quantize.restype = i32
     lib.higgs_quantize.argtypes = [P, vp, i32, vp, vp, vp, vp, vp, sz, vp]
+    lib.higgs_encoder_table_bytes.restype = sz
+    lib.higgs_encoder_table_bytes.argtypes = [i32, i32]
+    lib.higgs_make_encoder_table.restype = i32
+    lib.higgs_make_encoder_table.argtypes = [i32, i32, vp, vp, vp]
+    lib.higgs_quantize_prepared.restype = i32
+    lib.higgs_quantize_prepared.argtypes = [P, vp, i32, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.higgs_linear.restype = i32
     lib.higgs_linear.argtypes = [P, vp, i64, vp, vp, vp, vp, i32, vp, sz, vp]
     lib.higgs_rotate_activations.restype = i32
@@ -246,10 +253,23 @@ def higgs_selftest_wait(which: int, polls: int, device=None) -> torch.Tensor:
     return out
 
 
+def higgs_make_encoder_table(p: int, n: int, grid: torch.Tensor) -> torch.Tensor:
+    """The encoder's search table for a grid (cuda [n][p] fp32), to be passed to higgs_quantize(..., table=...) for
+    every layer that uses this grid."""
+    assert grid.is_cuda and grid.dtype == torch.float32 and grid.is_contiguous() and tuple(grid.shape) == (n, p)
+    size = lib.higgs_encoder_table_bytes(p, n)
+    if size == 0:
+        raise HiggsError(HIGGS_ERR_UNSUPPORTED, "higgs_encoder_table_bytes")
+    table = torch.empty(size, dtype=torch.uint8, device=grid.device)
+    _check(lib.higgs_make_encoder_table(p, n, _ptr(grid), _ptr(table), _stream()), "higgs_make_encoder_table")
+    return table
+
+
 def higgs_quantize(desc: higgs_desc, W: torch.Tensor, grid: torch.Tensor, want_canonical: bool = False,
-                   workspace: Optional[torch.Tensor] = None, out=None):
+                   workspace: Optional[torch.Tensor] = None, out=None, table: Optional[torch.Tensor] = None):
     """W: cuda [N][K] fp32 or bf16; grid: cuda [n][p] fp32.  Returns (packed u8, scales fp16 tile-major [N/16][K/g][16], canonical u8 or None).
-    out = (packed, scales) reuses existing output tensors."""
+    out = (packed, scales) reuses existing output tensors; table = higgs_make_encoder_table(p, n, grid) skips building
+    the search table in this call."""
     assert W.is_cuda and W.is_contiguous() and grid.is_cuda and grid.dtype == torch.float32 and grid.is_contiguous()
     dev = W.device
     if out is not None:
@@ -262,8 +282,17 @@ def higgs_quantize(desc: higgs_desc, W: torch.Tensor, grid: torch.Tensor, want_c
     canonical = torch.empty((desc.N, desc.K // desc.p), dtype=torch.uint8, device=dev) if want_canonical else None
     if workspace is None:
         workspace = _workspace(higgs_workspace_bytes(desc, HIGGS_OP_QUANTIZE), dev)
-    _check(lib.higgs_quantize(ctypes.byref(desc), _ptr(W), _dtype_code(W), _ptr(grid), _ptr(packed), _ptr(scales),
-                              _ptr(canonical), _ptr(workspace), workspace.numel(), _stream()), "higgs_quantize")
+    elif workspace is False:          # lend none (allowed with want_canonical): the library then packs in a second kernel
+        assert want_canonical
+        workspace = torch.empty(0, dtype=torch.uint8, device=dev)
+    if table is not None:
+        assert table.is_cuda and table.dtype == torch.uint8 and table.numel() >= lib.higgs_encoder_table_bytes(desc.p, desc.n)
+        _check(lib.higgs_quantize_prepared(ctypes.byref(desc), _ptr(W), _dtype_code(W), _ptr(grid), _ptr(table), _ptr(packed),
+                                           _ptr(scales), _ptr(canonical), _ptr(workspace), workspace.numel(), _stream()),
+               "higgs_quantize_prepared")
+    else:
+        _check(lib.higgs_quantize(ctypes.byref(desc), _ptr(W), _dtype_code(W), _ptr(grid), _ptr(packed), _ptr(scales),
+                                  _ptr(canonical), _ptr(workspace), workspace.numel(), _stream()), "higgs_quantize")
     return packed, scales, canonical
 
 

@@ -190,28 +190,60 @@ int higgs_make_uniform_grid(int n, float* grid_out, float* step_out, float* mse_
     return rc != HIGGS_OK ? rc : launch_stream_fence(as_stream(stream));
 }
 
-int higgs_quantize(const higgs_desc* d, const void* W, int w_dtype, const float* grid, void* packed_out,
-                   void* scales_out, uint8_t* canonical_out, void* workspace, size_t workspace_bytes, void* stream) {
+size_t higgs_encoder_table_bytes(int p, int n) {
+    return format_of(p, n) == Format::kNone ? 0 : encoder_table_bytes(p);
+}
+
+int higgs_make_encoder_table(int p, int n, const float* grid, void* table_out, void* stream) {
+    if (format_of(p, n) == Format::kNone) return HIGGS_ERR_UNSUPPORTED;
+    if (!grid || !table_out || !aligned(table_out, 16)) return HIGGS_ERR_INVALID_ARG;
+    const int rc = launch_encoder_table(p, n, grid, table_out, as_stream(stream));
+    return rc != HIGGS_OK ? rc : launch_stream_fence(as_stream(stream));
+}
+
+int higgs_quantize_prepared(const higgs_desc* d, const void* W, int w_dtype, const float* grid, const void* table,
+                            void* packed_out, void* scales_out, uint8_t* canonical_out, void* workspace,
+                            size_t workspace_bytes, void* stream) {
     int rc = check_desc(d);
     if (rc != HIGGS_OK) return rc;
     if (w_dtype != HIGGS_F32 && w_dtype != HIGGS_BF16) return HIGGS_ERR_UNSUPPORTED;
     if (d->N == 0 || d->K == 0) return HIGGS_OK;
     if (!W || !grid || !packed_out || !scales_out) return HIGGS_ERR_INVALID_ARG;
-    if (!aligned(W, 16) || !aligned(packed_out, 16) || !aligned(scales_out, 16)) return HIGGS_ERR_INVALID_ARG;
-    uint8_t* canonical = canonical_out;
-    if (!canonical) {
-        if (!workspace || !aligned(workspace, 256)) return HIGGS_ERR_INVALID_ARG;
-        if (workspace_bytes < higgs_workspace_bytes(d, HIGGS_OP_QUANTIZE, 0)) return HIGGS_ERR_WORKSPACE;
-        canonical = static_cast<uint8_t*>(workspace);
-    } else if (!aligned(canonical, 16)) {
+    if (!aligned(W, 16) || !aligned(packed_out, 16) || !aligned(scales_out, 16) || (table && !aligned(table, 16)))
         return HIGGS_ERR_INVALID_ARG;
+    if (canonical_out && !aligned(canonical_out, 16)) return HIGGS_ERR_INVALID_ARG;
+    if (workspace && !aligned(workspace, 256)) return HIGGS_ERR_INVALID_ARG;
+    if (!canonical_out) {
+        if (!workspace) return HIGGS_ERR_INVALID_ARG;
+        if (workspace_bytes < higgs_workspace_bytes(d, HIGGS_OP_QUANTIZE, 0)) return HIGGS_ERR_WORKSPACE;
     }
     cudaStream_t st = as_stream(stream);
-    // (the packed output is written by the pack kernel only: until then it lends the encoder its scratch space)
-    rc = launch_encode(*d, W, w_dtype, grid, canonical, scales_out, packed_out, higgs_packed_bytes(d), st);
+    // The workspace holds the cell table of a large layer (whose search kernel emits the packed stream itself and needs
+    // no canonical copy) or the canonical codes of a small one (exhaustive scan, then the pack kernel) - never both.
+    // Without a workspace (the caller wants the canonical codes and lends none) the table of a large layer is built in
+    // the packed output, which only the pack kernel writes, after the encoder has finished.
+    const bool ws_table = workspace && workspace_bytes >= encoder_table_bytes(d->p);
+    void* build_space = table ? nullptr : (ws_table ? workspace : packed_out);
+    const bool fuse = table || ws_table;
+    uint8_t* canonical = canonical_out ? canonical_out : static_cast<uint8_t*>(workspace);
+    // (a small layer ignores the table arguments; a large one ignores `canonical` when it is the workspace)
+    bool packed_done = false;
+    const int64_t tasks = d->N * (d->K / kGroup);
+    const bool large = tasks >= kPrunedMinTasks;
+    rc = launch_encode(*d, W, w_dtype, grid, table, build_space, large ? canonical_out : canonical,
+                       (large && fuse) ? packed_out : nullptr, scales_out, &packed_done, st);
     if (rc != HIGGS_OK) return rc;
-    rc = launch_pack(*d, canonical, packed_out, st);
-    return rc != HIGGS_OK ? rc : launch_stream_fence(st);
+    if (!packed_done) {
+        rc = launch_pack(*d, large ? canonical_out : canonical, packed_out, st);
+        if (rc != HIGGS_OK) return rc;
+    }
+    return launch_stream_fence(st);
+}
+
+int higgs_quantize(const higgs_desc* d, const void* W, int w_dtype, const float* grid, void* packed_out,
+                   void* scales_out, uint8_t* canonical_out, void* workspace, size_t workspace_bytes, void* stream) {
+    return higgs_quantize_prepared(d, W, w_dtype, grid, nullptr, packed_out, scales_out, canonical_out, workspace,
+                                   workspace_bytes, stream);
 }
 
 int higgs_dequantize(const higgs_desc* d, const void* packed, const void* scales, const float* grid, void* W_out,

@@ -181,8 +181,12 @@ int launch_rht_activations(const higgs_desc& d, const void* x, int64_t B, __half
                            size_t zero_floats, cudaStream_t st);
 int launch_rht_debug(const higgs_desc& d, const void* x, int x_dtype, int64_t rows, float* out, int normalised,
                      cudaStream_t st);
-int launch_encode(const higgs_desc& d, const void* W, int w_dtype, const float* grid, uint8_t* canonical,
-                  void* scales, void* scratch, size_t scratch_bytes, cudaStream_t st);
+// layers of at least this many (row, group) tasks are encoded with the pruned search
+constexpr int64_t kPrunedMinTasks = 2048;
+size_t encoder_table_bytes(int p);
+int launch_encoder_table(int p, int n, const float* grid, void* table, cudaStream_t st);
+int launch_encode(const higgs_desc& d, const void* W, int w_dtype, const float* grid, const void* table, void* build_space,
+                  uint8_t* canonical, void* packed, void* scales, bool* packed_done, cudaStream_t st);
 int launch_pack(const higgs_desc& d, const uint8_t* canonical, void* packed, cudaStream_t st);
 int launch_unpack(const higgs_desc& d, const void* packed, uint8_t* canonical, cudaStream_t st);
 int launch_dequantize(const higgs_desc& d, const uint8_t* canonical, const void* scales, const float* grid, void* W_out,
@@ -235,6 +239,7 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
                      const GatherTargets* more = nullptr);
 int read_tc_status(int clear);
 int read_grid_status(int clear);
+int read_encode_status(int clear);
 int launch_wait_selftest(uint32_t limit, int* result, cudaStream_t st);
 int launch_tc_wait_selftest(uint32_t limit, int* result, cudaStream_t st);
 int launch_stream_fence(cudaStream_t st);

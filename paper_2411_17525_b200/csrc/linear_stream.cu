@@ -1122,7 +1122,8 @@ int read_device_status(cudaStream_t st, int clear) {
     }
     const int tc = read_tc_status(clear);
     const int gf = read_grid_status(clear);
-    return v != 0 ? v : tc != 0 ? tc : gf;
+    const int en = read_encode_status(clear);
+    return v != 0 ? v : tc != 0 ? tc : gf != 0 ? gf : en;
 }
 
 }  // namespace higgs

@@ -35,6 +35,103 @@ __device__ __forceinline__ void load32<float>(const float* __restrict__ src, int
     }
 }
 
+// ---- packed layout -----------------------------------------------------------
+// The packed stream is a sequence of blocks, block (rt, kb) covering rows
+// [16 rt, 16 rt + 16) and inputs [64 kb, 64 kb + 64), stored at block index
+// rt * (K/64) + kb.  Inside a block, lane L of the consuming warp owns a
+// contiguous run of bytes holding exactly the table indices of the A-fragment
+// registers it feeds to four m16n8k16 tensor-core steps: step m (inputs
+// 16m..16m+15 of the block), register a in 0..3 is the fp16 pair
+//   row   = 16 rt + (L>>2) + 8 (a&1)
+//   pairs = inputs 64 kb + 16 m + 2 (L&3) + 8 (a>>1) + {0, 1}.
+// "Slot" s = 4m + a, 16 slots per lane.
+//   byte-LUT format: 16 bytes per lane, byte s = table index of slot s; a block is
+//                    512 contiguous bytes, lane L at byte offset 16 L.
+//   six-bit format : three 32-bit words per lane and block.  Words 0 and 1 hold the
+//                    low nibbles: slot 4m+a sits in word m>>1 at bit 8a + 4(m&1).
+//                    Word 2 holds the high bit-pairs: slot 4m+a at bit 8a + 2m.
+//                    (The consumer rebuilds four byte-aligned indices with one shift
+//                    and one three-input logic operation each, see linear_mma.cu.)
+//   nibble format  : (n = 16) two 32-bit words per lane and block, 256 bytes per block, lane L at
+//                    byte offset 8 L.  Byte 2m + h of the lane holds the slots 4m + 2h (low
+//                    nibble) and 4m + 2h + 1 (high nibble): the two registers of one row pair.
+//   8-bit format   : (p = 1, n = 256) one byte per input: slot 4m + a is the halfword a & 1 of the lane's
+//                    word 2m + (a >> 1) (low byte = first input of the pair); a block is 1024 bytes, two
+//                    512-byte halves holding words 0..3 and 4..7 of every lane (16 bytes per lane each).
+//                    Two neighbouring blocks (2j, 2j+1 along K) form a 768-byte
+//                    super-block of three 256-byte planes; plane w stores word w of
+//                    lane L, block half h at 32-bit index 2L + h, so a warp reads
+//                    each plane with one coalesced 64-bit load per lane.
+__device__ __forceinline__ void slot_coords(int64_t rt, int64_t kb, int L, int s, int64_t& row, int64_t& pair) {
+    const int m = s >> 2, a = s & 3;
+    row = rt * 16 + (L >> 2) + 8 * (a & 1);
+    pair = kb * 32 + m * 8 + (L & 3) + 4 * (a >> 1);   // index of the 2-input pair along K
+}
+
+__device__ __forceinline__ void six_bit_store(uint32_t (&w)[3], int s, uint32_t code) {
+    const int m = s >> 2, a = s & 3;
+    w[m >> 1] |= (code & 15u) << (8 * a + 4 * (m & 1));
+    w[2] |= ((code >> 4) & 3u) << (8 * a + 2 * m);
+}
+__device__ __forceinline__ uint32_t six_bit_load(const uint32_t (&w)[3], int s) {
+    const int m = s >> 2, a = s & 3;
+    const uint32_t lo = (w[m >> 1] >> (8 * a + 4 * (m & 1))) & 15u;
+    const uint32_t hi = (w[2] >> (8 * a + 2 * m)) & 3u;
+    return lo | (hi << 4);
+}
+// 32-bit index of word w of (block kb, lane L) in the six-bit stream
+__device__ __forceinline__ int64_t six_bit_word(int64_t rt, int64_t kb, int64_t kblocks, int L, int w) {
+    return ((rt * (kblocks >> 1) + (kb >> 1)) * 3 + w) * 64 + 2 * L + (kb & 1);
+}
+
+// The packed words of one (64-input block, lane) position, assembled from a tile of canonical codes in shared memory
+// (16 rows of the row tile, RS bytes apart; kbl = the 64-input block inside the tile's 1024 inputs) and stored.
+// fmt: 0 byte, 1 six-bit, 2 nibble, 3 8-bit (uniform over the block).
+template <int P>
+__device__ __forceinline__ void pack_item(const uint8_t* tile, int RS, int fmt, int bits, int kbl, int L, int64_t rt,
+                                          int64_t kb, int64_t kblocks, uint32_t* __restrict__ packed) {
+    const int64_t blk = rt * kblocks + kb, t = blk * 32 + L;
+    const uint32_t mask = (1u << bits) - 1u;
+    // table index of slot s = 4m + a of this lane (two consecutive inputs): row (L>>2) + 8(a&1) of the tile,
+    // pair kbl*32 + m*8 + (L&3) + 4(a>>1)
+    auto index_of = [&](int s) -> uint32_t {
+        const int m = s >> 2, a = s & 3;
+        const int row = (L >> 2) + 8 * (a & 1), pair = kbl * 32 + m * 8 + (L & 3) + 4 * (a >> 1);
+        if (P == 2) return tile[row * RS + pair];
+        const uint8_t* q = tile + row * RS + 2 * pair;       // two scalar codes of `bits` bits each
+        return (uint32_t)(q[0] & mask) | ((uint32_t)(q[1] & mask) << bits);
+    };
+    if (P == 1 && fmt == 3) {
+        uint32_t w[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int s = 0; s < 16; ++s) w[2 * (s >> 2) + ((s & 3) >> 1)] |= index_of(s) << (16 * (s & 1));
+        uint4* out = reinterpret_cast<uint4*>(packed) + blk * 64;      // 1024-byte block = 64 uint4
+        out[L] = make_uint4(w[0], w[1], w[2], w[3]);
+        out[32 + L] = make_uint4(w[4], w[5], w[6], w[7]);
+    } else if (fmt == 1) {
+        uint32_t w[3] = {0u, 0u, 0u};
+#pragma unroll
+        for (int s = 0; s < 16; ++s) six_bit_store(w, s, index_of(s) & 63u);
+#pragma unroll
+        for (int i = 0; i < 3; ++i) packed[six_bit_word(rt, kb, kblocks, L, i)] = w[i];
+    } else if (fmt == 2) {
+        uint32_t w[2] = {0u, 0u};
+#pragma unroll
+        for (int s = 0; s < 16; ++s) {
+            const int m = s >> 2, a = s & 3, byte = 2 * m + (a >> 1);
+            w[byte >> 2] |= (index_of(s) & 15u) << (8 * (byte & 3) + 4 * (a & 1));
+        }
+        reinterpret_cast<uint2*>(packed)[t] = make_uint2(w[0], w[1]);
+    } else {
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int s = 0; s < 16; ++s) w[s >> 2] |= index_of(s) << (8 * (s & 3));
+        reinterpret_cast<uint4*>(packed)[t] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
+__host__ __device__ constexpr int kTileRowBytes(int P) { return (P == 2 ? 512 : 1024) + 16; }   // rows 16 bytes apart in bank position
+
 // One warp per (row, group).  Steps in the order of Algorithm 1:
 //   s = ||w||_2 ; w+ = H diag(sign) (w/s) ; code = argmin_c ||w+_t - G[c]||^2 ; scale = s/sqrt(g).
 // Distances are fp32 in the plain (x-g)^2 form; '<' keeps the lowest index on ties.
@@ -129,7 +226,7 @@ __global__ void __launch_bounds__(128) encode_kernel(const T* __restrict__ W, co
 // bounds the winner's distance from any point of the cell, so only points whose distance to the cell is at most U (+ a
 // slack far above fp32 rounding) can be nearest.  (2) Of those, c is dropped if another candidate c' is nearer at all
 // corners of the cell by a margin: |z - c|^2 - |z - c'|^2 is affine in z, so its minimum over the cell is at a corner,
-// and c wins nowhere in the cell.  The surviving indices (at most four, else the cell is marked) are stored in
+// and c wins nowhere in the cell.  The surviving indices (at most four - two for p = 1 -, else the cell is marked) are stored in
 // ascending order, the last one repeated up to four: the encoder evaluates all four without a branch, and its strict
 // '<' keeps the lowest index on ties exactly like the exhaustive scan (a repeated candidate never replaces itself).
 // Marked cells and inputs outside the table take the exhaustive scan, done by the whole warp for one such point at a
@@ -215,7 +312,7 @@ __global__ void __launch_bounds__(256) build_cells_kernel(const float* __restric
             }
             const unsigned kept = __ballot_sync(0xffffffffu, have && !dominated);
             const int cnt = __popc(kept);
-            if (cnt >= 1 && cnt <= kMaxCand) {
+            if (cnt >= 1 && cnt <= (P == 2 ? kMaxCand : 2)) {      // the encoder evaluates four candidates for p = 2, two for p = 1
                 // the kept lane of rank r supplies byte r; the last one also fills the bytes above it
                 const int r = __popc(kept & ((1u << lane) - 1u));
                 const bool is_kept = (kept >> lane) & 1u;
@@ -228,13 +325,38 @@ __global__ void __launch_bounds__(256) build_cells_kernel(const float* __restric
     }
 }
 
-// the exhaustive scan of one point by the whole warp (lowest index among equal distances)
+// status of the encoder's bounded waits (HIGGS_ERR_TIMEOUT if one ran out), read by higgs_device_status
+__device__ int g_encode_status = 0;
+constexpr uint32_t kEncodeWaitLimit = 1u << 22;
+
+__device__ __forceinline__ uint32_t enc_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void enc_mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void enc_mbar_arrive(uint32_t bar) {
+    asm volatile("{\n\t.reg .b64 t;\n\tmbarrier.arrive.shared::cta.b64 t, [%0];\n\t}" ::"r"(bar) : "memory");
+}
+// waits for the phase of the given parity, at most kEncodeWaitLimit polls; a wait that runs out is recorded and the
+// caller carries on (wrong codes for that launch, which the status word reports, rather than a hung device)
+__device__ __forceinline__ void enc_mbar_wait(uint32_t bar, uint32_t parity) {
+    for (uint32_t it = 0; it < kEncodeWaitLimit; ++it) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+        if (done) return;
+    }
+    atomicExch(&g_encode_status, (int)HIGGS_ERR_TIMEOUT);
+}
+
+// the exhaustive scan of one point by the whole warp (lowest index among equal distances); point c is the first
+// eight (four for p = 1) bytes of row c of the replicated grid
 template <int P>
-__device__ __noinline__ int warp_scan(const float* sgrid, int n, float px, float py, int lane) {
+__device__ __noinline__ int warp_scan(const uint8_t* rep, int n, float px, float py, int lane) {
     float bd = INFINITY;
     int bc = 0x7fffffff;
     for (int c = lane; c < n; c += 32) {           // ascending within the lane: '<' keeps its lowest index
-        const float dx = px - sgrid[P * c], dy = P == 2 ? py - sgrid[2 * c + 1] : 0.f;
+        const float* g = reinterpret_cast<const float*>(rep + c * 128);
+        const float dx = px - g[0], dy = P == 2 ? py - g[1] : 0.f;
         const float d = P == 2 ? fmaf(dy, dy, dx * dx) : dx * dx;
         if (d < bd) { bd = d; bc = c; }
     }
@@ -247,40 +369,51 @@ __device__ __noinline__ int warp_scan(const float* sgrid, int n, float px, float
     return bc == 0x7fffffff ? 0 : bc;               // no distance compared below infinity (a NaN input): index 0, as the scan
 }
 
-// Persistent blocks of 16 warps, one (row, group) per warp and turn.  Shared memory: the cell table and the grid with
-// every point repeated across a 128-byte row (16 copies of an 8-byte point for p = 2, 32 copies of a float for p = 1), so
-// that a lane reads "its" copy and the 32 lookups of a warp never meet in a bank.
+// Persistent blocks of 16 warps; a block takes one row tile (16 rows) x one group per turn, warp w the tile's row w.
+// Shared memory: the cell table; the grid with every point repeated across a 128-byte row (16 copies of an 8-byte
+// point for p = 2, 32 copies of a float for p = 1: a lane reads "its" copy and the 32 lookups of a warp never meet in
+// a bank); two tiles of canonical codes, through which the block emits the packed stream itself (thread t assembles
+// the words of 64-input block t / 32, lane t % 32).  The warps of a block are not held in step: a warp puts its row
+// into the turn's tile and arrives on an mbarrier, and only a turn later - after its next search - waits for that
+// phase and packs the finished tile, so a warp may run up to one turn ahead of the slowest (a block-wide barrier per
+// turn made all sixteen warps wait for memory together and cost 20 %).  Writing tile t % 2 in turn t is safe: it was
+// last read when every warp packed tile t - 2, before its arrival of turn t - 1, which this warp has waited for.
+// canonical and packed may each be null (not both).
 template <typename T, int P>
 __global__ void __launch_bounds__(512, 2) encode_pruned_kernel(const T* __restrict__ W, const float* __restrict__ grid, int n,
                                                                const uint32_t* __restrict__ table,
-                                                               uint8_t* __restrict__ canonical, __half* __restrict__ scales,
+                                                               uint8_t* __restrict__ canonical, uint32_t* __restrict__ packed,
+                                                               int fmt, int bits, __half* __restrict__ scales,
                                                                int64_t N, int64_t K, uint64_t xi) {
     constexpr int NC = P == 2 ? kCells2 * kCells2 : kCells1;
     constexpr int CELLS = P == 2 ? kCells2 : kCells1;
+    constexpr int RS = kTileRowBytes(P);
     extern __shared__ __align__(128) uint8_t enc_smem[];
-    __shared__ float sgrid[256 * 2];
     uint32_t* cells = reinterpret_cast<uint32_t*>(enc_smem);
     uint8_t* rep = enc_smem + (size_t)NC * 4;
-    for (int i = threadIdx.x; i < n * P; i += blockDim.x) sgrid[i] = grid[i];
+    uint8_t* tiles_base = rep + (size_t)n * 128;
+    const uint32_t bar = enc_smem_u32(tiles_base + 2 * 16 * RS);      // mbarrier: one arrival per warp and turn
+    if (threadIdx.x == 0) enc_mbar_init(bar, 16);
     for (int i = threadIdx.x; i < NC / 4; i += blockDim.x)
         reinterpret_cast<uint4*>(cells)[i] = reinterpret_cast<const uint4*>(table)[i];
     for (int i = threadIdx.x; i < n * 32; i += blockDim.x)
         reinterpret_cast<float*>(rep)[i] = grid[P == 2 ? 2 * (i >> 5) + (i & 1) : (i >> 5)];
     __syncthreads();
 
-    const int lane = threadIdx.x & 31;
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const uint8_t* rep_lane = rep + (P == 2 ? (lane & 15) * 8 : lane * 4);
-    const int64_t groups = K / kGroup;
-    const int64_t tasks = N * groups;
-    const int64_t warps_total = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int64_t groups = K / kGroup, kblocks = K / kBlockK;
+    const int64_t turns = (N / 16) * groups;
     const float inv_w = CELLS / (2.0f * kCellR);
     const float magic = 8388608.0f + 0.5f * CELLS;
-    // (row, group) of the warp's task, advanced by the grid's stride without a division per task
-    const int64_t first = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    int64_t row = first / groups, gi = first % groups;
-    const int64_t step_rows = warps_total / groups, step_groups = warps_total % groups;
-    for (int64_t task = first; task < tasks; task += warps_total, row += step_rows, gi += step_groups) {
-        if (gi >= groups) { gi -= groups; ++row; }
+    // (row tile, group) of the block's turn, advanced by the grid's stride without a division per turn
+    int64_t rt = (int64_t)blockIdx.x / groups, gi = (int64_t)blockIdx.x % groups;
+    const int64_t step_tiles = (int64_t)gridDim.x / groups, step_groups = (int64_t)gridDim.x % groups;
+    int parity = 0;                  // tile of this turn
+    int64_t prev_rt = -1, prev_gi = 0;
+    for (int64_t turn = blockIdx.x; turn < turns; turn += gridDim.x, rt += step_tiles, gi += step_groups, parity ^= 1) {
+        if (gi >= groups) { gi -= groups; ++rt; }
+        const int64_t row = rt * 16 + wib;
         float v[32];
         load32<T>(W + row * K + gi * kGroup, lane, v);
         float ss = 0.0f;
@@ -294,7 +427,7 @@ __global__ void __launch_bounds__(512, 2) encode_pruned_kernel(const T* __restri
         for (int r = 0; r < 32; ++r) v[r] *= inv;
         apply_signs1024(v, xi, gi * kGroup, lane);
         fwht1024_warp(v, lane);
-        if (lane == 0) scales[((row >> 4) * groups + gi) * 16 + (row & 15)] = __float2half_rn(s * 0.03125f);
+        if (lane == 0) scales[(rt * groups + gi) * 16 + wib] = __float2half_rn(s * 0.03125f);
 
         uint32_t out[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};      // the lane's codes, one byte each, in storage order
         uint32_t slow = 0u;                                       // bit t: tuple t needs the exhaustive scan
@@ -335,81 +468,56 @@ __global__ void __launch_bounds__(512, 2) encode_pruned_kernel(const T* __restri
                     m &= m - 1;
                     const float px = __shfl_sync(0xffffffffu, v[P * t], src);
                     const float py = P == 2 ? __shfl_sync(0xffffffffu, v[2 * t + 1], src) : 0.f;
-                    const int bc = warp_scan<P>(sgrid, n, px, py, lane);
+                    const int bc = warp_scan<P>(rep, n, px, py, lane);
                     if (lane == src) out[t >> 2] = (out[t >> 2] & ~(0xffu << (8 * (t & 3)))) | ((uint32_t)bc << (8 * (t & 3)));
                 }
             }
         }
-        if (P == 2) {
-            // tuple t of chunk c sits at tuple index c*128 + lane*4 + (t&3): 4 consecutive bytes per chunk
-            uint8_t* dst = canonical + row * (K / 2) + gi * (kGroup / 2);
+        // tuple t of chunk c sits at tuple index c*128 + lane*4 + (t&3) (p = 2: four consecutive bytes per chunk);
+        // value t of chunk c at c*256 + lane*8 + t (p = 1: eight)
+        if (canonical) {
+            if (P == 2) {
+                uint8_t* dst = canonical + row * (K / 2) + gi * (kGroup / 2);
 #pragma unroll
-            for (int c = 0; c < 4; ++c) *reinterpret_cast<uint32_t*>(dst + c * 128 + lane * 4) = out[c];
-        } else {
-            uint8_t* dst = canonical + row * K + gi * kGroup;
+                for (int c = 0; c < 4; ++c) *reinterpret_cast<uint32_t*>(dst + c * 128 + lane * 4) = out[c];
+            } else {
+                uint8_t* dst = canonical + row * K + gi * kGroup;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) *reinterpret_cast<uint2*>(dst + c * 256 + lane * 8) = make_uint2(out[2 * c], out[2 * c + 1]);
+                for (int c = 0; c < 4; ++c) *reinterpret_cast<uint2*>(dst + c * 256 + lane * 8) = make_uint2(out[2 * c], out[2 * c + 1]);
+            }
         }
+        if (packed) {
+            if (prev_rt >= 0) {      // the tile of the turn before: complete once all sixteen warps have arrived
+                enc_mbar_wait(bar, (uint32_t)(parity ^ 1));
+                pack_item<P>(tiles_base + (parity ^ 1) * (16 * RS), RS, fmt, bits, wib, lane, prev_rt, prev_gi * 16 + wib, kblocks, packed);
+            }
+            uint8_t* mine = tiles_base + parity * (16 * RS) + wib * RS;
+            if (P == 2) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) *reinterpret_cast<uint32_t*>(mine + c * 128 + lane * 4) = out[c];
+            } else {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) *reinterpret_cast<uint2*>(mine + c * 256 + lane * 8) = make_uint2(out[2 * c], out[2 * c + 1]);
+            }
+            __syncwarp();
+            if (lane == 0) enc_mbar_arrive(bar);
+            prev_rt = rt;
+            prev_gi = gi;
+        }
+    }
+    if (packed && prev_rt >= 0) {
+        enc_mbar_wait(bar, (uint32_t)(parity ^ 1));
+        pack_item<P>(tiles_base + (parity ^ 1) * (16 * RS), RS, fmt, bits, wib, lane, prev_rt, prev_gi * 16 + wib, kblocks, packed);
     }
 }
 
-// ---- packed layout -----------------------------------------------------------
-// The packed stream is a sequence of blocks, block (rt, kb) covering rows
-// [16 rt, 16 rt + 16) and inputs [64 kb, 64 kb + 64), stored at block index
-// rt * (K/64) + kb.  Inside a block, lane L of the consuming warp owns a
-// contiguous run of bytes holding exactly the table indices of the A-fragment
-// registers it feeds to four m16n8k16 tensor-core steps: step m (inputs
-// 16m..16m+15 of the block), register a in 0..3 is the fp16 pair
-//   row   = 16 rt + (L>>2) + 8 (a&1)
-//   pairs = inputs 64 kb + 16 m + 2 (L&3) + 8 (a>>1) + {0, 1}.
-// "Slot" s = 4m + a, 16 slots per lane.
-//   byte-LUT format: 16 bytes per lane, byte s = table index of slot s; a block is
-//                    512 contiguous bytes, lane L at byte offset 16 L.
-//   six-bit format : three 32-bit words per lane and block.  Words 0 and 1 hold the
-//                    low nibbles: slot 4m+a sits in word m>>1 at bit 8a + 4(m&1).
-//                    Word 2 holds the high bit-pairs: slot 4m+a at bit 8a + 2m.
-//                    (The consumer rebuilds four byte-aligned indices with one shift
-//                    and one three-input logic operation each, see linear_mma.cu.)
-//   nibble format  : (n = 16) two 32-bit words per lane and block, 256 bytes per block, lane L at
-//                    byte offset 8 L.  Byte 2m + h of the lane holds the slots 4m + 2h (low
-//                    nibble) and 4m + 2h + 1 (high nibble): the two registers of one row pair.
-//   8-bit format   : (p = 1, n = 256) one byte per input: slot 4m + a is the halfword a & 1 of the lane's
-//                    word 2m + (a >> 1) (low byte = first input of the pair); a block is 1024 bytes, two
-//                    512-byte halves holding words 0..3 and 4..7 of every lane (16 bytes per lane each).
-//                    Two neighbouring blocks (2j, 2j+1 along K) form a 768-byte
-//                    super-block of three 256-byte planes; plane w stores word w of
-//                    lane L, block half h at 32-bit index 2L + h, so a warp reads
-//                    each plane with one coalesced 64-bit load per lane.
-__device__ __forceinline__ void slot_coords(int64_t rt, int64_t kb, int L, int s, int64_t& row, int64_t& pair) {
-    const int m = s >> 2, a = s & 3;
-    row = rt * 16 + (L >> 2) + 8 * (a & 1);
-    pair = kb * 32 + m * 8 + (L & 3) + 4 * (a >> 1);   // index of the 2-input pair along K
-}
-
-__device__ __forceinline__ void six_bit_store(uint32_t (&w)[3], int s, uint32_t code) {
-    const int m = s >> 2, a = s & 3;
-    w[m >> 1] |= (code & 15u) << (8 * a + 4 * (m & 1));
-    w[2] |= ((code >> 4) & 3u) << (8 * a + 2 * m);
-}
-__device__ __forceinline__ uint32_t six_bit_load(const uint32_t (&w)[3], int s) {
-    const int m = s >> 2, a = s & 3;
-    const uint32_t lo = (w[m >> 1] >> (8 * a + 4 * (m & 1))) & 15u;
-    const uint32_t hi = (w[2] >> (8 * a + 2 * m)) & 3u;
-    return lo | (hi << 4);
-}
-// 32-bit index of word w of (block kb, lane L) in the six-bit stream
-__device__ __forceinline__ int64_t six_bit_word(int64_t rt, int64_t kb, int64_t kblocks, int L, int w) {
-    return ((rt * (kblocks >> 1) + (kb >> 1)) * 3 + w) * 64 + 2 * L + (kb & 1);
-}
-
 // One block packs 16 rows x 1024 inputs: the canonical codes of the tile are staged in shared memory with coalesced
-// 16-byte loads (rows 16 bytes apart in bank position, so the byte gathers below meet no bank conflicts), then every
-// thread assembles the words of two (64-input block, lane) positions and stores them coalesced.
-template <int P, int FMT>
+// 16-byte loads (no bank conflicts in the byte gathers, see kTileRowBytes), then every thread assembles the words of
+// two (64-input block, lane) positions and stores them coalesced.
+template <int P>
 __global__ void __launch_bounds__(256) pack_kernel(const uint8_t* __restrict__ canonical, uint32_t* __restrict__ packed,
-                                                   int64_t N, int64_t K, int bits) {
-    constexpr int RB = P == 2 ? 512 : 1024;          // canonical bytes of one row and 1024 inputs
-    constexpr int RS = RB + 16;
+                                                   int64_t N, int64_t K, int fmt, int bits) {
+    constexpr int RS = kTileRowBytes(P), RB = RS - 16;          // RB canonical bytes of one row and 1024 inputs
     __shared__ __align__(16) uint8_t tile[16 * RS];
     const int64_t kblocks = K / kBlockK, ktiles = K / kGroup;
     const int64_t rt = blockIdx.x / ktiles, kt = blockIdx.x % ktiles;
@@ -419,48 +527,8 @@ __global__ void __launch_bounds__(256) pack_kernel(const uint8_t* __restrict__ c
             *reinterpret_cast<const uint4*>(canonical + ((rt * 16 + r) * ktiles + kt) * RB + c * 16);
     }
     __syncthreads();
-    constexpr bool SIX = FMT == 1, NIB = FMT == 2, B8 = FMT == 3;
-    const uint32_t mask = (1u << bits) - 1u;
-    for (int item = threadIdx.x; item < 512; item += 256) {
-        const int L = item & 31, kbl = item >> 5;
-        const int64_t kb = kt * 16 + kbl, blk = rt * kblocks + kb, t = blk * 32 + L;
-        // table index of slot s = 4m + a of this lane (two consecutive inputs): row (L>>2) + 8(a&1) of the tile,
-        // pair kbl*32 + m*8 + (L&3) + 4(a>>1)
-        auto index_of = [&](int s) -> uint32_t {
-            const int m = s >> 2, a = s & 3;
-            const int row = (L >> 2) + 8 * (a & 1), pair = kbl * 32 + m * 8 + (L & 3) + 4 * (a >> 1);
-            if (P == 2) return tile[row * RS + pair];
-            const uint8_t* q = tile + row * RS + 2 * pair;       // two scalar codes of `bits` bits each
-            return B8 ? ((uint32_t)q[0] | ((uint32_t)q[1] << 8)) : ((uint32_t)(q[0] & mask) | ((uint32_t)(q[1] & mask) << bits));
-        };
-        if (B8) {
-            uint32_t w[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
-#pragma unroll
-            for (int s = 0; s < 16; ++s) w[2 * (s >> 2) + ((s & 3) >> 1)] |= index_of(s) << (16 * (s & 1));
-            uint4* out = reinterpret_cast<uint4*>(packed) + blk * 64;      // 1024-byte block = 64 uint4
-            out[L] = make_uint4(w[0], w[1], w[2], w[3]);
-            out[32 + L] = make_uint4(w[4], w[5], w[6], w[7]);
-        } else if (SIX) {
-            uint32_t w[3] = {0u, 0u, 0u};
-#pragma unroll
-            for (int s = 0; s < 16; ++s) six_bit_store(w, s, index_of(s) & 63u);
-#pragma unroll
-            for (int i = 0; i < 3; ++i) packed[six_bit_word(rt, kb, kblocks, L, i)] = w[i];
-        } else if (NIB) {
-            uint32_t w[2] = {0u, 0u};
-#pragma unroll
-            for (int s = 0; s < 16; ++s) {
-                const int m = s >> 2, a = s & 3, byte = 2 * m + (a >> 1);
-                w[byte >> 2] |= (index_of(s) & 15u) << (8 * (byte & 3) + 4 * (a & 1));
-            }
-            reinterpret_cast<uint2*>(packed)[t] = make_uint2(w[0], w[1]);
-        } else {
-            uint32_t w[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-            for (int s = 0; s < 16; ++s) w[s >> 2] |= index_of(s) << (8 * (s & 3));
-            reinterpret_cast<uint4*>(packed)[t] = make_uint4(w[0], w[1], w[2], w[3]);
-        }
-    }
+    for (int item = threadIdx.x; item < 512; item += 256)
+        pack_item<P>(tile, RS, fmt, bits, item >> 5, item & 31, rt, kt * 16 + (item >> 5), kblocks, packed);
 }
 
 template <int P, int FMT>
@@ -525,43 +593,78 @@ int sm_count() {
 
 }  // namespace
 
-int launch_encode(const higgs_desc& d, const void* W, int w_dtype, const float* grid, uint8_t* canonical, void* scales,
-                  void* scratch, size_t scratch_bytes, cudaStream_t st) {
+int read_encode_status(int clear) {
+    int v = 0;
+    if (cudaMemcpyFromSymbol(&v, g_encode_status, sizeof(int)) != cudaSuccess) return HIGGS_ERR_CUDA;
+    if (clear && v != 0) {
+        const int zero = 0;
+        if (cudaMemcpyToSymbol(g_encode_status, &zero, sizeof(int)) != cudaSuccess) return HIGGS_ERR_CUDA;
+    }
+    return v;
+}
+
+size_t encoder_table_bytes(int p) { return (size_t)(p == 2 ? kCells2 * kCells2 : kCells1) * 4; }
+
+int launch_encoder_table(int p, int n, const float* grid, void* table, cudaStream_t st) {
+    if (p == 2) build_cells_kernel<2><<<592, 256, 0, st>>>(grid, n, static_cast<uint32_t*>(table));      // one warp per cell and turn
+    else build_cells_kernel<1><<<128, 256, 0, st>>>(grid, n, static_cast<uint32_t*>(table));
+    return cuda_status(cudaGetLastError());
+}
+
+// table: a prepared cell table, or null; build_space: where to build one (encoder_table_bytes, 16-byte aligned), or
+// null.  Large layers with a table take the pruned search, which also emits the packed stream when `packed` is given
+// (*packed_done = true); everything else is the exhaustive scan into `canonical`.
+int launch_encode(const higgs_desc& d, const void* W, int w_dtype, const float* grid, const void* table, void* build_space,
+                  uint8_t* canonical, void* packed, void* scales, bool* packed_done, cudaStream_t st) {
+    *packed_done = false;
     const int64_t warps = d.N * (d.K / kGroup);
     if (warps == 0) return HIGGS_OK;
-    const unsigned blocks = (unsigned)((warps + 3) / 4);
     __half* sc = static_cast<__half*>(scales);
-    // Large layers: the exact pruned search (persistent blocks that copy the candidate table once); otherwise the
-    // exhaustive scan, whose cost is small there.
-    const bool pruned = warps >= 2048 && scratch && scratch_bytes >= kCellTableBytes &&
-                        (reinterpret_cast<uintptr_t>(scratch) % 16) == 0;
-    uint32_t* table = static_cast<uint32_t*>(scratch);
-    const size_t smem = (size_t)(d.p == 2 ? kCells2 * kCells2 : kCells1) * 4 + (size_t)d.n * 128;
-    if (pruned) {
-        static int configured[64];
-        const int ok = device_once(configured, [] {
-            constexpr int kMax = kCells2 * kCells2 * 4 + 256 * 128;
-            bool good = true;
-            good = good && cudaFuncSetAttribute(encode_pruned_kernel<float, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMax) == cudaSuccess;
-            good = good && cudaFuncSetAttribute(encode_pruned_kernel<float, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMax) == cudaSuccess;
-            good = good && cudaFuncSetAttribute(encode_pruned_kernel<__nv_bfloat16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMax) == cudaSuccess;
-            good = good && cudaFuncSetAttribute(encode_pruned_kernel<__nv_bfloat16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMax) == cudaSuccess;
-            return good ? 1 : -1;
-        });
-        if (ok < 0) return HIGGS_ERR_CUDA;
-        if (d.p == 2) build_cells_kernel<2><<<592, 256, 0, st>>>(grid, d.n, table);      // one warp per cell and turn
-        else build_cells_kernel<1><<<128, 256, 0, st>>>(grid, d.n, table);
+    const bool pruned = warps >= kPrunedMinTasks && (table || build_space) && (canonical || packed);
+    if (!pruned) {
+        if (!canonical) return HIGGS_ERR_INVALID_ARG;
+        const unsigned blocks = (unsigned)((warps + 3) / 4);
+#define HIGGS_ENC(T, P) encode_kernel<T, P><<<blocks, 128, 0, st>>>(static_cast<const T*>(W), grid, d.n, canonical, sc, d.N, d.K, d.rht_seed)
+        if (w_dtype == HIGGS_F32 && d.p == 2) HIGGS_ENC(float, 2);
+        else if (w_dtype == HIGGS_F32 && d.p == 1) HIGGS_ENC(float, 1);
+        else if (w_dtype == HIGGS_BF16 && d.p == 2) HIGGS_ENC(__nv_bfloat16, 2);
+        else if (w_dtype == HIGGS_BF16 && d.p == 1) HIGGS_ENC(__nv_bfloat16, 1);
+        else return HIGGS_ERR_UNSUPPORTED;
+#undef HIGGS_ENC
+        return cuda_status(cudaGetLastError());
     }
-    const unsigned pblocks = 2u * (unsigned)sm_count();     // two blocks of 16 warps per SM; any count is correct
+    static int configured[64];
+    const int ok = device_once(configured, [] {
+        constexpr int kMax = kCells2 * kCells2 * 4 + 256 * 128 + 2 * 16 * kTileRowBytes(1) + 16;
+        bool good = true;
+        good = good && cudaFuncSetAttribute(encode_pruned_kernel<float, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMax) == cudaSuccess;
+        good = good && cudaFuncSetAttribute(encode_pruned_kernel<float, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMax) == cudaSuccess;
+        good = good && cudaFuncSetAttribute(encode_pruned_kernel<__nv_bfloat16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMax) == cudaSuccess;
+        good = good && cudaFuncSetAttribute(encode_pruned_kernel<__nv_bfloat16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMax) == cudaSuccess;
+        return good ? 1 : -1;
+    });
+    if (ok < 0) return HIGGS_ERR_CUDA;
+    if (!table) {
+        const int rc = launch_encoder_table(d.p, d.n, grid, build_space, st);
+        if (rc != HIGGS_OK) return rc;
+        table = build_space;
+    }
+    const uint32_t* tab = static_cast<const uint32_t*>(table);
+    uint32_t* pk = static_cast<uint32_t*>(packed);
+    const size_t smem = encoder_table_bytes(d.p) + (size_t)d.n * 128 + 2 * 16 * (size_t)kTileRowBytes(d.p) + 16;
+    const int64_t turns = (d.N / 16) * (d.K / kGroup);
+    const int64_t resident = 2 * (int64_t)sm_count();     // two blocks of 16 warps per SM; any count is correct
+    const unsigned blocks = (unsigned)(turns < resident ? turns : resident);
+    const int fmt = (int)format_of(d.p, d.n) - 1, bits = code_bits(d.n);
 #define HIGGS_ENC(T, P) \
-    if (pruned) encode_pruned_kernel<T, P><<<pblocks, 512, smem, st>>>(static_cast<const T*>(W), grid, d.n, table, canonical, sc, d.N, d.K, d.rht_seed); \
-    else encode_kernel<T, P><<<blocks, 128, 0, st>>>(static_cast<const T*>(W), grid, d.n, canonical, sc, d.N, d.K, d.rht_seed)
-    if (w_dtype == HIGGS_F32 && d.p == 2) { HIGGS_ENC(float, 2); }
-    else if (w_dtype == HIGGS_F32 && d.p == 1) { HIGGS_ENC(float, 1); }
-    else if (w_dtype == HIGGS_BF16 && d.p == 2) { HIGGS_ENC(__nv_bfloat16, 2); }
-    else if (w_dtype == HIGGS_BF16 && d.p == 1) { HIGGS_ENC(__nv_bfloat16, 1); }
+    encode_pruned_kernel<T, P><<<blocks, 512, smem, st>>>(static_cast<const T*>(W), grid, d.n, tab, canonical, pk, fmt, bits, sc, d.N, d.K, d.rht_seed)
+    if (w_dtype == HIGGS_F32 && d.p == 2) HIGGS_ENC(float, 2);
+    else if (w_dtype == HIGGS_F32 && d.p == 1) HIGGS_ENC(float, 1);
+    else if (w_dtype == HIGGS_BF16 && d.p == 2) HIGGS_ENC(__nv_bfloat16, 2);
+    else if (w_dtype == HIGGS_BF16 && d.p == 1) HIGGS_ENC(__nv_bfloat16, 1);
     else return HIGGS_ERR_UNSUPPORTED;
 #undef HIGGS_ENC
+    *packed_done = packed != nullptr;
     return cuda_status(cudaGetLastError());
 }
 
@@ -570,18 +673,11 @@ int launch_pack(const higgs_desc& d, const uint8_t* canonical, void* packed, cud
     if (tiles == 0) return HIGGS_OK;
     if (tiles > 0x7fffffff) return HIGGS_ERR_UNSUPPORTED;
     if (reinterpret_cast<uintptr_t>(canonical) % 16) return HIGGS_ERR_INVALID_ARG;
-    const unsigned blocks = (unsigned)tiles;
-    uint32_t* out = static_cast<uint32_t*>(packed);
     const Format f = format_of(d.p, d.n);
-    const int bits = code_bits(d.n);
-    if (f == Format::kByteLut && d.p == 2) pack_kernel<2, 0><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K, bits);
-    else if (f == Format::kByteLut && d.p == 1) pack_kernel<1, 0><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K, bits);
-    else if (f == Format::kSixBit && d.p == 2) pack_kernel<2, 1><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K, bits);
-    else if (f == Format::kSixBit) pack_kernel<1, 1><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K, bits);
-    else if (f == Format::kNibble && d.p == 2) pack_kernel<2, 2><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K, bits);
-    else if (f == Format::kNibble) pack_kernel<1, 2><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K, bits);
-    else if (f == Format::kByte8) pack_kernel<1, 3><<<blocks, 256, 0, st>>>(canonical, out, d.N, d.K, bits);
-    else return HIGGS_ERR_UNSUPPORTED;
+    if (f == Format::kNone) return HIGGS_ERR_UNSUPPORTED;
+    uint32_t* out = static_cast<uint32_t*>(packed);
+    if (d.p == 2) pack_kernel<2><<<(unsigned)tiles, 256, 0, st>>>(canonical, out, d.N, d.K, (int)f - 1, code_bits(d.n));
+    else pack_kernel<1><<<(unsigned)tiles, 256, 0, st>>>(canonical, out, d.N, d.K, (int)f - 1, code_bits(d.n));
     return cuda_status(cudaGetLastError());
 }
 

@@ -78,10 +78,13 @@ def test_full_size_layer_on_sampled_rows(name, N, K, p, n, batches):
         assert float((y2 - y).abs().max()) <= 1e-5 * float(y.abs().max())
 
 
-@pytest.mark.parametrize("p,n,N,K", [(2, 256, 8192, 2048), (2, 64, 4096, 4096), (1, 256, 8192, 1024)])
+@pytest.mark.parametrize("p,n,N,K", [(2, 256, 8192, 2048), (2, 64, 4096, 4096), (1, 256, 8192, 1024), (2, 16, 4096, 2048),
+                                     (1, 16, 2048, 4096), (1, 8, 4096, 2048), (1, 4, 8192, 1024)])
 def test_pruned_search_equals_exhaustive_scan(p, n, N, K):
-    """Large layers are encoded with the exact pruned nearest-point search, small ones with the exhaustive scan: rows are
-    independent, so re-encoding a slice of the rows as a small matrix must give the very same codes and scales."""
+    """Large layers are encoded with the exact pruned nearest-point search (which also emits the packed stream), small
+    ones with the exhaustive scan and the pack kernel: rows are independent, so re-encoding a slice of the rows as a
+    small matrix must give the very same codes, scales and packed bytes.  The same holds for the call with a search
+    table prepared beforehand and for the call that lends no workspace (pruned search, then the pack kernel)."""
     cfg = 2
     xi = inputs.rht_seed(cfg)
     W = inputs.make_weights(N, K, inputs.weight_seed(cfg, 5), bf16=True)
@@ -90,12 +93,51 @@ def test_pruned_search_equals_exhaustive_scan(p, n, N, K):
     W = inputs.bf16_round(W)
     _, gt = U.grid32(p, n)
     d = hb.make_desc(p, n, N, K, xi)
-    packed, scales, canon = hb.higgs_quantize(d, U.bf16_tensor(W), gt, want_canonical=True)
+    Wt = U.bf16_tensor(W)
+    packed, scales, canon = hb.higgs_quantize(d, Wt, gt, want_canonical=True)
     rows = 64
     ds = hb.make_desc(p, n, rows, K, xi)
     packed_s, scales_s, canon_s = hb.higgs_quantize(ds, U.bf16_tensor(W[:rows]), gt, want_canonical=True)
     assert torch.equal(canon[:rows], canon_s)
     assert torch.equal(hb.scales_from_tile_major(scales, N)[:rows], hb.scales_from_tile_major(scales_s, rows))
+    nb = hb.higgs_packed_bytes(ds)
+    assert torch.equal(packed[:nb], packed_s[:nb])
+    # the whole packed stream against the pack kernel on the canonical codes
+    assert torch.equal(packed[:hb.higgs_packed_bytes(d)], hb.higgs_pack_codes(d, canon)[:hb.higgs_packed_bytes(d)])
+    table = hb.higgs_make_encoder_table(p, n, gt)
+    for kwargs in ({"table": table}, {"table": table, "want_canonical": True}, {"want_canonical": True, "workspace": False}, {}):
+        packed2, scales2, canon2 = hb.higgs_quantize(d, Wt, gt, **kwargs)
+        assert torch.equal(packed2, packed) and torch.equal(scales2, scales), kwargs
+        assert canon2 is None or torch.equal(canon2, canon), kwargs
+    assert hb.higgs_device_status() == hb.HIGGS_OK
+
+
+@pytest.mark.parametrize("p,n", [(2, 256), (2, 64), (1, 256), (1, 16)])
+def test_pruned_search_on_a_crowded_grid_falls_back_to_the_scan(p, n):
+    """A grid that is nothing like the optimal one: its points crowd on a small circle (p = 2) or in a short interval
+    (p = 1), with exact duplicates, so cells near the middle have more candidates than a list holds and the encoder
+    must take the exhaustive scan for the points that land there - with the lowest index among equal distances."""
+    rng = np.random.default_rng(77)
+    if p == 2:
+        ang = np.sort(rng.uniform(0, 2 * np.pi, n))
+        g = np.stack([0.4 * np.cos(ang), 0.4 * np.sin(ang)], axis=1)
+    else:
+        g = np.sort(rng.uniform(-0.02, 0.02, n))[:, None]
+    g[n // 2] = g[n // 2 - 1]                           # a duplicate: equal distances, the lower index must win
+    gt = torch.from_numpy(g.astype(np.float32)).to(U.dev())
+    N, K, xi = 4096, 1024, inputs.rht_seed(3)
+    W = inputs.make_weights(N, K, inputs.weight_seed(3, 1), bf16=True)
+    d = hb.make_desc(p, n, N, K, xi)
+    packed, scales, canon = hb.higgs_quantize(d, U.bf16_tensor(W), gt, want_canonical=True)
+    rows = 32
+    ds = hb.make_desc(p, n, rows, K, xi)
+    _, _, canon_s = hb.higgs_quantize(ds, U.bf16_tensor(W[:rows]), gt, want_canonical=True)
+    assert torch.equal(canon[:rows], canon_s)
+    assert int((canon == n // 2).sum()) == 0            # the duplicate with the higher index never wins
+    # and the oracle agrees on a few rows (exact ties between duplicates aside, which the rule above settles)
+    q, _ = U.oracle_encode(W[:4], G, g.astype(np.float32).astype(np.float64), xi)
+    U.compare_codes(canon[:4].cpu().numpy(), q, max_frac=5e-3)
+    assert hb.higgs_device_status() == hb.HIGGS_OK
 
 
 def test_general_grid_encoder_full_size_on_sampled_rows():
