@@ -304,31 +304,25 @@ def divisor_at_most(steps: int, cap: int) -> int:
 class Quantized:
     """One layer encoded on the device (Algorithm 1) with everything a timed product or a parity check needs."""
 
-    def __init__(self, hb, torch, dev, name, N, K, pn, xi, grid, W, time_it=False):
+    def __init__(self, hb, torch, dev, name, N, K, pn, xi, grid, W, table=None):
         self.name, self.N, self.K, self.pn = name, N, K, pn
         self.desc = hb.make_desc(pn[0], pn[1], N, K, xi)
-        self.grid = grid
-        self.enc_ms = None
-        wsq = torch.empty(hb.higgs_workspace_bytes(self.desc, hb.HIGGS_OP_QUANTIZE), dtype=torch.uint8, device=dev)
-        pk, sc, _ = hb.higgs_quantize(self.desc, W, grid, workspace=wsq)
-        if time_it:      # second call into the same buffers: only the library's kernels are inside the timed region
-            torch.cuda.synchronize()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            hb.higgs_quantize(self.desc, W, grid, workspace=wsq, out=(pk, sc))
-            e1.record()
-            torch.cuda.synchronize()
-            self.enc_ms = e0.elapsed_time(e1)
-        del wsq
+        self.grid, self.table = grid, table
+        self.wsq = torch.empty(hb.higgs_workspace_bytes(self.desc, hb.HIGGS_OP_QUANTIZE), dtype=torch.uint8, device=dev)
+        pk, sc, _ = hb.higgs_quantize(self.desc, W, grid, workspace=self.wsq, table=table)
         self.packed, self.scales = [pk], [sc]
         self.bytes = layer_bytes(N, K, *pn)
+
+    def encode_again(self, hb, W):
+        """A second call into the same buffers: only the library's kernels are inside a timed region around it."""
+        hb.higgs_quantize(self.desc, W, self.grid, workspace=self.wsq, out=(self.packed[0], self.scales[0]), table=self.table)
 
     @classmethod
     def from_buffers(cls, name, desc, grid, packed, scales):
         """A layer whose packed buffers exist already (row-concatenated layers)."""
         q = cls.__new__(cls)
         q.name, q.N, q.K, q.pn, q.desc, q.grid = name, desc.N, desc.K, (desc.p, desc.n), desc, grid
-        q.packed, q.scales, q.bytes, q.enc_ms = list(packed), list(scales), layer_bytes(desc.N, desc.K, desc.p, desc.n), None
+        q.packed, q.scales, q.bytes, q.table, q.wsq = list(packed), list(scales), layer_bytes(desc.N, desc.K, desc.p, desc.n), None, None
         return q
 
     def ensure_copies(self, count):
@@ -521,11 +515,12 @@ def run_ours(args):
     set_bytes = sum(layer_bytes(N, K, *pn[li]) for li, (_, N, K) in enumerate(layers))
     copies = min(64, max(2, -(-2 * L2_BYTES // set_bytes)))      # rotating copies so that no step finds its codes in L2
     qs, xs, xs_host, xs32, ws, ys = [], [], [], [], [], []
+    tables = {key: hb.higgs_make_encoder_table(key[0], key[1], grids[key]) for key in set(pn)}     # once per grid
+    Ws = []
     for li, (name, N, K) in enumerate(layers):
         W = torch.from_numpy(inputs.make_weights(N, K, inputs.weight_seed(cfg, li), bf16=True)).to(dev).to(torch.bfloat16)
-        q = Quantized(hb, torch, dev, name, N, K, pn[li], xi, grids[pn[li]], W, time_it=True)
-        del W
-        q.ensure_copies(copies)
+        q = Quantized(hb, torch, dev, name, N, K, pn[li], xi, grids[pn[li]], W, table=tables[pn[li]])
+        Ws.append(W)
         qs.append(q)
         # q/k/v read the same block input, so do gate/up
         xi_of = {"k": "q", "v": "q", "up": "gate"}.get(name, name)
@@ -540,8 +535,20 @@ def run_ours(args):
         ws.append(torch.empty(hb.higgs_workspace_bytes(q.desc, hb.HIGGS_OP_LINEAR, B), dtype=torch.uint8, device=dev))
         ys.append(torch.empty((B, N), dtype=torch.float32, device=dev))
     descs = [q.desc for q in qs]
-    enc_ms = sum(q.enc_ms for q in qs)
+    # the encoder's time: one more pass over all layers into the same buffers, the calls enqueued back to back
+    torch.cuda.synchronize()
+    e0, e1 = ev(), ev()
+    e0.record()
+    for q, W in zip(qs, Ws):
+        q.encode_again(hb, W)
+    e1.record()
+    torch.cuda.synchronize()
+    enc_ms = e0.elapsed_time(e1)
     enc_weights = sum(N * K for _, N, K in layers)
+    del Ws
+    for q in qs:
+        q.wsq = None
+        q.ensure_copies(copies)
 
     # layers that read the same block input share one rotation (the transform is isolated from the product, Sec. 4.3);
     # a layer whose K is split across thread blocks goes through higgs_linear, whose rotation kernel also clears y
@@ -873,7 +880,9 @@ def run_ours(args):
             "clocks": clocks,
             "roofline": roofline,
             "cpu_baseline": cpu,
-            "quantize": {"weights_per_s": wps, "ms": enc_ms, "weights": enc_weights, "grid_fit": grid_info,
+            "quantize": {"weights_per_s": wps, "ms": enc_ms, "weights": enc_weights,
+                         "calls": f"{len(layers)} higgs_quantize_prepared calls back to back (search table built once per grid), second pass into the same buffers",
+                         "grid_fit": grid_info,
                          "rooflines": encoder_rooflines(wps, pn, [N * K for _, N, K in layers], clocks, peak, peak_src)},
             "detail": detail,
         }
