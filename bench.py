@@ -901,7 +901,7 @@ def split_units(total_units: int, world: int, rank: int):
 
 def run_sharded(args):
     """ONE layer set sharded over the ranks (strong scaling): every rank encodes and multiplies its shard of every matrix
-    and the kernels' epilogues write into peer-mapped buffers of all ranks (plain stores over NVLink, no multicast, no
+    and the kernels' epilogues write into peer-mapped buffers of all ranks (plain stores over NVLink, one per destination, no
     library kernel on peer memory).  rows: higgs_linear_gather, every rank ends a step holding the full outputs.  k:
     higgs_linear_kshard into slot buffers, a barrier, higgs_reduce_slots.  Between a step's writes and its readers
     stands the symmetric-memory barrier of the process group, enqueued on the timed stream."""

@@ -293,7 +293,7 @@ int higgs_linear_multi_launch_count(int32_t count, const higgs_desc* const* desc
  * written straight into columns [row_offset, row_offset + desc->N) of EVERY destination
  *   y_dsts[i] : device-accessible [B][ld] of y_dtype, i < n_dst <= 8 - this device's own output buffer first, then the
  *               peer-mapped pointers of the other devices' buffers (cudaDeviceEnablePeerAccess / IPC / symmetric
- *               memory; plain stores over NVLink, no multicast).
+ *               memory; plain stores over NVLink, one per destination).
  * The kernels store to all destinations from their epilogue (a K-split small-batch product sums into the workspace
  * first and a copy kernel spreads the result).  The call neither waits for nor signals other devices: the caller
  * orders "all shards written" before any reader (e.g. a barrier on the participating streams), and no two shards
@@ -322,7 +322,7 @@ int higgs_shard_rows(int64_t N, int32_t world, int32_t rank, int32_t multiple, i
  * of the unsharded layer.  (HOST function.)
  *
  * higgs_linear_kshard: this device's partial product, written from the kernels' epilogues (plain stores, own
- * memory and peer-mapped memory alike, no multicast) into slot `rank` of EVERY device's slot buffer
+ * memory and peer-mapped memory alike, one store per destination) into slot `rank` of EVERY device's slot buffer
  *   slot_bufs[i] : device-accessible fp32 [world][B][N] of device i (i = rank: this device's own), a HOST array;
  * desc/x_shard/packed/scales describe the shard (x_shard is [B][K_r] bf16).  It neither waits for nor signals other
  * devices: the caller orders "all partials written" before higgs_reduce_slots (a barrier of the process group).
