@@ -158,7 +158,6 @@ __device__ __forceinline__ void fwht1024_warp(float (&v)[32], int lane) {
 // Flips the signs of the 32 values of this lane (mapping above) for the group starting at input k0 (a multiple
 // of 1024): chunk c covers inputs k0 + c*256 + lane*8 .. +7, eight consecutive bits of one 64-bit sign word.
 __device__ __forceinline__ void apply_signs1024(float (&v)[32], uint64_t xi, int64_t k0, int lane) {
-#pragma unroll
     // the group's 16 sign words: lane l computes word l & 15, chunk c of a lane needs word 4c + lane/8
     const uint64_t word = sign_word(xi, ((uint64_t)k0 >> 6) + (uint64_t)(lane & 15));
     const uint32_t lo = (uint32_t)word, hi = (uint32_t)(word >> 32);

@@ -241,7 +241,6 @@ constexpr uint32_t kCellScan = 1u;     // bytes (1, 0, 0, 0) are not an ascendin
 constexpr float kCellR = 4.0f;
 constexpr float kCandSlack = 1e-3f;
 constexpr float kDominance = 1e-3f;    // margin of step (2) on squared distances (fp32 rounding there is below 1e-5)
-constexpr size_t kCellTableBytes = (size_t)(kCells2 * kCells2 > kCells1 ? kCells2 * kCells2 : kCells1) * 4;
 
 template <int P>
 __global__ void __launch_bounds__(256) build_cells_kernel(const float* __restrict__ grid, int n, uint32_t* __restrict__ table) {
