@@ -652,15 +652,20 @@ int launch_encode(const higgs_desc& d, const void* W, int w_dtype, const float* 
     uint32_t* pk = static_cast<uint32_t*>(packed);
     const size_t smem = encoder_table_bytes(d.p) + (size_t)d.n * 128 + 2 * 16 * (size_t)kTileRowBytes(d.p) + 16;
     const int64_t turns = (d.N / 16) * (d.K / kGroup);
-    const int64_t resident = 2 * (int64_t)sm_count();     // two blocks of 16 warps per SM; any count is correct
-    const unsigned blocks = (unsigned)(turns < resident ? turns : resident);
     const int fmt = (int)format_of(d.p, d.n) - 1, bits = code_bits(d.n);
+    // persistent grid: as many blocks as are resident at once (two of 16 warps per SM); any count is correct
 #define HIGGS_ENC(T, P) \
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, encode_pruned_kernel<T, P>, 512, smem) != cudaSuccess || per_sm < 1) per_sm = 1; \
+    resident = (int64_t)per_sm * sm_count(); \
+    blocks = (unsigned)(turns < resident ? turns : resident); \
     encode_pruned_kernel<T, P><<<blocks, 512, smem, st>>>(static_cast<const T*>(W), grid, d.n, tab, canonical, pk, fmt, bits, sc, d.N, d.K, d.rht_seed)
-    if (w_dtype == HIGGS_F32 && d.p == 2) HIGGS_ENC(float, 2);
-    else if (w_dtype == HIGGS_F32 && d.p == 1) HIGGS_ENC(float, 1);
-    else if (w_dtype == HIGGS_BF16 && d.p == 2) HIGGS_ENC(__nv_bfloat16, 2);
-    else if (w_dtype == HIGGS_BF16 && d.p == 1) HIGGS_ENC(__nv_bfloat16, 1);
+    int per_sm = 0;
+    int64_t resident = 0;
+    unsigned blocks = 0;
+    if (w_dtype == HIGGS_F32 && d.p == 2) { HIGGS_ENC(float, 2); }
+    else if (w_dtype == HIGGS_F32 && d.p == 1) { HIGGS_ENC(float, 1); }
+    else if (w_dtype == HIGGS_BF16 && d.p == 2) { HIGGS_ENC(__nv_bfloat16, 2); }
+    else if (w_dtype == HIGGS_BF16 && d.p == 1) { HIGGS_ENC(__nv_bfloat16, 1); }
     else return HIGGS_ERR_UNSUPPORTED;
 #undef HIGGS_ENC
     *packed_done = packed != nullptr;
