@@ -109,7 +109,7 @@ def measured_peaks():
 # the measured weights/s and a counted constant, not read from a counter in this run.  HBM: what the encoder must move
 # per weight - the bf16 weight in, log2(n)/p bits of code and 16/1024 bits of scale out - against the copy peak; this
 # is the floor an exact pruned search approaches.
-ENCODER_WARP_INSTR_PER_WEIGHT = {(2, 256): 1677.0 / 1024.0}
+ENCODER_WARP_INSTR_PER_WEIGHT = {(2, 256): 1776.0 / 1024.0}
 
 
 def encoder_rooflines(weights_per_s, pn, sizes, clocks, hbm_peak, peak_src):
