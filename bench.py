@@ -741,6 +741,17 @@ def run_ours(args):
                 t = tb if (li == big and Bk == B) else time_product(hb, torch, stream, q, Bk, xk, reps=100)
                 par = parity_on_sampled_rows(hb, oracle, q, x32, t["y"], xi, grids64[q.pn])
                 detail["layers"].append(product_row(hb, q, Bk, t, peak, peak_tf, par))
+        # the step itself, as timed (multi-matrix products, shared rotations, fused rotations): one more step, then every
+        # layer's output of that step against the oracle on sampled rows
+        with torch.cuda.stream(stream):
+            step(0)
+            stream.synchronize()
+        step_par = [parity_on_sampled_rows(hb, oracle, qs[li], xs32[li], ys[li], xi, grids64[qs[li].pn]) for li in range(len(layers))]
+        detail["step_parity"] = {"max_rel": float(f"{max(p[0] for p in step_par):.3g}"),
+                                 "max_over_rms": float(f"{max(p[1] for p in step_par):.3g}"),
+                                 "what": "outputs of one whole step (the launches that are timed) for all layers, 16 sampled rows each"}
+        if detail["step_parity"]["max_rel"] > 2e-3:
+            raise SystemExit(f"parity re-check failed on the step's outputs: {detail['step_parity']}")
         detail["parity_bound"] = "max |y - y^| / max |y^| <= 2e-3 on 16 sampled rows of every timed layer, fp64 oracle on the device's codes"
         worst = max(r["parity_max_rel"] for r in detail["layers"])
         if worst > 2e-3:
