@@ -145,3 +145,29 @@ def test_seeded_grid_and_helper_arguments():
     assert L.higgs_launch_floor(148, 2048, 0, None) == hb.HIGGS_ERR_INVALID_ARG
     assert L.higgs_selftest_wait(0, 100, None, None) == hb.HIGGS_ERR_INVALID_ARG
     assert L.higgs_selftest_wait(2, 100, a, None) == hb.HIGGS_ERR_INVALID_ARG
+
+
+def test_encoder_table_queries_and_arguments():
+    """The prepared search table: one 32-bit list per cell (128 x 128 cells for p = 2, 1024 for p = 1); argument
+    checks run before any CUDA call."""
+    L = binding.lib
+    a, odd = ctypes.c_void_p(0x1000), ctypes.c_void_p(0x1008)
+    assert L.higgs_encoder_table_bytes(2, 256) == 128 * 128 * 4
+    assert L.higgs_encoder_table_bytes(2, 64) == 128 * 128 * 4
+    assert L.higgs_encoder_table_bytes(1, 16) == 1024 * 4
+    assert L.higgs_encoder_table_bytes(3, 830) == 0 and L.higgs_encoder_table_bytes(2, 100) == 0
+    assert L.higgs_make_encoder_table(3, 830, a, a, None) == hb.HIGGS_ERR_UNSUPPORTED
+    assert L.higgs_make_encoder_table(2, 256, None, a, None) == hb.HIGGS_ERR_INVALID_ARG
+    assert L.higgs_make_encoder_table(2, 256, a, None, None) == hb.HIGGS_ERR_INVALID_ARG
+    assert L.higgs_make_encoder_table(2, 256, a, odd, None) == hb.HIGGS_ERR_INVALID_ARG
+    d = hb.make_desc(2, 256, 4096, 4096, 1)
+    P = ctypes.byref(d)
+    ws = hb.higgs_workspace_bytes(d, hb.HIGGS_OP_QUANTIZE)
+    assert ws >= L.higgs_encoder_table_bytes(2, 256)         # a large layer's workspace always holds the table
+    assert L.higgs_quantize_prepared(P, None, hb.HIGGS_BF16, a, a, a, a, None, a, ws, None) == hb.HIGGS_ERR_INVALID_ARG
+    assert L.higgs_quantize_prepared(P, a, hb.HIGGS_BF16, a, odd, a, a, None, a, ws, None) == hb.HIGGS_ERR_INVALID_ARG    # table alignment
+    assert L.higgs_quantize_prepared(P, a, hb.HIGGS_BF16, a, a, a, a, odd, a, ws, None) == hb.HIGGS_ERR_INVALID_ARG      # canonical alignment
+    assert L.higgs_quantize_prepared(P, a, hb.HIGGS_BF16, a, a, a, a, None, None, 0, None) == hb.HIGGS_ERR_INVALID_ARG   # no canonical_out: workspace needed
+    assert L.higgs_quantize_prepared(P, a, hb.HIGGS_BF16, a, a, a, a, None, a, 16, None) == hb.HIGGS_ERR_WORKSPACE
+    empty = hb.make_desc(2, 256, 0, 4096, 1)
+    assert L.higgs_quantize_prepared(ctypes.byref(empty), None, hb.HIGGS_BF16, None, None, None, None, None, None, 0, None) == hb.HIGGS_OK
