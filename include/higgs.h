@@ -184,6 +184,9 @@ int higgs_gaussian_samples(int p, uint64_t sample_seed, int64_t num_samples, flo
  *   scales_out     device, higgs_scales_bytes() bytes, 16-byte aligned: fp16 scales stored
  *                  tile-major, element (r, i) at index ((r / 16) * (K/g) + i) * 16 + r % 16
  *   canonical_out  device, optional, [N][K/p] one byte per code (for checking), 16-byte aligned
+ *   workspace      device, 256-byte aligned, higgs_workspace_bytes(desc, HIGGS_OP_QUANTIZE, 0) bytes: required when
+ *                  canonical_out is NULL (HIGGS_ERR_INVALID_ARG / HIGGS_ERR_WORKSPACE otherwise); optional with
+ *                  canonical_out (without it a large layer's packed stream is written by a second kernel)
  */
 int higgs_quantize(const higgs_desc* desc, const void* W, int w_dtype, const float* grid,
                    void* packed_out, void* scales_out, uint8_t* canonical_out,
