@@ -160,3 +160,19 @@ def test_general_grid_encoder_full_size_on_sampled_rows():
     assert ulp.max() <= 1
     t2_rows = oracle.layer_error(W[rows], q.codes, sc16.astype(np.float64), G, g64, xi)
     assert abs(t2 - t2_rows) <= 0.03 * t2_rows, (t2, t2_rows)
+
+
+@pytest.mark.parametrize("p,n,N,K", [(2, 256, 14336, 4096), (2, 64, 8192, 8192), (1, 16, 4096, 14336)])
+def test_encoder_is_reproducible_run_to_run(p, n, N, K):
+    """The warps of an encoder block run up to one turn apart and hand their rows over through a shared-memory tile: a
+    race there would show as packed bytes that differ between runs, or from the pack kernel on the canonical codes."""
+    _, gt = U.grid32(p, n)
+    W = U.bf16_tensor(inputs.make_weights(N, K, inputs.weight_seed(2, 9), bf16=True))
+    d = hb.make_desc(p, n, N, K, inputs.rht_seed(2))
+    table = hb.higgs_make_encoder_table(p, n, gt)
+    ref_p, ref_s, ref_c = hb.higgs_quantize(d, W, gt, want_canonical=True, workspace=False)      # search, then the pack kernel
+    assert torch.equal(hb.higgs_pack_codes(d, ref_c), ref_p)
+    for it in range(12):
+        pk, sc, _ = hb.higgs_quantize(d, W, gt, table=table if it % 2 else None)
+        assert torch.equal(pk, ref_p) and torch.equal(sc, ref_s), it
+    assert hb.higgs_device_status() == hb.HIGGS_OK
