@@ -73,6 +73,7 @@ constexpr uint32_t kMaxDynSmem = 232448;
 constexpr uint32_t kSmallBytes = 4096;  // barriers, recycle counters, abort flag
 constexpr int kWarps = 16;
 constexpr int kMaxDepth = 8;            // ring slots per warp
+constexpr int kArmFirst = 1;            // tasks a warp requests before its loop starts; the ring then fills two requests per consumed task
 constexpr int kMaxAccSlots = 32;        // items whose partial tiles may be parked at once
 constexpr uint32_t kWaitLimit = 1u << 22;
 constexpr uint32_t kNibbleTileBytes = 32768; // nibble format: the table rows are full, the partial tiles live at the end of shared memory
@@ -477,7 +478,8 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
             if (b < prm.B) xraw[b] = *reinterpret_cast<const uint4*>(prm.x + (int64_t)b * prm.K + kbase + lane * 8);
     }
     int issued = 0;
-    for (; issued < n_tasks && issued < D; ++issued) issue(issued);
+    for (; issued < n_tasks && issued < D && issued < kArmFirst; ++issued) issue(issued);
+    int d_issue = issued == D ? 0 : issued;      // slot of the next task to be requested
     auto scratch = [&](uint32_t off) { return part0 + (off >> 7) * kPieceStride + (off & 127u); };
     // (when K < 4096 several units own the same 1024-group: only the first of them transforms it - every warp of the
     // block would otherwise spend the same issue slots on the same butterflies - and the others read the result)
@@ -745,10 +747,16 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
         asm volatile("ld.shared.u16 %0, [%1];" : "=h"(shi16) : "r"(slot + Codes::kBytes + (uint32_t)g * 2u + 16u));
         __syncwarp();
         ++done;
-        if (issued < n_tasks) {                  // the slot's words are in registers: re-arm it for task i + D
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            issue(d);
-            ++issued;
+        // the slot's words are in registers: request further tasks - task i + D into this slot in the steady state, two
+        // per consumed task while the ring is still filling (the first kArmFirst were requested before the loop)
+        if (issued < n_tasks) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            if (issued < n_tasks && issued < i + 1 + D) {
+                issue(d_issue);
+                ++issued;
+                if (++d_issue == D) d_issue = 0;
+            }
         }
         if (++d == D) { d = 0; ph ^= 1u; }
 
