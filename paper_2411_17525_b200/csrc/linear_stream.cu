@@ -437,6 +437,11 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
     // (every lane runs the loop so that addresses stay warp-uniform - bulk copies take uniform operands - and one
     // elected lane issues)
     pdl_trigger();
+    // The first task's copy starts now: the weights are inputs that no kernel of the stream writes (a producer of
+    // weights ends with a fence kernel, so this kernel cannot have started while one was running).
+    int issued = 0;
+    for (; issued < n_tasks && issued < D && issued < kArmFirst; ++issued) issue(issued);
+    int d_issue = issued == D ? 0 : issued;      // slot of the next task to be requested
     // Everything above depends only on the weights.  The activations (and y, which the previous kernel in the
     // stream may still be reading or clearing) are touched only after the previous kernel has completed.
     pdl_wait();
@@ -477,9 +482,6 @@ __global__ void __launch_bounds__((kWarps + 1) * 32, 1) linear_stream_kernel(con
         for (int b = 0; b < 2; ++b)
             if (b < prm.B) xraw[b] = *reinterpret_cast<const uint4*>(prm.x + (int64_t)b * prm.K + kbase + lane * 8);
     }
-    int issued = 0;
-    for (; issued < n_tasks && issued < D && issued < kArmFirst; ++issued) issue(issued);
-    int d_issue = issued == D ? 0 : issued;      // slot of the next task to be requested
     auto scratch = [&](uint32_t off) { return part0 + (off >> 7) * kPieceStride + (off & 127u); };
     // (when K < 4096 several units own the same 1024-group: only the first of them transforms it - every warp of the
     // block would otherwise spend the same issue slots on the same butterflies - and the others read the result)
