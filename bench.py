@@ -396,6 +396,9 @@ def product_row(hb, q, B, t, peak, peak_tf, parity=None):
     else:
         gb = alg / (t["us"] * 1e-6) / 1e9
         row["roofline"] = {"bound": "hbm", "achieved": round(gb, 1), "peak": peak, "unit": "GB/s", "frac": round(gb / peak, 4)}
+        # table lookups alone as a share of one 32-lane shared-memory wavefront per SM and clock (148 SMs, 1965 MHz)
+        per_lookup = {(2, 256): 2, (2, 64): 2, (1, 16): 2, (1, 8): 2, (2, 16): 4, (1, 4): 4, (1, 256): 1}[(p, n)]
+        row["lut_gather_frac"] = round(q.N * q.K / per_lookup / 32.0 / (t["us"] * 1e-6) / (148 * 1965e6), 4)
     if parity is not None:
         row["parity_max_rel"], row["parity_max_over_rms"] = (float(f"{v:.3g}") for v in parity)
     return row
@@ -720,6 +723,16 @@ def run_ours(args):
     else:
         roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                     "peak_source": f"of {peak_src}", "algorithmic_bytes": alg, "frac_of_8TBps": achieved / 8000.0, **common}
+        # the secondary bound of a lookup-table kernel: every pair of weights (every weight of the 8-bit grid, every four
+        # of the 2-bit grids) is one 32-lane shared-memory gather; an SM serves one such wavefront per clock
+        per_lookup = {(2, 256): 2, (2, 64): 2, (1, 16): 2, (1, 8): 2, (2, 16): 4, (1, 4): 4, (1, 256): 1}[(p, n)]
+        gathers = qb.N * qb.K / per_lookup / 32.0
+        mhz = (clocks or {}).get("sm_mhz") or 1965.0
+        gpeak = 148 * mhz * 1e6
+        roofline["lut_gather"] = {"bound": "shared-memory gathers", "achieved": gathers / (tb["us"] * 1e-6) / 1e9,
+                                  "peak": gpeak / 1e9, "unit": "G wavefronts/s", "frac": gathers / (tb["us"] * 1e-6) / gpeak,
+                                  "note": "table lookups alone, 32 per wavefront, against 148 SMs x one wavefront per clock at "
+                                          "the sampled SM clock; the code words' own loads and stores share that path"}
 
     detail = None
     if not args.no_detail and rank == 0 and world == 1:      # (detail times more launches with collectives-free code paths: single-GPU runs only)
