@@ -346,16 +346,16 @@ def parity_on_sampled_rows(hb, oracle, q, x_host32, y, xi, grid64, rows=16, seed
     return float(err / np.max(np.abs(y_ref))), float(err / np.sqrt(np.mean(y_ref ** 2)))
 
 
-def time_product(hb, torch, stream, q, B, x_dev, reps=200, copies_bytes=2 * L2_BYTES):
+def time_product(hb, torch, stream, q, B, x_dev, reps=200, copies_bytes=512 << 20):
     """One launch of the product kernel (D2-D5 on already rotated activations) of layer `q` at batch B, timed with CUDA
-    events on the launching stream: a CUDA graph of back-to-back launches over rotating weight copies (>= 2 x L2, so no
+    events on the launching stream: a CUDA graph of back-to-back launches over rotating weight copies (>= 512 MB, so no
     launch finds its codes in L2), every replay timed separately.  Returns mean / median / min microseconds per launch
     over the replays, the kernels per call and the output of the last launch."""
     d = q.desc
     xdag = hb.higgs_rotate_activations(d, x_dev)
     yk = torch.empty((B, d.N), dtype=torch.float32, device=x_dev.device)
     wk = torch.empty(hb.higgs_workspace_bytes(d, hb.HIGGS_OP_LINEAR, B), dtype=torch.uint8, device=x_dev.device)
-    q.ensure_copies(min(64, max(2, -(-copies_bytes // q.bytes))))
+    q.ensure_copies(min(1024, max(2, -(-copies_bytes // q.bytes))))
     n = len(q.packed)
     ev = lambda: torch.cuda.Event(enable_timing=True)
     with torch.cuda.stream(stream):
@@ -516,7 +516,7 @@ def run_ours(args):
 
     # ---- E1-E4: encode every layer once on the device (Algorithm 1)
     set_bytes = sum(layer_bytes(N, K, *pn[li]) for li, (_, N, K) in enumerate(layers))
-    copies = min(64, max(2, -(-2 * L2_BYTES // set_bytes)))      # rotating copies so that no step finds its codes in L2
+    copies = min(64, max(2, -(-(512 << 20) // set_bytes)))      # rotating copies (>= 512 MB in all) so that no step finds its codes in L2
     qs, xs, xs_host, xs32, ws, ys = [], [], [], [], [], []
     tables = {key: hb.higgs_make_encoder_table(key[0], key[1], grids[key]) for key in set(pn)}     # once per grid
     Ws = []
