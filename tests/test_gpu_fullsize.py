@@ -176,3 +176,21 @@ def test_encoder_is_reproducible_run_to_run(p, n, N, K):
         pk, sc, _ = hb.higgs_quantize(d, W, gt, table=table if it % 2 else None)
         assert torch.equal(pk, ref_p) and torch.equal(sc, ref_s), it
     assert hb.higgs_device_status() == hb.HIGGS_OK
+
+
+@pytest.mark.parametrize("p,n,N,K", [(2, 256, 16, 131072), (2, 64, 48, 65536), (1, 16, 32768, 1024), (2, 256, 32784, 1024)])
+def test_encoder_on_extreme_aspect_ratios(p, n, N, K):
+    """One row tile with 128 groups, many row tiles with one group, a row count that is not a multiple of the grid of
+    blocks: the persistent encoder's (row tile, group) bookkeeping against the pack kernel and the exhaustive scan."""
+    _, gt = U.grid32(p, n)
+    W = U.bf16_tensor(inputs.make_weights(N, K, inputs.weight_seed(4, 2), bf16=True))
+    xi = inputs.rht_seed(4)
+    d = hb.make_desc(p, n, N, K, xi)
+    packed, scales, canon = hb.higgs_quantize(d, W, gt, want_canonical=True)
+    assert torch.equal(hb.higgs_pack_codes(d, canon), packed)
+    rows, Ks = 16, min(K, 65536)                        # 16 rows x at most 64 groups: a small layer, exhaustive scan
+    ds = hb.make_desc(p, n, rows, Ks, xi)
+    _, scales_s, canon_s = hb.higgs_quantize(ds, W[:rows, :Ks].contiguous(), gt, want_canonical=True)
+    assert torch.equal(canon[:rows, :Ks // p], canon_s)
+    assert torch.equal(hb.scales_from_tile_major(scales, N)[:rows, :Ks // G], hb.scales_from_tile_major(scales_s, rows))
+    assert hb.higgs_device_status() == hb.HIGGS_OK
