@@ -630,15 +630,27 @@ def run_ours(args):
                         for k in range(length):
                             step(c * length + k)
                     graphs[length].append(g)
+            # every graph once before anything is timed: the first launch of a graph also uploads it to the device
+            # (80 us for a graph of five steps), which is set-up, not a step
+            for gl in graphs.values():
+                for g in gl:
+                    g.replay()
+            stream.synchronize()
+
+    replay_marks = []                 # (event, steps covered) after every graph replay of the last run_steps call
 
     def run_steps(first, count):      # exactly `count` steps, starting with step number `first`
         length = spg if count % spg == 0 else spg_w
         i = first
+        replay_marks.clear()
         while count > 0:
             if graphs is not None and count >= length:
                 graphs[length][(i // length) % copies].replay()
                 i += length
                 count -= length
+                m = ev()
+                m.record(stream)
+                replay_marks.append((m, length))
             else:
                 step(i)
                 i += 1
@@ -663,6 +675,7 @@ def run_ours(args):
             fn(warmup, steps)
             b.record(stream)
             torch.cuda.synchronize()
+            timed.start_event = a
             barrier()
             ms = a.elapsed_time(b)
         return max_over_ranks(ms, dev, world)
@@ -672,6 +685,16 @@ def run_ours(args):
     if rank == 0:
         sampler.start()
     ms = timed(run_steps, args.steps, warm)
+    # where the time of the timed region goes: per graph replay (the first one also carries the launch latency of the
+    # first graph after the synchronisation that the protocol puts before the region)
+    per_replay = None
+    if replay_marks:
+        prev, per = timed.start_event, []
+        for m, length in replay_marks:
+            per.append(prev.elapsed_time(m) * 1e3 / length)
+            prev = m
+        per_replay = {"us_per_step_first_replay": round(per[0], 2), "us_per_step_median": round(statistics.median(per), 2),
+                      "us_per_step_min": round(min(per), 2), "replays": len(per)}
     ms_e2e = timed(run_steps_host, args.steps, warm)
     # nvidia-smi samples every 100 ms and the timed regions above last tens of milliseconds: keep the same load running
     # (untimed) for a second more so that the clock record has samples taken under it
@@ -897,6 +920,7 @@ def run_ours(args):
                        "launch": "direct" if args.no_graph else f"CUDA graphs of {spg} consecutive steps over rotating weight copies ({args.steps // spg} replays timed)",
                        "step": "one transformer block, 7 matrices: layers that read the same input and share a grid (here: " + merged_names + ") run as one product over their concatenated rows (higgs_linear_multi); other sharing layers share one rotation (higgs_linear_share + higgs_linear_prerotated); a layer with its own input goes through higgs_linear; for 1-2 tokens the rotation runs inside the product kernel"},
             "us_per_layer": ms_per_step * 1e3 / len(layers),
+            "per_replay": per_replay,
             "weight_bytes_per_step": set_bytes,
             "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": ms_e2e / args.steps},
