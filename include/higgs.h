@@ -465,9 +465,9 @@ int higgs_dequantize(const higgs_desc* desc, const void* packed, const void* sca
 
 /* "Measuring Grid Parameters": one entry of the database of per-layer errors.  For the layer W quantised as
  * (packed, scales, grid) it accumulates, without materialising the dequantised matrix,
- *   sums_out[0] = || W^ - W ||_F^2,   sums_out[1] = || W ||_F^2        (device, two doubles, 8-byte aligned),
- * so that t^2 = sums_out[0] / sums_out[1] is the relative error of the linearity theorem (Appendix E shows it
- * equals the grid's expected squared error for Gaussian-like rotated weights).
+ *   sums_out[0] = || W^ - W ||_F^2,   sums_out[1] = || W ||_F^2,   sums_out[2] = t^2 = sums_out[0] / sums_out[1]
+ * (device, three doubles, 8-byte aligned; t^2 = 0 for an all-zero layer): t^2 is the relative error of the linearity
+ * theorem (Appendix E shows it equals the grid's expected squared error for Gaussian-like rotated weights).
  * W: device [N][K], w_dtype in {HIGGS_F32, HIGGS_BF16}; workspace as for higgs_dequantize.  Asynchronous.    */
 int higgs_layer_error(const higgs_desc* desc, const void* W, int w_dtype, const void* packed, const void* scales,
                       const float* grid, double* sums_out, void* workspace, size_t workspace_bytes, void* stream);
@@ -482,8 +482,8 @@ int higgs_layer_error(const higgs_desc* desc, const void* W, int w_dtype, const 
  *                rotated coordinates [t p, (t+1) p).  When p does not divide 1024 the last tuple is completed with
  *                zeros and matched on all p coordinates; its completed coordinates are dropped on reconstruction.
  *   scales_out : device [N][K/1024] fp16, ROW-major (not the product kernels' tile-major order): ||w|| / sqrt(1024)
- *   sums_out   : device, two doubles, optional: || W^ - W ||_F^2 (with the fp16 scale) and || W ||_F^2, so that
- *                t^2 = sums_out[0] / sums_out[1]; cleared by the call.
+ *   sums_out   : device, three doubles, optional: || W^ - W ||_F^2 (with the fp16 scale), || W ||_F^2 and their
+ *                ratio t^2; cleared by the call.
  * HIGGS_ERR_UNSUPPORTED for p, n or K outside the above; HIGGS_ERR_INVALID_ARG for null pointers.  Asynchronous.  */
 int higgs_general_tuples(int p);
 int higgs_quantize_general(int p, int n, int64_t N, int64_t K, uint64_t rht_seed, const void* W, int w_dtype,

@@ -644,12 +644,11 @@ def higgs_make_uniform_grid(n: int, device=None):
 def higgs_layer_error(desc: higgs_desc, W: torch.Tensor, packed: torch.Tensor, scales: torch.Tensor, grid: torch.Tensor) -> float:
     """Relative quantisation error t^2 = ||W^ - W||^2 / ||W||^2 of the layer (Section 5, 'Measuring Grid Parameters')."""
     assert W.is_cuda and W.is_contiguous() and W.dtype in (torch.float32, torch.bfloat16)
-    sums = torch.zeros(2, dtype=torch.float64, device=W.device)
+    sums = torch.zeros(3, dtype=torch.float64, device=W.device)
     ws = _workspace(higgs_workspace_bytes(desc, HIGGS_OP_QUANTIZE, 0), W.device)
     _check(lib.higgs_layer_error(ctypes.byref(desc), _ptr(W), _dtype_code(W), _ptr(packed), _ptr(scales), _ptr(grid), _ptr(sums),
                                  _ptr(ws), ws.numel(), _stream()), "higgs_layer_error")
-    s = sums.cpu()
-    return float(s[0] / s[1]) if float(s[1]) > 0 else 0.0
+    return float(sums[2].item())
 
 
 def higgs_quantize_general(p: int, n: int, W: torch.Tensor, grid: torch.Tensor, rht_seed: int, want_error: bool = True):
@@ -661,14 +660,10 @@ def higgs_quantize_general(p: int, n: int, W: torch.Tensor, grid: torch.Tensor, 
     tuples = lib.higgs_general_tuples(p)
     codes = torch.empty((N, K // 1024, max(tuples, 1)), dtype=torch.uint16, device=W.device)
     scales = torch.empty((N, K // 1024), dtype=torch.float16, device=W.device)
-    sums = torch.zeros(2, dtype=torch.float64, device=W.device) if want_error else None
+    sums = torch.zeros(3, dtype=torch.float64, device=W.device) if want_error else None
     _check(lib.higgs_quantize_general(p, n, N, K, rht_seed, _ptr(W), _dtype_code(W), _ptr(grid), _ptr(codes), _ptr(scales),
                                       _ptr(sums), _stream()), "higgs_quantize_general")
-    t2 = None
-    if want_error:
-        s = sums.cpu()
-        t2 = float(s[0] / s[1]) if float(s[1]) > 0 else 0.0
-    return codes, scales, t2
+    return codes, scales, (float(sums[2].item()) if want_error else None)
 
 
 def higgs_allocate_bits(alpha, t2, bits64, sizes, budget64: int):

@@ -179,8 +179,9 @@ int higgs_quantize_general(int p, int n, int64_t N, int64_t K, uint64_t rht_seed
     if (!W || !grid || !codes_out || !scales_out) return HIGGS_ERR_INVALID_ARG;
     if (!aligned(W, 16) || !aligned(codes_out, 2) || !aligned(scales_out, 2) || (sums_out && !aligned(sums_out, 8)))
         return HIGGS_ERR_INVALID_ARG;
-    return launch_encode_general(p, n, N, K, rht_seed, W, w_dtype, grid, codes_out, scales_out, sums_out,
-                                 as_stream(stream));
+    const int rc = launch_encode_general(p, n, N, K, rht_seed, W, w_dtype, grid, codes_out, scales_out, sums_out,
+                                         as_stream(stream));
+    return rc != HIGGS_OK || !sums_out ? rc : launch_error_ratio(sums_out, as_stream(stream));
 }
 
 int higgs_make_uniform_grid(int n, float* grid_out, float* step_out, float* mse_out, void* stream) {
@@ -268,7 +269,7 @@ int higgs_layer_error(const higgs_desc* d, const void* W, int w_dtype, const voi
     if (rc != HIGGS_OK) return rc;
     if (w_dtype != HIGGS_F32 && w_dtype != HIGGS_BF16) return HIGGS_ERR_UNSUPPORTED;
     if (!sums_out || !aligned(sums_out, 8)) return HIGGS_ERR_INVALID_ARG;
-    if (d->N == 0 || d->K == 0) return cuda_status(cudaMemsetAsync(sums_out, 0, 2 * sizeof(double), as_stream(stream)));
+    if (d->N == 0 || d->K == 0) return cuda_status(cudaMemsetAsync(sums_out, 0, 3 * sizeof(double), as_stream(stream)));
     if (!W || !packed || !scales || !grid || !workspace) return HIGGS_ERR_INVALID_ARG;
     if (!aligned(W, 16) || !aligned(packed, 16) || !aligned(scales, 16) || !aligned(workspace, 256)) return HIGGS_ERR_INVALID_ARG;
     if (workspace_bytes < higgs_workspace_bytes(d, HIGGS_OP_QUANTIZE, 0)) return HIGGS_ERR_WORKSPACE;
@@ -276,7 +277,8 @@ int higgs_layer_error(const higgs_desc* d, const void* W, int w_dtype, const voi
     uint8_t* canonical = static_cast<uint8_t*>(workspace);
     rc = launch_unpack(*d, packed, canonical, st);
     if (rc != HIGGS_OK) return rc;
-    return launch_layer_error(*d, canonical, scales, grid, W, w_dtype, sums_out, st);
+    rc = launch_layer_error(*d, canonical, scales, grid, W, w_dtype, sums_out, st);
+    return rc != HIGGS_OK ? rc : launch_error_ratio(sums_out, st);
 }
 
 int higgs_allocate_bits(int32_t num_layers, int32_t num_options, const double* alpha, const double* t2, const int32_t* bits64,

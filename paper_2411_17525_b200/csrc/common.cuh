@@ -237,6 +237,7 @@ int launch_linear_tc(const higgs_desc& d, const __half* xdag_tc, int64_t B, cons
                      const float* grid, void* y, int y_mode, cudaStream_t st, int64_t ldy = 0,
                      const GatherTargets* more = nullptr);
 int read_tc_status(int clear);
+int launch_error_ratio(double* sums, cudaStream_t st);
 int read_grid_status(int clear);
 int read_encode_status(int clear);
 int launch_wait_selftest(uint32_t limit, int* result, cudaStream_t st);

@@ -64,6 +64,14 @@ int launch_reduce_slots(const float* slots, int world, int64_t count, void* y, i
                                   y_dtype == HIGGS_BF16 ? 1 : 0));
 }
 
+// t^2 = ||W^ - W||^2 / ||W||^2 from the two accumulated sums (0 for an all-zero layer)
+__global__ void error_ratio_kernel(double* sums) { sums[2] = sums[1] > 0.0 ? sums[0] / sums[1] : 0.0; }
+
+int launch_error_ratio(double* sums, cudaStream_t st) {
+    error_ratio_kernel<<<1, 1, 0, st>>>(sums);
+    return cuda_status(cudaGetLastError());
+}
+
 int launch_floor(int blocks, int threads, size_t smem, cudaStream_t st) {
     static int configured[64] = {0};
     const int ok = device_once(configured, [] {
